@@ -1,0 +1,179 @@
+/*
+ * libh1b -- decode-time attention read directly from a hybrid compressed KV
+ * cache (H1B-KV): every cached key is an m-bit sign sketch sign(R k) of a fixed
+ * Gaussian projection (Section IV-A, Eq. 2), every cached value is a vector of
+ * 4-bit codes with a scale and a zero-point (Section IV-B, Eq. 4), scores are
+ * normalised Hamming inner products (Eq. 3) and the output is
+ * softmax(alpha/tau) * V_dequant (Section IV-C, Eq. 5).
+ *
+ * C ABI, CUDA (sm_100a) behind it.  No C++ or framework types cross this
+ * boundary: plain pointers, marked HOST or DEVICE, and sizes.
+ *
+ * Conventions
+ *   - Every call returns 0 (H1B_OK) or a negative H1B_ERR_* code; the text of
+ *     the last error of a context is h1b_last_error().  Nothing aborts or
+ *     throws.  Argument errors are detected on the host before any launch, so
+ *     a failed call has written nothing.
+ *   - Ownership: the library owns only the host-side context.  The caller
+ *     allocates the device workspace (h1b_cache_bytes() bytes, 256-byte
+ *     aligned) and every input/output buffer, and keeps them alive until the
+ *     stream work that uses them has completed.  h1b_free() does not free the
+ *     workspace.
+ *   - Asynchrony: h1b_append_kv() and h1b_decode_attention() only enqueue work
+ *     on `stream` (a cudaStream_t passed as void*, NULL = the default stream).
+ *     Use one stream at a time per context.
+ *   - Symbols: d = head_dim, m = sketch_bits (the paper's b), G = group_size,
+ *     L = n_layers, Hq / Hkv = query / KV heads, B = sequences in the call.
+ *     The projection is held as Rt[d][m] (row-major), Rt[i][j] = R[j][i] for
+ *     the paper's R in R^{m x d}; one matrix per layer, shared by all heads and
+ *     by keys and queries.
+ *   - Sketch bit j of a vector x is 1 iff sum_i x_i * Rt[i][j] >= 0 (s_j = +1).
+ *   - Values: per token, per KV head, per group of G consecutive channels:
+ *     scale = fp16((max - min)/15), zero = min, code = clamp(rne((v - zero)/scale), 0, 15),
+ *     code = 0 when scale == 0.  Dequantised value = code * scale + zero.
+ *   - Score of token t for a query: m - 2 * popcount(s_q xor s_t); alpha = score / m.
+ *     All cached tokens [0, len) are attended, the one just appended included.
+ *     Query head h reads KV head h / (Hq / Hkv).  An empty sequence gives zeros.
+ */
+#ifndef H1B_H
+#define H1B_H
+
+#include <stddef.h>
+#include <stdint.h>
+
+#ifdef __cplusplus
+extern "C" {
+#endif
+
+#define H1B_OK               0
+#define H1B_ERR_INVALID_ARG (-1)  /* a size, index or flag is out of range            */
+#define H1B_ERR_NULL        (-2)  /* a required pointer is NULL                        */
+#define H1B_ERR_UNSUPPORTED (-3)  /* valid in principle, no kernel for this shape      */
+#define H1B_ERR_CAPACITY    (-4)  /* len + n_new > max_seq for some sequence           */
+#define H1B_ERR_WORKSPACE   (-5)  /* workspace too small or misaligned                 */
+#define H1B_ERR_CUDA        (-6)  /* a CUDA runtime call failed (text in last_error)   */
+#define H1B_ERR_TIMEOUT     (-7)  /* a bounded device-side wait gave up (poll_status)  */
+
+typedef struct h1b_ctx h1b_ctx;   /* opaque, host-side */
+
+typedef struct {
+    int32_t n_layers;      /* L >= 1                                                   */
+    int32_t n_q_heads;     /* Hq; Hq / Hkv must be 1, 2 or 4                           */
+    int32_t n_kv_heads;    /* Hkv                                                      */
+    int32_t head_dim;      /* d: 128                                                   */
+    int32_t sketch_bits;   /* m: 64, 128, 256 or 512                                   */
+    int32_t group_size;    /* G: 32                                                    */
+    int32_t max_batch;     /* sequences the cache can hold (<= 256)                    */
+    int32_t max_seq;       /* tokens per sequence the cache can hold                   */
+    int32_t device;        /* CUDA device ordinal                                      */
+    uint32_t flags;        /* reserved, must be 0                                      */
+} h1b_config;
+
+/* Bytes of one cached token of one KV head: m/8 + d/2 + (d/G)*4 (Section IV-B
+ * storage statement plus the fp16 scale and zero per group). 0 if invalid. */
+size_t h1b_entry_bytes(const h1b_config *cfg /* HOST */);
+
+/* Bytes of device workspace the caller must provide for this configuration
+ * (projection matrices, lengths, split-K scratch, staging and the packed cache
+ * itself). 0 if the configuration is invalid or unsupported. */
+size_t h1b_cache_bytes(const h1b_config *cfg /* HOST */);
+
+/* Create a context over a caller-owned workspace and install the projection
+ * matrices (Section IV-A: "a fixed, pre-generated Gaussian matrix").
+ *   seed       used only when Rt_host is NULL
+ *   Rt_host    HOST, nullable: float32 [L][d][m]; NULL = draw N(0,1) from `seed`
+ *              on the host (Box-Muller over a splitmix64 counter stream)
+ *   workspace  DEVICE, 256-byte aligned, workspace_bytes >= h1b_cache_bytes(cfg)
+ *   out        HOST: receives the context
+ * Zero-fills the workspace, copies Rt to the device, sets all lengths to 0 and
+ * synchronises the stream before returning. */
+int h1b_init_projection(const h1b_config *cfg, uint64_t seed, const float *Rt_host,
+                        void *workspace, size_t workspace_bytes, void *stream,
+                        h1b_ctx **out);
+
+/* Compress and append new key/value rows (Eq. 2 on keys, Eq. 4 on values).
+ *   k, v        DEVICE: fp16 [n_layers][B][Tn][Hkv][d]
+ *   n_new_host  HOST, nullable: int32 [B], 0 <= n_new[b] <= Tn rows of sequence b
+ *               are appended (the first n_new[b] of its Tn); NULL = Tn for all
+ * Sequence b of the call is sequence b of the cache.  Row tn of sequence b goes
+ * to position len[layer][b] + tn; afterwards len[layer][b] += n_new[b].
+ * H1B_ERR_CAPACITY (nothing written) if any sequence would exceed max_seq. */
+int h1b_append_kv(h1b_ctx *ctx, int layer_begin, int n_layers, const void *k, const void *v,
+                  const int32_t *n_new_host, int B, int Tn, void *stream);
+
+/* One decode step of attention over the compressed cache (Eq. 3 and Eq. 5):
+ * sketch the queries, score every cached token by popcount, softmax with
+ * temperature tau, weight the dequantised values.
+ *   q        DEVICE: fp16 [n_layers][B][Hq][d]
+ *   inv_tau  1/tau, finite and > 0
+ *   out      DEVICE: float32 [n_layers][B][Hq][d]
+ * Uses the split-K scratch inside the workspace: calls on one context must not
+ * overlap on the GPU. */
+int h1b_decode_attention(h1b_ctx *ctx, int layer_begin, int n_layers, const void *q,
+                         float inv_tau, void *out, int B, void *stream);
+
+/* The same step for callers whose tensors live in host memory: copies k, v, q
+ * (HOST, fp16, [L][B][1][Hkv][d], [L][B][1][Hkv][d], [L][B][Hq][d]; pinned
+ * memory makes the copies asynchronous) into staging inside the workspace,
+ * appends one token per sequence to all L layers, runs decode attention over
+ * all layers, copies the result to out (HOST, float32 [L][B][Hq][d]) and
+ * synchronises the stream. */
+int h1b_decode_step_host(h1b_ctx *ctx, const void *k_host, const void *v_host,
+                         const void *q_host, float inv_tau, void *out_host, int B,
+                         void *stream);
+
+/* Synchronise the context's device and release the host-side context. The
+ * workspace stays with the caller. */
+int h1b_free(h1b_ctx *ctx);
+
+/* ---- introspection and test helpers (synchronous) ------------------------ */
+
+/* Copy layer `layer`'s projection to Rt_host (HOST float32 [d][m]). */
+int h1b_get_projection(h1b_ctx *ctx, int layer, float *Rt_host);
+
+/* Copy layer `layer`'s lengths to len_host (HOST int32 [max_batch]); also
+ * checks them against the host mirror (H1B_ERR_INVALID_ARG on mismatch). */
+int h1b_get_lengths(h1b_ctx *ctx, int layer, int32_t *len_host);
+
+/* Forget the cached tokens of sequence `seq` in all layers (-1 = all
+ * sequences): lengths become 0; the bytes are not cleared. */
+int h1b_reset(h1b_ctx *ctx, int seq);
+
+/* Set the length of sequence `seq` (-1 = all) in all layers to new_len, which
+ * must not exceed any of their current lengths (roll back the last tokens). */
+int h1b_truncate(h1b_ctx *ctx, int seq, int new_len);
+
+/* Unpack cached tokens [t0, t0+n) of (layer, seq, kv_head) into a canonical
+ * layout, independent of the packed device layout (all HOST, any may be NULL):
+ *   words  uint32 [n][m/32]: sketch bit j is bit (j % 32) of word j / 32
+ *   codes  uint8  [n][d]:    one 4-bit code per byte
+ *   scale, zero  uint16 [n][d/G]: fp16 bit patterns */
+int h1b_export_cache(h1b_ctx *ctx, int layer, int seq, int kv_head, int t0, int n,
+                     uint32_t *words, uint8_t *codes, uint16_t *scale, uint16_t *zero);
+
+/* Sketch one query (DEVICE fp16 [d]) with layer `layer`'s projection and score
+ * it against every cached token of (layer, seq, kv_head):
+ *   qwords_host  HOST, nullable: uint32 [m/32]
+ *   score_host   HOST, nullable: int32 [len] = m - 2 * Hamming */
+int h1b_debug_scores(h1b_ctx *ctx, int layer, int seq, int kv_head, const void *q,
+                     uint32_t *qwords_host, int32_t *score_host);
+
+/* Force the number of sequence splits of the decode kernel (0 = automatic).
+ * H1B_ERR_INVALID_ARG if the split-K scratch cannot hold that many. */
+int h1b_set_splits(h1b_ctx *ctx, int splits);
+
+/* After the stream has been synchronised: 0, or H1B_ERR_TIMEOUT if a kernel
+ * gave up a bounded wait since the last poll (the flag is cleared). */
+int h1b_poll_status(h1b_ctx *ctx);
+
+/* Kernel launches enqueued by this context so far. */
+int64_t h1b_launch_count(const h1b_ctx *ctx);
+
+/* Text of the last error recorded on this context ("" if none). With ctx ==
+ * NULL: the text of the last failed h1b_init_projection() on this thread. */
+const char *h1b_last_error(const h1b_ctx *ctx);
+
+#ifdef __cplusplus
+}
+#endif
+#endif /* H1B_H */

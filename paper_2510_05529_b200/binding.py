@@ -1,0 +1,250 @@
+"""ctypes binding of libh1b.so: the same entry points as include/h1b.h.
+
+This module only marshals arguments. Every step of the path (sketching,
+quantisation, scores, softmax, weighted sum) runs in the CUDA library. PyTorch
+is used for device memory and streams. There is no CPU fallback: a missing or
+unloadable library raises.
+"""
+from __future__ import annotations
+
+import ctypes
+import os
+
+import numpy as np
+import torch
+
+from .build import LIB_PATH, build_library, is_stale
+
+H1B_OK = 0
+ERRORS = {
+    -1: "H1B_ERR_INVALID_ARG", -2: "H1B_ERR_NULL", -3: "H1B_ERR_UNSUPPORTED", -4: "H1B_ERR_CAPACITY",
+    -5: "H1B_ERR_WORKSPACE", -6: "H1B_ERR_CUDA", -7: "H1B_ERR_TIMEOUT",
+}
+
+
+class H1BError(RuntimeError):
+    def __init__(self, code: int, text: str = ""):
+        self.code = code
+        super().__init__("%s (%d)%s" % (ERRORS.get(code, "H1B_ERR_?"), code, ": " + text if text else ""))
+
+
+class h1b_config(ctypes.Structure):
+    _fields_ = [(n, ctypes.c_int32) for n in
+                ("n_layers", "n_q_heads", "n_kv_heads", "head_dim", "sketch_bits", "group_size",
+                 "max_batch", "max_seq", "device")] + [("flags", ctypes.c_uint32)]
+
+
+_lib = None
+
+
+def load_library(rebuild: bool = True) -> ctypes.CDLL:
+    """Load libh1b.so (building it with nvcc first when it is missing or stale)."""
+    global _lib
+    if _lib is not None:
+        return _lib
+    if rebuild and is_stale():
+        build_library()
+    if not os.path.exists(LIB_PATH):
+        raise RuntimeError("libh1b.so is missing and could not be built; there is no fallback path")
+    lib = ctypes.CDLL(LIB_PATH)
+    vp, cp = ctypes.c_void_p, ctypes.POINTER(h1b_config)
+    i32p = ctypes.POINTER(ctypes.c_int32)
+    sig = {
+        "h1b_entry_bytes": (ctypes.c_size_t, [cp]),
+        "h1b_cache_bytes": (ctypes.c_size_t, [cp]),
+        "h1b_init_projection": (ctypes.c_int, [cp, ctypes.c_uint64, vp, vp, ctypes.c_size_t, vp,
+                                               ctypes.POINTER(vp)]),
+        "h1b_append_kv": (ctypes.c_int, [vp, ctypes.c_int, ctypes.c_int, vp, vp, i32p, ctypes.c_int,
+                                         ctypes.c_int, vp]),
+        "h1b_decode_attention": (ctypes.c_int, [vp, ctypes.c_int, ctypes.c_int, vp, ctypes.c_float, vp,
+                                                ctypes.c_int, vp]),
+        "h1b_decode_step_host": (ctypes.c_int, [vp, vp, vp, vp, ctypes.c_float, vp, ctypes.c_int, vp]),
+        "h1b_free": (ctypes.c_int, [vp]),
+        "h1b_get_projection": (ctypes.c_int, [vp, ctypes.c_int, vp]),
+        "h1b_get_lengths": (ctypes.c_int, [vp, ctypes.c_int, vp]),
+        "h1b_reset": (ctypes.c_int, [vp, ctypes.c_int]),
+        "h1b_truncate": (ctypes.c_int, [vp, ctypes.c_int, ctypes.c_int]),
+        "h1b_export_cache": (ctypes.c_int, [vp, ctypes.c_int, ctypes.c_int, ctypes.c_int, ctypes.c_int,
+                                            ctypes.c_int, vp, vp, vp, vp]),
+        "h1b_debug_scores": (ctypes.c_int, [vp, ctypes.c_int, ctypes.c_int, ctypes.c_int, vp, vp, vp]),
+        "h1b_set_splits": (ctypes.c_int, [vp, ctypes.c_int]),
+        "h1b_poll_status": (ctypes.c_int, [vp]),
+        "h1b_launch_count": (ctypes.c_int64, [vp]),
+        "h1b_last_error": (ctypes.c_char_p, [vp]),
+    }
+    for name, (res, args) in sig.items():
+        fn = getattr(lib, name)
+        fn.restype, fn.argtypes = res, args
+    _lib = lib
+    return lib
+
+
+def make_config(n_layers, n_q_heads, n_kv_heads, head_dim=128, sketch_bits=128, group_size=32,
+                max_batch=1, max_seq=8192, device=0) -> h1b_config:
+    return h1b_config(n_layers, n_q_heads, n_kv_heads, head_dim, sketch_bits, group_size,
+                      max_batch, max_seq, device, 0)
+
+
+def h1b_entry_bytes(cfg: h1b_config) -> int:
+    return int(load_library().h1b_entry_bytes(ctypes.byref(cfg)))
+
+
+def h1b_cache_bytes(cfg: h1b_config) -> int:
+    return int(load_library().h1b_cache_bytes(ctypes.byref(cfg)))
+
+
+def _stream_ptr(stream) -> int:
+    if stream is None:
+        stream = torch.cuda.current_stream()
+    return int(stream.cuda_stream)
+
+
+def _dev_ptr(t: torch.Tensor, dtype, what: str) -> int:
+    if not (isinstance(t, torch.Tensor) and t.is_cuda and t.is_contiguous() and t.dtype == dtype):
+        raise TypeError("%s must be a contiguous CUDA tensor of dtype %s" % (what, dtype))
+    return t.data_ptr()
+
+
+class H1BCache:
+    """One library context over a torch-owned device workspace."""
+
+    def __init__(self, cfg: h1b_config, seed: int = 0, Rt: np.ndarray | None = None, stream=None):
+        self.lib = load_library()
+        self.cfg = cfg
+        nbytes = h1b_cache_bytes(cfg)
+        if nbytes == 0:
+            raise H1BError(-3, "invalid or unsupported configuration")
+        self.device = torch.device("cuda", cfg.device)
+        self.workspace = torch.empty(nbytes + 256, dtype=torch.uint8, device=self.device)
+        base = self.workspace.data_ptr()
+        self._ws_ptr = (base + 255) // 256 * 256
+        self.workspace_bytes = nbytes
+        rt_ptr = None
+        if Rt is not None:
+            Rt = np.ascontiguousarray(Rt, dtype=np.float32)
+            want = (cfg.n_layers, cfg.head_dim, cfg.sketch_bits)
+            if Rt.shape != want:
+                raise ValueError("Rt must have shape %s, got %s" % (want, Rt.shape))
+            rt_ptr = Rt.ctypes.data
+        handle = ctypes.c_void_p()
+        with torch.cuda.device(self.device):
+            rc = self.lib.h1b_init_projection(ctypes.byref(cfg), seed, rt_ptr, self._ws_ptr, nbytes,
+                                              _stream_ptr(stream), ctypes.byref(handle))
+        if rc != H1B_OK:
+            raise H1BError(rc, (self.lib.h1b_last_error(None) or b"").decode())
+        self._h = handle
+
+    # -- helpers ---------------------------------------------------------
+    def _check(self, rc: int):
+        if rc != H1B_OK:
+            raise H1BError(rc, (self.lib.h1b_last_error(self._h) or b"").decode())
+
+    def close(self):
+        if getattr(self, "_h", None):
+            self.lib.h1b_free(self._h)
+            self._h = None
+
+    def __del__(self):
+        try:
+            self.close()
+        except Exception:
+            pass
+
+    # -- the four calls of the path ----------------------------------------
+    def h1b_append_kv(self, k: torch.Tensor, v: torch.Tensor, layer_begin: int = 0, n_new=None, stream=None):
+        """k, v: fp16 CUDA [n_layers, B, Tn, Hkv, d]."""
+        kp = _dev_ptr(k, torch.float16, "k")
+        vp = _dev_ptr(v, torch.float16, "v")
+        if k.shape != v.shape or k.dim() != 5 or k.shape[3] != self.cfg.n_kv_heads or k.shape[4] != self.cfg.head_dim:
+            raise ValueError("k and v must be [n_layers, B, Tn, Hkv, d]")
+        nl, B, Tn = int(k.shape[0]), int(k.shape[1]), int(k.shape[2])
+        nn = None
+        if n_new is not None:
+            arr = np.ascontiguousarray(n_new, dtype=np.int32)
+            if arr.shape != (B,):
+                raise ValueError("n_new must have shape [B]")
+            nn = arr.ctypes.data_as(ctypes.POINTER(ctypes.c_int32))
+        self._check(self.lib.h1b_append_kv(self._h, layer_begin, nl, kp, vp, nn, B, Tn, _stream_ptr(stream)))
+
+    def h1b_decode_attention(self, q: torch.Tensor, inv_tau: float, out: torch.Tensor | None = None,
+                             layer_begin: int = 0, stream=None) -> torch.Tensor:
+        """q: fp16 CUDA [n_layers, B, Hq, d] -> out fp32 [n_layers, B, Hq, d]."""
+        qp = _dev_ptr(q, torch.float16, "q")
+        if q.dim() != 4 or q.shape[2] != self.cfg.n_q_heads or q.shape[3] != self.cfg.head_dim:
+            raise ValueError("q must be [n_layers, B, Hq, d]")
+        if out is None:
+            out = torch.empty(q.shape, dtype=torch.float32, device=q.device)
+        op = _dev_ptr(out, torch.float32, "out")
+        if out.shape != q.shape:
+            raise ValueError("out must have q's shape")
+        self._check(self.lib.h1b_decode_attention(self._h, layer_begin, int(q.shape[0]), qp, float(inv_tau), op,
+                                                  int(q.shape[1]), _stream_ptr(stream)))
+        return out
+
+    def h1b_decode_step_host(self, k: torch.Tensor, v: torch.Tensor, q: torch.Tensor, inv_tau: float,
+                             out: torch.Tensor, stream=None) -> torch.Tensor:
+        """Host tensors (pinned for asynchronous copies): k, v fp16 [L, B, 1, Hkv, d], q fp16 [L, B, Hq, d],
+        out fp32 [L, B, Hq, d]. Copies, appends, decodes, copies back, synchronises."""
+        for t, dt, name in ((k, torch.float16, "k"), (v, torch.float16, "v"), (q, torch.float16, "q"),
+                            (out, torch.float32, "out")):
+            if t.is_cuda or not t.is_contiguous() or t.dtype != dt:
+                raise TypeError("%s must be a contiguous host tensor of dtype %s" % (name, dt))
+        L, B = self.cfg.n_layers, int(q.shape[1])
+        if tuple(k.shape) != (L, B, 1, self.cfg.n_kv_heads, self.cfg.head_dim) or k.shape != v.shape or \
+                tuple(q.shape) != (L, B, self.cfg.n_q_heads, self.cfg.head_dim) or out.shape != q.shape:
+            raise ValueError("host step shapes: k, v [L, B, 1, Hkv, d]; q, out [L, B, Hq, d]")
+        self._check(self.lib.h1b_decode_step_host(self._h, k.data_ptr(), v.data_ptr(), q.data_ptr(), float(inv_tau),
+                                                  out.data_ptr(), B, _stream_ptr(stream)))
+        return out
+
+    # -- introspection -----------------------------------------------------
+    def h1b_get_projection(self, layer: int) -> np.ndarray:
+        Rt = np.empty((self.cfg.head_dim, self.cfg.sketch_bits), dtype=np.float32)
+        self._check(self.lib.h1b_get_projection(self._h, layer, Rt.ctypes.data))
+        return Rt
+
+    def h1b_get_lengths(self, layer: int) -> np.ndarray:
+        ln = np.empty((self.cfg.max_batch,), dtype=np.int32)
+        self._check(self.lib.h1b_get_lengths(self._h, layer, ln.ctypes.data))
+        return ln
+
+    def h1b_reset(self, seq: int = -1):
+        self._check(self.lib.h1b_reset(self._h, seq))
+
+    def h1b_truncate(self, seq: int, new_len: int):
+        self._check(self.lib.h1b_truncate(self._h, seq, new_len))
+
+    def h1b_export_cache(self, layer: int, seq: int, kv_head: int, t0: int, n: int):
+        """-> (words uint32 [n, m/32], codes uint8 [n, d], scale uint16 [n, d/G], zero uint16 [n, d/G])."""
+        c = self.cfg
+        words = np.empty((n, c.sketch_bits // 32), dtype=np.uint32)
+        codes = np.empty((n, c.head_dim), dtype=np.uint8)
+        scale = np.empty((n, c.head_dim // c.group_size), dtype=np.uint16)
+        zero = np.empty_like(scale)
+        self._check(self.lib.h1b_export_cache(self._h, layer, seq, kv_head, t0, n, words.ctypes.data,
+                                              codes.ctypes.data, scale.ctypes.data, zero.ctypes.data))
+        return words, codes, scale, zero
+
+    def h1b_debug_scores(self, layer: int, seq: int, kv_head: int, q_row: torch.Tensor, n_tokens: int):
+        """q_row: fp16 CUDA [d]. -> (qwords uint32 [m/32], score int32 [n_tokens])."""
+        qp = _dev_ptr(q_row, torch.float16, "q_row")
+        qwords = np.empty((self.cfg.sketch_bits // 32,), dtype=np.uint32)
+        score = np.empty((max(n_tokens, 1),), dtype=np.int32)
+        self._check(self.lib.h1b_debug_scores(self._h, layer, seq, kv_head, qp, qwords.ctypes.data, score.ctypes.data))
+        return qwords, score[:n_tokens]
+
+    def h1b_set_splits(self, splits: int):
+        self._check(self.lib.h1b_set_splits(self._h, splits))
+
+    def h1b_poll_status(self):
+        self._check(self.lib.h1b_poll_status(self._h))
+
+    def h1b_launch_count(self) -> int:
+        return int(self.lib.h1b_launch_count(self._h))
+
+
+def unpack_words(words: np.ndarray, m: int) -> np.ndarray:
+    """uint32 [n, m/32] -> bits uint8 [n, m] (bit j = bit j%32 of word j/32). Marshalling only."""
+    w = np.ascontiguousarray(words, dtype=np.uint32)
+    bits = ((w[:, :, None] >> np.arange(32, dtype=np.uint32)[None, None, :]) & 1).astype(np.uint8)
+    return bits.reshape(w.shape[0], m)

@@ -1,0 +1,463 @@
+// Host side of libh1b: the C ABI declared in include/h1b.h. Validation,
+// workspace carving, the host mirror of the lengths, launches. All device
+// arithmetic is in h1b_kernels.cu.
+#include <algorithm>
+#include <cmath>
+#include <cstdarg>
+#include <cstdio>
+#include <cstring>
+#include <new>
+#include <string>
+#include <vector>
+
+#include <cuda_runtime.h>
+
+#include "../../include/h1b.h"
+#include "h1b_kernels.h"
+
+using namespace h1b;
+
+namespace {
+
+constexpr long kTargetItems = 8192;   // decode work items aimed for (one warp each)
+constexpr int kMinSplitTokens = 256;
+
+struct Plan {
+    size_t rt, len, status, qwords, partial, stage_k, stage_v, stage_q, stage_out, dbg_q, dbg_s, cache, total;
+    size_t partial_items, slab_bytes;
+    int cap_tokens, m_words, gq;
+};
+
+size_t align_up(size_t x, size_t a) { return (x + a - 1) / a * a; }
+
+int check_config(const h1b_config *c) {
+    if (!c) return H1B_ERR_NULL;
+    if (c->n_layers < 1 || c->n_q_heads < 1 || c->n_kv_heads < 1 || c->max_batch < 1 || c->max_seq < 1 ||
+        c->head_dim < 1 || c->sketch_bits < 1 || c->group_size < 1 || c->device < 0 || c->flags != 0)
+        return H1B_ERR_INVALID_ARG;
+    if (c->n_q_heads % c->n_kv_heads != 0 || c->head_dim % c->group_size != 0 || c->sketch_bits % 32 != 0)
+        return H1B_ERR_INVALID_ARG;
+    if (c->max_batch > 256) return H1B_ERR_INVALID_ARG;
+    const int gq = c->n_q_heads / c->n_kv_heads;
+    if (gq != 1 && gq != 2 && gq != 4) return H1B_ERR_UNSUPPORTED;
+    if (c->head_dim != kHeadDim || c->group_size != kGroup) return H1B_ERR_UNSUPPORTED;
+    if (c->sketch_bits != 64 && c->sketch_bits != 128 && c->sketch_bits != 256 && c->sketch_bits != 512)
+        return H1B_ERR_UNSUPPORTED;
+    if ((long)c->n_layers * c->max_batch * c->n_kv_heads > (1L << 28)) return H1B_ERR_INVALID_ARG;
+    return H1B_OK;
+}
+
+int make_plan(const h1b_config *c, Plan *p) {
+    const int rc = check_config(c);
+    if (rc != H1B_OK) return rc;
+    p->m_words = c->sketch_bits / 32;
+    p->gq = c->n_q_heads / c->n_kv_heads;
+    const ChunkLayout cl = chunk_layout(p->m_words);
+    p->cap_tokens = (c->max_seq + kChunkTokens - 1) / kChunkTokens * kChunkTokens;
+    p->slab_bytes = (size_t)(p->cap_tokens / kChunkTokens) * cl.bytes;
+    const size_t L = c->n_layers, B = c->max_batch, Hq = c->n_q_heads, Hkv = c->n_kv_heads, d = c->head_dim;
+    const size_t slabs = L * B * Hkv;
+    p->partial_items = slabs > (size_t)kTargetItems ? slabs : (size_t)kTargetItems;
+    size_t o = 0;
+    auto take = [&](size_t bytes) { size_t at = o; o = align_up(o + bytes, 256); return at; };
+    p->rt = take(L * d * c->sketch_bits * sizeof(float));
+    p->len = take(L * B * sizeof(int32_t));
+    p->status = take(64);
+    p->qwords = take(L * B * Hq * p->m_words * sizeof(uint32_t));
+    p->partial = take(p->partial_items * p->gq * kPartStride * sizeof(float));
+    p->stage_k = take(L * B * Hkv * d * 2);
+    p->stage_v = take(L * B * Hkv * d * 2);
+    p->stage_q = take(L * B * Hq * d * 2);
+    p->stage_out = take(L * B * Hq * d * 4);
+    p->dbg_q = take(p->m_words * sizeof(uint32_t));
+    p->dbg_s = take((size_t)p->cap_tokens * sizeof(int32_t));
+    p->cache = take(slabs * p->slab_bytes);
+    p->total = o;
+    return H1B_OK;
+}
+
+thread_local std::string g_init_error;
+
+// N(0,1) from a counter-based stream (splitmix64 + Box-Muller), host only.
+uint64_t splitmix64(uint64_t x) {
+    x += 0x9E3779B97F4A7C15ull;
+    x = (x ^ (x >> 30)) * 0xBF58476D1CE4E5B9ull;
+    x = (x ^ (x >> 27)) * 0x94D049BB133111EBull;
+    return x ^ (x >> 31);
+}
+void fill_gaussian(float *dst, size_t n, uint64_t seed) {
+    for (size_t i = 0; i < n; i += 2) {
+        const uint64_t a = splitmix64(seed * 0x100000001B3ull + i), b = splitmix64(a ^ 0xD1B54A32D192ED03ull);
+        const double u1 = ((double)(a >> 11) + 1.0) / 9007199254740993.0;   // (0, 1)
+        const double u2 = (double)(b >> 11) / 9007199254740992.0;           // [0, 1)
+        const double r = std::sqrt(-2.0 * std::log(u1)), th = 6.283185307179586476925 * u2;
+        dst[i] = (float)(r * std::cos(th));
+        if (i + 1 < n) dst[i + 1] = (float)(r * std::sin(th));
+    }
+}
+
+}  // namespace
+
+struct h1b_ctx {
+    h1b_config cfg;
+    Plan plan;
+    ChunkLayout cl;
+    unsigned char *ws;
+    std::vector<int32_t> len_host;     // [L][max_batch], mirror of the device lengths
+    int forced_splits;
+    int64_t launches;
+    std::string err;
+};
+
+namespace {
+
+int fail(h1b_ctx *ctx, int code, const char *fmt, ...) {
+    char buf[512];
+    va_list ap;
+    va_start(ap, fmt);
+    vsnprintf(buf, sizeof buf, fmt, ap);
+    va_end(ap);
+    if (ctx) ctx->err = buf; else g_init_error = buf;
+    return code;
+}
+
+#define H1B_CUDA(ctx, expr)                                                                   \
+    do {                                                                                      \
+        cudaError_t e_ = (expr);                                                              \
+        if (e_ != cudaSuccess)                                                                \
+            return fail(ctx, H1B_ERR_CUDA, "%s: %s (%s:%d)", #expr, cudaGetErrorString(e_),   \
+                        __FILE__, __LINE__);                                                  \
+    } while (0)
+
+template <class T>
+T *at(h1b_ctx *ctx, size_t off) { return reinterpret_cast<T *>(ctx->ws + off); }
+
+unsigned char *slab_ptr(h1b_ctx *ctx, int layer, int seq, int kvh) {
+    return ctx->ws + ctx->plan.cache +
+           ((size_t)(layer * ctx->cfg.max_batch + seq) * ctx->cfg.n_kv_heads + kvh) * ctx->plan.slab_bytes;
+}
+
+int check_layers(h1b_ctx *ctx, int layer_begin, int n_layers, int B) {
+    if (!ctx) return H1B_ERR_NULL;
+    if (layer_begin < 0 || n_layers < 1 || layer_begin + n_layers > ctx->cfg.n_layers)
+        return fail(ctx, H1B_ERR_INVALID_ARG, "layers [%d, %d) outside [0, %d)", layer_begin,
+                    layer_begin + n_layers, ctx->cfg.n_layers);
+    if (B < 1 || B > ctx->cfg.max_batch)
+        return fail(ctx, H1B_ERR_INVALID_ARG, "B = %d outside [1, %d]", B, ctx->cfg.max_batch);
+    return H1B_OK;
+}
+
+}  // namespace
+
+extern "C" {
+
+size_t h1b_entry_bytes(const h1b_config *cfg) {
+    if (check_config(cfg) != H1B_OK) return 0;
+    return (size_t)cfg->sketch_bits / 8 + (size_t)cfg->head_dim / 2 + (size_t)(cfg->head_dim / cfg->group_size) * 4;
+}
+
+size_t h1b_cache_bytes(const h1b_config *cfg) {
+    Plan p;
+    if (make_plan(cfg, &p) != H1B_OK) return 0;
+    return p.total;
+}
+
+int h1b_init_projection(const h1b_config *cfg, uint64_t seed, const float *Rt_host, void *workspace,
+                        size_t workspace_bytes, void *stream, h1b_ctx **out) {
+    if (!cfg || !out) return fail(nullptr, H1B_ERR_NULL, "cfg or out is NULL");
+    *out = nullptr;
+    Plan plan;
+    const int rc = make_plan(cfg, &plan);
+    if (rc != H1B_OK) return fail(nullptr, rc, "invalid or unsupported configuration");
+    if (!workspace) return fail(nullptr, H1B_ERR_NULL, "workspace is NULL");
+    if (workspace_bytes < plan.total || (reinterpret_cast<uintptr_t>(workspace) & 255u))
+        return fail(nullptr, H1B_ERR_WORKSPACE, "workspace needs %zu bytes, 256-byte aligned (got %zu at %p)",
+                    plan.total, workspace_bytes, workspace);
+    h1b_ctx *ctx = new (std::nothrow) h1b_ctx();
+    if (!ctx) return fail(nullptr, H1B_ERR_INVALID_ARG, "out of host memory");
+    ctx->cfg = *cfg;
+    ctx->plan = plan;
+    ctx->cl = chunk_layout(plan.m_words);
+    ctx->ws = static_cast<unsigned char *>(workspace);
+    ctx->len_host.assign((size_t)cfg->n_layers * cfg->max_batch, 0);
+    ctx->forced_splits = 0;
+    ctx->launches = 0;
+    cudaStream_t st = static_cast<cudaStream_t>(stream);
+    auto bail = [&](cudaError_t e, const char *what) {
+        fail(nullptr, H1B_ERR_CUDA, "%s: %s", what, cudaGetErrorString(e));
+        delete ctx;
+        return H1B_ERR_CUDA;
+    };
+    cudaError_t e = cudaSetDevice(cfg->device);
+    if (e != cudaSuccess) return bail(e, "cudaSetDevice");
+    // Every byte of the cache is a finite fp16 / small integer from here on, so
+    // tokens past a sequence's end can be read and weighted by zero.
+    e = cudaMemsetAsync(workspace, 0, plan.total, st);
+    if (e != cudaSuccess) return bail(e, "cudaMemsetAsync");
+    const size_t nR = (size_t)cfg->n_layers * cfg->head_dim * cfg->sketch_bits;
+    std::vector<float> gen;
+    if (!Rt_host) {
+        gen.resize(nR);
+        fill_gaussian(gen.data(), nR, seed);
+        Rt_host = gen.data();
+    }
+    e = cudaMemcpyAsync(ctx->ws + plan.rt, Rt_host, nR * sizeof(float), cudaMemcpyHostToDevice, st);
+    if (e != cudaSuccess) return bail(e, "cudaMemcpyAsync(Rt)");
+    e = cudaStreamSynchronize(st);
+    if (e != cudaSuccess) return bail(e, "cudaStreamSynchronize");
+    *out = ctx;
+    return H1B_OK;
+}
+
+int h1b_append_kv(h1b_ctx *ctx, int layer_begin, int n_layers, const void *k, const void *v,
+                  const int32_t *n_new_host, int B, int Tn, void *stream) {
+    int rc = check_layers(ctx, layer_begin, n_layers, B);
+    if (rc != H1B_OK) return rc;
+    if (!k || !v) return fail(ctx, H1B_ERR_NULL, "k or v is NULL");
+    if (Tn < 1) return fail(ctx, H1B_ERR_INVALID_ARG, "Tn = %d < 1", Tn);
+    NewCounts nn;
+    std::memset(&nn, 0, sizeof nn);
+    for (int b = 0; b < B; ++b) {
+        const int n = n_new_host ? n_new_host[b] : Tn;
+        if (n < 0 || n > Tn) return fail(ctx, H1B_ERR_INVALID_ARG, "n_new[%d] = %d outside [0, %d]", b, n, Tn);
+        nn.v[b] = n;
+    }
+    for (int l = layer_begin; l < layer_begin + n_layers; ++l)
+        for (int b = 0; b < B; ++b)
+            if ((long)ctx->len_host[(size_t)l * ctx->cfg.max_batch + b] + nn.v[b] > ctx->cfg.max_seq)
+                return fail(ctx, H1B_ERR_CAPACITY, "layer %d sequence %d: %d + %d tokens exceed max_seq %d", l, b,
+                            ctx->len_host[(size_t)l * ctx->cfg.max_batch + b], nn.v[b], ctx->cfg.max_seq);
+    AppendParams p;
+    p.k = static_cast<const uint16_t *>(k);
+    p.v = static_cast<const uint16_t *>(v);
+    p.Rt = at<float>(ctx, ctx->plan.rt);
+    p.cache = ctx->ws + ctx->plan.cache;
+    p.len = at<int32_t>(ctx, ctx->plan.len);
+    p.slab_bytes = ctx->plan.slab_bytes;
+    p.layer_begin = layer_begin; p.n_layers = n_layers; p.B = B; p.Tn = Tn;
+    p.Hkv = ctx->cfg.n_kv_heads; p.max_batch = ctx->cfg.max_batch; p.m_words = ctx->plan.m_words;
+    int launches = 0;
+    H1B_CUDA(ctx, launch_append(p, nn, static_cast<cudaStream_t>(stream), &launches));
+    ctx->launches += launches;
+    for (int l = layer_begin; l < layer_begin + n_layers; ++l)
+        for (int b = 0; b < B; ++b) ctx->len_host[(size_t)l * ctx->cfg.max_batch + b] += nn.v[b];
+    return H1B_OK;
+}
+
+int h1b_decode_attention(h1b_ctx *ctx, int layer_begin, int n_layers, const void *q, float inv_tau, void *out,
+                         int B, void *stream) {
+    int rc = check_layers(ctx, layer_begin, n_layers, B);
+    if (rc != H1B_OK) return rc;
+    if (!q || !out) return fail(ctx, H1B_ERR_NULL, "q or out is NULL");
+    if (!(inv_tau > 0.f) || !std::isfinite(inv_tau))
+        return fail(ctx, H1B_ERR_INVALID_ARG, "inv_tau must be finite and > 0");
+    cudaStream_t st = static_cast<cudaStream_t>(stream);
+    int launches = 0;
+    SketchParams sp;
+    sp.q = static_cast<const uint16_t *>(q);
+    sp.Rt = at<float>(ctx, ctx->plan.rt);
+    sp.qwords = at<uint32_t>(ctx, ctx->plan.qwords);
+    sp.layer_begin = layer_begin; sp.n_layers = n_layers; sp.B = B; sp.Hq = ctx->cfg.n_q_heads;
+    sp.max_batch = ctx->cfg.max_batch; sp.m_words = ctx->plan.m_words;
+    H1B_CUDA(ctx, launch_sketch(sp, st, &launches));
+
+    // Split the sequence so that there are about kTargetItems work items; the
+    // last split of a sequence is open-ended, so the result does not depend on
+    // how well the host's view of the lengths matches the device's.
+    const long slabs = (long)n_layers * B * ctx->cfg.n_kv_heads;
+    int maxlen = 1;
+    for (int l = layer_begin; l < layer_begin + n_layers; ++l)
+        for (int b = 0; b < B; ++b) maxlen = std::max(maxlen, ctx->len_host[(size_t)l * ctx->cfg.max_batch + b]);
+    long splits = ctx->forced_splits > 0 ? ctx->forced_splits : kTargetItems / slabs;
+    const long max_splits = std::max(1, maxlen / kMinSplitTokens);
+    if (ctx->forced_splits <= 0 && splits > max_splits) splits = max_splits;
+    if (splits < 1) splits = 1;
+    if ((size_t)(slabs * splits) > ctx->plan.partial_items)
+        return fail(ctx, H1B_ERR_INVALID_ARG, "%ld splits of %ld slabs exceed the split-K scratch", splits, slabs);
+    const int span = (maxlen + 255) / 256 * 256;
+    int split_tokens = (int)((span + splits - 1) / splits);
+    split_tokens = (split_tokens + kChunkTokens - 1) / kChunkTokens * kChunkTokens;
+
+    DecodeParams dp;
+    dp.cache = ctx->ws + ctx->plan.cache;
+    dp.len = at<int32_t>(ctx, ctx->plan.len);
+    dp.qwords = sp.qwords;
+    dp.partial = at<float>(ctx, ctx->plan.partial);
+    dp.out = static_cast<float *>(out);
+    dp.status = at<int32_t>(ctx, ctx->plan.status);
+    dp.slab_bytes = ctx->plan.slab_bytes;
+    dp.layer_begin = layer_begin; dp.n_layers = n_layers; dp.B = B; dp.Hkv = ctx->cfg.n_kv_heads;
+    dp.Hq = ctx->cfg.n_q_heads; dp.max_batch = ctx->cfg.max_batch; dp.m_words = ctx->plan.m_words;
+    dp.splits = (int)splits; dp.split_tokens = split_tokens;
+    dp.c2 = (float)(2.0 * (double)inv_tau * 1.4426950408889634 / (double)ctx->cfg.sketch_bits);
+    H1B_CUDA(ctx, launch_decode(dp, st, &launches));
+    ctx->launches += launches;
+    return H1B_OK;
+}
+
+int h1b_decode_step_host(h1b_ctx *ctx, const void *k_host, const void *v_host, const void *q_host, float inv_tau,
+                         void *out_host, int B, void *stream) {
+    if (!ctx) return H1B_ERR_NULL;
+    if (!k_host || !v_host || !q_host || !out_host) return fail(ctx, H1B_ERR_NULL, "a host buffer is NULL");
+    int rc = check_layers(ctx, 0, ctx->cfg.n_layers, B);
+    if (rc != H1B_OK) return rc;
+    cudaStream_t st = static_cast<cudaStream_t>(stream);
+    const size_t L = ctx->cfg.n_layers, d = ctx->cfg.head_dim;
+    const size_t kv_bytes = L * B * ctx->cfg.n_kv_heads * d * 2, q_bytes = L * B * ctx->cfg.n_q_heads * d * 2;
+    H1B_CUDA(ctx, cudaMemcpyAsync(ctx->ws + ctx->plan.stage_k, k_host, kv_bytes, cudaMemcpyHostToDevice, st));
+    H1B_CUDA(ctx, cudaMemcpyAsync(ctx->ws + ctx->plan.stage_v, v_host, kv_bytes, cudaMemcpyHostToDevice, st));
+    H1B_CUDA(ctx, cudaMemcpyAsync(ctx->ws + ctx->plan.stage_q, q_host, q_bytes, cudaMemcpyHostToDevice, st));
+    rc = h1b_append_kv(ctx, 0, ctx->cfg.n_layers, ctx->ws + ctx->plan.stage_k, ctx->ws + ctx->plan.stage_v, nullptr,
+                       B, 1, stream);
+    if (rc != H1B_OK) return rc;
+    rc = h1b_decode_attention(ctx, 0, ctx->cfg.n_layers, ctx->ws + ctx->plan.stage_q, inv_tau,
+                              ctx->ws + ctx->plan.stage_out, B, stream);
+    if (rc != H1B_OK) return rc;
+    H1B_CUDA(ctx, cudaMemcpyAsync(out_host, ctx->ws + ctx->plan.stage_out, q_bytes * 2, cudaMemcpyDeviceToHost, st));
+    H1B_CUDA(ctx, cudaStreamSynchronize(st));
+    return H1B_OK;
+}
+
+int h1b_free(h1b_ctx *ctx) {
+    if (!ctx) return H1B_ERR_NULL;
+    int rc = H1B_OK;
+    if (cudaSetDevice(ctx->cfg.device) != cudaSuccess || cudaDeviceSynchronize() != cudaSuccess) rc = H1B_ERR_CUDA;
+    delete ctx;
+    return rc;
+}
+
+int h1b_get_projection(h1b_ctx *ctx, int layer, float *Rt_host) {
+    if (!ctx) return H1B_ERR_NULL;
+    if (!Rt_host) return fail(ctx, H1B_ERR_NULL, "Rt_host is NULL");
+    if (layer < 0 || layer >= ctx->cfg.n_layers) return fail(ctx, H1B_ERR_INVALID_ARG, "layer %d out of range", layer);
+    const size_t n = (size_t)ctx->cfg.head_dim * ctx->cfg.sketch_bits;
+    H1B_CUDA(ctx, cudaDeviceSynchronize());
+    H1B_CUDA(ctx, cudaMemcpy(Rt_host, at<float>(ctx, ctx->plan.rt) + (size_t)layer * n, n * sizeof(float),
+                             cudaMemcpyDeviceToHost));
+    return H1B_OK;
+}
+
+int h1b_get_lengths(h1b_ctx *ctx, int layer, int32_t *len_host) {
+    if (!ctx) return H1B_ERR_NULL;
+    if (!len_host) return fail(ctx, H1B_ERR_NULL, "len_host is NULL");
+    if (layer < 0 || layer >= ctx->cfg.n_layers) return fail(ctx, H1B_ERR_INVALID_ARG, "layer %d out of range", layer);
+    const int mb = ctx->cfg.max_batch;
+    H1B_CUDA(ctx, cudaDeviceSynchronize());
+    H1B_CUDA(ctx, cudaMemcpy(len_host, at<int32_t>(ctx, ctx->plan.len) + (size_t)layer * mb, mb * sizeof(int32_t),
+                             cudaMemcpyDeviceToHost));
+    for (int b = 0; b < mb; ++b)
+        if (len_host[b] != ctx->len_host[(size_t)layer * mb + b])
+            return fail(ctx, H1B_ERR_INVALID_ARG, "layer %d sequence %d: device length %d, host mirror %d", layer, b,
+                        len_host[b], ctx->len_host[(size_t)layer * mb + b]);
+    return H1B_OK;
+}
+
+int h1b_truncate(h1b_ctx *ctx, int seq, int new_len) {
+    if (!ctx) return H1B_ERR_NULL;
+    const int mb = ctx->cfg.max_batch;
+    if (seq < -1 || seq >= mb) return fail(ctx, H1B_ERR_INVALID_ARG, "sequence %d out of range", seq);
+    if (new_len < 0) return fail(ctx, H1B_ERR_INVALID_ARG, "new_len %d < 0", new_len);
+    for (int l = 0; l < ctx->cfg.n_layers; ++l)
+        for (int b = 0; b < mb; ++b)
+            if ((seq < 0 || b == seq) && new_len > 0 && ctx->len_host[(size_t)l * mb + b] < new_len)
+                return fail(ctx, H1B_ERR_INVALID_ARG, "layer %d sequence %d holds %d < %d tokens", l, b,
+                            ctx->len_host[(size_t)l * mb + b], new_len);
+    H1B_CUDA(ctx, cudaDeviceSynchronize());
+    H1B_CUDA(ctx, launch_set_len(at<int32_t>(ctx, ctx->plan.len), ctx->cfg.n_layers, mb, seq, new_len, nullptr));
+    H1B_CUDA(ctx, cudaDeviceSynchronize());
+    for (int l = 0; l < ctx->cfg.n_layers; ++l)
+        for (int b = 0; b < mb; ++b)
+            if (seq < 0 || b == seq) ctx->len_host[(size_t)l * mb + b] = new_len;
+    return H1B_OK;
+}
+
+int h1b_reset(h1b_ctx *ctx, int seq) { return h1b_truncate(ctx, seq, 0); }
+
+int h1b_export_cache(h1b_ctx *ctx, int layer, int seq, int kv_head, int t0, int n, uint32_t *words, uint8_t *codes,
+                     uint16_t *scale, uint16_t *zero) {
+    if (!ctx) return H1B_ERR_NULL;
+    if (layer < 0 || layer >= ctx->cfg.n_layers || seq < 0 || seq >= ctx->cfg.max_batch || kv_head < 0 ||
+        kv_head >= ctx->cfg.n_kv_heads)
+        return fail(ctx, H1B_ERR_INVALID_ARG, "(layer %d, seq %d, kv_head %d) out of range", layer, seq, kv_head);
+    const int len = ctx->len_host[(size_t)layer * ctx->cfg.max_batch + seq];
+    if (t0 < 0 || n < 0 || t0 + n > len)
+        return fail(ctx, H1B_ERR_INVALID_ARG, "tokens [%d, %d) outside the cached [0, %d)", t0, t0 + n, len);
+    if (n == 0) return H1B_OK;
+    const ChunkLayout &cl = ctx->cl;
+    const int c_lo = t0 / kChunkTokens, c_hi = (t0 + n - 1) / kChunkTokens;
+    std::vector<unsigned char> raw((size_t)(c_hi - c_lo + 1) * cl.bytes);
+    H1B_CUDA(ctx, cudaDeviceSynchronize());
+    H1B_CUDA(ctx, cudaMemcpy(raw.data(), slab_ptr(ctx, layer, seq, kv_head) + (size_t)c_lo * cl.bytes, raw.size(),
+                             cudaMemcpyDeviceToHost));
+    const int mw = cl.m_words, d = ctx->cfg.head_dim;
+    for (int i = 0; i < n; ++i) {
+        const int t = t0 + i, tt = t % kChunkTokens;
+        const unsigned char *ch = raw.data() + (size_t)(t / kChunkTokens - c_lo) * cl.bytes;
+        if (words)
+            for (int w = 0; w < mw; ++w) std::memcpy(&words[(size_t)i * mw + w], ch + key_word_off(w, tt), 4);
+        if (codes)
+            for (int cb = 0; cb < d / 16; ++cb)
+                for (int r = 0; r < 8; ++r) {
+                    const unsigned char byte = ch[code_byte_off(cl, tt, cb, r)];
+                    codes[(size_t)i * d + cb * 16 + r] = byte & 15;
+                    codes[(size_t)i * d + cb * 16 + r + 8] = byte >> 4;
+                }
+        for (int g = 0; g < kGroups; ++g) {
+            if (scale) std::memcpy(&scale[(size_t)i * kGroups + g], ch + scale_off(cl, tt, g), 2);
+            if (zero) std::memcpy(&zero[(size_t)i * kGroups + g], ch + zero_off(cl, tt, g), 2);
+        }
+    }
+    return H1B_OK;
+}
+
+int h1b_debug_scores(h1b_ctx *ctx, int layer, int seq, int kv_head, const void *q, uint32_t *qwords_host,
+                     int32_t *score_host) {
+    if (!ctx) return H1B_ERR_NULL;
+    if (!q) return fail(ctx, H1B_ERR_NULL, "q is NULL");
+    if (layer < 0 || layer >= ctx->cfg.n_layers || seq < 0 || seq >= ctx->cfg.max_batch || kv_head < 0 ||
+        kv_head >= ctx->cfg.n_kv_heads)
+        return fail(ctx, H1B_ERR_INVALID_ARG, "(layer %d, seq %d, kv_head %d) out of range", layer, seq, kv_head);
+    const int len = ctx->len_host[(size_t)layer * ctx->cfg.max_batch + seq];
+    const int mw = ctx->plan.m_words;
+    // sketch the single query row with the layer's projection into the debug slot
+    SketchParams sp;
+    sp.q = static_cast<const uint16_t *>(q);
+    sp.Rt = at<float>(ctx, ctx->plan.rt) + (size_t)layer * ctx->cfg.head_dim * ctx->cfg.sketch_bits;
+    sp.qwords = at<uint32_t>(ctx, ctx->plan.dbg_q);
+    sp.layer_begin = 0; sp.n_layers = 1; sp.B = 1; sp.Hq = 1; sp.max_batch = 1; sp.m_words = mw;
+    int launches = 0;
+    H1B_CUDA(ctx, cudaDeviceSynchronize());
+    H1B_CUDA(ctx, launch_sketch(sp, nullptr, &launches));
+    H1B_CUDA(ctx, launch_debug_scores(slab_ptr(ctx, layer, seq, kv_head), sp.qwords, mw, len,
+                                      at<int32_t>(ctx, ctx->plan.dbg_s), nullptr));
+    H1B_CUDA(ctx, cudaDeviceSynchronize());
+    if (qwords_host)
+        H1B_CUDA(ctx, cudaMemcpy(qwords_host, sp.qwords, mw * sizeof(uint32_t), cudaMemcpyDeviceToHost));
+    if (score_host && len > 0)
+        H1B_CUDA(ctx, cudaMemcpy(score_host, at<int32_t>(ctx, ctx->plan.dbg_s), (size_t)len * sizeof(int32_t),
+                                 cudaMemcpyDeviceToHost));
+    return H1B_OK;
+}
+
+int h1b_set_splits(h1b_ctx *ctx, int splits) {
+    if (!ctx) return H1B_ERR_NULL;
+    if (splits < 0 || (size_t)splits > ctx->plan.partial_items)
+        return fail(ctx, H1B_ERR_INVALID_ARG, "splits %d outside [0, %zu]", splits, ctx->plan.partial_items);
+    ctx->forced_splits = splits;
+    return H1B_OK;
+}
+
+int h1b_poll_status(h1b_ctx *ctx) {
+    if (!ctx) return H1B_ERR_NULL;
+    int32_t s = 0;
+    H1B_CUDA(ctx, cudaMemcpy(&s, at<int32_t>(ctx, ctx->plan.status), sizeof s, cudaMemcpyDeviceToHost));
+    if (s == kStatusOk) return H1B_OK;
+    H1B_CUDA(ctx, cudaMemset(at<int32_t>(ctx, ctx->plan.status), 0, sizeof s));
+    return fail(ctx, H1B_ERR_TIMEOUT, "a kernel gave up a bounded wait (status %d)", s);
+}
+
+int64_t h1b_launch_count(const h1b_ctx *ctx) { return ctx ? ctx->launches : 0; }
+
+const char *h1b_last_error(const h1b_ctx *ctx) { return ctx ? ctx->err.c_str() : g_init_error.c_str(); }
+
+}  // extern "C"

@@ -1,0 +1,18 @@
+// Launch functions of the H1B-KV kernels (internal to the library).
+#pragma once
+#include <cuda_runtime.h>
+
+#include "h1b_layout.cuh"
+
+namespace h1b {
+
+// Each launcher enqueues on `st`, adds the number of kernels it launched to
+// *launches and returns the launch error, if any.
+cudaError_t launch_append(const AppendParams &p, const NewCounts &nn, cudaStream_t st, int *launches);
+cudaError_t launch_sketch(const SketchParams &p, cudaStream_t st, int *launches);
+cudaError_t launch_decode(const DecodeParams &p, cudaStream_t st, int *launches);
+cudaError_t launch_set_len(int32_t *len, int n_layers, int max_batch, int seq, int value, cudaStream_t st);
+cudaError_t launch_debug_scores(const unsigned char *slab, const uint32_t *qwords, int m_words, int len,
+                                int32_t *score, cudaStream_t st);
+
+}  // namespace h1b

@@ -1,0 +1,111 @@
+// Packed device layout of the H1B-KV cache and the parameter blocks shared by
+// the host API and the kernels.
+//
+// One slab per (layer, sequence, KV head), made of chunks of 32 tokens that are
+// contiguous in memory, so that a decode warp streams a slab with one bulk
+// copy per chunk:
+//
+//   chunk = [ key words ][ value codes ][ zero ][ scale ]
+//
+//   key words   uint32 [m/32][32 tokens]        word w of token t at w*128 + t*4
+//   value codes 2 blocks of 16 tokens x 128 channels x 4 bit = 2 x 1024 B, each
+//               laid out as the A operand of mma.m16n8k16 (channels x tokens):
+//               [half: channels 0-63 | 64-127][lane 0..31][4 words], word i of a
+//               lane holds, for channel block cb = half*4+i (16 channels) and
+//               r = lane/4, j = lane%4, the 8 codes
+//                 nibble 0: (channel cb*16+r,   token 2j)    nibble 4: (.., token 2j+1)
+//                 nibble 1: (channel cb*16+r+8, token 2j)    nibble 5: (.., token 2j+1)
+//                 nibble 2: (channel cb*16+r,   token 2j+8)  nibble 6: (.., token 2j+9)
+//                 nibble 3: (channel cb*16+r+8, token 2j+8)  nibble 7: (.., token 2j+9)
+//               so one token of one word is exactly one byte (two channels), and an
+//               append never has to read-modify-write.
+//   zero        fp16 [32 tokens][4 groups]
+//   scale       fp16 [2 blocks][4 groups][16 tokens]
+//
+// Bytes per token: m/8 + 64 + 8 + 8, the count of Section IV-B's storage
+// statement plus the fp16 scale and zero of each group.
+#pragma once
+#include <cstdint>
+#include <cstddef>
+
+namespace h1b {
+
+constexpr int kHeadDim = 128;
+constexpr int kGroup = 32;
+constexpr int kGroups = kHeadDim / kGroup;       // 4
+constexpr int kChunkTokens = 32;
+constexpr int kValBlockBytes = 1024;             // 16 tokens x 128 channels x 4 bit
+constexpr int kPartStride = 132;                 // floats per (item, head): acc[128], min Hamming, sum, pad
+
+struct ChunkLayout {
+    int m_words;      // m / 32
+    int val_off;      // byte offset of the value codes
+    int zero_off;
+    int scale_off;
+    int bytes;        // chunk size
+};
+
+__host__ __device__ inline ChunkLayout chunk_layout(int m_words) {
+    ChunkLayout c;
+    c.m_words = m_words;
+    c.val_off = m_words * 4 * kChunkTokens;
+    c.zero_off = c.val_off + 2 * kValBlockBytes;
+    c.scale_off = c.zero_off + kChunkTokens * kGroups * 2;
+    c.bytes = c.scale_off + kChunkTokens * kGroups * 2;
+    return c;
+}
+
+// Byte offset, inside a chunk, of key word w of token tt (0..31).
+__host__ __device__ inline int key_word_off(int w, int tt) { return w * 128 + tt * 4; }
+
+// Byte offset, inside a chunk, of the byte that holds the codes of channels
+// (cb*16 + r) [low nibble] and (cb*16 + r + 8) [high nibble] of token tt.
+__host__ __device__ inline int code_byte_off(const ChunkLayout &c, int tt, int cb, int r) {
+    int vb = tt >> 4, k = tt & 15;
+    int j = (k & 7) >> 1, odd = k & 1, hi8 = k >> 3;
+    int lane = r * 4 + j;
+    return c.val_off + vb * kValBlockBytes + (cb >> 2) * 512 + lane * 16 + (cb & 3) * 4 + odd * 2 + hi8;
+}
+__host__ __device__ inline int zero_off(const ChunkLayout &c, int tt, int g) {
+    return c.zero_off + tt * 8 + g * 2;
+}
+__host__ __device__ inline int scale_off(const ChunkLayout &c, int tt, int g) {
+    return c.scale_off + (tt >> 4) * 128 + g * 32 + (tt & 15) * 2;
+}
+
+// Device status word values.
+constexpr int kStatusOk = 0;
+constexpr int kStatusWaitTimeout = 1;
+
+struct NewCounts { int32_t v[256]; };            // n_new per sequence, passed by value
+
+struct AppendParams {
+    const uint16_t *k, *v;      // fp16 [n_layers][B][Tn][Hkv][d]
+    const float *Rt;            // [L][d][m]
+    unsigned char *cache;       // slab 0
+    int32_t *len;               // [L][max_batch]
+    size_t slab_bytes;
+    int layer_begin, n_layers, B, Tn, Hkv, max_batch, m_words;
+};
+
+struct SketchParams {           // query sketch
+    const uint16_t *q;          // fp16 [n_layers][B][Hq][d]
+    const float *Rt;
+    uint32_t *qwords;           // [L][max_batch][Hq][m/32]
+    int layer_begin, n_layers, B, Hq, max_batch, m_words;
+};
+
+struct DecodeParams {
+    const unsigned char *cache;
+    const int32_t *len;         // [L][max_batch]
+    const uint32_t *qwords;     // [L][max_batch][Hq][m/32]
+    float *partial;             // [items][GQ][kPartStride]
+    float *out;                 // fp32 [n_layers][B][Hq][d]
+    int32_t *status;
+    size_t slab_bytes;
+    int layer_begin, n_layers, B, Hkv, Hq, max_batch, m_words;
+    int splits, split_tokens;   // split_tokens is a multiple of 32
+    float c2;                   // 2 * inv_tau * log2(e) / m : log2-weight per unit of Hamming distance
+};
+
+}  // namespace h1b
