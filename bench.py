@@ -1,0 +1,346 @@
+#!/usr/bin/env python
+"""Benchmark of the H1B-KV decode hot path on B200.
+
+A step is one pass of the whole path over one batch of synthetic input: append
+the new token's K/V to every layer's compressed cache (Eq. 2, Eq. 4), then decode
+attention over every layer's cache (Eq. 3, Eq. 5). Workload at 1 GPU: the 7B
+shape (32 layers x 32 heads, d = 128, m = 128), one sequence, 8192-token context.
+
+  python bench.py [--gpus N] [--steps K] [--warmup W] [--impl ours|reference]
+
+Prints one JSON line (rank 0). With N > 1 (launched by torch.distributed.run)
+every rank runs its own sequence on its own GPU: independent units, no
+collective on the data path, weak scaling.
+
+`--impl reference` times the fp64 CPU oracle, as it stands, on the host cores,
+on a bounded sample of the same workload.
+"""
+from __future__ import annotations
+
+import argparse
+import json
+import os
+import sys
+import threading
+import time
+
+import numpy as np
+
+ROOT = os.path.dirname(os.path.abspath(__file__))
+if ROOT not in sys.path:
+    sys.path.insert(0, ROOT)
+
+METRIC = "decode-attn tokens/s (7B shape, 8k ctx): append 1 token + decode attention over 32 layers"
+UNIT = "tokens/s"
+INV_TAU = 16.0
+# DRAM bytes of one decode_split_kernel launch on the bench workload, from the ncu capture
+# summarised under profiles/ (dram__bytes_read.sum + dram__bytes_write.sum); None = not captured.
+NCU_TRAFFIC_BYTES_PER_LAUNCH = None
+
+
+def measured_peaks():
+    path = os.path.join(ROOT, "MEASURED_PEAKS.json")
+    try:
+        with open(path) as fh:
+            return float(json.load(fh)["hbm_gbs"]), "measured"
+    except Exception:
+        return 6650.0, "fallback"
+
+
+class ClockSampler(threading.Thread):
+    """Samples SM clock and clock-event reasons through NVML (read-only) while a region runs."""
+
+    def __init__(self, index: int):
+        super().__init__(daemon=True)
+        self.index, self.samples, self.reasons, self.max_mhz = index, [], set(), None
+        self._stop_evt = threading.Event()
+        self.ok = False
+        try:
+            import pynvml
+            pynvml.nvmlInit()
+            self.nv = pynvml
+            self.h = pynvml.nvmlDeviceGetHandleByIndex(index)
+            self.max_mhz = int(pynvml.nvmlDeviceGetMaxClockInfo(self.h, pynvml.NVML_CLOCK_SM))
+            self.ok = True
+        except Exception:
+            self.ok = False
+
+    def run(self):
+        if not self.ok:
+            return
+        nv = self.nv
+        names = {
+            "hw_slowdown": getattr(nv, "nvmlClocksEventReasonHwSlowdown", 0x8),
+            "hw_thermal_slowdown": getattr(nv, "nvmlClocksEventReasonHwThermalSlowdown", 0x40),
+            "sw_thermal_slowdown": getattr(nv, "nvmlClocksEventReasonSwThermalSlowdown", 0x20),
+            "sw_power_cap": getattr(nv, "nvmlClocksEventReasonSwPowerCap", 0x4),
+            "hw_power_brake": getattr(nv, "nvmlClocksEventReasonHwPowerBrakeSlowdown", 0x80),
+        }
+        get = getattr(nv, "nvmlDeviceGetCurrentClocksEventReasons", None) or \
+            getattr(nv, "nvmlDeviceGetCurrentClocksThrottleReasons")
+        while not self._stop_evt.is_set():
+            try:
+                self.samples.append(int(nv.nvmlDeviceGetClockInfo(self.h, nv.NVML_CLOCK_SM)))
+                mask = int(get(self.h))
+                for k, bit in names.items():
+                    if mask & bit:
+                        self.reasons.add(k)
+            except Exception:
+                break
+            time.sleep(0.002)
+
+    def stop(self):
+        self._stop_evt.set()
+        self.join(timeout=2)
+        med = float(np.median(self.samples)) if self.samples else None
+        return {"sm_mhz": med, "sm_max_mhz": self.max_mhz, "reasons": sorted(self.reasons),
+                "samples": len(self.samples)}
+
+
+def gpu_index() -> int:
+    """Physical index of the device this rank uses (for NVML)."""
+    local = int(os.environ.get("LOCAL_RANK", "0"))
+    vis = os.environ.get("CUDA_VISIBLE_DEVICES")
+    if vis:
+        ids = [x for x in vis.split(",") if x.strip()]
+        try:
+            return int(ids[local])
+        except Exception:
+            return local
+    return local
+
+
+# --------------------------------------------------------------------------- ours
+def run_ours(args):
+    import torch
+
+    import h1b_synth
+    from paper_2510_05529_b200 import binding
+
+    rank = int(os.environ.get("RANK", "0"))
+    world = int(os.environ.get("WORLD_SIZE", "1"))
+    local = int(os.environ.get("LOCAL_RANK", "0"))
+    if not torch.cuda.is_available():
+        raise SystemExit("bench.py needs a CUDA device: the hot path has no CPU fallback")
+    torch.cuda.set_device(local)
+    dist = None
+    if world > 1:
+        import torch.distributed as dist_mod
+        dist_mod.init_process_group("nccl", device_id=torch.device("cuda", local))
+        dist = dist_mod
+    dev = torch.device("cuda", local)
+    w = h1b_synth.WORKLOADS["c2_7b_8k"]
+    steps, warmup = args.steps, args.warmup
+    total_steps = 2 * (steps + warmup) + 8           # device-resident run, then the host-buffer run
+    prefill = w.context - 1                           # the first step decodes exactly `context` tokens
+    cfg = binding.make_config(w.n_layers, w.n_q_heads, w.n_kv_heads, w.head_dim, w.sketch_bits, w.group_size,
+                              max_batch=w.batch, max_seq=prefill + total_steps, device=local)
+    # each rank is its own sequence: different seeds per rank
+    wr = h1b_synth.scaled(w, index=w.index + 10 * rank)
+    Rt = np.stack([h1b_synth.projection(h1b_synth.layer_seed(wr, l, 99), w.head_dim, w.sketch_bits)
+                   for l in range(w.n_layers)])
+    cache = binding.H1BCache(cfg, Rt=Rt)
+    for l in range(w.n_layers):                       # prefill, one layer at a time
+        K, V = h1b_synth.kv_rows(wr, l, prefill, device=str(dev))
+        cache.h1b_append_kv(K.unsqueeze(0), V.unsqueeze(0), layer_begin=l)
+    torch.cuda.synchronize()
+    # per-step inputs: a pool of new tokens and queries, resident in HBM
+    pool = 16
+    kn = [torch.stack([h1b_synth.kv_rows(wr, l, 1, device=str(dev), stream=100 + i)[0] for l in range(w.n_layers)])
+          for i in range(pool)]
+    vn = [torch.stack([h1b_synth.kv_rows(wr, l, 1, device=str(dev), stream=100 + i)[1] for l in range(w.n_layers)])
+          for i in range(pool)]
+    qn = [torch.stack([h1b_synth.queries(wr, l, device=str(dev), stream=i) for l in range(w.n_layers)])
+          for i in range(pool)]
+    out = torch.empty((w.n_layers, w.batch, w.n_q_heads, w.head_dim), dtype=torch.float32, device=dev)
+    stream = torch.cuda.current_stream()
+
+    def step(i):
+        cache.h1b_append_kv(kn[i % pool], vn[i % pool])
+        cache.h1b_decode_attention(qn[i % pool], INV_TAU, out=out)
+
+    def barrier():
+        if dist is not None:
+            dist.barrier()
+        torch.cuda.synchronize()
+
+    for i in range(warmup):
+        step(i)
+    barrier()
+    launches0 = cache.h1b_launch_count()
+    cache.h1b_set_profiling(True)
+    cache.h1b_read_profile()
+    sampler = ClockSampler(gpu_index())
+    sampler.start()
+    ev0, ev1 = torch.cuda.Event(enable_timing=True), torch.cuda.Event(enable_timing=True)
+    ctx_first = int(cache.h1b_get_lengths(0)[0]) + 1
+    barrier()
+    ev0.record(stream)
+    for i in range(steps):
+        step(warmup + i)
+    ev1.record(stream)
+    barrier()
+    clocks = sampler.stop()
+    ms_total = ev0.elapsed_time(ev1)
+    launches = cache.h1b_launch_count() - launches0
+    kern_ms, kern_n = cache.h1b_read_profile()
+    cache.h1b_set_profiling(False)
+    cache.h1b_poll_status()
+    ctx_last = int(cache.h1b_get_lengths(0)[0])
+
+    # end to end through the host-buffer entry point: pinned host inputs, H2D and D2H inside the timed region
+    kh = [t.cpu().pin_memory() for t in kn]
+    vh = [t.cpu().pin_memory() for t in vn]
+    qh = [t.cpu().pin_memory() for t in qn]
+    oh = torch.empty(out.shape, dtype=torch.float32).pin_memory()
+    for i in range(min(warmup, 8)):
+        cache.h1b_decode_step_host(kh[i % pool], vh[i % pool], qh[i % pool], INV_TAU, oh)
+    barrier()
+    e0, e1 = torch.cuda.Event(enable_timing=True), torch.cuda.Event(enable_timing=True)
+    e0.record(stream)
+    for i in range(steps):
+        cache.h1b_decode_step_host(kh[i % pool], vh[i % pool], qh[i % pool], INV_TAU, oh)
+    e1.record(stream)
+    barrier()
+    e2e_ms_total = e0.elapsed_time(e1)
+
+    t = torch.tensor([ms_total, e2e_ms_total], dtype=torch.float64, device=dev)
+    if dist is not None:
+        dist.all_reduce(t, op=dist.ReduceOp.MAX)
+    ms_total, e2e_ms_total = float(t[0]), float(t[1])
+    tokens_per_step = w.batch * world
+    ms_per_step = ms_total / steps
+    value = tokens_per_step / (ms_per_step * 1e-3)
+    e2e_value = tokens_per_step / (e2e_ms_total / steps * 1e-3)
+
+    # roofline of the dominant kernel (split-K decode attention), per launch
+    entry = binding.h1b_entry_bytes(cfg)
+    ctx_mean = 0.5 * (ctx_first + ctx_last)
+    slabs = w.n_layers * w.batch * w.n_kv_heads
+    alg_bytes = slabs * ctx_mean * entry + w.n_layers * w.batch * w.n_q_heads * (w.sketch_bits // 8)
+    peak, peak_kind = measured_peaks()
+    kern_ms_avg = kern_ms / max(kern_n, 1)
+    achieved = alg_bytes / (kern_ms_avg * 1e-3) / 1e9 if kern_n else None
+    roofline = {"bound": "hbm", "kernel": "decode_split_kernel", "achieved": achieved, "peak": peak,
+                "peak_kind": peak_kind + " (MEASURED_PEAKS.json hbm_gbs)" if peak_kind == "measured" else "fallback",
+                "unit": "GB/s", "frac": (achieved / peak) if achieved else None,
+                "frac_of_8tbs_nominal": (achieved / 8000.0) if achieved else None,
+                "traffic": NCU_TRAFFIC_BYTES_PER_LAUNCH, "alg_bytes_per_launch": alg_bytes,
+                "kernel_ms_avg": kern_ms_avg, "kernel_launches_timed": kern_n,
+                "step_gbs": alg_bytes / (ms_per_step * 1e-3) / 1e9}
+    line = {
+        "metric": METRIC, "value": value, "unit": UNIT, "n_gpus": world, "steps": steps, "warmup": warmup,
+        "ms_per_step": ms_per_step, "higher_is_better": True, "scaling": "weak", "vs_baseline": None,
+        "dtype": "f32", "data": "synthetic",
+        "config": {"workload": "c2_7b_8k: 32 layers x 32 heads, d=128, m=128, batch 1 per GPU, fp16 K/V ~ N(0,1) with 1% "
+                               "outlier channels x8, one projection per layer",
+                   "ctx_first": ctx_first, "ctx_last": ctx_last, "inv_tau": INV_TAU,
+                   "cache_bytes": int(slabs * ctx_mean * entry),
+                   "l2": "working set (%.0f MB per step) is larger than L2; nothing is flushed" % (alg_bytes / 1e6)},
+        "e2e": {"value": e2e_value, "unit": UNIT, "ms_per_step": e2e_ms_total / steps,
+                "h2d_bytes_per_step": int(sum(x[0].numel() * 2 for x in (kh, vh, qh))),
+                "d2h_bytes_per_step": int(oh.numel() * 4)},
+        "gpu_launches": int(launches),
+        "clocks": clocks,
+        "roofline": roofline,
+    }
+    if rank == 0 and world == 1 and not args.no_cpu_baseline:
+        line["cpu_baseline"] = cpu_baseline(sample_layers=1, steps=5, warmup=1)
+    cache.close()
+    if dist is not None:
+        dist.barrier()
+        dist.destroy_process_group()
+    if rank == 0:
+        print(json.dumps(line))
+
+
+# --------------------------------------------------------------------------- oracle on host cores
+class OracleSample:
+    """The fp64 oracle, as it stands, on a bounded sample of the bench workload:
+    `sample_layers` of the 32 layers (all 32 heads, 8192 cached tokens each). One
+    decode step = compress the new token (Eq. 2, Eq. 4) and attend over the cached
+    history (Eq. 2 on q, Eq. 3, Eq. 5). The history is compressed once, untimed."""
+
+    def __init__(self, sample_layers: int = 1):
+        import torch
+
+        import h1b_synth
+        import oracle
+        self.oracle, self.w = oracle, h1b_synth.WORKLOADS["c2_7b_8k"]
+        w, T = self.w, self.w.context
+        self.layers = []
+        for l in range(sample_layers):
+            Rt = h1b_synth.projection(h1b_synth.layer_seed(w, l, 99), w.head_dim, w.sketch_bits)
+            K, V = h1b_synth.kv_rows(w, l, T)
+            q = h1b_synth.queries(w, l)
+            Kb = K.view(dtype=torch.int16).numpy().view(np.uint16)
+            Vb = V.view(dtype=torch.int16).numpy().view(np.uint16)
+            qb = q.view(dtype=torch.int16).numpy().view(np.uint16)
+            # the whole layer is compressed once; each timed step recompresses the newest token into slot T-1
+            cache = oracle.compress(Kb, Vb, Rt)
+            self.layers.append((Rt, Kb[:, T - 1:], Vb[:, T - 1:], qb, cache))
+        self.lens = np.full((w.batch,), T, dtype=np.int32)
+
+    def step(self) -> float:
+        """Seconds for one decode step over the sampled layers."""
+        o, T = self.oracle, self.w.context
+        t0 = time.perf_counter()
+        for Rt, k_new, v_new, qb, cache in self.layers:
+            new = o.compress(k_new, v_new, Rt)
+            for dst, src in zip(cache, new):
+                dst[:, :, T - 1:T] = src
+            o.decode_cached(cache, self.lens, qb, Rt, INV_TAU)
+        return time.perf_counter() - t0
+
+    def describe(self, n_timed: int):
+        w = self.w
+        return ("%d of %d layers (%d heads x %d cached tokens each), mean of %d timed steps, scaled to %d layers; "
+                "history compressed once outside the timed region"
+                % (len(self.layers), w.n_layers, w.n_kv_heads, w.context, n_timed, w.n_layers))
+
+
+def cpu_baseline(sample_layers: int = 1, steps: int = 3, warmup: int = 1, sample: OracleSample | None = None):
+    s = sample or OracleSample(sample_layers)
+    for _ in range(warmup):
+        s.step()
+    times = [s.step() for _ in range(max(1, steps))]
+    step_s = float(np.mean(times)) * s.w.n_layers / len(s.layers)
+    return {"value": s.w.batch / step_s, "unit": UNIT, "cores": s.oracle.threads(), "kind": "oracle",
+            "sample": s.describe(len(times)), "ms_per_step": step_s * 1e3}
+
+
+def run_reference(args):
+    rank = int(os.environ.get("RANK", "0"))
+    if rank != 0:
+        return
+    world = int(os.environ.get("WORLD_SIZE", "1"))
+    t0 = time.perf_counter()
+    steps = max(1, min(args.steps, 20))
+    base = cpu_baseline(sample_layers=1, steps=steps, warmup=max(1, min(args.warmup, 3)))
+    v = base["value"]
+    line = {"impl": "reference", "metric": METRIC, "value": v, "unit": UNIT, "n_gpus": world,
+            "steps": steps, "warmup": max(1, min(args.warmup, 3)), "ms_per_step": 1e3 / v, "higher_is_better": True,
+            "scaling": "weak", "vs_baseline": None, "dtype": "f64", "data": "synthetic",
+            "config": {"workload": "c2_7b_8k (bounded sample of it per step, see cpu_baseline.sample)"},
+            "cpu_baseline": base,
+            "e2e": {"value": v, "unit": UNIT, "h2d_bytes_per_step": 0, "d2h_bytes_per_step": 0},
+            "wall_s": time.perf_counter() - t0}
+    print(json.dumps(line))
+
+
+def main():
+    ap = argparse.ArgumentParser()
+    ap.add_argument("--gpus", type=int, default=1)
+    ap.add_argument("--steps", type=int, default=300)
+    ap.add_argument("--warmup", type=int, default=30)
+    ap.add_argument("--impl", default="ours", choices=["ours", "reference"])
+    ap.add_argument("--no-cpu-baseline", action="store_true")
+    args = ap.parse_args()
+    if args.impl == "reference":
+        run_reference(args)
+    else:
+        run_ours(args)
+
+
+if __name__ == "__main__":
+    main()

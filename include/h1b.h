@@ -166,6 +166,16 @@ int h1b_set_splits(h1b_ctx *ctx, int splits);
  * gave up a bounded wait since the last poll (the flag is cleared). */
 int h1b_poll_status(h1b_ctx *ctx);
 
+/* Time the dominant kernel. While enabled, every h1b_decode_attention() brackets
+ * the launch of its split-K attention kernel with a pair of CUDA events on the
+ * call's stream (at most 4096 pairs between two reads; later launches are not
+ * recorded). Events are created on the first enabling call. */
+int h1b_set_profiling(h1b_ctx *ctx, int enable);
+
+/* Synchronise the device, return the summed duration (milliseconds) and the
+ * number of the recorded kernel launches (both HOST), and forget them. */
+int h1b_read_profile(h1b_ctx *ctx, double *decode_ms, int64_t *decode_launches);
+
 /* Kernel launches enqueued by this context so far. */
 int64_t h1b_launch_count(const h1b_ctx *ctx);
 

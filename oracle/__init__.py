@@ -64,6 +64,10 @@ def _load():
             lib.h1bo_layer.argtypes = [u16p, u16p, i32p, u16p, f32p, ctypes.c_int, ctypes.c_long,
                                        ctypes.c_int, ctypes.c_int, ctypes.c_int, ctypes.c_int,
                                        ctypes.c_int, ctypes.c_double, f64p]
+            lib.h1bo_decode_cached.restype = ctypes.c_long
+            lib.h1bo_decode_cached.argtypes = [u8p, u8p, u16p, u16p, i32p, u16p, f32p, ctypes.c_int,
+                                               ctypes.c_long, ctypes.c_int, ctypes.c_int, ctypes.c_int,
+                                               ctypes.c_int, ctypes.c_int, ctypes.c_double, f64p]
             lib.h1bo_entry_bytes.restype = ctypes.c_long
             lib.h1bo_entry_bytes.argtypes = [ctypes.c_int, ctypes.c_int, ctypes.c_int]
             lib.h1bo_threads.restype = ctypes.c_int
@@ -183,6 +187,40 @@ def layer(K, V, lens, q, Rt, inv_tau: float, G: int = 32):
                              _ptr(ln, ctypes.c_int32), _ptr(qb, ctypes.c_uint16),
                              _ptr(Rt, ctypes.c_float), B, T, Hq, Hkv, d, m, G, float(inv_tau),
                              _ptr(out, ctypes.c_double))
+    if bad:
+        raise AssertionError("oracle: score identity violated %d times" % bad)
+    return out
+
+
+def compress(K, V, Rt, G: int = 32):
+    """Eq. 2 and Eq. 4 on K, V [B, T, Hkv, d] fp16 -> the unpacked cache
+    (kbits [B, Hkv, T, m], codes [B, Hkv, T, d], scale16, zero16 [B, Hkv, T, d/G])."""
+    Kb, Vb = _as_u16(K), _as_u16(V)
+    B, T, Hkv, d = Kb.shape
+    Kr = np.ascontiguousarray(Kb.transpose(0, 2, 1, 3)).reshape(B * Hkv * T, d)
+    Vr = np.ascontiguousarray(Vb.transpose(0, 2, 1, 3)).reshape(B * Hkv * T, d)
+    m = np.asarray(Rt).shape[1]
+    kbits = sketch(Kr, Rt).reshape(B, Hkv, T, m)
+    codes, s16, z16 = quantize(Vr, G)
+    return (kbits, codes.reshape(B, Hkv, T, d), s16.reshape(B, Hkv, T, d // G), z16.reshape(B, Hkv, T, d // G))
+
+
+def decode_cached(cache, lens, q, Rt, inv_tau: float, G: int = 32):
+    """One decode step over an unpacked cache from compress(). q [B, Hq, d] fp16 -> out fp64 [B, Hq, d]."""
+    kbits, codes, s16, z16 = (np.ascontiguousarray(a) for a in cache)
+    B, Hkv, T, m = kbits.shape
+    d = codes.shape[3]
+    qb = _as_u16(q)
+    Hq = qb.shape[1]
+    Rt = np.ascontiguousarray(Rt, dtype=np.float32)
+    ln = np.ascontiguousarray(lens, dtype=np.int32)
+    assert ln.shape == (B,) and int(ln.max(initial=0)) <= T and Rt.shape == (d, m)
+    out = np.zeros((B, Hq, d), dtype=np.float64)
+    bad = _load().h1bo_decode_cached(_ptr(kbits, ctypes.c_uint8), _ptr(codes, ctypes.c_uint8),
+                                     _ptr(s16, ctypes.c_uint16), _ptr(z16, ctypes.c_uint16),
+                                     _ptr(ln, ctypes.c_int32), _ptr(qb, ctypes.c_uint16),
+                                     _ptr(Rt, ctypes.c_float), B, T, Hq, Hkv, d, m, G, float(inv_tau),
+                                     _ptr(out, ctypes.c_double))
     if bad:
         raise AssertionError("oracle: score identity violated %d times" % bad)
     return out

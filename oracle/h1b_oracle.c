@@ -288,6 +288,44 @@ long h1bo_layer(const uint16_t *K, const uint16_t *V, const int32_t *lens,
     return bad_total;
 }
 
+/* ------------------------------------------------------------------------ */
+/* Decode step over an existing compressed cache (what one generated token    */
+/* costs once the history has been compressed): Eq. 2 on the queries, Eq. 3   */
+/* and Eq. 5 against the cached sketches and codes.                           */
+/*   kbits  [B][Hkv][T][m] (0/1 bytes), codes [B][Hkv][T][d],                 */
+/*   scale16, zero16 [B][Hkv][T][d/G]; T = stride, lens[b] tokens are used    */
+/*   q [B][Hq][d] binary16, out [B][Hq][d] fp64                               */
+/* OpenMP over the independent (sequence, KV head) units only.                */
+/* ------------------------------------------------------------------------ */
+long h1bo_decode_cached(const uint8_t *kbits, const uint8_t *codes, const uint16_t *scale16,
+                        const uint16_t *zero16, const int32_t *lens, const uint16_t *q,
+                        const float *Rt, int B, long T, int Hq, int Hkv, int d, int m, int G,
+                        double inv_tau, double *out)
+{
+    long bad_total = 0;
+    int ng = d / G, rep = Hq / Hkv;
+    long units = (long)B * Hkv;
+#ifdef _OPENMP
+#pragma omp parallel for schedule(dynamic, 1) reduction(+ : bad_total)
+#endif
+    for (long u = 0; u < units; ++u) {
+        int b = (int)(u / Hkv);
+        long len = lens[b];
+        int32_t *score = (int32_t *)malloc(sizeof(int32_t) * (size_t)(len > 0 ? len : 1));
+        uint8_t *qbits = (uint8_t *)malloc((size_t)m);
+        for (int r = 0; r < rep; ++r) {
+            int h = (int)(u % Hkv) * rep + r;
+            h1bo_sketch(q + ((size_t)b * Hq + h) * d, 1, d, m, Rt, qbits, NULL, NULL);
+            bad_total += h1bo_scores(qbits, kbits + (size_t)u * T * m, len, m, score);
+            h1bo_attention(score, len, m, inv_tau, codes + (size_t)u * T * d,
+                           scale16 + (size_t)u * T * ng, zero16 + (size_t)u * T * ng, d, G,
+                           out + ((size_t)b * Hq + h) * d, NULL);
+        }
+        free(score); free(qbits);
+    }
+    return bad_total;
+}
+
 /* Section IV-B storage statement: a token holds an m-bit sketch and d 4-bit
  * codes; this build also stores a binary16 scale and zero per group. */
 long h1bo_entry_bytes(int d, int m, int G)

@@ -69,6 +69,8 @@ def load_library(rebuild: bool = True) -> ctypes.CDLL:
         "h1b_debug_scores": (ctypes.c_int, [vp, ctypes.c_int, ctypes.c_int, ctypes.c_int, vp, vp, vp]),
         "h1b_set_splits": (ctypes.c_int, [vp, ctypes.c_int]),
         "h1b_poll_status": (ctypes.c_int, [vp]),
+        "h1b_set_profiling": (ctypes.c_int, [vp, ctypes.c_int]),
+        "h1b_read_profile": (ctypes.c_int, [vp, ctypes.POINTER(ctypes.c_double), ctypes.POINTER(ctypes.c_int64)]),
         "h1b_launch_count": (ctypes.c_int64, [vp]),
         "h1b_last_error": (ctypes.c_char_p, [vp]),
     }
@@ -238,6 +240,15 @@ class H1BCache:
 
     def h1b_poll_status(self):
         self._check(self.lib.h1b_poll_status(self._h))
+
+    def h1b_set_profiling(self, enable: bool):
+        self._check(self.lib.h1b_set_profiling(self._h, int(bool(enable))))
+
+    def h1b_read_profile(self):
+        """-> (summed split-K kernel time in ms, number of recorded launches)."""
+        ms, n = ctypes.c_double(), ctypes.c_int64()
+        self._check(self.lib.h1b_read_profile(self._h, ctypes.byref(ms), ctypes.byref(n)))
+        return float(ms.value), int(n.value)
 
     def h1b_launch_count(self) -> int:
         return int(self.lib.h1b_launch_count(self._h))

@@ -106,6 +106,9 @@ struct h1b_ctx {
     std::vector<int32_t> len_host;     // [L][max_batch], mirror of the device lengths
     int forced_splits;
     int64_t launches;
+    bool profiling;
+    std::vector<cudaEvent_t> events;   // pairs (before, after) around the split-K kernel
+    size_t events_used;
     std::string err;
 };
 
@@ -182,6 +185,8 @@ int h1b_init_projection(const h1b_config *cfg, uint64_t seed, const float *Rt_ho
     ctx->len_host.assign((size_t)cfg->n_layers * cfg->max_batch, 0);
     ctx->forced_splits = 0;
     ctx->launches = 0;
+    ctx->profiling = false;
+    ctx->events_used = 0;
     cudaStream_t st = static_cast<cudaStream_t>(stream);
     auto bail = [&](cudaError_t e, const char *what) {
         fail(nullptr, H1B_ERR_CUDA, "%s: %s", what, cudaGetErrorString(e));
@@ -290,7 +295,13 @@ int h1b_decode_attention(h1b_ctx *ctx, int layer_begin, int n_layers, const void
     dp.Hq = ctx->cfg.n_q_heads; dp.max_batch = ctx->cfg.max_batch; dp.m_words = ctx->plan.m_words;
     dp.splits = (int)splits; dp.split_tokens = split_tokens;
     dp.c2 = (float)(2.0 * (double)inv_tau * 1.4426950408889634 / (double)ctx->cfg.sketch_bits);
-    H1B_CUDA(ctx, launch_decode(dp, st, &launches));
+    cudaEvent_t ev0 = nullptr, ev1 = nullptr;
+    if (ctx->profiling && ctx->events_used + 2 <= ctx->events.size()) {
+        ev0 = ctx->events[ctx->events_used];
+        ev1 = ctx->events[ctx->events_used + 1];
+        ctx->events_used += 2;
+    }
+    H1B_CUDA(ctx, launch_decode(dp, st, &launches, ev0, ev1));
     ctx->launches += launches;
     return H1B_OK;
 }
@@ -322,6 +333,7 @@ int h1b_free(h1b_ctx *ctx) {
     if (!ctx) return H1B_ERR_NULL;
     int rc = H1B_OK;
     if (cudaSetDevice(ctx->cfg.device) != cudaSuccess || cudaDeviceSynchronize() != cudaSuccess) rc = H1B_ERR_CUDA;
+    for (cudaEvent_t e : ctx->events) cudaEventDestroy(e);
     delete ctx;
     return rc;
 }
@@ -454,6 +466,36 @@ int h1b_poll_status(h1b_ctx *ctx) {
     if (s == kStatusOk) return H1B_OK;
     H1B_CUDA(ctx, cudaMemset(at<int32_t>(ctx, ctx->plan.status), 0, sizeof s));
     return fail(ctx, H1B_ERR_TIMEOUT, "a kernel gave up a bounded wait (status %d)", s);
+}
+
+int h1b_set_profiling(h1b_ctx *ctx, int enable) {
+    if (!ctx) return H1B_ERR_NULL;
+    if (enable && ctx->events.empty()) {
+        ctx->events.reserve(8192);
+        for (int i = 0; i < 8192; ++i) {
+            cudaEvent_t e;
+            H1B_CUDA(ctx, cudaEventCreate(&e));
+            ctx->events.push_back(e);
+        }
+    }
+    ctx->profiling = enable != 0;
+    return H1B_OK;
+}
+
+int h1b_read_profile(h1b_ctx *ctx, double *decode_ms, int64_t *decode_launches) {
+    if (!ctx) return H1B_ERR_NULL;
+    if (!decode_ms || !decode_launches) return fail(ctx, H1B_ERR_NULL, "an output pointer is NULL");
+    H1B_CUDA(ctx, cudaDeviceSynchronize());
+    double sum = 0.0;
+    for (size_t i = 0; i + 1 < ctx->events_used; i += 2) {
+        float ms = 0.f;
+        H1B_CUDA(ctx, cudaEventElapsedTime(&ms, ctx->events[i], ctx->events[i + 1]));
+        sum += ms;
+    }
+    *decode_ms = sum;
+    *decode_launches = (int64_t)(ctx->events_used / 2);
+    ctx->events_used = 0;
+    return H1B_OK;
 }
 
 int64_t h1b_launch_count(const h1b_ctx *ctx) { return ctx ? ctx->launches : 0; }

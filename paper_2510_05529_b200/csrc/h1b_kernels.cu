@@ -474,15 +474,18 @@ static cudaError_t launch_decode_t(const DecodeParams &p, cudaStream_t st) {
     return cudaGetLastError();
 }
 
-cudaError_t launch_decode(const DecodeParams &p, cudaStream_t st, int *launches) {
+cudaError_t launch_decode(const DecodeParams &p, cudaStream_t st, int *launches, cudaEvent_t before,
+                          cudaEvent_t after) {
     const int gq = p.Hq / p.Hkv;
     cudaError_t e = cudaErrorInvalidValue;
+    if (before) cudaEventRecord(before, st);
     H1B_DISPATCH_MW(p.m_words,
         if (gq == 1) e = launch_decode_t<MW, 1>(p, st);
         else if (gq == 2) e = launch_decode_t<MW, 2>(p, st);
         else if (gq == 4) e = launch_decode_t<MW, 4>(p, st);
     );
     if (e != cudaSuccess) return e;
+    if (after) cudaEventRecord(after, st);
     ++*launches;
     combine_kernel<<<p.n_layers * p.B * p.Hq, kHeadDim, 0, st>>>(p);
     ++*launches;

@@ -10,7 +10,9 @@ namespace h1b {
 // *launches and returns the launch error, if any.
 cudaError_t launch_append(const AppendParams &p, const NewCounts &nn, cudaStream_t st, int *launches);
 cudaError_t launch_sketch(const SketchParams &p, cudaStream_t st, int *launches);
-cudaError_t launch_decode(const DecodeParams &p, cudaStream_t st, int *launches);
+// `before` / `after`, when not null, are recorded around the split-K attention kernel alone.
+cudaError_t launch_decode(const DecodeParams &p, cudaStream_t st, int *launches, cudaEvent_t before = nullptr,
+                          cudaEvent_t after = nullptr);
 cudaError_t launch_set_len(int32_t *len, int n_layers, int max_batch, int seq, int value, cudaStream_t st);
 cudaError_t launch_debug_scores(const unsigned char *slab, const uint32_t *qwords, int m_words, int len,
                                 int32_t *score, cudaStream_t st);

@@ -192,3 +192,16 @@ def test_entry_bytes_and_paper_cache_sizes():
     # printed 58.7 MB: the 4-bit values alone are 9x larger. Recorded, not enforced.
     stated = L * H * T * (256 // 8 + 128 // 2) / 1e6
     assert stated > 9 * rows[("7B", "H1BKV")]
+
+
+def test_decode_cached_equals_layer_driver():
+    """The cached decode step and the straight-from-fp16 layer driver are two routes to Eq. 5."""
+    rng = np.random.default_rng(14)
+    B, T, Hq, Hkv, d, m = 2, 50, 4, 2, 128, 128
+    Rt = rng.standard_normal((d, m)).astype(np.float32)
+    K = rng.standard_normal((B, T, Hkv, d)).astype(np.float16)
+    V = rng.standard_normal((B, T, Hkv, d)).astype(np.float16)
+    q = rng.standard_normal((B, Hq, d)).astype(np.float16)
+    lens = np.array([50, 23], np.int32)
+    cache = oracle.compress(K, V, Rt)
+    assert np.array_equal(oracle.decode_cached(cache, lens, q, Rt, 16.0), oracle.layer(K, V, lens, q, Rt, 16.0))
