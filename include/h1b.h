@@ -112,6 +112,41 @@ int h1b_append_kv(h1b_ctx *ctx, int layer_begin, int n_layers, const void *k, co
 int h1b_decode_attention(h1b_ctx *ctx, int layer_begin, int n_layers, const void *q,
                          float inv_tau, void *out, int B, void *stream);
 
+/* h1b_decode_attention() for callers that must not allocate and cannot spare
+ * scratch of their own. (No counterpart in the paper: this is a deployment
+ * convenience, not a step of the method.)
+ *
+ * Who this is for: code that runs after its process has handed all device
+ * memory to a fixed arena, a plug-in inside another runtime's region where
+ * cudaMalloc/cudaFree (and anything that calls them, a tensor library's
+ * allocator included) is forbidden or would synchronise the device, or a
+ * latency-critical loop that may not take the allocator's lock. Such callers
+ * still own the cache, q and out; what they lack is a place for this call's
+ * temporaries. Here the temporaries (the query sketches and the split-K
+ * partial results) live in an 8 MiB array built into the library image, so the
+ * call allocates nothing, frees nothing and writes nothing in the workspace's
+ * scratch region. Every device that loads the library holds those 8 MiB until
+ * the process exits.
+ *
+ * Same arguments, same result and same errors as h1b_decode_attention(), plus:
+ *   - H1B_ERR_CAPACITY, with the needed and the available byte counts in
+ *     h1b_last_error(), when even one split per sequence does not fit:
+ *     n_layers * B * Hkv * (Hq/Hkv) * 528 bytes of partials plus
+ *     L * max_batch * Hq * m/8 bytes of sketches must be <= 8 MiB. When more
+ *     splits would fit the automatic choice, fewer are used (slower, same result
+ *     up to summation order).
+ *   - the context's device must be the current device.
+ *   - the first call on each device looks up the array's device address
+ *     (cudaGetSymbolAddress) and keeps it; make that first call outside any
+ *     stream capture.
+ * All contexts and all calls in the process share the one array per device, and
+ * it keeps whatever the last call left in it. Nothing in it has to start at
+ * zero: every element a call reads was written earlier by the same call. Two
+ * calls whose kernels overlap on the GPU (different streams, different
+ * contexts) race on it: order them on one stream or with events. */
+int h1b_decode_attention_static(h1b_ctx *ctx, int layer_begin, int n_layers, const void *q,
+                                float inv_tau, void *out, int B, void *stream);
+
 /* The same step for callers whose tensors live in host memory: copies k, v, q
  * (HOST, fp16, [L][B][1][Hkv][d], [L][B][1][Hkv][d], [L][B][Hq][d]; pinned
  * memory makes the copies asynchronous) into staging inside the workspace,

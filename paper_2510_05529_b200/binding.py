@@ -58,6 +58,8 @@ def load_library(rebuild: bool = True) -> ctypes.CDLL:
                                          ctypes.c_int, vp]),
         "h1b_decode_attention": (ctypes.c_int, [vp, ctypes.c_int, ctypes.c_int, vp, ctypes.c_float, vp,
                                                 ctypes.c_int, vp]),
+        "h1b_decode_attention_static": (ctypes.c_int, [vp, ctypes.c_int, ctypes.c_int, vp, ctypes.c_float, vp,
+                                                       ctypes.c_int, vp]),
         "h1b_decode_step_host": (ctypes.c_int, [vp, vp, vp, vp, ctypes.c_float, vp, ctypes.c_int, vp]),
         "h1b_free": (ctypes.c_int, [vp]),
         "h1b_get_projection": (ctypes.c_int, [vp, ctypes.c_int, vp]),
@@ -181,6 +183,20 @@ class H1BCache:
             raise ValueError("out must have q's shape")
         self._check(self.lib.h1b_decode_attention(self._h, layer_begin, int(q.shape[0]), qp, float(inv_tau), op,
                                                   int(q.shape[1]), _stream_ptr(stream)))
+        return out
+
+    def h1b_decode_attention_static(self, q: torch.Tensor, inv_tau: float, out: torch.Tensor,
+                                    layer_begin: int = 0, stream=None) -> torch.Tensor:
+        """h1b_decode_attention for callers that must not allocate: the temporaries live in the
+        library's built-in 8 MiB device array, and `out` has to be supplied (nothing is created
+        here either). q fp16 CUDA [n_layers, B, Hq, d], out fp32 CUDA of the same shape. The
+        context's device must be current; calls that overlap on the GPU race on the shared array."""
+        qp = _dev_ptr(q, torch.float16, "q")
+        op = _dev_ptr(out, torch.float32, "out")
+        if q.dim() != 4 or q.shape[2] != self.cfg.n_q_heads or q.shape[3] != self.cfg.head_dim or out.shape != q.shape:
+            raise ValueError("q and out must be [n_layers, B, Hq, d]")
+        self._check(self.lib.h1b_decode_attention_static(self._h, layer_begin, int(q.shape[0]), qp, float(inv_tau),
+                                                         op, int(q.shape[1]), _stream_ptr(stream)))
         return out
 
     def h1b_decode_step_host(self, k: torch.Tensor, v: torch.Tensor, q: torch.Tensor, inv_tau: float,

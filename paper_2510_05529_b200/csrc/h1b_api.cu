@@ -306,6 +306,93 @@ int h1b_decode_attention(h1b_ctx *ctx, int layer_begin, int n_layers, const void
     return H1B_OK;
 }
 
+// ---------------------------------------------------------------------------
+// Decode attention without touching the workspace's scratch region and without
+// allocating anything: the query sketches and the split-K partials live in a
+// fixed array that is part of the library image. Every device that loads the
+// library carries these bytes until the process exits.
+// ---------------------------------------------------------------------------
+#define H1B_STATIC_SCRATCH_BYTES (8u << 20)
+static __device__ __align__(256) unsigned char h1b_static_scratch[H1B_STATIC_SCRATCH_BYTES];
+
+// In host code the name above is only a stand-in for the symbol, not a device
+// address; the address each device gave the array is looked up once per device.
+static void *g_static_scratch_addr[64] = {};
+
+// Never launched: a device-side reference, so that the array is certain to be kept in the image.
+__global__ void h1b_static_scratch_anchor(unsigned char *dst) {
+    if (dst) *dst = h1b_static_scratch[0];
+}
+
+int h1b_decode_attention_static(h1b_ctx *ctx, int layer_begin, int n_layers, const void *q, float inv_tau,
+                                void *out, int B, void *stream) {
+    int rc = check_layers(ctx, layer_begin, n_layers, B);
+    if (rc != H1B_OK) return rc;
+    if (!q || !out) return fail(ctx, H1B_ERR_NULL, "q or out is NULL");
+    if (!(inv_tau > 0.f) || !std::isfinite(inv_tau))
+        return fail(ctx, H1B_ERR_INVALID_ARG, "inv_tau must be finite and > 0");
+    const int dev = ctx->cfg.device;
+    if (dev < 0 || dev >= 64) return fail(ctx, H1B_ERR_UNSUPPORTED, "device ordinal %d outside [0, 64)", dev);
+    int cur = -1;
+    H1B_CUDA(ctx, cudaGetDevice(&cur));
+    if (cur != dev)
+        return fail(ctx, H1B_ERR_INVALID_ARG, "device %d must be current (current is %d)", dev, cur);
+    if (!g_static_scratch_addr[dev]) {          // first call on this device: resolve the array's address
+        void *p = nullptr;
+        H1B_CUDA(ctx, cudaGetSymbolAddress(&p, h1b_static_scratch));
+        if (!p) return fail(ctx, H1B_ERR_CUDA, "cudaGetSymbolAddress returned a null address");
+        g_static_scratch_addr[dev] = p;
+    }
+    unsigned char *scratch = static_cast<unsigned char *>(g_static_scratch_addr[dev]);
+
+    // carve: query sketches for every (layer, sequence, head) slot the kernels index, then the partials
+    const size_t qw_bytes = align_up((size_t)ctx->cfg.n_layers * ctx->cfg.max_batch * ctx->cfg.n_q_heads *
+                                         ctx->plan.m_words * sizeof(uint32_t), 256);
+    const long slabs = (long)n_layers * B * ctx->cfg.n_kv_heads;
+    const size_t item_bytes = (size_t)ctx->plan.gq * kPartStride * sizeof(float);
+    if (qw_bytes + (size_t)slabs * item_bytes > H1B_STATIC_SCRATCH_BYTES)
+        return fail(ctx, H1B_ERR_CAPACITY,
+                    "static scratch too small: this call needs at least %zu bytes, the built-in array holds %u",
+                    qw_bytes + (size_t)slabs * item_bytes, (unsigned)H1B_STATIC_SCRATCH_BYTES);
+    const long fit_splits = (long)((H1B_STATIC_SCRATCH_BYTES - qw_bytes) / item_bytes / (size_t)slabs);
+    int maxlen = 1;
+    for (int l = layer_begin; l < layer_begin + n_layers; ++l)
+        for (int b = 0; b < B; ++b) maxlen = std::max(maxlen, ctx->len_host[(size_t)l * ctx->cfg.max_batch + b]);
+    long splits = ctx->forced_splits > 0 ? ctx->forced_splits : kTargetItems / slabs;
+    const long max_splits = std::max(1, maxlen / kMinSplitTokens);
+    if (ctx->forced_splits <= 0 && splits > max_splits) splits = max_splits;
+    if (splits > fit_splits) splits = fit_splits;
+    if (splits < 1) splits = 1;
+    const int span = (maxlen + 255) / 256 * 256;
+    int split_tokens = (int)((span + splits - 1) / splits);
+    split_tokens = (split_tokens + kChunkTokens - 1) / kChunkTokens * kChunkTokens;
+
+    cudaStream_t st = static_cast<cudaStream_t>(stream);
+    int launches = 0;
+    SketchParams sp;
+    sp.q = static_cast<const uint16_t *>(q);
+    sp.Rt = at<float>(ctx, ctx->plan.rt);
+    sp.qwords = reinterpret_cast<uint32_t *>(scratch);
+    sp.layer_begin = layer_begin; sp.n_layers = n_layers; sp.B = B; sp.Hq = ctx->cfg.n_q_heads;
+    sp.max_batch = ctx->cfg.max_batch; sp.m_words = ctx->plan.m_words;
+    H1B_CUDA(ctx, launch_sketch(sp, st, &launches));
+    DecodeParams dp;
+    dp.cache = ctx->ws + ctx->plan.cache;
+    dp.len = at<int32_t>(ctx, ctx->plan.len);
+    dp.qwords = sp.qwords;
+    dp.partial = reinterpret_cast<float *>(scratch + qw_bytes);
+    dp.out = static_cast<float *>(out);
+    dp.status = at<int32_t>(ctx, ctx->plan.status);
+    dp.slab_bytes = ctx->plan.slab_bytes;
+    dp.layer_begin = layer_begin; dp.n_layers = n_layers; dp.B = B; dp.Hkv = ctx->cfg.n_kv_heads;
+    dp.Hq = ctx->cfg.n_q_heads; dp.max_batch = ctx->cfg.max_batch; dp.m_words = ctx->plan.m_words;
+    dp.splits = (int)splits; dp.split_tokens = split_tokens;
+    dp.c2 = (float)(2.0 * (double)inv_tau * 1.4426950408889634 / (double)ctx->cfg.sketch_bits);
+    H1B_CUDA(ctx, launch_decode(dp, st, &launches));
+    ctx->launches += launches;
+    return H1B_OK;
+}
+
 int h1b_decode_step_host(h1b_ctx *ctx, const void *k_host, const void *v_host, const void *q_host, float inv_tau,
                          void *out_host, int B, void *stream) {
     if (!ctx) return H1B_ERR_NULL;
