@@ -42,11 +42,14 @@ def load_library(rebuild: bool = True) -> ctypes.CDLL:
     global _lib
     if _lib is not None:
         return _lib
-    if rebuild and is_stale():
-        build_library()
-    if not os.path.exists(LIB_PATH):
-        raise RuntimeError("libh1b.so is missing and could not be built; there is no fallback path")
-    lib = ctypes.CDLL(LIB_PATH)
+    path = os.environ.get("H1B_LIBRARY_PATH")          # a prebuilt library elsewhere; default: the in-tree one
+    if not path:
+        path = LIB_PATH
+        if rebuild and is_stale():
+            build_library()
+    if not os.path.exists(path):
+        raise RuntimeError("%s is missing and could not be built; there is no fallback path" % path)
+    lib = ctypes.CDLL(path)
     vp, cp = ctypes.c_void_p, ctypes.POINTER(h1b_config)
     i32p = ctypes.POINTER(ctypes.c_int32)
     sig = {

@@ -238,6 +238,7 @@ int h1b_append_kv(h1b_ctx *ctx, int layer_begin, int n_layers, const void *k, co
     p.Rt = at<float>(ctx, ctx->plan.rt);
     p.cache = ctx->ws + ctx->plan.cache;
     p.len = at<int32_t>(ctx, ctx->plan.len);
+    p.done = at<int32_t>(ctx, ctx->plan.status) + 4;
     p.slab_bytes = ctx->plan.slab_bytes;
     p.layer_begin = layer_begin; p.n_layers = n_layers; p.B = B; p.Tn = Tn;
     p.Hkv = ctx->cfg.n_kv_heads; p.max_batch = ctx->cfg.max_batch; p.m_words = ctx->plan.m_words;

@@ -1,15 +1,15 @@
 // CUDA kernels of the H1B-KV hot path (sm_100a).
 //
-//   append_rows_kernel   Eq. 2 on new keys (fp32 FMA projection in ascending
-//                        channel order, sign, ballot-pack) and Eq. 4 on new
-//                        values (group min/max, fp16 scale, round-half-even
-//                        codes), written straight into the packed cache.
-//   sketch_rows_kernel   Eq. 2 on the queries of a decode step.
+//   append_kernel        Eq. 2 on new keys (tiled fp32 FMA projection in ascending
+//                        channel order, sign, pack) and Eq. 4 on new values (group
+//                        min/max, fp16 scale, round-half-even codes), written straight
+//                        into the packed cache; the last block bumps the lengths.
+//   sketch_kernel        Eq. 2 on the queries of a decode step.
 //   decode_split_kernel  Eq. 3 + Eq. 5 over one split of one (layer, sequence,
 //                        KV head) slab per warp: bulk-async chunk ring in shared
 //                        memory, XOR/popcount scores, online softmax on integer
-//                        Hamming distances, bf16 tensor-core P.V on integer codes
-//                        with the weights split into two bf16 parts.
+//                        Hamming distances, fp16 tensor-core P.V on the integer codes
+//                        with each weight split into two fp16 parts.
 //   combine_kernel       merges the split partials (flash-decoding style).
 #include "h1b_kernels.h"
 #include "h1b_ptx.cuh"
@@ -17,58 +17,74 @@
 namespace h1b {
 
 // ===========================================================================
-// Eq. 2: one warp projects one row. Lane l owns columns l, l+32, ... ; the sum
-// over input channels runs in ascending order with one fused multiply-add per
-// term, so the fp32 result is within 128 * 2^-24 of the exact projection
-// relative to the sum of absolute terms.
+// Eq. 2 on a tile of 32 rows x 32 sketch columns (one packed word per row).
+//
+// 128 threads. The projection tile Rt[128][32] and the rows (transposed to
+// [channel][row], padded) are staged in shared memory. Lane = row, warp w owns
+// columns 8w..8w+7 of the word. For every (row, column) the sum over the 128
+// input channels runs in ascending order with one fused multiply-add per term,
+// so the fp32 result is within 128 * 2^-24 of the exact projection relative to
+// the sum of absolute terms, and every launch shape gives the same bits.
 // ===========================================================================
-template <int MW>
-__device__ __forceinline__ void project_row(const uint16_t *__restrict__ x, const float *__restrict__ Rt,
-                                            int lane, uint32_t (&words)[MW]) {
-    float acc[MW];
-#pragma unroll
-    for (int w = 0; w < MW; ++w) acc[w] = 0.f;
-    const __half *xh = reinterpret_cast<const __half *>(x);
-#pragma unroll 8
-    for (int i = 0; i < kHeadDim; ++i) {
-        const float xi = __half2float(xh[i]);
-        const float *r = Rt + (size_t)i * (MW * 32) + lane;
-#pragma unroll
-        for (int w = 0; w < MW; ++w) acc[w] = __fmaf_rn(xi, __ldg(r + 32 * w), acc[w]);
+constexpr int kProjThreads = 128;
+constexpr int kProjRows = 32;
+
+struct ProjSmem {
+    float r[kHeadDim][32];               // Rt[:, 32*word .. 32*word+31]
+    float x[kHeadDim][kProjRows + 1];    // rows, transposed
+    unsigned char sig[kProjRows][4];     // sign bits, one byte per (row, warp)
+};
+
+// Returns, for threads 0..31, the packed word of row `tid` of the tile (other threads: unspecified).
+// x_rows: fp16 [n_rows][128], row-contiguous; rows beyond n_rows read as zero.
+__device__ __forceinline__ uint32_t project_tile(ProjSmem &sm, const uint16_t *__restrict__ x_rows, int n_rows,
+                                                 const float *__restrict__ Rt_layer, int m, int word) {
+    const int tid = threadIdx.x, lane = tid & 31, warp = tid >> 5;
+    // Rt tile: 128 x 32 floats, 128-byte rows
+    for (int e = tid; e < kHeadDim * 8; e += kProjThreads) {
+        const int i = e >> 3, c4 = e & 7;
+        const float4 v = __ldg(reinterpret_cast<const float4 *>(Rt_layer + (size_t)i * m + word * 32) + c4);
+        *reinterpret_cast<float4 *>(&sm.r[i][c4 * 4]) = v;
     }
+    // rows: coalesced half2 reads, transposed padded writes (conflict-free both ways)
+    for (int e = tid; e < kProjRows * (kHeadDim / 2); e += kProjThreads) {
+        const int row = e >> 6, c2 = e & 63;
+        float2 v = make_float2(0.f, 0.f);
+        if (row < n_rows) v = __half22float2(reinterpret_cast<const __half2 *>(x_rows + (size_t)row * kHeadDim)[c2]);
+        sm.x[2 * c2][row] = v.x;
+        sm.x[2 * c2 + 1][row] = v.y;
+    }
+    __syncthreads();
+    float acc[8];
 #pragma unroll
-    for (int w = 0; w < MW; ++w) words[w] = __ballot_sync(0xffffffffu, acc[w] >= 0.f);
+    for (int c = 0; c < 8; ++c) acc[c] = 0.f;
+#pragma unroll 4
+    for (int i = 0; i < kHeadDim; ++i) {
+        const float xv = sm.x[i][lane];
+        const float4 ra = *reinterpret_cast<const float4 *>(&sm.r[i][warp * 8]);
+        const float4 rb = *reinterpret_cast<const float4 *>(&sm.r[i][warp * 8 + 4]);
+        acc[0] = __fmaf_rn(xv, ra.x, acc[0]); acc[1] = __fmaf_rn(xv, ra.y, acc[1]);
+        acc[2] = __fmaf_rn(xv, ra.z, acc[2]); acc[3] = __fmaf_rn(xv, ra.w, acc[3]);
+        acc[4] = __fmaf_rn(xv, rb.x, acc[4]); acc[5] = __fmaf_rn(xv, rb.y, acc[5]);
+        acc[6] = __fmaf_rn(xv, rb.z, acc[6]); acc[7] = __fmaf_rn(xv, rb.w, acc[7]);
+    }
+    uint32_t bits = 0;
+#pragma unroll
+    for (int c = 0; c < 8; ++c) bits |= (acc[c] >= 0.f ? 1u : 0u) << c;
+    sm.sig[lane][warp] = (unsigned char)bits;
+    __syncthreads();
+    uint32_t word_bits = 0;
+    if (tid < kProjRows) word_bits = *reinterpret_cast<const uint32_t *>(sm.sig[tid]);
+    __syncthreads();                                      // the tile buffers may be reused by the caller
+    return word_bits;
 }
 
-template <int MW>
-__global__ void __launch_bounds__(256) append_rows_kernel(AppendParams p, NewCounts nn) {
-    const int lane = threadIdx.x & 31;
-    const long row = (long)blockIdx.x * (blockDim.x >> 5) + (threadIdx.x >> 5);
-    const long rows = (long)p.n_layers * p.B * p.Tn * p.Hkv;
-    if (row >= rows) return;
-    const int kvh = (int)(row % p.Hkv);
-    const int tn = (int)((row / p.Hkv) % p.Tn);
-    const int b = (int)((row / ((long)p.Hkv * p.Tn)) % p.B);
-    const int ll = (int)(row / ((long)p.Hkv * p.Tn * p.B));
-    if (tn >= nn.v[b]) return;
-    const int layer = p.layer_begin + ll;
-    const int t = p.len[layer * p.max_batch + b] + tn;
-    const ChunkLayout cl = chunk_layout(MW);
-    unsigned char *chunk = p.cache + ((size_t)(layer * p.max_batch + b) * p.Hkv + kvh) * p.slab_bytes +
-                           (size_t)(t >> 5) * cl.bytes;
-    const int tt = t & 31;
-
-    // ---- key sketch -----------------------------------------------------
-    uint32_t words[MW];
-    project_row<MW>(p.k + row * kHeadDim, p.Rt + (size_t)layer * kHeadDim * (MW * 32), lane, words);
-#pragma unroll
-    for (int w = 0; w < MW; ++w)
-        if (lane == w) *reinterpret_cast<uint32_t *>(chunk + key_word_off(w, tt)) = words[w];
-
-    // ---- value codes ------------------------------------------------------
+// Eq. 4 on one row by one warp, written into the packed cache.
+__device__ __forceinline__ void quantize_row(const uint16_t *__restrict__ v_row, unsigned char *chunk,
+                                             const ChunkLayout &cl, int tt, int lane) {
     // lane -> channel block cb = lane/4 and the channel pairs (2jj, 2jj+1), (2jj+8, 2jj+9)
     const int cb = lane >> 2, jj = lane & 3, g = lane >> 3;
-    const __half2 *vrow = reinterpret_cast<const __half2 *>(p.v + row * kHeadDim);
+    const __half2 *vrow = reinterpret_cast<const __half2 *>(v_row);
     const float2 va = __half22float2(vrow[(cb * 16 + 2 * jj) >> 1]);
     const float2 vb = __half22float2(vrow[(cb * 16 + 2 * jj + 8) >> 1]);
     float mn = fminf(fminf(va.x, va.y), fminf(vb.x, vb.y));
@@ -97,11 +113,62 @@ __global__ void __launch_bounds__(256) append_rows_kernel(AppendParams p, NewCou
     }
 }
 
-__global__ void bump_len_kernel(int32_t *len, int layer_begin, int n_layers, int B, int max_batch, NewCounts nn) {
-    const int i = blockIdx.x * blockDim.x + threadIdx.x;
-    if (i >= n_layers * B) return;
-    const int ll = i / B, b = i % B;
-    len[(layer_begin + ll) * max_batch + b] += nn.v[b];
+// One launch appends: blocks [0, proj_blocks) sketch key tiles, the rest quantise value rows (one warp per
+// row); the block that finishes last adds n_new to the lengths (every block has read them by then).
+__global__ void __launch_bounds__(kProjThreads) append_kernel(AppendParams p, NewCounts nn) {
+    __shared__ ProjSmem sm;
+    const int mw = p.m_words, m = mw * 32;
+    const ChunkLayout cl = chunk_layout(mw);
+    const int rows_per_layer = p.B * p.Tn * p.Hkv;
+    const int tiles_per_layer = (rows_per_layer + kProjRows - 1) / kProjRows;
+    const int proj_blocks = p.n_layers * tiles_per_layer * mw;
+    if ((int)blockIdx.x < proj_blocks) {
+        const int word = blockIdx.x % mw;
+        const int tile = (blockIdx.x / mw) % tiles_per_layer;
+        const int ll = blockIdx.x / (mw * tiles_per_layer);
+        const int layer = p.layer_begin + ll;
+        const int row0 = tile * kProjRows;
+        const int n_rows = min(kProjRows, rows_per_layer - row0);
+        const uint32_t bits = project_tile(sm, p.k + ((size_t)ll * rows_per_layer + row0) * kHeadDim, n_rows,
+                                           p.Rt + (size_t)layer * kHeadDim * m, m, word);
+        if ((int)threadIdx.x < n_rows) {
+            const int row = row0 + threadIdx.x;
+            const int kvh = row % p.Hkv, tn = (row / p.Hkv) % p.Tn, b = row / (p.Hkv * p.Tn);
+            if (tn < nn.v[b]) {
+                const int t = p.len[layer * p.max_batch + b] + tn;
+                unsigned char *chunk = p.cache + ((size_t)(layer * p.max_batch + b) * p.Hkv + kvh) * p.slab_bytes +
+                                       (size_t)(t >> 5) * cl.bytes;
+                *reinterpret_cast<uint32_t *>(chunk + key_word_off(word, t & 31)) = bits;
+            }
+        }
+    } else {
+        const long row = (long)(blockIdx.x - proj_blocks) * (kProjThreads / 32) + (threadIdx.x >> 5);
+        const long rows = (long)p.n_layers * rows_per_layer;
+        if (row < rows) {
+            const int kvh = (int)(row % p.Hkv), tn = (int)((row / p.Hkv) % p.Tn);
+            const int b = (int)((row / ((long)p.Hkv * p.Tn)) % p.B), ll = (int)(row / rows_per_layer);
+            if (tn < nn.v[b]) {
+                const int layer = p.layer_begin + ll;
+                const int t = p.len[layer * p.max_batch + b] + tn;
+                unsigned char *chunk = p.cache + ((size_t)(layer * p.max_batch + b) * p.Hkv + kvh) * p.slab_bytes +
+                                       (size_t)(t >> 5) * cl.bytes;
+                quantize_row(p.v + row * kHeadDim, chunk, cl, t & 31, threadIdx.x & 31);
+            }
+        }
+    }
+    // ---- the last block to finish publishes the new lengths
+    __shared__ int is_last;
+    __syncthreads();
+    if (threadIdx.x == 0) {
+        __threadfence();
+        is_last = (atomicAdd(p.done, 1) == (int)gridDim.x - 1);
+    }
+    __syncthreads();
+    if (is_last) {
+        for (int i = threadIdx.x; i < p.n_layers * p.B; i += blockDim.x)
+            p.len[(p.layer_begin + i / p.B) * p.max_batch + (i % p.B)] += nn.v[i % p.B];
+        if (threadIdx.x == 0) *p.done = 0;
+    }
 }
 
 __global__ void set_len_kernel(int32_t *len, int n_layers, int max_batch, int seq, int value) {
@@ -110,29 +177,57 @@ __global__ void set_len_kernel(int32_t *len, int n_layers, int max_batch, int se
     if (seq < 0 || (i % max_batch) == seq) len[i] = value;
 }
 
-template <int MW>
-__global__ void __launch_bounds__(256) sketch_rows_kernel(SketchParams p) {
-    const int lane = threadIdx.x & 31;
-    const long row = (long)blockIdx.x * (blockDim.x >> 5) + (threadIdx.x >> 5);
-    const long rows = (long)p.n_layers * p.B * p.Hq;
-    if (row >= rows) return;
-    const int h = (int)(row % p.Hq);
-    const int b = (int)((row / p.Hq) % p.B);
-    const int ll = (int)(row / ((long)p.Hq * p.B));
+// Eq. 2 on the queries of a decode step: one block per (layer, tile of 32 query rows, word).
+__global__ void __launch_bounds__(kProjThreads) sketch_kernel(SketchParams p) {
+    __shared__ ProjSmem sm;
+    const int mw = p.m_words, m = mw * 32;
+    const int rows_per_layer = p.B * p.Hq;
+    const int tiles_per_layer = (rows_per_layer + kProjRows - 1) / kProjRows;
+    const int word = blockIdx.x % mw;
+    const int tile = (blockIdx.x / mw) % tiles_per_layer;
+    const int ll = blockIdx.x / (mw * tiles_per_layer);
     const int layer = p.layer_begin + ll;
-    uint32_t words[MW];
-    project_row<MW>(p.q + row * kHeadDim, p.Rt + (size_t)layer * kHeadDim * (MW * 32), lane, words);
-    uint32_t *dst = p.qwords + ((size_t)(layer * p.max_batch + b) * p.Hq + h) * MW;
-#pragma unroll
-    for (int w = 0; w < MW; ++w)
-        if (lane == w) dst[w] = words[w];
+    const int row0 = tile * kProjRows;
+    const int n_rows = min(kProjRows, rows_per_layer - row0);
+    const uint32_t bits = project_tile(sm, p.q + ((size_t)ll * rows_per_layer + row0) * kHeadDim, n_rows,
+                                       p.Rt + (size_t)layer * kHeadDim * m, m, word);
+    if ((int)threadIdx.x < n_rows) {
+        const int row = row0 + threadIdx.x;
+        const int h = row % p.Hq, b = row / p.Hq;
+        p.qwords[((size_t)(layer * p.max_batch + b) * p.Hq + h) * mw + word] = bits;
+    }
 }
 
 // ===========================================================================
 // Decode: one warp per work item (layer, sequence, KV head, split).
+//
+// Per 32-token chunk (one bulk copy into this warp's ring in shared memory):
+//   phase 1  lane = token: Hamming distance to each query head of the GQA group
+//            (XOR + popcount), running minimum over the warp (redux), softmax
+//            weight p = 2 * 2^((hmin - ham) * c2), running sum, and the zero-point
+//            term sum_t p_t * zero_tg, all per lane; p goes to shared memory.
+//   phase 2  two blocks of 16 tokens: out^T (channels x columns) += codes^T x W on
+//            the tensor cores (mma.m16n8k16, fp16 in, fp32 accumulate).
+//            A = codes, two per register, masked in place from the packed words as fp16
+//            subnormals (code * 2^-20): no bias to add or remove, no conversion; three
+//            shifts and four ANDs per 8 codes (see codes_to_f16x2).
+//            B = weights x = p * scale (fp32) split as hi = fp16(x) and
+//            lo = fp16((x - hi) * 2^11) in two columns with their own accumulators:
+//            x = hi + lo * 2^-11 to 2^-22 relative (2^-36 absolute), whatever the
+//            magnitudes, so fp16's narrow exponent never costs accuracy. x <= 2 * 8734.
 // ===========================================================================
-constexpr int kDecodeWarps = 4;
-constexpr int kStages = 4;
+// Build-time tunables of the decode kernel.
+#ifndef H1B_DECODE_WARPS
+#define H1B_DECODE_WARPS 4          // warps (work items) per block
+#endif
+#ifndef H1B_DECODE_STAGES
+#define H1B_DECODE_STAGES 3         // chunks in flight per warp
+#endif
+#ifndef H1B_DECODE_MIN_BLOCKS
+#define H1B_DECODE_MIN_BLOCKS 1     // resident blocks per SM the register allocation must allow
+#endif
+constexpr int kDecodeWarps = H1B_DECODE_WARPS;
+constexpr int kStages = H1B_DECODE_STAGES;
 constexpr unsigned long long kWaitLimitNs = 2000000000ull;   // 2 s, then give up
 constexpr int kHamSentinel = 1 << 20;
 
@@ -144,12 +239,125 @@ struct DecodeSmem {
 };
 
 template <int MW, int GQ>
-__global__ void __launch_bounds__(kDecodeWarps * 32) decode_split_kernel(DecodeParams p) {
-    using SM = DecodeSmem<MW, GQ>;
-    constexpr int CB = SM::kChunkBytes;
+struct DecodeState {
+    float acc[8][4];            // per channel block of 16: C fragment (rows r, r+8; columns 2jq, 2jq+1)
+    int hmin[GQ];               // running minimum Hamming distance (= running maximum logit)
+    float ssum[GQ];             // per-lane partial sum of the weights
+    float accz[GQ][kGroups];    // per-lane partial sum of p * zero
+    uint32_t qw[GQ][MW];        // query sketches
+};
+
+// One chunk. TAIL: tokens at or beyond t_end are masked (only the last chunk of a split needs it).
+template <int MW, int GQ, bool TAIL>
+__device__ __forceinline__ void decode_chunk(DecodeState<MW, GQ> &st, const unsigned char *ch, float *p_s,
+                                             int lane, int n_valid, float c2) {
     constexpr int NG = 4 / GQ;                 // value groups covered by one B fragment
     constexpr int NB = GQ;                     // B fragments per 16-token block
     constexpr int VAL = MW * 128, ZERO = VAL + 2048, SCALE = ZERO + 256;
+    const int jq = lane & 3;
+
+    // ---------------- phase 1
+    const bool valid = !TAIL || lane < n_valid;
+    uint32_t kw[MW];
+#pragma unroll
+    for (int w = 0; w < MW; ++w) kw[w] = *reinterpret_cast<const uint32_t *>(ch + w * 128 + lane * 4);
+    const uint2 zraw = *reinterpret_cast<const uint2 *>(ch + ZERO + lane * 8);
+    const float2 z01 = half2_bits_to_float2(zraw.x), z23 = half2_bits_to_float2(zraw.y);
+    float scl[GQ];
+#pragma unroll
+    for (int h = 0; h < GQ; ++h) {
+        int ham = 0;
+#pragma unroll
+        for (int w = 0; w < MW; ++w) ham += __popc(kw[w] ^ st.qw[h][w]);
+        const int cmin = __reduce_min_sync(0xffffffffu, (TAIL && !valid) ? kHamSentinel : ham);
+        scl[h] = 1.f;
+        if (cmin < st.hmin[h]) {                            // warp-uniform: the running max moved
+            scl[h] = ex2_approx((float)(cmin - st.hmin[h]) * c2);
+            st.hmin[h] = cmin;
+            st.ssum[h] *= scl[h];                           // rescale what predates this chunk
+#pragma unroll
+            for (int g = 0; g < kGroups; ++g) st.accz[h][g] *= scl[h];
+        }
+        // p carries the static factor 2 of the weights (removed when the partial is written)
+        float pv = ex2_approx(fmaf((float)(st.hmin[h] - ham), c2, 1.f));
+        if (TAIL) pv = valid ? pv : 0.f;
+        st.ssum[h] += pv;
+        st.accz[h][0] = fmaf(pv, z01.x, st.accz[h][0]);
+        st.accz[h][1] = fmaf(pv, z01.y, st.accz[h][1]);
+        st.accz[h][2] = fmaf(pv, z23.x, st.accz[h][2]);
+        st.accz[h][3] = fmaf(pv, z23.y, st.accz[h][3]);
+        p_s[h * 32 + lane] = pv;
+    }
+    // factors by which this lane's accumulator columns 2jq, 2jq+1 shrink when a running max moved (else 1)
+    float f0, f1;
+    if (GQ == 1) { f0 = scl[0]; f1 = scl[0]; }
+    else if (GQ == 2) { f0 = scl[0]; f1 = scl[GQ > 1 ? 1 : 0]; }
+    else { f0 = (jq & 1) ? scl[GQ > 2 ? 2 : 0] : scl[0]; f1 = (jq & 1) ? scl[GQ > 3 ? 3 : 0] : scl[GQ > 1 ? 1 : 0]; }
+    __syncwarp();
+
+    // ---------------- phase 2
+    // Column n = lane/4 of a B fragment is (part, idx): part 0 = hi, part 1 = lo; idx = value group (GQ 1),
+    // (group in pair, head) (GQ 2) or head (GQ 4). This lane computes the weights of ONE token pair
+    // (tokens 2jq, 2jq+1 if part 0, else 2jq+8, 2jq+9), both parts, and swaps one of them with lane ^ 16.
+    const int part = lane >> 4, idx = (lane >> 2) & 3;
+    const int bhead = (GQ == 1) ? 0 : (GQ == 2 ? (idx & 1) : idx);
+    const int bgsel = (GQ == 1) ? idx : (GQ == 2 ? (idx >> 1) : 0);
+    const int tp = 2 * jq + 8 * part;                       // first token of this lane's pair within a block
+    uint32_t bf[2][NB][2];
+#pragma unroll
+    for (int vb = 0; vb < 2; ++vb) {
+        const float2 pp = *reinterpret_cast<const float2 *>(p_s + bhead * 32 + vb * 16 + tp);
+#pragma unroll
+        for (int bi = 0; bi < NB; ++bi) {
+            const int g = bi * NG + bgsel;
+            const float2 dd = half2_bits_to_float2(
+                *reinterpret_cast<const uint32_t *>(ch + SCALE + vb * 128 + g * 32 + tp * 2));
+            const float x0 = pp.x * dd.x, x1 = pp.y * dd.y;
+            const uint32_t hi = pack_f16x2(x0, x1);
+            const float2 hf = half2_bits_to_float2(hi);
+            const uint32_t lo = pack_f16x2((x0 - hf.x) * 2048.f, (x1 - hf.y) * 2048.f);
+            const uint32_t got = __shfl_xor_sync(0xffffffffu, part ? hi : lo, 16);
+            bf[vb][bi][0] = part ? got : hi;                // tokens 2jq, 2jq+1 of this lane's column
+            bf[vb][bi][1] = part ? lo : got;                // tokens 2jq+8, 2jq+9
+        }
+    }
+    // The tensor core truncates when it adds into its fp32 accumulator, a bias that grows with the length of
+    // the chain. So each chunk's two MMAs per channel block start from zero, and their sum is folded into the
+    // running accumulators with one round-to-nearest FMA, which applies the softmax rescale at the same time.
+    // Four channel blocks at a time keep the temporaries to 16 registers.
+#pragma unroll
+    for (int half = 0; half < 2; ++half) {
+        float tmp[4][4];
+#pragma unroll
+        for (int vb = 0; vb < 2; ++vb) {
+            const uint4 wq = *reinterpret_cast<const uint4 *>(ch + VAL + vb * 1024 + half * 512 + lane * 16);
+            const uint32_t wv[4] = {wq.x, wq.y, wq.z, wq.w};
+#pragma unroll
+            for (int i = 0; i < 4; ++i) {
+                const int cb = half * 4 + i;
+                const int bi = (cb >> 1) / NG;
+                uint32_t a[4];
+                codes_to_f16x2(wv[i], a);
+                if (vb == 0) mma_f16_16816_zero(tmp[i], a[0], a[1], a[2], a[3], bf[vb][bi][0], bf[vb][bi][1]);
+                else mma_f16_16816(tmp[i], a[0], a[1], a[2], a[3], bf[vb][bi][0], bf[vb][bi][1]);
+            }
+        }
+#pragma unroll
+        for (int i = 0; i < 4; ++i) {
+            const int cb = half * 4 + i;
+            st.acc[cb][0] = fmaf(st.acc[cb][0], f0, tmp[i][0]);
+            st.acc[cb][1] = fmaf(st.acc[cb][1], f1, tmp[i][1]);
+            st.acc[cb][2] = fmaf(st.acc[cb][2], f0, tmp[i][2]);
+            st.acc[cb][3] = fmaf(st.acc[cb][3], f1, tmp[i][3]);
+        }
+    }
+    __syncwarp();
+}
+
+template <int MW, int GQ>
+__global__ void __launch_bounds__(kDecodeWarps * 32, H1B_DECODE_MIN_BLOCKS) decode_split_kernel(DecodeParams p) {
+    using SM = DecodeSmem<MW, GQ>;
+    constexpr int CB = SM::kChunkBytes;
     extern __shared__ __align__(128) unsigned char smem_raw[];
 
     const int lane = threadIdx.x & 31, warp = threadIdx.x >> 5;
@@ -167,7 +375,7 @@ __global__ void __launch_bounds__(kDecodeWarps * 32) decode_split_kernel(DecodeP
     if (t_begin >= len) return;                                 // empty item: combine skips it too
     // the last split of a sequence is open-ended: it runs to the sequence's end
     const int t_end = (split == p.splits - 1) ? len : min(len, t_begin + p.split_tokens);
-    const int c0 = t_begin >> 5, c1 = (t_end + 31) >> 5;
+    const int c0 = t_begin >> 5, c_full = t_end >> 5, c1 = (t_end + 31) >> 5;
 
     unsigned char *ring = smem_raw + warp * SM::kPerWarp;
     float *p_s = reinterpret_cast<float *>(ring + kStages * CB);
@@ -182,141 +390,59 @@ __global__ void __launch_bounds__(kDecodeWarps * 32) decode_split_kernel(DecodeP
         mbar_fence_init();
     }
     __syncwarp();
+    const unsigned char *src = slab + (size_t)c0 * CB;          // next chunk to request
+    int requested = c0;
     if (lane == 0) {
-        for (int s = 0; s < kStages && c0 + s < c1; ++s) {
+        for (int s = 0; s < kStages && requested < c1; ++s, ++requested, src += CB) {
             mbar_arrive_expect_tx(bar0 + 8 * s, CB);
-            bulk_copy_g2s(ring_a + s * CB, slab + (size_t)(c0 + s) * CB, CB, bar0 + 8 * s);
+            bulk_copy_g2s(ring_a + s * CB, src, CB, bar0 + 8 * s);
         }
     }
 
-    // query sketches of the GQ heads that share this KV head
-    uint32_t qw[GQ][MW];
+    DecodeState<MW, GQ> st;
     {
         const uint32_t *qp = p.qwords + ((size_t)(layer * p.max_batch + b) * p.Hq + kvh * GQ) * MW;
 #pragma unroll
         for (int h = 0; h < GQ; ++h)
 #pragma unroll
-            for (int w = 0; w < MW; ++w) qw[h][w] = __ldg(qp + h * MW + w);
+            for (int w = 0; w < MW; ++w) st.qw[h][w] = __ldg(qp + h * MW + w);
     }
-
-    float acc[8][4];
 #pragma unroll
     for (int cb = 0; cb < 8; ++cb)
 #pragma unroll
-        for (int i = 0; i < 4; ++i) acc[cb][i] = 0.f;
-    int hmin[GQ];
-    float ssum[GQ], accz[GQ][kGroups];
+        for (int i = 0; i < 4; ++i) st.acc[cb][i] = 0.f;
 #pragma unroll
     for (int h = 0; h < GQ; ++h) {
-        hmin[h] = kHamSentinel;
-        ssum[h] = 0.f;
+        st.hmin[h] = kHamSentinel;
+        st.ssum[h] = 0.f;
 #pragma unroll
-        for (int g = 0; g < kGroups; ++g) accz[h][g] = 0.f;
+        for (int g = 0; g < kGroups; ++g) st.accz[h][g] = 0.f;
     }
 
-    // role of this lane when it builds a B fragment: column n = lane/4 of the
-    // 16x8 operand is (part, idx): part 0 = high bf16 part of the weight, 1 = low
-    const int jq = lane & 3;
-    const int part = lane >> 4, idx = (lane >> 2) & 3;
-    const int bhead = (GQ == 1) ? 0 : (GQ == 2 ? (idx & 1) : idx);
-    const int bgsel = (GQ == 1) ? idx : (GQ == 2 ? (idx >> 1) : 0);
-
-    int it = 0;
+    int stage = 0;
+    uint32_t parity = 0;
     bool failed = false;
-    for (int c = c0; c < c1; ++c, ++it) {
-        const int s = it % kStages;
-        const uint32_t parity = (it / kStages) & 1;
-        if (!mbar_wait_bounded(bar0 + 8 * s, parity, kWaitLimitNs)) { failed = true; break; }
-        const unsigned char *ch = ring + s * CB;
-
-        // ---------------- phase 1: scores and softmax weights, lane = token
-        const bool valid = (c * 32 + lane) < t_end;
-        uint32_t kw[MW];
-#pragma unroll
-        for (int w = 0; w < MW; ++w) kw[w] = *reinterpret_cast<const uint32_t *>(ch + w * 128 + lane * 4);
-        const uint2 zraw = *reinterpret_cast<const uint2 *>(ch + ZERO + lane * 8);
-        const float2 z01 = half2_bits_to_float2(zraw.x), z23 = half2_bits_to_float2(zraw.y);
-        float scl[GQ];
-        bool any = false;
-#pragma unroll
-        for (int h = 0; h < GQ; ++h) {
-            int ham = 0;
-#pragma unroll
-            for (int w = 0; w < MW; ++w) ham += __popc(kw[w] ^ qw[h][w]);
-            const int cmin = __reduce_min_sync(0xffffffffu, valid ? ham : kHamSentinel);
-            scl[h] = 1.f;
-            if (cmin < hmin[h]) {                               // warp-uniform: the running max moved
-                scl[h] = ex2_approx((float)(cmin - hmin[h]) * p.c2);
-                hmin[h] = cmin;
-                any = true;
-                ssum[h] *= scl[h];                              // rescale what predates this chunk
-#pragma unroll
-                for (int g = 0; g < kGroups; ++g) accz[h][g] *= scl[h];
-            }
-            const float pv = valid ? ex2_approx((float)(hmin[h] - ham) * p.c2) : 0.f;
-            ssum[h] += pv;
-            accz[h][0] = fmaf(pv, z01.x, accz[h][0]);
-            accz[h][1] = fmaf(pv, z01.y, accz[h][1]);
-            accz[h][2] = fmaf(pv, z23.x, accz[h][2]);
-            accz[h][3] = fmaf(pv, z23.y, accz[h][3]);
-            p_s[h * 32 + lane] = pv;
+    for (int c = c0; c < c1; ++c) {
+        if (!mbar_wait_bounded(bar0 + 8 * stage, parity, kWaitLimitNs)) { failed = true; break; }
+        const unsigned char *ch = ring + stage * CB;
+        if (c < c_full) decode_chunk<MW, GQ, false>(st, ch, p_s, lane, 32, p.c2);
+        else decode_chunk<MW, GQ, true>(st, ch, p_s, lane, t_end - c * 32, p.c2);
+        // every lane is done with this stage (the chunk ends with a warp barrier): refill it
+        if (lane == 0 && requested < c1) {
+            mbar_arrive_expect_tx(bar0 + 8 * stage, CB);
+            bulk_copy_g2s(ring_a + stage * CB, src, CB, bar0 + 8 * stage);
+            ++requested;
+            src += CB;
         }
-        if (any) {                                              // rescale the P.V accumulators too
-            float f0, f1;                                       // factors of this lane's columns 2jq, 2jq+1
-            if (GQ == 1) { f0 = scl[0]; f1 = scl[0]; }
-            else if (GQ == 2) { f0 = scl[0]; f1 = scl[GQ > 1 ? 1 : 0]; }
-            else { f0 = (jq & 1) ? scl[GQ > 2 ? 2 : 0] : scl[0]; f1 = (jq & 1) ? scl[GQ > 3 ? 3 : 0] : scl[GQ > 1 ? 1 : 0]; }
-#pragma unroll
-            for (int cb = 0; cb < 8; ++cb) {
-                acc[cb][0] *= f0; acc[cb][1] *= f1; acc[cb][2] *= f0; acc[cb][3] *= f1;
-            }
-        }
-        __syncwarp();
-
-        // ---------------- phase 2: P.V on tensor cores, two blocks of 16 tokens
-#pragma unroll
-        for (int vb = 0; vb < 2; ++vb) {
-            const float2 pa = *reinterpret_cast<const float2 *>(p_s + bhead * 32 + vb * 16 + 2 * jq);
-            const float2 pb = *reinterpret_cast<const float2 *>(p_s + bhead * 32 + vb * 16 + 2 * jq + 8);
-            uint32_t bf[NB][2];
-#pragma unroll
-            for (int bi = 0; bi < NB; ++bi) {
-                const int g = bi * NG + bgsel;
-                const unsigned char *sp = ch + SCALE + vb * 128 + g * 32 + jq * 4;
-                const float2 d01 = half2_bits_to_float2(*reinterpret_cast<const uint32_t *>(sp));
-                const float2 d89 = half2_bits_to_float2(*reinterpret_cast<const uint32_t *>(sp + 16));
-                const float x0 = pa.x * d01.x, x1 = pa.y * d01.y, x2 = pb.x * d89.x, x3 = pb.y * d89.y;
-                const uint32_t hi01 = pack_bf16x2(x0, x1), hi23 = pack_bf16x2(x2, x3);
-                const uint32_t lo01 = pack_bf16x2(x0 - __uint_as_float(hi01 << 16), x1 - __uint_as_float(hi01 & 0xffff0000u));
-                const uint32_t lo23 = pack_bf16x2(x2 - __uint_as_float(hi23 << 16), x3 - __uint_as_float(hi23 & 0xffff0000u));
-                bf[bi][0] = part ? lo01 : hi01;
-                bf[bi][1] = part ? lo23 : hi23;
-            }
-            const uint4 wa = *reinterpret_cast<const uint4 *>(ch + VAL + vb * 1024 + lane * 16);
-            const uint4 wb = *reinterpret_cast<const uint4 *>(ch + VAL + vb * 1024 + 512 + lane * 16);
-            const uint32_t wv[8] = {wa.x, wa.y, wa.z, wa.w, wb.x, wb.y, wb.z, wb.w};
-#pragma unroll
-            for (int cb = 0; cb < 8; ++cb) {
-                const uint32_t w = wv[cb];
-                const uint32_t a0 = nibbles_to_bf16x2(w), a1 = nibbles_to_bf16x2(w >> 4);
-                const uint32_t a2 = nibbles_to_bf16x2(w >> 8), a3 = nibbles_to_bf16x2(w >> 12);
-                const int bi = (cb >> 1) / NG;
-                mma_bf16_16816(acc[cb], a0, a1, a2, a3, bf[bi][0], bf[bi][1]);
-            }
-        }
-        __syncwarp();
-        if (lane == 0 && c + kStages < c1) {
-            mbar_arrive_expect_tx(bar0 + 8 * s, CB);
-            bulk_copy_g2s(ring_a + s * CB, slab + (size_t)(c + kStages) * CB, CB, bar0 + 8 * s);
-        }
+        if (++stage == kStages) { stage = 0; parity ^= 1; }
     }
 
     if (failed) {
         if (lane == 0) atomicExch(p.status, kStatusWaitTimeout);
-        // give copies that may still be in flight a bounded time to land
-        for (int k = 0; k < kStages && it + k < c1 - c0; ++k) {
-            const int s = (it + k) % kStages;
-            (void)mbar_wait_bounded(bar0 + 8 * s, ((it + k) / kStages) & 1, 100000000ull);
+        // give copies that may still be in flight a bounded time to land before leaving
+        for (int k = 0; k < kStages; ++k) {
+            (void)mbar_wait_bounded(bar0 + 8 * stage, parity, 100000000ull);
+            if (++stage == kStages) { stage = 0; parity ^= 1; }
         }
         return;
     }
@@ -326,30 +452,38 @@ __global__ void __launch_bounds__(kDecodeWarps * 32) decode_split_kernel(DecodeP
     for (int h = 0; h < GQ; ++h) {
 #pragma unroll
         for (int o = 16; o > 0; o >>= 1) {
-            ssum[h] += __shfl_xor_sync(0xffffffffu, ssum[h], o);
+            st.ssum[h] += __shfl_xor_sync(0xffffffffu, st.ssum[h], o);
 #pragma unroll
-            for (int g = 0; g < kGroups; ++g) accz[h][g] += __shfl_xor_sync(0xffffffffu, accz[h][g], o);
+            for (int g = 0; g < kGroups; ++g) st.accz[h][g] += __shfl_xor_sync(0xffffffffu, st.accz[h][g], o);
         }
     }
+    // Undo the scales: codes were fed as code / kCodeScaleLo (rows r) and code / kCodeScaleHi (rows r + 8), the
+    // weights carry a factor 2, and the low parts a further 2^11. Everything below is in units of 2p, like ssum and accz, so
+    // the common factor 2 cancels in the final division.
+    constexpr float kRowLo = kCodeScaleLo, kRowHi = kCodeScaleHi, kLoPart = 1.f / 2048.f;
     float *part_out = p.partial + (size_t)item * GQ * kPartStride;
-    const int r = lane >> 2;
+    const int r = lane >> 2, jq = lane & 3;
 #pragma unroll
     for (int cb = 0; cb < 8; ++cb) {
         float v[4];
 #pragma unroll
-        for (int i = 0; i < 4; ++i) v[i] = acc[cb][i] + __shfl_xor_sync(0xffffffffu, acc[cb][i], 2);  // high + low part
+        for (int i = 0; i < 4; ++i) {
+            const float other = __shfl_xor_sync(0xffffffffu, st.acc[cb][i], 2);   // lanes jq and jq^2: hi and lo columns
+            const float hi = (jq & 2) ? other : st.acc[cb][i], lo = (jq & 2) ? st.acc[cb][i] : other;
+            v[i] = fmaf(lo, kLoPart, hi) * (i < 2 ? kRowLo : kRowHi);
+        }
         const int g = cb >> 1;
         if (GQ == 1) {
             if (jq == (g >> 1)) {
-                part_out[cb * 16 + r] = v[g & 1] + accz[0][g];
-                part_out[cb * 16 + r + 8] = v[2 + (g & 1)] + accz[0][g];
+                part_out[cb * 16 + r] = v[g & 1] + st.accz[0][g];
+                part_out[cb * 16 + r + 8] = v[2 + (g & 1)] + st.accz[0][g];
             }
         } else if (GQ == 2) {
             if (jq == (g & 1)) {
 #pragma unroll
                 for (int h = 0; h < 2; ++h) {
-                    part_out[h * kPartStride + cb * 16 + r] = v[h] + accz[h < GQ ? h : 0][g];
-                    part_out[h * kPartStride + cb * 16 + r + 8] = v[2 + h] + accz[h < GQ ? h : 0][g];
+                    part_out[h * kPartStride + cb * 16 + r] = v[h] + st.accz[h < GQ ? h : 0][g];
+                    part_out[h * kPartStride + cb * 16 + r + 8] = v[2 + h] + st.accz[h < GQ ? h : 0][g];
                 }
             }
         } else {
@@ -357,7 +491,7 @@ __global__ void __launch_bounds__(kDecodeWarps * 32) decode_split_kernel(DecodeP
 #pragma unroll
                 for (int hh = 0; hh < 2; ++hh) {
                     // head = 2*jq + hh, a lane-dependent index: select without dynamic indexing
-                    const float z = (jq == 0) ? accz[hh < GQ ? hh : 0][g] : accz[(2 + hh) < GQ ? (2 + hh) : 0][g];
+                    const float z = (jq == 0) ? st.accz[hh < GQ ? hh : 0][g] : st.accz[(2 + hh) < GQ ? (2 + hh) : 0][g];
                     float *dst = part_out + (size_t)(2 * jq + hh) * kPartStride;
                     dst[cb * 16 + r] = v[hh] + z;
                     dst[cb * 16 + r + 8] = v[2 + hh] + z;
@@ -366,11 +500,11 @@ __global__ void __launch_bounds__(kDecodeWarps * 32) decode_split_kernel(DecodeP
         }
     }
     if (lane < GQ) {
-        int hm = hmin[0];
-        float sv = ssum[0];
+        int hm = st.hmin[0];
+        float sv = st.ssum[0];
 #pragma unroll
         for (int h = 1; h < GQ; ++h)
-            if (lane == h) { hm = hmin[h]; sv = ssum[h]; }
+            if (lane == h) { hm = st.hmin[h]; sv = st.ssum[h]; }
         part_out[lane * kPartStride + 128] = (float)hm;
         part_out[lane * kPartStride + 129] = sv;
     }
@@ -427,15 +561,12 @@ __global__ void debug_scores_kernel(const unsigned char *slab, const uint32_t *q
     }
 
 cudaError_t launch_append(const AppendParams &p, const NewCounts &nn, cudaStream_t st, int *launches) {
-    const long rows = (long)p.n_layers * p.B * p.Tn * p.Hkv;
-    if (rows > 0) {
-        const int wpb = 8;
-        const unsigned grid = (unsigned)((rows + wpb - 1) / wpb);
-        H1B_DISPATCH_MW(p.m_words, append_rows_kernel<MW><<<grid, wpb * 32, 0, st>>>(p, nn));
-        ++*launches;
-    }
-    const int n = p.n_layers * p.B;
-    bump_len_kernel<<<(n + 127) / 128, 128, 0, st>>>(p.len, p.layer_begin, p.n_layers, p.B, p.max_batch, nn);
+    const long rows_per_layer = (long)p.B * p.Tn * p.Hkv;
+    const long tiles = (rows_per_layer + kProjRows - 1) / kProjRows;
+    const long proj_blocks = (long)p.n_layers * tiles * p.m_words;
+    const long quant_blocks = ((long)p.n_layers * rows_per_layer + kProjThreads / 32 - 1) / (kProjThreads / 32);
+    if (proj_blocks + quant_blocks > 0x7fffffffL) return cudaErrorInvalidConfiguration;
+    append_kernel<<<(unsigned)(proj_blocks + quant_blocks), kProjThreads, 0, st>>>(p, nn);
     ++*launches;
     return cudaGetLastError();
 }
@@ -447,11 +578,10 @@ cudaError_t launch_set_len(int32_t *len, int n_layers, int max_batch, int seq, i
 }
 
 cudaError_t launch_sketch(const SketchParams &p, cudaStream_t st, int *launches) {
-    const long rows = (long)p.n_layers * p.B * p.Hq;
-    if (rows <= 0) return cudaSuccess;
-    const int wpb = 8;
-    const unsigned grid = (unsigned)((rows + wpb - 1) / wpb);
-    H1B_DISPATCH_MW(p.m_words, sketch_rows_kernel<MW><<<grid, wpb * 32, 0, st>>>(p));
+    const long rows_per_layer = (long)p.B * p.Hq;
+    if (rows_per_layer <= 0) return cudaSuccess;
+    const long tiles = (rows_per_layer + kProjRows - 1) / kProjRows;
+    sketch_kernel<<<(unsigned)((long)p.n_layers * tiles * p.m_words), kProjThreads, 0, st>>>(p);
     ++*launches;
     return cudaGetLastError();
 }

@@ -84,6 +84,7 @@ struct AppendParams {
     const float *Rt;            // [L][d][m]
     unsigned char *cache;       // slab 0
     int32_t *len;               // [L][max_batch]
+    int32_t *done;              // block counter of the append launch (zero between launches)
     size_t slab_bytes;
     int layer_begin, n_layers, B, Tn, Hkv, max_batch, m_words;
 };

@@ -1,9 +1,8 @@
 // Thin inline-PTX wrappers used by the H1B-KV kernels (sm_100a): mbarrier with
 // bounded waits, non-multicast bulk async copies into this CTA's shared memory,
-// warp-level bf16 tensor-core MMA, and a few scalar helpers.
+// warp-level fp16 tensor-core MMA, and a few scalar helpers.
 #pragma once
 #include <cstdint>
-#include <cuda_bf16.h>
 #include <cuda_fp16.h>
 
 namespace h1b {
@@ -65,29 +64,56 @@ __device__ __forceinline__ float ex2_approx(float x) {
     return y;
 }
 
-// Two floats -> packed bf16x2, round to nearest even; `lo` lands in bits 0-15.
-__device__ __forceinline__ uint32_t pack_bf16x2(float lo, float hi) {
+// Two floats -> packed f16x2, round to nearest even; `lo` lands in bits 0-15.
+__device__ __forceinline__ uint32_t pack_f16x2(float lo, float hi) {
     uint32_t r;
-    asm("cvt.rn.bf16x2.f32 %0, %1, %2;" : "=r"(r) : "f"(hi), "f"(lo));
+    asm("cvt.rn.f16x2.f32 %0, %1, %2;" : "=r"(r) : "f"(hi), "f"(lo));
     return r;
 }
 
-// (w & 0x000F000F) | 0x43004300 is the bf16 pair (128 + code_lo, 128 + code_hi);
-// subtracting 128 (exact) leaves the two integer codes as bf16.
-__device__ __forceinline__ uint32_t nibbles_to_bf16x2(uint32_t w) {
-    uint32_t x = (w & 0x000F000Fu) | 0x43004300u;
-    uint32_t r;
-    asm("sub.rn.bf16x2 %0, %1, %2;" : "=r"(r) : "r"(x), "r"(0x43004300u));
-    return r;
-}
-
-// D(16x8, f32) += A(16x16, bf16, row) * B(16x8, bf16, col)
-__device__ __forceinline__ void mma_bf16_16816(float (&c)[4], uint32_t a0, uint32_t a1, uint32_t a2, uint32_t a3,
-                                               uint32_t b0, uint32_t b1) {
+// D(16x8, f32) += A(16x16, f16, row) * B(16x8, f16, col). Subnormal f16 inputs keep their value, but
+// lose alignment precision when summed with larger terms (see decode_chunk).
+__device__ __forceinline__ void mma_f16_16816(float (&c)[4], uint32_t a0, uint32_t a1, uint32_t a2, uint32_t a3,
+                                              uint32_t b0, uint32_t b1) {
     asm volatile(
-        "mma.sync.aligned.m16n8k16.row.col.f32.bf16.bf16.f32 {%0,%1,%2,%3}, {%4,%5,%6,%7}, {%8,%9}, {%0,%1,%2,%3};"
+        "mma.sync.aligned.m16n8k16.row.col.f32.f16.f16.f32 {%0,%1,%2,%3}, {%4,%5,%6,%7}, {%8,%9}, {%0,%1,%2,%3};"
         : "+f"(c[0]), "+f"(c[1]), "+f"(c[2]), "+f"(c[3])
         : "r"(a0), "r"(a1), "r"(a2), "r"(a3), "r"(b0), "r"(b1));
+}
+
+// Eight 4-bit codes of one packed word -> the four f16x2 registers of an MMA A fragment, as fp16
+// SUBNORMALS taken in place: a code c at bits 4-7 of a half, everything else masked off, is the
+// subnormal 16 * c * 2^-24 = c * 2^-20. The word holds codes at bits 0, 4, 8 and 12 of each half, so
+// three of the four registers need a shift first. Bits 4-7 are used for all of them (and not bits
+// 0-3, which would save two shifts) because the tensor core aligns the 16 products of one MMA by
+// their exponent FIELDS: a subnormal with six leading zero bits loses about ten bits whenever
+// weights of different magnitude meet in one block of tokens; with two leading zeros the loss is
+// about 1e-6 relative, measured.
+//   H1B_DEQUANT_TWO_SHIFTS (build option): codes at bits 2-5 and 6-9 instead, one shift fewer,
+//   about 4e-6 relative.
+#ifdef H1B_DEQUANT_TWO_SHIFTS
+constexpr float kCodeScaleLo = 4194304.f;     // rows r:     code * 2^-22
+constexpr float kCodeScaleHi = 262144.f;      // rows r + 8: code * 2^-18
+__device__ __forceinline__ void codes_to_f16x2(uint32_t w, uint32_t (&a)[4]) {
+    const uint32_t u = w << 2, t = w >> 6;
+    a[0] = u & 0x003C003Cu; a[1] = u & 0x03C003C0u; a[2] = t & 0x003C003Cu; a[3] = t & 0x03C003C0u;
+}
+#else
+constexpr float kCodeScaleLo = 1048576.f;     // every row: code * 2^-20
+constexpr float kCodeScaleHi = 1048576.f;
+__device__ __forceinline__ void codes_to_f16x2(uint32_t w, uint32_t (&a)[4]) {
+    a[0] = (w << 4) & 0x00F000F0u; a[1] = w & 0x00F000F0u;
+    a[2] = (w >> 4) & 0x00F000F0u; a[3] = (w >> 8) & 0x00F000F0u;
+}
+#endif
+
+// D = A * B (accumulator starts at zero).
+__device__ __forceinline__ void mma_f16_16816_zero(float (&d)[4], uint32_t a0, uint32_t a1, uint32_t a2, uint32_t a3,
+                                                   uint32_t b0, uint32_t b1) {
+    asm volatile(
+        "mma.sync.aligned.m16n8k16.row.col.f32.f16.f16.f32 {%0,%1,%2,%3}, {%4,%5,%6,%7}, {%8,%9}, {%10,%10,%10,%10};"
+        : "=f"(d[0]), "=f"(d[1]), "=f"(d[2]), "=f"(d[3])
+        : "r"(a0), "r"(a1), "r"(a2), "r"(a3), "r"(b0), "r"(b1), "f"(0.f));
 }
 
 __device__ __forceinline__ float2 half2_bits_to_float2(uint32_t h2) {
