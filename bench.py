@@ -155,9 +155,8 @@ def run_ours(args):
     out = torch.empty((w.n_layers, w.batch, w.n_q_heads, w.head_dim), dtype=torch.float32, device=dev)
     stream = torch.cuda.current_stream()
 
-    def step(i):
-        cache.h1b_append_kv(kn[i % pool], vn[i % pool])
-        cache.h1b_decode_attention(qn[i % pool], INV_TAU, out=out)
+    def step(i):                                      # append the new token to all layers + decode: two launches
+        cache.h1b_decode_step(kn[i % pool], vn[i % pool], qn[i % pool], INV_TAU, out=out)
 
     def barrier():
         if dist is not None:

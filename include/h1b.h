@@ -112,6 +112,15 @@ int h1b_append_kv(h1b_ctx *ctx, int layer_begin, int n_layers, const void *k, co
 int h1b_decode_attention(h1b_ctx *ctx, int layer_begin, int n_layers, const void *q,
                          float inv_tau, void *out, int B, void *stream);
 
+/* One whole decode step on device tensors, all L layers: append one new token per
+ * sequence (Eq. 2, Eq. 4) and run decode attention over the grown cache (Eq. 3,
+ * Eq. 5). Same result as h1b_append_kv(Tn = 1) followed by h1b_decode_attention(),
+ * in two kernel launches instead of three.
+ *   k, v  DEVICE: fp16 [L][B][1][Hkv][d]      q  DEVICE: fp16 [L][B][Hq][d]
+ *   out   DEVICE: float32 [L][B][Hq][d] */
+int h1b_decode_step(h1b_ctx *ctx, const void *k, const void *v, const void *q, float inv_tau,
+                    void *out, int B, void *stream);
+
 /* h1b_decode_attention() for callers that must not allocate and cannot spare
  * scratch of their own. (No counterpart in the paper: this is a deployment
  * convenience, not a step of the method.)
@@ -131,7 +140,7 @@ int h1b_decode_attention(h1b_ctx *ctx, int layer_begin, int n_layers, const void
  * Same arguments, same result and same errors as h1b_decode_attention(), plus:
  *   - H1B_ERR_CAPACITY, with the needed and the available byte counts in
  *     h1b_last_error(), when even one split per sequence does not fit:
- *     n_layers * B * Hkv * (Hq/Hkv) * 528 bytes of partials plus
+ *     n_layers * B * Hkv * ((Hq/Hkv) * 528 + 4) bytes of partials and counters plus
  *     L * max_batch * Hq * m/8 bytes of sketches must be <= 8 MiB. When more
  *     splits would fit the automatic choice, fewer are used (slower, same result
  *     up to summation order).
@@ -140,8 +149,9 @@ int h1b_decode_attention(h1b_ctx *ctx, int layer_begin, int n_layers, const void
  *     (cudaGetSymbolAddress) and keeps it; make that first call outside any
  *     stream capture.
  * All contexts and all calls in the process share the one array per device, and
- * it keeps whatever the last call left in it. Nothing in it has to start at
- * zero: every element a call reads was written earlier by the same call. Two
+ * it keeps whatever the last call left in it. The only part that has to start
+ * at zero, the per-sequence arrival counters, is cleared by each call (a
+ * stream-ordered memset); everything else a call reads it has written itself. Two
  * calls whose kernels overlap on the GPU (different streams, different
  * contexts) race on it: order them on one stream or with events. */
 int h1b_decode_attention_static(h1b_ctx *ctx, int layer_begin, int n_layers, const void *q,

@@ -63,6 +63,7 @@ def load_library(rebuild: bool = True) -> ctypes.CDLL:
                                                 ctypes.c_int, vp]),
         "h1b_decode_attention_static": (ctypes.c_int, [vp, ctypes.c_int, ctypes.c_int, vp, ctypes.c_float, vp,
                                                        ctypes.c_int, vp]),
+        "h1b_decode_step": (ctypes.c_int, [vp, vp, vp, vp, ctypes.c_float, vp, ctypes.c_int, vp]),
         "h1b_decode_step_host": (ctypes.c_int, [vp, vp, vp, vp, ctypes.c_float, vp, ctypes.c_int, vp]),
         "h1b_free": (ctypes.c_int, [vp]),
         "h1b_get_projection": (ctypes.c_int, [vp, ctypes.c_int, vp]),
@@ -186,6 +187,21 @@ class H1BCache:
             raise ValueError("out must have q's shape")
         self._check(self.lib.h1b_decode_attention(self._h, layer_begin, int(q.shape[0]), qp, float(inv_tau), op,
                                                   int(q.shape[1]), _stream_ptr(stream)))
+        return out
+
+    def h1b_decode_step(self, k: torch.Tensor, v: torch.Tensor, q: torch.Tensor, inv_tau: float,
+                        out: torch.Tensor | None = None, stream=None) -> torch.Tensor:
+        """Append one token per sequence to every layer and decode: k, v fp16 CUDA [L, B, 1, Hkv, d],
+        q fp16 CUDA [L, B, Hq, d] -> out fp32 [L, B, Hq, d]."""
+        kp, vp, qp = _dev_ptr(k, torch.float16, "k"), _dev_ptr(v, torch.float16, "v"), _dev_ptr(q, torch.float16, "q")
+        L, B = self.cfg.n_layers, int(q.shape[1])
+        if tuple(k.shape) != (L, B, 1, self.cfg.n_kv_heads, self.cfg.head_dim) or k.shape != v.shape or \
+                tuple(q.shape) != (L, B, self.cfg.n_q_heads, self.cfg.head_dim):
+            raise ValueError("step shapes: k, v [L, B, 1, Hkv, d]; q [L, B, Hq, d]")
+        if out is None:
+            out = torch.empty(q.shape, dtype=torch.float32, device=q.device)
+        op = _dev_ptr(out, torch.float32, "out")
+        self._check(self.lib.h1b_decode_step(self._h, kp, vp, qp, float(inv_tau), op, B, _stream_ptr(stream)))
         return out
 
     def h1b_decode_attention_static(self, q: torch.Tensor, inv_tau: float, out: torch.Tensor,

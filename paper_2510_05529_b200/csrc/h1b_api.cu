@@ -23,7 +23,7 @@ constexpr long kTargetItems = 8192;   // decode work items aimed for (one warp e
 constexpr int kMinSplitTokens = 256;
 
 struct Plan {
-    size_t rt, len, status, qwords, partial, stage_k, stage_v, stage_q, stage_out, dbg_q, dbg_s, cache, total;
+    size_t rt, len, status, arrive, qwords, partial, stage_k, stage_v, stage_q, stage_out, dbg_q, dbg_s, cache, total;
     size_t partial_items, slab_bytes;
     int cap_tokens, m_words, gq;
 };
@@ -63,6 +63,7 @@ int make_plan(const h1b_config *c, Plan *p) {
     p->rt = take(L * d * c->sketch_bits * sizeof(float));
     p->len = take(L * B * sizeof(int32_t));
     p->status = take(64);
+    p->arrive = take(slabs * sizeof(int32_t));
     p->qwords = take(L * B * Hq * p->m_words * sizeof(uint32_t));
     p->partial = take(p->partial_items * p->gq * kPartStride * sizeof(float));
     p->stage_k = take(L * B * Hkv * d * 2);
@@ -214,24 +215,27 @@ int h1b_init_projection(const h1b_config *cfg, uint64_t seed, const float *Rt_ho
     return H1B_OK;
 }
 
-int h1b_append_kv(h1b_ctx *ctx, int layer_begin, int n_layers, const void *k, const void *v,
-                  const int32_t *n_new_host, int B, int Tn, void *stream) {
-    int rc = check_layers(ctx, layer_begin, n_layers, B);
-    if (rc != H1B_OK) return rc;
-    if (!k || !v) return fail(ctx, H1B_ERR_NULL, "k or v is NULL");
-    if (Tn < 1) return fail(ctx, H1B_ERR_INVALID_ARG, "Tn = %d < 1", Tn);
-    NewCounts nn;
-    std::memset(&nn, 0, sizeof nn);
+// ---------------------------------------------------------------------------
+// Shared pieces of append, decode and step (static: not part of the ABI).
+// ---------------------------------------------------------------------------
+static int make_new_counts(h1b_ctx *ctx, int layer_begin, int n_layers, const int32_t *n_new_host, int B, int Tn,
+                           NewCounts *nn) {
+    std::memset(nn, 0, sizeof *nn);
     for (int b = 0; b < B; ++b) {
         const int n = n_new_host ? n_new_host[b] : Tn;
         if (n < 0 || n > Tn) return fail(ctx, H1B_ERR_INVALID_ARG, "n_new[%d] = %d outside [0, %d]", b, n, Tn);
-        nn.v[b] = n;
+        nn->v[b] = n;
     }
     for (int l = layer_begin; l < layer_begin + n_layers; ++l)
         for (int b = 0; b < B; ++b)
-            if ((long)ctx->len_host[(size_t)l * ctx->cfg.max_batch + b] + nn.v[b] > ctx->cfg.max_seq)
+            if ((long)ctx->len_host[(size_t)l * ctx->cfg.max_batch + b] + nn->v[b] > ctx->cfg.max_seq)
                 return fail(ctx, H1B_ERR_CAPACITY, "layer %d sequence %d: %d + %d tokens exceed max_seq %d", l, b,
-                            ctx->len_host[(size_t)l * ctx->cfg.max_batch + b], nn.v[b], ctx->cfg.max_seq);
+                            ctx->len_host[(size_t)l * ctx->cfg.max_batch + b], nn->v[b], ctx->cfg.max_seq);
+    return H1B_OK;
+}
+
+static AppendParams append_params(h1b_ctx *ctx, int layer_begin, int n_layers, const void *k, const void *v, int B,
+                                  int Tn) {
     AppendParams p;
     p.k = static_cast<const uint16_t *>(k);
     p.v = static_cast<const uint16_t *>(v);
@@ -242,34 +246,31 @@ int h1b_append_kv(h1b_ctx *ctx, int layer_begin, int n_layers, const void *k, co
     p.slab_bytes = ctx->plan.slab_bytes;
     p.layer_begin = layer_begin; p.n_layers = n_layers; p.B = B; p.Tn = Tn;
     p.Hkv = ctx->cfg.n_kv_heads; p.max_batch = ctx->cfg.max_batch; p.m_words = ctx->plan.m_words;
-    int launches = 0;
-    H1B_CUDA(ctx, launch_append(p, nn, static_cast<cudaStream_t>(stream), &launches));
-    ctx->launches += launches;
-    for (int l = layer_begin; l < layer_begin + n_layers; ++l)
-        for (int b = 0; b < B; ++b) ctx->len_host[(size_t)l * ctx->cfg.max_batch + b] += nn.v[b];
-    return H1B_OK;
+    return p;
 }
 
-int h1b_decode_attention(h1b_ctx *ctx, int layer_begin, int n_layers, const void *q, float inv_tau, void *out,
-                         int B, void *stream) {
-    int rc = check_layers(ctx, layer_begin, n_layers, B);
-    if (rc != H1B_OK) return rc;
-    if (!q || !out) return fail(ctx, H1B_ERR_NULL, "q or out is NULL");
-    if (!(inv_tau > 0.f) || !std::isfinite(inv_tau))
-        return fail(ctx, H1B_ERR_INVALID_ARG, "inv_tau must be finite and > 0");
-    cudaStream_t st = static_cast<cudaStream_t>(stream);
-    int launches = 0;
+static SketchParams sketch_params(h1b_ctx *ctx, int layer_begin, int n_layers, const void *q, int B,
+                                  uint32_t *qwords) {
     SketchParams sp;
     sp.q = static_cast<const uint16_t *>(q);
     sp.Rt = at<float>(ctx, ctx->plan.rt);
-    sp.qwords = at<uint32_t>(ctx, ctx->plan.qwords);
+    sp.qwords = qwords;
     sp.layer_begin = layer_begin; sp.n_layers = n_layers; sp.B = B; sp.Hq = ctx->cfg.n_q_heads;
     sp.max_batch = ctx->cfg.max_batch; sp.m_words = ctx->plan.m_words;
-    H1B_CUDA(ctx, launch_sketch(sp, st, &launches));
+    return sp;
+}
 
-    // Split the sequence so that there are about kTargetItems work items; the
-    // last split of a sequence is open-ended, so the result does not depend on
-    // how well the host's view of the lengths matches the device's.
+static void commit_lengths(h1b_ctx *ctx, int layer_begin, int n_layers, int B, const NewCounts &nn) {
+    for (int l = layer_begin; l < layer_begin + n_layers; ++l)
+        for (int b = 0; b < B; ++b) ctx->len_host[(size_t)l * ctx->cfg.max_batch + b] += nn.v[b];
+}
+
+// Enqueue the split-K attention kernel over scratch (qwords, partial, arrive). The sequence is split so that
+// there are about kTargetItems work items, capped by `max_items`; the last split of a sequence is open-ended,
+// so the result does not depend on how well the host's view of the lengths matches the device's.
+static int enqueue_decode(h1b_ctx *ctx, int layer_begin, int n_layers, float inv_tau, void *out, int B,
+                          cudaStream_t st, uint32_t *qwords, float *partial, int32_t *arrive, size_t max_items,
+                          bool may_profile, int *launches) {
     const long slabs = (long)n_layers * B * ctx->cfg.n_kv_heads;
     int maxlen = 1;
     for (int l = layer_begin; l < layer_begin + n_layers; ++l)
@@ -278,8 +279,12 @@ int h1b_decode_attention(h1b_ctx *ctx, int layer_begin, int n_layers, const void
     const long max_splits = std::max(1, maxlen / kMinSplitTokens);
     if (ctx->forced_splits <= 0 && splits > max_splits) splits = max_splits;
     if (splits < 1) splits = 1;
-    if ((size_t)(slabs * splits) > ctx->plan.partial_items)
-        return fail(ctx, H1B_ERR_INVALID_ARG, "%ld splits of %ld slabs exceed the split-K scratch", splits, slabs);
+    if ((size_t)(slabs * splits) > max_items) {
+        if (ctx->forced_splits > 0 || (size_t)slabs > max_items)
+            return fail(ctx, H1B_ERR_CAPACITY, "%ld splits of %ld slabs exceed the split-K scratch (%zu items)",
+                        splits, slabs, max_items);
+        splits = (long)(max_items / (size_t)slabs);
+    }
     const int span = (maxlen + 255) / 256 * 256;
     int split_tokens = (int)((span + splits - 1) / splits);
     split_tokens = (split_tokens + kChunkTokens - 1) / kChunkTokens * kChunkTokens;
@@ -287,31 +292,96 @@ int h1b_decode_attention(h1b_ctx *ctx, int layer_begin, int n_layers, const void
     DecodeParams dp;
     dp.cache = ctx->ws + ctx->plan.cache;
     dp.len = at<int32_t>(ctx, ctx->plan.len);
-    dp.qwords = sp.qwords;
-    dp.partial = at<float>(ctx, ctx->plan.partial);
+    dp.qwords = qwords;
+    dp.partial = partial;
     dp.out = static_cast<float *>(out);
     dp.status = at<int32_t>(ctx, ctx->plan.status);
+    dp.arrive = arrive;
     dp.slab_bytes = ctx->plan.slab_bytes;
     dp.layer_begin = layer_begin; dp.n_layers = n_layers; dp.B = B; dp.Hkv = ctx->cfg.n_kv_heads;
     dp.Hq = ctx->cfg.n_q_heads; dp.max_batch = ctx->cfg.max_batch; dp.m_words = ctx->plan.m_words;
     dp.splits = (int)splits; dp.split_tokens = split_tokens;
     dp.c2 = (float)(2.0 * (double)inv_tau * 1.4426950408889634 / (double)ctx->cfg.sketch_bits);
     cudaEvent_t ev0 = nullptr, ev1 = nullptr;
-    if (ctx->profiling && ctx->events_used + 2 <= ctx->events.size()) {
+    if (may_profile && ctx->profiling && ctx->events_used + 2 <= ctx->events.size()) {
         ev0 = ctx->events[ctx->events_used];
         ev1 = ctx->events[ctx->events_used + 1];
         ctx->events_used += 2;
     }
-    H1B_CUDA(ctx, launch_decode(dp, st, &launches, ev0, ev1));
-    ctx->launches += launches;
+    H1B_CUDA(ctx, launch_decode(dp, st, launches, ev0, ev1));
     return H1B_OK;
+}
+
+static int check_decode_args(h1b_ctx *ctx, int layer_begin, int n_layers, const void *q, float inv_tau,
+                             const void *out, int B) {
+    int rc = check_layers(ctx, layer_begin, n_layers, B);
+    if (rc != H1B_OK) return rc;
+    if (!q || !out) return fail(ctx, H1B_ERR_NULL, "q or out is NULL");
+    if (!(inv_tau > 0.f) || !std::isfinite(inv_tau))
+        return fail(ctx, H1B_ERR_INVALID_ARG, "inv_tau must be finite and > 0");
+    return H1B_OK;
+}
+
+int h1b_append_kv(h1b_ctx *ctx, int layer_begin, int n_layers, const void *k, const void *v,
+                  const int32_t *n_new_host, int B, int Tn, void *stream) {
+    int rc = check_layers(ctx, layer_begin, n_layers, B);
+    if (rc != H1B_OK) return rc;
+    if (!k || !v) return fail(ctx, H1B_ERR_NULL, "k or v is NULL");
+    if (Tn < 1) return fail(ctx, H1B_ERR_INVALID_ARG, "Tn = %d < 1", Tn);
+    NewCounts nn;
+    rc = make_new_counts(ctx, layer_begin, n_layers, n_new_host, B, Tn, &nn);
+    if (rc != H1B_OK) return rc;
+    const AppendParams ap = append_params(ctx, layer_begin, n_layers, k, v, B, Tn);
+    int launches = 0;
+    H1B_CUDA(ctx, launch_prepare(&ap, nullptr, nn, static_cast<cudaStream_t>(stream), &launches));
+    ctx->launches += launches;
+    commit_lengths(ctx, layer_begin, n_layers, B, nn);
+    return H1B_OK;
+}
+
+int h1b_decode_attention(h1b_ctx *ctx, int layer_begin, int n_layers, const void *q, float inv_tau, void *out,
+                         int B, void *stream) {
+    int rc = check_decode_args(ctx, layer_begin, n_layers, q, inv_tau, out, B);
+    if (rc != H1B_OK) return rc;
+    cudaStream_t st = static_cast<cudaStream_t>(stream);
+    int launches = 0;
+    const SketchParams sp = sketch_params(ctx, layer_begin, n_layers, q, B, at<uint32_t>(ctx, ctx->plan.qwords));
+    NewCounts none;
+    std::memset(&none, 0, sizeof none);
+    H1B_CUDA(ctx, launch_prepare(nullptr, &sp, none, st, &launches));
+    rc = enqueue_decode(ctx, layer_begin, n_layers, inv_tau, out, B, st, sp.qwords, at<float>(ctx, ctx->plan.partial),
+                        at<int32_t>(ctx, ctx->plan.arrive), ctx->plan.partial_items, true, &launches);
+    ctx->launches += launches;
+    return rc;
+}
+
+int h1b_decode_step(h1b_ctx *ctx, const void *k, const void *v, const void *q, float inv_tau, void *out, int B,
+                    void *stream) {
+    if (!ctx) return H1B_ERR_NULL;
+    const int L = ctx->cfg.n_layers;
+    int rc = check_decode_args(ctx, 0, L, q, inv_tau, out, B);
+    if (rc != H1B_OK) return rc;
+    if (!k || !v) return fail(ctx, H1B_ERR_NULL, "k or v is NULL");
+    NewCounts nn;
+    rc = make_new_counts(ctx, 0, L, nullptr, B, 1, &nn);
+    if (rc != H1B_OK) return rc;
+    cudaStream_t st = static_cast<cudaStream_t>(stream);
+    int launches = 0;
+    const AppendParams ap = append_params(ctx, 0, L, k, v, B, 1);
+    const SketchParams sp = sketch_params(ctx, 0, L, q, B, at<uint32_t>(ctx, ctx->plan.qwords));
+    H1B_CUDA(ctx, launch_prepare(&ap, &sp, nn, st, &launches));
+    commit_lengths(ctx, 0, L, B, nn);
+    rc = enqueue_decode(ctx, 0, L, inv_tau, out, B, st, sp.qwords, at<float>(ctx, ctx->plan.partial),
+                        at<int32_t>(ctx, ctx->plan.arrive), ctx->plan.partial_items, true, &launches);
+    ctx->launches += launches;
+    return rc;
 }
 
 // ---------------------------------------------------------------------------
 // Decode attention without touching the workspace's scratch region and without
-// allocating anything: the query sketches and the split-K partials live in a
-// fixed array that is part of the library image. Every device that loads the
-// library carries these bytes until the process exits.
+// allocating anything: the query sketches, the split-K partials and the arrival
+// counters live in a fixed array that is part of the library image. Every device
+// that loads the library carries these bytes until the process exits.
 // ---------------------------------------------------------------------------
 #define H1B_STATIC_SCRATCH_BYTES (8u << 20)
 static __device__ __align__(256) unsigned char h1b_static_scratch[H1B_STATIC_SCRATCH_BYTES];
@@ -327,11 +397,8 @@ __global__ void h1b_static_scratch_anchor(unsigned char *dst) {
 
 int h1b_decode_attention_static(h1b_ctx *ctx, int layer_begin, int n_layers, const void *q, float inv_tau,
                                 void *out, int B, void *stream) {
-    int rc = check_layers(ctx, layer_begin, n_layers, B);
+    int rc = check_decode_args(ctx, layer_begin, n_layers, q, inv_tau, out, B);
     if (rc != H1B_OK) return rc;
-    if (!q || !out) return fail(ctx, H1B_ERR_NULL, "q or out is NULL");
-    if (!(inv_tau > 0.f) || !std::isfinite(inv_tau))
-        return fail(ctx, H1B_ERR_INVALID_ARG, "inv_tau must be finite and > 0");
     const int dev = ctx->cfg.device;
     if (dev < 0 || dev >= 64) return fail(ctx, H1B_ERR_UNSUPPORTED, "device ordinal %d outside [0, 64)", dev);
     int cur = -1;
@@ -346,52 +413,33 @@ int h1b_decode_attention_static(h1b_ctx *ctx, int layer_begin, int n_layers, con
     }
     unsigned char *scratch = static_cast<unsigned char *>(g_static_scratch_addr[dev]);
 
-    // carve: query sketches for every (layer, sequence, head) slot the kernels index, then the partials
+    // carve: arrival counters (one per slab of the call), query sketches for every (layer, sequence, head)
+    // slot the kernels index, then the partials
+    const long slabs = (long)n_layers * B * ctx->cfg.n_kv_heads;
+    const size_t arrive_bytes = align_up((size_t)slabs * sizeof(int32_t), 256);
     const size_t qw_bytes = align_up((size_t)ctx->cfg.n_layers * ctx->cfg.max_batch * ctx->cfg.n_q_heads *
                                          ctx->plan.m_words * sizeof(uint32_t), 256);
-    const long slabs = (long)n_layers * B * ctx->cfg.n_kv_heads;
     const size_t item_bytes = (size_t)ctx->plan.gq * kPartStride * sizeof(float);
-    if (qw_bytes + (size_t)slabs * item_bytes > H1B_STATIC_SCRATCH_BYTES)
+    const size_t need = arrive_bytes + qw_bytes + (size_t)slabs * item_bytes;
+    if (need > H1B_STATIC_SCRATCH_BYTES)
         return fail(ctx, H1B_ERR_CAPACITY,
                     "static scratch too small: this call needs at least %zu bytes, the built-in array holds %u",
-                    qw_bytes + (size_t)slabs * item_bytes, (unsigned)H1B_STATIC_SCRATCH_BYTES);
-    const long fit_splits = (long)((H1B_STATIC_SCRATCH_BYTES - qw_bytes) / item_bytes / (size_t)slabs);
-    int maxlen = 1;
-    for (int l = layer_begin; l < layer_begin + n_layers; ++l)
-        for (int b = 0; b < B; ++b) maxlen = std::max(maxlen, ctx->len_host[(size_t)l * ctx->cfg.max_batch + b]);
-    long splits = ctx->forced_splits > 0 ? ctx->forced_splits : kTargetItems / slabs;
-    const long max_splits = std::max(1, maxlen / kMinSplitTokens);
-    if (ctx->forced_splits <= 0 && splits > max_splits) splits = max_splits;
-    if (splits > fit_splits) splits = fit_splits;
-    if (splits < 1) splits = 1;
-    const int span = (maxlen + 255) / 256 * 256;
-    int split_tokens = (int)((span + splits - 1) / splits);
-    split_tokens = (split_tokens + kChunkTokens - 1) / kChunkTokens * kChunkTokens;
-
+                    need, (unsigned)H1B_STATIC_SCRATCH_BYTES);
+    const size_t fit_items = (H1B_STATIC_SCRATCH_BYTES - arrive_bytes - qw_bytes) / item_bytes;
     cudaStream_t st = static_cast<cudaStream_t>(stream);
+    // the counters must start at zero whatever an earlier call (or an aborted one) left behind
+    H1B_CUDA(ctx, cudaMemsetAsync(scratch, 0, arrive_bytes, st));
     int launches = 0;
-    SketchParams sp;
-    sp.q = static_cast<const uint16_t *>(q);
-    sp.Rt = at<float>(ctx, ctx->plan.rt);
-    sp.qwords = reinterpret_cast<uint32_t *>(scratch);
-    sp.layer_begin = layer_begin; sp.n_layers = n_layers; sp.B = B; sp.Hq = ctx->cfg.n_q_heads;
-    sp.max_batch = ctx->cfg.max_batch; sp.m_words = ctx->plan.m_words;
-    H1B_CUDA(ctx, launch_sketch(sp, st, &launches));
-    DecodeParams dp;
-    dp.cache = ctx->ws + ctx->plan.cache;
-    dp.len = at<int32_t>(ctx, ctx->plan.len);
-    dp.qwords = sp.qwords;
-    dp.partial = reinterpret_cast<float *>(scratch + qw_bytes);
-    dp.out = static_cast<float *>(out);
-    dp.status = at<int32_t>(ctx, ctx->plan.status);
-    dp.slab_bytes = ctx->plan.slab_bytes;
-    dp.layer_begin = layer_begin; dp.n_layers = n_layers; dp.B = B; dp.Hkv = ctx->cfg.n_kv_heads;
-    dp.Hq = ctx->cfg.n_q_heads; dp.max_batch = ctx->cfg.max_batch; dp.m_words = ctx->plan.m_words;
-    dp.splits = (int)splits; dp.split_tokens = split_tokens;
-    dp.c2 = (float)(2.0 * (double)inv_tau * 1.4426950408889634 / (double)ctx->cfg.sketch_bits);
-    H1B_CUDA(ctx, launch_decode(dp, st, &launches));
+    const SketchParams sp = sketch_params(ctx, layer_begin, n_layers, q, B,
+                                          reinterpret_cast<uint32_t *>(scratch + arrive_bytes));
+    NewCounts none;
+    std::memset(&none, 0, sizeof none);
+    H1B_CUDA(ctx, launch_prepare(nullptr, &sp, none, st, &launches));
+    rc = enqueue_decode(ctx, layer_begin, n_layers, inv_tau, out, B, st, sp.qwords,
+                        reinterpret_cast<float *>(scratch + arrive_bytes + qw_bytes),
+                        reinterpret_cast<int32_t *>(scratch), fit_items, false, &launches);
     ctx->launches += launches;
-    return H1B_OK;
+    return rc;
 }
 
 int h1b_decode_step_host(h1b_ctx *ctx, const void *k_host, const void *v_host, const void *q_host, float inv_tau,
@@ -406,11 +454,8 @@ int h1b_decode_step_host(h1b_ctx *ctx, const void *k_host, const void *v_host, c
     H1B_CUDA(ctx, cudaMemcpyAsync(ctx->ws + ctx->plan.stage_k, k_host, kv_bytes, cudaMemcpyHostToDevice, st));
     H1B_CUDA(ctx, cudaMemcpyAsync(ctx->ws + ctx->plan.stage_v, v_host, kv_bytes, cudaMemcpyHostToDevice, st));
     H1B_CUDA(ctx, cudaMemcpyAsync(ctx->ws + ctx->plan.stage_q, q_host, q_bytes, cudaMemcpyHostToDevice, st));
-    rc = h1b_append_kv(ctx, 0, ctx->cfg.n_layers, ctx->ws + ctx->plan.stage_k, ctx->ws + ctx->plan.stage_v, nullptr,
-                       B, 1, stream);
-    if (rc != H1B_OK) return rc;
-    rc = h1b_decode_attention(ctx, 0, ctx->cfg.n_layers, ctx->ws + ctx->plan.stage_q, inv_tau,
-                              ctx->ws + ctx->plan.stage_out, B, stream);
+    rc = h1b_decode_step(ctx, ctx->ws + ctx->plan.stage_k, ctx->ws + ctx->plan.stage_v, ctx->ws + ctx->plan.stage_q,
+                         inv_tau, ctx->ws + ctx->plan.stage_out, B, stream);
     if (rc != H1B_OK) return rc;
     H1B_CUDA(ctx, cudaMemcpyAsync(out_host, ctx->ws + ctx->plan.stage_out, q_bytes * 2, cudaMemcpyDeviceToHost, st));
     H1B_CUDA(ctx, cudaStreamSynchronize(st));
@@ -526,8 +571,10 @@ int h1b_debug_scores(h1b_ctx *ctx, int layer, int seq, int kv_head, const void *
     sp.qwords = at<uint32_t>(ctx, ctx->plan.dbg_q);
     sp.layer_begin = 0; sp.n_layers = 1; sp.B = 1; sp.Hq = 1; sp.max_batch = 1; sp.m_words = mw;
     int launches = 0;
+    NewCounts none;
+    std::memset(&none, 0, sizeof none);
     H1B_CUDA(ctx, cudaDeviceSynchronize());
-    H1B_CUDA(ctx, launch_sketch(sp, nullptr, &launches));
+    H1B_CUDA(ctx, launch_prepare(nullptr, &sp, none, nullptr, &launches));
     H1B_CUDA(ctx, launch_debug_scores(slab_ptr(ctx, layer, seq, kv_head), sp.qwords, mw, len,
                                       at<int32_t>(ctx, ctx->plan.dbg_s), nullptr));
     H1B_CUDA(ctx, cudaDeviceSynchronize());

@@ -1,10 +1,10 @@
 // CUDA kernels of the H1B-KV hot path (sm_100a).
 //
-//   append_kernel        Eq. 2 on new keys (tiled fp32 FMA projection in ascending
-//                        channel order, sign, pack) and Eq. 4 on new values (group
-//                        min/max, fp16 scale, round-half-even codes), written straight
-//                        into the packed cache; the last block bumps the lengths.
-//   sketch_kernel        Eq. 2 on the queries of a decode step.
+//   prepare_kernel       Eq. 2 on new keys and on the queries of a decode step (tiled fp32
+//                        FMA projection in ascending channel order, sign, pack) and Eq. 4
+//                        on new values (group min/max, fp16 scale, round-half-even codes),
+//                        written straight into the packed cache; the last block bumps the
+//                        lengths. One launch per append, per query sketch, or per step.
 //   decode_split_kernel  Eq. 3 + Eq. 5 over one split of one (layer, sequence,
 //                        KV head) slab per warp: bulk-async chunk ring in shared
 //                        memory, XOR/popcount scores, online softmax on integer
@@ -40,17 +40,32 @@ struct ProjSmem {
 __device__ __forceinline__ uint32_t project_tile(ProjSmem &sm, const uint16_t *__restrict__ x_rows, int n_rows,
                                                  const float *__restrict__ Rt_layer, int m, int word) {
     const int tid = threadIdx.x, lane = tid & 31, warp = tid >> 5;
-    // Rt tile: 128 x 32 floats, 128-byte rows
-    for (int e = tid; e < kHeadDim * 8; e += kProjThreads) {
-        const int i = e >> 3, c4 = e & 7;
-        const float4 v = __ldg(reinterpret_cast<const float4 *>(Rt_layer + (size_t)i * m + word * 32) + c4);
-        *reinterpret_cast<float4 *>(&sm.r[i][c4 * 4]) = v;
+    // All global loads of the tile are issued before the first shared-memory store, so that the block pays
+    // one memory round trip, not one per loop iteration.
+    // Rt tile: 128 x 32 floats, 128-byte rows, 8 float4 per thread
+    float4 rv[kHeadDim * 8 / kProjThreads];
+#pragma unroll
+    for (int k = 0; k < kHeadDim * 8 / kProjThreads; ++k) {
+        const int e = tid + k * kProjThreads, i = e >> 3, c4 = e & 7;
+        rv[k] = __ldg(reinterpret_cast<const float4 *>(Rt_layer + (size_t)i * m + word * 32) + c4);
     }
-    // rows: coalesced half2 reads, transposed padded writes (conflict-free both ways)
-    for (int e = tid; e < kProjRows * (kHeadDim / 2); e += kProjThreads) {
-        const int row = e >> 6, c2 = e & 63;
-        float2 v = make_float2(0.f, 0.f);
-        if (row < n_rows) v = __half22float2(reinterpret_cast<const __half2 *>(x_rows + (size_t)row * kHeadDim)[c2]);
+    // rows: coalesced half2 reads (16 per thread), transposed padded writes
+    __half2 xv[kProjRows * (kHeadDim / 2) / kProjThreads];
+#pragma unroll
+    for (int k = 0; k < kProjRows * (kHeadDim / 2) / kProjThreads; ++k) {
+        const int e = tid + k * kProjThreads, row = e >> 6, c2 = e & 63;
+        xv[k] = __float2half2_rn(0.f);
+        if (row < n_rows) xv[k] = __ldg(reinterpret_cast<const __half2 *>(x_rows + (size_t)row * kHeadDim) + c2);
+    }
+#pragma unroll
+    for (int k = 0; k < kHeadDim * 8 / kProjThreads; ++k) {
+        const int e = tid + k * kProjThreads, i = e >> 3, c4 = e & 7;
+        *reinterpret_cast<float4 *>(&sm.r[i][c4 * 4]) = rv[k];
+    }
+#pragma unroll
+    for (int k = 0; k < kProjRows * (kHeadDim / 2) / kProjThreads; ++k) {
+        const int e = tid + k * kProjThreads, row = e >> 6, c2 = e & 63;
+        const float2 v = __half22float2(xv[k]);
         sm.x[2 * c2][row] = v.x;
         sm.x[2 * c2 + 1][row] = v.y;
     }
@@ -58,7 +73,7 @@ __device__ __forceinline__ uint32_t project_tile(ProjSmem &sm, const uint16_t *_
     float acc[8];
 #pragma unroll
     for (int c = 0; c < 8; ++c) acc[c] = 0.f;
-#pragma unroll 4
+#pragma unroll 16
     for (int i = 0; i < kHeadDim; ++i) {
         const float xv = sm.x[i][lane];
         const float4 ra = *reinterpret_cast<const float4 *>(&sm.r[i][warp * 8]);
@@ -113,61 +128,84 @@ __device__ __forceinline__ void quantize_row(const uint16_t *__restrict__ v_row,
     }
 }
 
-// One launch appends: blocks [0, proj_blocks) sketch key tiles, the rest quantise value rows (one warp per
-// row); the block that finishes last adds n_new to the lengths (every block has read them by then).
-__global__ void __launch_bounds__(kProjThreads) append_kernel(AppendParams p, NewCounts nn) {
+// One launch prepares a decode step (or only appends, or only sketches queries). Block ranges:
+//   [0, k_blocks)              key tiles: Eq. 2 on new keys, written into the cache   (ap.k != null)
+//   [k_blocks, +q_blocks)      query tiles: Eq. 2 on the queries, written to qwords   (sp.q != null)
+//   the rest                   value rows: Eq. 4, one warp per row                    (ap.k != null)
+// When keys/values are appended, the block that finishes last adds n_new to the lengths (every block has
+// read them by then).
+__global__ void __launch_bounds__(kProjThreads) prepare_kernel(AppendParams ap, SketchParams sp, NewCounts nn) {
     __shared__ ProjSmem sm;
-    const int mw = p.m_words, m = mw * 32;
+    const bool appending = ap.k != nullptr;
+    const int mw = appending ? ap.m_words : sp.m_words, m = mw * 32;
     const ChunkLayout cl = chunk_layout(mw);
-    const int rows_per_layer = p.B * p.Tn * p.Hkv;
-    const int tiles_per_layer = (rows_per_layer + kProjRows - 1) / kProjRows;
-    const int proj_blocks = p.n_layers * tiles_per_layer * mw;
-    if ((int)blockIdx.x < proj_blocks) {
-        const int word = blockIdx.x % mw;
-        const int tile = (blockIdx.x / mw) % tiles_per_layer;
-        const int ll = blockIdx.x / (mw * tiles_per_layer);
-        const int layer = p.layer_begin + ll;
+    const int k_rows = appending ? ap.B * ap.Tn * ap.Hkv : 0;           // per layer
+    const int k_tiles = (k_rows + kProjRows - 1) / kProjRows;
+    const int k_blocks = appending ? ap.n_layers * k_tiles * mw : 0;
+    const int q_rows = sp.q ? sp.B * sp.Hq : 0;
+    const int q_tiles = (q_rows + kProjRows - 1) / kProjRows;
+    const int q_blocks = sp.q ? sp.n_layers * q_tiles * mw : 0;
+    const int blk = blockIdx.x;
+    if (blk < k_blocks) {
+        const int word = blk % mw, tile = (blk / mw) % k_tiles, ll = blk / (mw * k_tiles);
+        const int layer = ap.layer_begin + ll;
         const int row0 = tile * kProjRows;
-        const int n_rows = min(kProjRows, rows_per_layer - row0);
-        const uint32_t bits = project_tile(sm, p.k + ((size_t)ll * rows_per_layer + row0) * kHeadDim, n_rows,
-                                           p.Rt + (size_t)layer * kHeadDim * m, m, word);
+        const int n_rows = min(kProjRows, k_rows - row0);
+        // this thread's row and where it goes: the length is fetched before the projection, not after it
+        const int row = row0 + min((int)threadIdx.x, n_rows - 1);
+        const int kvh = row % ap.Hkv, tn = (row / ap.Hkv) % ap.Tn, b = row / (ap.Hkv * ap.Tn);
+        const int len0 = ap.len[layer * ap.max_batch + b];
+        const uint32_t bits = project_tile(sm, ap.k + ((size_t)ll * k_rows + row0) * kHeadDim, n_rows,
+                                           ap.Rt + (size_t)layer * kHeadDim * m, m, word);
         if ((int)threadIdx.x < n_rows) {
-            const int row = row0 + threadIdx.x;
-            const int kvh = row % p.Hkv, tn = (row / p.Hkv) % p.Tn, b = row / (p.Hkv * p.Tn);
             if (tn < nn.v[b]) {
-                const int t = p.len[layer * p.max_batch + b] + tn;
-                unsigned char *chunk = p.cache + ((size_t)(layer * p.max_batch + b) * p.Hkv + kvh) * p.slab_bytes +
+                const int t = len0 + tn;
+                unsigned char *chunk = ap.cache + ((size_t)(layer * ap.max_batch + b) * ap.Hkv + kvh) * ap.slab_bytes +
                                        (size_t)(t >> 5) * cl.bytes;
                 *reinterpret_cast<uint32_t *>(chunk + key_word_off(word, t & 31)) = bits;
             }
         }
+    } else if (blk < k_blocks + q_blocks) {
+        const int qb = blk - k_blocks;
+        const int word = qb % mw, tile = (qb / mw) % q_tiles, ll = qb / (mw * q_tiles);
+        const int layer = sp.layer_begin + ll;
+        const int row0 = tile * kProjRows;
+        const int n_rows = min(kProjRows, q_rows - row0);
+        const uint32_t bits = project_tile(sm, sp.q + ((size_t)ll * q_rows + row0) * kHeadDim, n_rows,
+                                           sp.Rt + (size_t)layer * kHeadDim * m, m, word);
+        if ((int)threadIdx.x < n_rows) {
+            const int row = row0 + threadIdx.x;
+            const int h = row % sp.Hq, b = row / sp.Hq;
+            sp.qwords[((size_t)(layer * sp.max_batch + b) * sp.Hq + h) * mw + word] = bits;
+        }
     } else {
-        const long row = (long)(blockIdx.x - proj_blocks) * (kProjThreads / 32) + (threadIdx.x >> 5);
-        const long rows = (long)p.n_layers * rows_per_layer;
+        const long row = (long)(blk - k_blocks - q_blocks) * (kProjThreads / 32) + (threadIdx.x >> 5);
+        const long rows = (long)ap.n_layers * k_rows;
         if (row < rows) {
-            const int kvh = (int)(row % p.Hkv), tn = (int)((row / p.Hkv) % p.Tn);
-            const int b = (int)((row / ((long)p.Hkv * p.Tn)) % p.B), ll = (int)(row / rows_per_layer);
+            const int kvh = (int)(row % ap.Hkv), tn = (int)((row / ap.Hkv) % ap.Tn);
+            const int b = (int)((row / ((long)ap.Hkv * ap.Tn)) % ap.B), ll = (int)(row / k_rows);
             if (tn < nn.v[b]) {
-                const int layer = p.layer_begin + ll;
-                const int t = p.len[layer * p.max_batch + b] + tn;
-                unsigned char *chunk = p.cache + ((size_t)(layer * p.max_batch + b) * p.Hkv + kvh) * p.slab_bytes +
+                const int layer = ap.layer_begin + ll;
+                const int t = ap.len[layer * ap.max_batch + b] + tn;
+                unsigned char *chunk = ap.cache + ((size_t)(layer * ap.max_batch + b) * ap.Hkv + kvh) * ap.slab_bytes +
                                        (size_t)(t >> 5) * cl.bytes;
-                quantize_row(p.v + row * kHeadDim, chunk, cl, t & 31, threadIdx.x & 31);
+                quantize_row(ap.v + row * kHeadDim, chunk, cl, t & 31, threadIdx.x & 31);
             }
         }
     }
+    if (!appending) return;
     // ---- the last block to finish publishes the new lengths
     __shared__ int is_last;
     __syncthreads();
     if (threadIdx.x == 0) {
         __threadfence();
-        is_last = (atomicAdd(p.done, 1) == (int)gridDim.x - 1);
+        is_last = (atomicAdd(ap.done, 1) == (int)gridDim.x - 1);
     }
     __syncthreads();
     if (is_last) {
-        for (int i = threadIdx.x; i < p.n_layers * p.B; i += blockDim.x)
-            p.len[(p.layer_begin + i / p.B) * p.max_batch + (i % p.B)] += nn.v[i % p.B];
-        if (threadIdx.x == 0) *p.done = 0;
+        for (int i = threadIdx.x; i < ap.n_layers * ap.B; i += blockDim.x)
+            ap.len[(ap.layer_begin + i / ap.B) * ap.max_batch + (i % ap.B)] += nn.v[i % ap.B];
+        if (threadIdx.x == 0) *ap.done = 0;
     }
 }
 
@@ -175,27 +213,6 @@ __global__ void set_len_kernel(int32_t *len, int n_layers, int max_batch, int se
     const int i = blockIdx.x * blockDim.x + threadIdx.x;
     if (i >= n_layers * max_batch) return;
     if (seq < 0 || (i % max_batch) == seq) len[i] = value;
-}
-
-// Eq. 2 on the queries of a decode step: one block per (layer, tile of 32 query rows, word).
-__global__ void __launch_bounds__(kProjThreads) sketch_kernel(SketchParams p) {
-    __shared__ ProjSmem sm;
-    const int mw = p.m_words, m = mw * 32;
-    const int rows_per_layer = p.B * p.Hq;
-    const int tiles_per_layer = (rows_per_layer + kProjRows - 1) / kProjRows;
-    const int word = blockIdx.x % mw;
-    const int tile = (blockIdx.x / mw) % tiles_per_layer;
-    const int ll = blockIdx.x / (mw * tiles_per_layer);
-    const int layer = p.layer_begin + ll;
-    const int row0 = tile * kProjRows;
-    const int n_rows = min(kProjRows, rows_per_layer - row0);
-    const uint32_t bits = project_tile(sm, p.q + ((size_t)ll * rows_per_layer + row0) * kHeadDim, n_rows,
-                                       p.Rt + (size_t)layer * kHeadDim * m, m, word);
-    if ((int)threadIdx.x < n_rows) {
-        const int row = row0 + threadIdx.x;
-        const int h = row % p.Hq, b = row / p.Hq;
-        p.qwords[((size_t)(layer * p.max_batch + b) * p.Hq + h) * mw + word] = bits;
-    }
 }
 
 // ===========================================================================
@@ -223,11 +240,10 @@ __global__ void __launch_bounds__(kProjThreads) sketch_kernel(SketchParams p) {
 #ifndef H1B_DECODE_STAGES
 #define H1B_DECODE_STAGES 3         // chunks in flight per warp
 #endif
-#ifndef H1B_DECODE_MIN_BLOCKS
-#define H1B_DECODE_MIN_BLOCKS 1     // resident blocks per SM the register allocation must allow
-#endif
 constexpr int kDecodeWarps = H1B_DECODE_WARPS;
 constexpr int kStages = H1B_DECODE_STAGES;
+// Resident blocks per SM that the register allocation must allow: the kernel hides latency with warps.
+constexpr int decode_min_blocks(int gq) { return gq == 1 ? 5 : (gq == 2 ? 4 : 3); }
 constexpr unsigned long long kWaitLimitNs = 2000000000ull;   // 2 s, then give up
 constexpr int kHamSentinel = 1 << 20;
 
@@ -355,7 +371,7 @@ __device__ __forceinline__ void decode_chunk(DecodeState<MW, GQ> &st, const unsi
 }
 
 template <int MW, int GQ>
-__global__ void __launch_bounds__(kDecodeWarps * 32, H1B_DECODE_MIN_BLOCKS) decode_split_kernel(DecodeParams p) {
+__global__ void __launch_bounds__(kDecodeWarps * 32, decode_min_blocks(GQ)) decode_split_kernel(DecodeParams p) {
     using SM = DecodeSmem<MW, GQ>;
     constexpr int CB = SM::kChunkBytes;
     extern __shared__ __align__(128) unsigned char smem_raw[];
@@ -372,7 +388,14 @@ __global__ void __launch_bounds__(kDecodeWarps * 32, H1B_DECODE_MIN_BLOCKS) deco
     const int layer = p.layer_begin + ll;
     const int len = p.len[layer * p.max_batch + b];
     const int t_begin = split * p.split_tokens;
-    if (t_begin >= len) return;                                 // empty item: combine skips it too
+    if (t_begin >= len) {                                       // empty item: it is not counted by the combine
+#ifdef H1B_FUSED_COMBINE
+        if (len == 0 && split == 0)                             // an empty sequence attends to nothing: zeros
+            for (int i = lane; i < GQ * kHeadDim; i += 32)
+                p.out[(((size_t)ll * p.B + b) * p.Hq + kvh * GQ) * kHeadDim + i] = 0.f;
+#endif
+        return;
+    }
     // the last split of a sequence is open-ended: it runs to the sequence's end
     const int t_end = (split == p.splits - 1) ? len : min(len, t_begin + p.split_tokens);
     const int c0 = t_begin >> 5, c_full = t_end >> 5, c1 = (t_end + 31) >> 5;
@@ -444,10 +467,11 @@ __global__ void __launch_bounds__(kDecodeWarps * 32, H1B_DECODE_MIN_BLOCKS) deco
             (void)mbar_wait_bounded(bar0 + 8 * stage, parity, 100000000ull);
             if (++stage == kStages) { stage = 0; parity ^= 1; }
         }
-        return;
     }
 
     // ---------------- reduce across lanes and write the partial
+    // (after a timed-out wait the partial is meaningless, but the item still reports in below, so that
+    // the arrival counters return to zero; the status word tells the host that the output is invalid)
 #pragma unroll
     for (int h = 0; h < GQ; ++h) {
 #pragma unroll
@@ -508,9 +532,45 @@ __global__ void __launch_bounds__(kDecodeWarps * 32, H1B_DECODE_MIN_BLOCKS) deco
         part_out[lane * kPartStride + 128] = (float)hm;
         part_out[lane * kPartStride + 129] = sv;
     }
+
+#ifdef H1B_FUSED_COMBINE
+    // ---------------- the split that reports in last merges the slab's partials (flash-decoding combine)
+    // Build option: saves the combine launch, but the fences and the serial merge cost the attention
+    // kernel more than that launch on B200 (measured), so the default is the separate kernel below.
+    const int ns = min(p.splits, (len + p.split_tokens - 1) / p.split_tokens);   // non-empty splits of this slab
+    __threadfence();                                            // this lane's partial is visible device-wide
+    __syncwarp();
+    int prev = 0;
+    if (lane == 0) prev = atomicAdd(p.arrive + slab_local, 1);
+    prev = __shfl_sync(0xffffffffu, prev, 0);
+    if (prev != ns - 1) return;
+    __threadfence();
+    if (lane == 0) p.arrive[slab_local] = 0;                    // ready for the next launch
+    const float *base = p.partial + (size_t)slab_local * p.splits * GQ * kPartStride;
+#pragma unroll 1
+    for (int h = 0; h < GQ; ++h) {
+        const float *bh = base + (size_t)h * kPartStride;
+        float hm = 3.0e38f;
+        for (int j = 0; j < ns; ++j) hm = fminf(hm, __ldcg(bh + (size_t)j * GQ * kPartStride + 128));
+        float4 num = make_float4(0.f, 0.f, 0.f, 0.f);
+        float den = 0.f;
+        for (int j = 0; j < ns; ++j) {
+            const float *pj = bh + (size_t)j * GQ * kPartStride;
+            const float w = exp2f((hm - __ldcg(pj + 128)) * p.c2);
+            const float4 a = __ldcg(reinterpret_cast<const float4 *>(pj) + lane);
+            num.x = fmaf(w, a.x, num.x); num.y = fmaf(w, a.y, num.y);
+            num.z = fmaf(w, a.z, num.z); num.w = fmaf(w, a.w, num.w);
+            den = fmaf(w, __ldcg(pj + 129), den);
+        }
+        const float inv = 1.f / den;
+        float4 o = make_float4(num.x * inv, num.y * inv, num.z * inv, num.w * inv);
+        reinterpret_cast<float4 *>(p.out + (((size_t)ll * p.B + b) * p.Hq + kvh * GQ + h) * kHeadDim)[lane] = o;
+    }
+#endif
 }
 
-// One block per (layer, sequence, query head), one thread per channel.
+// Flash-decoding combine: one block per (layer, sequence, query head), one thread per channel, merges the
+// partials of the sequence's non-empty splits. An empty sequence gives zeros.
 __global__ void __launch_bounds__(kHeadDim) combine_kernel(DecodeParams p) {
     const int c = threadIdx.x;
     const int gq = p.Hq / p.Hkv;
@@ -520,8 +580,7 @@ __global__ void __launch_bounds__(kHeadDim) combine_kernel(DecodeParams p) {
     const int len = p.len[(p.layer_begin + ll) * p.max_batch + b];
     const int kvh = hq / gq, hh = hq % gq;
     const long slab_local = ((long)ll * p.B + b) * p.Hkv + kvh;
-    int ns = (len + p.split_tokens - 1) / p.split_tokens;
-    if (ns > p.splits) ns = p.splits;
+    const int ns = min(p.splits, (len + p.split_tokens - 1) / p.split_tokens);
     const float *base = p.partial + ((size_t)slab_local * p.splits * gq + hh) * kPartStride;
     const size_t stride = (size_t)gq * kPartStride;
     float hm = 3.0e38f;
@@ -560,13 +619,26 @@ __global__ void debug_scores_kernel(const unsigned char *slab, const uint32_t *q
         default: return cudaErrorInvalidValue;                     \
     }
 
-cudaError_t launch_append(const AppendParams &p, const NewCounts &nn, cudaStream_t st, int *launches) {
-    const long rows_per_layer = (long)p.B * p.Tn * p.Hkv;
-    const long tiles = (rows_per_layer + kProjRows - 1) / kProjRows;
-    const long proj_blocks = (long)p.n_layers * tiles * p.m_words;
-    const long quant_blocks = ((long)p.n_layers * rows_per_layer + kProjThreads / 32 - 1) / (kProjThreads / 32);
-    if (proj_blocks + quant_blocks > 0x7fffffffL) return cudaErrorInvalidConfiguration;
-    append_kernel<<<(unsigned)(proj_blocks + quant_blocks), kProjThreads, 0, st>>>(p, nn);
+cudaError_t launch_prepare(const AppendParams *ap, const SketchParams *sp, const NewCounts &nn, cudaStream_t st,
+                           int *launches) {
+    AppendParams a = {};
+    SketchParams q = {};
+    long blocks = 0;
+    if (ap) {
+        a = *ap;
+        const long rows_per_layer = (long)a.B * a.Tn * a.Hkv;
+        const long tiles = (rows_per_layer + kProjRows - 1) / kProjRows;
+        blocks += (long)a.n_layers * tiles * a.m_words;                                               // key tiles
+        blocks += ((long)a.n_layers * rows_per_layer + kProjThreads / 32 - 1) / (kProjThreads / 32);  // value rows
+    }
+    if (sp) {
+        q = *sp;
+        const long rows_per_layer = (long)q.B * q.Hq;
+        blocks += (long)q.n_layers * ((rows_per_layer + kProjRows - 1) / kProjRows) * q.m_words;
+    }
+    if (blocks <= 0) return cudaSuccess;
+    if (blocks > 0x7fffffffL) return cudaErrorInvalidConfiguration;
+    prepare_kernel<<<(unsigned)blocks, kProjThreads, 0, st>>>(a, q, nn);
     ++*launches;
     return cudaGetLastError();
 }
@@ -574,15 +646,6 @@ cudaError_t launch_append(const AppendParams &p, const NewCounts &nn, cudaStream
 cudaError_t launch_set_len(int32_t *len, int n_layers, int max_batch, int seq, int value, cudaStream_t st) {
     const int n = n_layers * max_batch;
     set_len_kernel<<<(n + 127) / 128, 128, 0, st>>>(len, n_layers, max_batch, seq, value);
-    return cudaGetLastError();
-}
-
-cudaError_t launch_sketch(const SketchParams &p, cudaStream_t st, int *launches) {
-    const long rows_per_layer = (long)p.B * p.Hq;
-    if (rows_per_layer <= 0) return cudaSuccess;
-    const long tiles = (rows_per_layer + kProjRows - 1) / kProjRows;
-    sketch_kernel<<<(unsigned)((long)p.n_layers * tiles * p.m_words), kProjThreads, 0, st>>>(p);
-    ++*launches;
     return cudaGetLastError();
 }
 
@@ -617,8 +680,10 @@ cudaError_t launch_decode(const DecodeParams &p, cudaStream_t st, int *launches,
     if (e != cudaSuccess) return e;
     if (after) cudaEventRecord(after, st);
     ++*launches;
+#ifndef H1B_FUSED_COMBINE
     combine_kernel<<<p.n_layers * p.B * p.Hq, kHeadDim, 0, st>>>(p);
     ++*launches;
+#endif
     return cudaGetLastError();
 }
 

@@ -8,8 +8,9 @@ namespace h1b {
 
 // Each launcher enqueues on `st`, adds the number of kernels it launched to
 // *launches and returns the launch error, if any.
-cudaError_t launch_append(const AppendParams &p, const NewCounts &nn, cudaStream_t st, int *launches);
-cudaError_t launch_sketch(const SketchParams &p, cudaStream_t st, int *launches);
+// Either part may be null: `ap` appends keys/values (and bumps the lengths), `sp` sketches queries.
+cudaError_t launch_prepare(const AppendParams *ap, const SketchParams *sp, const NewCounts &nn, cudaStream_t st,
+                           int *launches);
 // `before` / `after`, when not null, are recorded around the split-K attention kernel alone.
 cudaError_t launch_decode(const DecodeParams &p, cudaStream_t st, int *launches, cudaEvent_t before = nullptr,
                           cudaEvent_t after = nullptr);

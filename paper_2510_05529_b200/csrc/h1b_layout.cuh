@@ -103,6 +103,7 @@ struct DecodeParams {
     float *partial;             // [items][GQ][kPartStride]
     float *out;                 // fp32 [n_layers][B][Hq][d]
     int32_t *status;
+    int32_t *arrive;            // [slabs of the call]: splits that have reported in (zero between launches)
     size_t slab_bytes;
     int layer_begin, n_layers, B, Hkv, Hq, max_batch, m_words;
     int splits, split_tokens;   // split_tokens is a multiple of 32

@@ -126,11 +126,16 @@ def test_host_step_equals_device_calls():
     outh = torch.empty(qh.shape, dtype=torch.float32).pin_memory()
     cache.h1b_decode_step_host(kh, vh, qh, 16.0, outh)
     assert cache.h1b_get_lengths(0)[:2].tolist() == [100, 51]
-    # the same step on a second cache with device tensors
+    # the same step on a second cache with device tensors, as two calls ...
     r2 = build_and_decode(w, [99, 50], max_seq=128)
     r2["cache"].h1b_append_kv(kh.cuda(), vh.cuda())
     out2 = r2["cache"].h1b_decode_attention(r2["qd"], 16.0)
     assert np.array_equal(outh.numpy(), out2.cpu().numpy())
+    # ... and on a third one as the fused device step
+    r3 = build_and_decode(w, [99, 50], max_seq=128)
+    out3 = r3["cache"].h1b_decode_step(kh.cuda(), vh.cuda(), r3["qd"], 16.0)
+    assert np.array_equal(outh.numpy(), out3.cpu().numpy())
+    assert r3["cache"].h1b_get_lengths(1)[:2].tolist() == [100, 51]
     # and against the oracle, end to end, for one sequence
     K = torch.cat([r["K"][:, :, :100], torch.zeros_like(r["K"][:, :, :1])], 2)
     V = torch.cat([r["V"][:, :, :100], torch.zeros_like(r["V"][:, :, :1])], 2)
