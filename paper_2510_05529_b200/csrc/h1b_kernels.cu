@@ -261,6 +261,7 @@ struct DecodeState {
     float ssum[GQ];             // per-lane partial sum of the weights
     float accz[GQ][kGroups];    // per-lane partial sum of p * zero
     uint32_t qw[GQ][MW];        // query sketches
+    float zero[4];              // an opaque quad of zeros: C operand of each chunk's first MMA
 };
 
 // One chunk. TAIL: tokens at or beyond t_end are masked (only the last chunk of a split needs it).
@@ -354,7 +355,7 @@ __device__ __forceinline__ void decode_chunk(DecodeState<MW, GQ> &st, const unsi
                 const int bi = (cb >> 1) / NG;
                 uint32_t a[4];
                 codes_to_f16x2(wv[i], a);
-                if (vb == 0) mma_f16_16816_zero(tmp[i], a[0], a[1], a[2], a[3], bf[vb][bi][0], bf[vb][bi][1]);
+                if (vb == 0) mma_f16_16816_from(tmp[i], a[0], a[1], a[2], a[3], bf[vb][bi][0], bf[vb][bi][1], st.zero);
                 else mma_f16_16816(tmp[i], a[0], a[1], a[2], a[3], bf[vb][bi][0], bf[vb][bi][1]);
             }
         }
@@ -423,6 +424,7 @@ __global__ void __launch_bounds__(kDecodeWarps * 32, decode_min_blocks(GQ)) deco
     }
 
     DecodeState<MW, GQ> st;
+    zero_quad(st.zero);
     {
         const uint32_t *qp = p.qwords + ((size_t)(layer * p.max_batch + b) * p.Hq + kvh * GQ) * MW;
 #pragma unroll

@@ -107,13 +107,21 @@ __device__ __forceinline__ void codes_to_f16x2(uint32_t w, uint32_t (&a)[4]) {
 }
 #endif
 
-// D = A * B (accumulator starts at zero).
-__device__ __forceinline__ void mma_f16_16816_zero(float (&d)[4], uint32_t a0, uint32_t a1, uint32_t a2, uint32_t a3,
-                                                   uint32_t b0, uint32_t b1) {
+// D = A * B + Z, where Z is a quad of registers that the caller keeps at zero (see zero_quad): the
+// accumulator starts at zero without four register moves per MMA.
+__device__ __forceinline__ void mma_f16_16816_from(float (&d)[4], uint32_t a0, uint32_t a1, uint32_t a2, uint32_t a3,
+                                                   uint32_t b0, uint32_t b1, const float (&z)[4]) {
     asm volatile(
-        "mma.sync.aligned.m16n8k16.row.col.f32.f16.f16.f32 {%0,%1,%2,%3}, {%4,%5,%6,%7}, {%8,%9}, {%10,%10,%10,%10};"
+        "mma.sync.aligned.m16n8k16.row.col.f32.f16.f16.f32 {%0,%1,%2,%3}, {%4,%5,%6,%7}, {%8,%9}, {%10,%11,%12,%13};"
         : "=f"(d[0]), "=f"(d[1]), "=f"(d[2]), "=f"(d[3])
-        : "r"(a0), "r"(a1), "r"(a2), "r"(a3), "r"(b0), "r"(b1), "f"(0.f));
+        : "r"(a0), "r"(a1), "r"(a2), "r"(a3), "r"(b0), "r"(b1), "f"(z[0]), "f"(z[1]), "f"(z[2]), "f"(z[3]));
+}
+
+// Four zeros the compiler cannot see through, so that it keeps them in one register quad for the
+// whole kernel instead of re-creating them wherever they are used.
+__device__ __forceinline__ void zero_quad(float (&z)[4]) {
+    asm volatile("mov.f32 %0, 0f00000000;\n\tmov.f32 %1, 0f00000000;\n\tmov.f32 %2, 0f00000000;\n\tmov.f32 %3, 0f00000000;"
+                 : "=f"(z[0]), "=f"(z[1]), "=f"(z[2]), "=f"(z[3]));
 }
 
 __device__ __forceinline__ float2 half2_bits_to_float2(uint32_t h2) {
