@@ -33,9 +33,11 @@ if ROOT not in sys.path:
 METRIC = "decode-attn tokens/s (7B shape, 8k ctx): append 1 token + decode attention over 32 layers"
 UNIT = "tokens/s"
 INV_TAU = 16.0
-# DRAM bytes of one decode_split_kernel launch on the bench workload, from the ncu capture
-# summarised under profiles/ (dram__bytes_read.sum + dram__bytes_write.sum); None = not captured.
-NCU_TRAFFIC_BYTES_PER_LAUNCH = None
+# DRAM traffic of one decode_split_kernel launch (dram__bytes_read.sum + dram__bytes_write.sum) per
+# algorithmic byte, from the ncu capture summarised in profiles/decode_split_kernel_c2_7b_8k.md
+# (815.8 MB moved for 806.0 MB needed at 8199 cached tokens). Traffic grows in proportion to the cached
+# tokens, so the bench scales it to the context it actually ran.
+NCU_TRAFFIC_PER_ALGORITHMIC_BYTE = 1.0122
 
 
 def measured_peaks():
@@ -117,17 +119,12 @@ def run_ours(args):
     import h1b_synth
     from paper_2510_05529_b200 import binding
 
-    rank = int(os.environ.get("RANK", "0"))
-    world = int(os.environ.get("WORLD_SIZE", "1"))
-    local = int(os.environ.get("LOCAL_RANK", "0"))
+    from paper_2510_05529_b200 import dist as pdist
+    rank, world, local = pdist.world()
     if not torch.cuda.is_available():
         raise SystemExit("bench.py needs a CUDA device: the hot path has no CPU fallback")
     torch.cuda.set_device(local)
-    dist = None
-    if world > 1:
-        import torch.distributed as dist_mod
-        dist_mod.init_process_group("nccl", device_id=torch.device("cuda", local))
-        dist = dist_mod
+    pdist.init("nccl", torch.device("cuda", local))
     dev = torch.device("cuda", local)
     w = h1b_synth.WORKLOADS["c2_7b_8k"]
     steps, warmup = args.steps, args.warmup
@@ -159,8 +156,7 @@ def run_ours(args):
         cache.h1b_decode_step(kn[i % pool], vn[i % pool], qn[i % pool], INV_TAU, out=out)
 
     def barrier():
-        if dist is not None:
-            dist.barrier()
+        pdist.barrier()
         torch.cuda.synchronize()
 
     for i in range(warmup):
@@ -203,14 +199,10 @@ def run_ours(args):
     barrier()
     e2e_ms_total = e0.elapsed_time(e1)
 
-    t = torch.tensor([ms_total, e2e_ms_total], dtype=torch.float64, device=dev)
-    if dist is not None:
-        dist.all_reduce(t, op=dist.ReduceOp.MAX)
-    ms_total, e2e_ms_total = float(t[0]), float(t[1])
-    tokens_per_step = w.batch * world
+    ms_total, e2e_ms_total = pdist.max_over_ranks([ms_total, e2e_ms_total], dev)     # slowest rank
     ms_per_step = ms_total / steps
-    value = tokens_per_step / (ms_per_step * 1e-3)
-    e2e_value = tokens_per_step / (e2e_ms_total / steps * 1e-3)
+    value = pdist.whole_job_rate(w.batch, world, ms_per_step * 1e-3)
+    e2e_value = pdist.whole_job_rate(w.batch, world, e2e_ms_total / steps * 1e-3)
 
     # roofline of the dominant kernel (split-K decode attention), per launch
     entry = binding.h1b_entry_bytes(cfg)
@@ -224,7 +216,8 @@ def run_ours(args):
                 "peak_kind": peak_kind + " (MEASURED_PEAKS.json hbm_gbs)" if peak_kind == "measured" else "fallback",
                 "unit": "GB/s", "frac": (achieved / peak) if achieved else None,
                 "frac_of_8tbs_nominal": (achieved / 8000.0) if achieved else None,
-                "traffic": NCU_TRAFFIC_BYTES_PER_LAUNCH, "alg_bytes_per_launch": alg_bytes,
+                "traffic": NCU_TRAFFIC_PER_ALGORITHMIC_BYTE * alg_bytes, "traffic_source": "ncu capture at 8199 tokens, scaled by algorithmic bytes",
+                "alg_bytes_per_launch": alg_bytes,
                 "kernel_ms_avg": kern_ms_avg, "kernel_launches_timed": kern_n,
                 "step_gbs": alg_bytes / (ms_per_step * 1e-3) / 1e9}
     line = {
@@ -246,9 +239,7 @@ def run_ours(args):
     if rank == 0 and world == 1 and not args.no_cpu_baseline:
         line["cpu_baseline"] = cpu_baseline(sample_layers=1, steps=5, warmup=1)
     cache.close()
-    if dist is not None:
-        dist.barrier()
-        dist.destroy_process_group()
+    pdist.finish()
     if rank == 0:
         print(json.dumps(line))
 
