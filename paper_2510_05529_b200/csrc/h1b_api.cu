@@ -21,9 +21,10 @@ namespace {
 
 constexpr long kTargetItems = 8192;   // decode work items aimed for (one warp each)
 constexpr int kMinSplitTokens = 256;
+constexpr int kPrefillMinTokens = 64;   // appends of at least this many tokens per sequence take the tensor-core path
 
 struct Plan {
-    size_t rt, len, status, arrive, qwords, partial, stage_k, stage_v, stage_q, stage_out, dbg_q, dbg_s, cache, total;
+    size_t rt, rh, len, status, arrive, qwords, partial, stage_k, stage_v, stage_q, stage_out, dbg_q, dbg_s, cache, total;
     size_t partial_items, slab_bytes;
     int cap_tokens, m_words, gq;
 };
@@ -61,6 +62,7 @@ int make_plan(const h1b_config *c, Plan *p) {
     size_t o = 0;
     auto take = [&](size_t bytes) { size_t at = o; o = align_up(o + bytes, 256); return at; };
     p->rt = take(L * d * c->sketch_bits * sizeof(float));
+    p->rh = take(L * 2 * d * c->sketch_bits * sizeof(uint16_t));     // fp16 pieces of Rt for the tensor-core prefill
     p->len = take(L * B * sizeof(int32_t));
     p->status = take(64);
     p->arrive = take(slabs * sizeof(int32_t));
@@ -209,6 +211,8 @@ int h1b_init_projection(const h1b_config *cfg, uint64_t seed, const float *Rt_ho
     }
     e = cudaMemcpyAsync(ctx->ws + plan.rt, Rt_host, nR * sizeof(float), cudaMemcpyHostToDevice, st);
     if (e != cudaSuccess) return bail(e, "cudaMemcpyAsync(Rt)");
+    e = launch_split_projection(at<float>(ctx, plan.rt), at<uint16_t>(ctx, plan.rh), cfg->n_layers, cfg->sketch_bits, st);
+    if (e != cudaSuccess) return bail(e, "split_projection_kernel");
     e = cudaStreamSynchronize(st);
     if (e != cudaSuccess) return bail(e, "cudaStreamSynchronize");
     *out = ctx;
@@ -331,9 +335,32 @@ int h1b_append_kv(h1b_ctx *ctx, int layer_begin, int n_layers, const void *k, co
     NewCounts nn;
     rc = make_new_counts(ctx, layer_begin, n_layers, n_new_host, B, Tn, &nn);
     if (rc != H1B_OK) return rc;
-    const AppendParams ap = append_params(ctx, layer_begin, n_layers, k, v, B, Tn);
     int launches = 0;
-    H1B_CUDA(ctx, launch_prepare(&ap, nullptr, nn, static_cast<cudaStream_t>(stream), &launches));
+    if (Tn >= kPrefillMinTokens) {
+        // long append: tensor-core projection over tiles of 128 cache positions
+        PrefillParams pp;
+        pp.k = static_cast<const uint16_t *>(k);
+        pp.v = static_cast<const uint16_t *>(v);
+        pp.Rh = at<uint16_t>(ctx, ctx->plan.rh);
+        pp.cache = ctx->ws + ctx->plan.cache;
+        pp.len = at<int32_t>(ctx, ctx->plan.len);
+        pp.done = at<int32_t>(ctx, ctx->plan.status) + 4;
+        pp.slab_bytes = ctx->plan.slab_bytes;
+        pp.layer_begin = layer_begin; pp.n_layers = n_layers; pp.B = B; pp.Tn = Tn;
+        pp.Hkv = ctx->cfg.n_kv_heads; pp.max_batch = ctx->cfg.max_batch; pp.m_words = ctx->plan.m_words;
+        int tiles = 1;
+        for (int l = layer_begin; l < layer_begin + n_layers; ++l)
+            for (int b = 0; b < B; ++b) {
+                const int len0 = ctx->len_host[(size_t)l * ctx->cfg.max_batch + b];
+                if (nn.v[b] > 0) tiles = std::max(tiles, (len0 + nn.v[b] + 127) / 128 - len0 / 128);
+            }
+        pp.tiles_per_seq = tiles;
+        pp.tiles_per_block = std::min(tiles, 8);
+        H1B_CUDA(ctx, launch_prefill(pp, nn, static_cast<cudaStream_t>(stream), &launches));
+    } else {
+        const AppendParams ap = append_params(ctx, layer_begin, n_layers, k, v, B, Tn);
+        H1B_CUDA(ctx, launch_prepare(&ap, nullptr, nn, static_cast<cudaStream_t>(stream), &launches));
+    }
     ctx->launches += launches;
     commit_lengths(ctx, layer_begin, n_layers, B, nn);
     return H1B_OK;

@@ -209,6 +209,241 @@ __global__ void __launch_bounds__(kProjThreads) prepare_kernel(AppendParams ap, 
     }
 }
 
+// ===========================================================================
+// Prefill: long appends. One block = up to `tiles_per_block` tiles of 128 consecutive cache positions
+// of ONE slab (layer, sequence, KV head) x one block of up to 128 sketch columns.
+//
+//   Eq. 2 as a dense contraction on the tensor cores: y = K (fp16, exact) x [Rh1 + Rh2], where
+//   Rh1 = fp16(Rt) and Rh2 = fp16(Rt - Rh1): |Rt - Rh1 - Rh2| <= 2^-22 |Rt| (or 2^-25 absolute), so y is within
+//   ~1e-6 * sum|terms| of the exact projection, well inside the 1e-5 sign-boundary window. ldmatrix from
+//   XOR-swizzled shared memory, mma.sync.m16n8k16 fp16 -> fp32; warp w owns rows 16w..16w+15 of the tile.
+//   The signs are packed from the accumulator fragments (2 bits per thread per n-tile, OR-reduced over
+//   the quad) and stored as the tile's key words.
+//   Eq. 4: warp w quantises tokens 16w..16w+15 = one 16-token value block: codes are assembled in shared
+//   memory in the block's packed order and written with 16-byte stores. The division (v - min)/scale is
+//   q1 = q0 + (t - q0*scale)*inv with inv = RN(1/scale), q0 = RN(t*inv): correctly rounded (Markstein), i.e.
+//   the same bits as IEEE division; the scale (max-min)/15 -> fp16 is taken in fp32 when that is provably
+//   the correctly rounded result and in fp64 otherwise.
+// ===========================================================================
+constexpr int kPrefillThreads = 256;
+constexpr int kPrefillTile = 128;              // cache positions per tile
+
+template <int NBC>                             // sketch columns per block: 128 or 64
+struct PrefillSmem {
+    static constexpr int kRBytes = 2 * kHeadDim * NBC * 2;          // two fp16 pieces of the projection block
+    static constexpr int kABytes = kPrefillTile * kHeadDim * 2;     // the key tile
+    static constexpr int kVBytes = (kPrefillThreads / 32) * 1280;   // per warp: 1024 B codes + 128 B scale + 128 B zero
+    static constexpr int kTotal = kRBytes + kABytes + kVBytes;
+};
+
+// fp16((mx - mn) / 15), correctly rounded from the exact quotient.
+__device__ __forceinline__ __half exact_scale(float mx, float mn) {
+    const float d = __fsub_rn(mx, mn);
+    const float r = __fdiv_rn(d, 15.f);
+    // fp32 is enough when the subtraction is exact (magnitudes within 2^12 of each other: the difference of two
+    // fp16 numbers then fits 24 bits), the quotient is a normal fp16 and not on an fp16 rounding midpoint.
+    const float amx = fabsf(mx), amn = fabsf(mn);
+    const bool close = (amx <= amn * 4096.f) && (amn <= amx * 4096.f);
+    const uint32_t low = __float_as_uint(r) & 0x1FFFu;              // the 13 bits fp16 drops
+    const bool off_mid = (low < 0x0FFFu) || (low > 0x1001u);
+    if ((close || d == 0.f) && off_mid && (r >= 6.2e-5f || d == 0.f)) return __float2half_rn(r);
+    return __double2half(((double)mx - (double)mn) / 15.0);
+}
+
+template <int NBC>
+__global__ void __launch_bounds__(kPrefillThreads, 2) prefill_kernel(PrefillParams p, NewCounts nn) {
+    using SM = PrefillSmem<NBC>;
+    constexpr int NT = NBC / 8;                // n-tiles of 8 columns
+    constexpr int RCH = NBC / 8;               // 16-byte chunks per projection row
+    extern __shared__ __align__(128) unsigned char smem[];
+    unsigned char *Rs = smem, *As = smem + SM::kRBytes, *Vs = As + SM::kABytes;
+    const int tid = threadIdx.x, lane = tid & 31, warp = tid >> 5;
+    const int m = p.m_words * 32;
+    const ChunkLayout cl = chunk_layout(p.m_words);
+    const int groups_per_slab = (p.tiles_per_seq + p.tiles_per_block - 1) / p.tiles_per_block;
+    const int tg = blockIdx.x % groups_per_slab;
+    const long slab_local = blockIdx.x / groups_per_slab;
+    const int kvh = (int)(slab_local % p.Hkv), b = (int)((slab_local / p.Hkv) % p.B), ll = (int)(slab_local / ((long)p.Hkv * p.B));
+    const int layer = p.layer_begin + ll;
+    const int col0 = blockIdx.y * NBC;         // first sketch column of this block
+    const int len0 = p.len[layer * p.max_batch + b];
+    const int n_new = nn.v[b];
+    unsigned char *slab = p.cache + ((size_t)(layer * p.max_batch + b) * p.Hkv + kvh) * p.slab_bytes;
+
+    // ---- the two fp16 pieces of Rt[:, col0 .. col0+NBC), swizzled: chunk c of row k at c ^ (k & 7)
+    {
+        const uint16_t *src = p.Rh + (size_t)layer * 2 * kHeadDim * m;
+        for (int e = tid; e < 2 * kHeadDim * RCH; e += kPrefillThreads) {
+            const int c = e % RCH, k = (e / RCH) % kHeadDim, piece = e / (RCH * kHeadDim);
+            cp_async_16(smem_addr(Rs + ((size_t)(piece * kHeadDim + k) * RCH + (c ^ (k & 7))) * 16),
+                        src + ((size_t)piece * kHeadDim + k) * m + col0 + c * 8, 16);
+        }
+    }
+    const int first_tile = len0 / kPrefillTile + tg * p.tiles_per_block;
+    for (int ti = 0; ti < p.tiles_per_block; ++ti) {
+        const int P0 = (first_tile + ti) * kPrefillTile;
+        if (P0 >= len0 + n_new) break;                          // block-uniform
+        // ---- key tile: row r = position P0 + r, chunk c at c ^ (r & 7); rows outside the appended range are zero
+        for (int e = tid; e < kPrefillTile * 16; e += kPrefillThreads) {
+            const int c = e & 15, r = e >> 4;
+            const int tn = P0 + r - len0;
+            const bool ok = tn >= 0 && tn < n_new;
+            const uint16_t *src = p.k + ((((size_t)ll * p.B + b) * p.Tn + (ok ? tn : 0)) * p.Hkv + kvh) * kHeadDim + c * 8;
+            cp_async_16(smem_addr(As + (size_t)r * 256 + ((c ^ (r & 7)) << 4)), src, ok ? 16u : 0u);
+        }
+        cp_async_wait_all();
+        __syncthreads();
+
+        // ---- y = K x (Rh1 + Rh2): warp w, rows 16w..16w+15, all NBC columns
+        float acc[NT][4];
+#pragma unroll
+        for (int nt = 0; nt < NT; ++nt) { acc[nt][0] = 0.f; acc[nt][1] = 0.f; acc[nt][2] = 0.f; acc[nt][3] = 0.f; }
+        const uint32_t a_base = smem_addr(As), r_base = smem_addr(Rs);
+        const int lrow = (lane & 7) + ((lane >> 3) & 1) * 8, lhalf = lane >> 4;     // ldmatrix row / second-8 selector
+#pragma unroll
+        for (int ks = 0; ks < kHeadDim / 16; ++ks) {
+            uint32_t a[4];
+            {
+                const int r = warp * 16 + lrow, c = ks * 2 + lhalf;
+                ldmatrix_x4(a, a_base + r * 256 + ((c ^ (r & 7)) << 4));
+            }
+#pragma unroll
+            for (int piece = 0; piece < 2; ++piece) {
+#pragma unroll
+                for (int np = 0; np < NT / 2; ++np) {           // two n-tiles per ldmatrix
+                    uint32_t bq[4];
+                    const int k = ks * 16 + lrow, c = np * 2 + lhalf;
+                    ldmatrix_x4_trans(bq, r_base + ((piece * kHeadDim + k) * RCH + (c ^ (k & 7))) * 16);
+                    mma_f16_16816(acc[2 * np], a[0], a[1], a[2], a[3], bq[0], bq[1]);
+                    mma_f16_16816(acc[2 * np + 1], a[0], a[1], a[2], a[3], bq[2], bq[3]);
+                }
+            }
+        }
+        // ---- signs -> words. Thread (g = lane/4, jq = lane%4) holds rows g, g+8 and columns nt*8 + 2jq, +1.
+        {
+            constexpr int NW = NBC / 32;                        // words per row in this column block
+            uint32_t w_lo[NW], w_hi[NW];
+#pragma unroll
+            for (int w = 0; w < NW; ++w) { w_lo[w] = 0; w_hi[w] = 0; }
+            const int jq = lane & 3, g = lane >> 2;
+#pragma unroll
+            for (int nt = 0; nt < NT; ++nt) {
+                const int sh = (nt & 3) * 8 + 2 * jq;
+                w_lo[nt >> 2] |= ((acc[nt][0] >= 0.f ? 1u : 0u) | (acc[nt][1] >= 0.f ? 2u : 0u)) << sh;
+                w_hi[nt >> 2] |= ((acc[nt][2] >= 0.f ? 1u : 0u) | (acc[nt][3] >= 0.f ? 2u : 0u)) << sh;
+            }
+#pragma unroll
+            for (int w = 0; w < NW; ++w) {
+                w_lo[w] |= __shfl_xor_sync(0xffffffffu, w_lo[w], 1); w_lo[w] |= __shfl_xor_sync(0xffffffffu, w_lo[w], 2);
+                w_hi[w] |= __shfl_xor_sync(0xffffffffu, w_hi[w], 1); w_hi[w] |= __shfl_xor_sync(0xffffffffu, w_hi[w], 2);
+            }
+            // quad lane jq stores word jq (and jq + 4, ... when there are more than four)
+#pragma unroll
+            for (int w = 0; w < NW; ++w) {
+                if ((w & 3) == jq) {
+#pragma unroll
+                    for (int hi = 0; hi < 2; ++hi) {
+                        const int pos = P0 + warp * 16 + g + hi * 8, tn = pos - len0;
+                        if (tn >= 0 && tn < n_new)
+                            *reinterpret_cast<uint32_t *>(slab + (size_t)(pos >> 5) * cl.bytes +
+                                                          key_word_off(col0 / 32 + w, pos & 31)) = hi ? w_hi[w] : w_lo[w];
+                    }
+                }
+            }
+        }
+        // ---- values: warp w quantises tokens P0 + 16w .. +15 (one value block); only the first column block does it
+        if (blockIdx.y == 0) {
+            const int pos0 = P0 + warp * 16;
+            const int tn0 = pos0 - len0;
+            unsigned char *chunk = slab + (size_t)(pos0 >> 5) * cl.bytes;
+            const int vb = (pos0 >> 4) & 1;
+            if (tn0 >= 0 && tn0 + 16 <= n_new) {                // a whole block: assemble it in shared memory
+                unsigned char *vs = Vs + warp * 1280;
+                const int cb = lane >> 2, jj = lane & 3, grp = lane >> 3;
+                const size_t row_stride = (size_t)p.Hkv * kHeadDim;
+                const uint16_t *v0 = p.v + ((((size_t)ll * p.B + b) * p.Tn + tn0) * p.Hkv + kvh) * kHeadDim;
+#pragma unroll 4
+                for (int k = 0; k < 16; ++k) {
+                    const __half2 *vrow = reinterpret_cast<const __half2 *>(v0 + (size_t)k * row_stride);
+                    const float2 va = __half22float2(__ldg(vrow + ((cb * 16 + 2 * jj) >> 1)));
+                    const float2 vb2 = __half22float2(__ldg(vrow + ((cb * 16 + 2 * jj + 8) >> 1)));
+                    float mn = fminf(fminf(va.x, va.y), fminf(vb2.x, vb2.y));
+                    float mx = fmaxf(fmaxf(va.x, va.y), fmaxf(vb2.x, vb2.y));
+#pragma unroll
+                    for (int s = 1; s < 8; s <<= 1) {
+                        mn = fminf(mn, __shfl_xor_sync(0xffffffffu, mn, s));
+                        mx = fmaxf(mx, __shfl_xor_sync(0xffffffffu, mx, s));
+                    }
+                    if (mn == 0.f) mn = 0.f;
+                    const __half hd = exact_scale(mx, mn);
+                    const float delta = __half2float(hd);
+                    const float inv = (delta == 0.f) ? 0.f : __frcp_rn(delta);
+                    auto code = [&](float v) -> uint32_t {
+                        const float t = __fsub_rn(v, mn);
+                        const float q0 = __fmul_rn(t, inv);
+                        const float q1 = __fmaf_rn(__fmaf_rn(-q0, delta, t), inv, q0);      // = RN(t / delta)
+                        const float x = fminf(fmaxf(q1, 0.f), 15.f) + 12582912.f;           // round half to even
+                        return (delta == 0.f) ? 0u : (__float_as_uint(x) & 15u);
+                    };
+                    const uint32_t q0 = code(va.x), q1 = code(va.y), q8 = code(vb2.x), q9 = code(vb2.y);
+                    // in-block byte of (token k, channel block cb, row r): see code_byte_off
+                    const int jt = (k & 7) >> 1, byte = (k & 1) * 2 + (k >> 3);
+                    vs[(cb >> 2) * 512 + ((2 * jj) * 4 + jt) * 16 + (cb & 3) * 4 + byte] = (unsigned char)(q0 | (q8 << 4));
+                    vs[(cb >> 2) * 512 + ((2 * jj + 1) * 4 + jt) * 16 + (cb & 3) * 4 + byte] = (unsigned char)(q1 | (q9 << 4));
+                    if ((lane & 7) == 0) {
+                        *reinterpret_cast<__half *>(vs + 1024 + grp * 32 + k * 2) = hd;                    // scale [g][16 tokens]
+                        *reinterpret_cast<__half *>(vs + 1152 + k * 8 + grp * 2) = __float2half_rn(mn);    // zero  [16 tokens][g]
+                    }
+                }
+                __syncwarp();
+                const uint4 *src = reinterpret_cast<const uint4 *>(vs);
+                uint4 *dst = reinterpret_cast<uint4 *>(chunk + cl.val_off + vb * kValBlockBytes);
+                dst[lane] = src[lane];
+                dst[32 + lane] = src[32 + lane];
+                if (lane < 8) reinterpret_cast<uint4 *>(chunk + cl.scale_off + vb * 128)[lane] = src[64 + lane];
+                else if (lane < 16) reinterpret_cast<uint4 *>(chunk + cl.zero_off + vb * 128)[lane - 8] = src[72 + lane - 8];
+                __syncwarp();
+            } else {                                            // ragged edge of the appended range: row by row
+                for (int k = 0; k < 16; ++k) {
+                    const int tn = tn0 + k;
+                    if (tn >= 0 && tn < n_new)
+                        quantize_row(p.v + ((((size_t)ll * p.B + b) * p.Tn + tn) * p.Hkv + kvh) * kHeadDim,
+                                     slab + (size_t)((pos0 + k) >> 5) * cl.bytes, cl, (pos0 + k) & 31, lane);
+                }
+            }
+        }
+        __syncthreads();                                        // the key tile is overwritten by the next iteration
+    }
+    cp_async_wait_all();
+    // ---- the last block to finish publishes the new lengths
+    __shared__ int is_last;
+    __syncthreads();
+    if (tid == 0) {
+        __threadfence();
+        is_last = (atomicAdd(p.done, 1) == (int)(gridDim.x * gridDim.y) - 1);
+    }
+    __syncthreads();
+    if (is_last) {
+        for (int i = tid; i < p.n_layers * p.B; i += blockDim.x)
+            p.len[(p.layer_begin + i / p.B) * p.max_batch + (i % p.B)] += nn.v[i % p.B];
+        if (tid == 0) *p.done = 0;
+    }
+}
+
+// Rt (fp32) -> its two fp16 pieces, [L][2][d][m].
+__global__ void split_projection_kernel(const float *Rt, uint16_t *Rh, int n_layers, int m) {
+    const long n = (long)n_layers * kHeadDim * m;
+    for (long e = (long)blockIdx.x * blockDim.x + threadIdx.x; e < n; e += (long)gridDim.x * blockDim.x) {
+        const long l = e / ((long)kHeadDim * m), rest = e % ((long)kHeadDim * m);
+        const float r = Rt[e];
+        const __half h1 = __float2half_rn(r);
+        const __half h2 = __float2half_rn(r - __half2float(h1));
+        __half *dst = reinterpret_cast<__half *>(Rh) + l * 2 * kHeadDim * m;
+        dst[rest] = h1;
+        dst[(long)kHeadDim * m + rest] = h2;
+    }
+}
+
 __global__ void set_len_kernel(int32_t *len, int n_layers, int max_batch, int seq, int value) {
     const int i = blockIdx.x * blockDim.x + threadIdx.x;
     if (i >= n_layers * max_batch) return;
@@ -642,6 +877,37 @@ cudaError_t launch_prepare(const AppendParams *ap, const SketchParams *sp, const
     if (blocks > 0x7fffffffL) return cudaErrorInvalidConfiguration;
     prepare_kernel<<<(unsigned)blocks, kProjThreads, 0, st>>>(a, q, nn);
     ++*launches;
+    return cudaGetLastError();
+}
+
+template <int NBC>
+static cudaError_t launch_prefill_t(const PrefillParams &p, const NewCounts &nn, cudaStream_t st) {
+    using SM = PrefillSmem<NBC>;
+    static bool attr_set[64] = {};
+    int dev = 0;
+    cudaGetDevice(&dev);
+    if (dev >= 0 && dev < 64 && !attr_set[dev]) {
+        cudaError_t e = cudaFuncSetAttribute(prefill_kernel<NBC>, cudaFuncAttributeMaxDynamicSharedMemorySize, SM::kTotal);
+        if (e != cudaSuccess) return e;
+        attr_set[dev] = true;
+    }
+    const long groups = (p.tiles_per_seq + p.tiles_per_block - 1) / p.tiles_per_block;
+    const long gx = (long)p.n_layers * p.B * p.Hkv * groups;
+    if (gx <= 0 || gx > 0x7fffffffL) return cudaErrorInvalidConfiguration;
+    const int m = p.m_words * 32;
+    dim3 grid((unsigned)gx, (unsigned)((m + NBC - 1) / NBC));
+    prefill_kernel<NBC><<<grid, kPrefillThreads, SM::kTotal, st>>>(p, nn);
+    return cudaGetLastError();
+}
+
+cudaError_t launch_prefill(const PrefillParams &p, const NewCounts &nn, cudaStream_t st, int *launches) {
+    cudaError_t e = (p.m_words * 32 >= 128) ? launch_prefill_t<128>(p, nn, st) : launch_prefill_t<64>(p, nn, st);
+    if (e == cudaSuccess) ++*launches;
+    return e;
+}
+
+cudaError_t launch_split_projection(const float *Rt, uint16_t *Rh, int n_layers, int m, cudaStream_t st) {
+    split_projection_kernel<<<148 * 4, 256, 0, st>>>(Rt, Rh, n_layers, m);
     return cudaGetLastError();
 }
 

@@ -89,6 +89,18 @@ struct AppendParams {
     int layer_begin, n_layers, B, Tn, Hkv, max_batch, m_words;
 };
 
+struct PrefillParams {          // long appends: tensor-core projection
+    const uint16_t *k, *v;      // fp16 [n_layers][B][Tn][Hkv][d]
+    const uint16_t *Rh;         // fp16 [L][2][d][m]: Rt split exactly-enough as fp16(Rt) + fp16(Rt - fp16(Rt))
+    unsigned char *cache;
+    int32_t *len;               // [L][max_batch]
+    int32_t *done;              // block counter (zero between launches)
+    size_t slab_bytes;
+    int layer_begin, n_layers, B, Tn, Hkv, max_batch, m_words;
+    int tiles_per_seq;          // 128-position tiles that can overlap the appended range of a sequence
+    int tiles_per_block;        // consecutive tiles handled by one block (the projection is loaded once per block)
+};
+
 struct SketchParams {           // query sketch
     const uint16_t *q;          // fp16 [n_layers][B][Hq][d]
     const float *Rt;
