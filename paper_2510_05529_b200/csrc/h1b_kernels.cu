@@ -239,7 +239,9 @@ struct PrefillSmem {
 // fp16((mx - mn) / 15), correctly rounded from the exact quotient.
 __device__ __forceinline__ __half exact_scale(float mx, float mn) {
     const float d = __fsub_rn(mx, mn);
-    const float r = __fdiv_rn(d, 15.f);
+    // d / 15, correctly rounded: q0 = RN(d * RN(1/15)), one exact-residual correction (Markstein)
+    const float q0 = __fmul_rn(d, 0.0666666701436042786f);
+    const float r = __fmaf_rn(__fmaf_rn(-q0, 15.f, d), 0.0666666701436042786f, q0);
     // fp32 is enough when the subtraction is exact (magnitudes within 2^12 of each other: the difference of two
     // fp16 numbers then fits 24 bits), the quotient is a normal fp16 and not on an fp16 rounding midpoint.
     const float amx = fabsf(mx), amn = fabsf(mn);
@@ -358,42 +360,58 @@ __global__ void __launch_bounds__(kPrefillThreads, 2) prefill_kernel(PrefillPara
             unsigned char *chunk = slab + (size_t)(pos0 >> 5) * cl.bytes;
             const int vb = (pos0 >> 4) & 1;
             if (tn0 >= 0 && tn0 + 16 <= n_new) {                // a whole block: assemble it in shared memory
+                // lane = (row rsub of 8, group grp of 4): 32 channels of one row per lane and pass, two passes
                 unsigned char *vs = Vs + warp * 1280;
-                const int cb = lane >> 2, jj = lane & 3, grp = lane >> 3;
+                const int rsub = lane >> 2, grp = lane & 3;
                 const size_t row_stride = (size_t)p.Hkv * kHeadDim;
-                const uint16_t *v0 = p.v + ((((size_t)ll * p.B + b) * p.Tn + tn0) * p.Hkv + kvh) * kHeadDim;
-#pragma unroll 4
-                for (int k = 0; k < 16; ++k) {
-                    const __half2 *vrow = reinterpret_cast<const __half2 *>(v0 + (size_t)k * row_stride);
-                    const float2 va = __half22float2(__ldg(vrow + ((cb * 16 + 2 * jj) >> 1)));
-                    const float2 vb2 = __half22float2(__ldg(vrow + ((cb * 16 + 2 * jj + 8) >> 1)));
-                    float mn = fminf(fminf(va.x, va.y), fminf(vb2.x, vb2.y));
-                    float mx = fmaxf(fmaxf(va.x, va.y), fmaxf(vb2.x, vb2.y));
+                const uint16_t *v0 = p.v + ((((size_t)ll * p.B + b) * p.Tn + tn0) * p.Hkv + kvh) * kHeadDim + grp * 32;
+                uint4 raw[2][4];
 #pragma unroll
-                    for (int s = 1; s < 8; s <<= 1) {
-                        mn = fminf(mn, __shfl_xor_sync(0xffffffffu, mn, s));
-                        mx = fmaxf(mx, __shfl_xor_sync(0xffffffffu, mx, s));
+                for (int it = 0; it < 2; ++it)
+#pragma unroll
+                    for (int j = 0; j < 4; ++j)
+                        raw[it][j] = __ldg(reinterpret_cast<const uint4 *>(v0 + (size_t)(it * 8 + rsub) * row_stride) + j);
+#pragma unroll
+                for (int it = 0; it < 2; ++it) {
+                    float x[32];
+#pragma unroll
+                    for (int j = 0; j < 4; ++j) {
+                        const uint32_t w4[4] = {raw[it][j].x, raw[it][j].y, raw[it][j].z, raw[it][j].w};
+#pragma unroll
+                        for (int h = 0; h < 4; ++h) {
+                            const float2 f = half2_bits_to_float2(w4[h]);
+                            x[j * 8 + h * 2] = f.x;
+                            x[j * 8 + h * 2 + 1] = f.y;
+                        }
                     }
+                    float mn = x[0], mx = x[0];
+#pragma unroll
+                    for (int i = 1; i < 32; ++i) { mn = fminf(mn, x[i]); mx = fmaxf(mx, x[i]); }
                     if (mn == 0.f) mn = 0.f;
                     const __half hd = exact_scale(mx, mn);
                     const float delta = __half2float(hd);
-                    const float inv = (delta == 0.f) ? 0.f : __frcp_rn(delta);
-                    auto code = [&](float v) -> uint32_t {
-                        const float t = __fsub_rn(v, mn);
+                    const float inv = (delta == 0.f) ? 0.f : __frcp_rn(delta);   // scale 0: every code comes out 0
+                    uint32_t q[32];
+#pragma unroll
+                    for (int i = 0; i < 32; ++i) {
+                        const float t = __fsub_rn(x[i], mn);
                         const float q0 = __fmul_rn(t, inv);
                         const float q1 = __fmaf_rn(__fmaf_rn(-q0, delta, t), inv, q0);      // = RN(t / delta)
-                        const float x = fminf(fmaxf(q1, 0.f), 15.f) + 12582912.f;           // round half to even
-                        return (delta == 0.f) ? 0u : (__float_as_uint(x) & 15u);
-                    };
-                    const uint32_t q0 = code(va.x), q1 = code(va.y), q8 = code(vb2.x), q9 = code(vb2.y);
-                    // in-block byte of (token k, channel block cb, row r): see code_byte_off
-                    const int jt = (k & 7) >> 1, byte = (k & 1) * 2 + (k >> 3);
-                    vs[(cb >> 2) * 512 + ((2 * jj) * 4 + jt) * 16 + (cb & 3) * 4 + byte] = (unsigned char)(q0 | (q8 << 4));
-                    vs[(cb >> 2) * 512 + ((2 * jj + 1) * 4 + jt) * 16 + (cb & 3) * 4 + byte] = (unsigned char)(q1 | (q9 << 4));
-                    if ((lane & 7) == 0) {
-                        *reinterpret_cast<__half *>(vs + 1024 + grp * 32 + k * 2) = hd;                    // scale [g][16 tokens]
-                        *reinterpret_cast<__half *>(vs + 1152 + k * 8 + grp * 2) = __float2half_rn(mn);    // zero  [16 tokens][g]
+                        const float y = fminf(fmaxf(q1, 0.f), 15.f) + 12582912.f;           // round half to even
+                        q[i] = __float_as_uint(y) & 15u;
                     }
+                    // token k = it*8 + rsub of the block; in-block byte of (channel block cb, row r): see code_byte_off
+                    const int jt = rsub >> 1, bytepos = (rsub & 1) * 2 + it;
+#pragma unroll
+                    for (int cbl = 0; cbl < 2; ++cbl) {
+                        const int cb = 2 * grp + cbl;
+                        unsigned char *dstb = vs + (cb >> 2) * 512 + jt * 16 + (cb & 3) * 4 + bytepos;
+#pragma unroll
+                        for (int r = 0; r < 8; ++r) dstb[r * 64] = (unsigned char)(q[cbl * 16 + r] | (q[cbl * 16 + r + 8] << 4));
+                    }
+                    const int k = it * 8 + rsub;
+                    *reinterpret_cast<__half *>(vs + 1024 + grp * 32 + k * 2) = hd;                     // scale [g][16 tokens]
+                    *reinterpret_cast<__half *>(vs + 1152 + k * 8 + grp * 2) = __float2half_rn(mn);     // zero  [16 tokens][g]
                 }
                 __syncwarp();
                 const uint4 *src = reinterpret_cast<const uint4 *>(vs);
