@@ -282,10 +282,8 @@ __global__ void __launch_bounds__(kPrefillThreads, 2) prefill_kernel(PrefillPara
         }
     }
     const int first_tile = len0 / kPrefillTile + tg * p.tiles_per_block;
-    for (int ti = 0; ti < p.tiles_per_block; ++ti) {
-        const int P0 = (first_tile + ti) * kPrefillTile;
-        if (P0 >= len0 + n_new) break;                          // block-uniform
-        // ---- key tile: row r = position P0 + r, chunk c at c ^ (r & 7); rows outside the appended range are zero
+    // key tile: row r = position P0 + r, chunk c at c ^ (r & 7); rows outside the appended range are zero
+    auto load_key_tile = [&](int P0) {
         for (int e = tid; e < kPrefillTile * 16; e += kPrefillThreads) {
             const int c = e & 15, r = e >> 4;
             const int tn = P0 + r - len0;
@@ -293,6 +291,11 @@ __global__ void __launch_bounds__(kPrefillThreads, 2) prefill_kernel(PrefillPara
             const uint16_t *src = p.k + ((((size_t)ll * p.B + b) * p.Tn + (ok ? tn : 0)) * p.Hkv + kvh) * kHeadDim + c * 8;
             cp_async_16(smem_addr(As + (size_t)r * 256 + ((c ^ (r & 7)) << 4)), src, ok ? 16u : 0u);
         }
+    };
+    for (int ti = 0; ti < p.tiles_per_block; ++ti) {
+        const int P0 = (first_tile + ti) * kPrefillTile;
+        if (P0 >= len0 + n_new) break;                          // block-uniform
+        if (ti == 0) load_key_tile(P0);                         // later tiles were requested during the previous one
         cp_async_wait_all();
         __syncthreads();
 
@@ -321,6 +324,10 @@ __global__ void __launch_bounds__(kPrefillThreads, 2) prefill_kernel(PrefillPara
                 }
             }
         }
+        // every warp is done reading the key tile: request the next one now, so that its latency hides behind
+        // the sign packing and the value quantisation below
+        __syncthreads();
+        if (ti + 1 < p.tiles_per_block && P0 + kPrefillTile < len0 + n_new) load_key_tile(P0 + kPrefillTile);
         // ---- signs -> words. Thread (g = lane/4, jq = lane%4) holds rows g, g+8 and columns nt*8 + 2jq, +1.
         {
             constexpr int NW = NBC / 32;                        // words per row in this column block
@@ -430,7 +437,6 @@ __global__ void __launch_bounds__(kPrefillThreads, 2) prefill_kernel(PrefillPara
                 }
             }
         }
-        __syncthreads();                                        // the key tile is overwritten by the next iteration
     }
     cp_async_wait_all();
     // ---- the last block to finish publishes the new lengths
