@@ -126,20 +126,23 @@ def run_ours(args):
     torch.cuda.set_device(local)
     pdist.init("nccl", torch.device("cuda", local))
     dev = torch.device("cuda", local)
-    w = h1b_synth.WORKLOADS["c2_7b_8k"]
+    w = h1b_synth.WORKLOADS[args.workload]
+    if args.workload == "c5_prefill":
+        return run_prefill(args, w, pdist, rank, world, local)
     steps, warmup = args.steps, args.warmup
     total_steps = 2 * (steps + warmup) + 8           # device-resident run, then the host-buffer run
-    prefill = w.context - 1                           # the first step decodes exactly `context` tokens
+    lens0 = h1b_synth.lengths(w) - 1                  # the first step decodes exactly the workload's context
     cfg = binding.make_config(w.n_layers, w.n_q_heads, w.n_kv_heads, w.head_dim, w.sketch_bits, w.group_size,
-                              max_batch=w.batch, max_seq=prefill + total_steps, device=local)
+                              max_batch=w.batch, max_seq=w.context - 1 + total_steps, device=local)
     # each rank is its own sequence: different seeds per rank
     wr = h1b_synth.scaled(w, index=w.index + 10 * rank)
     Rt = np.stack([h1b_synth.projection(h1b_synth.layer_seed(wr, l, 99), w.head_dim, w.sketch_bits)
                    for l in range(w.n_layers)])
     cache = binding.H1BCache(cfg, Rt=Rt)
     for l in range(w.n_layers):                       # prefill, one layer at a time
-        K, V = h1b_synth.kv_rows(wr, l, prefill, device=str(dev))
-        cache.h1b_append_kv(K.unsqueeze(0), V.unsqueeze(0), layer_begin=l)
+        K, V = h1b_synth.kv_rows(wr, l, w.context - 1, device=str(dev))
+        cache.h1b_append_kv(K.unsqueeze(0), V.unsqueeze(0), layer_begin=l, n_new=lens0)
+        del K, V
     torch.cuda.synchronize()
     # per-step inputs: a pool of new tokens and queries, resident in HBM
     pool = 16
@@ -168,7 +171,8 @@ def run_ours(args):
     sampler = ClockSampler(gpu_index())
     sampler.start()
     ev0, ev1 = torch.cuda.Event(enable_timing=True), torch.cuda.Event(enable_timing=True)
-    ctx_first = int(cache.h1b_get_lengths(0)[0]) + 1
+    len_first = cache.h1b_get_lengths(0)[:w.batch].astype(np.int64) + 1
+    ctx_first = int(len_first.max())
     barrier()
     ev0.record(stream)
     for i in range(steps):
@@ -181,7 +185,8 @@ def run_ours(args):
     kern_ms, kern_n = cache.h1b_read_profile()
     cache.h1b_set_profiling(False)
     cache.h1b_poll_status()
-    ctx_last = int(cache.h1b_get_lengths(0)[0])
+    len_last = cache.h1b_get_lengths(0)[:w.batch].astype(np.int64)
+    ctx_last = int(len_last.max())
 
     # end to end through the host-buffer entry point: pinned host inputs, H2D and D2H inside the timed region
     kh = [t.cpu().pin_memory() for t in kn]
@@ -206,9 +211,9 @@ def run_ours(args):
 
     # roofline of the dominant kernel (split-K decode attention), per launch
     entry = binding.h1b_entry_bytes(cfg)
-    ctx_mean = 0.5 * (ctx_first + ctx_last)
-    slabs = w.n_layers * w.batch * w.n_kv_heads
-    alg_bytes = slabs * ctx_mean * entry + w.n_layers * w.batch * w.n_q_heads * (w.sketch_bits // 8)
+    tokens_mean = float((0.5 * (len_first + len_last)).sum())         # cached tokens over the batch, mean over the run
+    token_heads = w.n_layers * w.n_kv_heads * tokens_mean
+    alg_bytes = token_heads * entry + w.n_layers * w.batch * w.n_q_heads * (w.sketch_bits // 8)
     peak, peak_kind = measured_peaks()
     kern_ms_avg = kern_ms / max(kern_n, 1)
     achieved = alg_bytes / (kern_ms_avg * 1e-3) / 1e9 if kern_n else None
@@ -224,10 +229,12 @@ def run_ours(args):
         "metric": METRIC, "value": value, "unit": UNIT, "n_gpus": world, "steps": steps, "warmup": warmup,
         "ms_per_step": ms_per_step, "higher_is_better": True, "scaling": "weak", "vs_baseline": None,
         "dtype": "f32", "data": "synthetic",
-        "config": {"workload": "c2_7b_8k: 32 layers x 32 heads, d=128, m=128, batch 1 per GPU, fp16 K/V ~ N(0,1) with 1% "
-                               "outlier channels x8, one projection per layer",
+        "config": {"workload": "%s: %d layers x %d/%d heads, d=%d, m=%d, batch %d per GPU, %s; fp16 K/V ~ N(0,1)%s, one "
+                               "projection per layer" % (w.name, w.n_layers, w.n_q_heads, w.n_kv_heads, w.head_dim,
+                                                         w.sketch_bits, w.batch, w.notes,
+                                                         " with 1% outlier channels x8" if w.outlier_frac else ""),
                    "ctx_first": ctx_first, "ctx_last": ctx_last, "inv_tau": INV_TAU,
-                   "cache_bytes": int(slabs * ctx_mean * entry),
+                   "cache_bytes": int(token_heads * entry),
                    "l2": "working set (%.0f MB per step) is larger than L2; nothing is flushed" % (alg_bytes / 1e6)},
         "e2e": {"value": e2e_value, "unit": UNIT, "ms_per_step": e2e_ms_total / steps,
                 "h2d_bytes_per_step": int(sum(x[0].numel() * 2 for x in (kh, vh, qh))),
@@ -236,8 +243,53 @@ def run_ours(args):
         "clocks": clocks,
         "roofline": roofline,
     }
-    if rank == 0 and world == 1 and not args.no_cpu_baseline:
+    if rank == 0 and world == 1 and not args.no_cpu_baseline and args.workload == "c2_7b_8k":
         line["cpu_baseline"] = cpu_baseline(sample_layers=1, steps=5, warmup=1)
+    cache.close()
+    pdist.finish()
+    if rank == 0:
+        print(json.dumps(line))
+
+
+def run_prefill(args, w, pdist, rank, world, local):
+    """c5: a step is the compression of an 8192-token prompt into all layers' caches (h1b_append_kv)."""
+    import torch
+
+    import h1b_synth
+    from paper_2510_05529_b200 import binding
+    dev = torch.device("cuda", local)
+    cfg = binding.make_config(w.n_layers, w.n_q_heads, w.n_kv_heads, w.head_dim, w.sketch_bits, w.group_size,
+                              max_batch=w.batch, max_seq=w.context, device=local)
+    cache = binding.H1BCache(cfg, seed=11 + rank)
+    K = torch.stack([h1b_synth.kv_rows(w, l, w.context, device=str(dev))[0] for l in range(w.n_layers)])
+    V = torch.stack([h1b_synth.kv_rows(w, l, w.context, device=str(dev))[1] for l in range(w.n_layers)])
+    stream = torch.cuda.current_stream()
+    times = []
+    for i in range(args.warmup + args.steps):
+        cache.h1b_reset(-1)                           # synchronous, outside the timed call
+        e0, e1 = torch.cuda.Event(enable_timing=True), torch.cuda.Event(enable_timing=True)
+        pdist.barrier(); torch.cuda.synchronize()
+        e0.record(stream)
+        cache.h1b_append_kv(K, V)
+        e1.record(stream)
+        torch.cuda.synchronize()
+        if i >= args.warmup:
+            times.append(e0.elapsed_time(e1))
+    cache.h1b_poll_status()
+    ms = pdist.max_over_ranks([float(np.mean(times))], dev)[0]
+    rows = w.n_layers * w.batch * w.context * w.n_kv_heads
+    alg_bytes = rows * (2 * w.head_dim * 2 + binding.h1b_entry_bytes(cfg))       # fp16 K and V in, packed entry out
+    peak, peak_kind = measured_peaks()
+    line = {"metric": "prefill compression tokens/s (7B shape, 8192-token prompt into 32 layers' caches)",
+            "value": pdist.whole_job_rate(w.batch * w.context, world, ms * 1e-3), "unit": UNIT, "n_gpus": world,
+            "steps": args.steps, "warmup": args.warmup, "ms_per_step": ms, "higher_is_better": True,
+            "scaling": "weak", "vs_baseline": None, "dtype": "f16 x f16 -> f32 (projection), f32 (quantiser)",
+            "data": "synthetic", "config": {"workload": "%s: %s" % (w.name, w.notes), "l2": "5.1 GB per step, larger than L2"},
+            "gpu_launches": int(args.steps),
+            "roofline": {"bound": "hbm", "kernel": "prefill_kernel", "achieved": alg_bytes / (ms * 1e-3) / 1e9,
+                         "peak": peak, "peak_kind": peak_kind, "unit": "GB/s", "frac": alg_bytes / (ms * 1e-3) / 1e9 / peak,
+                         "alg_bytes_per_launch": alg_bytes, "traffic": None,
+                         "tensor_tflops": rows * 128 * w.sketch_bits * 2 * 2 / (ms * 1e-3) / 1e12}}
     cache.close()
     pdist.finish()
     if rank == 0:
@@ -325,6 +377,9 @@ def main():
     ap.add_argument("--warmup", type=int, default=30)
     ap.add_argument("--impl", default="ours", choices=["ours", "reference"])
     ap.add_argument("--no-cpu-baseline", action="store_true")
+    ap.add_argument("--workload", default="c2_7b_8k",
+                    choices=["c2_7b_8k", "c3_7b_batched", "c4_gqa_32k", "c5_prefill"],
+                    help="default: the configuration the metric is quoted on; the others are reported in DESIGN.md")
     args = ap.parse_args()
     if args.impl == "reference":
         run_reference(args)

@@ -344,6 +344,7 @@ int h1b_append_kv(h1b_ctx *ctx, int layer_begin, int n_layers, const void *k, co
         pp.Rh = at<uint16_t>(ctx, ctx->plan.rh);
         pp.cache = ctx->ws + ctx->plan.cache;
         pp.len = at<int32_t>(ctx, ctx->plan.len);
+        pp.status = at<int32_t>(ctx, ctx->plan.status);
         pp.done = at<int32_t>(ctx, ctx->plan.status) + 4;
         pp.slab_bytes = ctx->plan.slab_bytes;
         pp.layer_begin = layer_begin; pp.n_layers = n_layers; pp.B = B; pp.Tn = Tn;

@@ -26,6 +26,7 @@ namespace h1b {
 // so the fp32 result is within 128 * 2^-24 of the exact projection relative to
 // the sum of absolute terms, and every launch shape gives the same bits.
 // ===========================================================================
+constexpr unsigned long long kWaitLimitNs = 2000000000ull;   // bounded device-side waits: 2 s, then give up
 constexpr int kProjThreads = 128;
 constexpr int kProjRows = 32;
 
@@ -213,28 +214,37 @@ __global__ void __launch_bounds__(kProjThreads) prepare_kernel(AppendParams ap, 
 // Prefill: long appends. One block = up to `tiles_per_block` tiles of 128 consecutive cache positions
 // of ONE slab (layer, sequence, KV head) x one block of up to 128 sketch columns.
 //
-//   Eq. 2 as a dense contraction on the tensor cores: y = K (fp16, exact) x [Rh1 + Rh2], where
+//   Eq. 2 as a dense contraction on the 5th-generation tensor cores: y = K (fp16, exact) x [Rh1 + Rh2]^T, where
 //   Rh1 = fp16(Rt) and Rh2 = fp16(Rt - Rh1): |Rt - Rh1 - Rh2| <= 2^-22 |Rt| (or 2^-25 absolute), so y is within
-//   ~1e-6 * sum|terms| of the exact projection, well inside the 1e-5 sign-boundary window. ldmatrix from
-//   XOR-swizzled shared memory, mma.sync.m16n8k16 fp16 -> fp32; warp w owns rows 16w..16w+15 of the tile.
-//   The signs are packed from the accumulator fragments (2 bits per thread per n-tile, OR-reduced over
-//   the quad) and stored as the tile's key words.
+//   ~1e-6 * sum|terms| of the exact projection, well inside the 1e-5 sign-boundary window. The key tile
+//   (128 rows x 128 channels) and the two transposed pieces (columns x channels) sit in shared memory as
+//   K-major operands with the 128-byte swizzle; ONE thread issues the 16 tcgen05.mma (M = 128, N = columns,
+//   K = 16 each) of a tile into a TMEM accumulator and commits them to an mbarrier; they run while all
+//   warps quantise the tile's values. Four warps then read their 32 accumulator rows with tcgen05.ld
+//   (thread = row) and pack the signs thread-locally into the tile's key words.
 //   Eq. 4: warp w quantises tokens 16w..16w+15 = one 16-token value block: codes are assembled in shared
 //   memory in the block's packed order and written with 16-byte stores. The division (v - min)/scale is
 //   q1 = q0 + (t - q0*scale)*inv with inv = RN(1/scale), q0 = RN(t*inv): correctly rounded (Markstein), i.e.
 //   the same bits as IEEE division; the scale (max-min)/15 -> fp16 is taken in fp32 when that is provably
 //   the correctly rounded result and in fp64 otherwise.
+//   Every wait is bounded; TMEM is allocated once per block and always released before the block exits.
 // ===========================================================================
 constexpr int kPrefillThreads = 256;
 constexpr int kPrefillTile = 128;              // cache positions per tile
 
 template <int NBC>                             // sketch columns per block: 128 or 64
 struct PrefillSmem {
-    static constexpr int kRBytes = 2 * kHeadDim * NBC * 2;          // two fp16 pieces of the projection block
-    static constexpr int kABytes = kPrefillTile * kHeadDim * 2;     // the key tile
+    static constexpr int kRBytes = 2 * NBC * kHeadDim * 2;          // two fp16 pieces of the projection block, [col][channel]
+    static constexpr int kABytes = kPrefillTile * kHeadDim * 2;     // the key tile, [row][channel]
     static constexpr int kVBytes = (kPrefillThreads / 32) * 1280;   // per warp: 1024 B codes + 128 B scale + 128 B zero
-    static constexpr int kTotal = kRBytes + kABytes + kVBytes;
+    static constexpr int kTotal = kRBytes + kABytes + kVBytes + 1024;   // + slack to align the operands to 1024 B
 };
+
+// Byte offset of element (row, k) of a K-major operand tile [rows][128 channels] held as two 64-channel halves,
+// each with rows of 128 bytes and the 128-byte swizzle (16-byte chunk index XOR row % 8).
+__device__ __forceinline__ int kmajor_sw128_off(int rows, int row, int chunk16 /* k / 8 */) {
+    return (chunk16 >> 3) * rows * 128 + row * 128 + (((chunk16 & 7) ^ (row & 7)) << 4);
+}
 
 // fp16((mx - mn) / 15), correctly rounded from the exact quotient.
 __device__ __forceinline__ __half exact_scale(float mx, float mn) {
@@ -255,10 +265,12 @@ __device__ __forceinline__ __half exact_scale(float mx, float mn) {
 template <int NBC>
 __global__ void __launch_bounds__(kPrefillThreads, 2) prefill_kernel(PrefillParams p, NewCounts nn) {
     using SM = PrefillSmem<NBC>;
-    constexpr int NT = NBC / 8;                // n-tiles of 8 columns
-    constexpr int RCH = NBC / 8;               // 16-byte chunks per projection row
-    extern __shared__ __align__(128) unsigned char smem[];
+    extern __shared__ unsigned char smem_unaligned[];
+    unsigned char *smem = smem_unaligned + ((1024u - (smem_addr(smem_unaligned) & 1023u)) & 1023u);
     unsigned char *Rs = smem, *As = smem + SM::kRBytes, *Vs = As + SM::kABytes;
+    __shared__ uint32_t tmem_base_s;
+    __shared__ __align__(8) unsigned long long mma_bar_s;
+    __shared__ int is_last, gave_up;
     const int tid = threadIdx.x, lane = tid & 31, warp = tid >> 5;
     const int m = p.m_words * 32;
     const ChunkLayout cl = chunk_layout(p.m_words);
@@ -271,94 +283,60 @@ __global__ void __launch_bounds__(kPrefillThreads, 2) prefill_kernel(PrefillPara
     const int len0 = p.len[layer * p.max_batch + b];
     const int n_new = nn.v[b];
     unsigned char *slab = p.cache + ((size_t)(layer * p.max_batch + b) * p.Hkv + kvh) * p.slab_bytes;
+    const uint32_t bar = smem_addr(&mma_bar_s);
 
-    // ---- the two fp16 pieces of Rt[:, col0 .. col0+NBC), swizzled: chunk c of row k at c ^ (k & 7)
+    // a block that starts after some other block has given up a wait does nothing (keeps a failure short)
+    if (tid == 0) gave_up = (*reinterpret_cast<volatile const int32_t *>(p.status) != kStatusOk);
+    __syncthreads();
+    const bool skip_all = gave_up != 0;                         // block-uniform
+    if (warp == 0 && !skip_all) tmem_alloc(smem_addr(&tmem_base_s), NBC);    // NBC fp32 accumulator columns x 128 lanes
+    if (tid == 0) { mbar_init(bar, 1); mbar_fence_init(); }
+    // ---- the two fp16 pieces of Rt[:, col0 .. col0+NBC), transposed: operand B[col][channel]
     {
-        const uint16_t *src = p.Rh + (size_t)layer * 2 * kHeadDim * m;
-        for (int e = tid; e < 2 * kHeadDim * RCH; e += kPrefillThreads) {
-            const int c = e % RCH, k = (e / RCH) % kHeadDim, piece = e / (RCH * kHeadDim);
-            cp_async_16(smem_addr(Rs + ((size_t)(piece * kHeadDim + k) * RCH + (c ^ (k & 7))) * 16),
-                        src + ((size_t)piece * kHeadDim + k) * m + col0 + c * 8, 16);
+        const uint16_t *src = p.Rh + ((size_t)layer * 2 * m + col0) * kHeadDim;        // [L][2][m][128]
+        for (int e = tid; e < 2 * NBC * 16; e += kPrefillThreads) {
+            const int c = e & 15, n = (e >> 4) % NBC, piece = e / (16 * NBC);
+            cp_async_16(smem_addr(Rs + piece * (NBC * 256) + kmajor_sw128_off(NBC, n, c)),
+                        src + ((size_t)piece * m + n) * kHeadDim + c * 8, 16);
         }
     }
+    tc_fence_before_sync();
+    __syncthreads();
+    tc_fence_after_sync();
+    const uint32_t tmem_d = skip_all ? 0u : tmem_base_s;
+    const uint32_t idesc = umma_idesc_f16_m128(NBC);
     const int first_tile = len0 / kPrefillTile + tg * p.tiles_per_block;
-    // key tile: row r = position P0 + r, chunk c at c ^ (r & 7); rows outside the appended range are zero
+    // key tile: row r = position P0 + r; rows outside the appended range are zero
     auto load_key_tile = [&](int P0) {
         for (int e = tid; e < kPrefillTile * 16; e += kPrefillThreads) {
             const int c = e & 15, r = e >> 4;
             const int tn = P0 + r - len0;
             const bool ok = tn >= 0 && tn < n_new;
             const uint16_t *src = p.k + ((((size_t)ll * p.B + b) * p.Tn + (ok ? tn : 0)) * p.Hkv + kvh) * kHeadDim + c * 8;
-            cp_async_16(smem_addr(As + (size_t)r * 256 + ((c ^ (r & 7)) << 4)), src, ok ? 16u : 0u);
+            cp_async_16(smem_addr(As + kmajor_sw128_off(kPrefillTile, r, c)), src, ok ? 16u : 0u);
         }
     };
-    for (int ti = 0; ti < p.tiles_per_block; ++ti) {
+    uint32_t parity = 0;
+    for (int ti = 0; ti < p.tiles_per_block && !skip_all; ++ti) {
         const int P0 = (first_tile + ti) * kPrefillTile;
         if (P0 >= len0 + n_new) break;                          // block-uniform
-        if (ti == 0) load_key_tile(P0);                         // later tiles were requested during the previous one
+        load_key_tile(P0);
         cp_async_wait_all();
+        fence_proxy_async_smem();                               // generic-proxy writes -> visible to the tensor cores
         __syncthreads();
-
-        // ---- y = K x (Rh1 + Rh2): warp w, rows 16w..16w+15, all NBC columns
-        float acc[NT][4];
+        // ---- y = K x (Rh1 + Rh2)^T: one thread issues 2 pieces x 8 K-slices of 16
+        if (tid == 0) {
+            tc_fence_after_sync();
+            const uint32_t a_base = smem_addr(As), r_base = smem_addr(Rs);
 #pragma unroll
-        for (int nt = 0; nt < NT; ++nt) { acc[nt][0] = 0.f; acc[nt][1] = 0.f; acc[nt][2] = 0.f; acc[nt][3] = 0.f; }
-        const uint32_t a_base = smem_addr(As), r_base = smem_addr(Rs);
-        const int lrow = (lane & 7) + ((lane >> 3) & 1) * 8, lhalf = lane >> 4;     // ldmatrix row / second-8 selector
+            for (int piece = 0; piece < 2; ++piece)
 #pragma unroll
-        for (int ks = 0; ks < kHeadDim / 16; ++ks) {
-            uint32_t a[4];
-            {
-                const int r = warp * 16 + lrow, c = ks * 2 + lhalf;
-                ldmatrix_x4(a, a_base + r * 256 + ((c ^ (r & 7)) << 4));
-            }
-#pragma unroll
-            for (int piece = 0; piece < 2; ++piece) {
-#pragma unroll
-                for (int np = 0; np < NT / 2; ++np) {           // two n-tiles per ldmatrix
-                    uint32_t bq[4];
-                    const int k = ks * 16 + lrow, c = np * 2 + lhalf;
-                    ldmatrix_x4_trans(bq, r_base + ((piece * kHeadDim + k) * RCH + (c ^ (k & 7))) * 16);
-                    mma_f16_16816(acc[2 * np], a[0], a[1], a[2], a[3], bq[0], bq[1]);
-                    mma_f16_16816(acc[2 * np + 1], a[0], a[1], a[2], a[3], bq[2], bq[3]);
+                for (int ks = 0; ks < kHeadDim / 16; ++ks) {
+                    const uint64_t ad = umma_desc_k_sw128(a_base + (ks >> 2) * (kPrefillTile * 128) + (ks & 3) * 32);
+                    const uint64_t bd = umma_desc_k_sw128(r_base + piece * (NBC * 256) + (ks >> 2) * (NBC * 128) + (ks & 3) * 32);
+                    umma_f16(tmem_d, ad, bd, idesc, (piece | ks) ? 1u : 0u);
                 }
-            }
-        }
-        // every warp is done reading the key tile: request the next one now, so that its latency hides behind
-        // the sign packing and the value quantisation below
-        __syncthreads();
-        if (ti + 1 < p.tiles_per_block && P0 + kPrefillTile < len0 + n_new) load_key_tile(P0 + kPrefillTile);
-        // ---- signs -> words. Thread (g = lane/4, jq = lane%4) holds rows g, g+8 and columns nt*8 + 2jq, +1.
-        {
-            constexpr int NW = NBC / 32;                        // words per row in this column block
-            uint32_t w_lo[NW], w_hi[NW];
-#pragma unroll
-            for (int w = 0; w < NW; ++w) { w_lo[w] = 0; w_hi[w] = 0; }
-            const int jq = lane & 3, g = lane >> 2;
-#pragma unroll
-            for (int nt = 0; nt < NT; ++nt) {
-                const int sh = (nt & 3) * 8 + 2 * jq;
-                w_lo[nt >> 2] |= ((acc[nt][0] >= 0.f ? 1u : 0u) | (acc[nt][1] >= 0.f ? 2u : 0u)) << sh;
-                w_hi[nt >> 2] |= ((acc[nt][2] >= 0.f ? 1u : 0u) | (acc[nt][3] >= 0.f ? 2u : 0u)) << sh;
-            }
-#pragma unroll
-            for (int w = 0; w < NW; ++w) {
-                w_lo[w] |= __shfl_xor_sync(0xffffffffu, w_lo[w], 1); w_lo[w] |= __shfl_xor_sync(0xffffffffu, w_lo[w], 2);
-                w_hi[w] |= __shfl_xor_sync(0xffffffffu, w_hi[w], 1); w_hi[w] |= __shfl_xor_sync(0xffffffffu, w_hi[w], 2);
-            }
-            // quad lane jq stores word jq (and jq + 4, ... when there are more than four)
-#pragma unroll
-            for (int w = 0; w < NW; ++w) {
-                if ((w & 3) == jq) {
-#pragma unroll
-                    for (int hi = 0; hi < 2; ++hi) {
-                        const int pos = P0 + warp * 16 + g + hi * 8, tn = pos - len0;
-                        if (tn >= 0 && tn < n_new)
-                            *reinterpret_cast<uint32_t *>(slab + (size_t)(pos >> 5) * cl.bytes +
-                                                          key_word_off(col0 / 32 + w, pos & 31)) = hi ? w_hi[w] : w_lo[w];
-                    }
-                }
-            }
+            umma_commit(bar);
         }
         // ---- values: warp w quantises tokens P0 + 16w .. +15 (one value block); only the first column block does it
         if (blockIdx.y == 0) {
@@ -437,11 +415,37 @@ __global__ void __launch_bounds__(kPrefillThreads, 2) prefill_kernel(PrefillPara
                 }
             }
         }
+        // ---- signs: warps 0-3 read the accumulator (thread = row 32*warp + lane of the tile)
+        if (warp < 4) {
+            const bool done = mbar_wait_bounded(bar, parity, kWaitLimitNs);
+            tc_fence_after_sync();
+            if (done) {
+                const int pos = P0 + warp * 32 + lane, tn = pos - len0;
+                unsigned char *kw = slab + (size_t)(pos >> 5) * cl.bytes + (pos & 31) * 4;
+#pragma unroll
+                for (int w = 0; w < NBC / 32; ++w) {
+                    uint32_t y[32];
+                    tmem_ld_32cols(tmem_d + ((uint32_t)(warp * 32) << 16) + w * 32, y);
+                    uint32_t word = 0;
+#pragma unroll
+                    for (int j = 0; j < 32; ++j) word |= (__uint_as_float(y[j]) >= 0.f ? 1u : 0u) << j;
+                    if (tn >= 0 && tn < n_new) *reinterpret_cast<uint32_t *>(kw + (col0 / 32 + w) * 128) = word;
+                }
+            } else if (lane == 0) {
+                atomicExch(p.status, kStatusWaitTimeout);
+                gave_up = 1;
+            }
+            tc_fence_before_sync();
+        }
+        parity ^= 1;
+        __syncthreads();                                        // the key tile and the accumulator are free again
+        if (gave_up) break;
     }
     cp_async_wait_all();
-    // ---- the last block to finish publishes the new lengths
-    __shared__ int is_last;
+    tc_fence_before_sync();
     __syncthreads();
+    if (warp == 0 && !skip_all) { tc_fence_after_sync(); tmem_dealloc(tmem_d, NBC); }
+    // ---- the last block to finish publishes the new lengths
     if (tid == 0) {
         __threadfence();
         is_last = (atomicAdd(p.done, 1) == (int)(gridDim.x * gridDim.y) - 1);
@@ -454,17 +458,18 @@ __global__ void __launch_bounds__(kPrefillThreads, 2) prefill_kernel(PrefillPara
     }
 }
 
-// Rt (fp32) -> its two fp16 pieces, [L][2][d][m].
+// Rt (fp32, [L][d][m]) -> its two fp16 pieces, transposed to [L][2][m][d] (channel contiguous).
 __global__ void split_projection_kernel(const float *Rt, uint16_t *Rh, int n_layers, int m) {
     const long n = (long)n_layers * kHeadDim * m;
     for (long e = (long)blockIdx.x * blockDim.x + threadIdx.x; e < n; e += (long)gridDim.x * blockDim.x) {
-        const long l = e / ((long)kHeadDim * m), rest = e % ((long)kHeadDim * m);
+        const long l = e / ((long)kHeadDim * m);
+        const int i = (int)((e / m) % kHeadDim), j = (int)(e % m);
         const float r = Rt[e];
         const __half h1 = __float2half_rn(r);
         const __half h2 = __float2half_rn(r - __half2float(h1));
         __half *dst = reinterpret_cast<__half *>(Rh) + l * 2 * kHeadDim * m;
-        dst[rest] = h1;
-        dst[(long)kHeadDim * m + rest] = h2;
+        dst[(long)j * kHeadDim + i] = h1;
+        dst[(long)(m + j) * kHeadDim + i] = h2;
     }
 }
 
@@ -503,7 +508,6 @@ constexpr int kDecodeWarps = H1B_DECODE_WARPS;
 constexpr int kStages = H1B_DECODE_STAGES;
 // Resident blocks per SM that the register allocation must allow: the kernel hides latency with warps.
 constexpr int decode_min_blocks(int gq) { return gq == 1 ? 5 : (gq == 2 ? 4 : 3); }
-constexpr unsigned long long kWaitLimitNs = 2000000000ull;   // 2 s, then give up
 constexpr int kHamSentinel = 1 << 20;
 
 template <int MW, int GQ>

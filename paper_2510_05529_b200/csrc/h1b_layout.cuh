@@ -91,9 +91,10 @@ struct AppendParams {
 
 struct PrefillParams {          // long appends: tensor-core projection
     const uint16_t *k, *v;      // fp16 [n_layers][B][Tn][Hkv][d]
-    const uint16_t *Rh;         // fp16 [L][2][d][m]: Rt split exactly-enough as fp16(Rt) + fp16(Rt - fp16(Rt))
+    const uint16_t *Rh;         // fp16 [L][2][m][d]: Rt^T split as fp16(Rt) + fp16(Rt - fp16(Rt))
     unsigned char *cache;
     int32_t *len;               // [L][max_batch]
+    int32_t *status;            // device status word (bounded-wait timeouts)
     int32_t *done;              // block counter (zero between launches)
     size_t slab_bytes;
     int layer_begin, n_layers, B, Tn, Hkv, max_batch, m_words;
