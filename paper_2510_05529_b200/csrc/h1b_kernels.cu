@@ -320,7 +320,7 @@ __global__ void __launch_bounds__(kPrefillThreads, 2) prefill_kernel(PrefillPara
     for (int ti = 0; ti < p.tiles_per_block && !skip_all; ++ti) {
         const int P0 = (first_tile + ti) * kPrefillTile;
         if (P0 >= len0 + n_new) break;                          // block-uniform
-        load_key_tile(P0);
+        if (ti == 0) load_key_tile(P0);                         // later tiles were requested during the previous one
         cp_async_wait_all();
         fence_proxy_async_smem();                               // generic-proxy writes -> visible to the tensor cores
         __syncthreads();
@@ -419,6 +419,18 @@ __global__ void __launch_bounds__(kPrefillThreads, 2) prefill_kernel(PrefillPara
         if (warp < 4) {
             const bool done = mbar_wait_bounded(bar, parity, kWaitLimitNs);
             tc_fence_after_sync();
+            // the tensor cores are done with the key tile: these four warps request the next one right away, so
+            // that its latency hides behind the sign packing and the rest of the value quantisation
+            if (done && ti + 1 < p.tiles_per_block && P0 + kPrefillTile < len0 + n_new) {
+                const int Pn = P0 + kPrefillTile;
+                for (int e = tid; e < kPrefillTile * 16; e += 128) {
+                    const int c = e & 15, r = e >> 4;
+                    const int tnn = Pn + r - len0;
+                    const bool ok = tnn >= 0 && tnn < n_new;
+                    const uint16_t *src = p.k + ((((size_t)ll * p.B + b) * p.Tn + (ok ? tnn : 0)) * p.Hkv + kvh) * kHeadDim + c * 8;
+                    cp_async_16(smem_addr(As + kmajor_sw128_off(kPrefillTile, r, c)), src, ok ? 16u : 0u);
+                }
+            }
             if (done) {
                 const int pos = P0 + warp * 32 + lane, tn = pos - len0;
                 unsigned char *kw = slab + (size_t)(pos >> 5) * cl.bytes + (pos & 31) * 4;
