@@ -415,15 +415,16 @@ __global__ void __launch_bounds__(kPrefillThreads, 2) prefill_kernel(PrefillPara
                 }
             }
         }
-        // ---- signs: warps 0-3 read the accumulator (thread = row 32*warp + lane of the tile)
-        if (warp < 4) {
+        // ---- signs: thread = accumulator row 32*(warp%4) + lane (a warp can only read the TMEM lanes of its
+        // quarter); warps 0-3 take the lower half of the columns, warps 4-7 the upper half
+        {
             const bool done = mbar_wait_bounded(bar, parity, kWaitLimitNs);
             tc_fence_after_sync();
-            // the tensor cores are done with the key tile: these four warps request the next one right away, so
+            // the tensor cores are done with the key tile: request the next one right away, so
             // that its latency hides behind the sign packing and the rest of the value quantisation
             if (done && ti + 1 < p.tiles_per_block && P0 + kPrefillTile < len0 + n_new) {
                 const int Pn = P0 + kPrefillTile;
-                for (int e = tid; e < kPrefillTile * 16; e += 128) {
+                for (int e = tid; e < kPrefillTile * 16; e += kPrefillThreads) {
                     const int c = e & 15, r = e >> 4;
                     const int tnn = Pn + r - len0;
                     const bool ok = tnn >= 0 && tnn < n_new;
@@ -432,12 +433,14 @@ __global__ void __launch_bounds__(kPrefillThreads, 2) prefill_kernel(PrefillPara
                 }
             }
             if (done) {
-                const int pos = P0 + warp * 32 + lane, tn = pos - len0;
+                const int quarter = warp & 3, whalf = warp >> 2;
+                const int pos = P0 + quarter * 32 + lane, tn = pos - len0;
                 unsigned char *kw = slab + (size_t)(pos >> 5) * cl.bytes + (pos & 31) * 4;
 #pragma unroll
-                for (int w = 0; w < NBC / 32; ++w) {
+                for (int wi = 0; wi < NBC / 64; ++wi) {
+                    const int w = whalf * (NBC / 64) + wi;
                     uint32_t y[32];
-                    tmem_ld_32cols(tmem_d + ((uint32_t)(warp * 32) << 16) + w * 32, y);
+                    tmem_ld_32cols(tmem_d + ((uint32_t)(quarter * 32) << 16) + w * 32, y);
                     uint32_t word = 0;
 #pragma unroll
                     for (int j = 0; j < 32; ++j) word |= (__uint_as_float(y[j]) >= 0.f ? 1u : 0u) << j;
