@@ -137,6 +137,7 @@ __device__ __forceinline__ void quantize_row(const uint16_t *__restrict__ v_row,
 // read them by then).
 __global__ void __launch_bounds__(kProjThreads) prepare_kernel(AppendParams ap, SketchParams sp, NewCounts nn) {
     __shared__ ProjSmem sm;
+    launch_dependents();                                        // the attention grid may be scheduled behind this one
     const bool appending = ap.k != nullptr;
     const int mw = appending ? ap.m_words : sp.m_words, m = mw * 32;
     const ChunkLayout cl = chunk_layout(mw);
@@ -665,6 +666,8 @@ __global__ void __launch_bounds__(kDecodeWarps * 32, decode_min_blocks(GQ)) deco
     const int b = (int)((slab_local / p.Hkv) % p.B);
     const int ll = (int)(slab_local / ((long)p.Hkv * p.B));
     const int layer = p.layer_begin + ll;
+    launch_dependents();                                        // the combine grid may be scheduled behind this one
+    grid_dependency_wait();                                     // lengths, query sketches and the new token come from the prepare kernel
     const int len = p.len[layer * p.max_batch + b];
     const int t_begin = split * p.split_tokens;
     if (t_begin >= len) {                                       // empty item: it is not counted by the combine
@@ -857,6 +860,7 @@ __global__ void __launch_bounds__(kHeadDim) combine_kernel(DecodeParams p) {
     const int hq = blockIdx.x % p.Hq;
     const int b = (blockIdx.x / p.Hq) % p.B;
     const int ll = blockIdx.x / (p.Hq * p.B);
+    grid_dependency_wait();                                     // the partials come from the attention kernel
     const int len = p.len[(p.layer_begin + ll) * p.max_batch + b];
     const int kvh = hq / gq, hh = hq % gq;
     const long slab_local = ((long)ll * p.B + b) * p.Hkv + kvh;
@@ -974,8 +978,17 @@ static cudaError_t launch_decode_t(const DecodeParams &p, cudaStream_t st) {
     }
     const long items = (long)p.n_layers * p.B * p.Hkv * p.splits;
     const unsigned grid = (unsigned)((items + kDecodeWarps - 1) / kDecodeWarps);
-    decode_split_kernel<MW, GQ><<<grid, kDecodeWarps * 32, SM::kTotal, st>>>(p);
-    return cudaGetLastError();
+    cudaLaunchConfig_t cfg = {};
+    cfg.gridDim = dim3(grid);
+    cfg.blockDim = dim3(kDecodeWarps * 32);
+    cfg.dynamicSmemBytes = SM::kTotal;
+    cfg.stream = st;
+    cudaLaunchAttribute attr[1];
+    attr[0].id = cudaLaunchAttributeProgrammaticStreamSerialization;     // may overlap the tail of the prepare kernel
+    attr[0].val.programmaticStreamSerializationAllowed = 1;
+    cfg.attrs = attr;
+    cfg.numAttrs = 1;
+    return cudaLaunchKernelEx(&cfg, decode_split_kernel<MW, GQ>, p);
 }
 
 cudaError_t launch_decode(const DecodeParams &p, cudaStream_t st, int *launches, cudaEvent_t before,
@@ -992,7 +1005,19 @@ cudaError_t launch_decode(const DecodeParams &p, cudaStream_t st, int *launches,
     if (after) cudaEventRecord(after, st);
     ++*launches;
 #ifndef H1B_FUSED_COMBINE
-    combine_kernel<<<p.n_layers * p.B * p.Hq, kHeadDim, 0, st>>>(p);
+    {
+        cudaLaunchConfig_t cfg = {};
+        cfg.gridDim = dim3(p.n_layers * p.B * p.Hq);
+        cfg.blockDim = dim3(kHeadDim);
+        cfg.stream = st;
+        cudaLaunchAttribute attr[1];
+        attr[0].id = cudaLaunchAttributeProgrammaticStreamSerialization; // may overlap the tail of the attention kernel
+        attr[0].val.programmaticStreamSerializationAllowed = 1;
+        cfg.attrs = attr;
+        cfg.numAttrs = 1;
+        cudaError_t ec = cudaLaunchKernelEx(&cfg, combine_kernel, p);
+        if (ec != cudaSuccess) return ec;
+    }
     ++*launches;
 #endif
     return cudaGetLastError();
