@@ -62,7 +62,7 @@ typedef struct {
     int32_t n_kv_heads;    /* Hkv                                                      */
     int32_t head_dim;      /* d: 128                                                   */
     int32_t sketch_bits;   /* m: 64, 128, 256 or 512                                   */
-    int32_t group_size;    /* G: 32                                                    */
+    int32_t group_size;    /* G: 32, or 128 (= d: one scale and zero per value vector)  */
     int32_t max_batch;     /* sequences the cache can hold (<= 256)                    */
     int32_t max_seq;       /* tokens per sequence the cache can hold                   */
     int32_t device;        /* CUDA device ordinal                                      */

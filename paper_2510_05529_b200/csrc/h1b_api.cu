@@ -26,7 +26,7 @@ constexpr int kPrefillMinTokens = 64;   // appends of at least this many tokens 
 struct Plan {
     size_t rt, rh, len, status, arrive, qwords, partial, stage_k, stage_v, stage_q, stage_out, dbg_q, dbg_s, cache, total;
     size_t partial_items, slab_bytes;
-    int cap_tokens, m_words, gq;
+    int cap_tokens, m_words, gq, groups;
 };
 
 size_t align_up(size_t x, size_t a) { return (x + a - 1) / a * a; }
@@ -41,7 +41,7 @@ int check_config(const h1b_config *c) {
     if (c->max_batch > 256) return H1B_ERR_INVALID_ARG;
     const int gq = c->n_q_heads / c->n_kv_heads;
     if (gq != 1 && gq != 2 && gq != 4) return H1B_ERR_UNSUPPORTED;
-    if (c->head_dim != kHeadDim || c->group_size != kGroup) return H1B_ERR_UNSUPPORTED;
+    if (c->head_dim != kHeadDim || (c->group_size != kGroup && c->group_size != kHeadDim)) return H1B_ERR_UNSUPPORTED;
     if (c->sketch_bits != 64 && c->sketch_bits != 128 && c->sketch_bits != 256 && c->sketch_bits != 512)
         return H1B_ERR_UNSUPPORTED;
     if ((long)c->n_layers * c->max_batch * c->n_kv_heads > (1L << 28)) return H1B_ERR_INVALID_ARG;
@@ -53,7 +53,8 @@ int make_plan(const h1b_config *c, Plan *p) {
     if (rc != H1B_OK) return rc;
     p->m_words = c->sketch_bits / 32;
     p->gq = c->n_q_heads / c->n_kv_heads;
-    const ChunkLayout cl = chunk_layout(p->m_words);
+    p->groups = c->head_dim / c->group_size;
+    const ChunkLayout cl = chunk_layout(p->m_words, p->groups);
     p->cap_tokens = (c->max_seq + kChunkTokens - 1) / kChunkTokens * kChunkTokens;
     p->slab_bytes = (size_t)(p->cap_tokens / kChunkTokens) * cl.bytes;
     const size_t L = c->n_layers, B = c->max_batch, Hq = c->n_q_heads, Hkv = c->n_kv_heads, d = c->head_dim;
@@ -183,7 +184,7 @@ int h1b_init_projection(const h1b_config *cfg, uint64_t seed, const float *Rt_ho
     if (!ctx) return fail(nullptr, H1B_ERR_INVALID_ARG, "out of host memory");
     ctx->cfg = *cfg;
     ctx->plan = plan;
-    ctx->cl = chunk_layout(plan.m_words);
+    ctx->cl = chunk_layout(plan.m_words, plan.groups);
     ctx->ws = static_cast<unsigned char *>(workspace);
     ctx->len_host.assign((size_t)cfg->n_layers * cfg->max_batch, 0);
     ctx->forced_splits = 0;
@@ -250,6 +251,7 @@ static AppendParams append_params(h1b_ctx *ctx, int layer_begin, int n_layers, c
     p.slab_bytes = ctx->plan.slab_bytes;
     p.layer_begin = layer_begin; p.n_layers = n_layers; p.B = B; p.Tn = Tn;
     p.Hkv = ctx->cfg.n_kv_heads; p.max_batch = ctx->cfg.max_batch; p.m_words = ctx->plan.m_words;
+    p.groups = ctx->plan.groups;
     return p;
 }
 
@@ -304,6 +306,7 @@ static int enqueue_decode(h1b_ctx *ctx, int layer_begin, int n_layers, float inv
     dp.slab_bytes = ctx->plan.slab_bytes;
     dp.layer_begin = layer_begin; dp.n_layers = n_layers; dp.B = B; dp.Hkv = ctx->cfg.n_kv_heads;
     dp.Hq = ctx->cfg.n_q_heads; dp.max_batch = ctx->cfg.max_batch; dp.m_words = ctx->plan.m_words;
+    dp.groups = ctx->plan.groups;
     dp.splits = (int)splits; dp.split_tokens = split_tokens;
     dp.c2 = (float)(2.0 * (double)inv_tau * 1.4426950408889634 / (double)ctx->cfg.sketch_bits);
     cudaEvent_t ev0 = nullptr, ev1 = nullptr;
@@ -349,6 +352,7 @@ int h1b_append_kv(h1b_ctx *ctx, int layer_begin, int n_layers, const void *k, co
         pp.slab_bytes = ctx->plan.slab_bytes;
         pp.layer_begin = layer_begin; pp.n_layers = n_layers; pp.B = B; pp.Tn = Tn;
         pp.Hkv = ctx->cfg.n_kv_heads; pp.max_batch = ctx->cfg.max_batch; pp.m_words = ctx->plan.m_words;
+        pp.groups = ctx->plan.groups;
         int tiles = 1;
         for (int l = layer_begin; l < layer_begin + n_layers; ++l)
             for (int b = 0; b < B; ++b) {
@@ -575,9 +579,9 @@ int h1b_export_cache(h1b_ctx *ctx, int layer, int seq, int kv_head, int t0, int 
                     codes[(size_t)i * d + cb * 16 + r] = byte & 15;
                     codes[(size_t)i * d + cb * 16 + r + 8] = byte >> 4;
                 }
-        for (int g = 0; g < kGroups; ++g) {
-            if (scale) std::memcpy(&scale[(size_t)i * kGroups + g], ch + scale_off(cl, tt, g), 2);
-            if (zero) std::memcpy(&zero[(size_t)i * kGroups + g], ch + zero_off(cl, tt, g), 2);
+        for (int g = 0; g < cl.groups; ++g) {
+            if (scale) std::memcpy(&scale[(size_t)i * cl.groups + g], ch + scale_off(cl, tt, g), 2);
+            if (zero) std::memcpy(&zero[(size_t)i * cl.groups + g], ch + zero_off(cl, tt, g), 2);
         }
     }
     return H1B_OK;
@@ -603,7 +607,7 @@ int h1b_debug_scores(h1b_ctx *ctx, int layer, int seq, int kv_head, const void *
     std::memset(&none, 0, sizeof none);
     H1B_CUDA(ctx, cudaDeviceSynchronize());
     H1B_CUDA(ctx, launch_prepare(nullptr, &sp, none, nullptr, &launches));
-    H1B_CUDA(ctx, launch_debug_scores(slab_ptr(ctx, layer, seq, kv_head), sp.qwords, mw, len,
+    H1B_CUDA(ctx, launch_debug_scores(slab_ptr(ctx, layer, seq, kv_head), sp.qwords, mw, ctx->plan.groups, len,
                                       at<int32_t>(ctx, ctx->plan.dbg_s), nullptr));
     H1B_CUDA(ctx, cudaDeviceSynchronize());
     if (qwords_host)

@@ -99,16 +99,20 @@ __device__ __forceinline__ uint32_t project_tile(ProjSmem &sm, const uint16_t *_
 __device__ __forceinline__ void quantize_row(const uint16_t *__restrict__ v_row, unsigned char *chunk,
                                              const ChunkLayout &cl, int tt, int lane) {
     // lane -> channel block cb = lane/4 and the channel pairs (2jj, 2jj+1), (2jj+8, 2jj+9)
-    const int cb = lane >> 2, jj = lane & 3, g = lane >> 3;
+    const int cb = lane >> 2, jj = lane & 3;
+    const int span = cl.groups == 4 ? 8 : 32;                 // lanes that share one scale/zero
+    const int g = cl.groups == 4 ? (lane >> 3) : 0;
     const __half2 *vrow = reinterpret_cast<const __half2 *>(v_row);
     const float2 va = __half22float2(vrow[(cb * 16 + 2 * jj) >> 1]);
     const float2 vb = __half22float2(vrow[(cb * 16 + 2 * jj + 8) >> 1]);
     float mn = fminf(fminf(va.x, va.y), fminf(vb.x, vb.y));
     float mx = fmaxf(fmaxf(va.x, va.y), fmaxf(vb.x, vb.y));
 #pragma unroll
-    for (int s = 1; s < 8; s <<= 1) {
-        mn = fminf(mn, __shfl_xor_sync(0xffffffffu, mn, s));
-        mx = fmaxf(mx, __shfl_xor_sync(0xffffffffu, mx, s));
+    for (int s = 1; s < 32; s <<= 1) {
+        if (s < span) {
+            mn = fminf(mn, __shfl_xor_sync(0xffffffffu, mn, s));
+            mx = fmaxf(mx, __shfl_xor_sync(0xffffffffu, mx, s));
+        }
     }
     if (mn == 0.f) mn = 0.f;                                  // one spelling of zero
     // (max - min)/15 in fp64, rounded once to fp16: identical to the definition.
@@ -123,7 +127,7 @@ __device__ __forceinline__ void quantize_row(const uint16_t *__restrict__ v_row,
     const uint32_t q0 = code(va.x), q1 = code(va.y), q8 = code(vb.x), q9 = code(vb.y);
     chunk[code_byte_off(cl, tt, cb, 2 * jj)] = (unsigned char)(q0 | (q8 << 4));
     chunk[code_byte_off(cl, tt, cb, 2 * jj + 1)] = (unsigned char)(q1 | (q9 << 4));
-    if ((lane & 7) == 0) {
+    if ((lane & (span - 1)) == 0) {
         *reinterpret_cast<__half *>(chunk + scale_off(cl, tt, g)) = hd;
         *reinterpret_cast<__half *>(chunk + zero_off(cl, tt, g)) = __float2half_rn(mn);
     }
@@ -140,7 +144,7 @@ __global__ void __launch_bounds__(kProjThreads) prepare_kernel(AppendParams ap, 
     launch_dependents();                                        // the attention grid may be scheduled behind this one
     const bool appending = ap.k != nullptr;
     const int mw = appending ? ap.m_words : sp.m_words, m = mw * 32;
-    const ChunkLayout cl = chunk_layout(mw);
+    const ChunkLayout cl = chunk_layout(mw, appending ? ap.groups : kGroups);
     const int k_rows = appending ? ap.B * ap.Tn * ap.Hkv : 0;           // per layer
     const int k_tiles = (k_rows + kProjRows - 1) / kProjRows;
     const int k_blocks = appending ? ap.n_layers * k_tiles * mw : 0;
@@ -274,7 +278,7 @@ __global__ void __launch_bounds__(kPrefillThreads, 2) prefill_kernel(PrefillPara
     __shared__ int is_last, gave_up;
     const int tid = threadIdx.x, lane = tid & 31, warp = tid >> 5;
     const int m = p.m_words * 32;
-    const ChunkLayout cl = chunk_layout(p.m_words);
+    const ChunkLayout cl = chunk_layout(p.m_words, p.groups);
     const int groups_per_slab = (p.tiles_per_seq + p.tiles_per_block - 1) / p.tiles_per_block;
     const int tg = blockIdx.x % groups_per_slab;
     const long slab_local = blockIdx.x / groups_per_slab;
@@ -373,6 +377,10 @@ __global__ void __launch_bounds__(kPrefillThreads, 2) prefill_kernel(PrefillPara
                     float mn = x[0], mx = x[0];
 #pragma unroll
                     for (int i = 1; i < 32; ++i) { mn = fminf(mn, x[i]); mx = fmaxf(mx, x[i]); }
+                    if (p.groups == 1) {                        // one scale per vector: the row's four lanes agree
+                        mn = fminf(mn, __shfl_xor_sync(0xffffffffu, mn, 1)); mx = fmaxf(mx, __shfl_xor_sync(0xffffffffu, mx, 1));
+                        mn = fminf(mn, __shfl_xor_sync(0xffffffffu, mn, 2)); mx = fmaxf(mx, __shfl_xor_sync(0xffffffffu, mx, 2));
+                    }
                     if (mn == 0.f) mn = 0.f;
                     const __half hd = exact_scale(mx, mn);
                     const float delta = __half2float(hd);
@@ -396,16 +404,21 @@ __global__ void __launch_bounds__(kPrefillThreads, 2) prefill_kernel(PrefillPara
                         for (int r = 0; r < 8; ++r) dstb[r * 64] = (unsigned char)(q[cbl * 16 + r] | (q[cbl * 16 + r + 8] << 4));
                     }
                     const int k = it * 8 + rsub;
-                    *reinterpret_cast<__half *>(vs + 1024 + grp * 32 + k * 2) = hd;                     // scale [g][16 tokens]
-                    *reinterpret_cast<__half *>(vs + 1152 + k * 8 + grp * 2) = __float2half_rn(mn);     // zero  [16 tokens][g]
+                    if (p.groups == 4 || grp == 0) {
+                        const int gs = p.groups == 4 ? grp : 0;
+                        *reinterpret_cast<__half *>(vs + 1024 + gs * 32 + k * 2) = hd;                              // scale [g][16 tokens]
+                        *reinterpret_cast<__half *>(vs + 1152 + k * (2 * p.groups) + gs * 2) = __float2half_rn(mn); // zero  [16 tokens][g]
+                    }
                 }
                 __syncwarp();
                 const uint4 *src = reinterpret_cast<const uint4 *>(vs);
                 uint4 *dst = reinterpret_cast<uint4 *>(chunk + cl.val_off + vb * kValBlockBytes);
                 dst[lane] = src[lane];
                 dst[32 + lane] = src[32 + lane];
-                if (lane < 8) reinterpret_cast<uint4 *>(chunk + cl.scale_off + vb * 128)[lane] = src[64 + lane];
-                else if (lane < 16) reinterpret_cast<uint4 *>(chunk + cl.zero_off + vb * 128)[lane - 8] = src[72 + lane - 8];
+                const int n16 = 2 * p.groups;                   // 16-byte pieces of a block's scale (and zero) plane
+                if (lane < n16) reinterpret_cast<uint4 *>(chunk + cl.scale_off + vb * (32 * p.groups))[lane] = src[64 + lane];
+                else if (lane >= 8 && lane < 8 + n16)
+                    reinterpret_cast<uint4 *>(chunk + cl.zero_off + vb * (32 * p.groups))[lane - 8] = src[72 + lane - 8];
                 __syncwarp();
             } else {                                            // ragged edge of the appended range: row by row
                 for (int k = 0; k < 16; ++k) {
@@ -526,30 +539,30 @@ constexpr int kStages = H1B_DECODE_STAGES;
 constexpr int decode_min_blocks(int gq) { return gq == 1 ? 5 : (gq == 2 ? 4 : 3); }
 constexpr int kHamSentinel = 1 << 20;
 
-template <int MW, int GQ>
+template <int MW, int GQ, int NG>                 // NG: scale/zero pairs per value vector (4 or 1)
 struct DecodeSmem {
-    static constexpr int kChunkBytes = MW * 128 + 2560;
+    static constexpr int kChunkBytes = MW * 128 + 2048 + 128 * NG;
     static constexpr int kPerWarp = kStages * kChunkBytes + GQ * 32 * 4 + 128;   // ring, p buffer, barriers
     static constexpr int kTotal = kDecodeWarps * kPerWarp;
 };
 
-template <int MW, int GQ>
+template <int MW, int GQ, int NG>
 struct DecodeState {
     float acc[8][4];            // per channel block of 16: C fragment (rows r, r+8; columns 2jq, 2jq+1)
     int hmin[GQ];               // running minimum Hamming distance (= running maximum logit)
     float ssum[GQ];             // per-lane partial sum of the weights
-    float accz[GQ][kGroups];    // per-lane partial sum of p * zero
+    float accz[GQ][NG];         // per-lane partial sum of p * zero
     uint32_t qw[GQ][MW];        // query sketches
     float zero[4];              // an opaque quad of zeros: C operand of each chunk's first MMA
 };
 
 // One chunk. TAIL: tokens at or beyond t_end are masked (only the last chunk of a split needs it).
-template <int MW, int GQ, bool TAIL>
-__device__ __forceinline__ void decode_chunk(DecodeState<MW, GQ> &st, const unsigned char *ch, float *p_s,
+template <int MW, int GQ, int NG, bool TAIL>
+__device__ __forceinline__ void decode_chunk(DecodeState<MW, GQ, NG> &st, const unsigned char *ch, float *p_s,
                                              int lane, int n_valid, float c2) {
-    constexpr int NG = 4 / GQ;                 // value groups covered by one B fragment
-    constexpr int NB = GQ;                     // B fragments per 16-token block
-    constexpr int VAL = MW * 128, ZERO = VAL + 2048, SCALE = ZERO + 256;
+    constexpr int GPF = 4 / GQ;                // value groups covered by one B fragment (4 groups per vector)
+    constexpr int NB = (NG == 1) ? 1 : GQ;     // B fragments per 16-token block (one scale per vector: one fragment)
+    constexpr int VAL = MW * 128, ZERO = VAL + 2048, SCALE = ZERO + 64 * NG;
     const int jq = lane & 3;
 
     // ---------------- phase 1
@@ -557,8 +570,14 @@ __device__ __forceinline__ void decode_chunk(DecodeState<MW, GQ> &st, const unsi
     uint32_t kw[MW];
 #pragma unroll
     for (int w = 0; w < MW; ++w) kw[w] = *reinterpret_cast<const uint32_t *>(ch + w * 128 + lane * 4);
-    const uint2 zraw = *reinterpret_cast<const uint2 *>(ch + ZERO + lane * 8);
-    const float2 z01 = half2_bits_to_float2(zraw.x), z23 = half2_bits_to_float2(zraw.y);
+    float zf[NG];
+    if (NG == 4) {
+        const uint2 zraw = *reinterpret_cast<const uint2 *>(ch + ZERO + lane * 8);
+        const float2 z01 = half2_bits_to_float2(zraw.x), z23 = half2_bits_to_float2(zraw.y);
+        zf[0] = z01.x; zf[NG > 1 ? 1 : 0] = z01.y; zf[NG > 2 ? 2 : 0] = z23.x; zf[NG > 3 ? 3 : 0] = z23.y;
+    } else {
+        zf[0] = __half2float(*reinterpret_cast<const __half *>(ch + ZERO + lane * 2));
+    }
     float scl[GQ];
 #pragma unroll
     for (int h = 0; h < GQ; ++h) {
@@ -572,16 +591,14 @@ __device__ __forceinline__ void decode_chunk(DecodeState<MW, GQ> &st, const unsi
             st.hmin[h] = cmin;
             st.ssum[h] *= scl[h];                           // rescale what predates this chunk
 #pragma unroll
-            for (int g = 0; g < kGroups; ++g) st.accz[h][g] *= scl[h];
+            for (int g = 0; g < NG; ++g) st.accz[h][g] *= scl[h];
         }
         // p carries the static factor 2 of the weights (removed when the partial is written)
         float pv = ex2_approx(fmaf((float)(st.hmin[h] - ham), c2, 1.f));
         if (TAIL) pv = valid ? pv : 0.f;
         st.ssum[h] += pv;
-        st.accz[h][0] = fmaf(pv, z01.x, st.accz[h][0]);
-        st.accz[h][1] = fmaf(pv, z01.y, st.accz[h][1]);
-        st.accz[h][2] = fmaf(pv, z23.x, st.accz[h][2]);
-        st.accz[h][3] = fmaf(pv, z23.y, st.accz[h][3]);
+#pragma unroll
+        for (int g = 0; g < NG; ++g) st.accz[h][g] = fmaf(pv, zf[g], st.accz[h][g]);
         p_s[h * 32 + lane] = pv;
     }
     // factors by which this lane's accumulator columns 2jq, 2jq+1 shrink when a running max moved (else 1)
@@ -605,9 +622,9 @@ __device__ __forceinline__ void decode_chunk(DecodeState<MW, GQ> &st, const unsi
         const float2 pp = *reinterpret_cast<const float2 *>(p_s + bhead * 32 + vb * 16 + tp);
 #pragma unroll
         for (int bi = 0; bi < NB; ++bi) {
-            const int g = bi * NG + bgsel;
+            const int g = (NG == 1) ? 0 : bi * GPF + bgsel;
             const float2 dd = half2_bits_to_float2(
-                *reinterpret_cast<const uint32_t *>(ch + SCALE + vb * 128 + g * 32 + tp * 2));
+                *reinterpret_cast<const uint32_t *>(ch + SCALE + vb * (32 * NG) + g * 32 + tp * 2));
             const float x0 = pp.x * dd.x, x1 = pp.y * dd.y;
             const uint32_t hi = pack_f16x2(x0, x1);
             const float2 hf = half2_bits_to_float2(hi);
@@ -631,7 +648,7 @@ __device__ __forceinline__ void decode_chunk(DecodeState<MW, GQ> &st, const unsi
 #pragma unroll
             for (int i = 0; i < 4; ++i) {
                 const int cb = half * 4 + i;
-                const int bi = (cb >> 1) / NG;
+                const int bi = (NG == 1) ? 0 : (cb >> 1) / GPF;
                 uint32_t a[4];
                 codes_to_f16x2(wv[i], a);
                 if (vb == 0) mma_f16_16816_from(tmp[i], a[0], a[1], a[2], a[3], bf[vb][bi][0], bf[vb][bi][1], st.zero);
@@ -650,9 +667,9 @@ __device__ __forceinline__ void decode_chunk(DecodeState<MW, GQ> &st, const unsi
     __syncwarp();
 }
 
-template <int MW, int GQ>
+template <int MW, int GQ, int NG>
 __global__ void __launch_bounds__(kDecodeWarps * 32, decode_min_blocks(GQ)) decode_split_kernel(DecodeParams p) {
-    using SM = DecodeSmem<MW, GQ>;
+    using SM = DecodeSmem<MW, GQ, NG>;
     constexpr int CB = SM::kChunkBytes;
     extern __shared__ __align__(128) unsigned char smem_raw[];
 
@@ -704,7 +721,7 @@ __global__ void __launch_bounds__(kDecodeWarps * 32, decode_min_blocks(GQ)) deco
         }
     }
 
-    DecodeState<MW, GQ> st;
+    DecodeState<MW, GQ, NG> st;
     zero_quad(st.zero);
     {
         const uint32_t *qp = p.qwords + ((size_t)(layer * p.max_batch + b) * p.Hq + kvh * GQ) * MW;
@@ -722,7 +739,7 @@ __global__ void __launch_bounds__(kDecodeWarps * 32, decode_min_blocks(GQ)) deco
         st.hmin[h] = kHamSentinel;
         st.ssum[h] = 0.f;
 #pragma unroll
-        for (int g = 0; g < kGroups; ++g) st.accz[h][g] = 0.f;
+        for (int g = 0; g < NG; ++g) st.accz[h][g] = 0.f;
     }
 
     int stage = 0;
@@ -731,8 +748,8 @@ __global__ void __launch_bounds__(kDecodeWarps * 32, decode_min_blocks(GQ)) deco
     for (int c = c0; c < c1; ++c) {
         if (!mbar_wait_bounded(bar0 + 8 * stage, parity, kWaitLimitNs)) { failed = true; break; }
         const unsigned char *ch = ring + stage * CB;
-        if (c < c_full) decode_chunk<MW, GQ, false>(st, ch, p_s, lane, 32, p.c2);
-        else decode_chunk<MW, GQ, true>(st, ch, p_s, lane, t_end - c * 32, p.c2);
+        if (c < c_full) decode_chunk<MW, GQ, NG, false>(st, ch, p_s, lane, 32, p.c2);
+        else decode_chunk<MW, GQ, NG, true>(st, ch, p_s, lane, t_end - c * 32, p.c2);
         // every lane is done with this stage (the chunk ends with a warp barrier): refill it
         if (lane == 0 && requested < c1) {
             mbar_arrive_expect_tx(bar0 + 8 * stage, CB);
@@ -761,7 +778,7 @@ __global__ void __launch_bounds__(kDecodeWarps * 32, decode_min_blocks(GQ)) deco
         for (int o = 16; o > 0; o >>= 1) {
             st.ssum[h] += __shfl_xor_sync(0xffffffffu, st.ssum[h], o);
 #pragma unroll
-            for (int g = 0; g < kGroups; ++g) st.accz[h][g] += __shfl_xor_sync(0xffffffffu, st.accz[h][g], o);
+            for (int g = 0; g < NG; ++g) st.accz[h][g] += __shfl_xor_sync(0xffffffffu, st.accz[h][g], o);
         }
     }
     // Undo the scales: codes were fed as code / kCodeScaleLo (rows r) and code / kCodeScaleHi (rows r + 8), the
@@ -779,18 +796,18 @@ __global__ void __launch_bounds__(kDecodeWarps * 32, decode_min_blocks(GQ)) deco
             const float hi = (jq & 2) ? other : st.acc[cb][i], lo = (jq & 2) ? st.acc[cb][i] : other;
             v[i] = fmaf(lo, kLoPart, hi) * (i < 2 ? kRowLo : kRowHi);
         }
-        const int g = cb >> 1;
+        const int g = cb >> 1, gz = (NG == 1) ? 0 : g;          // gz: which zero-point sum belongs to this channel block
         if (GQ == 1) {
             if (jq == (g >> 1)) {
-                part_out[cb * 16 + r] = v[g & 1] + st.accz[0][g];
-                part_out[cb * 16 + r + 8] = v[2 + (g & 1)] + st.accz[0][g];
+                part_out[cb * 16 + r] = v[g & 1] + st.accz[0][gz];
+                part_out[cb * 16 + r + 8] = v[2 + (g & 1)] + st.accz[0][gz];
             }
         } else if (GQ == 2) {
             if (jq == (g & 1)) {
 #pragma unroll
                 for (int h = 0; h < 2; ++h) {
-                    part_out[h * kPartStride + cb * 16 + r] = v[h] + st.accz[h < GQ ? h : 0][g];
-                    part_out[h * kPartStride + cb * 16 + r + 8] = v[2 + h] + st.accz[h < GQ ? h : 0][g];
+                    part_out[h * kPartStride + cb * 16 + r] = v[h] + st.accz[h < GQ ? h : 0][gz];
+                    part_out[h * kPartStride + cb * 16 + r + 8] = v[2 + h] + st.accz[h < GQ ? h : 0][gz];
                 }
             }
         } else {
@@ -798,7 +815,7 @@ __global__ void __launch_bounds__(kDecodeWarps * 32, decode_min_blocks(GQ)) deco
 #pragma unroll
                 for (int hh = 0; hh < 2; ++hh) {
                     // head = 2*jq + hh, a lane-dependent index: select without dynamic indexing
-                    const float z = (jq == 0) ? st.accz[hh < GQ ? hh : 0][g] : st.accz[(2 + hh) < GQ ? (2 + hh) : 0][g];
+                    const float z = (jq == 0) ? st.accz[hh < GQ ? hh : 0][gz] : st.accz[(2 + hh) < GQ ? (2 + hh) : 0][gz];
                     float *dst = part_out + (size_t)(2 * jq + hh) * kPartStride;
                     dst[cb * 16 + r] = v[hh] + z;
                     dst[cb * 16 + r + 8] = v[2 + hh] + z;
@@ -879,11 +896,11 @@ __global__ void __launch_bounds__(kHeadDim) combine_kernel(DecodeParams p) {
 }
 
 // Test helper: score of every cached token of one slab against one sketch.
-__global__ void debug_scores_kernel(const unsigned char *slab, const uint32_t *qwords, int m_words, int len,
+__global__ void debug_scores_kernel(const unsigned char *slab, const uint32_t *qwords, int m_words, int groups, int len,
                                     int32_t *score) {
     const int t = blockIdx.x * blockDim.x + threadIdx.x;
     if (t >= len) return;
-    const ChunkLayout cl = chunk_layout(m_words);
+    const ChunkLayout cl = chunk_layout(m_words, groups);
     const unsigned char *chunk = slab + (size_t)(t >> 5) * cl.bytes;
     int ham = 0;
     for (int w = 0; w < m_words; ++w)
@@ -964,14 +981,14 @@ cudaError_t launch_set_len(int32_t *len, int n_layers, int max_batch, int seq, i
     return cudaGetLastError();
 }
 
-template <int MW, int GQ>
+template <int MW, int GQ, int NG>
 static cudaError_t launch_decode_t(const DecodeParams &p, cudaStream_t st) {
-    using SM = DecodeSmem<MW, GQ>;
+    using SM = DecodeSmem<MW, GQ, NG>;
     static bool attr_set[64] = {};
     int dev = 0;
     cudaGetDevice(&dev);
     if (dev >= 0 && dev < 64 && !attr_set[dev]) {
-        cudaError_t e = cudaFuncSetAttribute(decode_split_kernel<MW, GQ>,
+        cudaError_t e = cudaFuncSetAttribute(decode_split_kernel<MW, GQ, NG>,
                                              cudaFuncAttributeMaxDynamicSharedMemorySize, SM::kTotal);
         if (e != cudaSuccess) return e;
         attr_set[dev] = true;
@@ -988,7 +1005,7 @@ static cudaError_t launch_decode_t(const DecodeParams &p, cudaStream_t st) {
     attr[0].val.programmaticStreamSerializationAllowed = 1;
     cfg.attrs = attr;
     cfg.numAttrs = 1;
-    return cudaLaunchKernelEx(&cfg, decode_split_kernel<MW, GQ>, p);
+    return cudaLaunchKernelEx(&cfg, decode_split_kernel<MW, GQ, NG>, p);
 }
 
 cudaError_t launch_decode(const DecodeParams &p, cudaStream_t st, int *launches, cudaEvent_t before,
@@ -997,9 +1014,15 @@ cudaError_t launch_decode(const DecodeParams &p, cudaStream_t st, int *launches,
     cudaError_t e = cudaErrorInvalidValue;
     if (before) cudaEventRecord(before, st);
     H1B_DISPATCH_MW(p.m_words,
-        if (gq == 1) e = launch_decode_t<MW, 1>(p, st);
-        else if (gq == 2) e = launch_decode_t<MW, 2>(p, st);
-        else if (gq == 4) e = launch_decode_t<MW, 4>(p, st);
+        if (p.groups == 4) {
+            if (gq == 1) e = launch_decode_t<MW, 1, 4>(p, st);
+            else if (gq == 2) e = launch_decode_t<MW, 2, 4>(p, st);
+            else if (gq == 4) e = launch_decode_t<MW, 4, 4>(p, st);
+        } else if (p.groups == 1) {
+            if (gq == 1) e = launch_decode_t<MW, 1, 1>(p, st);
+            else if (gq == 2) e = launch_decode_t<MW, 2, 1>(p, st);
+            else if (gq == 4) e = launch_decode_t<MW, 4, 1>(p, st);
+        }
     );
     if (e != cudaSuccess) return e;
     if (after) cudaEventRecord(after, st);
@@ -1023,10 +1046,10 @@ cudaError_t launch_decode(const DecodeParams &p, cudaStream_t st, int *launches,
     return cudaGetLastError();
 }
 
-cudaError_t launch_debug_scores(const unsigned char *slab, const uint32_t *qwords, int m_words, int len,
+cudaError_t launch_debug_scores(const unsigned char *slab, const uint32_t *qwords, int m_words, int groups, int len,
                                 int32_t *score, cudaStream_t st) {
     if (len <= 0) return cudaSuccess;
-    debug_scores_kernel<<<(len + 127) / 128, 128, 0, st>>>(slab, qwords, m_words, len, score);
+    debug_scores_kernel<<<(len + 127) / 128, 128, 0, st>>>(slab, qwords, m_words, groups, len, score);
     return cudaGetLastError();
 }
 

@@ -18,7 +18,7 @@ cudaError_t launch_split_projection(const float *Rt, uint16_t *Rh, int n_layers,
 cudaError_t launch_decode(const DecodeParams &p, cudaStream_t st, int *launches, cudaEvent_t before = nullptr,
                           cudaEvent_t after = nullptr);
 cudaError_t launch_set_len(int32_t *len, int n_layers, int max_batch, int seq, int value, cudaStream_t st);
-cudaError_t launch_debug_scores(const unsigned char *slab, const uint32_t *qwords, int m_words, int len,
+cudaError_t launch_debug_scores(const unsigned char *slab, const uint32_t *qwords, int m_words, int groups, int len,
                                 int32_t *score, cudaStream_t st);
 
 }  // namespace h1b

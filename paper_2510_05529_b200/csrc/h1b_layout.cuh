@@ -19,11 +19,12 @@
 //                 nibble 3: (channel cb*16+r+8, token 2j+8)  nibble 7: (.., token 2j+9)
 //               so one token of one word is exactly one byte (two channels), and an
 //               append never has to read-modify-write.
-//   zero        fp16 [32 tokens][4 groups]
-//   scale       fp16 [2 blocks][4 groups][16 tokens]
+//   zero        fp16 [32 tokens][groups]
+//   scale       fp16 [2 blocks][groups][16 tokens]
 //
-// Bytes per token: m/8 + 64 + 8 + 8, the count of Section IV-B's storage
-// statement plus the fp16 scale and zero of each group.
+// groups = 128 / group_size: 4 (groups of 32 channels) or 1 (one scale and zero per value vector, the
+// per-vector scheme of Section IV-B). Bytes per token: m/8 + 64 + 4 * groups, the count of Section IV-B's
+// storage statement plus the fp16 scale and zero of each group.
 #pragma once
 #include <cstdint>
 #include <cstddef>
@@ -32,26 +33,28 @@ namespace h1b {
 
 constexpr int kHeadDim = 128;
 constexpr int kGroup = 32;
-constexpr int kGroups = kHeadDim / kGroup;       // 4
+constexpr int kGroups = kHeadDim / kGroup;       // 4: the most groups a value vector can have
 constexpr int kChunkTokens = 32;
 constexpr int kValBlockBytes = 1024;             // 16 tokens x 128 channels x 4 bit
 constexpr int kPartStride = 132;                 // floats per (item, head): acc[128], min Hamming, sum, pad
 
 struct ChunkLayout {
     int m_words;      // m / 32
+    int groups;       // scale/zero pairs per value vector: 4 or 1
     int val_off;      // byte offset of the value codes
     int zero_off;
     int scale_off;
     int bytes;        // chunk size
 };
 
-__host__ __device__ inline ChunkLayout chunk_layout(int m_words) {
+__host__ __device__ inline ChunkLayout chunk_layout(int m_words, int groups) {
     ChunkLayout c;
     c.m_words = m_words;
+    c.groups = groups;
     c.val_off = m_words * 4 * kChunkTokens;
     c.zero_off = c.val_off + 2 * kValBlockBytes;
-    c.scale_off = c.zero_off + kChunkTokens * kGroups * 2;
-    c.bytes = c.scale_off + kChunkTokens * kGroups * 2;
+    c.scale_off = c.zero_off + kChunkTokens * groups * 2;
+    c.bytes = c.scale_off + kChunkTokens * groups * 2;
     return c;
 }
 
@@ -67,10 +70,10 @@ __host__ __device__ inline int code_byte_off(const ChunkLayout &c, int tt, int c
     return c.val_off + vb * kValBlockBytes + (cb >> 2) * 512 + lane * 16 + (cb & 3) * 4 + odd * 2 + hi8;
 }
 __host__ __device__ inline int zero_off(const ChunkLayout &c, int tt, int g) {
-    return c.zero_off + tt * 8 + g * 2;
+    return c.zero_off + tt * (2 * c.groups) + g * 2;
 }
 __host__ __device__ inline int scale_off(const ChunkLayout &c, int tt, int g) {
-    return c.scale_off + (tt >> 4) * 128 + g * 32 + (tt & 15) * 2;
+    return c.scale_off + (tt >> 4) * (32 * c.groups) + g * 32 + (tt & 15) * 2;
 }
 
 // Device status word values.
@@ -86,7 +89,7 @@ struct AppendParams {
     int32_t *len;               // [L][max_batch]
     int32_t *done;              // block counter of the append launch (zero between launches)
     size_t slab_bytes;
-    int layer_begin, n_layers, B, Tn, Hkv, max_batch, m_words;
+    int layer_begin, n_layers, B, Tn, Hkv, max_batch, m_words, groups;
 };
 
 struct PrefillParams {          // long appends: tensor-core projection
@@ -97,7 +100,7 @@ struct PrefillParams {          // long appends: tensor-core projection
     int32_t *status;            // device status word (bounded-wait timeouts)
     int32_t *done;              // block counter (zero between launches)
     size_t slab_bytes;
-    int layer_begin, n_layers, B, Tn, Hkv, max_batch, m_words;
+    int layer_begin, n_layers, B, Tn, Hkv, max_batch, m_words, groups;
     int tiles_per_seq;          // 128-position tiles that can overlap the appended range of a sequence
     int tiles_per_block;        // consecutive tiles handled by one block (the projection is loaded once per block)
 };
@@ -118,7 +121,7 @@ struct DecodeParams {
     int32_t *status;
     int32_t *arrive;            // [slabs of the call]: splits that have reported in (zero between launches)
     size_t slab_bytes;
-    int layer_begin, n_layers, B, Hkv, Hq, max_batch, m_words;
+    int layer_begin, n_layers, B, Hkv, Hq, max_batch, m_words, groups;
     int splits, split_tokens;   // split_tokens is a multiple of 32
     float c2;                   // 2 * inv_tau * log2(e) / m : log2-weight per unit of Hamming distance
 };

@@ -41,6 +41,10 @@ def test_entry_and_workspace_bytes(lib):
     c4 = binding.make_config(32, 32, 8, 128, 256, 32, max_batch=8, max_seq=32768)
     assert binding.h1b_entry_bytes(c4) == 112
     assert binding.h1b_cache_bytes(c4) >= 32 * 8 * 8 * 32768 * 112
+    # one scale and zero per value vector (G = d) shrinks the entry to 84 bytes
+    cv = binding.make_config(32, 32, 32, 128, 128, 128, max_batch=1, max_seq=8192)
+    assert binding.h1b_entry_bytes(cv) == 84
+    assert 32 * 32 * 8192 * 84 <= binding.h1b_cache_bytes(cv) < total
     # capacity is rounded up to whole 32-token chunks
     a = binding.h1b_cache_bytes(binding.make_config(1, 1, 1, max_seq=33))
     b = binding.h1b_cache_bytes(binding.make_config(1, 1, 1, max_seq=64))

@@ -39,6 +39,19 @@ def test_gqa_and_sketch_widths(hq, hkv, m):
     print("gqa", hq, hkv, m, tot)
 
 
+@pytest.mark.parametrize("hq,hkv,m", [(2, 2, 128), (8, 2, 256), (4, 2, 64), (1, 1, 512)])
+def test_per_vector_quantisation_group_size_equals_head_dim(hq, hkv, m):
+    """G = d: one scale and zero per value vector, the literal scheme of Section IV-B (84 B per token at m = 128)."""
+    w = small("c2_7b_8k", n_layers=2, n_q_heads=hq, n_kv_heads=hkv, sketch_bits=m, group_size=128, batch=2,
+              context=300, outlier_frac=0.02)
+    cache, _ = make_cache(w, max_seq=8)
+    assert binding.h1b_entry_bytes(cache.cfg) == m // 8 + 64 + 4
+    cache.close()
+    # a long append (tensor-core path), a short one, then single tokens
+    tot = full_parity(w, [300, 131], appends=[200, 40] + [1] * 60)
+    print("G=128", hq, hkv, m, tot)
+
+
 @pytest.mark.parametrize("inv_tau", [1e-6, 1.0, 16.0, 50.0, 1000.0])
 def test_temperatures_from_uniform_to_argmax(inv_tau):
     w = small("c2_7b_8k", n_layers=1, n_q_heads=2, n_kv_heads=2, batch=1, context=700)
