@@ -127,6 +127,9 @@ def run_ours(args):
     pdist.init("nccl", torch.device("cuda", local))
     dev = torch.device("cuda", local)
     w = h1b_synth.WORKLOADS[args.workload]
+    if args.sketch_bits or args.group_size:           # the paper's ablation axes (Table V) as throughput variants
+        w = h1b_synth.scaled(w, sketch_bits=args.sketch_bits or w.sketch_bits, group_size=args.group_size or w.group_size,
+                             name="%s[m=%d,G=%d]" % (w.name, args.sketch_bits or w.sketch_bits, args.group_size or w.group_size))
     if args.workload == "c5_prefill":
         return run_prefill(args, w, pdist, rank, world, local)
     steps, warmup = args.steps, args.warmup
@@ -243,7 +246,7 @@ def run_ours(args):
         "clocks": clocks,
         "roofline": roofline,
     }
-    if rank == 0 and world == 1 and not args.no_cpu_baseline and args.workload == "c2_7b_8k":
+    if rank == 0 and world == 1 and not args.no_cpu_baseline and w.name == "c2_7b_8k":
         line["cpu_baseline"] = cpu_baseline(sample_layers=1, steps=5, warmup=1)
     cache.close()
     pdist.finish()
@@ -377,6 +380,8 @@ def main():
     ap.add_argument("--warmup", type=int, default=30)
     ap.add_argument("--impl", default="ours", choices=["ours", "reference"])
     ap.add_argument("--no-cpu-baseline", action="store_true")
+    ap.add_argument("--sketch-bits", type=int, default=0, help="override m (64, 128, 256, 512)")
+    ap.add_argument("--group-size", type=int, default=0, help="override G (32, or 128 = one scale per value vector)")
     ap.add_argument("--workload", default="c2_7b_8k",
                     choices=["c2_7b_8k", "c3_7b_batched", "c4_gqa_32k", "c5_prefill"],
                     help="default: the configuration the metric is quoted on; the others are reported in DESIGN.md")

@@ -1,5 +1,5 @@
 // Thin inline-PTX wrappers used by the H1B-KV kernels (sm_100a): mbarrier with
-// bounded waits, non-multicast bulk async copies into this CTA's shared memory,
+// bounded waits, bulk async copies into this CTA's own shared memory (one destination CTA),
 // warp-level fp16 tensor-core MMA, and a few scalar helpers.
 #pragma once
 #include <cstdint>
@@ -49,7 +49,7 @@ __device__ __forceinline__ bool mbar_wait_bounded(uint32_t bar, uint32_t parity,
     }
 }
 
-// Bulk async copy global -> this CTA's shared memory (no multicast); completion
+// Bulk async copy global -> this CTA's shared memory (one destination CTA); completion
 // is signalled on `bar` as transferred bytes. Both addresses 16-byte aligned,
 // `bytes` a multiple of 16.
 __device__ __forceinline__ void bulk_copy_g2s(uint32_t dst, const void *src, uint32_t bytes, uint32_t bar) {
