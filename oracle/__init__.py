@@ -68,6 +68,13 @@ def _load():
             lib.h1bo_decode_cached.argtypes = [u8p, u8p, u16p, u16p, i32p, u16p, f32p, ctypes.c_int,
                                                ctypes.c_long, ctypes.c_int, ctypes.c_int, ctypes.c_int,
                                                ctypes.c_int, ctypes.c_int, ctypes.c_double, f64p]
+            lib.h1bo_attention_fp16_values.restype = None
+            lib.h1bo_attention_fp16_values.argtypes = [i32p, ctypes.c_long, ctypes.c_int, ctypes.c_double, u16p,
+                                                       ctypes.c_int, f64p]
+            lib.h1bo_layer_fp16_values.restype = ctypes.c_long
+            lib.h1bo_layer_fp16_values.argtypes = [u16p, u16p, i32p, u16p, f32p, ctypes.c_int, ctypes.c_long,
+                                                   ctypes.c_int, ctypes.c_int, ctypes.c_int, ctypes.c_int,
+                                                   ctypes.c_double, f64p]
             lib.h1bo_entry_bytes.restype = ctypes.c_long
             lib.h1bo_entry_bytes.argtypes = [ctypes.c_int, ctypes.c_int, ctypes.c_int]
             lib.h1bo_threads.restype = ctypes.c_int
@@ -221,6 +228,35 @@ def decode_cached(cache, lens, q, Rt, inv_tau: float, G: int = 32):
                                      _ptr(ln, ctypes.c_int32), _ptr(qb, ctypes.c_uint16),
                                      _ptr(Rt, ctypes.c_float), B, T, Hq, Hkv, d, m, G, float(inv_tau),
                                      _ptr(out, ctypes.c_double))
+    if bad:
+        raise AssertionError("oracle: score identity violated %d times" % bad)
+    return out
+
+
+def attention_fp16_values(score, m: int, inv_tau: float, v16):
+    """Eq. 5 with uncompressed fp16 values (the key-only ablation). score [T], v16 [T, d] -> out fp64 [d]."""
+    sc = np.ascontiguousarray(score, dtype=np.int32)
+    vb = _as_u16(v16)
+    T, d = vb.shape
+    assert sc.shape == (T,)
+    out = np.zeros((d,), dtype=np.float64)
+    _load().h1bo_attention_fp16_values(_ptr(sc, ctypes.c_int32), T, m, float(inv_tau), _ptr(vb, ctypes.c_uint16), d,
+                                       _ptr(out, ctypes.c_double))
+    return out
+
+
+def layer_fp16_values(K, V, lens, q, Rt, inv_tau: float):
+    """The key-only variant for one layer: 1-bit key sketches, values kept in fp16."""
+    Kb, Vb, qb = _as_u16(K), _as_u16(V), _as_u16(q)
+    B, T, Hkv, d = Kb.shape
+    Hq = qb.shape[1]
+    Rt = np.ascontiguousarray(Rt, dtype=np.float32)
+    m = Rt.shape[1]
+    ln = np.ascontiguousarray(lens, dtype=np.int32)
+    out = np.zeros((B, Hq, d), dtype=np.float64)
+    bad = _load().h1bo_layer_fp16_values(_ptr(Kb, ctypes.c_uint16), _ptr(Vb, ctypes.c_uint16), _ptr(ln, ctypes.c_int32),
+                                         _ptr(qb, ctypes.c_uint16), _ptr(Rt, ctypes.c_float), B, T, Hq, Hkv, d, m,
+                                         float(inv_tau), _ptr(out, ctypes.c_double))
     if bad:
         raise AssertionError("oracle: score identity violated %d times" % bad)
     return out

@@ -36,7 +36,8 @@
  * Prop. 1); bit agreement rate tracks 1 - theta/pi (Eq. 1); round trip error
  * <= Delta/2; T = 1, equal keys, tau -> infinity and tau -> 0 limits; a
  * lossless 16-level grid reduces Eq. 5 to a library softmax @ V; hand-worked
- * tiny cases.  Parity unpinned (conventions of this build, nothing in the
+ * tiny cases; the fp16-value variant reduces to a library softmax @ V directly.
+ * Parity unpinned (conventions of this build, nothing in the
  * paper fixes them): the min/max rule for Delta and zero, round-half-to-even,
  * and the value of tau.
  */
@@ -233,6 +234,66 @@ void h1bo_attention(const int32_t *score, long T, int m, double inv_tau,
         }
     }
     free(w);
+}
+
+/* ------------------------------------------------------------------------ */
+/* Eq. 5 with uncompressed values: the "1-bit-key only" row of the ablation   */
+/* (Table V): out = softmax(alpha / tau) * V, V kept as binary16.              */
+/*   score [T] from h1bo_scores, v16 [T][d] binary16, out [d] fp64             */
+/* ------------------------------------------------------------------------ */
+void h1bo_attention_fp16_values(const int32_t *score, long T, int m, double inv_tau,
+                                const uint16_t *v16, int d, double *out)
+{
+    for (int c = 0; c < d; ++c) out[c] = 0.0;
+    if (T <= 0) return;
+    double *w = (double *)malloc(sizeof(double) * (size_t)T);
+    double mx = -INFINITY, sum = 0.0;
+    for (long t = 0; t < T; ++t) {
+        w[t] = ((double)score[t] / (double)m) * inv_tau;
+        if (w[t] > mx) mx = w[t];
+    }
+    for (long t = 0; t < T; ++t) { w[t] = exp(w[t] - mx); sum += w[t]; }
+    for (long t = 0; t < T; ++t) {
+        double pt = w[t] / sum;
+        for (int c = 0; c < d; ++c) out[c] += pt * h1bo_half_to_double(v16[t * d + c]);
+    }
+    free(w);
+}
+
+/* Layer driver of the key-only variant: like h1bo_layer, values uncompressed. */
+long h1bo_layer_fp16_values(const uint16_t *K, const uint16_t *V, const int32_t *lens,
+                            const uint16_t *q, const float *Rt, int B, long T, int Hq,
+                            int Hkv, int d, int m, double inv_tau, double *out)
+{
+    long bad_total = 0;
+    int rep = Hq / Hkv;
+    long units = (long)B * Hkv;
+#ifdef _OPENMP
+#pragma omp parallel for schedule(dynamic, 1) reduction(+ : bad_total)
+#endif
+    for (long u = 0; u < units; ++u) {
+        int b = (int)(u / Hkv), g = (int)(u % Hkv);
+        long len = lens[b];
+        size_t n = (size_t)(len > 0 ? len : 1);
+        uint16_t *krow = (uint16_t *)malloc(n * d * sizeof(uint16_t));
+        uint16_t *vrow = (uint16_t *)malloc(n * d * sizeof(uint16_t));
+        uint8_t *kbits = (uint8_t *)malloc(n * m);
+        int32_t *score = (int32_t *)malloc(n * sizeof(int32_t));
+        uint8_t *qbits = (uint8_t *)malloc((size_t)m);
+        for (long t = 0; t < len; ++t) {
+            memcpy(krow + t * d, K + (((size_t)b * T + t) * Hkv + g) * d, d * sizeof(uint16_t));
+            memcpy(vrow + t * d, V + (((size_t)b * T + t) * Hkv + g) * d, d * sizeof(uint16_t));
+        }
+        h1bo_sketch(krow, len, d, m, Rt, kbits, NULL, NULL);
+        for (int r = 0; r < rep; ++r) {
+            int h = g * rep + r;
+            h1bo_sketch(q + ((size_t)b * Hq + h) * d, 1, d, m, Rt, qbits, NULL, NULL);
+            bad_total += h1bo_scores(qbits, kbits, len, m, score);
+            h1bo_attention_fp16_values(score, len, m, inv_tau, vrow, d, out + ((size_t)b * Hq + h) * d);
+        }
+        free(krow); free(vrow); free(kbits); free(score); free(qbits);
+    }
+    return bad_total;
 }
 
 /* ------------------------------------------------------------------------ */

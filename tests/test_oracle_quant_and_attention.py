@@ -205,3 +205,27 @@ def test_decode_cached_equals_layer_driver():
     lens = np.array([50, 23], np.int32)
     cache = oracle.compress(K, V, Rt)
     assert np.array_equal(oracle.decode_cached(cache, lens, q, Rt, 16.0), oracle.layer(K, V, lens, q, Rt, 16.0))
+
+
+def test_fp16_value_variant_is_softmax_matmul():
+    """Key-only ablation: the oracle's output is scipy's softmax(alpha/tau) @ V on numpy-made sketches."""
+    rng = np.random.default_rng(15)
+    B, T, Hq, Hkv, d, m = 2, 70, 4, 2, 128, 128
+    Rt = rng.standard_normal((d, m)).astype(np.float32)
+    K = rng.standard_normal((B, T, Hkv, d)).astype(np.float16)
+    V = rng.standard_normal((B, T, Hkv, d)).astype(np.float16)
+    q = rng.standard_normal((B, Hq, d)).astype(np.float16)
+    lens = np.array([70, 9], np.int32)
+    out = oracle.layer_fp16_values(K, V, lens, q, Rt, 16.0)
+    R64 = Rt.astype(np.float64)
+    for b in range(B):
+        L = int(lens[b])
+        for h in range(Hq):
+            g = h // 2
+            sk = np.where(K[b, :L, g].astype(np.float64) @ R64 >= 0, 1.0, -1.0)
+            sq = np.where(q[b, h].astype(np.float64) @ R64 >= 0, 1.0, -1.0)
+            want = softmax(sk @ sq / m * 16.0) @ V[b, :L, g].astype(np.float64)
+            assert np.allclose(out[b, h], want, rtol=0, atol=1e-12)
+    sc = np.array([4, 0, -4], np.int32)
+    o = oracle.attention_fp16_values(sc, 4, 1.0, V[0, :3, 0])
+    assert np.allclose(o, np.array([0.66524096, 0.24472847, 0.09003057]) @ V[0, :3, 0].astype(np.float64), atol=2e-8)
