@@ -130,13 +130,16 @@ def run_ours(args):
     if args.sketch_bits or args.group_size:           # the paper's ablation axes (Table V) as throughput variants
         w = h1b_synth.scaled(w, sketch_bits=args.sketch_bits or w.sketch_bits, group_size=args.group_size or w.group_size,
                              name="%s[m=%d,G=%d]" % (w.name, args.sketch_bits or w.sketch_bits, args.group_size or w.group_size))
+    if args.fp16_values:                              # Table V's "1-bit keys only" row: values stay fp16
+        w = h1b_synth.scaled(w, name=w.name + "[fp16 values]")
     if args.workload == "c5_prefill":
         return run_prefill(args, w, pdist, rank, world, local)
     steps, warmup = args.steps, args.warmup
     total_steps = 2 * (steps + warmup) + 8           # device-resident run, then the host-buffer run
     lens0 = h1b_synth.lengths(w) - 1                  # the first step decodes exactly the workload's context
     cfg = binding.make_config(w.n_layers, w.n_q_heads, w.n_kv_heads, w.head_dim, w.sketch_bits, w.group_size,
-                              max_batch=w.batch, max_seq=w.context - 1 + total_steps, device=local)
+                              max_batch=w.batch, max_seq=w.context - 1 + total_steps, device=local,
+                              fp16_values=args.fp16_values)
     # each rank is its own sequence: different seeds per rank
     wr = h1b_synth.scaled(w, index=w.index + 10 * rank)
     Rt = np.stack([h1b_synth.projection(h1b_synth.layer_seed(wr, l, 99), w.head_dim, w.sketch_bits)
@@ -224,7 +227,9 @@ def run_ours(args):
                 "peak_kind": peak_kind + " (MEASURED_PEAKS.json hbm_gbs)" if peak_kind == "measured" else "fallback",
                 "unit": "GB/s", "frac": (achieved / peak) if achieved else None,
                 "frac_of_8tbs_nominal": (achieved / 8000.0) if achieved else None,
-                "traffic": NCU_TRAFFIC_PER_ALGORITHMIC_BYTE * alg_bytes, "traffic_source": "ncu capture at 8199 tokens, scaled by algorithmic bytes",
+                # the capture is of the default configuration's kernel; variants have no captured traffic
+                "traffic": (NCU_TRAFFIC_PER_ALGORITHMIC_BYTE * alg_bytes) if w.name == "c2_7b_8k" else None,
+                "traffic_source": "ncu capture at 8199 tokens, scaled by algorithmic bytes" if w.name == "c2_7b_8k" else None,
                 "alg_bytes_per_launch": alg_bytes,
                 "kernel_ms_avg": kern_ms_avg, "kernel_launches_timed": kern_n,
                 "step_gbs": alg_bytes / (ms_per_step * 1e-3) / 1e9}
@@ -262,7 +267,7 @@ def run_prefill(args, w, pdist, rank, world, local):
     from paper_2510_05529_b200 import binding
     dev = torch.device("cuda", local)
     cfg = binding.make_config(w.n_layers, w.n_q_heads, w.n_kv_heads, w.head_dim, w.sketch_bits, w.group_size,
-                              max_batch=w.batch, max_seq=w.context, device=local)
+                              max_batch=w.batch, max_seq=w.context, device=local, fp16_values=args.fp16_values)
     cache = binding.H1BCache(cfg, seed=11 + rank)
     K = torch.stack([h1b_synth.kv_rows(w, l, w.context, device=str(dev))[0] for l in range(w.n_layers)])
     V = torch.stack([h1b_synth.kv_rows(w, l, w.context, device=str(dev))[1] for l in range(w.n_layers)])
@@ -382,6 +387,7 @@ def main():
     ap.add_argument("--no-cpu-baseline", action="store_true")
     ap.add_argument("--sketch-bits", type=int, default=0, help="override m (64, 128, 256, 512)")
     ap.add_argument("--group-size", type=int, default=0, help="override G (32, or 128 = one scale per value vector)")
+    ap.add_argument("--fp16-values", action="store_true", help="keep values in fp16 (the 1-bit-keys-only ablation row)")
     ap.add_argument("--workload", default="c2_7b_8k",
                     choices=["c2_7b_8k", "c3_7b_batched", "c4_gqa_32k", "c5_prefill"],
                     help="default: the configuration the metric is quoted on; the others are reported in DESIGN.md")

@@ -34,6 +34,9 @@
  *   - Score of token t for a query: m - 2 * popcount(s_q xor s_t); alpha = score / m.
  *     All cached tokens [0, len) are attended, the one just appended included.
  *     Query head h reads KV head h / (Hq / Hkv).  An empty sequence gives zeros.
+ *   - With H1B_FLAG_FP16_VALUES (the "1-bit keys only" row of the ablation,
+ *     Table V) values are cached as the fp16 numbers they arrive as: no codes,
+ *     scales or zero-points; the output is softmax(alpha/tau) * V.
  */
 #ifndef H1B_H
 #define H1B_H
@@ -66,11 +69,16 @@ typedef struct {
     int32_t max_batch;     /* sequences the cache can hold (<= 256)                    */
     int32_t max_seq;       /* tokens per sequence the cache can hold                   */
     int32_t device;        /* CUDA device ordinal                                      */
-    uint32_t flags;        /* reserved, must be 0                                      */
+    uint32_t flags;        /* H1B_FLAG_* bits; every other bit must be 0               */
 } h1b_config;
 
+/* Keep values in fp16 (keys are still 1-bit sketches); group_size must still be a
+ * supported value but is not used. */
+#define H1B_FLAG_FP16_VALUES 1u
+
 /* Bytes of one cached token of one KV head: m/8 + d/2 + (d/G)*4 (Section IV-B
- * storage statement plus the fp16 scale and zero per group). 0 if invalid. */
+ * storage statement plus the fp16 scale and zero per group); m/8 + 2d with
+ * H1B_FLAG_FP16_VALUES. 0 if invalid. */
 size_t h1b_entry_bytes(const h1b_config *cfg /* HOST */);
 
 /* Bytes of device workspace the caller must provide for this configuration
@@ -192,9 +200,17 @@ int h1b_truncate(h1b_ctx *ctx, int seq, int new_len);
  * layout, independent of the packed device layout (all HOST, any may be NULL):
  *   words  uint32 [n][m/32]: sketch bit j is bit (j % 32) of word j / 32
  *   codes  uint8  [n][d]:    one 4-bit code per byte
- *   scale, zero  uint16 [n][d/G]: fp16 bit patterns */
+ *   scale, zero  uint16 [n][d/G]: fp16 bit patterns
+ * With H1B_FLAG_FP16_VALUES only `words` exists: codes, scale and zero must be
+ * NULL (H1B_ERR_INVALID_ARG otherwise); see h1b_export_values(). */
 int h1b_export_cache(h1b_ctx *ctx, int layer, int seq, int kv_head, int t0, int n,
                      uint32_t *words, uint8_t *codes, uint16_t *scale, uint16_t *zero);
+
+/* H1B_FLAG_FP16_VALUES only (H1B_ERR_INVALID_ARG otherwise): the cached values
+ * of tokens [t0, t0+n) of (layer, seq, kv_head).
+ *   values  HOST: uint16 [n][d], fp16 bit patterns, channel-contiguous */
+int h1b_export_values(h1b_ctx *ctx, int layer, int seq, int kv_head, int t0, int n,
+                      uint16_t *values);
 
 /* Sketch one query (DEVICE fp16 [d]) with layer `layer`'s projection and score
  * it against every cached token of (layer, seq, kv_head):

@@ -72,6 +72,8 @@ def load_library(rebuild: bool = True) -> ctypes.CDLL:
         "h1b_truncate": (ctypes.c_int, [vp, ctypes.c_int, ctypes.c_int]),
         "h1b_export_cache": (ctypes.c_int, [vp, ctypes.c_int, ctypes.c_int, ctypes.c_int, ctypes.c_int,
                                             ctypes.c_int, vp, vp, vp, vp]),
+        "h1b_export_values": (ctypes.c_int, [vp, ctypes.c_int, ctypes.c_int, ctypes.c_int, ctypes.c_int,
+                                             ctypes.c_int, vp]),
         "h1b_debug_scores": (ctypes.c_int, [vp, ctypes.c_int, ctypes.c_int, ctypes.c_int, vp, vp, vp]),
         "h1b_set_splits": (ctypes.c_int, [vp, ctypes.c_int]),
         "h1b_poll_status": (ctypes.c_int, [vp]),
@@ -87,10 +89,13 @@ def load_library(rebuild: bool = True) -> ctypes.CDLL:
     return lib
 
 
+H1B_FLAG_FP16_VALUES = 1      # h1b_config.flags: values stay fp16 (the 1-bit-keys-only configuration)
+
+
 def make_config(n_layers, n_q_heads, n_kv_heads, head_dim=128, sketch_bits=128, group_size=32,
-                max_batch=1, max_seq=8192, device=0) -> h1b_config:
+                max_batch=1, max_seq=8192, device=0, fp16_values=False) -> h1b_config:
     return h1b_config(n_layers, n_q_heads, n_kv_heads, head_dim, sketch_bits, group_size,
-                      max_batch, max_seq, device, 0)
+                      max_batch, max_seq, device, H1B_FLAG_FP16_VALUES if fp16_values else 0)
 
 
 def h1b_entry_bytes(cfg: h1b_config) -> int:
@@ -255,12 +260,22 @@ class H1BCache:
         """-> (words uint32 [n, m/32], codes uint8 [n, d], scale uint16 [n, d/G], zero uint16 [n, d/G])."""
         c = self.cfg
         words = np.empty((n, c.sketch_bits // 32), dtype=np.uint32)
+        if c.flags & H1B_FLAG_FP16_VALUES:              # no codes, scales or zero-points in this cache
+            self._check(self.lib.h1b_export_cache(self._h, layer, seq, kv_head, t0, n, words.ctypes.data,
+                                                  None, None, None))
+            return words, None, None, None
         codes = np.empty((n, c.head_dim), dtype=np.uint8)
         scale = np.empty((n, c.head_dim // c.group_size), dtype=np.uint16)
         zero = np.empty_like(scale)
         self._check(self.lib.h1b_export_cache(self._h, layer, seq, kv_head, t0, n, words.ctypes.data,
                                               codes.ctypes.data, scale.ctypes.data, zero.ctypes.data))
         return words, codes, scale, zero
+
+    def h1b_export_values(self, layer: int, seq: int, kv_head: int, t0: int, n: int) -> np.ndarray:
+        """fp16-value caches only -> values uint16 [n, d] (fp16 bit patterns)."""
+        values = np.empty((n, self.cfg.head_dim), dtype=np.uint16)
+        self._check(self.lib.h1b_export_values(self._h, layer, seq, kv_head, t0, n, values.ctypes.data))
+        return values
 
     def h1b_debug_scores(self, layer: int, seq: int, kv_head: int, q_row: torch.Tensor, n_tokens: int):
         """q_row: fp16 CUDA [d]. -> (qwords uint32 [m/32], score int32 [n_tokens])."""

@@ -34,7 +34,8 @@ size_t align_up(size_t x, size_t a) { return (x + a - 1) / a * a; }
 int check_config(const h1b_config *c) {
     if (!c) return H1B_ERR_NULL;
     if (c->n_layers < 1 || c->n_q_heads < 1 || c->n_kv_heads < 1 || c->max_batch < 1 || c->max_seq < 1 ||
-        c->head_dim < 1 || c->sketch_bits < 1 || c->group_size < 1 || c->device < 0 || c->flags != 0)
+        c->head_dim < 1 || c->sketch_bits < 1 || c->group_size < 1 || c->device < 0 ||
+        (c->flags & ~H1B_FLAG_FP16_VALUES) != 0)
         return H1B_ERR_INVALID_ARG;
     if (c->n_q_heads % c->n_kv_heads != 0 || c->head_dim % c->group_size != 0 || c->sketch_bits % 32 != 0)
         return H1B_ERR_INVALID_ARG;
@@ -53,7 +54,7 @@ int make_plan(const h1b_config *c, Plan *p) {
     if (rc != H1B_OK) return rc;
     p->m_words = c->sketch_bits / 32;
     p->gq = c->n_q_heads / c->n_kv_heads;
-    p->groups = c->head_dim / c->group_size;
+    p->groups = (c->flags & H1B_FLAG_FP16_VALUES) ? 0 : c->head_dim / c->group_size;   // 0: values stay fp16
     const ChunkLayout cl = chunk_layout(p->m_words, p->groups);
     p->cap_tokens = (c->max_seq + kChunkTokens - 1) / kChunkTokens * kChunkTokens;
     p->slab_bytes = (size_t)(p->cap_tokens / kChunkTokens) * cl.bytes;
@@ -160,6 +161,7 @@ extern "C" {
 
 size_t h1b_entry_bytes(const h1b_config *cfg) {
     if (check_config(cfg) != H1B_OK) return 0;
+    if (cfg->flags & H1B_FLAG_FP16_VALUES) return (size_t)cfg->sketch_bits / 8 + (size_t)cfg->head_dim * 2;
     return (size_t)cfg->sketch_bits / 8 + (size_t)cfg->head_dim / 2 + (size_t)(cfg->head_dim / cfg->group_size) * 4;
 }
 
@@ -559,6 +561,8 @@ int h1b_export_cache(h1b_ctx *ctx, int layer, int seq, int kv_head, int t0, int 
     const int len = ctx->len_host[(size_t)layer * ctx->cfg.max_batch + seq];
     if (t0 < 0 || n < 0 || t0 + n > len)
         return fail(ctx, H1B_ERR_INVALID_ARG, "tokens [%d, %d) outside the cached [0, %d)", t0, t0 + n, len);
+    if (ctx->plan.groups == 0 && (codes || scale || zero))
+        return fail(ctx, H1B_ERR_INVALID_ARG, "this cache keeps fp16 values: it has no codes, scales or zero-points");
     if (n == 0) return H1B_OK;
     const ChunkLayout &cl = ctx->cl;
     const int c_lo = t0 / kChunkTokens, c_hi = (t0 + n - 1) / kChunkTokens;
@@ -583,6 +587,32 @@ int h1b_export_cache(h1b_ctx *ctx, int layer, int seq, int kv_head, int t0, int 
             if (scale) std::memcpy(&scale[(size_t)i * cl.groups + g], ch + scale_off(cl, tt, g), 2);
             if (zero) std::memcpy(&zero[(size_t)i * cl.groups + g], ch + zero_off(cl, tt, g), 2);
         }
+    }
+    return H1B_OK;
+}
+
+int h1b_export_values(h1b_ctx *ctx, int layer, int seq, int kv_head, int t0, int n, uint16_t *values) {
+    if (!ctx) return H1B_ERR_NULL;
+    if (ctx->plan.groups != 0) return fail(ctx, H1B_ERR_INVALID_ARG, "this cache keeps 4-bit codes, not fp16 values");
+    if (!values) return fail(ctx, H1B_ERR_NULL, "values is NULL");
+    if (layer < 0 || layer >= ctx->cfg.n_layers || seq < 0 || seq >= ctx->cfg.max_batch || kv_head < 0 ||
+        kv_head >= ctx->cfg.n_kv_heads)
+        return fail(ctx, H1B_ERR_INVALID_ARG, "(layer %d, seq %d, kv_head %d) out of range", layer, seq, kv_head);
+    const int len = ctx->len_host[(size_t)layer * ctx->cfg.max_batch + seq];
+    if (t0 < 0 || n < 0 || t0 + n > len)
+        return fail(ctx, H1B_ERR_INVALID_ARG, "tokens [%d, %d) outside the cached [0, %d)", t0, t0 + n, len);
+    if (n == 0) return H1B_OK;
+    const ChunkLayout &cl = ctx->cl;
+    const int c_lo = t0 / kChunkTokens, c_hi = (t0 + n - 1) / kChunkTokens;
+    std::vector<unsigned char> raw((size_t)(c_hi - c_lo + 1) * cl.bytes);
+    H1B_CUDA(ctx, cudaDeviceSynchronize());
+    H1B_CUDA(ctx, cudaMemcpy(raw.data(), slab_ptr(ctx, layer, seq, kv_head) + (size_t)c_lo * cl.bytes, raw.size(),
+                             cudaMemcpyDeviceToHost));
+    const int d = ctx->cfg.head_dim;
+    for (int i = 0; i < n; ++i) {
+        const int t = t0 + i, tt = t % kChunkTokens;
+        const unsigned char *ch = raw.data() + (size_t)(t / kChunkTokens - c_lo) * cl.bytes;
+        for (int c = 0; c < d; ++c) std::memcpy(&values[(size_t)i * d + c], ch + value_half_off(cl, tt, c), 2);
     }
     return H1B_OK;
 }

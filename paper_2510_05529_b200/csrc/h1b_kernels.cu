@@ -133,6 +133,24 @@ __device__ __forceinline__ void quantize_row(const uint16_t *__restrict__ v_row,
     }
 }
 
+// fp16-value cache (groups == 0): one row by one warp, copied into the packed value plane.
+__device__ __forceinline__ void store_row_f16(const uint16_t *__restrict__ v_row, unsigned char *chunk,
+                                              const ChunkLayout &cl, int tt, int lane) {
+    const uint2 raw = __ldg(reinterpret_cast<const uint2 *>(v_row) + lane);      // channels 4*lane .. 4*lane+3
+    const uint16_t h[4] = {(uint16_t)(raw.x & 0xffffu), (uint16_t)(raw.x >> 16), (uint16_t)(raw.y & 0xffffu),
+                           (uint16_t)(raw.y >> 16)};
+#pragma unroll
+    for (int i = 0; i < 4; ++i)
+        *reinterpret_cast<uint16_t *>(chunk + value_half_off(cl, tt, lane * 4 + i)) = h[i];
+}
+
+// Eq. 4 (or, for an fp16-value cache, the plain copy) of one row by one warp.
+__device__ __forceinline__ void store_value_row(const uint16_t *__restrict__ v_row, unsigned char *chunk,
+                                                const ChunkLayout &cl, int tt, int lane) {
+    if (cl.groups == 0) store_row_f16(v_row, chunk, cl, tt, lane);
+    else quantize_row(v_row, chunk, cl, tt, lane);
+}
+
 // One launch prepares a decode step (or only appends, or only sketches queries). Block ranges:
 //   [0, k_blocks)              key tiles: Eq. 2 on new keys, written into the cache   (ap.k != null)
 //   [k_blocks, +q_blocks)      query tiles: Eq. 2 on the queries, written to qwords   (sp.q != null)
@@ -195,7 +213,7 @@ __global__ void __launch_bounds__(kProjThreads) prepare_kernel(AppendParams ap, 
                 const int t = ap.len[layer * ap.max_batch + b] + tn;
                 unsigned char *chunk = ap.cache + ((size_t)(layer * ap.max_batch + b) * ap.Hkv + kvh) * ap.slab_bytes +
                                        (size_t)(t >> 5) * cl.bytes;
-                quantize_row(ap.v + row * kHeadDim, chunk, cl, t & 31, threadIdx.x & 31);
+                store_value_row(ap.v + row * kHeadDim, chunk, cl, t & 31, threadIdx.x & 31);
             }
         }
     }
@@ -349,7 +367,39 @@ __global__ void __launch_bounds__(kPrefillThreads, 2) prefill_kernel(PrefillPara
             const int tn0 = pos0 - len0;
             unsigned char *chunk = slab + (size_t)(pos0 >> 5) * cl.bytes;
             const int vb = (pos0 >> 4) & 1;
-            if (tn0 >= 0 && tn0 + 16 <= n_new) {                // a whole block: assemble it in shared memory
+            if (p.groups == 0 && tn0 >= 0 && tn0 + 16 <= n_new) {
+                // fp16 values, a whole block of 16 tokens: transposed through shared memory into the A-operand
+                // order, 32 channels (two channel blocks, 1024 contiguous bytes of the cache) per pass
+                unsigned char *vs = Vs + warp * 1280;
+                const size_t row_stride = (size_t)p.Hkv * kHeadDim;
+                const uint16_t *v0 = p.v + ((((size_t)ll * p.B + b) * p.Tn + tn0) * p.Hkv + kvh) * kHeadDim;
+                unsigned char *dst_block = chunk + cl.val_off + vb * kHalfBlockBytes;
+#pragma unroll 1
+                for (int pass = 0; pass < 4; ++pass) {
+                    uint4 raw[2];
+#pragma unroll
+                    for (int i = 0; i < 2; ++i) {               // piece e: token e/4, channels pass*32 + (e%4)*8 .. +7
+                        const int e = lane + 32 * i;
+                        raw[i] = __ldg(reinterpret_cast<const uint4 *>(v0 + (size_t)(e >> 2) * row_stride + pass * 32) + (e & 3));
+                    }
+#pragma unroll
+                    for (int i = 0; i < 2; ++i) {
+                        const int e = lane + 32 * i, k = e >> 2, c16 = e & 3;
+                        const int j = (k & 7) >> 1, odd = k & 1, hi8 = k >> 3;
+                        unsigned char *base = vs + (c16 >> 1) * 512 + j * 16 + (hi8 * 2 + (c16 & 1)) * 4 + odd * 2;
+                        const uint32_t w4[4] = {raw[i].x, raw[i].y, raw[i].z, raw[i].w};
+#pragma unroll
+                        for (int x = 0; x < 8; ++x)             // channel row r = x of the channel block
+                            *reinterpret_cast<uint16_t *>(base + x * 64) = (uint16_t)(w4[x >> 1] >> ((x & 1) * 16));
+                    }
+                    __syncwarp();
+                    const uint4 *src = reinterpret_cast<const uint4 *>(vs);
+                    uint4 *dst = reinterpret_cast<uint4 *>(dst_block + pass * 1024);
+                    dst[lane] = src[lane];
+                    dst[32 + lane] = src[32 + lane];
+                    __syncwarp();
+                }
+            } else if (p.groups != 0 && tn0 >= 0 && tn0 + 16 <= n_new) {   // a whole block: assemble it in shared memory
                 // lane = (row rsub of 8, group grp of 4): 32 channels of one row per lane and pass, two passes
                 unsigned char *vs = Vs + warp * 1280;
                 const int rsub = lane >> 2, grp = lane & 3;
@@ -424,8 +474,8 @@ __global__ void __launch_bounds__(kPrefillThreads, 2) prefill_kernel(PrefillPara
                 for (int k = 0; k < 16; ++k) {
                     const int tn = tn0 + k;
                     if (tn >= 0 && tn < n_new)
-                        quantize_row(p.v + ((((size_t)ll * p.B + b) * p.Tn + tn) * p.Hkv + kvh) * kHeadDim,
-                                     slab + (size_t)((pos0 + k) >> 5) * cl.bytes, cl, (pos0 + k) & 31, lane);
+                        store_value_row(p.v + ((((size_t)ll * p.B + b) * p.Tn + tn) * p.Hkv + kvh) * kHeadDim,
+                                        slab + (size_t)((pos0 + k) >> 5) * cl.bytes, cl, (pos0 + k) & 31, lane);
                 }
             }
         }
@@ -536,13 +586,15 @@ __global__ void set_len_kernel(int32_t *len, int n_layers, int max_batch, int se
 constexpr int kDecodeWarps = H1B_DECODE_WARPS;
 constexpr int kStages = H1B_DECODE_STAGES;
 // Resident blocks per SM that the register allocation must allow: the kernel hides latency with warps.
-constexpr int decode_min_blocks(int gq) { return gq == 1 ? 5 : (gq == 2 ? 4 : 3); }
+constexpr int decode_min_blocks(int gq, int ng) { return ng == 0 ? 3 : (gq == 1 ? 5 : (gq == 2 ? 4 : 3)); }
 constexpr int kHamSentinel = 1 << 20;
 
-template <int MW, int GQ, int NG>                 // NG: scale/zero pairs per value vector (4 or 1)
+template <int MW, int GQ, int NG>                 // NG: scale/zero pairs per value vector (4 or 1); 0 = fp16 values
 struct DecodeSmem {
-    static constexpr int kChunkBytes = MW * 128 + 2048 + 128 * NG;
-    static constexpr int kPerWarp = kStages * kChunkBytes + GQ * 32 * 4 + 128;   // ring, p buffer, barriers
+    static constexpr int kChunkBytes = MW * 128 + (NG == 0 ? 8192 : 2048 + 128 * NG);
+    // fp16-value chunks are four times larger: two in flight per warp, so that three blocks still fit an SM
+    static constexpr int kNStages = (NG == 0 && kStages > 2) ? 2 : kStages;
+    static constexpr int kPerWarp = kNStages * kChunkBytes + GQ * 32 * 4 + 128;   // ring, p buffer, barriers
     static constexpr int kTotal = kDecodeWarps * kPerWarp;
 };
 
@@ -551,7 +603,7 @@ struct DecodeState {
     float acc[8][4];            // per channel block of 16: C fragment (rows r, r+8; columns 2jq, 2jq+1)
     int hmin[GQ];               // running minimum Hamming distance (= running maximum logit)
     float ssum[GQ];             // per-lane partial sum of the weights
-    float accz[GQ][NG];         // per-lane partial sum of p * zero
+    float accz[GQ][NG ? NG : 1]; // per-lane partial sum of p * zero (unused with fp16 values)
     uint32_t qw[GQ][MW];        // query sketches
     float zero[4];              // an opaque quad of zeros: C operand of each chunk's first MMA
 };
@@ -570,8 +622,10 @@ __device__ __forceinline__ void decode_chunk(DecodeState<MW, GQ, NG> &st, const 
     uint32_t kw[MW];
 #pragma unroll
     for (int w = 0; w < MW; ++w) kw[w] = *reinterpret_cast<const uint32_t *>(ch + w * 128 + lane * 4);
-    float zf[NG];
-    if (NG == 4) {
+    float zf[NG ? NG : 1];
+    if (NG == 0) {
+        zf[0] = 0.f;
+    } else if (NG == 4) {
         const uint2 zraw = *reinterpret_cast<const uint2 *>(ch + ZERO + lane * 8);
         const float2 z01 = half2_bits_to_float2(zraw.x), z23 = half2_bits_to_float2(zraw.y);
         zf[0] = z01.x; zf[NG > 1 ? 1 : 0] = z01.y; zf[NG > 2 ? 2 : 0] = z23.x; zf[NG > 3 ? 3 : 0] = z23.y;
@@ -607,6 +661,52 @@ __device__ __forceinline__ void decode_chunk(DecodeState<MW, GQ, NG> &st, const 
     else if (GQ == 2) { f0 = scl[0]; f1 = scl[GQ > 1 ? 1 : 0]; }
     else { f0 = (jq & 1) ? scl[GQ > 2 ? 2 : 0] : scl[0]; f1 = (jq & 1) ? scl[GQ > 3 ? 3 : 0] : scl[GQ > 1 ? 1 : 0]; }
     __syncwarp();
+
+    if constexpr (NG == 0) {
+        // ---------------- phase 2, fp16 values: out^T (channels x columns) += V^T x W with A = the cached values as
+        // they are (one 16-byte load per channel block and lane) and B = the weights p split into hi and lo parts;
+        // column n = lane/4 = (part, head). Same per-chunk zero start and fold as below.
+        const int part = lane >> 4, idx = (lane >> 2) & 3;
+        const int bhead = idx < GQ ? idx : 0;                   // columns of heads the group does not have: ignored
+        const int tp = 2 * jq + 8 * part;
+        uint32_t bf[2][2];
+#pragma unroll
+        for (int vb = 0; vb < 2; ++vb) {
+            const float2 pp = *reinterpret_cast<const float2 *>(p_s + bhead * 32 + vb * 16 + tp);
+            const uint32_t hi = pack_f16x2(pp.x, pp.y);
+            const float2 hf = half2_bits_to_float2(hi);
+            const uint32_t lo = pack_f16x2((pp.x - hf.x) * 2048.f, (pp.y - hf.y) * 2048.f);
+            const uint32_t got = __shfl_xor_sync(0xffffffffu, part ? hi : lo, 16);
+            bf[vb][0] = part ? got : hi;
+            bf[vb][1] = part ? lo : got;
+        }
+        const float g0 = (jq & 1) ? (GQ > 2 ? scl[GQ > 2 ? 2 : 0] : 1.f) : scl[0];
+        const float g1 = (jq & 1) ? (GQ > 3 ? scl[GQ > 3 ? 3 : 0] : 1.f) : (GQ > 1 ? scl[GQ > 1 ? 1 : 0] : 1.f);
+#pragma unroll
+        for (int half = 0; half < 2; ++half) {
+            float tmp[4][4];
+#pragma unroll
+            for (int vb = 0; vb < 2; ++vb) {
+#pragma unroll
+                for (int i = 0; i < 4; ++i) {
+                    const int cb = half * 4 + i;
+                    const uint4 a = *reinterpret_cast<const uint4 *>(ch + VAL + vb * kHalfBlockBytes + cb * 512 + lane * 16);
+                    if (vb == 0) mma_f16_16816_from(tmp[i], a.x, a.y, a.z, a.w, bf[vb][0], bf[vb][1], st.zero);
+                    else mma_f16_16816(tmp[i], a.x, a.y, a.z, a.w, bf[vb][0], bf[vb][1]);
+                }
+            }
+#pragma unroll
+            for (int i = 0; i < 4; ++i) {
+                const int cb = half * 4 + i;
+                st.acc[cb][0] = fmaf(st.acc[cb][0], g0, tmp[i][0]);
+                st.acc[cb][1] = fmaf(st.acc[cb][1], g1, tmp[i][1]);
+                st.acc[cb][2] = fmaf(st.acc[cb][2], g0, tmp[i][2]);
+                st.acc[cb][3] = fmaf(st.acc[cb][3], g1, tmp[i][3]);
+            }
+        }
+        __syncwarp();
+        return;
+    }
 
     // ---------------- phase 2
     // Column n = lane/4 of a B fragment is (part, idx): part 0 = hi, part 1 = lo; idx = value group (GQ 1),
@@ -668,9 +768,10 @@ __device__ __forceinline__ void decode_chunk(DecodeState<MW, GQ, NG> &st, const 
 }
 
 template <int MW, int GQ, int NG>
-__global__ void __launch_bounds__(kDecodeWarps * 32, decode_min_blocks(GQ)) decode_split_kernel(DecodeParams p) {
+__global__ void __launch_bounds__(kDecodeWarps * 32, decode_min_blocks(GQ, NG)) decode_split_kernel(DecodeParams p) {
     using SM = DecodeSmem<MW, GQ, NG>;
     constexpr int CB = SM::kChunkBytes;
+    constexpr int kStages = SM::kNStages;                       // shadows the build-time default
     extern __shared__ __align__(128) unsigned char smem_raw[];
 
     const int lane = threadIdx.x & 31, warp = threadIdx.x >> 5;
@@ -784,7 +885,8 @@ __global__ void __launch_bounds__(kDecodeWarps * 32, decode_min_blocks(GQ)) deco
     // Undo the scales: codes were fed as code / kCodeScaleLo (rows r) and code / kCodeScaleHi (rows r + 8), the
     // weights carry a factor 2, and the low parts a further 2^11. Everything below is in units of 2p, like ssum and accz, so
     // the common factor 2 cancels in the final division.
-    constexpr float kRowLo = kCodeScaleLo, kRowHi = kCodeScaleHi, kLoPart = 1.f / 2048.f;
+    // (fp16 values: A held the values themselves, so only the low parts' 2^11 is undone and there is no zero-point term.)
+    constexpr float kRowLo = NG ? kCodeScaleLo : 1.f, kRowHi = NG ? kCodeScaleHi : 1.f, kLoPart = 1.f / 2048.f;
     float *part_out = p.partial + (size_t)item * GQ * kPartStride;
     const int r = lane >> 2, jq = lane & 3;
 #pragma unroll
@@ -796,8 +898,19 @@ __global__ void __launch_bounds__(kDecodeWarps * 32, decode_min_blocks(GQ)) deco
             const float hi = (jq & 2) ? other : st.acc[cb][i], lo = (jq & 2) ? st.acc[cb][i] : other;
             v[i] = fmaf(lo, kLoPart, hi) * (i < 2 ? kRowLo : kRowHi);
         }
-        const int g = cb >> 1, gz = (NG == 1) ? 0 : g;          // gz: which zero-point sum belongs to this channel block
-        if (GQ == 1) {
+        const int g = cb >> 1, gz = (NG <= 1) ? 0 : g;          // gz: which zero-point sum belongs to this channel block
+        if (NG == 0) {                                          // columns 2jq, 2jq+1 = heads 2jq, 2jq+1 (lanes jq < 2)
+            if (jq < 2) {
+#pragma unroll
+                for (int hh = 0; hh < 2; ++hh) {
+                    if (2 * jq + hh < GQ) {
+                        float *dst = part_out + (size_t)(2 * jq + hh) * kPartStride;
+                        dst[cb * 16 + r] = v[hh];
+                        dst[cb * 16 + r + 8] = v[2 + hh];
+                    }
+                }
+            }
+        } else if (GQ == 1) {
             if (jq == (g >> 1)) {
                 part_out[cb * 16 + r] = v[g & 1] + st.accz[0][gz];
                 part_out[cb * 16 + r + 8] = v[2 + (g & 1)] + st.accz[0][gz];
@@ -1022,6 +1135,10 @@ cudaError_t launch_decode(const DecodeParams &p, cudaStream_t st, int *launches,
             if (gq == 1) e = launch_decode_t<MW, 1, 1>(p, st);
             else if (gq == 2) e = launch_decode_t<MW, 2, 1>(p, st);
             else if (gq == 4) e = launch_decode_t<MW, 4, 1>(p, st);
+        } else if (p.groups == 0) {
+            if (gq == 1) e = launch_decode_t<MW, 1, 0>(p, st);
+            else if (gq == 2) e = launch_decode_t<MW, 2, 0>(p, st);
+            else if (gq == 4) e = launch_decode_t<MW, 4, 0>(p, st);
         }
     );
     if (e != cudaSuccess) return e;

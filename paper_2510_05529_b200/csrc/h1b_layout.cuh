@@ -25,6 +25,14 @@
 // groups = 128 / group_size: 4 (groups of 32 channels) or 1 (one scale and zero per value vector, the
 // per-vector scheme of Section IV-B). Bytes per token: m/8 + 64 + 4 * groups, the count of Section IV-B's
 // storage statement plus the fp16 scale and zero of each group.
+//
+// groups = 0 selects the "1-bit keys only" configuration of the ablation (Table V): values stay fp16.
+//   chunk = [ key words ][ values ]
+//   values      2 blocks of 16 tokens x 128 channels x fp16 = 2 x 4096 B, each again in A-operand order:
+//               [channel block cb 0..7][lane 0..31][4 words]; word i of lane (r = lane/4, j = lane%4) holds
+//               channel cb*16 + r + 8*(i&1), tokens 2j + 8*(i>>1) (low half) and 2j + 8*(i>>1) + 1 (high half),
+//               so a decode lane fetches the four A registers of a channel block with one 16-byte load.
+// Bytes per token: m/8 + 256.
 #pragma once
 #include <cstdint>
 #include <cstddef>
@@ -36,11 +44,12 @@ constexpr int kGroup = 32;
 constexpr int kGroups = kHeadDim / kGroup;       // 4: the most groups a value vector can have
 constexpr int kChunkTokens = 32;
 constexpr int kValBlockBytes = 1024;             // 16 tokens x 128 channels x 4 bit
+constexpr int kHalfBlockBytes = 4096;            // 16 tokens x 128 channels x fp16 (groups == 0)
 constexpr int kPartStride = 132;                 // floats per (item, head): acc[128], min Hamming, sum, pad
 
 struct ChunkLayout {
     int m_words;      // m / 32
-    int groups;       // scale/zero pairs per value vector: 4 or 1
+    int groups;       // scale/zero pairs per value vector: 4 or 1; 0 = fp16 values, no scale or zero
     int val_off;      // byte offset of the value codes
     int zero_off;
     int scale_off;
@@ -52,7 +61,7 @@ __host__ __device__ inline ChunkLayout chunk_layout(int m_words, int groups) {
     c.m_words = m_words;
     c.groups = groups;
     c.val_off = m_words * 4 * kChunkTokens;
-    c.zero_off = c.val_off + 2 * kValBlockBytes;
+    c.zero_off = c.val_off + 2 * (groups == 0 ? kHalfBlockBytes : kValBlockBytes);
     c.scale_off = c.zero_off + kChunkTokens * groups * 2;
     c.bytes = c.scale_off + kChunkTokens * groups * 2;
     return c;
@@ -68,6 +77,13 @@ __host__ __device__ inline int code_byte_off(const ChunkLayout &c, int tt, int c
     int j = (k & 7) >> 1, odd = k & 1, hi8 = k >> 3;
     int lane = r * 4 + j;
     return c.val_off + vb * kValBlockBytes + (cb >> 2) * 512 + lane * 16 + (cb & 3) * 4 + odd * 2 + hi8;
+}
+// groups == 0: byte offset, inside a chunk, of the fp16 value of channel ch (0..127) of token tt.
+__host__ __device__ inline int value_half_off(const ChunkLayout &c, int tt, int ch) {
+    int vb = tt >> 4, k = tt & 15;
+    int j = (k & 7) >> 1, odd = k & 1, hi8 = k >> 3;
+    int cb = ch >> 4, r = ch & 7, hi = (ch >> 3) & 1;
+    return c.val_off + vb * kHalfBlockBytes + cb * 512 + (r * 4 + j) * 16 + (hi8 * 2 + hi) * 4 + odd * 2;
 }
 __host__ __device__ inline int zero_off(const ChunkLayout &c, int tt, int g) {
     return c.zero_off + tt * (2 * c.groups) + g * 2;
