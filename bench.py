@@ -135,7 +135,7 @@ def run_ours(args):
     if args.workload == "c5_prefill":
         return run_prefill(args, w, pdist, rank, world, local)
     steps, warmup = args.steps, args.warmup
-    total_steps = 2 * (steps + warmup) + 8           # device-resident run, then the host-buffer run
+    total_steps = 3 * (steps + warmup) + 16          # device-resident run, the host-buffer run, the per-layer graph run
     lens0 = h1b_synth.lengths(w) - 1                  # the first step decodes exactly the workload's context
     cfg = binding.make_config(w.n_layers, w.n_q_heads, w.n_kv_heads, w.head_dim, w.sketch_bits, w.group_size,
                               max_batch=w.batch, max_seq=w.context - 1 + total_steps, device=local,
@@ -210,7 +210,39 @@ def run_ours(args):
     barrier()
     e2e_ms_total = e0.elapsed_time(e1)
 
+    # layer-sequential: one (append + attention) call per layer, the order a model that runs its layers one
+    # after the other imposes, recorded once into a CUDA graph (3 kernels per layer) and replayed
+    seq_ms_total = None
+    if not args.no_layer_sequential:
+        pdist.barrier()
+        cache.h1b_sync_lengths()
+        ks, vs, qs = kn[0].clone(), vn[0].clone(), qn[0].clone()
+
+        def per_layer():
+            for l in range(w.n_layers):
+                cache.h1b_decode_step_layers(l, ks[l:l + 1], vs[l:l + 1], qs[l:l + 1], INV_TAU, out=out[l:l + 1])
+
+        per_layer()
+        torch.cuda.synchronize()
+        graph = torch.cuda.CUDAGraph()
+        with torch.cuda.graph(graph, capture_error_mode="thread_local"):   # other threads (NCCL's watchdog) may call CUDA
+            per_layer()
+        for i in range(min(warmup, 8)):
+            graph.replay()
+        barrier()
+        g0, g1 = torch.cuda.Event(enable_timing=True), torch.cuda.Event(enable_timing=True)
+        g0.record(stream)
+        for i in range(steps):
+            graph.replay()
+        g1.record(stream)
+        barrier()
+        seq_ms_total = g0.elapsed_time(g1)
+        cache.h1b_sync_lengths()
+        cache.h1b_poll_status()
+
     ms_total, e2e_ms_total = pdist.max_over_ranks([ms_total, e2e_ms_total], dev)     # slowest rank
+    if seq_ms_total is not None:
+        seq_ms_total = pdist.max_over_ranks([seq_ms_total], dev)[0]
     ms_per_step = ms_total / steps
     value = pdist.whole_job_rate(w.batch, world, ms_per_step * 1e-3)
     e2e_value = pdist.whole_job_rate(w.batch, world, e2e_ms_total / steps * 1e-3)
@@ -251,6 +283,10 @@ def run_ours(args):
         "clocks": clocks,
         "roofline": roofline,
     }
+    if seq_ms_total is not None:                      # not the headline: the same step issued layer by layer
+        line["layer_sequential"] = {"value": pdist.whole_job_rate(w.batch, world, seq_ms_total / steps * 1e-3), "unit": UNIT,
+                                    "ms_per_step": seq_ms_total / steps, "launches_per_step": 3 * w.n_layers,
+                                    "how": "h1b_decode_step_layers once per layer, one CUDA graph per step, replayed"}
     if rank == 0 and world == 1 and not args.no_cpu_baseline and w.name == "c2_7b_8k":
         line["cpu_baseline"] = cpu_baseline(sample_layers=1, steps=5, warmup=1)
     cache.close()
@@ -387,6 +423,7 @@ def main():
     ap.add_argument("--no-cpu-baseline", action="store_true")
     ap.add_argument("--sketch-bits", type=int, default=0, help="override m (64, 128, 256, 512)")
     ap.add_argument("--group-size", type=int, default=0, help="override G (32, or 128 = one scale per value vector)")
+    ap.add_argument("--no-layer-sequential", action="store_true", help="skip the per-layer CUDA-graph measurement")
     ap.add_argument("--fp16-values", action="store_true", help="keep values in fp16 (the 1-bit-keys-only ablation row)")
     ap.add_argument("--workload", default="c2_7b_8k",
                     choices=["c2_7b_8k", "c3_7b_batched", "c4_gqa_32k", "c5_prefill"],

@@ -129,6 +129,30 @@ int h1b_decode_attention(h1b_ctx *ctx, int layer_begin, int n_layers, const void
 int h1b_decode_step(h1b_ctx *ctx, const void *k, const void *v, const void *q, float inv_tau,
                     void *out, int B, void *stream);
 
+/* The same for layers [layer_begin, layer_begin + n_layers) only: what a model
+ * that runs its layers one after the other calls once per layer.
+ *   k, v  DEVICE: fp16 [n_layers][B][1][Hkv][d]   q  DEVICE: fp16 [n_layers][B][Hq][d]
+ *   out   DEVICE: float32 [n_layers][B][Hq][d] */
+int h1b_decode_step_layers(h1b_ctx *ctx, int layer_begin, int n_layers, const void *k,
+                           const void *v, const void *q, float inv_tau, void *out, int B,
+                           void *stream);
+
+/* Stream capture. h1b_append_kv(), h1b_decode_attention(), h1b_decode_step() and
+ * h1b_decode_step_layers() only enqueue kernels, so they may be recorded into a
+ * CUDA graph (make one ordinary call of each kind first: the first call sets
+ * kernel attributes). The kernels read the sequence lengths from device memory,
+ * so every replay appends at, and attends up to, the then-current end of each
+ * sequence. Frozen at capture time: the pointers, B, n_new and the split plan
+ * (its last split is open-ended, so growth is still covered). The host's copy of
+ * the lengths only sees the captured calls, not their replays: call
+ * h1b_sync_lengths() after replaying and before any other call on the context.
+ * A replay that finds a sequence full writes nothing for it, leaves its length
+ * alone and raises H1B_ERR_CAPACITY at the next h1b_poll_status().
+ *
+ * h1b_sync_lengths: copy the device's lengths into the host's copy; synchronises
+ * `stream`. */
+int h1b_sync_lengths(h1b_ctx *ctx, void *stream);
+
 /* h1b_decode_attention() for callers that must not allocate and cannot spare
  * scratch of their own. (No counterpart in the paper: this is a deployment
  * convenience, not a step of the method.)
@@ -223,8 +247,9 @@ int h1b_debug_scores(h1b_ctx *ctx, int layer, int seq, int kv_head, const void *
  * H1B_ERR_INVALID_ARG if the split-K scratch cannot hold that many. */
 int h1b_set_splits(h1b_ctx *ctx, int splits);
 
-/* After the stream has been synchronised: 0, or H1B_ERR_TIMEOUT if a kernel
- * gave up a bounded wait since the last poll (the flag is cleared). */
+/* After the stream has been synchronised: 0, H1B_ERR_TIMEOUT if a kernel gave
+ * up a bounded wait since the last poll, or H1B_ERR_CAPACITY if a replayed append
+ * found a sequence full (the flag is cleared). */
 int h1b_poll_status(h1b_ctx *ctx);
 
 /* Time the dominant kernel. While enabled, every h1b_decode_attention() brackets

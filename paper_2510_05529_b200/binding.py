@@ -64,6 +64,9 @@ def load_library(rebuild: bool = True) -> ctypes.CDLL:
         "h1b_decode_attention_static": (ctypes.c_int, [vp, ctypes.c_int, ctypes.c_int, vp, ctypes.c_float, vp,
                                                        ctypes.c_int, vp]),
         "h1b_decode_step": (ctypes.c_int, [vp, vp, vp, vp, ctypes.c_float, vp, ctypes.c_int, vp]),
+        "h1b_decode_step_layers": (ctypes.c_int, [vp, ctypes.c_int, ctypes.c_int, vp, vp, vp, ctypes.c_float, vp,
+                                                  ctypes.c_int, vp]),
+        "h1b_sync_lengths": (ctypes.c_int, [vp, vp]),
         "h1b_decode_step_host": (ctypes.c_int, [vp, vp, vp, vp, ctypes.c_float, vp, ctypes.c_int, vp]),
         "h1b_free": (ctypes.c_int, [vp]),
         "h1b_get_projection": (ctypes.c_int, [vp, ctypes.c_int, vp]),
@@ -208,6 +211,26 @@ class H1BCache:
         op = _dev_ptr(out, torch.float32, "out")
         self._check(self.lib.h1b_decode_step(self._h, kp, vp, qp, float(inv_tau), op, B, _stream_ptr(stream)))
         return out
+
+    def h1b_decode_step_layers(self, layer_begin: int, k: torch.Tensor, v: torch.Tensor, q: torch.Tensor,
+                               inv_tau: float, out: torch.Tensor | None = None, stream=None) -> torch.Tensor:
+        """The step for layers [layer_begin, layer_begin + n): k, v fp16 CUDA [n, B, 1, Hkv, d],
+        q fp16 CUDA [n, B, Hq, d] -> out fp32 [n, B, Hq, d]."""
+        kp, vp, qp = _dev_ptr(k, torch.float16, "k"), _dev_ptr(v, torch.float16, "v"), _dev_ptr(q, torch.float16, "q")
+        n, B = int(q.shape[0]), int(q.shape[1])
+        if tuple(k.shape) != (n, B, 1, self.cfg.n_kv_heads, self.cfg.head_dim) or k.shape != v.shape or \
+                tuple(q.shape) != (n, B, self.cfg.n_q_heads, self.cfg.head_dim):
+            raise ValueError("step shapes: k, v [n, B, 1, Hkv, d]; q [n, B, Hq, d]")
+        if out is None:
+            out = torch.empty(q.shape, dtype=torch.float32, device=q.device)
+        op = _dev_ptr(out, torch.float32, "out")
+        self._check(self.lib.h1b_decode_step_layers(self._h, layer_begin, n, kp, vp, qp, float(inv_tau), op, B,
+                                                    _stream_ptr(stream)))
+        return out
+
+    def h1b_sync_lengths(self, stream=None):
+        """After replaying a captured graph that appends: refresh the host's copy of the lengths."""
+        self._check(self.lib.h1b_sync_lengths(self._h, _stream_ptr(stream)))
 
     def h1b_decode_attention_static(self, q: torch.Tensor, inv_tau: float, out: torch.Tensor,
                                     layer_begin: int = 0, stream=None) -> torch.Tensor:

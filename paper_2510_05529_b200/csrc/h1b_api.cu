@@ -250,10 +250,12 @@ static AppendParams append_params(h1b_ctx *ctx, int layer_begin, int n_layers, c
     p.cache = ctx->ws + ctx->plan.cache;
     p.len = at<int32_t>(ctx, ctx->plan.len);
     p.done = at<int32_t>(ctx, ctx->plan.status) + 4;
+    p.status = at<int32_t>(ctx, ctx->plan.status);
     p.slab_bytes = ctx->plan.slab_bytes;
     p.layer_begin = layer_begin; p.n_layers = n_layers; p.B = B; p.Tn = Tn;
     p.Hkv = ctx->cfg.n_kv_heads; p.max_batch = ctx->cfg.max_batch; p.m_words = ctx->plan.m_words;
     p.groups = ctx->plan.groups;
+    p.max_seq = ctx->cfg.max_seq;
     return p;
 }
 
@@ -389,26 +391,39 @@ int h1b_decode_attention(h1b_ctx *ctx, int layer_begin, int n_layers, const void
     return rc;
 }
 
-int h1b_decode_step(h1b_ctx *ctx, const void *k, const void *v, const void *q, float inv_tau, void *out, int B,
-                    void *stream) {
-    if (!ctx) return H1B_ERR_NULL;
-    const int L = ctx->cfg.n_layers;
-    int rc = check_decode_args(ctx, 0, L, q, inv_tau, out, B);
+int h1b_decode_step_layers(h1b_ctx *ctx, int layer_begin, int n_layers, const void *k, const void *v, const void *q,
+                           float inv_tau, void *out, int B, void *stream) {
+    int rc = check_decode_args(ctx, layer_begin, n_layers, q, inv_tau, out, B);
     if (rc != H1B_OK) return rc;
     if (!k || !v) return fail(ctx, H1B_ERR_NULL, "k or v is NULL");
     NewCounts nn;
-    rc = make_new_counts(ctx, 0, L, nullptr, B, 1, &nn);
+    rc = make_new_counts(ctx, layer_begin, n_layers, nullptr, B, 1, &nn);
     if (rc != H1B_OK) return rc;
     cudaStream_t st = static_cast<cudaStream_t>(stream);
     int launches = 0;
-    const AppendParams ap = append_params(ctx, 0, L, k, v, B, 1);
-    const SketchParams sp = sketch_params(ctx, 0, L, q, B, at<uint32_t>(ctx, ctx->plan.qwords));
+    const AppendParams ap = append_params(ctx, layer_begin, n_layers, k, v, B, 1);
+    const SketchParams sp = sketch_params(ctx, layer_begin, n_layers, q, B, at<uint32_t>(ctx, ctx->plan.qwords));
     H1B_CUDA(ctx, launch_prepare(&ap, &sp, nn, st, &launches));
-    commit_lengths(ctx, 0, L, B, nn);
-    rc = enqueue_decode(ctx, 0, L, inv_tau, out, B, st, sp.qwords, at<float>(ctx, ctx->plan.partial),
+    commit_lengths(ctx, layer_begin, n_layers, B, nn);
+    rc = enqueue_decode(ctx, layer_begin, n_layers, inv_tau, out, B, st, sp.qwords, at<float>(ctx, ctx->plan.partial),
                         at<int32_t>(ctx, ctx->plan.arrive), ctx->plan.partial_items, true, &launches);
     ctx->launches += launches;
     return rc;
+}
+
+int h1b_decode_step(h1b_ctx *ctx, const void *k, const void *v, const void *q, float inv_tau, void *out, int B,
+                    void *stream) {
+    if (!ctx) return H1B_ERR_NULL;
+    return h1b_decode_step_layers(ctx, 0, ctx->cfg.n_layers, k, v, q, inv_tau, out, B, stream);
+}
+
+int h1b_sync_lengths(h1b_ctx *ctx, void *stream) {
+    if (!ctx) return H1B_ERR_NULL;
+    cudaStream_t st = static_cast<cudaStream_t>(stream);
+    H1B_CUDA(ctx, cudaMemcpyAsync(ctx->len_host.data(), at<int32_t>(ctx, ctx->plan.len),
+                                  ctx->len_host.size() * sizeof(int32_t), cudaMemcpyDeviceToHost, st));
+    H1B_CUDA(ctx, cudaStreamSynchronize(st));
+    return H1B_OK;
 }
 
 // ---------------------------------------------------------------------------
@@ -662,6 +677,8 @@ int h1b_poll_status(h1b_ctx *ctx) {
     H1B_CUDA(ctx, cudaMemcpy(&s, at<int32_t>(ctx, ctx->plan.status), sizeof s, cudaMemcpyDeviceToHost));
     if (s == kStatusOk) return H1B_OK;
     H1B_CUDA(ctx, cudaMemset(at<int32_t>(ctx, ctx->plan.status), 0, sizeof s));
+    if (s == kStatusCapacity)
+        return fail(ctx, H1B_ERR_CAPACITY, "a replayed append found a sequence full: its rows were dropped");
     return fail(ctx, H1B_ERR_TIMEOUT, "a kernel gave up a bounded wait (status %d)", s);
 }
 

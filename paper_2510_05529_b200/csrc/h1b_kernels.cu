@@ -182,7 +182,7 @@ __global__ void __launch_bounds__(kProjThreads) prepare_kernel(AppendParams ap, 
         const uint32_t bits = project_tile(sm, ap.k + ((size_t)ll * k_rows + row0) * kHeadDim, n_rows,
                                            ap.Rt + (size_t)layer * kHeadDim * m, m, word);
         if ((int)threadIdx.x < n_rows) {
-            if (tn < nn.v[b]) {
+            if (tn < nn.v[b] && len0 + nn.v[b] <= ap.max_seq) {
                 const int t = len0 + tn;
                 unsigned char *chunk = ap.cache + ((size_t)(layer * ap.max_batch + b) * ap.Hkv + kvh) * ap.slab_bytes +
                                        (size_t)(t >> 5) * cl.bytes;
@@ -208,9 +208,10 @@ __global__ void __launch_bounds__(kProjThreads) prepare_kernel(AppendParams ap, 
         if (row < rows) {
             const int kvh = (int)(row % ap.Hkv), tn = (int)((row / ap.Hkv) % ap.Tn);
             const int b = (int)((row / ((long)ap.Hkv * ap.Tn)) % ap.B), ll = (int)(row / k_rows);
-            if (tn < nn.v[b]) {
-                const int layer = ap.layer_begin + ll;
-                const int t = ap.len[layer * ap.max_batch + b] + tn;
+            const int layer = ap.layer_begin + ll;
+            const int len0 = ap.len[layer * ap.max_batch + b];
+            if (tn < nn.v[b] && len0 + nn.v[b] <= ap.max_seq) {
+                const int t = len0 + tn;
                 unsigned char *chunk = ap.cache + ((size_t)(layer * ap.max_batch + b) * ap.Hkv + kvh) * ap.slab_bytes +
                                        (size_t)(t >> 5) * cl.bytes;
                 store_value_row(ap.v + row * kHeadDim, chunk, cl, t & 31, threadIdx.x & 31);
@@ -227,8 +228,12 @@ __global__ void __launch_bounds__(kProjThreads) prepare_kernel(AppendParams ap, 
     }
     __syncthreads();
     if (is_last) {
-        for (int i = threadIdx.x; i < ap.n_layers * ap.B; i += blockDim.x)
-            ap.len[(ap.layer_begin + i / ap.B) * ap.max_batch + (i % ap.B)] += nn.v[i % ap.B];
+        for (int i = threadIdx.x; i < ap.n_layers * ap.B; i += blockDim.x) {
+            int32_t *len = ap.len + (ap.layer_begin + i / ap.B) * ap.max_batch + (i % ap.B);
+            const int n = nn.v[i % ap.B];
+            if (*len + n <= ap.max_seq) *len += n;
+            else atomicExch(ap.status, kStatusCapacity);        // full: nothing of this sequence's rows was written
+        }
         if (threadIdx.x == 0) *ap.done = 0;
     }
 }
@@ -982,10 +987,15 @@ __global__ void __launch_bounds__(kDecodeWarps * 32, decode_min_blocks(GQ, NG)) 
 #endif
 }
 
-// Flash-decoding combine: one block per (layer, sequence, query head), one thread per channel, merges the
-// partials of the sequence's non-empty splits. An empty sequence gives zeros.
+// Flash-decoding combine: one block per (layer, sequence, query head) merges the partials of the sequence's
+// non-empty splits. Warp w takes splits w, w+4, ...; a lane owns four channels (one 16-byte load per split), so
+// the loads of a warp's splits are independent and overlap; the four warps' sums meet in shared memory.
+// An empty sequence gives zeros.
 __global__ void __launch_bounds__(kHeadDim) combine_kernel(DecodeParams p) {
-    const int c = threadIdx.x;
+    __shared__ float s_min[4];
+    __shared__ float s_den[4];
+    __shared__ __align__(16) float s_num[4][kHeadDim];
+    const int tid = threadIdx.x, lane = tid & 31, warp = tid >> 5;
     const int gq = p.Hq / p.Hkv;
     const int hq = blockIdx.x % p.Hq;
     const int b = (blockIdx.x / p.Hq) % p.B;
@@ -997,15 +1007,31 @@ __global__ void __launch_bounds__(kHeadDim) combine_kernel(DecodeParams p) {
     const int ns = min(p.splits, (len + p.split_tokens - 1) / p.split_tokens);
     const float *base = p.partial + ((size_t)slab_local * p.splits * gq + hh) * kPartStride;
     const size_t stride = (size_t)gq * kPartStride;
+    // the smallest Hamming distance any split saw (= the largest logit)
     float hm = 3.0e38f;
-    for (int j = 0; j < ns; ++j) hm = fminf(hm, base[j * stride + 128]);
-    float num = 0.f, den = 0.f;
-    for (int j = 0; j < ns; ++j) {
-        const float w = exp2f((hm - base[j * stride + 128]) * p.c2);
-        num = fmaf(w, base[j * stride + c], num);
-        den = fmaf(w, base[j * stride + 129], den);
+    for (int j = tid; j < ns; j += kHeadDim) hm = fminf(hm, base[j * stride + 128]);
+#pragma unroll
+    for (int o = 16; o > 0; o >>= 1) hm = fminf(hm, __shfl_xor_sync(0xffffffffu, hm, o));
+    if (lane == 0) s_min[warp] = hm;
+    __syncthreads();
+    hm = fminf(fminf(s_min[0], s_min[1]), fminf(s_min[2], s_min[3]));
+    float4 num = make_float4(0.f, 0.f, 0.f, 0.f);
+    float den = 0.f;
+#pragma unroll 4
+    for (int j = warp; j < ns; j += 4) {
+        const float *pj = base + j * stride;
+        const float wgt = exp2f((hm - pj[128]) * p.c2);
+        const float4 a = reinterpret_cast<const float4 *>(pj)[lane];
+        num.x = fmaf(wgt, a.x, num.x); num.y = fmaf(wgt, a.y, num.y);
+        num.z = fmaf(wgt, a.z, num.z); num.w = fmaf(wgt, a.w, num.w);
+        den = fmaf(wgt, pj[129], den);
     }
-    p.out[(size_t)blockIdx.x * kHeadDim + c] = (ns > 0) ? num / den : 0.f;
+    reinterpret_cast<float4 *>(s_num[warp])[lane] = num;
+    if (lane == 0) s_den[warp] = den;
+    __syncthreads();
+    const float n4 = (s_num[0][tid] + s_num[1][tid]) + (s_num[2][tid] + s_num[3][tid]);
+    const float d4 = (s_den[0] + s_den[1]) + (s_den[2] + s_den[3]);
+    p.out[(size_t)blockIdx.x * kHeadDim + tid] = (ns > 0) ? n4 / d4 : 0.f;
 }
 
 // Test helper: score of every cached token of one slab against one sketch.

@@ -95,6 +95,8 @@ __host__ __device__ inline int scale_off(const ChunkLayout &c, int tt, int g) {
 // Device status word values.
 constexpr int kStatusOk = 0;
 constexpr int kStatusWaitTimeout = 1;
+constexpr int kStatusCapacity = 2;      // an append found a sequence full (only reachable when a captured graph is replayed
+                                        // more often than the cache has room for: direct calls are checked on the host)
 
 struct NewCounts { int32_t v[256]; };            // n_new per sequence, passed by value
 
@@ -104,8 +106,10 @@ struct AppendParams {
     unsigned char *cache;       // slab 0
     int32_t *len;               // [L][max_batch]
     int32_t *done;              // block counter of the append launch (zero between launches)
+    int32_t *status;            // device status word
     size_t slab_bytes;
     int layer_begin, n_layers, B, Tn, Hkv, max_batch, m_words, groups;
+    int max_seq;                // capacity of a sequence: rows that would land at or beyond it are dropped and flagged
 };
 
 struct PrefillParams {          // long appends: tensor-core projection
