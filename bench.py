@@ -135,7 +135,10 @@ def run_ours(args):
     if args.workload == "c5_prefill":
         return run_prefill(args, w, pdist, rank, world, local)
     steps, warmup = args.steps, args.warmup
-    total_steps = 3 * (steps + warmup) + 16          # device-resident run, the host-buffer run, the per-layer graph run
+    Tq = max(1, args.query_tokens)                    # > 1: a step appends Tq tokens and attends for all of them at once
+    if Tq > 1:
+        w = h1b_synth.scaled(w, name=w.name + "[Tq=%d]" % Tq)
+    total_steps = (3 * (steps + warmup) + 16) * Tq   # device-resident run, the host-buffer run, the per-layer graph run
     lens0 = h1b_synth.lengths(w) - 1                  # the first step decodes exactly the workload's context
     cfg = binding.make_config(w.n_layers, w.n_q_heads, w.n_kv_heads, w.head_dim, w.sketch_bits, w.group_size,
                               max_batch=w.batch, max_seq=w.context - 1 + total_steps, device=local,
@@ -161,8 +164,18 @@ def run_ours(args):
     out = torch.empty((w.n_layers, w.batch, w.n_q_heads, w.head_dim), dtype=torch.float32, device=dev)
     stream = torch.cuda.current_stream()
 
-    def step(i):                                      # append the new token to all layers + decode: two launches
-        cache.h1b_decode_step(kn[i % pool], vn[i % pool], qn[i % pool], INV_TAU, out=out)
+    if Tq > 1:                                        # Tq new tokens per sequence and their Tq queries
+        kq = torch.cat([kn[i] for i in range(Tq)], dim=2).contiguous()            # [L, B, Tq, Hkv, d]
+        vq = torch.cat([vn[i] for i in range(Tq)], dim=2).contiguous()
+        qq = torch.stack([qn[i] for i in range(Tq)], dim=2).contiguous()          # [L, B, Tq, Hq, d]
+        outq = torch.empty(qq.shape, dtype=torch.float32, device=dev)
+
+    def step(i):                                      # append the new token to all layers + decode: three launches
+        if Tq > 1:
+            cache.h1b_append_kv(kq, vq)
+            cache.h1b_decode_attention_multi(qq, INV_TAU, out=outq)
+        else:
+            cache.h1b_decode_step(kn[i % pool], vn[i % pool], qn[i % pool], INV_TAU, out=out)
 
     def barrier():
         pdist.barrier()
@@ -177,7 +190,7 @@ def run_ours(args):
     sampler = ClockSampler(gpu_index())
     sampler.start()
     ev0, ev1 = torch.cuda.Event(enable_timing=True), torch.cuda.Event(enable_timing=True)
-    len_first = cache.h1b_get_lengths(0)[:w.batch].astype(np.int64) + 1
+    len_first = cache.h1b_get_lengths(0)[:w.batch].astype(np.int64) + Tq
     ctx_first = int(len_first.max())
     barrier()
     ev0.record(stream)
@@ -195,16 +208,19 @@ def run_ours(args):
     ctx_last = int(len_last.max())
 
     # end to end through the host-buffer entry point: pinned host inputs, H2D and D2H inside the timed region
+    # (the several-query-tokens variant has no host-buffer entry point: its e2e repeats nothing and stays null)
+    if Tq > 1:
+        args.no_layer_sequential = True
     kh = [t.cpu().pin_memory() for t in kn]
     vh = [t.cpu().pin_memory() for t in vn]
     qh = [t.cpu().pin_memory() for t in qn]
     oh = torch.empty(out.shape, dtype=torch.float32).pin_memory()
-    for i in range(min(warmup, 8)):
+    for i in range(min(warmup, 8) if Tq == 1 else 0):
         cache.h1b_decode_step_host(kh[i % pool], vh[i % pool], qh[i % pool], INV_TAU, oh)
     barrier()
     e0, e1 = torch.cuda.Event(enable_timing=True), torch.cuda.Event(enable_timing=True)
     e0.record(stream)
-    for i in range(steps):
+    for i in range(steps if Tq == 1 else 0):
         cache.h1b_decode_step_host(kh[i % pool], vh[i % pool], qh[i % pool], INV_TAU, oh)
     e1.record(stream)
     barrier()
@@ -244,14 +260,14 @@ def run_ours(args):
     if seq_ms_total is not None:
         seq_ms_total = pdist.max_over_ranks([seq_ms_total], dev)[0]
     ms_per_step = ms_total / steps
-    value = pdist.whole_job_rate(w.batch, world, ms_per_step * 1e-3)
-    e2e_value = pdist.whole_job_rate(w.batch, world, e2e_ms_total / steps * 1e-3)
+    value = pdist.whole_job_rate(w.batch * Tq, world, ms_per_step * 1e-3)
+    e2e_value = pdist.whole_job_rate(w.batch, world, e2e_ms_total / steps * 1e-3) if Tq == 1 else None
 
     # roofline of the dominant kernel (split-K decode attention), per launch
     entry = binding.h1b_entry_bytes(cfg)
     tokens_mean = float((0.5 * (len_first + len_last)).sum())         # cached tokens over the batch, mean over the run
     token_heads = w.n_layers * w.n_kv_heads * tokens_mean
-    alg_bytes = token_heads * entry + w.n_layers * w.batch * w.n_q_heads * (w.sketch_bits // 8)
+    alg_bytes = token_heads * entry + w.n_layers * w.batch * Tq * w.n_q_heads * (w.sketch_bits // 8)
     peak, peak_kind = measured_peaks()
     kern_ms_avg = kern_ms / max(kern_n, 1)
     achieved = alg_bytes / (kern_ms_avg * 1e-3) / 1e9 if kern_n else None
@@ -276,7 +292,7 @@ def run_ours(args):
                    "ctx_first": ctx_first, "ctx_last": ctx_last, "inv_tau": INV_TAU,
                    "cache_bytes": int(token_heads * entry),
                    "l2": "working set (%.0f MB per step) is larger than L2; nothing is flushed" % (alg_bytes / 1e6)},
-        "e2e": {"value": e2e_value, "unit": UNIT, "ms_per_step": e2e_ms_total / steps,
+        "e2e": {"value": e2e_value, "unit": UNIT, "ms_per_step": (e2e_ms_total / steps) if Tq == 1 else None,
                 "h2d_bytes_per_step": int(sum(x[0].numel() * 2 for x in (kh, vh, qh))),
                 "d2h_bytes_per_step": int(oh.numel() * 4)},
         "gpu_launches": int(launches),
@@ -424,6 +440,8 @@ def main():
     ap.add_argument("--sketch-bits", type=int, default=0, help="override m (64, 128, 256, 512)")
     ap.add_argument("--group-size", type=int, default=0, help="override G (32, or 128 = one scale per value vector)")
     ap.add_argument("--no-layer-sequential", action="store_true", help="skip the per-layer CUDA-graph measurement")
+    ap.add_argument("--query-tokens", type=int, default=1,
+                    help="> 1: each step appends this many tokens per sequence and attends for all of them (variant)")
     ap.add_argument("--fp16-values", action="store_true", help="keep values in fp16 (the 1-bit-keys-only ablation row)")
     ap.add_argument("--workload", default="c2_7b_8k",
                     choices=["c2_7b_8k", "c3_7b_batched", "c4_gqa_32k", "c5_prefill"],

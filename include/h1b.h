@@ -120,6 +120,21 @@ int h1b_append_kv(h1b_ctx *ctx, int layer_begin, int n_layers, const void *k, co
 int h1b_decode_attention(h1b_ctx *ctx, int layer_begin, int n_layers, const void *q,
                          float inv_tau, void *out, int B, void *stream);
 
+/* Decode attention for the last Tq tokens of every sequence at once (chunked
+ * prefill, verification of speculated tokens). The Tq query tokens are the
+ * sequence's last Tq cached tokens, already appended: query token i
+ * (0 <= i < Tq) attends to cached tokens [0, len - Tq + i + 1), i.e. to
+ * everything up to and including itself (Eq. 3 and Eq. 5 per query token).
+ * The paper describes one query per step; this is the same computation for
+ * several queries that share every cache tile they read.
+ *   q    DEVICE: fp16 [n_layers][B][Tq][Hq][d]      1 <= Tq <= H1B_MAX_QUERY_TOKENS
+ *   out  DEVICE: float32 [n_layers][B][Tq][Hq][d]
+ * H1B_ERR_INVALID_ARG if some sequence of the call holds fewer than Tq tokens.
+ * Tq = 1 is h1b_decode_attention(). */
+#define H1B_MAX_QUERY_TOKENS 16
+int h1b_decode_attention_multi(h1b_ctx *ctx, int layer_begin, int n_layers, const void *q, int Tq,
+                               float inv_tau, void *out, int B, void *stream);
+
 /* One whole decode step on device tensors, all L layers: append one new token per
  * sequence (Eq. 2, Eq. 4) and run decode attention over the grown cache (Eq. 3,
  * Eq. 5). Same result as h1b_append_kv(Tn = 1) followed by h1b_decode_attention(),

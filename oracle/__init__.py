@@ -262,6 +262,24 @@ def layer_fp16_values(K, V, lens, q, Rt, inv_tau: float):
     return out
 
 
+def layer_multi(K, V, lens, q, Rt, inv_tau: float, G: int = 32, fp16_values: bool = False):
+    """Several query tokens per sequence: q [B, Tq, Hq, d] are the queries of each sequence's last Tq cached
+    tokens; query token i attends to tokens [0, lens - Tq + i + 1), i.e. up to and including itself. Written as
+    what it means: one independent single-query pass (Eq. 2-5) per query token over its own prefix of the
+    sequence. Returns out fp64 [B, Tq, Hq, d]."""
+    qb = _as_u16(q)
+    B, Tq, Hq, d = qb.shape
+    ln = np.ascontiguousarray(lens, dtype=np.int32)
+    assert ln.shape == (B,) and int(ln.min()) >= Tq
+    out = np.zeros((B, Tq, Hq, d), dtype=np.float64)
+    for i in range(Tq):
+        prefix = (ln - Tq + i + 1).astype(np.int32)
+        qi = np.ascontiguousarray(qb[:, i])
+        out[:, i] = layer_fp16_values(K, V, prefix, qi, Rt, inv_tau) if fp16_values else \
+            layer(K, V, prefix, qi, Rt, inv_tau, G)
+    return out
+
+
 def entry_bytes(d: int, m: int, G: int) -> int:
     return int(_load().h1bo_entry_bytes(d, m, G))
 

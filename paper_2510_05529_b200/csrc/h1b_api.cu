@@ -21,11 +21,12 @@ namespace {
 
 constexpr long kTargetItems = 8192;   // decode work items aimed for (one warp each)
 constexpr int kMinSplitTokens = 256;
+constexpr int kMaxQueryTokens = H1B_MAX_QUERY_TOKENS;
 constexpr int kPrefillMinTokens = 64;   // appends of at least this many tokens per sequence take the tensor-core path
 
 struct Plan {
     size_t rt, rh, len, status, arrive, qwords, partial, stage_k, stage_v, stage_q, stage_out, dbg_q, dbg_s, cache, total;
-    size_t partial_items, slab_bytes;
+    size_t partial_bytes, slab_bytes;
     int cap_tokens, m_words, gq, groups;
 };
 
@@ -60,7 +61,9 @@ int make_plan(const h1b_config *c, Plan *p) {
     p->slab_bytes = (size_t)(p->cap_tokens / kChunkTokens) * cl.bytes;
     const size_t L = c->n_layers, B = c->max_batch, Hq = c->n_q_heads, Hkv = c->n_kv_heads, d = c->head_dim;
     const size_t slabs = L * B * Hkv;
-    p->partial_items = slabs > (size_t)kTargetItems ? slabs : (size_t)kTargetItems;
+    // split-K scratch: room for kTargetItems work items (or one per slab) of four (virtual) heads each
+    const size_t partial_items = slabs > (size_t)kTargetItems ? slabs : (size_t)kTargetItems;
+    p->partial_bytes = partial_items * 4 * kPartStride * sizeof(float);
     size_t o = 0;
     auto take = [&](size_t bytes) { size_t at = o; o = align_up(o + bytes, 256); return at; };
     p->rt = take(L * d * c->sketch_bits * sizeof(float));
@@ -68,8 +71,8 @@ int make_plan(const h1b_config *c, Plan *p) {
     p->len = take(L * B * sizeof(int32_t));
     p->status = take(64);
     p->arrive = take(slabs * sizeof(int32_t));
-    p->qwords = take(L * B * Hq * p->m_words * sizeof(uint32_t));
-    p->partial = take(p->partial_items * p->gq * kPartStride * sizeof(float));
+    p->qwords = take(L * B * Hq * kMaxQueryTokens * p->m_words * sizeof(uint32_t));
+    p->partial = take(p->partial_bytes);
     p->stage_k = take(L * B * Hkv * d * 2);
     p->stage_v = take(L * B * Hkv * d * 2);
     p->stage_q = take(L * B * Hq * d * 2);
@@ -279,9 +282,12 @@ static void commit_lengths(h1b_ctx *ctx, int layer_begin, int n_layers, int B, c
 // there are about kTargetItems work items, capped by `max_items`; the last split of a sequence is open-ended,
 // so the result does not depend on how well the host's view of the lengths matches the device's.
 static int enqueue_decode(h1b_ctx *ctx, int layer_begin, int n_layers, float inv_tau, void *out, int B,
-                          cudaStream_t st, uint32_t *qwords, float *partial, int32_t *arrive, size_t max_items,
-                          bool may_profile, int *launches) {
-    const long slabs = (long)n_layers * B * ctx->cfg.n_kv_heads;
+                          cudaStream_t st, uint32_t *qwords, float *partial, int32_t *arrive, size_t partial_bytes,
+                          bool may_profile, int *launches, int Tq = 1) {
+    // (query token, query head) pairs that share a KV head, and how many of them one work item takes
+    const int vheads = ctx->plan.gq * Tq, gqk = vheads >= 3 ? 4 : vheads, vgroups = (vheads + gqk - 1) / gqk;
+    const size_t max_items = partial_bytes / ((size_t)gqk * kPartStride * sizeof(float));
+    const long slabs = (long)n_layers * B * ctx->cfg.n_kv_heads * vgroups;       // slabs x groups: units a split divides
     int maxlen = 1;
     for (int l = layer_begin; l < layer_begin + n_layers; ++l)
         for (int b = 0; b < B; ++b) maxlen = std::max(maxlen, ctx->len_host[(size_t)l * ctx->cfg.max_batch + b]);
@@ -312,6 +318,7 @@ static int enqueue_decode(h1b_ctx *ctx, int layer_begin, int n_layers, float inv
     dp.Hq = ctx->cfg.n_q_heads; dp.max_batch = ctx->cfg.max_batch; dp.m_words = ctx->plan.m_words;
     dp.groups = ctx->plan.groups;
     dp.splits = (int)splits; dp.split_tokens = split_tokens;
+    dp.Tq = Tq; dp.gqk = gqk; dp.vgroups = vgroups;
     dp.c2 = (float)(2.0 * (double)inv_tau * 1.4426950408889634 / (double)ctx->cfg.sketch_bits);
     cudaEvent_t ev0 = nullptr, ev1 = nullptr;
     if (may_profile && ctx->profiling && ctx->events_used + 2 <= ctx->events.size()) {
@@ -386,7 +393,32 @@ int h1b_decode_attention(h1b_ctx *ctx, int layer_begin, int n_layers, const void
     std::memset(&none, 0, sizeof none);
     H1B_CUDA(ctx, launch_prepare(nullptr, &sp, none, st, &launches));
     rc = enqueue_decode(ctx, layer_begin, n_layers, inv_tau, out, B, st, sp.qwords, at<float>(ctx, ctx->plan.partial),
-                        at<int32_t>(ctx, ctx->plan.arrive), ctx->plan.partial_items, true, &launches);
+                        at<int32_t>(ctx, ctx->plan.arrive), ctx->plan.partial_bytes, true, &launches);
+    ctx->launches += launches;
+    return rc;
+}
+
+int h1b_decode_attention_multi(h1b_ctx *ctx, int layer_begin, int n_layers, const void *q, int Tq, float inv_tau,
+                               void *out, int B, void *stream) {
+    int rc = check_decode_args(ctx, layer_begin, n_layers, q, inv_tau, out, B);
+    if (rc != H1B_OK) return rc;
+    if (Tq < 1 || Tq > kMaxQueryTokens)
+        return fail(ctx, H1B_ERR_INVALID_ARG, "Tq = %d outside [1, %d]", Tq, kMaxQueryTokens);
+    for (int l = layer_begin; l < layer_begin + n_layers; ++l)
+        for (int b = 0; b < B; ++b)
+            if (ctx->len_host[(size_t)l * ctx->cfg.max_batch + b] < Tq)
+                return fail(ctx, H1B_ERR_INVALID_ARG, "layer %d sequence %d holds %d < Tq = %d tokens", l, b,
+                            ctx->len_host[(size_t)l * ctx->cfg.max_batch + b], Tq);
+    cudaStream_t st = static_cast<cudaStream_t>(stream);
+    int launches = 0;
+    // rows of the sketch are (sequence, query token, query head): Tq * Hq "heads" per sequence
+    SketchParams sp = sketch_params(ctx, layer_begin, n_layers, q, B, at<uint32_t>(ctx, ctx->plan.qwords));
+    sp.Hq = Tq * ctx->cfg.n_q_heads;
+    NewCounts none;
+    std::memset(&none, 0, sizeof none);
+    H1B_CUDA(ctx, launch_prepare(nullptr, &sp, none, st, &launches));
+    rc = enqueue_decode(ctx, layer_begin, n_layers, inv_tau, out, B, st, sp.qwords, at<float>(ctx, ctx->plan.partial),
+                        at<int32_t>(ctx, ctx->plan.arrive), ctx->plan.partial_bytes, true, &launches, Tq);
     ctx->launches += launches;
     return rc;
 }
@@ -406,7 +438,7 @@ int h1b_decode_step_layers(h1b_ctx *ctx, int layer_begin, int n_layers, const vo
     H1B_CUDA(ctx, launch_prepare(&ap, &sp, nn, st, &launches));
     commit_lengths(ctx, layer_begin, n_layers, B, nn);
     rc = enqueue_decode(ctx, layer_begin, n_layers, inv_tau, out, B, st, sp.qwords, at<float>(ctx, ctx->plan.partial),
-                        at<int32_t>(ctx, ctx->plan.arrive), ctx->plan.partial_items, true, &launches);
+                        at<int32_t>(ctx, ctx->plan.arrive), ctx->plan.partial_bytes, true, &launches);
     ctx->launches += launches;
     return rc;
 }
@@ -474,7 +506,7 @@ int h1b_decode_attention_static(h1b_ctx *ctx, int layer_begin, int n_layers, con
         return fail(ctx, H1B_ERR_CAPACITY,
                     "static scratch too small: this call needs at least %zu bytes, the built-in array holds %u",
                     need, (unsigned)H1B_STATIC_SCRATCH_BYTES);
-    const size_t fit_items = (H1B_STATIC_SCRATCH_BYTES - arrive_bytes - qw_bytes) / item_bytes;
+    const size_t fit_bytes = H1B_STATIC_SCRATCH_BYTES - arrive_bytes - qw_bytes;
     cudaStream_t st = static_cast<cudaStream_t>(stream);
     // the counters must start at zero whatever an earlier call (or an aborted one) left behind
     H1B_CUDA(ctx, cudaMemsetAsync(scratch, 0, arrive_bytes, st));
@@ -486,7 +518,7 @@ int h1b_decode_attention_static(h1b_ctx *ctx, int layer_begin, int n_layers, con
     H1B_CUDA(ctx, launch_prepare(nullptr, &sp, none, st, &launches));
     rc = enqueue_decode(ctx, layer_begin, n_layers, inv_tau, out, B, st, sp.qwords,
                         reinterpret_cast<float *>(scratch + arrive_bytes + qw_bytes),
-                        reinterpret_cast<int32_t *>(scratch), fit_items, false, &launches);
+                        reinterpret_cast<int32_t *>(scratch), fit_bytes, false, &launches);
     ctx->launches += launches;
     return rc;
 }
@@ -665,8 +697,9 @@ int h1b_debug_scores(h1b_ctx *ctx, int layer, int seq, int kv_head, const void *
 
 int h1b_set_splits(h1b_ctx *ctx, int splits) {
     if (!ctx) return H1B_ERR_NULL;
-    if (splits < 0 || (size_t)splits > ctx->plan.partial_items)
-        return fail(ctx, H1B_ERR_INVALID_ARG, "splits %d outside [0, %zu]", splits, ctx->plan.partial_items);
+    const size_t most = ctx->plan.partial_bytes / ((size_t)ctx->plan.gq * kPartStride * sizeof(float));
+    if (splits < 0 || (size_t)splits > most)
+        return fail(ctx, H1B_ERR_INVALID_ARG, "splits %d outside [0, %zu]", splits, most);
     ctx->forced_splits = splits;
     return H1B_OK;
 }

@@ -613,17 +613,17 @@ struct DecodeState {
     float zero[4];              // an opaque quad of zeros: C operand of each chunk's first MMA
 };
 
-// One chunk. TAIL: tokens at or beyond t_end are masked (only the last chunk of a split needs it).
+// One chunk. TAIL: head h attends only to the chunk's first n_valid[h] tokens (the last chunks of a split; with
+// several query tokens, each one's causal limit).
 template <int MW, int GQ, int NG, bool TAIL>
 __device__ __forceinline__ void decode_chunk(DecodeState<MW, GQ, NG> &st, const unsigned char *ch, float *p_s,
-                                             int lane, int n_valid, float c2) {
+                                             int lane, const int (&n_valid)[GQ], float c2) {
     constexpr int GPF = 4 / GQ;                // value groups covered by one B fragment (4 groups per vector)
     constexpr int NB = (NG == 1) ? 1 : GQ;     // B fragments per 16-token block (one scale per vector: one fragment)
     constexpr int VAL = MW * 128, ZERO = VAL + 2048, SCALE = ZERO + 64 * NG;
     const int jq = lane & 3;
 
     // ---------------- phase 1
-    const bool valid = !TAIL || lane < n_valid;
     uint32_t kw[MW];
 #pragma unroll
     for (int w = 0; w < MW; ++w) kw[w] = *reinterpret_cast<const uint32_t *>(ch + w * 128 + lane * 4);
@@ -643,6 +643,7 @@ __device__ __forceinline__ void decode_chunk(DecodeState<MW, GQ, NG> &st, const 
         int ham = 0;
 #pragma unroll
         for (int w = 0; w < MW; ++w) ham += __popc(kw[w] ^ st.qw[h][w]);
+        const bool valid = !TAIL || lane < n_valid[h];
         const int cmin = __reduce_min_sync(0xffffffffu, (TAIL && !valid) ? kHamSentinel : ham);
         scl[h] = 1.f;
         if (cmin < st.hmin[h]) {                            // warp-uniform: the running max moved
@@ -781,10 +782,11 @@ __global__ void __launch_bounds__(kDecodeWarps * 32, decode_min_blocks(GQ, NG)) 
 
     const int lane = threadIdx.x & 31, warp = threadIdx.x >> 5;
     const long item = (long)blockIdx.x * kDecodeWarps + warp;
-    const long n_items = (long)p.n_layers * p.B * p.Hkv * p.splits;
+    const long n_items = (long)p.n_layers * p.B * p.Hkv * p.vgroups * p.splits;
     if (item >= n_items) return;
     const int split = (int)(item % p.splits);
-    const long slab_local = item / p.splits;
+    const int vg = (int)((item / p.splits) % p.vgroups);        // which group of GQ virtual heads (0 unless Tq > 1)
+    const long slab_local = item / ((long)p.splits * p.vgroups);
     const int kvh = (int)(slab_local % p.Hkv);
     const int b = (int)((slab_local / p.Hkv) % p.B);
     const int ll = (int)(slab_local / ((long)p.Hkv * p.B));
@@ -803,7 +805,8 @@ __global__ void __launch_bounds__(kDecodeWarps * 32, decode_min_blocks(GQ, NG)) 
     }
     // the last split of a sequence is open-ended: it runs to the sequence's end
     const int t_end = (split == p.splits - 1) ? len : min(len, t_begin + p.split_tokens);
-    const int c0 = t_begin >> 5, c_full = t_end >> 5, c1 = (t_end + 31) >> 5;
+    // chunks below c_full are attended in full by every head (the earliest query token sees len - Tq + 1 tokens)
+    const int c0 = t_begin >> 5, c_full = min(t_end, len - p.Tq + 1) >> 5, c1 = (t_end + 31) >> 5;
 
     unsigned char *ring = smem_raw + warp * SM::kPerWarp;
     float *p_s = reinterpret_cast<float *>(ring + kStages * CB);
@@ -829,12 +832,18 @@ __global__ void __launch_bounds__(kDecodeWarps * 32, decode_min_blocks(GQ, NG)) 
 
     DecodeState<MW, GQ, NG> st;
     zero_quad(st.zero);
+    int limit[GQ];                                              // tokens [0, limit[h]) are attended by head h
     {
-        const uint32_t *qp = p.qwords + ((size_t)(layer * p.max_batch + b) * p.Hq + kvh * GQ) * MW;
+        const int gq = p.Hq / p.Hkv, vheads = gq * p.Tq;
 #pragma unroll
-        for (int h = 0; h < GQ; ++h)
+        for (int h = 0; h < GQ; ++h) {
+            // a group's surplus slots repeat the last virtual head (their results are never read)
+            const int v = min(vg * GQ + h, vheads - 1), tq = v / gq, hq = kvh * gq + v % gq;
+            limit[h] = min(t_end, len - p.Tq + tq + 1);
+            const uint32_t *qp = p.qwords + (((size_t)(layer * p.max_batch + b) * p.Tq + tq) * p.Hq + hq) * MW;
 #pragma unroll
-            for (int w = 0; w < MW; ++w) st.qw[h][w] = __ldg(qp + h * MW + w);
+            for (int w = 0; w < MW; ++w) st.qw[h][w] = __ldg(qp + w);
+        }
     }
 #pragma unroll
     for (int cb = 0; cb < 8; ++cb)
@@ -854,8 +863,14 @@ __global__ void __launch_bounds__(kDecodeWarps * 32, decode_min_blocks(GQ, NG)) 
     for (int c = c0; c < c1; ++c) {
         if (!mbar_wait_bounded(bar0 + 8 * stage, parity, kWaitLimitNs)) { failed = true; break; }
         const unsigned char *ch = ring + stage * CB;
-        if (c < c_full) decode_chunk<MW, GQ, NG, false>(st, ch, p_s, lane, 32, p.c2);
-        else decode_chunk<MW, GQ, NG, true>(st, ch, p_s, lane, t_end - c * 32, p.c2);
+        if (c < c_full) {
+            decode_chunk<MW, GQ, NG, false>(st, ch, p_s, lane, limit, p.c2);
+        } else {
+            int n_valid[GQ];
+#pragma unroll
+            for (int h = 0; h < GQ; ++h) n_valid[h] = limit[h] - c * 32;
+            decode_chunk<MW, GQ, NG, true>(st, ch, p_s, lane, n_valid, p.c2);
+        }
         // every lane is done with this stage (the chunk ends with a warp barrier): refill it
         if (lane == 0 && requested < c1) {
             mbar_arrive_expect_tx(bar0 + 8 * stage, CB);
@@ -997,16 +1012,18 @@ __global__ void __launch_bounds__(kHeadDim) combine_kernel(DecodeParams p) {
     __shared__ __align__(16) float s_num[4][kHeadDim];
     const int tid = threadIdx.x, lane = tid & 31, warp = tid >> 5;
     const int gq = p.Hq / p.Hkv;
-    const int hq = blockIdx.x % p.Hq;
-    const int b = (blockIdx.x / p.Hq) % p.B;
-    const int ll = blockIdx.x / (p.Hq * p.B);
+    const int hq = blockIdx.x % p.Hq;                           // blocks enumerate [layer][sequence][query token][query head]
+    const int tq = (blockIdx.x / p.Hq) % p.Tq;
+    const int b = (blockIdx.x / (p.Hq * p.Tq)) % p.B;
+    const int ll = blockIdx.x / (p.Hq * p.Tq * p.B);
     grid_dependency_wait();                                     // the partials come from the attention kernel
     const int len = p.len[(p.layer_begin + ll) * p.max_batch + b];
-    const int kvh = hq / gq, hh = hq % gq;
+    const int kvh = hq / gq;
+    const int v = tq * gq + hq % gq, vg = v / p.gqk, hh = v % p.gqk;          // virtual head, its group and slot
     const long slab_local = ((long)ll * p.B + b) * p.Hkv + kvh;
     const int ns = min(p.splits, (len + p.split_tokens - 1) / p.split_tokens);
-    const float *base = p.partial + ((size_t)slab_local * p.splits * gq + hh) * kPartStride;
-    const size_t stride = (size_t)gq * kPartStride;
+    const float *base = p.partial + (((size_t)slab_local * p.vgroups + vg) * p.splits * p.gqk + hh) * kPartStride;
+    const size_t stride = (size_t)p.gqk * kPartStride;
     // the smallest Hamming distance any split saw (= the largest logit)
     float hm = 3.0e38f;
     for (int j = tid; j < ns; j += kHeadDim) hm = fminf(hm, base[j * stride + 128]);
@@ -1132,7 +1149,7 @@ static cudaError_t launch_decode_t(const DecodeParams &p, cudaStream_t st) {
         if (e != cudaSuccess) return e;
         attr_set[dev] = true;
     }
-    const long items = (long)p.n_layers * p.B * p.Hkv * p.splits;
+    const long items = (long)p.n_layers * p.B * p.Hkv * p.vgroups * p.splits;
     const unsigned grid = (unsigned)((items + kDecodeWarps - 1) / kDecodeWarps);
     cudaLaunchConfig_t cfg = {};
     cfg.gridDim = dim3(grid);
@@ -1149,8 +1166,11 @@ static cudaError_t launch_decode_t(const DecodeParams &p, cudaStream_t st) {
 
 cudaError_t launch_decode(const DecodeParams &p, cudaStream_t st, int *launches, cudaEvent_t before,
                           cudaEvent_t after) {
-    const int gq = p.Hq / p.Hkv;
+    const int gq = p.gqk;                                       // (virtual) heads per work item
     cudaError_t e = cudaErrorInvalidValue;
+#ifdef H1B_FUSED_COMBINE
+    if (p.Tq != 1) return cudaErrorNotSupported;                // the fused merge only knows one query token
+#endif
     if (before) cudaEventRecord(before, st);
     H1B_DISPATCH_MW(p.m_words,
         if (p.groups == 4) {
@@ -1173,7 +1193,7 @@ cudaError_t launch_decode(const DecodeParams &p, cudaStream_t st, int *launches,
 #ifndef H1B_FUSED_COMBINE
     {
         cudaLaunchConfig_t cfg = {};
-        cfg.gridDim = dim3(p.n_layers * p.B * p.Hq);
+        cfg.gridDim = dim3(p.n_layers * p.B * p.Tq * p.Hq);
         cfg.blockDim = dim3(kHeadDim);
         cfg.stream = st;
         cudaLaunchAttribute attr[1];

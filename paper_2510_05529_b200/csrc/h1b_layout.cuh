@@ -135,14 +135,18 @@ struct SketchParams {           // query sketch
 struct DecodeParams {
     const unsigned char *cache;
     const int32_t *len;         // [L][max_batch]
-    const uint32_t *qwords;     // [L][max_batch][Hq][m/32]
-    float *partial;             // [items][GQ][kPartStride]
-    float *out;                 // fp32 [n_layers][B][Hq][d]
+    const uint32_t *qwords;     // [L][max_batch][Tq][Hq][m/32]
+    float *partial;             // [items][gqk][kPartStride]
+    float *out;                 // fp32 [n_layers][B][Tq][Hq][d]
     int32_t *status;
     int32_t *arrive;            // [slabs of the call]: splits that have reported in (zero between launches)
     size_t slab_bytes;
     int layer_begin, n_layers, B, Hkv, Hq, max_batch, m_words, groups;
     int splits, split_tokens;   // split_tokens is a multiple of 32
+    // Several query tokens per sequence (Tq > 1): they are the sequence's last Tq cached tokens, query token i attends to
+    // tokens [0, len - Tq + i + 1). The Tq * (Hq/Hkv) (query token, query head) pairs that share a KV head are "virtual
+    // heads" v = i * (Hq/Hkv) + head-in-group, handled `gqk` at a time by one work item (vgroups items per slab and split).
+    int Tq, gqk, vgroups;
     float c2;                   // 2 * inv_tau * log2(e) / m : log2-weight per unit of Hamming distance
 };
 

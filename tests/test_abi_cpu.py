@@ -37,7 +37,7 @@ def test_entry_and_workspace_bytes(lib):
     assert binding.h1b_entry_bytes(c) == 96
     payload = 32 * 32 * 8192 * 96
     total = binding.h1b_cache_bytes(c)
-    assert payload <= total <= payload + 16 * 2 ** 20     # cache + projections + scratch
+    assert payload <= total <= payload + 32 * 2 ** 20     # cache + projections + split-K scratch (17 MiB) + staging
     c4 = binding.make_config(32, 32, 8, 128, 256, 32, max_batch=8, max_seq=32768)
     assert binding.h1b_entry_bytes(c4) == 112
     assert binding.h1b_cache_bytes(c4) >= 32 * 8 * 8 * 32768 * 112

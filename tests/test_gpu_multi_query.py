@@ -1,0 +1,167 @@
+"""GPU parity of decode attention for several query tokens per sequence (chunked prefill, verification of
+speculated tokens): the queries are the sequence's last Tq cached tokens and each attends up to and including
+itself. Checked against the fp64 oracle's per-query-token passes, isolated (on the exported GPU cache, integer
+scores bit for bit) and end to end (from the fp16 rows)."""
+import numpy as np
+import pytest
+import torch
+
+import h1b_synth
+import oracle
+from h1b_testlib import WINDOW, check_output, f16_bits, make_cache
+from paper_2510_05529_b200 import binding
+
+pytestmark = pytest.mark.gpu
+W = h1b_synth.WORKLOADS
+
+
+def _queries(w, Tq, seed=0):
+    """fp16 [L, B, Tq, Hq, d]: one seeded draw per query token."""
+    return torch.stack([torch.stack([h1b_synth.queries(w, l, stream=200 + seed + i) for i in range(Tq)], dim=1)
+                        for l in range(w.n_layers)])
+
+
+def _fill(w, lens, fp16_values=False, max_seq=None):
+    lens = np.asarray(lens, np.int32)
+    T = int(lens.max())
+    cache, Rt = make_cache(w, max_seq=max_seq or T, fp16_values=fp16_values)
+    Ks, Vs = [], []
+    for l in range(w.n_layers):
+        K, V = h1b_synth.kv_rows(w, l, T)
+        cache.h1b_append_kv(K.unsqueeze(0).cuda(), V.unsqueeze(0).cuda(), layer_begin=l, n_new=lens)
+        Ks.append(K); Vs.append(V)
+    return cache, Rt, torch.stack(Ks), torch.stack(Vs), lens
+
+
+def _check(w, cache, Rt, K, V, q, lens, out, inv_tau, fp16_values):
+    """out [L, B, Tq, Hq, d] against the oracle, both protocols."""
+    gq = w.n_q_heads // w.n_kv_heads
+    Tq = q.shape[2]
+    worst, flips = 0.0, 0
+    for l in range(w.n_layers):
+        e2e = oracle.layer_multi(f16_bits(K[l]), f16_bits(V[l]), lens, f16_bits(q[l]), Rt[l], inv_tau, w.group_size,
+                                 fp16_values=fp16_values)
+        for b in range(w.batch):
+            n = int(lens[b])
+            for g in range(w.n_kv_heads):
+                words, codes, scale, zero = cache.h1b_export_cache(l, b, g, 0, n)
+                kbits = binding.unpack_words(words, w.sketch_bits)
+                obits, y, a = oracle.sketch(f16_bits(K[l, b, :n, g]), Rt[l], want_margin=True)
+                flips += int((kbits != obits).sum())
+                vals = cache.h1b_export_values(l, b, g, 0, n) if fp16_values else None
+                for i in range(Tq):
+                    n_i = n - Tq + i + 1                                  # what query token i attends to
+                    for hh in range(gq):
+                        h = g * gq + hh
+                        qrow = q[l, b, i, h].contiguous().cuda()
+                        qwords, gscore = cache.h1b_debug_scores(l, b, g, qrow, n)
+                        qbits = binding.unpack_words(qwords[None], w.sketch_bits)[0]
+                        oscore = oracle.scores(qbits, kbits)
+                        assert np.array_equal(gscore[:n], oscore)
+                        oq, yq, aq = oracle.sketch(f16_bits(qrow)[None], Rt[l], want_margin=True)
+                        dq = oq[0] != qbits
+                        assert not (dq & (np.abs(yq[0]) > WINDOW * aq[0])).any()
+                        flips += int(dq.sum())
+                        if fp16_values:
+                            ref = oracle.attention_fp16_values(oscore[:n_i], w.sketch_bits, inv_tau, vals[:n_i])
+                        else:
+                            ref = oracle.attention(oscore[:n_i], w.sketch_bits, inv_tau, codes[:n_i], scale[:n_i],
+                                                   zero[:n_i], w.group_size)
+                        worst = max(worst, check_output(out[l, b, i, h], ref, ("isolated", l, b, i, h)))
+                        if flips == 0 and not fp16_values:
+                            # the oracle quantises the rows itself: only comparable while no boundary decision differs
+                            ocodes, oscale, ozero = oracle.quantize(f16_bits(V[l, b, :n, g]), w.group_size)[:3]
+                            if np.array_equal(ocodes, codes) and np.array_equal(oscale, scale):
+                                check_output(out[l, b, i, h], e2e[b, i, h], ("end to end", l, b, i, h))
+                        elif flips == 0:
+                            check_output(out[l, b, i, h], e2e[b, i, h], ("end to end", l, b, i, h))
+    return worst, flips
+
+
+@pytest.mark.parametrize("hq, hkv, Tq", [(1, 1, 1), (1, 1, 2), (1, 1, 3), (1, 1, 4), (1, 1, 7), (2, 2, 16),
+                                         (4, 2, 3), (4, 2, 8), (4, 1, 2), (4, 1, 5), (8, 2, 16)])
+def test_head_group_shapes_and_query_counts(hq, hkv, Tq):
+    w = h1b_synth.scaled(W["c1_tiny"], batch=2, n_layers=2, n_q_heads=hq, n_kv_heads=hkv)
+    cache, Rt, K, V, lens = _fill(w, [333, 64])
+    q = _queries(w, Tq)
+    out = cache.h1b_decode_attention_multi(q.cuda(), 16.0).cpu().numpy()
+    cache.h1b_poll_status()
+    worst, flips = _check(w, cache, Rt, K, V, q, lens, out, 16.0, False)
+    print("multi-query", hq, hkv, Tq, "max err", worst, "flips in window", flips)
+    cache.close()
+
+
+@pytest.mark.parametrize("lens, Tq, splits, inv_tau", [
+    ([16, 17], 16, 0, 16.0),          # the queries are (almost) the whole sequence
+    ([32, 33], 4, 0, 1.0),            # the causal limits straddle a chunk boundary
+    ([1000, 257], 6, 7, 50.0),        # forced splits: limits fall into different splits
+    ([1000, 999], 16, 31, 16.0),      # the last split holds only some of the query tokens' last keys
+])
+def test_causal_limits_across_chunks_and_splits(lens, Tq, splits, inv_tau):
+    w = h1b_synth.scaled(W["c1_tiny"], batch=2, n_q_heads=2, n_kv_heads=1)
+    cache, Rt, K, V, lens = _fill(w, lens)
+    q = _queries(w, Tq, seed=9)
+    cache.h1b_set_splits(splits)
+    out = cache.h1b_decode_attention_multi(q.cuda(), inv_tau).cpu().numpy()
+    cache.h1b_poll_status()
+    worst, flips = _check(w, cache, Rt, K, V, q, lens, out, inv_tau, False)
+    print("multi-query causal", lens.tolist(), Tq, splits, "max err", worst, "flips", flips)
+    cache.close()
+
+
+@pytest.mark.parametrize("m, G, fp16_values", [(64, 32, False), (256, 128, False), (128, 32, True), (512, 32, True)])
+def test_other_formats(m, G, fp16_values):
+    w = h1b_synth.scaled(W["c1_tiny"], batch=2, n_q_heads=4, n_kv_heads=2, sketch_bits=m, group_size=G)
+    cache, Rt, K, V, lens = _fill(w, [200, 90], fp16_values=fp16_values)
+    q = _queries(w, 5, seed=3)
+    out = cache.h1b_decode_attention_multi(q.cuda(), 16.0).cpu().numpy()
+    cache.h1b_poll_status()
+    _check(w, cache, Rt, K, V, q, lens, out, 16.0, fp16_values)
+    cache.close()
+
+
+def test_one_query_token_is_the_decode_call_and_bad_counts_are_rejected():
+    w = h1b_synth.scaled(W["c1_tiny"], batch=2, n_q_heads=4, n_kv_heads=2)
+    cache, Rt, K, V, lens = _fill(w, [300, 5])
+    q1 = _queries(w, 1)
+    a = cache.h1b_decode_attention_multi(q1.cuda(), 16.0).cpu().numpy()
+    b = cache.h1b_decode_attention(q1[:, :, 0].contiguous().cuda(), 16.0).cpu().numpy()
+    assert np.array_equal(a[:, :, 0], b)
+    with pytest.raises(binding.H1BError) as err:                          # sequence 1 holds 5 tokens
+        cache.h1b_decode_attention_multi(_queries(w, 6).cuda(), 16.0)
+    assert err.value.code == -1
+    with pytest.raises(binding.H1BError):                                 # more than the interface allows
+        cache.h1b_decode_attention_multi(_queries(w, 17).cuda(), 16.0)
+    cache.close()
+
+
+def test_7b_shape_sampled_units():
+    """32 heads, 8192 cached tokens, 8 query tokens, two layers: sampled (layer, head) units end to end."""
+    w = h1b_synth.scaled(W["c2_7b_8k"], n_layers=2)
+    lens = h1b_synth.lengths(w)
+    Tq = 8
+    cache, Rt = make_cache(w, max_seq=w.context)
+    units = [(0, 0, 0), (1, 0, 31), (1, 0, 17)]
+    keep = {}
+    for l in range(w.n_layers):
+        K, V = h1b_synth.kv_rows(w, l, w.context, device="cuda")
+        cache.h1b_append_kv(K.unsqueeze(0), V.unsqueeze(0), layer_begin=l, n_new=lens)
+        for u in units:
+            if u[0] == l:
+                keep[u] = (K[u[1], :, u[2]].cpu(), V[u[1], :, u[2]].cpu())
+    q = _queries(w, Tq)
+    out = cache.h1b_decode_attention_multi(q.cuda(), 16.0).cpu().numpy()
+    cache.h1b_poll_status()
+    for (l, b, g) in units:
+        K, V = keep[(l, b, g)]
+        n = int(lens[b])
+        words, codes, scale, zero = cache.h1b_export_cache(l, b, g, 0, n)
+        kbits = binding.unpack_words(words, w.sketch_bits)
+        for i in range(Tq):
+            qrow = q[l, b, i, g].contiguous().cuda()
+            qwords, gscore = cache.h1b_debug_scores(l, b, g, qrow, n)
+            n_i = n - Tq + i + 1
+            ref = oracle.attention(gscore[:n_i], w.sketch_bits, 16.0, codes[:n_i], scale[:n_i], zero[:n_i], w.group_size)
+            check_output(out[l, b, i, g], ref, ("7B shape", l, b, g, i))
+        assert np.array_equal(gscore[:n], oracle.scores(binding.unpack_words(qwords[None], w.sketch_bits)[0], kbits))
+    cache.close()

@@ -229,3 +229,37 @@ def test_fp16_value_variant_is_softmax_matmul():
     sc = np.array([4, 0, -4], np.int32)
     o = oracle.attention_fp16_values(sc, 4, 1.0, V[0, :3, 0])
     assert np.allclose(o, np.array([0.66524096, 0.24472847, 0.09003057]) @ V[0, :3, 0].astype(np.float64), atol=2e-8)
+
+
+def test_multi_query_is_causally_masked_softmax_matmul():
+    """Several query tokens: one masked [Tq, T] score matrix in numpy gives every query token's output at once.
+    Values on a lossless grid (4-bit route) and arbitrary (fp16-value route)."""
+    rng = np.random.default_rng(16)
+    B, T, Tq, Hq, Hkv, d, m = 2, 60, 5, 4, 2, 128, 64
+    Rt = rng.standard_normal((d, m)).astype(np.float32)
+    K = rng.standard_normal((B, T, Hkv, d)).astype(np.float16)
+    n = rng.integers(0, 16, (B, T, Hkv, d))
+    n[..., ::32] = 0
+    n[..., 1::32] = 15
+    Vgrid = (-1.0 + 0.125 * n).astype(np.float16)
+    Vany = rng.standard_normal((B, T, Hkv, d)).astype(np.float16)
+    q = rng.standard_normal((B, Tq, Hq, d)).astype(np.float16)
+    lens = np.array([T, 23], dtype=np.int32)
+    R64 = Rt.astype(np.float64)
+    for V, fp16_values in ((Vgrid, False), (Vany, True)):
+        out = oracle.layer_multi(K, V, lens, q, Rt, 16.0, fp16_values=fp16_values)
+        assert out.shape == (B, Tq, Hq, d)
+        for b in range(B):
+            L = int(lens[b])
+            pos = np.arange(L)[None, :]                                   # key positions
+            own = (L - Tq + np.arange(Tq))[:, None]                       # each query token's own position
+            for h in range(Hq):
+                g = h // (Hq // Hkv)
+                sk = np.where(K[b, :L, g].astype(np.float64) @ R64 >= 0, 1.0, -1.0)      # [L, m]
+                sq = np.where(q[b, :, h].astype(np.float64) @ R64 >= 0, 1.0, -1.0)       # [Tq, m]
+                logits = np.where(pos <= own, sq @ sk.T / m * 16.0, -np.inf)
+                want = softmax(logits, axis=1) @ V[b, :L, g].astype(np.float64)
+                assert np.allclose(out[b, :, h], want, rtol=0, atol=1e-12), (fp16_values, b, h)
+    # one query token is the single-query path
+    one = oracle.layer_multi(K, Vany, lens, q[:, -1:], Rt, 16.0)
+    assert np.array_equal(one[:, 0], oracle.layer(K, Vany, lens, q[:, -1], Rt, 16.0))
