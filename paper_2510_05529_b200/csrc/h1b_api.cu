@@ -371,7 +371,12 @@ int h1b_append_kv(h1b_ctx *ctx, int layer_begin, int n_layers, const void *k, co
                 if (nn.v[b] > 0) tiles = std::max(tiles, (len0 + nn.v[b] + 127) / 128 - len0 / 128);
             }
         pp.tiles_per_seq = tiles;
-        pp.tiles_per_block = std::min(tiles, 8);
+        // one block streams consecutive tiles of a slab through a two-deep pipeline: long runs amortise its start-up,
+        // as long as there are still several blocks for every SM
+        const long slabs = (long)n_layers * B * ctx->cfg.n_kv_heads * ((ctx->cfg.sketch_bits + 127) / 128);
+        int tpb = std::min(tiles, 32);
+        while (tpb > 4 && slabs * ((tiles + tpb - 1) / tpb) < 148 * 4) tpb = (tpb + 1) / 2;
+        pp.tiles_per_block = tpb;
         H1B_CUDA(ctx, launch_prefill(pp, nn, static_cast<cudaStream_t>(stream), &launches));
     } else {
         const AppendParams ap = append_params(ctx, layer_begin, n_layers, k, v, B, Tn);

@@ -259,13 +259,13 @@ __global__ void __launch_bounds__(kProjThreads) prepare_kernel(AppendParams ap, 
 // ===========================================================================
 constexpr int kPrefillThreads = 256;
 constexpr int kPrefillTile = 128;              // cache positions per tile
+constexpr int kKeyStages = 4;                  // key tile buffers: tiles are requested three ahead of the MMAs that read them
 
 template <int NBC>                             // sketch columns per block: 128 or 64
 struct PrefillSmem {
     static constexpr int kRBytes = 2 * NBC * kHeadDim * 2;          // two fp16 pieces of the projection block, [col][channel]
     static constexpr int kABytes = kPrefillTile * kHeadDim * 2;     // the key tile, [row][channel]
-    static constexpr int kVBytes = (kPrefillThreads / 32) * 1280;   // per warp: 1024 B codes + 128 B scale + 128 B zero
-    static constexpr int kTotal = kRBytes + kABytes + kVBytes + 1024;   // + slack to align the operands to 1024 B
+    static constexpr int kTotal = kRBytes + kKeyStages * kABytes + 1024;   // + slack to align the operands to 1024 B
 };
 
 // Byte offset of element (row, k) of a K-major operand tile [rows][128 channels] held as two 64-channel halves,
@@ -290,14 +290,156 @@ __device__ __forceinline__ __half exact_scale(float mx, float mn) {
     return __double2half(((double)mx - (double)mn) / 15.0);
 }
 
+// Eq. 4 (or the fp16 copy) for the 16 cache positions pos0 .. pos0+15 of one slab, by one warp. `vs` is 1280 bytes of
+// shared memory owned by the warp. Positions outside the appended range [len0, len0 + n_new) are left alone.
+__device__ __forceinline__ void store_value_block16(const PrefillParams &p, const ChunkLayout &cl, unsigned char *slab,
+                                                    int ll, int b, int kvh, int len0, int n_new, int pos0,
+                                                    unsigned char *vs, int lane) {
+    const int tn0 = pos0 - len0;
+    unsigned char *chunk = slab + (size_t)(pos0 >> 5) * cl.bytes;
+    const int vb = (pos0 >> 4) & 1;
+    if (p.groups == 0 && tn0 >= 0 && tn0 + 16 <= n_new) {
+        // fp16 values, a whole block of 16 tokens: transposed through shared memory into the A-operand
+        // order, 32 channels (two channel blocks, 1024 contiguous bytes of the cache) per pass
+        const size_t row_stride = (size_t)p.Hkv * kHeadDim;
+        const uint16_t *v0 = p.v + ((((size_t)ll * p.B + b) * p.Tn + tn0) * p.Hkv + kvh) * kHeadDim;
+        unsigned char *dst_block = chunk + cl.val_off + vb * kHalfBlockBytes;
+#pragma unroll 1
+        for (int pass = 0; pass < 4; ++pass) {
+            uint4 raw[2];
+#pragma unroll
+            for (int i = 0; i < 2; ++i) {               // piece e: token e/4, channels pass*32 + (e%4)*8 .. +7
+                const int e = lane + 32 * i;
+                raw[i] = __ldg(reinterpret_cast<const uint4 *>(v0 + (size_t)(e >> 2) * row_stride + pass * 32) + (e & 3));
+            }
+#pragma unroll
+            for (int i = 0; i < 2; ++i) {
+                const int e = lane + 32 * i, k = e >> 2, c16 = e & 3;
+                const int j = (k & 7) >> 1, odd = k & 1, hi8 = k >> 3;
+                unsigned char *base = vs + (c16 >> 1) * 512 + j * 16 + (hi8 * 2 + (c16 & 1)) * 4 + odd * 2;
+                const uint32_t w4[4] = {raw[i].x, raw[i].y, raw[i].z, raw[i].w};
+#pragma unroll
+                for (int x = 0; x < 8; ++x)             // channel row r = x of the channel block
+                    *reinterpret_cast<uint16_t *>(base + x * 64) = (uint16_t)(w4[x >> 1] >> ((x & 1) * 16));
+            }
+            __syncwarp();
+            const uint4 *src = reinterpret_cast<const uint4 *>(vs);
+            uint4 *dst = reinterpret_cast<uint4 *>(dst_block + pass * 1024);
+            dst[lane] = src[lane];
+            dst[32 + lane] = src[32 + lane];
+            __syncwarp();
+        }
+    } else if (p.groups != 0 && tn0 >= 0 && tn0 + 16 <= n_new) {   // a whole block: assemble it in shared memory
+        // lane = (row rsub of 8, group grp of 4): 32 channels of one row per lane and pass, two passes
+                const int rsub = lane >> 2, grp = lane & 3;
+        const size_t row_stride = (size_t)p.Hkv * kHeadDim;
+        const uint16_t *v0 = p.v + ((((size_t)ll * p.B + b) * p.Tn + tn0) * p.Hkv + kvh) * kHeadDim + grp * 32;
+        uint4 raw[2][4];
+#pragma unroll
+        for (int it = 0; it < 2; ++it)
+#pragma unroll
+            for (int j = 0; j < 4; ++j)
+                raw[it][j] = __ldg(reinterpret_cast<const uint4 *>(v0 + (size_t)(it * 8 + rsub) * row_stride) + j);
+#pragma unroll
+        for (int it = 0; it < 2; ++it) {
+            float x[32];
+#pragma unroll
+            for (int j = 0; j < 4; ++j) {
+                const uint32_t w4[4] = {raw[it][j].x, raw[it][j].y, raw[it][j].z, raw[it][j].w};
+#pragma unroll
+                for (int h = 0; h < 4; ++h) {
+                    const float2 f = half2_bits_to_float2(w4[h]);
+                    x[j * 8 + h * 2] = f.x;
+                    x[j * 8 + h * 2 + 1] = f.y;
+                }
+            }
+            float mn = x[0], mx = x[0];
+#pragma unroll
+            for (int i = 1; i < 32; ++i) { mn = fminf(mn, x[i]); mx = fmaxf(mx, x[i]); }
+            if (p.groups == 1) {                        // one scale per vector: the row's four lanes agree
+                mn = fminf(mn, __shfl_xor_sync(0xffffffffu, mn, 1)); mx = fmaxf(mx, __shfl_xor_sync(0xffffffffu, mx, 1));
+                mn = fminf(mn, __shfl_xor_sync(0xffffffffu, mn, 2)); mx = fmaxf(mx, __shfl_xor_sync(0xffffffffu, mx, 2));
+            }
+            if (mn == 0.f) mn = 0.f;
+            const __half hd = exact_scale(mx, mn);
+            const float delta = __half2float(hd);
+            const float inv = (delta == 0.f) ? 0.f : __frcp_rn(delta);   // scale 0: every code comes out 0
+            uint32_t q[32];
+#pragma unroll
+            for (int i = 0; i < 32; ++i) {
+                const float t = __fsub_rn(x[i], mn);
+                const float q0 = __fmul_rn(t, inv);
+                const float q1 = __fmaf_rn(__fmaf_rn(-q0, delta, t), inv, q0);      // = RN(t / delta)
+                const float y = fminf(fmaxf(q1, 0.f), 15.f) + 12582912.f;           // round half to even
+                q[i] = __float_as_uint(y) & 15u;
+            }
+            // token k = it*8 + rsub of the block; in-block byte of (channel block cb, row r): see code_byte_off
+            const int jt = rsub >> 1, bytepos = (rsub & 1) * 2 + it;
+#pragma unroll
+            for (int cbl = 0; cbl < 2; ++cbl) {
+                const int cb = 2 * grp + cbl;
+                unsigned char *dstb = vs + (cb >> 2) * 512 + jt * 16 + (cb & 3) * 4 + bytepos;
+#pragma unroll
+                for (int r = 0; r < 8; ++r) dstb[r * 64] = (unsigned char)(q[cbl * 16 + r] | (q[cbl * 16 + r + 8] << 4));
+            }
+            const int k = it * 8 + rsub;
+            if (p.groups == 4 || grp == 0) {
+                const int gs = p.groups == 4 ? grp : 0;
+                *reinterpret_cast<__half *>(vs + 1024 + gs * 32 + k * 2) = hd;                              // scale [g][16 tokens]
+                *reinterpret_cast<__half *>(vs + 1152 + k * (2 * p.groups) + gs * 2) = __float2half_rn(mn); // zero  [16 tokens][g]
+            }
+        }
+        __syncwarp();
+        const uint4 *src = reinterpret_cast<const uint4 *>(vs);
+        uint4 *dst = reinterpret_cast<uint4 *>(chunk + cl.val_off + vb * kValBlockBytes);
+        dst[lane] = src[lane];
+        dst[32 + lane] = src[32 + lane];
+        const int n16 = 2 * p.groups;                   // 16-byte pieces of a block's scale (and zero) plane
+        if (lane < n16) reinterpret_cast<uint4 *>(chunk + cl.scale_off + vb * (32 * p.groups))[lane] = src[64 + lane];
+        else if (lane >= 8 && lane < 8 + n16)
+            reinterpret_cast<uint4 *>(chunk + cl.zero_off + vb * (32 * p.groups))[lane - 8] = src[72 + lane - 8];
+        __syncwarp();
+    } else {                                            // ragged edge of the appended range: row by row
+        for (int k = 0; k < 16; ++k) {
+            const int tn = tn0 + k;
+            if (tn >= 0 && tn < n_new)
+                store_value_row(p.v + ((((size_t)ll * p.B + b) * p.Tn + tn) * p.Hkv + kvh) * kHeadDim,
+                                slab + (size_t)((pos0 + k) >> 5) * cl.bytes, cl, (pos0 + k) & 31, lane);
+        }
+    }
+}
+
+// Long appends, value side: one warp per block of 16 cache positions of one slab, no block-level synchronisation.
+// Units enumerate (slab, 16-position block) over the 128-aligned range that the appended tokens can touch.
+constexpr int kValueWarps = 4;
+__global__ void __launch_bounds__(kValueWarps * 32) prefill_values_kernel(PrefillParams p, NewCounts nn) {
+    __shared__ __align__(16) unsigned char vs_all[kValueWarps][1280];
+    const int lane = threadIdx.x & 31, warp = threadIdx.x >> 5;
+    const ChunkLayout cl = chunk_layout(p.m_words, p.groups);
+    const int blocks_per_seq = p.tiles_per_seq * (kPrefillTile / 16);
+    const long unit = (long)blockIdx.x * kValueWarps + warp;
+    const long n_units = (long)p.n_layers * p.B * p.Hkv * blocks_per_seq;
+    if (unit >= n_units) return;
+    const int blk = (int)(unit % blocks_per_seq);
+    const long slab_local = unit / blocks_per_seq;
+    const int kvh = (int)(slab_local % p.Hkv), b = (int)((slab_local / p.Hkv) % p.B), ll = (int)(slab_local / ((long)p.Hkv * p.B));
+    const int layer = p.layer_begin + ll;
+    const int len0 = p.len[layer * p.max_batch + b];
+    const int n_new = nn.v[b];
+    const int pos0 = (len0 / kPrefillTile) * kPrefillTile + blk * 16;
+    if (pos0 + 16 <= len0 || pos0 >= len0 + n_new) return;
+    unsigned char *slab = p.cache + ((size_t)(layer * p.max_batch + b) * p.Hkv + kvh) * p.slab_bytes;
+    store_value_block16(p, cl, slab, ll, b, kvh, len0, n_new, pos0, vs_all[warp], lane);
+}
+
 template <int NBC>
-__global__ void __launch_bounds__(kPrefillThreads, 2) prefill_kernel(PrefillParams p, NewCounts nn) {
+__global__ void __launch_bounds__(kPrefillThreads, 1) prefill_kernel(PrefillParams p, NewCounts nn) {
     using SM = PrefillSmem<NBC>;
     extern __shared__ unsigned char smem_unaligned[];
     unsigned char *smem = smem_unaligned + ((1024u - (smem_addr(smem_unaligned) & 1023u)) & 1023u);
-    unsigned char *Rs = smem, *As = smem + SM::kRBytes, *Vs = As + SM::kABytes;
+    unsigned char *Rs = smem, *As0 = smem + SM::kRBytes;        // key tile ti sits in buffer ti % kKeyStages at As0 + that * kABytes
     __shared__ uint32_t tmem_base_s;
-    __shared__ __align__(8) unsigned long long mma_bar_s;
+    __shared__ __align__(8) unsigned long long mma_bar_s[2];
     __shared__ int is_last, gave_up;
     const int tid = threadIdx.x, lane = tid & 31, warp = tid >> 5;
     const int m = p.m_words * 32;
@@ -311,14 +453,15 @@ __global__ void __launch_bounds__(kPrefillThreads, 2) prefill_kernel(PrefillPara
     const int len0 = p.len[layer * p.max_batch + b];
     const int n_new = nn.v[b];
     unsigned char *slab = p.cache + ((size_t)(layer * p.max_batch + b) * p.Hkv + kvh) * p.slab_bytes;
-    const uint32_t bar = smem_addr(&mma_bar_s);
+    const uint32_t bar0 = smem_addr(&mma_bar_s[0]);
 
     // a block that starts after some other block has given up a wait does nothing (keeps a failure short)
     if (tid == 0) gave_up = (*reinterpret_cast<volatile const int32_t *>(p.status) != kStatusOk);
     __syncthreads();
     const bool skip_all = gave_up != 0;                         // block-uniform
-    if (warp == 0 && !skip_all) tmem_alloc(smem_addr(&tmem_base_s), NBC);    // NBC fp32 accumulator columns x 128 lanes
-    if (tid == 0) { mbar_init(bar, 1); mbar_fence_init(); }
+    // two accumulators of NBC fp32 columns x 128 lanes: the MMAs of one tile run while the previous tile's signs are packed
+    if (warp == 0 && !skip_all) tmem_alloc(smem_addr(&tmem_base_s), 2 * NBC);
+    if (tid == 0) { mbar_init(bar0, 1); mbar_init(bar0 + 8, 1); mbar_fence_init(); }
     // ---- the two fp16 pieces of Rt[:, col0 .. col0+NBC), transposed: operand B[col][channel]
     {
         const uint16_t *src = p.Rh + ((size_t)layer * 2 * m + col0) * kHeadDim;        // [L][2][m][128]
@@ -328,207 +471,114 @@ __global__ void __launch_bounds__(kPrefillThreads, 2) prefill_kernel(PrefillPara
                         src + ((size_t)piece * m + n) * kHeadDim + c * 8, 16);
         }
     }
+    const int first_tile = len0 / kPrefillTile + tg * p.tiles_per_block;
+    // tiles of this block that overlap the appended range (block-uniform)
+    const int n_tiles = skip_all ? 0 : max(0, min(p.tiles_per_block,
+                                                   (len0 + n_new - first_tile * kPrefillTile + kPrefillTile - 1) / kPrefillTile));
+    // key tile ti -> buffer ti % kKeyStages: row r = position P0 + r; rows outside the appended range are zero
+    // A thread always copies the same 16-byte column piece c of rows r0, r0 + 16, ...: the shared-memory offsets and the
+    // global row pointers advance by constants (r0 + 16 k keeps r % 8, so the swizzle term is fixed).
+    const int ld_c = tid & 15, ld_r0 = tid >> 4;
+    constexpr int kRowsPerPass = kPrefillThreads / 16;
+    const uint32_t ld_soff = (uint32_t)kmajor_sw128_off(kPrefillTile, ld_r0, ld_c);
+    const size_t k_row_stride = (size_t)p.Hkv * kHeadDim;       // elements between consecutive tokens of one KV head
+    const uint16_t *k_seq = p.k + (((size_t)ll * p.B + b) * p.Tn * p.Hkv + kvh) * kHeadDim + ld_c * 8;   // token 0 of this head
+    auto load_key_tile = [&](int ti) {
+        const int tn0 = (first_tile + ti) * kPrefillTile + ld_r0 - len0;        // appended-token index of this thread's first row
+        const uint32_t dst0 = smem_addr(As0 + (ti % kKeyStages) * SM::kABytes) + ld_soff;
+#pragma unroll
+        for (int k = 0; k < kPrefillTile / kRowsPerPass; ++k) {
+            const int tn = tn0 + k * kRowsPerPass;
+            const bool ok = tn >= 0 && tn < n_new;
+            cp_async_16(dst0 + k * (kRowsPerPass * 128), k_seq + (size_t)(ok ? tn : 0) * k_row_stride, ok ? 16u : 0u);
+        }
+    };
     tc_fence_before_sync();
     __syncthreads();
     tc_fence_after_sync();
     const uint32_t tmem_d = skip_all ? 0u : tmem_base_s;
     const uint32_t idesc = umma_idesc_f16_m128(NBC);
-    const int first_tile = len0 / kPrefillTile + tg * p.tiles_per_block;
-    // key tile: row r = position P0 + r; rows outside the appended range are zero
-    auto load_key_tile = [&](int P0) {
-        for (int e = tid; e < kPrefillTile * 16; e += kPrefillThreads) {
-            const int c = e & 15, r = e >> 4;
-            const int tn = P0 + r - len0;
-            const bool ok = tn >= 0 && tn < n_new;
-            const uint16_t *src = p.k + ((((size_t)ll * p.B + b) * p.Tn + (ok ? tn : 0)) * p.Hkv + kvh) * kHeadDim + c * 8;
-            cp_async_16(smem_addr(As + kmajor_sw128_off(kPrefillTile, r, c)), src, ok ? 16u : 0u);
-        }
-    };
-    uint32_t parity = 0;
-    for (int ti = 0; ti < p.tiles_per_block && !skip_all; ++ti) {
-        const int P0 = (first_tile + ti) * kPrefillTile;
-        if (P0 >= len0 + n_new) break;                          // block-uniform
-        if (ti == 0) load_key_tile(P0);                         // later tiles were requested during the previous one
-        cp_async_wait_all();
-        fence_proxy_async_smem();                               // generic-proxy writes -> visible to the tensor cores
-        __syncthreads();
-        // ---- y = K x (Rh1 + Rh2)^T: one thread issues 2 pieces x 8 K-slices of 16
+    // y = K x (Rh1 + Rh2)^T for tile ti into accumulator ti % 2: one thread issues 2 pieces x 8 K-slices of 16
+    auto issue_mma = [&](int ti) {
         if (tid == 0) {
             tc_fence_after_sync();
-            const uint32_t a_base = smem_addr(As), r_base = smem_addr(Rs);
+            const uint32_t a_base = smem_addr(As0 + (ti % kKeyStages) * SM::kABytes), r_base = smem_addr(Rs);
+            const uint32_t acc = tmem_d + (uint32_t)((ti & 1) * NBC);
 #pragma unroll
             for (int piece = 0; piece < 2; ++piece)
 #pragma unroll
                 for (int ks = 0; ks < kHeadDim / 16; ++ks) {
                     const uint64_t ad = umma_desc_k_sw128(a_base + (ks >> 2) * (kPrefillTile * 128) + (ks & 3) * 32);
                     const uint64_t bd = umma_desc_k_sw128(r_base + piece * (NBC * 256) + (ks >> 2) * (NBC * 128) + (ks & 3) * 32);
-                    umma_f16(tmem_d, ad, bd, idesc, (piece | ks) ? 1u : 0u);
+                    umma_f16(acc, ad, bd, idesc, (piece | ks) ? 1u : 0u);
                 }
-            umma_commit(bar);
+            umma_commit(bar0 + 8 * (ti & 1));
         }
-        // ---- values: warp w quantises tokens P0 + 16w .. +15 (one value block); only the first column block does it
-        if (blockIdx.y == 0) {
-            const int pos0 = P0 + warp * 16;
-            const int tn0 = pos0 - len0;
-            unsigned char *chunk = slab + (size_t)(pos0 >> 5) * cl.bytes;
-            const int vb = (pos0 >> 4) & 1;
-            if (p.groups == 0 && tn0 >= 0 && tn0 + 16 <= n_new) {
-                // fp16 values, a whole block of 16 tokens: transposed through shared memory into the A-operand
-                // order, 32 channels (two channel blocks, 1024 contiguous bytes of the cache) per pass
-                unsigned char *vs = Vs + warp * 1280;
-                const size_t row_stride = (size_t)p.Hkv * kHeadDim;
-                const uint16_t *v0 = p.v + ((((size_t)ll * p.B + b) * p.Tn + tn0) * p.Hkv + kvh) * kHeadDim;
-                unsigned char *dst_block = chunk + cl.val_off + vb * kHalfBlockBytes;
-#pragma unroll 1
-                for (int pass = 0; pass < 4; ++pass) {
-                    uint4 raw[2];
+    };
+    int issued = 0, waited = 0;
+    // One copy group per tile, in tile order (an empty one where there is no tile), so that "all but the newest
+    // kKeyStages - 2 groups" always means "up to the tile whose MMAs start next".
+    if (n_tiles > 0) {
 #pragma unroll
-                    for (int i = 0; i < 2; ++i) {               // piece e: token e/4, channels pass*32 + (e%4)*8 .. +7
-                        const int e = lane + 32 * i;
-                        raw[i] = __ldg(reinterpret_cast<const uint4 *>(v0 + (size_t)(e >> 2) * row_stride + pass * 32) + (e & 3));
-                    }
-#pragma unroll
-                    for (int i = 0; i < 2; ++i) {
-                        const int e = lane + 32 * i, k = e >> 2, c16 = e & 3;
-                        const int j = (k & 7) >> 1, odd = k & 1, hi8 = k >> 3;
-                        unsigned char *base = vs + (c16 >> 1) * 512 + j * 16 + (hi8 * 2 + (c16 & 1)) * 4 + odd * 2;
-                        const uint32_t w4[4] = {raw[i].x, raw[i].y, raw[i].z, raw[i].w};
-#pragma unroll
-                        for (int x = 0; x < 8; ++x)             // channel row r = x of the channel block
-                            *reinterpret_cast<uint16_t *>(base + x * 64) = (uint16_t)(w4[x >> 1] >> ((x & 1) * 16));
-                    }
-                    __syncwarp();
-                    const uint4 *src = reinterpret_cast<const uint4 *>(vs);
-                    uint4 *dst = reinterpret_cast<uint4 *>(dst_block + pass * 1024);
-                    dst[lane] = src[lane];
-                    dst[32 + lane] = src[32 + lane];
-                    __syncwarp();
-                }
-            } else if (p.groups != 0 && tn0 >= 0 && tn0 + 16 <= n_new) {   // a whole block: assemble it in shared memory
-                // lane = (row rsub of 8, group grp of 4): 32 channels of one row per lane and pass, two passes
-                unsigned char *vs = Vs + warp * 1280;
-                const int rsub = lane >> 2, grp = lane & 3;
-                const size_t row_stride = (size_t)p.Hkv * kHeadDim;
-                const uint16_t *v0 = p.v + ((((size_t)ll * p.B + b) * p.Tn + tn0) * p.Hkv + kvh) * kHeadDim + grp * 32;
-                uint4 raw[2][4];
-#pragma unroll
-                for (int it = 0; it < 2; ++it)
-#pragma unroll
-                    for (int j = 0; j < 4; ++j)
-                        raw[it][j] = __ldg(reinterpret_cast<const uint4 *>(v0 + (size_t)(it * 8 + rsub) * row_stride) + j);
-#pragma unroll
-                for (int it = 0; it < 2; ++it) {
-                    float x[32];
-#pragma unroll
-                    for (int j = 0; j < 4; ++j) {
-                        const uint32_t w4[4] = {raw[it][j].x, raw[it][j].y, raw[it][j].z, raw[it][j].w};
-#pragma unroll
-                        for (int h = 0; h < 4; ++h) {
-                            const float2 f = half2_bits_to_float2(w4[h]);
-                            x[j * 8 + h * 2] = f.x;
-                            x[j * 8 + h * 2 + 1] = f.y;
-                        }
-                    }
-                    float mn = x[0], mx = x[0];
-#pragma unroll
-                    for (int i = 1; i < 32; ++i) { mn = fminf(mn, x[i]); mx = fmaxf(mx, x[i]); }
-                    if (p.groups == 1) {                        // one scale per vector: the row's four lanes agree
-                        mn = fminf(mn, __shfl_xor_sync(0xffffffffu, mn, 1)); mx = fmaxf(mx, __shfl_xor_sync(0xffffffffu, mx, 1));
-                        mn = fminf(mn, __shfl_xor_sync(0xffffffffu, mn, 2)); mx = fmaxf(mx, __shfl_xor_sync(0xffffffffu, mx, 2));
-                    }
-                    if (mn == 0.f) mn = 0.f;
-                    const __half hd = exact_scale(mx, mn);
-                    const float delta = __half2float(hd);
-                    const float inv = (delta == 0.f) ? 0.f : __frcp_rn(delta);   // scale 0: every code comes out 0
-                    uint32_t q[32];
-#pragma unroll
-                    for (int i = 0; i < 32; ++i) {
-                        const float t = __fsub_rn(x[i], mn);
-                        const float q0 = __fmul_rn(t, inv);
-                        const float q1 = __fmaf_rn(__fmaf_rn(-q0, delta, t), inv, q0);      // = RN(t / delta)
-                        const float y = fminf(fmaxf(q1, 0.f), 15.f) + 12582912.f;           // round half to even
-                        q[i] = __float_as_uint(y) & 15u;
-                    }
-                    // token k = it*8 + rsub of the block; in-block byte of (channel block cb, row r): see code_byte_off
-                    const int jt = rsub >> 1, bytepos = (rsub & 1) * 2 + it;
-#pragma unroll
-                    for (int cbl = 0; cbl < 2; ++cbl) {
-                        const int cb = 2 * grp + cbl;
-                        unsigned char *dstb = vs + (cb >> 2) * 512 + jt * 16 + (cb & 3) * 4 + bytepos;
-#pragma unroll
-                        for (int r = 0; r < 8; ++r) dstb[r * 64] = (unsigned char)(q[cbl * 16 + r] | (q[cbl * 16 + r + 8] << 4));
-                    }
-                    const int k = it * 8 + rsub;
-                    if (p.groups == 4 || grp == 0) {
-                        const int gs = p.groups == 4 ? grp : 0;
-                        *reinterpret_cast<__half *>(vs + 1024 + gs * 32 + k * 2) = hd;                              // scale [g][16 tokens]
-                        *reinterpret_cast<__half *>(vs + 1152 + k * (2 * p.groups) + gs * 2) = __float2half_rn(mn); // zero  [16 tokens][g]
-                    }
-                }
-                __syncwarp();
-                const uint4 *src = reinterpret_cast<const uint4 *>(vs);
-                uint4 *dst = reinterpret_cast<uint4 *>(chunk + cl.val_off + vb * kValBlockBytes);
-                dst[lane] = src[lane];
-                dst[32 + lane] = src[32 + lane];
-                const int n16 = 2 * p.groups;                   // 16-byte pieces of a block's scale (and zero) plane
-                if (lane < n16) reinterpret_cast<uint4 *>(chunk + cl.scale_off + vb * (32 * p.groups))[lane] = src[64 + lane];
-                else if (lane >= 8 && lane < 8 + n16)
-                    reinterpret_cast<uint4 *>(chunk + cl.zero_off + vb * (32 * p.groups))[lane - 8] = src[72 + lane - 8];
-                __syncwarp();
-            } else {                                            // ragged edge of the appended range: row by row
-                for (int k = 0; k < 16; ++k) {
-                    const int tn = tn0 + k;
-                    if (tn >= 0 && tn < n_new)
-                        store_value_row(p.v + ((((size_t)ll * p.B + b) * p.Tn + tn) * p.Hkv + kvh) * kHeadDim,
-                                        slab + (size_t)((pos0 + k) >> 5) * cl.bytes, cl, (pos0 + k) & 31, lane);
-                }
-            }
+        for (int t = 0; t < kKeyStages; ++t) {                  // the projection pieces travel with tile 0's group
+            if (t < n_tiles) load_key_tile(t);
+            cp_async_commit();
         }
+        cp_async_wait_group<kKeyStages - 1>();
+        fence_proxy_async_smem();                               // generic-proxy writes -> visible to the tensor cores
+        __syncthreads();
+        issue_mma(0);
+        issued = 1;
+    }
+    // Steady state of iteration ti: the MMAs of tile ti are running or done, tiles up to ti + kKeyStages - 1 are landing.
+    for (int ti = 0; ti < n_tiles; ++ti) {
+        if (ti + 1 < n_tiles) {                                 // start tile ti+1's MMAs behind tile ti's
+            cp_async_wait_group<kKeyStages - 2>();
+            fence_proxy_async_smem();
+            __syncthreads();                                    // also: every thread is done with accumulator (ti+1) % 2
+            if (gave_up) break;
+            issue_mma(ti + 1);
+            issued = ti + 2;
+        }
+        const bool done = mbar_wait_bounded(bar0 + 8 * (ti & 1), (uint32_t)((ti >> 1) & 1), kWaitLimitNs);
+        waited = ti + 1;
+        tc_fence_after_sync();
+        // the tensor cores are done with this tile's key buffer: request the tile that will use it next
+        if (done && ti + kKeyStages < n_tiles) load_key_tile(ti + kKeyStages);
+        cp_async_commit();
         // ---- signs: thread = accumulator row 32*(warp%4) + lane (a warp can only read the TMEM lanes of its
         // quarter); warps 0-3 take the lower half of the columns, warps 4-7 the upper half
-        {
-            const bool done = mbar_wait_bounded(bar, parity, kWaitLimitNs);
-            tc_fence_after_sync();
-            // the tensor cores are done with the key tile: request the next one right away, so
-            // that its latency hides behind the sign packing and the rest of the value quantisation
-            if (done && ti + 1 < p.tiles_per_block && P0 + kPrefillTile < len0 + n_new) {
-                const int Pn = P0 + kPrefillTile;
-                for (int e = tid; e < kPrefillTile * 16; e += kPrefillThreads) {
-                    const int c = e & 15, r = e >> 4;
-                    const int tnn = Pn + r - len0;
-                    const bool ok = tnn >= 0 && tnn < n_new;
-                    const uint16_t *src = p.k + ((((size_t)ll * p.B + b) * p.Tn + (ok ? tnn : 0)) * p.Hkv + kvh) * kHeadDim + c * 8;
-                    cp_async_16(smem_addr(As + kmajor_sw128_off(kPrefillTile, r, c)), src, ok ? 16u : 0u);
-                }
-            }
-            if (done) {
-                const int quarter = warp & 3, whalf = warp >> 2;
-                const int pos = P0 + quarter * 32 + lane, tn = pos - len0;
-                unsigned char *kw = slab + (size_t)(pos >> 5) * cl.bytes + (pos & 31) * 4;
+        if (done) {
+            const int P0 = (first_tile + ti) * kPrefillTile;
+            const int quarter = warp & 3, whalf = warp >> 2;
+            const int pos = P0 + quarter * 32 + lane, tn = pos - len0;
+            unsigned char *kw = slab + (size_t)(pos >> 5) * cl.bytes + (pos & 31) * 4;
 #pragma unroll
-                for (int wi = 0; wi < NBC / 64; ++wi) {
-                    const int w = whalf * (NBC / 64) + wi;
-                    uint32_t y[32];
-                    tmem_ld_32cols(tmem_d + ((uint32_t)(quarter * 32) << 16) + w * 32, y);
-                    uint32_t word = 0;
+            for (int wi = 0; wi < NBC / 64; ++wi) {
+                const int w = whalf * (NBC / 64) + wi;
+                uint32_t y[32];
+                tmem_ld_32cols(tmem_d + ((uint32_t)(quarter * 32) << 16) + (uint32_t)((ti & 1) * NBC) + w * 32, y);
+                // bit j = (y_j >= 0): shift the sign bits in from column 31 down to 0, then invert. Adding +0 first
+                // turns a negative zero into a positive one, so that it counts as >= 0 like every other zero.
+                uint32_t neg = 0;
 #pragma unroll
-                    for (int j = 0; j < 32; ++j) word |= (__uint_as_float(y[j]) >= 0.f ? 1u : 0u) << j;
-                    if (tn >= 0 && tn < n_new) *reinterpret_cast<uint32_t *>(kw + (col0 / 32 + w) * 128) = word;
-                }
-            } else if (lane == 0) {
-                atomicExch(p.status, kStatusWaitTimeout);
-                gave_up = 1;
+                for (int j = 31; j >= 0; --j)
+                    neg = __funnelshift_l(__float_as_uint(__uint_as_float(y[j]) + 0.f), neg, 1);
+                if (tn >= 0 && tn < n_new) *reinterpret_cast<uint32_t *>(kw + (col0 / 32 + w) * 128) = ~neg;
             }
-            tc_fence_before_sync();
+        } else if (lane == 0) {
+            atomicExch(p.status, kStatusWaitTimeout);
+            gave_up = 1;
         }
-        parity ^= 1;
-        __syncthreads();                                        // the key tile and the accumulator are free again
-        if (gave_up) break;
+        tc_fence_before_sync();
     }
+    // after a failed wait: give MMAs that were issued but not waited for a bounded time before the TMEM goes back
+    for (int ti = waited; ti < issued; ++ti)
+        (void)mbar_wait_bounded(bar0 + 8 * (ti & 1), (uint32_t)((ti >> 1) & 1), 100000000ull);
     cp_async_wait_all();
     tc_fence_before_sync();
     __syncthreads();
-    if (warp == 0 && !skip_all) { tc_fence_after_sync(); tmem_dealloc(tmem_d, NBC); }
+    if (warp == 0 && !skip_all) { tc_fence_after_sync(); tmem_dealloc(tmem_d, 2 * NBC); }
     // ---- the last block to finish publishes the new lengths
     if (tid == 0) {
         __threadfence();
@@ -1121,7 +1171,15 @@ static cudaError_t launch_prefill_t(const PrefillParams &p, const NewCounts &nn,
 }
 
 cudaError_t launch_prefill(const PrefillParams &p, const NewCounts &nn, cudaStream_t st, int *launches) {
-    cudaError_t e = (p.m_words * 32 >= 128) ? launch_prefill_t<128>(p, nn, st) : launch_prefill_t<64>(p, nn, st);
+    // values first; the key kernel's last block then publishes the new lengths
+    const long units = (long)p.n_layers * p.B * p.Hkv * p.tiles_per_seq * (kPrefillTile / 16);
+    const long vblocks = (units + kValueWarps - 1) / kValueWarps;
+    if (vblocks <= 0 || vblocks > 0x7fffffffL) return cudaErrorInvalidConfiguration;
+    prefill_values_kernel<<<(unsigned)vblocks, kValueWarps * 32, 0, st>>>(p, nn);
+    cudaError_t e = cudaGetLastError();
+    if (e != cudaSuccess) return e;
+    ++*launches;
+    e = (p.m_words * 32 >= 128) ? launch_prefill_t<128>(p, nn, st) : launch_prefill_t<64>(p, nn, st);
     if (e == cudaSuccess) ++*launches;
     return e;
 }
