@@ -257,7 +257,7 @@ __global__ void __launch_bounds__(kProjThreads) prepare_kernel(AppendParams ap, 
 //   the correctly rounded result and in fp64 otherwise.
 //   Every wait is bounded; TMEM is allocated once per block and always released before the block exits.
 // ===========================================================================
-constexpr int kPrefillThreads = 256;
+constexpr int kPrefillThreads = 512;
 constexpr int kPrefillTile = 128;              // cache positions per tile
 constexpr int kKeyStages = 4;                  // key tile buffers: tiles are requested three ahead of the MMAs that read them
 
@@ -353,25 +353,54 @@ __device__ __forceinline__ void store_value_block16(const PrefillParams &p, cons
                     x[j * 8 + h * 2 + 1] = f.y;
                 }
             }
-            float mn = x[0], mx = x[0];
+            // minimum and maximum on the packed halves (comparisons only: exact), two channels per instruction
+            __half2 mn2, mx2;
+            {
+                const uint32_t w0 = raw[it][0].x;
+                mn2 = *reinterpret_cast<const __half2 *>(&w0);
+                mx2 = mn2;
+            }
 #pragma unroll
-            for (int i = 1; i < 32; ++i) { mn = fminf(mn, x[i]); mx = fmaxf(mx, x[i]); }
+            for (int j = 0; j < 4; ++j) {
+                const uint32_t w4[4] = {raw[it][j].x, raw[it][j].y, raw[it][j].z, raw[it][j].w};
+#pragma unroll
+                for (int h = 0; h < 4; ++h) {
+                    if (j == 0 && h == 0) continue;
+                    const __half2 hv = *reinterpret_cast<const __half2 *>(&w4[h]);
+                    mn2 = __hmin2(mn2, hv);
+                    mx2 = __hmax2(mx2, hv);
+                }
+            }
+            float mn = fminf(__low2float(mn2), __high2float(mn2)), mx = fmaxf(__low2float(mx2), __high2float(mx2));
             if (p.groups == 1) {                        // one scale per vector: the row's four lanes agree
                 mn = fminf(mn, __shfl_xor_sync(0xffffffffu, mn, 1)); mx = fmaxf(mx, __shfl_xor_sync(0xffffffffu, mx, 1));
                 mn = fminf(mn, __shfl_xor_sync(0xffffffffu, mn, 2)); mx = fmaxf(mx, __shfl_xor_sync(0xffffffffu, mx, 2));
             }
-            if (mn == 0.f) mn = 0.f;
+            if (mn == 0.f) mn = 0.f;                    // one spelling of zero
+            if (mx == 0.f) mx = 0.f;
             const __half hd = exact_scale(mx, mn);
             const float delta = __half2float(hd);
             const float inv = (delta == 0.f) ? 0.f : __frcp_rn(delta);   // scale 0: every code comes out 0
+            // q[i]: the bits of code + 1.5 * 2^23, i.e. the code in the low four bits and zeros up to bit 21.
+            // t >= 0, and with a normal fp16 scale t / scale <= 15 / (1 - 2^-11) < 15.5: nothing to clamp. Only a
+            // subnormal scale (a range below 15 * 2^-14) can overshoot.
             uint32_t q[32];
+            if (delta >= 6.103515625e-05f || delta == 0.f) {
 #pragma unroll
-            for (int i = 0; i < 32; ++i) {
-                const float t = __fsub_rn(x[i], mn);
-                const float q0 = __fmul_rn(t, inv);
-                const float q1 = __fmaf_rn(__fmaf_rn(-q0, delta, t), inv, q0);      // = RN(t / delta)
-                const float y = fminf(fmaxf(q1, 0.f), 15.f) + 12582912.f;           // round half to even
-                q[i] = __float_as_uint(y) & 15u;
+                for (int i = 0; i < 32; ++i) {
+                    const float t = __fsub_rn(x[i], mn);
+                    const float q0 = __fmul_rn(t, inv);
+                    const float q1 = __fmaf_rn(__fmaf_rn(-q0, delta, t), inv, q0);  // = RN(t / delta)
+                    q[i] = __float_as_uint(q1 + 12582912.f);                        // round half to even
+                }
+            } else {
+#pragma unroll
+                for (int i = 0; i < 32; ++i) {
+                    const float t = __fsub_rn(x[i], mn);
+                    const float q0 = __fmul_rn(t, inv);
+                    const float q1 = __fmaf_rn(__fmaf_rn(-q0, delta, t), inv, q0);
+                    q[i] = __float_as_uint(fminf(q1, 15.f) + 12582912.f);
+                }
             }
             // token k = it*8 + rsub of the block; in-block byte of (channel block cb, row r): see code_byte_off
             const int jt = rsub >> 1, bytepos = (rsub & 1) * 2 + it;
@@ -380,7 +409,8 @@ __device__ __forceinline__ void store_value_block16(const PrefillParams &p, cons
                 const int cb = 2 * grp + cbl;
                 unsigned char *dstb = vs + (cb >> 2) * 512 + jt * 16 + (cb & 3) * 4 + bytepos;
 #pragma unroll
-                for (int r = 0; r < 8; ++r) dstb[r * 64] = (unsigned char)(q[cbl * 16 + r] | (q[cbl * 16 + r + 8] << 4));
+                for (int r = 0; r < 8; ++r)             // low byte of lo + 16 * hi = the two codes (the constant's low byte is 0)
+                    dstb[r * 64] = (unsigned char)(q[cbl * 16 + r] + 16u * q[cbl * 16 + r + 8]);
             }
             const int k = it * 8 + rsub;
             if (p.groups == 4 || grp == 0) {
@@ -459,15 +489,17 @@ __global__ void __launch_bounds__(kPrefillThreads, 1) prefill_kernel(PrefillPara
     if (tid == 0) gave_up = (*reinterpret_cast<volatile const int32_t *>(p.status) != kStatusOk);
     __syncthreads();
     const bool skip_all = gave_up != 0;                         // block-uniform
-    // two accumulators of NBC fp32 columns x 128 lanes: the MMAs of one tile run while the previous tile's signs are packed
-    if (warp == 0 && !skip_all) tmem_alloc(smem_addr(&tmem_base_s), 2 * NBC);
+    // two accumulators of 2 * NBC fp32 columns x 128 lanes (the products with the two pieces of the projection side by
+    // side): the MMAs of one tile run while the previous tile's signs are packed
+    if (warp == 0 && !skip_all) tmem_alloc(smem_addr(&tmem_base_s), 4 * NBC);
     if (tid == 0) { mbar_init(bar0, 1); mbar_init(bar0 + 8, 1); mbar_fence_init(); }
     // ---- the two fp16 pieces of Rt[:, col0 .. col0+NBC), transposed: operand B[col][channel]
     {
         const uint16_t *src = p.Rh + ((size_t)layer * 2 * m + col0) * kHeadDim;        // [L][2][m][128]
         for (int e = tid; e < 2 * NBC * 16; e += kPrefillThreads) {
             const int c = e & 15, n = (e >> 4) % NBC, piece = e / (16 * NBC);
-            cp_async_16(smem_addr(Rs + piece * (NBC * 256) + kmajor_sw128_off(NBC, n, c)),
+            // one operand of 2 * NBC rows: row piece * NBC + n
+            cp_async_16(smem_addr(Rs + kmajor_sw128_off(2 * NBC, piece * NBC + n, c)),
                         src + ((size_t)piece * m + n) * kHeadDim + c * 8, 16);
         }
     }
@@ -497,21 +529,19 @@ __global__ void __launch_bounds__(kPrefillThreads, 1) prefill_kernel(PrefillPara
     __syncthreads();
     tc_fence_after_sync();
     const uint32_t tmem_d = skip_all ? 0u : tmem_base_s;
-    const uint32_t idesc = umma_idesc_f16_m128(NBC);
-    // y = K x (Rh1 + Rh2)^T for tile ti into accumulator ti % 2: one thread issues 2 pieces x 8 K-slices of 16
+    const uint32_t idesc = umma_idesc_f16_m128(2 * NBC);
+    // [K x Rh1^T | K x Rh2^T] for tile ti into accumulator ti % 2: one thread issues 8 K-slices of 16, N = 2 * NBC
     auto issue_mma = [&](int ti) {
         if (tid == 0) {
             tc_fence_after_sync();
             const uint32_t a_base = smem_addr(As0 + (ti % kKeyStages) * SM::kABytes), r_base = smem_addr(Rs);
-            const uint32_t acc = tmem_d + (uint32_t)((ti & 1) * NBC);
+            const uint32_t acc = tmem_d + (uint32_t)((ti & 1) * 2 * NBC);
 #pragma unroll
-            for (int piece = 0; piece < 2; ++piece)
-#pragma unroll
-                for (int ks = 0; ks < kHeadDim / 16; ++ks) {
-                    const uint64_t ad = umma_desc_k_sw128(a_base + (ks >> 2) * (kPrefillTile * 128) + (ks & 3) * 32);
-                    const uint64_t bd = umma_desc_k_sw128(r_base + piece * (NBC * 256) + (ks >> 2) * (NBC * 128) + (ks & 3) * 32);
-                    umma_f16(acc, ad, bd, idesc, (piece | ks) ? 1u : 0u);
-                }
+            for (int ks = 0; ks < kHeadDim / 16; ++ks) {
+                const uint64_t ad = umma_desc_k_sw128(a_base + (ks >> 2) * (kPrefillTile * 128) + (ks & 3) * 32);
+                const uint64_t bd = umma_desc_k_sw128(r_base + (ks >> 2) * (2 * NBC * 128) + (ks & 3) * 32);
+                umma_f16(acc, ad, bd, idesc, ks ? 1u : 0u);
+            }
             umma_commit(bar0 + 8 * (ti & 1));
         }
     };
@@ -547,24 +577,29 @@ __global__ void __launch_bounds__(kPrefillThreads, 1) prefill_kernel(PrefillPara
         if (done && ti + kKeyStages < n_tiles) load_key_tile(ti + kKeyStages);
         cp_async_commit();
         // ---- signs: thread = accumulator row 32*(warp%4) + lane (a warp can only read the TMEM lanes of its
-        // quarter); warps 0-3 take the lower half of the columns, warps 4-7 the upper half
+        // quarter); warps 4g..4g+3 take columns 32g..32g+31 = one key word per thread
         if (done) {
             const int P0 = (first_tile + ti) * kPrefillTile;
-            const int quarter = warp & 3, whalf = warp >> 2;
+            const int quarter = warp & 3, w = warp >> 2;
             const int pos = P0 + quarter * 32 + lane, tn = pos - len0;
-            unsigned char *kw = slab + (size_t)(pos >> 5) * cl.bytes + (pos & 31) * 4;
+            if (w < NBC / 32) {
+                uint32_t y[32], y2[32];
+                const uint32_t acc = tmem_d + ((uint32_t)(quarter * 32) << 16) + (uint32_t)((ti & 1) * 2 * NBC) + w * 32;
+                tmem_ld_32cols(acc, y);
+                tmem_ld_32cols(acc + NBC, y2);
+                // bit j = (y_j >= 0): the sign bits are shifted in (four independent chains of eight columns), then
+                // inverted. Adding +0 first turns a negative zero into a positive one, so that it counts as >= 0
+                // like every other zero.
+                uint32_t part[4] = {0u, 0u, 0u, 0u};
 #pragma unroll
-            for (int wi = 0; wi < NBC / 64; ++wi) {
-                const int w = whalf * (NBC / 64) + wi;
-                uint32_t y[32];
-                tmem_ld_32cols(tmem_d + ((uint32_t)(quarter * 32) << 16) + (uint32_t)((ti & 1) * NBC) + w * 32, y);
-                // bit j = (y_j >= 0): shift the sign bits in from column 31 down to 0, then invert. Adding +0 first
-                // turns a negative zero into a positive one, so that it counts as >= 0 like every other zero.
-                uint32_t neg = 0;
+                for (int j = 7; j >= 0; --j)
 #pragma unroll
-                for (int j = 31; j >= 0; --j)
-                    neg = __funnelshift_l(__float_as_uint(__uint_as_float(y[j]) + 0.f), neg, 1);
-                if (tn >= 0 && tn < n_new) *reinterpret_cast<uint32_t *>(kw + (col0 / 32 + w) * 128) = ~neg;
+                    for (int k = 0; k < 4; ++k)
+                        part[k] = __funnelshift_l(__float_as_uint(__uint_as_float(y[8 * k + j]) + __uint_as_float(y2[8 * k + j]) + 0.f),
+                                                  part[k], 1);
+                const uint32_t neg = part[0] | (part[1] << 8) | (part[2] << 16) | (part[3] << 24);
+                if (tn >= 0 && tn < n_new)
+                    *reinterpret_cast<uint32_t *>(slab + (size_t)(pos >> 5) * cl.bytes + (pos & 31) * 4 + (col0 / 32 + w) * 128) = ~neg;
             }
         } else if (lane == 0) {
             atomicExch(p.status, kStatusWaitTimeout);
@@ -578,7 +613,7 @@ __global__ void __launch_bounds__(kPrefillThreads, 1) prefill_kernel(PrefillPara
     cp_async_wait_all();
     tc_fence_before_sync();
     __syncthreads();
-    if (warp == 0 && !skip_all) { tc_fence_after_sync(); tmem_dealloc(tmem_d, 2 * NBC); }
+    if (warp == 0 && !skip_all) { tc_fence_after_sync(); tmem_dealloc(tmem_d, 4 * NBC); }
     // ---- the last block to finish publishes the new lengths
     if (tid == 0) {
         __threadfence();
