@@ -117,6 +117,8 @@ struct h1b_ctx {
     bool profiling;
     std::vector<cudaEvent_t> events;   // pairs (before, after) around the split-K kernel
     size_t events_used;
+    cudaStream_t side;                 // long appends: the value kernel runs here, beside the key kernel
+    cudaEvent_t fork, join;            // ... forked from and joined back into the caller's stream
     std::string err;
 };
 
@@ -196,6 +198,7 @@ int h1b_init_projection(const h1b_config *cfg, uint64_t seed, const float *Rt_ho
     ctx->launches = 0;
     ctx->profiling = false;
     ctx->events_used = 0;
+    ctx->side = nullptr; ctx->fork = nullptr; ctx->join = nullptr;
     cudaStream_t st = static_cast<cudaStream_t>(stream);
     auto bail = [&](cudaError_t e, const char *what) {
         fail(nullptr, H1B_ERR_CUDA, "%s: %s", what, cudaGetErrorString(e));
@@ -221,6 +224,16 @@ int h1b_init_projection(const h1b_config *cfg, uint64_t seed, const float *Rt_ho
     if (e != cudaSuccess) return bail(e, "split_projection_kernel");
     e = cudaStreamSynchronize(st);
     if (e != cudaSuccess) return bail(e, "cudaStreamSynchronize");
+    // without these three the two long-append kernels simply run one after the other
+    if (cudaStreamCreateWithFlags(&ctx->side, cudaStreamNonBlocking) != cudaSuccess ||
+        cudaEventCreateWithFlags(&ctx->fork, cudaEventDisableTiming) != cudaSuccess ||
+        cudaEventCreateWithFlags(&ctx->join, cudaEventDisableTiming) != cudaSuccess) {
+        (void)cudaGetLastError();
+        if (ctx->join) cudaEventDestroy(ctx->join);
+        if (ctx->fork) cudaEventDestroy(ctx->fork);
+        if (ctx->side) cudaStreamDestroy(ctx->side);
+        ctx->side = nullptr; ctx->fork = nullptr; ctx->join = nullptr;
+    }
     *out = ctx;
     return H1B_OK;
 }
@@ -377,7 +390,7 @@ int h1b_append_kv(h1b_ctx *ctx, int layer_begin, int n_layers, const void *k, co
         int tpb = std::min(tiles, 32);
         while (tpb > 4 && slabs * ((tiles + tpb - 1) / tpb) < 148 * 4) tpb = (tpb + 1) / 2;
         pp.tiles_per_block = tpb;
-        H1B_CUDA(ctx, launch_prefill(pp, nn, static_cast<cudaStream_t>(stream), &launches));
+        H1B_CUDA(ctx, launch_prefill(pp, nn, static_cast<cudaStream_t>(stream), ctx->side, ctx->fork, ctx->join, &launches));
     } else {
         const AppendParams ap = append_params(ctx, layer_begin, n_layers, k, v, B, Tn);
         H1B_CUDA(ctx, launch_prepare(&ap, nullptr, nn, static_cast<cudaStream_t>(stream), &launches));
@@ -553,6 +566,9 @@ int h1b_free(h1b_ctx *ctx) {
     int rc = H1B_OK;
     if (cudaSetDevice(ctx->cfg.device) != cudaSuccess || cudaDeviceSynchronize() != cudaSuccess) rc = H1B_ERR_CUDA;
     for (cudaEvent_t e : ctx->events) cudaEventDestroy(e);
+    if (ctx->join) cudaEventDestroy(ctx->join);
+    if (ctx->fork) cudaEventDestroy(ctx->fork);
+    if (ctx->side) cudaStreamDestroy(ctx->side);
     delete ctx;
     return rc;
 }

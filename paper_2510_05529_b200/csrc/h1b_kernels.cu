@@ -257,7 +257,7 @@ __global__ void __launch_bounds__(kProjThreads) prepare_kernel(AppendParams ap, 
 //   the correctly rounded result and in fp64 otherwise.
 //   Every wait is bounded; TMEM is allocated once per block and always released before the block exits.
 // ===========================================================================
-constexpr int kPrefillThreads = 512;
+constexpr int kPrefillThreads = 256;       // few enough registers in use that blocks of the value kernel fit beside it
 constexpr int kPrefillTile = 128;              // cache positions per tile
 constexpr int kKeyStages = 4;                  // key tile buffers: tiles are requested three ahead of the MMAs that read them
 
@@ -439,27 +439,47 @@ __device__ __forceinline__ void store_value_block16(const PrefillParams &p, cons
     }
 }
 
+// End of both long-append kernels: the block that finishes last of all (key and value kernel together) adds the new
+// tokens to the lengths. Every block of both kernels has read the lengths by then.
+__device__ __forceinline__ void prefill_publish_lengths(const PrefillParams &p, const NewCounts &nn, int *is_last_s) {
+    __syncthreads();
+    if (threadIdx.x == 0) {
+        __threadfence();
+        *is_last_s = (atomicAdd(p.done, 1) == p.total_blocks - 1);
+    }
+    __syncthreads();
+    if (*is_last_s) {
+        for (int i = threadIdx.x; i < p.n_layers * p.B; i += blockDim.x)
+            p.len[(p.layer_begin + i / p.B) * p.max_batch + (i % p.B)] += nn.v[i % p.B];
+        if (threadIdx.x == 0) *p.done = 0;
+    }
+}
+
 // Long appends, value side: one warp per block of 16 cache positions of one slab, no block-level synchronisation.
 // Units enumerate (slab, 16-position block) over the 128-aligned range that the appended tokens can touch.
 constexpr int kValueWarps = 4;
 __global__ void __launch_bounds__(kValueWarps * 32) prefill_values_kernel(PrefillParams p, NewCounts nn) {
     __shared__ __align__(16) unsigned char vs_all[kValueWarps][1280];
+    __shared__ int is_last;
     const int lane = threadIdx.x & 31, warp = threadIdx.x >> 5;
     const ChunkLayout cl = chunk_layout(p.m_words, p.groups);
     const int blocks_per_seq = p.tiles_per_seq * (kPrefillTile / 16);
     const long unit = (long)blockIdx.x * kValueWarps + warp;
     const long n_units = (long)p.n_layers * p.B * p.Hkv * blocks_per_seq;
-    if (unit >= n_units) return;
-    const int blk = (int)(unit % blocks_per_seq);
-    const long slab_local = unit / blocks_per_seq;
-    const int kvh = (int)(slab_local % p.Hkv), b = (int)((slab_local / p.Hkv) % p.B), ll = (int)(slab_local / ((long)p.Hkv * p.B));
-    const int layer = p.layer_begin + ll;
-    const int len0 = p.len[layer * p.max_batch + b];
-    const int n_new = nn.v[b];
-    const int pos0 = (len0 / kPrefillTile) * kPrefillTile + blk * 16;
-    if (pos0 + 16 <= len0 || pos0 >= len0 + n_new) return;
-    unsigned char *slab = p.cache + ((size_t)(layer * p.max_batch + b) * p.Hkv + kvh) * p.slab_bytes;
-    store_value_block16(p, cl, slab, ll, b, kvh, len0, n_new, pos0, vs_all[warp], lane);
+    if (unit < n_units) {
+        const int blk = (int)(unit % blocks_per_seq);
+        const long slab_local = unit / blocks_per_seq;
+        const int kvh = (int)(slab_local % p.Hkv), b = (int)((slab_local / p.Hkv) % p.B), ll = (int)(slab_local / ((long)p.Hkv * p.B));
+        const int layer = p.layer_begin + ll;
+        const int len0 = p.len[layer * p.max_batch + b];
+        const int n_new = nn.v[b];
+        const int pos0 = (len0 / kPrefillTile) * kPrefillTile + blk * 16;
+        if (pos0 + 16 > len0 && pos0 < len0 + n_new) {
+            unsigned char *slab = p.cache + ((size_t)(layer * p.max_batch + b) * p.Hkv + kvh) * p.slab_bytes;
+            store_value_block16(p, cl, slab, ll, b, kvh, len0, n_new, pos0, vs_all[warp], lane);
+        }
+    }
+    prefill_publish_lengths(p, nn, &is_last);
 }
 
 template <int NBC>
@@ -467,7 +487,7 @@ __global__ void __launch_bounds__(kPrefillThreads, 1) prefill_kernel(PrefillPara
     using SM = PrefillSmem<NBC>;
     extern __shared__ unsigned char smem_unaligned[];
     unsigned char *smem = smem_unaligned + ((1024u - (smem_addr(smem_unaligned) & 1023u)) & 1023u);
-    unsigned char *Rs = smem, *As0 = smem + SM::kRBytes;        // key tile ti sits in buffer ti % kKeyStages at As0 + that * kABytes
+    unsigned char *Rs = smem, *As0 = smem + SM::kRBytes;        // key tile number t sits in buffer t % kKeyStages at As0 + that * kABytes
     __shared__ uint32_t tmem_base_s;
     __shared__ __align__(8) unsigned long long mma_bar_s[2];
     __shared__ int is_last, gave_up;
@@ -475,14 +495,8 @@ __global__ void __launch_bounds__(kPrefillThreads, 1) prefill_kernel(PrefillPara
     const int m = p.m_words * 32;
     const ChunkLayout cl = chunk_layout(p.m_words, p.groups);
     const int groups_per_slab = (p.tiles_per_seq + p.tiles_per_block - 1) / p.tiles_per_block;
-    const int tg = blockIdx.x % groups_per_slab;
-    const long slab_local = blockIdx.x / groups_per_slab;
-    const int kvh = (int)(slab_local % p.Hkv), b = (int)((slab_local / p.Hkv) % p.B), ll = (int)(slab_local / ((long)p.Hkv * p.B));
-    const int layer = p.layer_begin + ll;
-    const int col0 = blockIdx.y * NBC;         // first sketch column of this block
-    const int len0 = p.len[layer * p.max_batch + b];
-    const int n_new = nn.v[b];
-    unsigned char *slab = p.cache + ((size_t)(layer * p.max_batch + b) * p.Hkv + kvh) * p.slab_bytes;
+    const int col_blocks = (m + NBC - 1) / NBC;
+    const long n_work = (long)p.n_layers * p.B * p.Hkv * groups_per_slab * col_blocks;
     const uint32_t bar0 = smem_addr(&mma_bar_s[0]);
 
     // a block that starts after some other block has given up a wait does nothing (keeps a failure short)
@@ -493,62 +507,81 @@ __global__ void __launch_bounds__(kPrefillThreads, 1) prefill_kernel(PrefillPara
     // side): the MMAs of one tile run while the previous tile's signs are packed
     if (warp == 0 && !skip_all) tmem_alloc(smem_addr(&tmem_base_s), 4 * NBC);
     if (tid == 0) { mbar_init(bar0, 1); mbar_init(bar0 + 8, 1); mbar_fence_init(); }
-    // ---- the two fp16 pieces of Rt[:, col0 .. col0+NBC), transposed: operand B[col][channel]
-    {
-        const uint16_t *src = p.Rh + ((size_t)layer * 2 * m + col0) * kHeadDim;        // [L][2][m][128]
-        for (int e = tid; e < 2 * NBC * 16; e += kPrefillThreads) {
-            const int c = e & 15, n = (e >> 4) % NBC, piece = e / (16 * NBC);
-            // one operand of 2 * NBC rows: row piece * NBC + n
-            cp_async_16(smem_addr(Rs + kmajor_sw128_off(2 * NBC, piece * NBC + n, c)),
-                        src + ((size_t)piece * m + n) * kHeadDim + c * 8, 16);
-        }
-    }
-    const int first_tile = len0 / kPrefillTile + tg * p.tiles_per_block;
-    // tiles of this block that overlap the appended range (block-uniform)
-    const int n_tiles = skip_all ? 0 : max(0, min(p.tiles_per_block,
-                                                   (len0 + n_new - first_tile * kPrefillTile + kPrefillTile - 1) / kPrefillTile));
-    // key tile ti -> buffer ti % kKeyStages: row r = position P0 + r; rows outside the appended range are zero
+    tc_fence_before_sync();
+    __syncthreads();
+    tc_fence_after_sync();
+    const uint32_t tmem_d = skip_all ? 0u : tmem_base_s;
+    const uint32_t idesc = umma_idesc_f16_m128(2 * NBC);
     // A thread always copies the same 16-byte column piece c of rows r0, r0 + 16, ...: the shared-memory offsets and the
     // global row pointers advance by constants (r0 + 16 k keeps r % 8, so the swizzle term is fixed).
     const int ld_c = tid & 15, ld_r0 = tid >> 4;
     constexpr int kRowsPerPass = kPrefillThreads / 16;
     const uint32_t ld_soff = (uint32_t)kmajor_sw128_off(kPrefillTile, ld_r0, ld_c);
     const size_t k_row_stride = (size_t)p.Hkv * kHeadDim;       // elements between consecutive tokens of one KV head
-    const uint16_t *k_seq = p.k + (((size_t)ll * p.B + b) * p.Tn * p.Hkv + kvh) * kHeadDim + ld_c * 8;   // token 0 of this head
-    auto load_key_tile = [&](int ti) {
-        const int tn0 = (first_tile + ti) * kPrefillTile + ld_r0 - len0;        // appended-token index of this thread's first row
-        const uint32_t dst0 = smem_addr(As0 + (ti % kKeyStages) * SM::kABytes) + ld_soff;
-#pragma unroll
-        for (int k = 0; k < kPrefillTile / kRowsPerPass; ++k) {
-            const int tn = tn0 + k * kRowsPerPass;
-            const bool ok = tn >= 0 && tn < n_new;
-            cp_async_16(dst0 + k * (kRowsPerPass * 128), k_seq + (size_t)(ok ? tn : 0) * k_row_stride, ok ? 16u : 0u);
-        }
-    };
-    tc_fence_before_sync();
-    __syncthreads();
-    tc_fence_after_sync();
-    const uint32_t tmem_d = skip_all ? 0u : tmem_base_s;
-    const uint32_t idesc = umma_idesc_f16_m128(2 * NBC);
-    // [K x Rh1^T | K x Rh2^T] for tile ti into accumulator ti % 2: one thread issues 8 K-slices of 16, N = 2 * NBC
-    auto issue_mma = [&](int ti) {
-        if (tid == 0) {
-            tc_fence_after_sync();
-            const uint32_t a_base = smem_addr(As0 + (ti % kKeyStages) * SM::kABytes), r_base = smem_addr(Rs);
-            const uint32_t acc = tmem_d + (uint32_t)((ti & 1) * 2 * NBC);
-#pragma unroll
-            for (int ks = 0; ks < kHeadDim / 16; ++ks) {
-                const uint64_t ad = umma_desc_k_sw128(a_base + (ks >> 2) * (kPrefillTile * 128) + (ks & 3) * 32);
-                const uint64_t bd = umma_desc_k_sw128(r_base + (ks >> 2) * (2 * NBC * 128) + (ks & 3) * 32);
-                umma_f16(acc, ad, bd, idesc, ks ? 1u : 0u);
+
+    // The grid is at most one block per SM; a block walks over work items = (slab, run of up to tiles_per_block
+    // consecutive tiles, block of NBC sketch columns). `seq` numbers the tiles this block has pushed through the
+    // pipeline so far: buffer seq % kKeyStages, accumulator and barrier seq % 2, barrier parity (seq / 2) % 2.
+    int seq = 0;
+    int loaded_layer = -1, loaded_col0 = -1;                    // which projection block the shared memory holds
+    int issued = 0, waited = 0;                                 // tiles (by seq) whose MMAs were issued / waited for
+    for (long work = blockIdx.x; work < n_work && !skip_all; work += gridDim.x) {
+        const int cbk = (int)(work % col_blocks);
+        const int tg = (int)((work / col_blocks) % groups_per_slab);
+        const long slab_local = work / ((long)col_blocks * groups_per_slab);
+        const int kvh = (int)(slab_local % p.Hkv), b = (int)((slab_local / p.Hkv) % p.B), ll = (int)(slab_local / ((long)p.Hkv * p.B));
+        const int layer = p.layer_begin + ll;
+        const int col0 = cbk * NBC;                             // first sketch column of this work item
+        const int len0 = p.len[layer * p.max_batch + b];
+        const int n_new = nn.v[b];
+        unsigned char *slab = p.cache + ((size_t)(layer * p.max_batch + b) * p.Hkv + kvh) * p.slab_bytes;
+        const int first_tile = len0 / kPrefillTile + tg * p.tiles_per_block;
+        // tiles of this work item that overlap the appended range (block-uniform)
+        const int n_tiles = max(0, min(p.tiles_per_block,
+                                       (len0 + n_new - first_tile * kPrefillTile + kPrefillTile - 1) / kPrefillTile));
+        if (n_tiles == 0) continue;
+        // ---- the two fp16 pieces of Rt[:, col0 .. col0+NBC), transposed: one operand B[2 * NBC rows][channel].
+        // (All MMAs of the previous work item have completed: its last tile was waited for.)
+        if (layer != loaded_layer || col0 != loaded_col0) {
+            const uint16_t *src = p.Rh + ((size_t)layer * 2 * m + col0) * kHeadDim;        // [L][2][m][128]
+            for (int e = tid; e < 2 * NBC * 16; e += kPrefillThreads) {
+                const int c = e & 15, n = (e >> 4) % NBC, piece = e / (16 * NBC);
+                cp_async_16(smem_addr(Rs + kmajor_sw128_off(2 * NBC, piece * NBC + n, c)),
+                            src + ((size_t)piece * m + n) * kHeadDim + c * 8, 16);
             }
-            umma_commit(bar0 + 8 * (ti & 1));
+            loaded_layer = layer;
+            loaded_col0 = col0;
         }
-    };
-    int issued = 0, waited = 0;
-    // One copy group per tile, in tile order (an empty one where there is no tile), so that "all but the newest
-    // kKeyStages - 2 groups" always means "up to the tile whose MMAs start next".
-    if (n_tiles > 0) {
+        const uint16_t *k_seq = p.k + (((size_t)ll * p.B + b) * p.Tn * p.Hkv + kvh) * kHeadDim + ld_c * 8;   // token 0 of this head
+        // key tile ti of the work item: row r = position P0 + r; rows outside the appended range are zero
+        auto load_key_tile = [&](int ti) {
+            const int tn0 = (first_tile + ti) * kPrefillTile + ld_r0 - len0;    // appended-token index of this thread's first row
+            const uint32_t dst0 = smem_addr(As0 + ((seq + ti) % kKeyStages) * SM::kABytes) + ld_soff;
+#pragma unroll
+            for (int k = 0; k < kPrefillTile / kRowsPerPass; ++k) {
+                const int tn = tn0 + k * kRowsPerPass;
+                const bool ok = tn >= 0 && tn < n_new;
+                cp_async_16(dst0 + k * (kRowsPerPass * 128), k_seq + (size_t)(ok ? tn : 0) * k_row_stride, ok ? 16u : 0u);
+            }
+        };
+        // [K x Rh1^T | K x Rh2^T] for tile ti: one thread issues 8 K-slices of 16, N = 2 * NBC
+        auto issue_mma = [&](int ti) {
+            if (tid == 0) {
+                tc_fence_after_sync();
+                const int sq = seq + ti;
+                const uint32_t a_base = smem_addr(As0 + (sq % kKeyStages) * SM::kABytes), r_base = smem_addr(Rs);
+                const uint32_t acc = tmem_d + (uint32_t)((sq & 1) * 2 * NBC);
+#pragma unroll
+                for (int ks = 0; ks < kHeadDim / 16; ++ks) {
+                    const uint64_t ad = umma_desc_k_sw128(a_base + (ks >> 2) * (kPrefillTile * 128) + (ks & 3) * 32);
+                    const uint64_t bd = umma_desc_k_sw128(r_base + (ks >> 2) * (2 * NBC * 128) + (ks & 3) * 32);
+                    umma_f16(acc, ad, bd, idesc, ks ? 1u : 0u);
+                }
+                umma_commit(bar0 + 8 * (sq & 1));
+            }
+        };
+        // One copy group per tile, in tile order (an empty one where there is no tile), so that "all but the newest
+        // kKeyStages - 2 groups" always means "up to the tile whose MMAs start next".
 #pragma unroll
         for (int t = 0; t < kKeyStages; ++t) {                  // the projection pieces travel with tile 0's group
             if (t < n_tiles) load_key_tile(t);
@@ -558,73 +591,69 @@ __global__ void __launch_bounds__(kPrefillThreads, 1) prefill_kernel(PrefillPara
         fence_proxy_async_smem();                               // generic-proxy writes -> visible to the tensor cores
         __syncthreads();
         issue_mma(0);
-        issued = 1;
-    }
-    // Steady state of iteration ti: the MMAs of tile ti are running or done, tiles up to ti + kKeyStages - 1 are landing.
-    for (int ti = 0; ti < n_tiles; ++ti) {
-        if (ti + 1 < n_tiles) {                                 // start tile ti+1's MMAs behind tile ti's
-            cp_async_wait_group<kKeyStages - 2>();
-            fence_proxy_async_smem();
-            __syncthreads();                                    // also: every thread is done with accumulator (ti+1) % 2
-            if (gave_up) break;
-            issue_mma(ti + 1);
-            issued = ti + 2;
-        }
-        const bool done = mbar_wait_bounded(bar0 + 8 * (ti & 1), (uint32_t)((ti >> 1) & 1), kWaitLimitNs);
-        waited = ti + 1;
-        tc_fence_after_sync();
-        // the tensor cores are done with this tile's key buffer: request the tile that will use it next
-        if (done && ti + kKeyStages < n_tiles) load_key_tile(ti + kKeyStages);
-        cp_async_commit();
-        // ---- signs: thread = accumulator row 32*(warp%4) + lane (a warp can only read the TMEM lanes of its
-        // quarter); warps 4g..4g+3 take columns 32g..32g+31 = one key word per thread
-        if (done) {
-            const int P0 = (first_tile + ti) * kPrefillTile;
-            const int quarter = warp & 3, w = warp >> 2;
-            const int pos = P0 + quarter * 32 + lane, tn = pos - len0;
-            if (w < NBC / 32) {
-                uint32_t y[32], y2[32];
-                const uint32_t acc = tmem_d + ((uint32_t)(quarter * 32) << 16) + (uint32_t)((ti & 1) * 2 * NBC) + w * 32;
-                tmem_ld_32cols(acc, y);
-                tmem_ld_32cols(acc + NBC, y2);
-                // bit j = (y_j >= 0): the sign bits are shifted in (four independent chains of eight columns), then
-                // inverted. Adding +0 first turns a negative zero into a positive one, so that it counts as >= 0
-                // like every other zero.
-                uint32_t part[4] = {0u, 0u, 0u, 0u};
-#pragma unroll
-                for (int j = 7; j >= 0; --j)
-#pragma unroll
-                    for (int k = 0; k < 4; ++k)
-                        part[k] = __funnelshift_l(__float_as_uint(__uint_as_float(y[8 * k + j]) + __uint_as_float(y2[8 * k + j]) + 0.f),
-                                                  part[k], 1);
-                const uint32_t neg = part[0] | (part[1] << 8) | (part[2] << 16) | (part[3] << 24);
-                if (tn >= 0 && tn < n_new)
-                    *reinterpret_cast<uint32_t *>(slab + (size_t)(pos >> 5) * cl.bytes + (pos & 31) * 4 + (col0 / 32 + w) * 128) = ~neg;
+        issued = seq + 1;
+        // Steady state of iteration ti: the MMAs of tile ti are running or done, tiles up to ti + kKeyStages - 1 are landing.
+        bool stop = false;
+        for (int ti = 0; ti < n_tiles; ++ti) {
+            if (ti + 1 < n_tiles) {                             // start tile ti+1's MMAs behind tile ti's
+                cp_async_wait_group<kKeyStages - 2>();
+                fence_proxy_async_smem();
+                __syncthreads();                                // also: every thread is done with the accumulator that comes next
+                if (gave_up) { stop = true; break; }
+                issue_mma(ti + 1);
+                issued = seq + ti + 2;
             }
-        } else if (lane == 0) {
-            atomicExch(p.status, kStatusWaitTimeout);
-            gave_up = 1;
+            const int sq = seq + ti;
+            const bool done = mbar_wait_bounded(bar0 + 8 * (sq & 1), (uint32_t)((sq >> 1) & 1), kWaitLimitNs);
+            waited = sq + 1;
+            tc_fence_after_sync();
+            // the tensor cores are done with this tile's key buffer: request the tile that will use it next
+            if (done && ti + kKeyStages < n_tiles) load_key_tile(ti + kKeyStages);
+            cp_async_commit();
+            // ---- signs: thread = accumulator row 32*(warp%4) + lane (a warp can only read the TMEM lanes of its
+            // quarter); a warp packs one key word (32 columns) per thread at a time
+            if (done) {
+                const int P0 = (first_tile + ti) * kPrefillTile;
+                const int quarter = warp & 3;
+                const int pos = P0 + quarter * 32 + lane, tn = pos - len0;
+#pragma unroll
+                for (int w = warp >> 2; w < NBC / 32; w += kPrefillThreads / 128) {
+                    uint32_t y[32], y2[32];
+                    const uint32_t acc = tmem_d + ((uint32_t)(quarter * 32) << 16) + (uint32_t)((sq & 1) * 2 * NBC) + w * 32;
+                    tmem_ld_32cols(acc, y);
+                    tmem_ld_32cols(acc + NBC, y2);
+                    // bit j = (y_j >= 0): the sign bits are shifted in (four independent chains of eight columns), then
+                    // inverted. Adding +0 first turns a negative zero into a positive one, so that it counts as >= 0
+                    // like every other zero.
+                    uint32_t part[4] = {0u, 0u, 0u, 0u};
+#pragma unroll
+                    for (int j = 7; j >= 0; --j)
+#pragma unroll
+                        for (int k = 0; k < 4; ++k)
+                            part[k] = __funnelshift_l(__float_as_uint(__uint_as_float(y[8 * k + j]) + __uint_as_float(y2[8 * k + j]) + 0.f),
+                                                      part[k], 1);
+                    const uint32_t neg = part[0] | (part[1] << 8) | (part[2] << 16) | (part[3] << 24);
+                    if (tn >= 0 && tn < n_new)
+                        *reinterpret_cast<uint32_t *>(slab + (size_t)(pos >> 5) * cl.bytes + (pos & 31) * 4 + (col0 / 32 + w) * 128) = ~neg;
+                }
+            } else if (lane == 0) {
+                atomicExch(p.status, kStatusWaitTimeout);
+                gave_up = 1;
+            }
+            tc_fence_before_sync();
         }
-        tc_fence_before_sync();
+        seq += n_tiles;
+        __syncthreads();                                        // the accumulators, the key buffers and gave_up are settled
+        if (stop || gave_up) break;
     }
     // after a failed wait: give MMAs that were issued but not waited for a bounded time before the TMEM goes back
-    for (int ti = waited; ti < issued; ++ti)
-        (void)mbar_wait_bounded(bar0 + 8 * (ti & 1), (uint32_t)((ti >> 1) & 1), 100000000ull);
+    for (int sq = waited; sq < issued; ++sq)
+        (void)mbar_wait_bounded(bar0 + 8 * (sq & 1), (uint32_t)((sq >> 1) & 1), 100000000ull);
     cp_async_wait_all();
     tc_fence_before_sync();
     __syncthreads();
     if (warp == 0 && !skip_all) { tc_fence_after_sync(); tmem_dealloc(tmem_d, 4 * NBC); }
-    // ---- the last block to finish publishes the new lengths
-    if (tid == 0) {
-        __threadfence();
-        is_last = (atomicAdd(p.done, 1) == (int)(gridDim.x * gridDim.y) - 1);
-    }
-    __syncthreads();
-    if (is_last) {
-        for (int i = tid; i < p.n_layers * p.B; i += blockDim.x)
-            p.len[(p.layer_begin + i / p.B) * p.max_batch + (i % p.B)] += nn.v[i % p.B];
-        if (tid == 0) *p.done = 0;
-    }
+    prefill_publish_lengths(p, nn, &is_last);
 }
 
 // Rt (fp32, [L][d][m]) -> its two fp16 pieces, transposed to [L][2][m][d] (channel contiguous).
@@ -1185,8 +1214,13 @@ cudaError_t launch_prepare(const AppendParams *ap, const SketchParams *sp, const
     return cudaGetLastError();
 }
 
+static long prefill_key_blocks(const PrefillParams &p, int nbc) {
+    const long groups = (p.tiles_per_seq + p.tiles_per_block - 1) / p.tiles_per_block;
+    return (long)p.n_layers * p.B * p.Hkv * groups * ((p.m_words * 32 + nbc - 1) / nbc);
+}
+
 template <int NBC>
-static cudaError_t launch_prefill_t(const PrefillParams &p, const NewCounts &nn, cudaStream_t st) {
+static cudaError_t launch_prefill_t(const PrefillParams &p, const NewCounts &nn, cudaStream_t st, int grid) {
     using SM = PrefillSmem<NBC>;
     static bool attr_set[64] = {};
     int dev = 0;
@@ -1194,29 +1228,68 @@ static cudaError_t launch_prefill_t(const PrefillParams &p, const NewCounts &nn,
     if (dev >= 0 && dev < 64 && !attr_set[dev]) {
         cudaError_t e = cudaFuncSetAttribute(prefill_kernel<NBC>, cudaFuncAttributeMaxDynamicSharedMemorySize, SM::kTotal);
         if (e != cudaSuccess) return e;
+        // the largest shared-memory split, not the smallest that fits this kernel: the rest is for the value kernel's blocks
+        e = cudaFuncSetAttribute(prefill_kernel<NBC>, cudaFuncAttributePreferredSharedMemoryCarveout, cudaSharedmemCarveoutMaxShared);
+        if (e != cudaSuccess) return e;
         attr_set[dev] = true;
     }
-    const long groups = (p.tiles_per_seq + p.tiles_per_block - 1) / p.tiles_per_block;
-    const long gx = (long)p.n_layers * p.B * p.Hkv * groups;
-    if (gx <= 0 || gx > 0x7fffffffL) return cudaErrorInvalidConfiguration;
-    const int m = p.m_words * 32;
-    dim3 grid((unsigned)gx, (unsigned)((m + NBC - 1) / NBC));
-    prefill_kernel<NBC><<<grid, kPrefillThreads, SM::kTotal, st>>>(p, nn);
+    prefill_kernel<NBC><<<(unsigned)grid, kPrefillThreads, SM::kTotal, st>>>(p, nn);
     return cudaGetLastError();
 }
 
-cudaError_t launch_prefill(const PrefillParams &p, const NewCounts &nn, cudaStream_t st, int *launches) {
-    // values first; the key kernel's last block then publishes the new lengths
+// The value kernel (instruction-bound) and the key kernel (latency-bound around the tensor cores) are independent
+// until the lengths are published, so they run side by side: the value kernel on `side`, forked from and joined
+// back into `st` with the two events (all three may be null: then one after the other on `st`).
+cudaError_t launch_prefill(const PrefillParams &p_in, const NewCounts &nn, cudaStream_t st, cudaStream_t side,
+                           cudaEvent_t fork, cudaEvent_t join, int *launches) {
+    PrefillParams p = p_in;
+    const int nbc = (p.m_words * 32 >= 128) ? 128 : 64;
     const long units = (long)p.n_layers * p.B * p.Hkv * p.tiles_per_seq * (kPrefillTile / 16);
     const long vblocks = (units + kValueWarps - 1) / kValueWarps;
-    if (vblocks <= 0 || vblocks > 0x7fffffffL) return cudaErrorInvalidConfiguration;
-    prefill_values_kernel<<<(unsigned)vblocks, kValueWarps * 32, 0, st>>>(p, nn);
-    cudaError_t e = cudaGetLastError();
+    // key kernel: at most one block per SM, each walking over its share of the work items, so that all of its blocks
+    // are resident from the start and the value kernel's blocks can settle beside them
+    static int n_sm[64] = {};
+    int dev = 0;
+    cudaGetDevice(&dev);
+    if (dev < 0 || dev >= 64) return cudaErrorInvalidDevice;
+    if (!n_sm[dev]) {
+        cudaError_t ea = cudaDeviceGetAttribute(&n_sm[dev], cudaDevAttrMultiProcessorCount, dev);
+        if (ea != cudaSuccess) return ea;
+    }
+    const long kwork = prefill_key_blocks(p, nbc);
+    const long kblocks = kwork < n_sm[dev] ? kwork : n_sm[dev];
+    if (vblocks <= 0 || kblocks <= 0 || vblocks + kblocks > 0x7fffffffL) return cudaErrorInvalidConfiguration;
+    p.total_blocks = (int)(vblocks + kblocks);
+    const bool forked = side && fork && join;
+    cudaError_t e;
+    {   // both kernels ask for the same shared-memory / L1 split, or an SM set up for one would not take the other
+        static bool attr_set[64] = {};
+        int dev = 0;
+        cudaGetDevice(&dev);
+        if (dev >= 0 && dev < 64 && !attr_set[dev]) {
+            e = cudaFuncSetAttribute(prefill_values_kernel, cudaFuncAttributePreferredSharedMemoryCarveout,
+                                     cudaSharedmemCarveoutMaxShared);
+            if (e != cudaSuccess) return e;
+            attr_set[dev] = true;
+        }
+    }
+    if (forked) {
+        if ((e = cudaEventRecord(fork, st)) != cudaSuccess) return e;
+        if ((e = cudaStreamWaitEvent(side, fork, 0)) != cudaSuccess) return e;
+    }
+    // the key kernel first: one block of it settles on every SM (its shared memory allows no more), and the value
+    // kernel's small blocks fill the registers and issue slots that are left
+    e = (nbc == 128) ? launch_prefill_t<128>(p, nn, st, (int)kblocks) : launch_prefill_t<64>(p, nn, st, (int)kblocks);
     if (e != cudaSuccess) return e;
     ++*launches;
-    e = (p.m_words * 32 >= 128) ? launch_prefill_t<128>(p, nn, st) : launch_prefill_t<64>(p, nn, st);
-    if (e == cudaSuccess) ++*launches;
-    return e;
+    prefill_values_kernel<<<(unsigned)vblocks, kValueWarps * 32, 0, forked ? side : st>>>(p, nn);
+    if ((e = cudaGetLastError()) != cudaSuccess) return e;
+    ++*launches;
+    if (forked) {
+        if ((e = cudaEventRecord(join, side)) != cudaSuccess) return e;
+        if ((e = cudaStreamWaitEvent(st, join, 0)) != cudaSuccess) return e;
+    }
+    return cudaSuccess;
 }
 
 cudaError_t launch_split_projection(const float *Rt, uint16_t *Rh, int n_layers, int m, cudaStream_t st) {

@@ -13,7 +13,8 @@ cudaError_t launch_prepare(const AppendParams *ap, const SketchParams *sp, const
                            int *launches);
 // `before` / `after`, when not null, are recorded around the split-K attention kernel alone.
 // Long appends: tensor-core projection (Rh holds the two fp16 pieces made by launch_split_projection).
-cudaError_t launch_prefill(const PrefillParams &p, const NewCounts &nn, cudaStream_t st, int *launches);
+cudaError_t launch_prefill(const PrefillParams &p, const NewCounts &nn, cudaStream_t st, cudaStream_t side,
+                           cudaEvent_t fork, cudaEvent_t join, int *launches);
 cudaError_t launch_split_projection(const float *Rt, uint16_t *Rh, int n_layers, int m, cudaStream_t st);
 cudaError_t launch_decode(const DecodeParams &p, cudaStream_t st, int *launches, cudaEvent_t before = nullptr,
                           cudaEvent_t after = nullptr);

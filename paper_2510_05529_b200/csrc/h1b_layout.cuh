@@ -123,6 +123,8 @@ struct PrefillParams {          // long appends: tensor-core projection
     int layer_begin, n_layers, B, Tn, Hkv, max_batch, m_words, groups;
     int tiles_per_seq;          // 128-position tiles that can overlap the appended range of a sequence
     int tiles_per_block;        // consecutive tiles handled by one block (the projection is loaded once per block)
+    int total_blocks;           // blocks of the key kernel plus blocks of the value kernel: the last of them all to finish
+                                // publishes the new lengths (the two kernels may run side by side)
 };
 
 struct SketchParams {           // query sketch
