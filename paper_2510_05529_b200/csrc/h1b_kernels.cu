@@ -503,15 +503,14 @@ __global__ void __launch_bounds__(kPrefillThreads, 1) prefill_kernel(PrefillPara
     if (tid == 0) gave_up = (*reinterpret_cast<volatile const int32_t *>(p.status) != kStatusOk);
     __syncthreads();
     const bool skip_all = gave_up != 0;                         // block-uniform
-    // two accumulators of 2 * NBC fp32 columns x 128 lanes (the products with the two pieces of the projection side by
-    // side): the MMAs of one tile run while the previous tile's signs are packed
-    if (warp == 0 && !skip_all) tmem_alloc(smem_addr(&tmem_base_s), 4 * NBC);
+    // two accumulators of NBC fp32 columns x 128 lanes: the MMAs of one tile run while the previous tile's signs are packed
+    if (warp == 0 && !skip_all) tmem_alloc(smem_addr(&tmem_base_s), 2 * NBC);
     if (tid == 0) { mbar_init(bar0, 1); mbar_init(bar0 + 8, 1); mbar_fence_init(); }
     tc_fence_before_sync();
     __syncthreads();
     tc_fence_after_sync();
     const uint32_t tmem_d = skip_all ? 0u : tmem_base_s;
-    const uint32_t idesc = umma_idesc_f16_m128(2 * NBC);
+    const uint32_t idesc = umma_idesc_f16_m128(NBC);
     // A thread always copies the same 16-byte column piece c of rows r0, r0 + 16, ...: the shared-memory offsets and the
     // global row pointers advance by constants (r0 + 16 k keeps r % 8, so the swizzle term is fixed).
     const int ld_c = tid & 15, ld_r0 = tid >> 4;
@@ -540,7 +539,7 @@ __global__ void __launch_bounds__(kPrefillThreads, 1) prefill_kernel(PrefillPara
         const int n_tiles = max(0, min(p.tiles_per_block,
                                        (len0 + n_new - first_tile * kPrefillTile + kPrefillTile - 1) / kPrefillTile));
         if (n_tiles == 0) continue;
-        // ---- the two fp16 pieces of Rt[:, col0 .. col0+NBC), transposed: one operand B[2 * NBC rows][channel].
+        // ---- the two fp16 pieces of Rt[:, col0 .. col0+NBC), transposed and stacked: B[2 * NBC rows][channel].
         // (All MMAs of the previous work item have completed: its last tile was waited for.)
         if (layer != loaded_layer || col0 != loaded_col0) {
             const uint16_t *src = p.Rh + ((size_t)layer * 2 * m + col0) * kHeadDim;        // [L][2][m][128]
@@ -564,19 +563,21 @@ __global__ void __launch_bounds__(kPrefillThreads, 1) prefill_kernel(PrefillPara
                 cp_async_16(dst0 + k * (kRowsPerPass * 128), k_seq + (size_t)(ok ? tn : 0) * k_row_stride, ok ? 16u : 0u);
             }
         };
-        // [K x Rh1^T | K x Rh2^T] for tile ti: one thread issues 8 K-slices of 16, N = 2 * NBC
+        // y = K x (Rh1 + Rh2)^T for tile ti: one thread issues 2 pieces x 8 K-slices of 16 into one accumulator
         auto issue_mma = [&](int ti) {
             if (tid == 0) {
                 tc_fence_after_sync();
                 const int sq = seq + ti;
                 const uint32_t a_base = smem_addr(As0 + (sq % kKeyStages) * SM::kABytes), r_base = smem_addr(Rs);
-                const uint32_t acc = tmem_d + (uint32_t)((sq & 1) * 2 * NBC);
+                const uint32_t acc = tmem_d + (uint32_t)((sq & 1) * NBC);
 #pragma unroll
-                for (int ks = 0; ks < kHeadDim / 16; ++ks) {
-                    const uint64_t ad = umma_desc_k_sw128(a_base + (ks >> 2) * (kPrefillTile * 128) + (ks & 3) * 32);
-                    const uint64_t bd = umma_desc_k_sw128(r_base + (ks >> 2) * (2 * NBC * 128) + (ks & 3) * 32);
-                    umma_f16(acc, ad, bd, idesc, ks ? 1u : 0u);
-                }
+                for (int piece = 0; piece < 2; ++piece)         // rows piece * NBC .. of the stacked projection operand
+#pragma unroll
+                    for (int ks = 0; ks < kHeadDim / 16; ++ks) {
+                        const uint64_t ad = umma_desc_k_sw128(a_base + (ks >> 2) * (kPrefillTile * 128) + (ks & 3) * 32);
+                        const uint64_t bd = umma_desc_k_sw128(r_base + piece * (NBC * 128) + (ks >> 2) * (2 * NBC * 128) + (ks & 3) * 32);
+                        umma_f16(acc, ad, bd, idesc, (piece | ks) ? 1u : 0u);
+                    }
                 umma_commit(bar0 + 8 * (sq & 1));
             }
         };
@@ -618,10 +619,8 @@ __global__ void __launch_bounds__(kPrefillThreads, 1) prefill_kernel(PrefillPara
                 const int pos = P0 + quarter * 32 + lane, tn = pos - len0;
 #pragma unroll
                 for (int w = warp >> 2; w < NBC / 32; w += kPrefillThreads / 128) {
-                    uint32_t y[32], y2[32];
-                    const uint32_t acc = tmem_d + ((uint32_t)(quarter * 32) << 16) + (uint32_t)((sq & 1) * 2 * NBC) + w * 32;
-                    tmem_ld_32cols(acc, y);
-                    tmem_ld_32cols(acc + NBC, y2);
+                    uint32_t y[32];
+                    tmem_ld_32cols(tmem_d + ((uint32_t)(quarter * 32) << 16) + (uint32_t)((sq & 1) * NBC) + w * 32, y);
                     // bit j = (y_j >= 0): the sign bits are shifted in (four independent chains of eight columns), then
                     // inverted. Adding +0 first turns a negative zero into a positive one, so that it counts as >= 0
                     // like every other zero.
@@ -630,8 +629,7 @@ __global__ void __launch_bounds__(kPrefillThreads, 1) prefill_kernel(PrefillPara
                     for (int j = 7; j >= 0; --j)
 #pragma unroll
                         for (int k = 0; k < 4; ++k)
-                            part[k] = __funnelshift_l(__float_as_uint(__uint_as_float(y[8 * k + j]) + __uint_as_float(y2[8 * k + j]) + 0.f),
-                                                      part[k], 1);
+                            part[k] = __funnelshift_l(__float_as_uint(__uint_as_float(y[8 * k + j]) + 0.f), part[k], 1);
                     const uint32_t neg = part[0] | (part[1] << 8) | (part[2] << 16) | (part[3] << 24);
                     if (tn >= 0 && tn < n_new)
                         *reinterpret_cast<uint32_t *>(slab + (size_t)(pos >> 5) * cl.bytes + (pos & 31) * 4 + (col0 / 32 + w) * 128) = ~neg;
@@ -652,7 +650,7 @@ __global__ void __launch_bounds__(kPrefillThreads, 1) prefill_kernel(PrefillPara
     cp_async_wait_all();
     tc_fence_before_sync();
     __syncthreads();
-    if (warp == 0 && !skip_all) { tc_fence_after_sync(); tmem_dealloc(tmem_d, 4 * NBC); }
+    if (warp == 0 && !skip_all) { tc_fence_after_sync(); tmem_dealloc(tmem_d, 2 * NBC); }
     prefill_publish_lengths(p, nn, &is_last);
 }
 
