@@ -467,9 +467,12 @@ __global__ void __launch_bounds__(kValueWarps * 32) prefill_values_kernel(Prefil
     const long unit = (long)blockIdx.x * kValueWarps + warp;
     const long n_units = (long)p.n_layers * p.B * p.Hkv * blocks_per_seq;
     if (unit < n_units) {
-        const int blk = (int)(unit % blocks_per_seq);
-        const long slab_local = unit / blocks_per_seq;
-        const int kvh = (int)(slab_local % p.Hkv), b = (int)((slab_local / p.Hkv) % p.B), ll = (int)(slab_local / ((long)p.Hkv * p.B));
+        // KV head fastest: warps that run at the same time read the same token rows of neighbouring heads, i.e. whole
+        // contiguous [Hkv][d] rows of the input between them
+        const int kvh = (int)(unit % p.Hkv);
+        const int blk = (int)((unit / p.Hkv) % blocks_per_seq);
+        const long seq_local = unit / ((long)p.Hkv * blocks_per_seq);
+        const int b = (int)(seq_local % p.B), ll = (int)(seq_local / p.B);
         const int layer = p.layer_begin + ll;
         const int len0 = p.len[layer * p.max_batch + b];
         const int n_new = nn.v[b];
