@@ -209,7 +209,8 @@ int h1b_decode_attention_static(h1b_ctx *ctx, int layer_begin, int n_layers, con
  * memory makes the copies asynchronous) into staging inside the workspace,
  * appends one token per sequence to all L layers, runs decode attention over
  * all layers, copies the result to out (HOST, float32 [L][B][Hq][d]) and
- * synchronises the stream. */
+ * synchronises the stream. When k, v and q lie back to back in host memory (in
+ * that order) they travel in one copy. */
 int h1b_decode_step_host(h1b_ctx *ctx, const void *k_host, const void *v_host,
                          const void *q_host, float inv_tau, void *out_host, int B,
                          void *stream);

@@ -550,9 +550,23 @@ int h1b_decode_step_host(h1b_ctx *ctx, const void *k_host, const void *v_host, c
     cudaStream_t st = static_cast<cudaStream_t>(stream);
     const size_t L = ctx->cfg.n_layers, d = ctx->cfg.head_dim;
     const size_t kv_bytes = L * B * ctx->cfg.n_kv_heads * d * 2, q_bytes = L * B * ctx->cfg.n_q_heads * d * 2;
-    H1B_CUDA(ctx, cudaMemcpyAsync(ctx->ws + ctx->plan.stage_k, k_host, kv_bytes, cudaMemcpyHostToDevice, st));
-    H1B_CUDA(ctx, cudaMemcpyAsync(ctx->ws + ctx->plan.stage_v, v_host, kv_bytes, cudaMemcpyHostToDevice, st));
-    H1B_CUDA(ctx, cudaMemcpyAsync(ctx->ws + ctx->plan.stage_q, q_host, q_bytes, cudaMemcpyHostToDevice, st));
+    const unsigned char *kh = static_cast<const unsigned char *>(k_host);
+    bool one_copy = false;
+    if (static_cast<const unsigned char *>(v_host) == kh + kv_bytes &&
+        static_cast<const unsigned char *>(q_host) == kh + 2 * kv_bytes &&
+        ctx->plan.stage_v == ctx->plan.stage_k + kv_bytes && ctx->plan.stage_q == ctx->plan.stage_v + kv_bytes) {
+        // the three inputs lie back to back in host memory (and so does the staging): one copy instead of three.
+        // Neighbours that belong to different page-locked allocations are refused by the runtime before anything
+        // is enqueued: then the three copies below do the job.
+        one_copy = cudaMemcpyAsync(ctx->ws + ctx->plan.stage_k, k_host, 2 * kv_bytes + q_bytes, cudaMemcpyHostToDevice, st) ==
+                   cudaSuccess;
+        if (!one_copy) (void)cudaGetLastError();
+    }
+    if (!one_copy) {
+        H1B_CUDA(ctx, cudaMemcpyAsync(ctx->ws + ctx->plan.stage_k, k_host, kv_bytes, cudaMemcpyHostToDevice, st));
+        H1B_CUDA(ctx, cudaMemcpyAsync(ctx->ws + ctx->plan.stage_v, v_host, kv_bytes, cudaMemcpyHostToDevice, st));
+        H1B_CUDA(ctx, cudaMemcpyAsync(ctx->ws + ctx->plan.stage_q, q_host, q_bytes, cudaMemcpyHostToDevice, st));
+    }
     rc = h1b_decode_step(ctx, ctx->ws + ctx->plan.stage_k, ctx->ws + ctx->plan.stage_v, ctx->ws + ctx->plan.stage_q,
                          inv_tau, ctx->ws + ctx->plan.stage_out, B, stream);
     if (rc != H1B_OK) return rc;

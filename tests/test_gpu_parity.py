@@ -149,6 +149,16 @@ def test_host_step_equals_device_calls():
     out3 = r3["cache"].h1b_decode_step(kh.cuda(), vh.cuda(), r3["qd"], 16.0)
     assert np.array_equal(outh.numpy(), out3.cpu().numpy())
     assert r3["cache"].h1b_get_lengths(1)[:2].tolist() == [100, 51]
+    # ... and on a fourth one through the host entry point again, with k, v and q back to back in one pinned
+    # buffer (they then travel in a single copy)
+    r4 = build_and_decode(w, [99, 50], max_seq=128)
+    nk, nq = kh.numel(), qh.numel()
+    buf = torch.empty(2 * nk + nq, dtype=torch.float16).pin_memory()
+    k4, v4, q4 = buf[:nk].view(kh.shape), buf[nk:2 * nk].view(vh.shape), buf[2 * nk:].view(qh.shape)
+    k4.copy_(kh); v4.copy_(vh); q4.copy_(qh)
+    out4 = torch.empty(qh.shape, dtype=torch.float32).pin_memory()
+    r4["cache"].h1b_decode_step_host(k4, v4, q4, 16.0, out4)
+    assert np.array_equal(outh.numpy(), out4.numpy())
     # and against the oracle, end to end, for one sequence
     K = torch.cat([r["K"][:, :, :100], torch.zeros_like(r["K"][:, :, :1])], 2)
     V = torch.cat([r["V"][:, :, :100], torch.zeros_like(r["V"][:, :, :1])], 2)
