@@ -157,8 +157,9 @@ int h1b_decode_step_layers(h1b_ctx *ctx, int layer_begin, int n_layers, const vo
  * CUDA graph (make one ordinary call of each kind first: the first call sets
  * kernel attributes). The kernels read the sequence lengths from device memory,
  * so every replay appends at, and attends up to, the then-current end of each
- * sequence. Frozen at capture time: the pointers, B, n_new and the split plan
- * (its last split is open-ended, so growth is still covered). The host's copy of
+ * sequence. Frozen at capture time: the pointers, B, n_new and the number of
+ * splits per sequence (which chunks a split takes is worked out on the device
+ * from the length at that moment, so growth is covered). The host's copy of
  * the lengths only sees the captured calls, not their replays: call
  * h1b_sync_lengths() after replaying and before any other call on the context.
  * A replay that finds a sequence full writes nothing for it, leaves its length
@@ -187,7 +188,7 @@ int h1b_sync_lengths(h1b_ctx *ctx, void *stream);
  * Same arguments, same result and same errors as h1b_decode_attention(), plus:
  *   - H1B_ERR_CAPACITY, with the needed and the available byte counts in
  *     h1b_last_error(), when even one split per sequence does not fit:
- *     n_layers * B * Hkv * ((Hq/Hkv) * 528 + 4) bytes of partials and counters plus
+ *     n_layers * B * Hkv * (Hq/Hkv) * 528 bytes of partials plus
  *     L * max_batch * Hq * m/8 bytes of sketches must be <= 8 MiB. When more
  *     splits would fit the automatic choice, fewer are used (slower, same result
  *     up to summation order).
@@ -196,11 +197,10 @@ int h1b_sync_lengths(h1b_ctx *ctx, void *stream);
  *     (cudaGetSymbolAddress) and keeps it; make that first call outside any
  *     stream capture.
  * All contexts and all calls in the process share the one array per device, and
- * it keeps whatever the last call left in it. The only part that has to start
- * at zero, the per-sequence arrival counters, is cleared by each call (a
- * stream-ordered memset); everything else a call reads it has written itself. Two
- * calls whose kernels overlap on the GPU (different streams, different
- * contexts) race on it: order them on one stream or with events. */
+ * it keeps whatever the last call left in it; nothing in it has to be
+ * initialised, since a call reads only what it has written itself. Two calls
+ * whose kernels overlap on the GPU (different streams, different contexts)
+ * race on it: order them on one stream or with events. */
 int h1b_decode_attention_static(h1b_ctx *ctx, int layer_begin, int n_layers, const void *q,
                                 float inv_tau, void *out, int B, void *stream);
 

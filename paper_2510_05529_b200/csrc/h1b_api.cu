@@ -25,7 +25,7 @@ constexpr int kMaxQueryTokens = H1B_MAX_QUERY_TOKENS;
 constexpr int kPrefillMinTokens = 64;   // appends of at least this many tokens per sequence take the tensor-core path
 
 struct Plan {
-    size_t rt, rh, len, status, arrive, qwords, partial, stage_k, stage_v, stage_q, stage_out, dbg_q, dbg_s, cache, total;
+    size_t rt, rh, len, status, qwords, partial, stage_k, stage_v, stage_q, stage_out, dbg_q, dbg_s, cache, total;
     size_t partial_bytes, slab_bytes;
     int cap_tokens, m_words, gq, groups;
 };
@@ -70,7 +70,6 @@ int make_plan(const h1b_config *c, Plan *p) {
     p->rh = take(L * 2 * d * c->sketch_bits * sizeof(uint16_t));     // fp16 pieces of Rt for the tensor-core prefill
     p->len = take(L * B * sizeof(int32_t));
     p->status = take(64);
-    p->arrive = take(slabs * sizeof(int32_t));
     p->qwords = take(L * B * Hq * kMaxQueryTokens * p->m_words * sizeof(uint32_t));
     p->partial = take(p->partial_bytes);
     p->stage_k = take(L * B * Hkv * d * 2);
@@ -291,11 +290,12 @@ static void commit_lengths(h1b_ctx *ctx, int layer_begin, int n_layers, int B, c
         for (int b = 0; b < B; ++b) ctx->len_host[(size_t)l * ctx->cfg.max_batch + b] += nn.v[b];
 }
 
-// Enqueue the split-K attention kernel over scratch (qwords, partial, arrive). The sequence is split so that
-// there are about kTargetItems work items, capped by `max_items`; the last split of a sequence is open-ended,
-// so the result does not depend on how well the host's view of the lengths matches the device's.
+// Enqueue the split-K attention kernel over scratch (qwords, partial). Every sequence is split so that there are
+// about kTargetItems work items, capped by what the scratch holds. The host only chooses how many splits; which
+// chunks a split takes is worked out on the device from the sequence's length at that moment, so the result does
+// not depend on how well the host's view of the lengths matches the device's.
 static int enqueue_decode(h1b_ctx *ctx, int layer_begin, int n_layers, float inv_tau, void *out, int B,
-                          cudaStream_t st, uint32_t *qwords, float *partial, int32_t *arrive, size_t partial_bytes,
+                          cudaStream_t st, uint32_t *qwords, float *partial, size_t partial_bytes,
                           bool may_profile, int *launches, int Tq = 1) {
     // (query token, query head) pairs that share a KV head, and how many of them one work item takes
     const int vheads = ctx->plan.gq * Tq, gqk = vheads >= 3 ? 4 : vheads, vgroups = (vheads + gqk - 1) / gqk;
@@ -314,9 +314,6 @@ static int enqueue_decode(h1b_ctx *ctx, int layer_begin, int n_layers, float inv
                         splits, slabs, max_items);
         splits = (long)(max_items / (size_t)slabs);
     }
-    const int span = (maxlen + 255) / 256 * 256;
-    int split_tokens = (int)((span + splits - 1) / splits);
-    split_tokens = (split_tokens + kChunkTokens - 1) / kChunkTokens * kChunkTokens;
 
     DecodeParams dp;
     dp.cache = ctx->ws + ctx->plan.cache;
@@ -325,12 +322,11 @@ static int enqueue_decode(h1b_ctx *ctx, int layer_begin, int n_layers, float inv
     dp.partial = partial;
     dp.out = static_cast<float *>(out);
     dp.status = at<int32_t>(ctx, ctx->plan.status);
-    dp.arrive = arrive;
     dp.slab_bytes = ctx->plan.slab_bytes;
     dp.layer_begin = layer_begin; dp.n_layers = n_layers; dp.B = B; dp.Hkv = ctx->cfg.n_kv_heads;
     dp.Hq = ctx->cfg.n_q_heads; dp.max_batch = ctx->cfg.max_batch; dp.m_words = ctx->plan.m_words;
     dp.groups = ctx->plan.groups;
-    dp.splits = (int)splits; dp.split_tokens = split_tokens;
+    dp.splits = (int)splits;
     dp.Tq = Tq; dp.gqk = gqk; dp.vgroups = vgroups;
     dp.c2 = (float)(2.0 * (double)inv_tau * 1.4426950408889634 / (double)ctx->cfg.sketch_bits);
     cudaEvent_t ev0 = nullptr, ev1 = nullptr;
@@ -411,7 +407,7 @@ int h1b_decode_attention(h1b_ctx *ctx, int layer_begin, int n_layers, const void
     std::memset(&none, 0, sizeof none);
     H1B_CUDA(ctx, launch_prepare(nullptr, &sp, none, st, &launches));
     rc = enqueue_decode(ctx, layer_begin, n_layers, inv_tau, out, B, st, sp.qwords, at<float>(ctx, ctx->plan.partial),
-                        at<int32_t>(ctx, ctx->plan.arrive), ctx->plan.partial_bytes, true, &launches);
+                        ctx->plan.partial_bytes, true, &launches);
     ctx->launches += launches;
     return rc;
 }
@@ -436,7 +432,7 @@ int h1b_decode_attention_multi(h1b_ctx *ctx, int layer_begin, int n_layers, cons
     std::memset(&none, 0, sizeof none);
     H1B_CUDA(ctx, launch_prepare(nullptr, &sp, none, st, &launches));
     rc = enqueue_decode(ctx, layer_begin, n_layers, inv_tau, out, B, st, sp.qwords, at<float>(ctx, ctx->plan.partial),
-                        at<int32_t>(ctx, ctx->plan.arrive), ctx->plan.partial_bytes, true, &launches, Tq);
+                        ctx->plan.partial_bytes, true, &launches, Tq);
     ctx->launches += launches;
     return rc;
 }
@@ -456,7 +452,7 @@ int h1b_decode_step_layers(h1b_ctx *ctx, int layer_begin, int n_layers, const vo
     H1B_CUDA(ctx, launch_prepare(&ap, &sp, nn, st, &launches));
     commit_lengths(ctx, layer_begin, n_layers, B, nn);
     rc = enqueue_decode(ctx, layer_begin, n_layers, inv_tau, out, B, st, sp.qwords, at<float>(ctx, ctx->plan.partial),
-                        at<int32_t>(ctx, ctx->plan.arrive), ctx->plan.partial_bytes, true, &launches);
+                        ctx->plan.partial_bytes, true, &launches);
     ctx->launches += launches;
     return rc;
 }
@@ -478,9 +474,9 @@ int h1b_sync_lengths(h1b_ctx *ctx, void *stream) {
 
 // ---------------------------------------------------------------------------
 // Decode attention without touching the workspace's scratch region and without
-// allocating anything: the query sketches, the split-K partials and the arrival
-// counters live in a fixed array that is part of the library image. Every device
-// that loads the library carries these bytes until the process exits.
+// allocating anything: the query sketches and the split-K partials live in a
+// fixed array that is part of the library image. Every device that loads the
+// library carries these bytes until the process exits.
 // ---------------------------------------------------------------------------
 #define H1B_STATIC_SCRATCH_BYTES (8u << 20)
 static __device__ __align__(256) unsigned char h1b_static_scratch[H1B_STATIC_SCRATCH_BYTES];
@@ -512,31 +508,25 @@ int h1b_decode_attention_static(h1b_ctx *ctx, int layer_begin, int n_layers, con
     }
     unsigned char *scratch = static_cast<unsigned char *>(g_static_scratch_addr[dev]);
 
-    // carve: arrival counters (one per slab of the call), query sketches for every (layer, sequence, head)
-    // slot the kernels index, then the partials
+    // carve: query sketches for every (layer, sequence, head) slot the kernels index, then the partials
     const long slabs = (long)n_layers * B * ctx->cfg.n_kv_heads;
-    const size_t arrive_bytes = align_up((size_t)slabs * sizeof(int32_t), 256);
     const size_t qw_bytes = align_up((size_t)ctx->cfg.n_layers * ctx->cfg.max_batch * ctx->cfg.n_q_heads *
                                          ctx->plan.m_words * sizeof(uint32_t), 256);
     const size_t item_bytes = (size_t)ctx->plan.gq * kPartStride * sizeof(float);
-    const size_t need = arrive_bytes + qw_bytes + (size_t)slabs * item_bytes;
+    const size_t need = qw_bytes + (size_t)slabs * item_bytes;
     if (need > H1B_STATIC_SCRATCH_BYTES)
         return fail(ctx, H1B_ERR_CAPACITY,
                     "static scratch too small: this call needs at least %zu bytes, the built-in array holds %u",
                     need, (unsigned)H1B_STATIC_SCRATCH_BYTES);
-    const size_t fit_bytes = H1B_STATIC_SCRATCH_BYTES - arrive_bytes - qw_bytes;
+    const size_t fit_bytes = H1B_STATIC_SCRATCH_BYTES - qw_bytes;
     cudaStream_t st = static_cast<cudaStream_t>(stream);
-    // the counters must start at zero whatever an earlier call (or an aborted one) left behind
-    H1B_CUDA(ctx, cudaMemsetAsync(scratch, 0, arrive_bytes, st));
     int launches = 0;
-    const SketchParams sp = sketch_params(ctx, layer_begin, n_layers, q, B,
-                                          reinterpret_cast<uint32_t *>(scratch + arrive_bytes));
+    const SketchParams sp = sketch_params(ctx, layer_begin, n_layers, q, B, reinterpret_cast<uint32_t *>(scratch));
     NewCounts none;
     std::memset(&none, 0, sizeof none);
     H1B_CUDA(ctx, launch_prepare(nullptr, &sp, none, st, &launches));
     rc = enqueue_decode(ctx, layer_begin, n_layers, inv_tau, out, B, st, sp.qwords,
-                        reinterpret_cast<float *>(scratch + arrive_bytes + qw_bytes),
-                        reinterpret_cast<int32_t *>(scratch), fit_bytes, false, &launches);
+                        reinterpret_cast<float *>(scratch + qw_bytes), fit_bytes, false, &launches);
     ctx->launches += launches;
     return rc;
 }

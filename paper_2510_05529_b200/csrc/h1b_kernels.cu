@@ -888,6 +888,17 @@ __device__ __forceinline__ void decode_chunk(DecodeState<MW, GQ, NG> &st, const 
     __syncwarp();
 }
 
+// n_chunks chunks dealt out evenly over n_splits splits: every split gets `q`, the first `r` of them one more.
+struct SplitShare { int q, r; };
+__device__ __forceinline__ SplitShare split_share(int n_chunks, int n_splits) {
+    SplitShare s;
+    s.q = n_chunks / n_splits;
+    s.r = n_chunks - s.q * n_splits;
+    return s;
+}
+__device__ __forceinline__ int split_first_chunk(int s, const SplitShare &sh) { return s * sh.q + min(s, sh.r); }
+__device__ __forceinline__ bool split_is_empty(int s, const SplitShare &sh) { return sh.q == 0 && s >= sh.r; }
+
 template <int MW, int GQ, int NG>
 __global__ void __launch_bounds__(kDecodeWarps * 32, decode_min_blocks(GQ, NG)) decode_split_kernel(DecodeParams p) {
     using SM = DecodeSmem<MW, GQ, NG>;
@@ -909,19 +920,14 @@ __global__ void __launch_bounds__(kDecodeWarps * 32, decode_min_blocks(GQ, NG)) 
     launch_dependents();                                        // the combine grid may be scheduled behind this one
     grid_dependency_wait();                                     // lengths, query sketches and the new token come from the prepare kernel
     const int len = p.len[layer * p.max_batch + b];
-    const int t_begin = split * p.split_tokens;
-    if (t_begin >= len) {                                       // empty item: it is not counted by the combine
-#ifdef H1B_FUSED_COMBINE
-        if (len == 0 && split == 0)                             // an empty sequence attends to nothing: zeros
-            for (int i = lane; i < GQ * kHeadDim; i += 32)
-                p.out[(((size_t)ll * p.B + b) * p.Hq + kvh * GQ) * kHeadDim + i] = 0.f;
-#endif
-        return;
-    }
-    // the last split of a sequence is open-ended: it runs to the sequence's end
-    const int t_end = (split == p.splits - 1) ? len : min(len, t_begin + p.split_tokens);
+    // The sequence's chunks are dealt out evenly: split s takes chunks [s C / S, (s + 1) C / S) of the C the
+    // sequence has now (whatever the host believed when it chose S), so the items of a sequence differ by one chunk at most.
+    const SplitShare share = split_share((len + 31) >> 5, p.splits);
+    const int c0 = split_first_chunk(split, share), c1 = split_first_chunk(split + 1, share);
+    if (c0 >= c1) return;                                       // empty item: the combine skips it too
+    const int t_end = min(len, c1 * 32);
     // chunks below c_full are attended in full by every head (the earliest query token sees len - Tq + 1 tokens)
-    const int c0 = t_begin >> 5, c_full = min(t_end, len - p.Tq + 1) >> 5, c1 = (t_end + 31) >> 5;
+    const int c_full = min(t_end, len - p.Tq + 1) >> 5;
 
     unsigned char *ring = smem_raw + warp * SM::kPerWarp;
     float *p_s = reinterpret_cast<float *>(ring + kStages * CB);
@@ -1006,8 +1012,7 @@ __global__ void __launch_bounds__(kDecodeWarps * 32, decode_min_blocks(GQ, NG)) 
     }
 
     // ---------------- reduce across lanes and write the partial
-    // (after a timed-out wait the partial is meaningless, but the item still reports in below, so that
-    // the arrival counters return to zero; the status word tells the host that the output is invalid)
+    // (after a timed-out wait the partial is meaningless; the status word tells the host that the output is invalid)
 #pragma unroll
     for (int h = 0; h < GQ; ++h) {
 #pragma unroll
@@ -1081,40 +1086,6 @@ __global__ void __launch_bounds__(kDecodeWarps * 32, decode_min_blocks(GQ, NG)) 
         part_out[lane * kPartStride + 129] = sv;
     }
 
-#ifdef H1B_FUSED_COMBINE
-    // ---------------- the split that reports in last merges the slab's partials (flash-decoding combine)
-    // Build option: saves the combine launch, but the fences and the serial merge cost the attention
-    // kernel more than that launch on B200 (measured), so the default is the separate kernel below.
-    const int ns = min(p.splits, (len + p.split_tokens - 1) / p.split_tokens);   // non-empty splits of this slab
-    __threadfence();                                            // this lane's partial is visible device-wide
-    __syncwarp();
-    int prev = 0;
-    if (lane == 0) prev = atomicAdd(p.arrive + slab_local, 1);
-    prev = __shfl_sync(0xffffffffu, prev, 0);
-    if (prev != ns - 1) return;
-    __threadfence();
-    if (lane == 0) p.arrive[slab_local] = 0;                    // ready for the next launch
-    const float *base = p.partial + (size_t)slab_local * p.splits * GQ * kPartStride;
-#pragma unroll 1
-    for (int h = 0; h < GQ; ++h) {
-        const float *bh = base + (size_t)h * kPartStride;
-        float hm = 3.0e38f;
-        for (int j = 0; j < ns; ++j) hm = fminf(hm, __ldcg(bh + (size_t)j * GQ * kPartStride + 128));
-        float4 num = make_float4(0.f, 0.f, 0.f, 0.f);
-        float den = 0.f;
-        for (int j = 0; j < ns; ++j) {
-            const float *pj = bh + (size_t)j * GQ * kPartStride;
-            const float w = exp2f((hm - __ldcg(pj + 128)) * p.c2);
-            const float4 a = __ldcg(reinterpret_cast<const float4 *>(pj) + lane);
-            num.x = fmaf(w, a.x, num.x); num.y = fmaf(w, a.y, num.y);
-            num.z = fmaf(w, a.z, num.z); num.w = fmaf(w, a.w, num.w);
-            den = fmaf(w, __ldcg(pj + 129), den);
-        }
-        const float inv = 1.f / den;
-        float4 o = make_float4(num.x * inv, num.y * inv, num.z * inv, num.w * inv);
-        reinterpret_cast<float4 *>(p.out + (((size_t)ll * p.B + b) * p.Hq + kvh * GQ + h) * kHeadDim)[lane] = o;
-    }
-#endif
 }
 
 // Flash-decoding combine: one block per (layer, sequence, query head) merges the partials of the sequence's
@@ -1136,12 +1107,14 @@ __global__ void __launch_bounds__(kHeadDim) combine_kernel(DecodeParams p) {
     const int kvh = hq / gq;
     const int v = tq * gq + hq % gq, vg = v / p.gqk, hh = v % p.gqk;          // virtual head, its group and slot
     const long slab_local = ((long)ll * p.B + b) * p.Hkv + kvh;
-    const int ns = min(p.splits, (len + p.split_tokens - 1) / p.split_tokens);
+    const int n_chunks = (len + 31) >> 5, ns = p.splits;       // splits that got no chunk wrote nothing: skipped below
+    const SplitShare share = split_share(n_chunks, ns);
     const float *base = p.partial + (((size_t)slab_local * p.vgroups + vg) * p.splits * p.gqk + hh) * kPartStride;
     const size_t stride = (size_t)p.gqk * kPartStride;
     // the smallest Hamming distance any split saw (= the largest logit)
     float hm = 3.0e38f;
-    for (int j = tid; j < ns; j += kHeadDim) hm = fminf(hm, base[j * stride + 128]);
+    for (int j = tid; j < ns; j += kHeadDim)
+        if (!split_is_empty(j, share)) hm = fminf(hm, base[j * stride + 128]);
 #pragma unroll
     for (int o = 16; o > 0; o >>= 1) hm = fminf(hm, __shfl_xor_sync(0xffffffffu, hm, o));
     if (lane == 0) s_min[warp] = hm;
@@ -1151,6 +1124,7 @@ __global__ void __launch_bounds__(kHeadDim) combine_kernel(DecodeParams p) {
     float den = 0.f;
 #pragma unroll 4
     for (int j = warp; j < ns; j += 4) {
+        if (split_is_empty(j, share)) continue;
         const float *pj = base + j * stride;
         const float wgt = exp2f((hm - pj[128]) * p.c2);
         const float4 a = reinterpret_cast<const float4 *>(pj)[lane];
@@ -1163,7 +1137,7 @@ __global__ void __launch_bounds__(kHeadDim) combine_kernel(DecodeParams p) {
     __syncthreads();
     const float n4 = (s_num[0][tid] + s_num[1][tid]) + (s_num[2][tid] + s_num[3][tid]);
     const float d4 = (s_den[0] + s_den[1]) + (s_den[2] + s_den[3]);
-    p.out[(size_t)blockIdx.x * kHeadDim + tid] = (ns > 0) ? n4 / d4 : 0.f;
+    p.out[(size_t)blockIdx.x * kHeadDim + tid] = (n_chunks > 0) ? n4 / d4 : 0.f;
 }
 
 // Test helper: score of every cached token of one slab against one sketch.
@@ -1335,9 +1309,6 @@ cudaError_t launch_decode(const DecodeParams &p, cudaStream_t st, int *launches,
                           cudaEvent_t after) {
     const int gq = p.gqk;                                       // (virtual) heads per work item
     cudaError_t e = cudaErrorInvalidValue;
-#ifdef H1B_FUSED_COMBINE
-    if (p.Tq != 1) return cudaErrorNotSupported;                // the fused merge only knows one query token
-#endif
     if (before) cudaEventRecord(before, st);
     H1B_DISPATCH_MW(p.m_words,
         if (p.groups == 4) {
@@ -1357,7 +1328,6 @@ cudaError_t launch_decode(const DecodeParams &p, cudaStream_t st, int *launches,
     if (e != cudaSuccess) return e;
     if (after) cudaEventRecord(after, st);
     ++*launches;
-#ifndef H1B_FUSED_COMBINE
     {
         cudaLaunchConfig_t cfg = {};
         cfg.gridDim = dim3(p.n_layers * p.B * p.Tq * p.Hq);
@@ -1372,7 +1342,6 @@ cudaError_t launch_decode(const DecodeParams &p, cudaStream_t st, int *launches,
         if (ec != cudaSuccess) return ec;
     }
     ++*launches;
-#endif
     return cudaGetLastError();
 }
 

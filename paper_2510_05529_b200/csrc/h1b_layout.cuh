@@ -141,10 +141,9 @@ struct DecodeParams {
     float *partial;             // [items][gqk][kPartStride]
     float *out;                 // fp32 [n_layers][B][Tq][Hq][d]
     int32_t *status;
-    int32_t *arrive;            // [slabs of the call]: splits that have reported in (zero between launches)
     size_t slab_bytes;
     int layer_begin, n_layers, B, Hkv, Hq, max_batch, m_words, groups;
-    int splits, split_tokens;   // split_tokens is a multiple of 32
+    int splits;                 // work items per (slab, group of virtual heads): each takes an even share of the chunks
     // Several query tokens per sequence (Tq > 1): they are the sequence's last Tq cached tokens, query token i attends to
     // tokens [0, len - Tq + i + 1). The Tq * (Hq/Hkv) (query token, query head) pairs that share a KV head are "virtual
     // heads" v = i * (Hq/Hkv) + head-in-group, handled `gqk` at a time by one work item (vgroups items per slab and split).
