@@ -25,7 +25,7 @@ constexpr int kMaxQueryTokens = H1B_MAX_QUERY_TOKENS;
 constexpr int kPrefillMinTokens = 64;   // appends of at least this many tokens per sequence take the tensor-core path
 
 struct Plan {
-    size_t rt, rh, len, status, qwords, partial, stage_k, stage_v, stage_q, stage_out, dbg_q, dbg_s, cache, total;
+    size_t rt, rh, len, status, qwords, partial, stage_k, stage_v, stage_q, stage_out, dbg_q, dbg_row, dbg_s, cache, total;
     size_t partial_bytes, slab_bytes;
     int cap_tokens, m_words, gq, groups;
 };
@@ -43,16 +43,37 @@ int check_config(const h1b_config *c) {
     if (c->max_batch > 256) return H1B_ERR_INVALID_ARG;
     const int gq = c->n_q_heads / c->n_kv_heads;
     if (gq != 1 && gq != 2 && gq != 4) return H1B_ERR_UNSUPPORTED;
-    if (c->head_dim != kHeadDim || (c->group_size != kGroup && c->group_size != kHeadDim)) return H1B_ERR_UNSUPPORTED;
     if (c->sketch_bits != 64 && c->sketch_bits != 128 && c->sketch_bits != 256 && c->sketch_bits != 512)
         return H1B_ERR_UNSUPPORTED;
+    if (c->head_dim == kHeadDim / 2) {
+        // 64-wide heads travel in pairs through the 128-wide kernels: multi-head attention with an even number of
+        // heads, groups of 32 channels (or fp16 values), and both sketches of a pair within 512 bits
+        if (gq != 1 || (c->n_kv_heads & 1) || c->group_size != kGroup || c->sketch_bits > 256) return H1B_ERR_UNSUPPORTED;
+    } else if (c->head_dim != kHeadDim || (c->group_size != kGroup && c->group_size != kHeadDim)) {
+        return H1B_ERR_UNSUPPORTED;
+    }
     if ((long)c->n_layers * c->max_batch * c->n_kv_heads > (1L << 28)) return H1B_ERR_INVALID_ARG;
     return H1B_OK;
 }
 
-int make_plan(const h1b_config *c, Plan *p) {
-    const int rc = check_config(c);
+// The configuration the kernels see. Head dimension 128: the caller's. Head dimension 64: heads 2s and 2s+1 form
+// slab s of 128 channels, so there are half as many slabs as heads (which the kernels call KV heads), the sketch
+// words of both heads sit side by side (twice the bits), and the projection is the block-diagonal [[R, 0], [0, R]].
+bool is_paired(const h1b_config *c) { return c->head_dim == kHeadDim / 2; }
+h1b_config internal_config(const h1b_config *c) {
+    h1b_config ic = *c;
+    if (is_paired(c)) {
+        ic.head_dim = kHeadDim;
+        ic.n_kv_heads = c->n_kv_heads / 2;
+        ic.sketch_bits = 2 * c->sketch_bits;
+    }
+    return ic;
+}
+
+int make_plan(const h1b_config *user, Plan *p) {
+    const int rc = check_config(user);
     if (rc != H1B_OK) return rc;
+    const h1b_config ic = internal_config(user), *c = &ic;
     p->m_words = c->sketch_bits / 32;
     p->gq = c->n_q_heads / c->n_kv_heads;
     p->groups = (c->flags & H1B_FLAG_FP16_VALUES) ? 0 : c->head_dim / c->group_size;   // 0: values stay fp16
@@ -77,6 +98,7 @@ int make_plan(const h1b_config *c, Plan *p) {
     p->stage_q = take(L * B * Hq * d * 2);
     p->stage_out = take(L * B * Hq * d * 4);
     p->dbg_q = take(p->m_words * sizeof(uint32_t));
+    p->dbg_row = take(kHeadDim * 2);
     p->dbg_s = take((size_t)p->cap_tokens * sizeof(int32_t));
     p->cache = take(slabs * p->slab_bytes);
     p->total = o;
@@ -106,7 +128,9 @@ void fill_gaussian(float *dst, size_t n, uint64_t seed) {
 }  // namespace
 
 struct h1b_ctx {
-    h1b_config cfg;
+    h1b_config cfg;                    // what the kernels see (see internal_config)
+    h1b_config ucfg;                   // what the caller asked for
+    bool paired;                       // head dimension 64: two heads per slab
     Plan plan;
     ChunkLayout cl;
     unsigned char *ws;
@@ -188,7 +212,9 @@ int h1b_init_projection(const h1b_config *cfg, uint64_t seed, const float *Rt_ho
                     plan.total, workspace_bytes, workspace);
     h1b_ctx *ctx = new (std::nothrow) h1b_ctx();
     if (!ctx) return fail(nullptr, H1B_ERR_INVALID_ARG, "out of host memory");
-    ctx->cfg = *cfg;
+    ctx->ucfg = *cfg;
+    ctx->cfg = internal_config(cfg);
+    ctx->paired = is_paired(cfg);
     ctx->plan = plan;
     ctx->cl = chunk_layout(plan.m_words, plan.groups);
     ctx->ws = static_cast<unsigned char *>(workspace);
@@ -211,15 +237,29 @@ int h1b_init_projection(const h1b_config *cfg, uint64_t seed, const float *Rt_ho
     e = cudaMemsetAsync(workspace, 0, plan.total, st);
     if (e != cudaSuccess) return bail(e, "cudaMemsetAsync");
     const size_t nR = (size_t)cfg->n_layers * cfg->head_dim * cfg->sketch_bits;
-    std::vector<float> gen;
+    std::vector<float> gen, wide;
     if (!Rt_host) {
         gen.resize(nR);
         fill_gaussian(gen.data(), nR, seed);
         Rt_host = gen.data();
     }
-    e = cudaMemcpyAsync(ctx->ws + plan.rt, Rt_host, nR * sizeof(float), cudaMemcpyHostToDevice, st);
+    size_t nR_dev = nR;
+    if (ctx->paired) {                          // [[R, 0], [0, R]] per layer: [128][2m]
+        const size_t d = cfg->head_dim, m = cfg->sketch_bits;
+        nR_dev = (size_t)cfg->n_layers * 2 * d * 2 * m;
+        wide.assign(nR_dev, 0.f);
+        for (size_t l = 0; l < (size_t)cfg->n_layers; ++l)
+            for (size_t i = 0; i < d; ++i)
+                for (size_t j = 0; j < m; ++j) {
+                    const float r = Rt_host[(l * d + i) * m + j];
+                    wide[(l * 2 * d + i) * 2 * m + j] = r;
+                    wide[(l * 2 * d + d + i) * 2 * m + m + j] = r;
+                }
+        Rt_host = wide.data();
+    }
+    e = cudaMemcpyAsync(ctx->ws + plan.rt, Rt_host, nR_dev * sizeof(float), cudaMemcpyHostToDevice, st);
     if (e != cudaSuccess) return bail(e, "cudaMemcpyAsync(Rt)");
-    e = launch_split_projection(at<float>(ctx, plan.rt), at<uint16_t>(ctx, plan.rh), cfg->n_layers, cfg->sketch_bits, st);
+    e = launch_split_projection(at<float>(ctx, plan.rt), at<uint16_t>(ctx, plan.rh), cfg->n_layers, ctx->cfg.sketch_bits, st);
     if (e != cudaSuccess) return bail(e, "split_projection_kernel");
     e = cudaStreamSynchronize(st);
     if (e != cudaSuccess) return bail(e, "cudaStreamSynchronize");
@@ -280,7 +320,9 @@ static SketchParams sketch_params(h1b_ctx *ctx, int layer_begin, int n_layers, c
     sp.q = static_cast<const uint16_t *>(q);
     sp.Rt = at<float>(ctx, ctx->plan.rt);
     sp.qwords = qwords;
-    sp.layer_begin = layer_begin; sp.n_layers = n_layers; sp.B = B; sp.Hq = ctx->cfg.n_q_heads;
+    // (paired heads: a row of the sketch is a pair of query heads, 128 channels, and yields both heads' words)
+    sp.layer_begin = layer_begin; sp.n_layers = n_layers; sp.B = B;
+    sp.Hq = ctx->paired ? ctx->cfg.n_q_heads / 2 : ctx->cfg.n_q_heads;
     sp.max_batch = ctx->cfg.max_batch; sp.m_words = ctx->plan.m_words;
     return sp;
 }
@@ -328,7 +370,9 @@ static int enqueue_decode(h1b_ctx *ctx, int layer_begin, int n_layers, float inv
     dp.groups = ctx->plan.groups;
     dp.splits = (int)splits;
     dp.Tq = Tq; dp.gqk = gqk; dp.vgroups = vgroups;
-    dp.c2 = (float)(2.0 * (double)inv_tau * 1.4426950408889634 / (double)ctx->cfg.sketch_bits);
+    dp.paired = ctx->paired ? 1 : 0;
+    dp.out_dim = ctx->ucfg.head_dim;
+    dp.c2 = (float)(2.0 * (double)inv_tau * 1.4426950408889634 / (double)ctx->ucfg.sketch_bits);
     cudaEvent_t ev0 = nullptr, ev1 = nullptr;
     if (may_profile && ctx->profiling && ctx->events_used + 2 <= ctx->events.size()) {
         ev0 = ctx->events[ctx->events_used];
@@ -418,6 +462,8 @@ int h1b_decode_attention_multi(h1b_ctx *ctx, int layer_begin, int n_layers, cons
     if (rc != H1B_OK) return rc;
     if (Tq < 1 || Tq > kMaxQueryTokens)
         return fail(ctx, H1B_ERR_INVALID_ARG, "Tq = %d outside [1, %d]", Tq, kMaxQueryTokens);
+    if (ctx->paired && Tq > 1)
+        return fail(ctx, H1B_ERR_UNSUPPORTED, "several query tokens are not built for head dimension 64");
     for (int l = layer_begin; l < layer_begin + n_layers; ++l)
         for (int b = 0; b < B; ++b)
             if (ctx->len_host[(size_t)l * ctx->cfg.max_batch + b] < Tq)
@@ -538,8 +584,8 @@ int h1b_decode_step_host(h1b_ctx *ctx, const void *k_host, const void *v_host, c
     int rc = check_layers(ctx, 0, ctx->cfg.n_layers, B);
     if (rc != H1B_OK) return rc;
     cudaStream_t st = static_cast<cudaStream_t>(stream);
-    const size_t L = ctx->cfg.n_layers, d = ctx->cfg.head_dim;
-    const size_t kv_bytes = L * B * ctx->cfg.n_kv_heads * d * 2, q_bytes = L * B * ctx->cfg.n_q_heads * d * 2;
+    const size_t L = ctx->ucfg.n_layers, d = ctx->ucfg.head_dim;
+    const size_t kv_bytes = L * B * ctx->ucfg.n_kv_heads * d * 2, q_bytes = L * B * ctx->ucfg.n_q_heads * d * 2;
     const unsigned char *kh = static_cast<const unsigned char *>(k_host);
     bool one_copy = false;
     if (static_cast<const unsigned char *>(v_host) == kh + kv_bytes &&
@@ -583,8 +629,17 @@ int h1b_get_projection(h1b_ctx *ctx, int layer, float *Rt_host) {
     if (layer < 0 || layer >= ctx->cfg.n_layers) return fail(ctx, H1B_ERR_INVALID_ARG, "layer %d out of range", layer);
     const size_t n = (size_t)ctx->cfg.head_dim * ctx->cfg.sketch_bits;
     H1B_CUDA(ctx, cudaDeviceSynchronize());
-    H1B_CUDA(ctx, cudaMemcpy(Rt_host, at<float>(ctx, ctx->plan.rt) + (size_t)layer * n, n * sizeof(float),
+    if (!ctx->paired) {
+        H1B_CUDA(ctx, cudaMemcpy(Rt_host, at<float>(ctx, ctx->plan.rt) + (size_t)layer * n, n * sizeof(float),
+                                 cudaMemcpyDeviceToHost));
+        return H1B_OK;
+    }
+    // the caller's [64][m] is the upper left block of the block-diagonal [128][2m] the device holds
+    std::vector<float> wide(n);
+    H1B_CUDA(ctx, cudaMemcpy(wide.data(), at<float>(ctx, ctx->plan.rt) + (size_t)layer * n, n * sizeof(float),
                              cudaMemcpyDeviceToHost));
+    const size_t d = ctx->ucfg.head_dim, m = ctx->ucfg.sketch_bits;
+    for (size_t i = 0; i < d; ++i) std::memcpy(Rt_host + i * m, wide.data() + i * 2 * m, m * sizeof(float));
     return H1B_OK;
 }
 
@@ -628,7 +683,7 @@ int h1b_export_cache(h1b_ctx *ctx, int layer, int seq, int kv_head, int t0, int 
                      uint16_t *scale, uint16_t *zero) {
     if (!ctx) return H1B_ERR_NULL;
     if (layer < 0 || layer >= ctx->cfg.n_layers || seq < 0 || seq >= ctx->cfg.max_batch || kv_head < 0 ||
-        kv_head >= ctx->cfg.n_kv_heads)
+        kv_head >= ctx->ucfg.n_kv_heads)
         return fail(ctx, H1B_ERR_INVALID_ARG, "(layer %d, seq %d, kv_head %d) out of range", layer, seq, kv_head);
     const int len = ctx->len_host[(size_t)layer * ctx->cfg.max_batch + seq];
     if (t0 < 0 || n < 0 || t0 + n > len)
@@ -639,25 +694,29 @@ int h1b_export_cache(h1b_ctx *ctx, int layer, int seq, int kv_head, int t0, int 
     const ChunkLayout &cl = ctx->cl;
     const int c_lo = t0 / kChunkTokens, c_hi = (t0 + n - 1) / kChunkTokens;
     std::vector<unsigned char> raw((size_t)(c_hi - c_lo + 1) * cl.bytes);
+    // with paired heads, head kv_head is half `half` of slab kv_head / 2: its share of the words, channel blocks and groups
+    const int slab = ctx->paired ? kv_head / 2 : kv_head, half = ctx->paired ? (kv_head & 1) : 0;
     H1B_CUDA(ctx, cudaDeviceSynchronize());
-    H1B_CUDA(ctx, cudaMemcpy(raw.data(), slab_ptr(ctx, layer, seq, kv_head) + (size_t)c_lo * cl.bytes, raw.size(),
+    H1B_CUDA(ctx, cudaMemcpy(raw.data(), slab_ptr(ctx, layer, seq, slab) + (size_t)c_lo * cl.bytes, raw.size(),
                              cudaMemcpyDeviceToHost));
-    const int mw = cl.m_words, d = ctx->cfg.head_dim;
+    const int d = ctx->ucfg.head_dim, mw = ctx->ucfg.sketch_bits / 32;
+    const int ng = ctx->paired ? cl.groups / 2 : cl.groups;
+    const int w0 = half * mw, cb0 = half * (d / 16), g0 = half * ng;
     for (int i = 0; i < n; ++i) {
         const int t = t0 + i, tt = t % kChunkTokens;
         const unsigned char *ch = raw.data() + (size_t)(t / kChunkTokens - c_lo) * cl.bytes;
         if (words)
-            for (int w = 0; w < mw; ++w) std::memcpy(&words[(size_t)i * mw + w], ch + key_word_off(w, tt), 4);
+            for (int w = 0; w < mw; ++w) std::memcpy(&words[(size_t)i * mw + w], ch + key_word_off(w0 + w, tt), 4);
         if (codes)
             for (int cb = 0; cb < d / 16; ++cb)
                 for (int r = 0; r < 8; ++r) {
-                    const unsigned char byte = ch[code_byte_off(cl, tt, cb, r)];
+                    const unsigned char byte = ch[code_byte_off(cl, tt, cb0 + cb, r)];
                     codes[(size_t)i * d + cb * 16 + r] = byte & 15;
                     codes[(size_t)i * d + cb * 16 + r + 8] = byte >> 4;
                 }
-        for (int g = 0; g < cl.groups; ++g) {
-            if (scale) std::memcpy(&scale[(size_t)i * cl.groups + g], ch + scale_off(cl, tt, g), 2);
-            if (zero) std::memcpy(&zero[(size_t)i * cl.groups + g], ch + zero_off(cl, tt, g), 2);
+        for (int g = 0; g < ng; ++g) {
+            if (scale) std::memcpy(&scale[(size_t)i * ng + g], ch + scale_off(cl, tt, g0 + g), 2);
+            if (zero) std::memcpy(&zero[(size_t)i * ng + g], ch + zero_off(cl, tt, g0 + g), 2);
         }
     }
     return H1B_OK;
@@ -668,7 +727,7 @@ int h1b_export_values(h1b_ctx *ctx, int layer, int seq, int kv_head, int t0, int
     if (ctx->plan.groups != 0) return fail(ctx, H1B_ERR_INVALID_ARG, "this cache keeps 4-bit codes, not fp16 values");
     if (!values) return fail(ctx, H1B_ERR_NULL, "values is NULL");
     if (layer < 0 || layer >= ctx->cfg.n_layers || seq < 0 || seq >= ctx->cfg.max_batch || kv_head < 0 ||
-        kv_head >= ctx->cfg.n_kv_heads)
+        kv_head >= ctx->ucfg.n_kv_heads)
         return fail(ctx, H1B_ERR_INVALID_ARG, "(layer %d, seq %d, kv_head %d) out of range", layer, seq, kv_head);
     const int len = ctx->len_host[(size_t)layer * ctx->cfg.max_batch + seq];
     if (t0 < 0 || n < 0 || t0 + n > len)
@@ -677,14 +736,15 @@ int h1b_export_values(h1b_ctx *ctx, int layer, int seq, int kv_head, int t0, int
     const ChunkLayout &cl = ctx->cl;
     const int c_lo = t0 / kChunkTokens, c_hi = (t0 + n - 1) / kChunkTokens;
     std::vector<unsigned char> raw((size_t)(c_hi - c_lo + 1) * cl.bytes);
+    const int slab = ctx->paired ? kv_head / 2 : kv_head, half = ctx->paired ? (kv_head & 1) : 0;
     H1B_CUDA(ctx, cudaDeviceSynchronize());
-    H1B_CUDA(ctx, cudaMemcpy(raw.data(), slab_ptr(ctx, layer, seq, kv_head) + (size_t)c_lo * cl.bytes, raw.size(),
+    H1B_CUDA(ctx, cudaMemcpy(raw.data(), slab_ptr(ctx, layer, seq, slab) + (size_t)c_lo * cl.bytes, raw.size(),
                              cudaMemcpyDeviceToHost));
-    const int d = ctx->cfg.head_dim;
+    const int d = ctx->ucfg.head_dim;
     for (int i = 0; i < n; ++i) {
         const int t = t0 + i, tt = t % kChunkTokens;
         const unsigned char *ch = raw.data() + (size_t)(t / kChunkTokens - c_lo) * cl.bytes;
-        for (int c = 0; c < d; ++c) std::memcpy(&values[(size_t)i * d + c], ch + value_half_off(cl, tt, c), 2);
+        for (int c = 0; c < d; ++c) std::memcpy(&values[(size_t)i * d + c], ch + value_half_off(cl, tt, half * d + c), 2);
     }
     return H1B_OK;
 }
@@ -694,10 +754,19 @@ int h1b_debug_scores(h1b_ctx *ctx, int layer, int seq, int kv_head, const void *
     if (!ctx) return H1B_ERR_NULL;
     if (!q) return fail(ctx, H1B_ERR_NULL, "q is NULL");
     if (layer < 0 || layer >= ctx->cfg.n_layers || seq < 0 || seq >= ctx->cfg.max_batch || kv_head < 0 ||
-        kv_head >= ctx->cfg.n_kv_heads)
+        kv_head >= ctx->ucfg.n_kv_heads)
         return fail(ctx, H1B_ERR_INVALID_ARG, "(layer %d, seq %d, kv_head %d) out of range", layer, seq, kv_head);
     const int len = ctx->len_host[(size_t)layer * ctx->cfg.max_batch + seq];
-    const int mw = ctx->plan.m_words;
+    const int mw = ctx->plan.m_words, mwh = ctx->ucfg.sketch_bits / 32;
+    const int slab = ctx->paired ? kv_head / 2 : kv_head, half = ctx->paired ? (kv_head & 1) : 0;
+    H1B_CUDA(ctx, cudaDeviceSynchronize());
+    if (ctx->paired) {
+        // a 128-channel row with the 64-channel query in front and zeros behind: the upper left block of the
+        // block-diagonal projection then gives the query's sketch in the first m/32 words
+        H1B_CUDA(ctx, cudaMemset(ctx->ws + ctx->plan.dbg_row, 0, kHeadDim * 2));
+        H1B_CUDA(ctx, cudaMemcpy(ctx->ws + ctx->plan.dbg_row, q, (size_t)ctx->ucfg.head_dim * 2, cudaMemcpyDeviceToDevice));
+        q = ctx->ws + ctx->plan.dbg_row;
+    }
     // sketch the single query row with the layer's projection into the debug slot
     SketchParams sp;
     sp.q = static_cast<const uint16_t *>(q);
@@ -707,13 +776,12 @@ int h1b_debug_scores(h1b_ctx *ctx, int layer, int seq, int kv_head, const void *
     int launches = 0;
     NewCounts none;
     std::memset(&none, 0, sizeof none);
-    H1B_CUDA(ctx, cudaDeviceSynchronize());
     H1B_CUDA(ctx, launch_prepare(nullptr, &sp, none, nullptr, &launches));
-    H1B_CUDA(ctx, launch_debug_scores(slab_ptr(ctx, layer, seq, kv_head), sp.qwords, mw, ctx->plan.groups, len,
+    H1B_CUDA(ctx, launch_debug_scores(slab_ptr(ctx, layer, seq, slab), sp.qwords, mw, ctx->plan.groups, len, half * mwh, mwh,
                                       at<int32_t>(ctx, ctx->plan.dbg_s), nullptr));
     H1B_CUDA(ctx, cudaDeviceSynchronize());
     if (qwords_host)
-        H1B_CUDA(ctx, cudaMemcpy(qwords_host, sp.qwords, mw * sizeof(uint32_t), cudaMemcpyDeviceToHost));
+        H1B_CUDA(ctx, cudaMemcpy(qwords_host, sp.qwords, mwh * sizeof(uint32_t), cudaMemcpyDeviceToHost));
     if (score_host && len > 0)
         H1B_CUDA(ctx, cudaMemcpy(score_host, at<int32_t>(ctx, ctx->plan.dbg_s), (size_t)len * sizeof(int32_t),
                                  cudaMemcpyDeviceToHost));

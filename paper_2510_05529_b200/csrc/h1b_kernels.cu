@@ -730,11 +730,17 @@ struct DecodeState {
 
 // One chunk. TAIL: head h attends only to the chunk's first n_valid[h] tokens (the last chunks of a split; with
 // several query tokens, each one's causal limit).
-template <int MW, int GQ, int NG, bool TAIL>
+// PAIRED (head dimension 64): the slab holds two heads side by side, head h in channels 64h..64h+63 and in key words
+// [h MW/2, (h+1) MW/2). GQ = 2 then counts those two heads; the accumulator columns are laid out as for one head,
+// (value group, part), and group g simply takes the weights of head g / 2.
+template <int MW, int GQ, int NG, bool TAIL, bool PAIRED>
 __device__ __forceinline__ void decode_chunk(DecodeState<MW, GQ, NG> &st, const unsigned char *ch, float *p_s,
                                              int lane, const int (&n_valid)[GQ], float c2) {
-    constexpr int GPF = 4 / GQ;                // value groups covered by one B fragment (4 groups per vector)
-    constexpr int NB = (NG == 1) ? 1 : GQ;     // B fragments per 16-token block (one scale per vector: one fragment)
+    static_assert(!PAIRED || (GQ == 2 && (NG == 4 || NG == 0)), "two 64-wide heads per slab, groups of 32 or fp16 values");
+    constexpr int GQL = PAIRED ? 1 : GQ;       // heads the accumulator columns are laid out for
+    constexpr int GPF = 4 / GQL;               // value groups covered by one B fragment (4 groups per vector)
+    constexpr int NB = (NG == 1) ? 1 : GQL;    // B fragments per 16-token block (one scale per vector: one fragment)
+    constexpr int MWH = PAIRED ? MW / 2 : MW;  // key words of one head
     constexpr int VAL = MW * 128, ZERO = VAL + 2048, SCALE = ZERO + 64 * NG;
     const int jq = lane & 3;
 
@@ -757,7 +763,7 @@ __device__ __forceinline__ void decode_chunk(DecodeState<MW, GQ, NG> &st, const 
     for (int h = 0; h < GQ; ++h) {
         int ham = 0;
 #pragma unroll
-        for (int w = 0; w < MW; ++w) ham += __popc(kw[w] ^ st.qw[h][w]);
+        for (int w = 0; w < MWH; ++w) ham += __popc(kw[(PAIRED ? h * MWH : 0) + w] ^ st.qw[h][w]);
         const bool valid = !TAIL || lane < n_valid[h];
         const int cmin = __reduce_min_sync(0xffffffffu, (TAIL && !valid) ? kHamSentinel : ham);
         scl[h] = 1.f;
@@ -778,7 +784,8 @@ __device__ __forceinline__ void decode_chunk(DecodeState<MW, GQ, NG> &st, const 
     }
     // factors by which this lane's accumulator columns 2jq, 2jq+1 shrink when a running max moved (else 1)
     float f0, f1;
-    if (GQ == 1) { f0 = scl[0]; f1 = scl[0]; }
+    if (PAIRED && NG != 0) { f0 = (jq & 1) ? scl[GQ > 1 ? 1 : 0] : scl[0]; f1 = f0; }   // columns 2jq, 2jq+1: groups of head jq % 2
+    else if (GQ == 1) { f0 = scl[0]; f1 = scl[0]; }
     else if (GQ == 2) { f0 = scl[0]; f1 = scl[GQ > 1 ? 1 : 0]; }
     else { f0 = (jq & 1) ? scl[GQ > 2 ? 2 : 0] : scl[0]; f1 = (jq & 1) ? scl[GQ > 3 ? 3 : 0] : scl[GQ > 1 ? 1 : 0]; }
     __syncwarp();
@@ -834,8 +841,8 @@ __device__ __forceinline__ void decode_chunk(DecodeState<MW, GQ, NG> &st, const 
     // (group in pair, head) (GQ 2) or head (GQ 4). This lane computes the weights of ONE token pair
     // (tokens 2jq, 2jq+1 if part 0, else 2jq+8, 2jq+9), both parts, and swaps one of them with lane ^ 16.
     const int part = lane >> 4, idx = (lane >> 2) & 3;
-    const int bhead = (GQ == 1) ? 0 : (GQ == 2 ? (idx & 1) : idx);
-    const int bgsel = (GQ == 1) ? idx : (GQ == 2 ? (idx >> 1) : 0);
+    const int bhead = PAIRED ? (idx >> 1) : ((GQ == 1) ? 0 : (GQ == 2 ? (idx & 1) : idx));
+    const int bgsel = (GQL == 1) ? idx : (GQL == 2 ? (idx >> 1) : 0);
     const int tp = 2 * jq + 8 * part;                       // first token of this lane's pair within a block
     uint32_t bf[2][NB][2];
 #pragma unroll
@@ -899,9 +906,10 @@ __device__ __forceinline__ SplitShare split_share(int n_chunks, int n_splits) {
 __device__ __forceinline__ int split_first_chunk(int s, const SplitShare &sh) { return s * sh.q + min(s, sh.r); }
 __device__ __forceinline__ bool split_is_empty(int s, const SplitShare &sh) { return sh.q == 0 && s >= sh.r; }
 
-template <int MW, int GQ, int NG>
+template <int MW, int GQ, int NG, bool PAIRED>
 __global__ void __launch_bounds__(kDecodeWarps * 32, decode_min_blocks(GQ, NG)) decode_split_kernel(DecodeParams p) {
     using SM = DecodeSmem<MW, GQ, NG>;
+    constexpr int MWH = PAIRED ? MW / 2 : MW;                   // key words of one head
     constexpr int CB = SM::kChunkBytes;
     constexpr int kStages = SM::kNStages;                       // shadows the build-time default
     extern __shared__ __align__(128) unsigned char smem_raw[];
@@ -961,9 +969,9 @@ __global__ void __launch_bounds__(kDecodeWarps * 32, decode_min_blocks(GQ, NG)) 
             // a group's surplus slots repeat the last virtual head (their results are never read)
             const int v = min(vg * GQ + h, vheads - 1), tq = v / gq, hq = kvh * gq + v % gq;
             limit[h] = min(t_end, len - p.Tq + tq + 1);
-            const uint32_t *qp = p.qwords + (((size_t)(layer * p.max_batch + b) * p.Tq + tq) * p.Hq + hq) * MW;
+            const uint32_t *qp = p.qwords + (((size_t)(layer * p.max_batch + b) * p.Tq + tq) * p.Hq + hq) * MWH;
 #pragma unroll
-            for (int w = 0; w < MW; ++w) st.qw[h][w] = __ldg(qp + w);
+            for (int w = 0; w < MWH; ++w) st.qw[h][w] = __ldg(qp + w);
         }
     }
 #pragma unroll
@@ -985,12 +993,12 @@ __global__ void __launch_bounds__(kDecodeWarps * 32, decode_min_blocks(GQ, NG)) 
         if (!mbar_wait_bounded(bar0 + 8 * stage, parity, kWaitLimitNs)) { failed = true; break; }
         const unsigned char *ch = ring + stage * CB;
         if (c < c_full) {
-            decode_chunk<MW, GQ, NG, false>(st, ch, p_s, lane, limit, p.c2);
+            decode_chunk<MW, GQ, NG, false, PAIRED>(st, ch, p_s, lane, limit, p.c2);
         } else {
             int n_valid[GQ];
 #pragma unroll
             for (int h = 0; h < GQ; ++h) n_valid[h] = limit[h] - c * 32;
-            decode_chunk<MW, GQ, NG, true>(st, ch, p_s, lane, n_valid, p.c2);
+            decode_chunk<MW, GQ, NG, true, PAIRED>(st, ch, p_s, lane, n_valid, p.c2);
         }
         // every lane is done with this stage (the chunk ends with a warp barrier): refill it
         if (lane == 0 && requested < c1) {
@@ -1043,12 +1051,26 @@ __global__ void __launch_bounds__(kDecodeWarps * 32, decode_min_blocks(GQ, NG)) 
             if (jq < 2) {
 #pragma unroll
                 for (int hh = 0; hh < 2; ++hh) {
-                    if (2 * jq + hh < GQ) {
+                    if (PAIRED) {                               // head hh owns channel blocks 4hh .. 4hh+3: its channels 0..63
+                        if (jq == 0 && (cb >> 2) == hh) {
+                            float *dst = part_out + (size_t)hh * kPartStride;
+                            dst[(cb & 3) * 16 + r] = v[hh];
+                            dst[(cb & 3) * 16 + r + 8] = v[2 + hh];
+                        }
+                    } else if (2 * jq + hh < GQ) {
                         float *dst = part_out + (size_t)(2 * jq + hh) * kPartStride;
                         dst[cb * 16 + r] = v[hh];
                         dst[cb * 16 + r + 8] = v[2 + hh];
                     }
                 }
+            }
+        } else if (PAIRED) {                                    // group g belongs to head g / 2 = cb / 4
+            if (jq == (g >> 1)) {
+                const int hh = cb >> 2;
+                const float z = hh ? st.accz[GQ > 1 ? 1 : 0][gz] : st.accz[0][gz];
+                float *dst = part_out + (size_t)hh * kPartStride;
+                dst[(cb & 3) * 16 + r] = v[g & 1] + z;
+                dst[(cb & 3) * 16 + r + 8] = v[2 + (g & 1)] + z;
             }
         } else if (GQ == 1) {
             if (jq == (g >> 1)) {
@@ -1127,7 +1149,7 @@ __global__ void __launch_bounds__(kHeadDim) combine_kernel(DecodeParams p) {
         if (split_is_empty(j, share)) continue;
         const float *pj = base + j * stride;
         const float wgt = exp2f((hm - pj[128]) * p.c2);
-        const float4 a = reinterpret_cast<const float4 *>(pj)[lane];
+        const float4 a = (lane * 4 < p.out_dim) ? reinterpret_cast<const float4 *>(pj)[lane] : make_float4(0.f, 0.f, 0.f, 0.f);
         num.x = fmaf(wgt, a.x, num.x); num.y = fmaf(wgt, a.y, num.y);
         num.z = fmaf(wgt, a.z, num.z); num.w = fmaf(wgt, a.w, num.w);
         den = fmaf(wgt, pj[129], den);
@@ -1137,20 +1159,21 @@ __global__ void __launch_bounds__(kHeadDim) combine_kernel(DecodeParams p) {
     __syncthreads();
     const float n4 = (s_num[0][tid] + s_num[1][tid]) + (s_num[2][tid] + s_num[3][tid]);
     const float d4 = (s_den[0] + s_den[1]) + (s_den[2] + s_den[3]);
-    p.out[(size_t)blockIdx.x * kHeadDim + tid] = (n_chunks > 0) ? n4 / d4 : 0.f;
+    if (tid < p.out_dim) p.out[(size_t)blockIdx.x * p.out_dim + tid] = (n_chunks > 0) ? n4 / d4 : 0.f;
 }
 
 // Test helper: score of every cached token of one slab against one sketch.
+// Key words [w0, w0 + nw) of the slab (one head's sketch) against qwords[0 .. nw).
 __global__ void debug_scores_kernel(const unsigned char *slab, const uint32_t *qwords, int m_words, int groups, int len,
-                                    int32_t *score) {
+                                    int w0, int nw, int32_t *score) {
     const int t = blockIdx.x * blockDim.x + threadIdx.x;
     if (t >= len) return;
     const ChunkLayout cl = chunk_layout(m_words, groups);
     const unsigned char *chunk = slab + (size_t)(t >> 5) * cl.bytes;
     int ham = 0;
-    for (int w = 0; w < m_words; ++w)
-        ham += __popc(*reinterpret_cast<const uint32_t *>(chunk + key_word_off(w, t & 31)) ^ qwords[w]);
-    score[t] = m_words * 32 - 2 * ham;
+    for (int w = 0; w < nw; ++w)
+        ham += __popc(*reinterpret_cast<const uint32_t *>(chunk + key_word_off(w0 + w, t & 31)) ^ qwords[w]);
+    score[t] = nw * 32 - 2 * ham;
 }
 
 // ===========================================================================
@@ -1278,14 +1301,14 @@ cudaError_t launch_set_len(int32_t *len, int n_layers, int max_batch, int seq, i
     return cudaGetLastError();
 }
 
-template <int MW, int GQ, int NG>
+template <int MW, int GQ, int NG, bool PAIRED = false>
 static cudaError_t launch_decode_t(const DecodeParams &p, cudaStream_t st) {
     using SM = DecodeSmem<MW, GQ, NG>;
     static bool attr_set[64] = {};
     int dev = 0;
     cudaGetDevice(&dev);
     if (dev >= 0 && dev < 64 && !attr_set[dev]) {
-        cudaError_t e = cudaFuncSetAttribute(decode_split_kernel<MW, GQ, NG>,
+        cudaError_t e = cudaFuncSetAttribute(decode_split_kernel<MW, GQ, NG, PAIRED>,
                                              cudaFuncAttributeMaxDynamicSharedMemorySize, SM::kTotal);
         if (e != cudaSuccess) return e;
         attr_set[dev] = true;
@@ -1302,7 +1325,7 @@ static cudaError_t launch_decode_t(const DecodeParams &p, cudaStream_t st) {
     attr[0].val.programmaticStreamSerializationAllowed = 1;
     cfg.attrs = attr;
     cfg.numAttrs = 1;
-    return cudaLaunchKernelEx(&cfg, decode_split_kernel<MW, GQ, NG>, p);
+    return cudaLaunchKernelEx(&cfg, decode_split_kernel<MW, GQ, NG, PAIRED>, p);
 }
 
 cudaError_t launch_decode(const DecodeParams &p, cudaStream_t st, int *launches, cudaEvent_t before,
@@ -1311,7 +1334,10 @@ cudaError_t launch_decode(const DecodeParams &p, cudaStream_t st, int *launches,
     cudaError_t e = cudaErrorInvalidValue;
     if (before) cudaEventRecord(before, st);
     H1B_DISPATCH_MW(p.m_words,
-        if (p.groups == 4) {
+        if (p.paired) {                                         // two 64-wide heads per slab
+            if (gq == 2 && p.groups == 4) e = launch_decode_t<MW, 2, 4, true>(p, st);
+            else if (gq == 2 && p.groups == 0) e = launch_decode_t<MW, 2, 0, true>(p, st);
+        } else if (p.groups == 4) {
             if (gq == 1) e = launch_decode_t<MW, 1, 4>(p, st);
             else if (gq == 2) e = launch_decode_t<MW, 2, 4>(p, st);
             else if (gq == 4) e = launch_decode_t<MW, 4, 4>(p, st);
@@ -1346,9 +1372,9 @@ cudaError_t launch_decode(const DecodeParams &p, cudaStream_t st, int *launches,
 }
 
 cudaError_t launch_debug_scores(const unsigned char *slab, const uint32_t *qwords, int m_words, int groups, int len,
-                                int32_t *score, cudaStream_t st) {
+                                int w0, int nw, int32_t *score, cudaStream_t st) {
     if (len <= 0) return cudaSuccess;
-    debug_scores_kernel<<<(len + 127) / 128, 128, 0, st>>>(slab, qwords, m_words, groups, len, score);
+    debug_scores_kernel<<<(len + 127) / 128, 128, 0, st>>>(slab, qwords, m_words, groups, len, w0, nw, score);
     return cudaGetLastError();
 }
 

@@ -148,6 +148,9 @@ struct DecodeParams {
     // tokens [0, len - Tq + i + 1). The Tq * (Hq/Hkv) (query token, query head) pairs that share a KV head are "virtual
     // heads" v = i * (Hq/Hkv) + head-in-group, handled `gqk` at a time by one work item (vgroups items per slab and split).
     int Tq, gqk, vgroups;
+    // Head dimension 64: two heads share a 128-channel slab (head h of the pair in channels 64h.., key words [h m/32, ..)),
+    // so Hkv counts pairs, Hq heads, m_words the words of both sketches, and a head's output has out_dim = 64 channels.
+    int paired, out_dim;
     float c2;                   // 2 * inv_tau * log2(e) / m : log2-weight per unit of Hamming distance
 };
 

@@ -45,6 +45,10 @@ def test_entry_and_workspace_bytes(lib):
     cv = binding.make_config(32, 32, 32, 128, 128, 128, max_batch=1, max_seq=8192)
     assert binding.h1b_entry_bytes(cv) == 84
     assert 32 * 32 * 8192 * 84 <= binding.h1b_cache_bytes(cv) < total
+    # 64-wide heads (12 layers x 8 heads, the small model of the paper): 16 + 32 + 2 * 4 bytes per token and head
+    c64 = binding.make_config(12, 8, 8, 64, 128, 32, max_batch=1, max_seq=4096)
+    assert binding.h1b_entry_bytes(c64) == 56
+    assert binding.h1b_cache_bytes(c64) >= 12 * 8 * 4096 * 56
     # capacity is rounded up to whole 32-token chunks
     a = binding.h1b_cache_bytes(binding.make_config(1, 1, 1, max_seq=33))
     b = binding.h1b_cache_bytes(binding.make_config(1, 1, 1, max_seq=64))
@@ -52,7 +56,8 @@ def test_entry_and_workspace_bytes(lib):
 
 
 @pytest.mark.parametrize("kw", [
-    dict(n_layers=0), dict(n_q_heads=3, n_kv_heads=2), dict(head_dim=64), dict(sketch_bits=100),
+    dict(n_layers=0), dict(n_q_heads=3, n_kv_heads=2), dict(head_dim=32), dict(head_dim=64, n_q_heads=8, n_kv_heads=4),
+    dict(head_dim=64, n_q_heads=3, n_kv_heads=3), dict(head_dim=64, sketch_bits=512), dict(sketch_bits=100),
     dict(sketch_bits=96), dict(group_size=64), dict(max_batch=0), dict(max_batch=257), dict(max_seq=0),
     dict(n_q_heads=8, n_kv_heads=1),
 ])
