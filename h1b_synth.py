@@ -47,6 +47,10 @@ WORKLOADS = {
                            notes="GQA 32/8, m=256, 32k context, batch 8"),
     "c5_prefill": Workload("c5_prefill", 32, 32, 32, 128, 128, 32, 1, 8192, index=5,
                            notes="prefill compression of 8192 tokens per layer, then one decode"),
+    # the paper's small model (12 layers, 8 heads of dimension 64, sketch width 256, 8k context); a batch of 32
+    # sequences, so that the cache (1.8 GB) does not sit in the L2
+    "c6_60m_8k": Workload("c6_60m_8k", 12, 8, 8, 64, 256, 32, 32, 8192, index=6,
+                          notes="60M GPT-2-style shape, head dimension 64, m=256, 8k context, batch 32"),
 }
 
 

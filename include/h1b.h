@@ -34,6 +34,11 @@
  *   - Score of token t for a query: m - 2 * popcount(s_q xor s_t); alpha = score / m.
  *     All cached tokens [0, len) are attended, the one just appended included.
  *     Query head h reads KV head h / (Hq / Hkv).  An empty sequence gives zeros.
+ *   - d = 64 (the paper's 60M model: 12 layers, 8 heads of 64 channels) runs
+ *     through the same 128-channel kernels, two heads per cache slab; nothing
+ *     of that shows at this interface (shapes, exports and results are per
+ *     head), except the restrictions listed at h1b_config.head_dim and that
+ *     h1b_decode_attention_multi() takes one query token only.
  *   - With H1B_FLAG_FP16_VALUES (the "1-bit keys only" row of the ablation,
  *     Table V) values are cached as the fp16 numbers they arrive as: no codes,
  *     scales or zero-points; the output is softmax(alpha/tau) * V.
@@ -63,7 +68,7 @@ typedef struct {
     int32_t n_layers;      /* L >= 1                                                   */
     int32_t n_q_heads;     /* Hq; Hq / Hkv must be 1, 2 or 4                           */
     int32_t n_kv_heads;    /* Hkv                                                      */
-    int32_t head_dim;      /* d: 128                                                   */
+    int32_t head_dim;      /* d: 128, or 64 (then Hq == Hkv, even, G = 32, m <= 256)    */
     int32_t sketch_bits;   /* m: 64, 128, 256 or 512                                   */
     int32_t group_size;    /* G: 32, or 128 (= d: one scale and zero per value vector)  */
     int32_t max_batch;     /* sequences the cache can hold (<= 256)                    */
