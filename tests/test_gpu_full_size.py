@@ -130,3 +130,12 @@ def test_c5_prefill_compression_then_decode_full_size():
     stats = _check_units(w, cache, Rt, units, kept, q, out, lens)
     print("c5 full size", stats)
     cache.close()
+
+
+def test_c6_60m_shape_head_dim_64_full_size():
+    """12 layers x 8 heads of 64 channels, m = 256, 8k context, 32 sequences: two heads per slab inside the library."""
+    w = W["c6_60m_8k"]
+    cache, Rt, units, kept, q, out, lens = _run_full(w, n_samples=4)
+    stats = _check_units(w, cache, Rt, units, kept, q, out, lens)
+    print("c6 full size", stats)
+    cache.close()
