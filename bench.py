@@ -140,14 +140,22 @@ def run_ours(args):
         w = h1b_synth.scaled(w, name=w.name + "[Tq=%d]" % Tq)
     total_steps = (3 * (steps + warmup) + 16) * Tq   # device-resident run, the host-buffer run, the per-layer graph run
     lens0 = h1b_synth.lengths(w) - 1                  # the first step decodes exactly the workload's context
+    page_tokens = max(0, args.page_tokens)
+    pages_per_seq = (w.context - 1 + total_steps + page_tokens - 1) // page_tokens if page_tokens else 0
+    if page_tokens:
+        w = h1b_synth.scaled(w, name=w.name + "[pages of %d tokens]" % page_tokens)
     cfg = binding.make_config(w.n_layers, w.n_q_heads, w.n_kv_heads, w.head_dim, w.sketch_bits, w.group_size,
                               max_batch=w.batch, max_seq=w.context - 1 + total_steps, device=local,
-                              fp16_values=args.fp16_values)
+                              fp16_values=args.fp16_values, page_tokens=page_tokens, n_pages=pages_per_seq * w.batch)
     # each rank is its own sequence: different seeds per rank
     wr = h1b_synth.scaled(w, index=w.index + 10 * rank)
     Rt = np.stack([h1b_synth.projection(h1b_synth.layer_seed(wr, l, 99), w.head_dim, w.sketch_bits)
                    for l in range(w.n_layers)])
     cache = binding.H1BCache(cfg, Rt=Rt)
+    if page_tokens:                                   # every sequence gets a seeded, scattered set of pool pages
+        perm = np.random.default_rng(7 + rank).permutation(pages_per_seq * w.batch)
+        for b in range(w.batch):
+            cache.h1b_set_block_table(b, perm[b * pages_per_seq:(b + 1) * pages_per_seq])
     for l in range(w.n_layers):                       # prefill, one layer at a time
         K, V = h1b_synth.kv_rows(wr, l, w.context - 1, device=str(dev))
         cache.h1b_append_kv(K.unsqueeze(0), V.unsqueeze(0), layer_begin=l, n_new=lens0)
@@ -451,6 +459,8 @@ def main():
     ap.add_argument("--no-layer-sequential", action="store_true", help="skip the per-layer CUDA-graph measurement")
     ap.add_argument("--query-tokens", type=int, default=1,
                     help="> 1: each step appends this many tokens per sequence and attends for all of them (variant)")
+    ap.add_argument("--page-tokens", type=int, default=0,
+                    help="> 0: a paged cache with pages of this many tokens, scattered over the pool (variant)")
     ap.add_argument("--fp16-values", action="store_true", help="keep values in fp16 (the 1-bit-keys-only ablation row)")
     ap.add_argument("--workload", default="c2_7b_8k",
                     choices=["c2_7b_8k", "c3_7b_batched", "c4_gqa_32k", "c5_prefill", "c6_60m_8k"],

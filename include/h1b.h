@@ -75,6 +75,9 @@ typedef struct {
     int32_t max_seq;       /* tokens per sequence the cache can hold                   */
     int32_t device;        /* CUDA device ordinal                                      */
     uint32_t flags;        /* H1B_FLAG_* bits; every other bit must be 0               */
+    int32_t page_tokens;   /* 0: one contiguous slab per sequence; > 0 (a multiple of
+                              32): paged cache, tokens per page                        */
+    int32_t n_pages;       /* paged cache: pages in each layer's pool (else 0)         */
 } h1b_config;
 
 /* Keep values in fp16 (keys are still 1-bit sketches); group_size must still be a
@@ -85,6 +88,24 @@ typedef struct {
  * storage statement plus the fp16 scale and zero per group); m/8 + 2d with
  * H1B_FLAG_FP16_VALUES. 0 if invalid. */
 size_t h1b_entry_bytes(const h1b_config *cfg /* HOST */);
+
+/* Paged cache (page_tokens > 0; not a step of the paper's method: the cache
+ * layout serving systems use for ragged batches). A page holds page_tokens
+ * consecutive tokens of every KV head of one layer; each layer has its own pool
+ * of n_pages pages; ONE block table per sequence, shared by all layers and
+ * heads, names the pool page that holds tokens [k * page_tokens, (k+1) *
+ * page_tokens) of the sequence. max_seq bounds a sequence's table, the pool
+ * bounds the total. A new context has empty tables: give every sequence its
+ * pages with h1b_set_block_table() before appending to it.
+ *
+ * h1b_set_block_table: sequence `seq` owns pages_host[0 .. n) (HOST int32, each
+ * in [0, n_pages), n * page_tokens <= max_seq rounded up to whole pages), in
+ * this order. May grow or shrink a table between steps; entries that cover
+ * cached tokens must keep their pages. The library does not check that two
+ * sequences do not share a page. Stream-ordered like the other calls.
+ * H1B_ERR_INVALID_ARG on a contiguous cache, on bad page numbers, or when fewer
+ * pages than the sequence's cached tokens need. */
+int h1b_set_block_table(h1b_ctx *ctx, int seq, const int32_t *pages_host, int n, void *stream);
 
 /* Bytes of device workspace the caller must provide for this configuration
  * (projection matrices, lengths, split-K scratch, staging and the packed cache
@@ -110,7 +131,8 @@ int h1b_init_projection(const h1b_config *cfg, uint64_t seed, const float *Rt_ho
  *               are appended (the first n_new[b] of its Tn); NULL = Tn for all
  * Sequence b of the call is sequence b of the cache.  Row tn of sequence b goes
  * to position len[layer][b] + tn; afterwards len[layer][b] += n_new[b].
- * H1B_ERR_CAPACITY (nothing written) if any sequence would exceed max_seq. */
+ * H1B_ERR_CAPACITY (nothing written) if any sequence would exceed max_seq or,
+ * with a paged cache, the pages its block table holds. */
 int h1b_append_kv(h1b_ctx *ctx, int layer_begin, int n_layers, const void *k, const void *v,
                   const int32_t *n_new_host, int B, int Tn, void *stream);
 

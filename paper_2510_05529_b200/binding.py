@@ -31,7 +31,8 @@ class H1BError(RuntimeError):
 class h1b_config(ctypes.Structure):
     _fields_ = [(n, ctypes.c_int32) for n in
                 ("n_layers", "n_q_heads", "n_kv_heads", "head_dim", "sketch_bits", "group_size",
-                 "max_batch", "max_seq", "device")] + [("flags", ctypes.c_uint32)]
+                 "max_batch", "max_seq", "device")] + [("flags", ctypes.c_uint32), ("page_tokens", ctypes.c_int32),
+                                                       ("n_pages", ctypes.c_int32)]
 
 
 _lib = None
@@ -69,6 +70,7 @@ def load_library(rebuild: bool = True) -> ctypes.CDLL:
         "h1b_decode_step_layers": (ctypes.c_int, [vp, ctypes.c_int, ctypes.c_int, vp, vp, vp, ctypes.c_float, vp,
                                                   ctypes.c_int, vp]),
         "h1b_sync_lengths": (ctypes.c_int, [vp, vp]),
+        "h1b_set_block_table": (ctypes.c_int, [vp, ctypes.c_int, i32p, ctypes.c_int, vp]),
         "h1b_decode_step_host": (ctypes.c_int, [vp, vp, vp, vp, ctypes.c_float, vp, ctypes.c_int, vp]),
         "h1b_free": (ctypes.c_int, [vp]),
         "h1b_get_projection": (ctypes.c_int, [vp, ctypes.c_int, vp]),
@@ -98,9 +100,10 @@ H1B_FLAG_FP16_VALUES = 1      # h1b_config.flags: values stay fp16 (the 1-bit-ke
 
 
 def make_config(n_layers, n_q_heads, n_kv_heads, head_dim=128, sketch_bits=128, group_size=32,
-                max_batch=1, max_seq=8192, device=0, fp16_values=False) -> h1b_config:
+                max_batch=1, max_seq=8192, device=0, fp16_values=False, page_tokens=0, n_pages=0) -> h1b_config:
+    """page_tokens > 0: a paged cache with n_pages pages of that many tokens in each layer's pool."""
     return h1b_config(n_layers, n_q_heads, n_kv_heads, head_dim, sketch_bits, group_size,
-                      max_batch, max_seq, device, H1B_FLAG_FP16_VALUES if fp16_values else 0)
+                      max_batch, max_seq, device, H1B_FLAG_FP16_VALUES if fp16_values else 0, page_tokens, n_pages)
 
 
 def h1b_entry_bytes(cfg: h1b_config) -> int:
@@ -242,6 +245,12 @@ class H1BCache:
         self._check(self.lib.h1b_decode_step_layers(self._h, layer_begin, n, kp, vp, qp, float(inv_tau), op, B,
                                                     _stream_ptr(stream)))
         return out
+
+    def h1b_set_block_table(self, seq: int, pages, stream=None):
+        """Paged cache: sequence `seq` owns these pool pages, in this order."""
+        arr = np.ascontiguousarray(pages, dtype=np.int32)
+        self._check(self.lib.h1b_set_block_table(self._h, seq, arr.ctypes.data_as(ctypes.POINTER(ctypes.c_int32)),
+                                                 int(arr.size), _stream_ptr(stream)))
 
     def h1b_sync_lengths(self, stream=None):
         """After replaying a captured graph that appends: refresh the host's copy of the lengths."""

@@ -27,6 +27,8 @@ constexpr int kPrefillMinTokens = 64;   // appends of at least this many tokens 
 struct Plan {
     size_t rt, rh, len, status, qwords, partial, stage_k, stage_v, stage_q, stage_out, dbg_q, dbg_row, dbg_s, cache, total;
     size_t partial_bytes, slab_bytes;
+    size_t table, seq_cap, layer_bytes;     // paged cache: block tables [max_batch][table_stride], capacities [max_batch]
+    int table_stride, page_chunks;          // 0 when the cache is contiguous
     int cap_tokens, m_words, gq, groups;
 };
 
@@ -53,6 +55,12 @@ int check_config(const h1b_config *c) {
         return H1B_ERR_UNSUPPORTED;
     }
     if ((long)c->n_layers * c->max_batch * c->n_kv_heads > (1L << 28)) return H1B_ERR_INVALID_ARG;
+    if (c->page_tokens < 0 || c->n_pages < 0) return H1B_ERR_INVALID_ARG;
+    if (c->page_tokens > 0) {
+        if (c->page_tokens % kChunkTokens != 0 || c->n_pages < 1) return H1B_ERR_INVALID_ARG;
+    } else if (c->n_pages != 0) {
+        return H1B_ERR_INVALID_ARG;
+    }
     return H1B_OK;
 }
 
@@ -80,6 +88,9 @@ int make_plan(const h1b_config *user, Plan *p) {
     const ChunkLayout cl = chunk_layout(p->m_words, p->groups);
     p->cap_tokens = (c->max_seq + kChunkTokens - 1) / kChunkTokens * kChunkTokens;
     p->slab_bytes = (size_t)(p->cap_tokens / kChunkTokens) * cl.bytes;
+    p->page_chunks = c->page_tokens / kChunkTokens;
+    p->table_stride = c->page_tokens > 0 ? (c->max_seq + c->page_tokens - 1) / c->page_tokens : 0;
+    p->layer_bytes = (size_t)c->n_pages * c->n_kv_heads * p->page_chunks * cl.bytes;
     const size_t L = c->n_layers, B = c->max_batch, Hq = c->n_q_heads, Hkv = c->n_kv_heads, d = c->head_dim;
     const size_t slabs = L * B * Hkv;
     // split-K scratch: room for kTargetItems work items (or one per slab) of four (virtual) heads each
@@ -100,7 +111,9 @@ int make_plan(const h1b_config *user, Plan *p) {
     p->dbg_q = take(p->m_words * sizeof(uint32_t));
     p->dbg_row = take(kHeadDim * 2);
     p->dbg_s = take((size_t)p->cap_tokens * sizeof(int32_t));
-    p->cache = take(slabs * p->slab_bytes);
+    p->table = take((size_t)c->max_batch * (p->table_stride ? p->table_stride : 1) * sizeof(int32_t));
+    p->seq_cap = take((size_t)c->max_batch * sizeof(int32_t));
+    p->cache = take(c->page_tokens > 0 ? L * p->layer_bytes : slabs * p->slab_bytes);
     p->total = o;
     return H1B_OK;
 }
@@ -135,6 +148,8 @@ struct h1b_ctx {
     ChunkLayout cl;
     unsigned char *ws;
     std::vector<int32_t> len_host;     // [L][max_batch], mirror of the device lengths
+    std::vector<int32_t> table_host;   // paged cache: mirror of the block tables [max_batch][table_stride], -1 = none
+    std::vector<int32_t> cap_host;     // tokens each sequence has room for (max_seq, or what its pages hold)
     int forced_splits;
     int64_t launches;
     bool profiling;
@@ -168,9 +183,33 @@ int fail(h1b_ctx *ctx, int code, const char *fmt, ...) {
 template <class T>
 T *at(h1b_ctx *ctx, size_t off) { return reinterpret_cast<T *>(ctx->ws + off); }
 
-unsigned char *slab_ptr(h1b_ctx *ctx, int layer, int seq, int kvh) {
-    return ctx->ws + ctx->plan.cache +
-           ((size_t)(layer * ctx->cfg.max_batch + seq) * ctx->cfg.n_kv_heads + kvh) * ctx->plan.slab_bytes;
+CacheAddr cache_addr(h1b_ctx *ctx) {
+    CacheAddr a;
+    a.base = ctx->ws + ctx->plan.cache;
+    a.table = ctx->plan.page_chunks ? at<int32_t>(ctx, ctx->plan.table) : nullptr;
+    a.slab_bytes = ctx->plan.slab_bytes;
+    a.layer_bytes = ctx->plan.layer_bytes;
+    a.table_stride = ctx->plan.table_stride; a.page_chunks = ctx->plan.page_chunks;
+    a.Hkv = ctx->cfg.n_kv_heads; a.max_batch = ctx->cfg.max_batch; a.chunk_bytes = ctx->cl.bytes;
+    return a;
+}
+
+// Chunks [c_lo, c_hi] of one slab, copied to the host (one copy when they are contiguous, one per chunk when paged).
+int fetch_chunks(h1b_ctx *ctx, int layer, int seq, int slab, int c_lo, int c_hi, std::vector<unsigned char> *raw) {
+    const CacheAddr a = cache_addr(ctx);
+    const size_t cb = ctx->cl.bytes;
+    raw->resize((size_t)(c_hi - c_lo + 1) * cb);
+    H1B_CUDA(ctx, cudaDeviceSynchronize());
+    if (!a.table) {
+        H1B_CUDA(ctx, cudaMemcpy(raw->data(), a.base + chunk_offset(a, nullptr, layer, seq, slab, c_lo), raw->size(),
+                                 cudaMemcpyDeviceToHost));
+        return H1B_OK;
+    }
+    for (int c = c_lo; c <= c_hi; ++c)
+        H1B_CUDA(ctx, cudaMemcpy(raw->data() + (size_t)(c - c_lo) * cb,
+                                 a.base + chunk_offset(a, ctx->table_host.data(), layer, seq, slab, c), cb,
+                                 cudaMemcpyDeviceToHost));
+    return H1B_OK;
 }
 
 int check_layers(h1b_ctx *ctx, int layer_begin, int n_layers, int B) {
@@ -219,6 +258,8 @@ int h1b_init_projection(const h1b_config *cfg, uint64_t seed, const float *Rt_ho
     ctx->cl = chunk_layout(plan.m_words, plan.groups);
     ctx->ws = static_cast<unsigned char *>(workspace);
     ctx->len_host.assign((size_t)cfg->n_layers * cfg->max_batch, 0);
+    ctx->table_host.assign((size_t)cfg->max_batch * (plan.table_stride ? plan.table_stride : 1), -1);
+    ctx->cap_host.assign((size_t)cfg->max_batch, plan.page_chunks ? 0 : cfg->max_seq);
     ctx->forced_splits = 0;
     ctx->launches = 0;
     ctx->profiling = false;
@@ -259,6 +300,12 @@ int h1b_init_projection(const h1b_config *cfg, uint64_t seed, const float *Rt_ho
     }
     e = cudaMemcpyAsync(ctx->ws + plan.rt, Rt_host, nR_dev * sizeof(float), cudaMemcpyHostToDevice, st);
     if (e != cudaSuccess) return bail(e, "cudaMemcpyAsync(Rt)");
+    e = cudaMemcpyAsync(ctx->ws + plan.table, ctx->table_host.data(), ctx->table_host.size() * sizeof(int32_t),
+                        cudaMemcpyHostToDevice, st);
+    if (e != cudaSuccess) return bail(e, "cudaMemcpyAsync(block tables)");
+    e = cudaMemcpyAsync(ctx->ws + plan.seq_cap, ctx->cap_host.data(), ctx->cap_host.size() * sizeof(int32_t),
+                        cudaMemcpyHostToDevice, st);
+    if (e != cudaSuccess) return bail(e, "cudaMemcpyAsync(capacities)");
     e = launch_split_projection(at<float>(ctx, plan.rt), at<uint16_t>(ctx, plan.rh), cfg->n_layers, ctx->cfg.sketch_bits, st);
     if (e != cudaSuccess) return bail(e, "split_projection_kernel");
     e = cudaStreamSynchronize(st);
@@ -290,9 +337,9 @@ static int make_new_counts(h1b_ctx *ctx, int layer_begin, int n_layers, const in
     }
     for (int l = layer_begin; l < layer_begin + n_layers; ++l)
         for (int b = 0; b < B; ++b)
-            if ((long)ctx->len_host[(size_t)l * ctx->cfg.max_batch + b] + nn->v[b] > ctx->cfg.max_seq)
-                return fail(ctx, H1B_ERR_CAPACITY, "layer %d sequence %d: %d + %d tokens exceed max_seq %d", l, b,
-                            ctx->len_host[(size_t)l * ctx->cfg.max_batch + b], nn->v[b], ctx->cfg.max_seq);
+            if ((long)ctx->len_host[(size_t)l * ctx->cfg.max_batch + b] + nn->v[b] > ctx->cap_host[b])
+                return fail(ctx, H1B_ERR_CAPACITY, "layer %d sequence %d: %d + %d tokens exceed its capacity of %d", l, b,
+                            ctx->len_host[(size_t)l * ctx->cfg.max_batch + b], nn->v[b], ctx->cap_host[b]);
     return H1B_OK;
 }
 
@@ -302,15 +349,14 @@ static AppendParams append_params(h1b_ctx *ctx, int layer_begin, int n_layers, c
     p.k = static_cast<const uint16_t *>(k);
     p.v = static_cast<const uint16_t *>(v);
     p.Rt = at<float>(ctx, ctx->plan.rt);
-    p.cache = ctx->ws + ctx->plan.cache;
+    p.ca = cache_addr(ctx);
     p.len = at<int32_t>(ctx, ctx->plan.len);
     p.done = at<int32_t>(ctx, ctx->plan.status) + 4;
     p.status = at<int32_t>(ctx, ctx->plan.status);
-    p.slab_bytes = ctx->plan.slab_bytes;
+    p.seq_cap = at<int32_t>(ctx, ctx->plan.seq_cap);
     p.layer_begin = layer_begin; p.n_layers = n_layers; p.B = B; p.Tn = Tn;
     p.Hkv = ctx->cfg.n_kv_heads; p.max_batch = ctx->cfg.max_batch; p.m_words = ctx->plan.m_words;
     p.groups = ctx->plan.groups;
-    p.max_seq = ctx->cfg.max_seq;
     return p;
 }
 
@@ -358,13 +404,12 @@ static int enqueue_decode(h1b_ctx *ctx, int layer_begin, int n_layers, float inv
     }
 
     DecodeParams dp;
-    dp.cache = ctx->ws + ctx->plan.cache;
+    dp.ca = cache_addr(ctx);
     dp.len = at<int32_t>(ctx, ctx->plan.len);
     dp.qwords = qwords;
     dp.partial = partial;
     dp.out = static_cast<float *>(out);
     dp.status = at<int32_t>(ctx, ctx->plan.status);
-    dp.slab_bytes = ctx->plan.slab_bytes;
     dp.layer_begin = layer_begin; dp.n_layers = n_layers; dp.B = B; dp.Hkv = ctx->cfg.n_kv_heads;
     dp.Hq = ctx->cfg.n_q_heads; dp.max_batch = ctx->cfg.max_batch; dp.m_words = ctx->plan.m_words;
     dp.groups = ctx->plan.groups;
@@ -409,11 +454,11 @@ int h1b_append_kv(h1b_ctx *ctx, int layer_begin, int n_layers, const void *k, co
         pp.k = static_cast<const uint16_t *>(k);
         pp.v = static_cast<const uint16_t *>(v);
         pp.Rh = at<uint16_t>(ctx, ctx->plan.rh);
-        pp.cache = ctx->ws + ctx->plan.cache;
+        pp.ca = cache_addr(ctx);
+        pp.seq_cap = at<int32_t>(ctx, ctx->plan.seq_cap);
         pp.len = at<int32_t>(ctx, ctx->plan.len);
         pp.status = at<int32_t>(ctx, ctx->plan.status);
         pp.done = at<int32_t>(ctx, ctx->plan.status) + 4;
-        pp.slab_bytes = ctx->plan.slab_bytes;
         pp.layer_begin = layer_begin; pp.n_layers = n_layers; pp.B = B; pp.Tn = Tn;
         pp.Hkv = ctx->cfg.n_kv_heads; pp.max_batch = ctx->cfg.max_batch; pp.m_words = ctx->plan.m_words;
         pp.groups = ctx->plan.groups;
@@ -693,12 +738,10 @@ int h1b_export_cache(h1b_ctx *ctx, int layer, int seq, int kv_head, int t0, int 
     if (n == 0) return H1B_OK;
     const ChunkLayout &cl = ctx->cl;
     const int c_lo = t0 / kChunkTokens, c_hi = (t0 + n - 1) / kChunkTokens;
-    std::vector<unsigned char> raw((size_t)(c_hi - c_lo + 1) * cl.bytes);
+    std::vector<unsigned char> raw;
     // with paired heads, head kv_head is half `half` of slab kv_head / 2: its share of the words, channel blocks and groups
     const int slab = ctx->paired ? kv_head / 2 : kv_head, half = ctx->paired ? (kv_head & 1) : 0;
-    H1B_CUDA(ctx, cudaDeviceSynchronize());
-    H1B_CUDA(ctx, cudaMemcpy(raw.data(), slab_ptr(ctx, layer, seq, slab) + (size_t)c_lo * cl.bytes, raw.size(),
-                             cudaMemcpyDeviceToHost));
+    { const int rcf = fetch_chunks(ctx, layer, seq, slab, c_lo, c_hi, &raw); if (rcf != H1B_OK) return rcf; }
     const int d = ctx->ucfg.head_dim, mw = ctx->ucfg.sketch_bits / 32;
     const int ng = ctx->paired ? cl.groups / 2 : cl.groups;
     const int w0 = half * mw, cb0 = half * (d / 16), g0 = half * ng;
@@ -735,11 +778,9 @@ int h1b_export_values(h1b_ctx *ctx, int layer, int seq, int kv_head, int t0, int
     if (n == 0) return H1B_OK;
     const ChunkLayout &cl = ctx->cl;
     const int c_lo = t0 / kChunkTokens, c_hi = (t0 + n - 1) / kChunkTokens;
-    std::vector<unsigned char> raw((size_t)(c_hi - c_lo + 1) * cl.bytes);
+    std::vector<unsigned char> raw;
     const int slab = ctx->paired ? kv_head / 2 : kv_head, half = ctx->paired ? (kv_head & 1) : 0;
-    H1B_CUDA(ctx, cudaDeviceSynchronize());
-    H1B_CUDA(ctx, cudaMemcpy(raw.data(), slab_ptr(ctx, layer, seq, slab) + (size_t)c_lo * cl.bytes, raw.size(),
-                             cudaMemcpyDeviceToHost));
+    { const int rcf = fetch_chunks(ctx, layer, seq, slab, c_lo, c_hi, &raw); if (rcf != H1B_OK) return rcf; }
     const int d = ctx->ucfg.head_dim;
     for (int i = 0; i < n; ++i) {
         const int t = t0 + i, tt = t % kChunkTokens;
@@ -777,7 +818,7 @@ int h1b_debug_scores(h1b_ctx *ctx, int layer, int seq, int kv_head, const void *
     NewCounts none;
     std::memset(&none, 0, sizeof none);
     H1B_CUDA(ctx, launch_prepare(nullptr, &sp, none, nullptr, &launches));
-    H1B_CUDA(ctx, launch_debug_scores(slab_ptr(ctx, layer, seq, slab), sp.qwords, mw, ctx->plan.groups, len, half * mwh, mwh,
+    H1B_CUDA(ctx, launch_debug_scores(cache_addr(ctx), layer, seq, slab, sp.qwords, len, half * mwh, mwh,
                                       at<int32_t>(ctx, ctx->plan.dbg_s), nullptr));
     H1B_CUDA(ctx, cudaDeviceSynchronize());
     if (qwords_host)
@@ -785,6 +826,34 @@ int h1b_debug_scores(h1b_ctx *ctx, int layer, int seq, int kv_head, const void *
     if (score_host && len > 0)
         H1B_CUDA(ctx, cudaMemcpy(score_host, at<int32_t>(ctx, ctx->plan.dbg_s), (size_t)len * sizeof(int32_t),
                                  cudaMemcpyDeviceToHost));
+    return H1B_OK;
+}
+
+int h1b_set_block_table(h1b_ctx *ctx, int seq, const int32_t *pages_host, int n, void *stream) {
+    if (!ctx) return H1B_ERR_NULL;
+    if (!ctx->plan.page_chunks) return fail(ctx, H1B_ERR_INVALID_ARG, "this cache is not paged");
+    if (seq < 0 || seq >= ctx->cfg.max_batch) return fail(ctx, H1B_ERR_INVALID_ARG, "sequence %d out of range", seq);
+    if (n < 0 || n > ctx->plan.table_stride)
+        return fail(ctx, H1B_ERR_INVALID_ARG, "%d pages outside [0, %d]", n, ctx->plan.table_stride);
+    if (n > 0 && !pages_host) return fail(ctx, H1B_ERR_NULL, "pages_host is NULL");
+    for (int i = 0; i < n; ++i)
+        if (pages_host[i] < 0 || pages_host[i] >= ctx->cfg.n_pages)
+            return fail(ctx, H1B_ERR_INVALID_ARG, "page %d (entry %d) outside the pool of %d", pages_host[i], i, ctx->cfg.n_pages);
+    const int page_tokens = ctx->cfg.page_tokens;
+    int held = 0;
+    for (int l = 0; l < ctx->cfg.n_layers; ++l) held = std::max(held, ctx->len_host[(size_t)l * ctx->cfg.max_batch + seq]);
+    if ((long)n * page_tokens < held)
+        return fail(ctx, H1B_ERR_INVALID_ARG, "sequence %d holds %d tokens: %d pages of %d are too few", seq, held, n, page_tokens);
+    int32_t *row = ctx->table_host.data() + (size_t)seq * ctx->plan.table_stride;
+    for (int i = 0; i < ctx->plan.table_stride; ++i) row[i] = i < n ? pages_host[i] : -1;
+    ctx->cap_host[seq] = (int)std::min<long>((long)n * page_tokens, ctx->cfg.max_seq);
+    cudaStream_t st = static_cast<cudaStream_t>(stream);
+    // (the host copies are the source, and they may change before the copies run: synchronise)
+    H1B_CUDA(ctx, cudaMemcpyAsync(at<int32_t>(ctx, ctx->plan.table) + (size_t)seq * ctx->plan.table_stride, row,
+                                  (size_t)ctx->plan.table_stride * sizeof(int32_t), cudaMemcpyHostToDevice, st));
+    H1B_CUDA(ctx, cudaMemcpyAsync(at<int32_t>(ctx, ctx->plan.seq_cap) + seq, &ctx->cap_host[seq], sizeof(int32_t),
+                                  cudaMemcpyHostToDevice, st));
+    H1B_CUDA(ctx, cudaStreamSynchronize(st));
     return H1B_OK;
 }
 

@@ -182,10 +182,9 @@ __global__ void __launch_bounds__(kProjThreads) prepare_kernel(AppendParams ap, 
         const uint32_t bits = project_tile(sm, ap.k + ((size_t)ll * k_rows + row0) * kHeadDim, n_rows,
                                            ap.Rt + (size_t)layer * kHeadDim * m, m, word);
         if ((int)threadIdx.x < n_rows) {
-            if (tn < nn.v[b] && len0 + nn.v[b] <= ap.max_seq) {
+            if (tn < nn.v[b] && len0 + nn.v[b] <= ap.seq_cap[b]) {
                 const int t = len0 + tn;
-                unsigned char *chunk = ap.cache + ((size_t)(layer * ap.max_batch + b) * ap.Hkv + kvh) * ap.slab_bytes +
-                                       (size_t)(t >> 5) * cl.bytes;
+                unsigned char *chunk = chunk_ptr(ap.ca, layer, b, kvh, t >> 5);
                 *reinterpret_cast<uint32_t *>(chunk + key_word_off(word, t & 31)) = bits;
             }
         }
@@ -210,10 +209,9 @@ __global__ void __launch_bounds__(kProjThreads) prepare_kernel(AppendParams ap, 
             const int b = (int)((row / ((long)ap.Hkv * ap.Tn)) % ap.B), ll = (int)(row / k_rows);
             const int layer = ap.layer_begin + ll;
             const int len0 = ap.len[layer * ap.max_batch + b];
-            if (tn < nn.v[b] && len0 + nn.v[b] <= ap.max_seq) {
+            if (tn < nn.v[b] && len0 + nn.v[b] <= ap.seq_cap[b]) {
                 const int t = len0 + tn;
-                unsigned char *chunk = ap.cache + ((size_t)(layer * ap.max_batch + b) * ap.Hkv + kvh) * ap.slab_bytes +
-                                       (size_t)(t >> 5) * cl.bytes;
+                unsigned char *chunk = chunk_ptr(ap.ca, layer, b, kvh, t >> 5);
                 store_value_row(ap.v + row * kHeadDim, chunk, cl, t & 31, threadIdx.x & 31);
             }
         }
@@ -231,7 +229,7 @@ __global__ void __launch_bounds__(kProjThreads) prepare_kernel(AppendParams ap, 
         for (int i = threadIdx.x; i < ap.n_layers * ap.B; i += blockDim.x) {
             int32_t *len = ap.len + (ap.layer_begin + i / ap.B) * ap.max_batch + (i % ap.B);
             const int n = nn.v[i % ap.B];
-            if (*len + n <= ap.max_seq) *len += n;
+            if (*len + n <= ap.seq_cap[i % ap.B]) *len += n;
             else atomicExch(ap.status, kStatusCapacity);        // full: nothing of this sequence's rows was written
         }
         if (threadIdx.x == 0) *ap.done = 0;
@@ -292,11 +290,11 @@ __device__ __forceinline__ __half exact_scale(float mx, float mn) {
 
 // Eq. 4 (or the fp16 copy) for the 16 cache positions pos0 .. pos0+15 of one slab, by one warp. `vs` is 1280 bytes of
 // shared memory owned by the warp. Positions outside the appended range [len0, len0 + n_new) are left alone.
-__device__ __forceinline__ void store_value_block16(const PrefillParams &p, const ChunkLayout &cl, unsigned char *slab,
+__device__ __forceinline__ void store_value_block16(const PrefillParams &p, const ChunkLayout &cl, int layer,
                                                     int ll, int b, int kvh, int len0, int n_new, int pos0,
                                                     unsigned char *vs, int lane) {
     const int tn0 = pos0 - len0;
-    unsigned char *chunk = slab + (size_t)(pos0 >> 5) * cl.bytes;
+    unsigned char *chunk = chunk_ptr(p.ca, layer, b, kvh, pos0 >> 5);
     const int vb = (pos0 >> 4) & 1;
     if (p.groups == 0 && tn0 >= 0 && tn0 + 16 <= n_new) {
         // fp16 values, a whole block of 16 tokens: transposed through shared memory into the A-operand
@@ -434,7 +432,7 @@ __device__ __forceinline__ void store_value_block16(const PrefillParams &p, cons
             const int tn = tn0 + k;
             if (tn >= 0 && tn < n_new)
                 store_value_row(p.v + ((((size_t)ll * p.B + b) * p.Tn + tn) * p.Hkv + kvh) * kHeadDim,
-                                slab + (size_t)((pos0 + k) >> 5) * cl.bytes, cl, (pos0 + k) & 31, lane);
+                                chunk, cl, (pos0 + k) & 31, lane);     // 16 aligned positions: all in this chunk
         }
     }
 }
@@ -449,8 +447,12 @@ __device__ __forceinline__ void prefill_publish_lengths(const PrefillParams &p, 
     }
     __syncthreads();
     if (*is_last_s) {
-        for (int i = threadIdx.x; i < p.n_layers * p.B; i += blockDim.x)
-            p.len[(p.layer_begin + i / p.B) * p.max_batch + (i % p.B)] += nn.v[i % p.B];
+        for (int i = threadIdx.x; i < p.n_layers * p.B; i += blockDim.x) {
+            int32_t *len = p.len + (p.layer_begin + i / p.B) * p.max_batch + (i % p.B);
+            const int n = nn.v[i % p.B];
+            if (*len + n <= p.seq_cap[i % p.B]) *len += n;
+            else atomicExch(p.status, kStatusCapacity);         // full: nothing of this sequence's rows was written
+        }
         if (threadIdx.x == 0) *p.done = 0;
     }
 }
@@ -475,11 +477,10 @@ __global__ void __launch_bounds__(kValueWarps * 32) prefill_values_kernel(Prefil
         const int b = (int)(seq_local % p.B), ll = (int)(seq_local / p.B);
         const int layer = p.layer_begin + ll;
         const int len0 = p.len[layer * p.max_batch + b];
-        const int n_new = nn.v[b];
+        const int n_new = (len0 + nn.v[b] <= p.seq_cap[b]) ? nn.v[b] : 0;       // no room: nothing is written
         const int pos0 = (len0 / kPrefillTile) * kPrefillTile + blk * 16;
         if (pos0 + 16 > len0 && pos0 < len0 + n_new) {
-            unsigned char *slab = p.cache + ((size_t)(layer * p.max_batch + b) * p.Hkv + kvh) * p.slab_bytes;
-            store_value_block16(p, cl, slab, ll, b, kvh, len0, n_new, pos0, vs_all[warp], lane);
+            store_value_block16(p, cl, layer, ll, b, kvh, len0, n_new, pos0, vs_all[warp], lane);
         }
     }
     prefill_publish_lengths(p, nn, &is_last);
@@ -535,8 +536,7 @@ __global__ void __launch_bounds__(kPrefillThreads, 1) prefill_kernel(PrefillPara
         const int layer = p.layer_begin + ll;
         const int col0 = cbk * NBC;                             // first sketch column of this work item
         const int len0 = p.len[layer * p.max_batch + b];
-        const int n_new = nn.v[b];
-        unsigned char *slab = p.cache + ((size_t)(layer * p.max_batch + b) * p.Hkv + kvh) * p.slab_bytes;
+        const int n_new = (len0 + nn.v[b] <= p.seq_cap[b]) ? nn.v[b] : 0;       // no room: nothing is written
         const int first_tile = len0 / kPrefillTile + tg * p.tiles_per_block;
         // tiles of this work item that overlap the appended range (block-uniform)
         const int n_tiles = max(0, min(p.tiles_per_block,
@@ -620,6 +620,8 @@ __global__ void __launch_bounds__(kPrefillThreads, 1) prefill_kernel(PrefillPara
                 const int P0 = (first_tile + ti) * kPrefillTile;
                 const int quarter = warp & 3;
                 const int pos = P0 + quarter * 32 + lane, tn = pos - len0;
+                // this warp's 32 rows are the 32 tokens of one chunk
+                unsigned char *chunk = chunk_ptr(p.ca, layer, b, kvh, (P0 >> 5) + quarter);
 #pragma unroll
                 for (int w = warp >> 2; w < NBC / 32; w += kPrefillThreads / 128) {
                     uint32_t y[32];
@@ -635,7 +637,7 @@ __global__ void __launch_bounds__(kPrefillThreads, 1) prefill_kernel(PrefillPara
                             part[k] = __funnelshift_l(__float_as_uint(__uint_as_float(y[8 * k + j]) + 0.f), part[k], 1);
                     const uint32_t neg = part[0] | (part[1] << 8) | (part[2] << 16) | (part[3] << 24);
                     if (tn >= 0 && tn < n_new)
-                        *reinterpret_cast<uint32_t *>(slab + (size_t)(pos >> 5) * cl.bytes + (pos & 31) * 4 + (col0 / 32 + w) * 128) = ~neg;
+                        *reinterpret_cast<uint32_t *>(chunk + lane * 4 + (col0 / 32 + w) * 128) = ~neg;
                 }
             } else if (lane == 0) {
                 atomicExch(p.status, kStatusWaitTimeout);
@@ -906,7 +908,7 @@ __device__ __forceinline__ SplitShare split_share(int n_chunks, int n_splits) {
 __device__ __forceinline__ int split_first_chunk(int s, const SplitShare &sh) { return s * sh.q + min(s, sh.r); }
 __device__ __forceinline__ bool split_is_empty(int s, const SplitShare &sh) { return sh.q == 0 && s >= sh.r; }
 
-template <int MW, int GQ, int NG, bool PAIRED>
+template <int MW, int GQ, int NG, bool PAIRED, bool PAGED>
 __global__ void __launch_bounds__(kDecodeWarps * 32, decode_min_blocks(GQ, NG)) decode_split_kernel(DecodeParams p) {
     using SM = DecodeSmem<MW, GQ, NG>;
     constexpr int MWH = PAIRED ? MW / 2 : MW;                   // key words of one head
@@ -941,21 +943,44 @@ __global__ void __launch_bounds__(kDecodeWarps * 32, decode_min_blocks(GQ, NG)) 
     float *p_s = reinterpret_cast<float *>(ring + kStages * CB);
     const uint32_t bar0 = smem_addr(ring + kStages * CB + GQ * 128);
     const uint32_t ring_a = smem_addr(ring);
-    const unsigned char *slab =
-        p.cache + ((size_t)(layer * p.max_batch + b) * p.Hkv + kvh) * p.slab_bytes;
-
     if (lane == 0) {
 #pragma unroll
         for (int s = 0; s < kStages; ++s) mbar_init(bar0 + 8 * s, 1);
         mbar_fence_init();
     }
     __syncwarp();
-    const unsigned char *src = slab + (size_t)c0 * CB;          // next chunk to request
+    // Next chunk to request (lane 0 does the requesting). A slab's chunks follow one another in memory, except from
+    // page to page of a paged cache: there the walk keeps its place in the page and in the sequence's block table, and
+    // reads the number of the page after the current one ahead of time. That state lives in this warp's shared
+    // memory (three words behind the barriers); the contiguous case (PAGED false) has none of it.
+    const unsigned char *src = chunk_ptr(p.ca, layer, b, kvh, c0);
     int requested = c0;
+    int *walk = reinterpret_cast<int *>(ring + kStages * CB + GQ * 128 + 64);     // left in page, page index, next page
+    if (PAGED && lane == 0) {
+        const int32_t *table_row = p.ca.table + (size_t)b * p.ca.table_stride;
+        const int page_idx = c0 / p.ca.page_chunks;
+        walk[0] = p.ca.page_chunks - (c0 - page_idx * p.ca.page_chunks);
+        walk[1] = page_idx;
+        walk[2] = (page_idx + 1 < p.ca.table_stride) ? table_row[page_idx + 1] : 0;
+    }
+#define H1B_NEXT_CHUNK()                                                                                        \
+    do {                                                                                                        \
+        ++requested;                                                                                            \
+        src += CB;                                                                                              \
+        if (PAGED && --walk[0] == 0) {                                                                          \
+            const int page_idx = ++walk[1];                                                                     \
+            walk[0] = p.ca.page_chunks;                                                                         \
+            src = p.ca.base + (size_t)layer * p.ca.layer_bytes +                                                \
+                  ((size_t)walk[2] * p.ca.Hkv + kvh) * ((size_t)p.ca.page_chunks * CB);                         \
+            walk[2] = (page_idx + 1 < p.ca.table_stride && requested < c1)                                      \
+                          ? p.ca.table[(size_t)b * p.ca.table_stride + page_idx + 1] : 0;                       \
+        }                                                                                                       \
+    } while (0)
     if (lane == 0) {
-        for (int s = 0; s < kStages && requested < c1; ++s, ++requested, src += CB) {
+        for (int s = 0; s < kStages && requested < c1; ++s) {
             mbar_arrive_expect_tx(bar0 + 8 * s, CB);
             bulk_copy_g2s(ring_a + s * CB, src, CB, bar0 + 8 * s);
+            H1B_NEXT_CHUNK();
         }
     }
 
@@ -1004,11 +1029,11 @@ __global__ void __launch_bounds__(kDecodeWarps * 32, decode_min_blocks(GQ, NG)) 
         if (lane == 0 && requested < c1) {
             mbar_arrive_expect_tx(bar0 + 8 * stage, CB);
             bulk_copy_g2s(ring_a + stage * CB, src, CB, bar0 + 8 * stage);
-            ++requested;
-            src += CB;
+            H1B_NEXT_CHUNK();
         }
         if (++stage == kStages) { stage = 0; parity ^= 1; }
     }
+#undef H1B_NEXT_CHUNK
 
     if (failed) {
         if (lane == 0) atomicExch(p.status, kStatusWaitTimeout);
@@ -1164,12 +1189,11 @@ __global__ void __launch_bounds__(kHeadDim) combine_kernel(DecodeParams p) {
 
 // Test helper: score of every cached token of one slab against one sketch.
 // Key words [w0, w0 + nw) of the slab (one head's sketch) against qwords[0 .. nw).
-__global__ void debug_scores_kernel(const unsigned char *slab, const uint32_t *qwords, int m_words, int groups, int len,
+__global__ void debug_scores_kernel(CacheAddr ca, int layer, int b, int kvh, const uint32_t *qwords, int len,
                                     int w0, int nw, int32_t *score) {
     const int t = blockIdx.x * blockDim.x + threadIdx.x;
     if (t >= len) return;
-    const ChunkLayout cl = chunk_layout(m_words, groups);
-    const unsigned char *chunk = slab + (size_t)(t >> 5) * cl.bytes;
+    const unsigned char *chunk = chunk_ptr(ca, layer, b, kvh, t >> 5);
     int ham = 0;
     for (int w = 0; w < nw; ++w)
         ham += __popc(*reinterpret_cast<const uint32_t *>(chunk + key_word_off(w0 + w, t & 31)) ^ qwords[w]);
@@ -1301,14 +1325,14 @@ cudaError_t launch_set_len(int32_t *len, int n_layers, int max_batch, int seq, i
     return cudaGetLastError();
 }
 
-template <int MW, int GQ, int NG, bool PAIRED = false>
-static cudaError_t launch_decode_t(const DecodeParams &p, cudaStream_t st) {
+template <int MW, int GQ, int NG, bool PAIRED, bool PAGED>
+static cudaError_t launch_decode_tt(const DecodeParams &p, cudaStream_t st) {
     using SM = DecodeSmem<MW, GQ, NG>;
     static bool attr_set[64] = {};
     int dev = 0;
     cudaGetDevice(&dev);
     if (dev >= 0 && dev < 64 && !attr_set[dev]) {
-        cudaError_t e = cudaFuncSetAttribute(decode_split_kernel<MW, GQ, NG, PAIRED>,
+        cudaError_t e = cudaFuncSetAttribute(decode_split_kernel<MW, GQ, NG, PAIRED, PAGED>,
                                              cudaFuncAttributeMaxDynamicSharedMemorySize, SM::kTotal);
         if (e != cudaSuccess) return e;
         attr_set[dev] = true;
@@ -1325,7 +1349,12 @@ static cudaError_t launch_decode_t(const DecodeParams &p, cudaStream_t st) {
     attr[0].val.programmaticStreamSerializationAllowed = 1;
     cfg.attrs = attr;
     cfg.numAttrs = 1;
-    return cudaLaunchKernelEx(&cfg, decode_split_kernel<MW, GQ, NG, PAIRED>, p);
+    return cudaLaunchKernelEx(&cfg, decode_split_kernel<MW, GQ, NG, PAIRED, PAGED>, p);
+}
+
+template <int MW, int GQ, int NG, bool PAIRED = false>
+static cudaError_t launch_decode_t(const DecodeParams &p, cudaStream_t st) {
+    return p.ca.table ? launch_decode_tt<MW, GQ, NG, PAIRED, true>(p, st) : launch_decode_tt<MW, GQ, NG, PAIRED, false>(p, st);
 }
 
 cudaError_t launch_decode(const DecodeParams &p, cudaStream_t st, int *launches, cudaEvent_t before,
@@ -1371,10 +1400,10 @@ cudaError_t launch_decode(const DecodeParams &p, cudaStream_t st, int *launches,
     return cudaGetLastError();
 }
 
-cudaError_t launch_debug_scores(const unsigned char *slab, const uint32_t *qwords, int m_words, int groups, int len,
+cudaError_t launch_debug_scores(const CacheAddr &ca, int layer, int b, int kvh, const uint32_t *qwords, int len,
                                 int w0, int nw, int32_t *score, cudaStream_t st) {
     if (len <= 0) return cudaSuccess;
-    debug_scores_kernel<<<(len + 127) / 128, 128, 0, st>>>(slab, qwords, m_words, groups, len, w0, nw, score);
+    debug_scores_kernel<<<(len + 127) / 128, 128, 0, st>>>(ca, layer, b, kvh, qwords, len, w0, nw, score);
     return cudaGetLastError();
 }
 

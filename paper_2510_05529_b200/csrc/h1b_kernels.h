@@ -20,7 +20,7 @@ cudaError_t launch_decode(const DecodeParams &p, cudaStream_t st, int *launches,
                           cudaEvent_t after = nullptr);
 cudaError_t launch_set_len(int32_t *len, int n_layers, int max_batch, int seq, int value, cudaStream_t st);
 // Scores of key words [w0, w0 + nw) of every cached token of one slab against qwords[0 .. nw).
-cudaError_t launch_debug_scores(const unsigned char *slab, const uint32_t *qwords, int m_words, int groups, int len,
+cudaError_t launch_debug_scores(const CacheAddr &ca, int layer, int b, int kvh, const uint32_t *qwords, int len,
                                 int w0, int nw, int32_t *score, cudaStream_t st);
 
 }  // namespace h1b

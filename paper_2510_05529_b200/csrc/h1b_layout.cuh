@@ -92,6 +92,26 @@ __host__ __device__ inline int scale_off(const ChunkLayout &c, int tt, int g) {
     return c.scale_off + (tt >> 4) * (32 * c.groups) + g * 32 + (tt & 15) * 2;
 }
 
+// Where the chunks of a slab live. Contiguous cache: slab (layer, sequence, KV head) is one run of chunks. Paged cache:
+// a page holds `page_chunks` consecutive chunks of every KV head of one layer ([Hkv][page_chunks] chunks); every layer has
+// its own pool of pages, and one block table per sequence (shared by all layers and heads) says which page of the pool
+// holds the sequence's k-th run of page_chunks chunks.
+struct CacheAddr {
+    unsigned char *base;        // contiguous: slab 0; paged: page 0 of layer 0
+    const int32_t *table;       // paged: [max_batch][table_stride] page numbers; null = contiguous
+    size_t slab_bytes;          // contiguous: bytes of one slab
+    size_t layer_bytes;         // paged: bytes of one layer's pool
+    int table_stride, page_chunks, Hkv, max_batch, chunk_bytes;
+};
+__host__ __device__ inline size_t chunk_offset(const CacheAddr &a, const int32_t *table, int layer, int b, int kvh, int c) {
+    if (!table) return ((size_t)(layer * a.max_batch + b) * a.Hkv + kvh) * a.slab_bytes + (size_t)c * a.chunk_bytes;
+    const int page = table[(size_t)b * a.table_stride + c / a.page_chunks];
+    return (size_t)layer * a.layer_bytes + (((size_t)page * a.Hkv + kvh) * a.page_chunks + c % a.page_chunks) * (size_t)a.chunk_bytes;
+}
+__device__ inline unsigned char *chunk_ptr(const CacheAddr &a, int layer, int b, int kvh, int c) {
+    return a.base + chunk_offset(a, a.table, layer, b, kvh, c);
+}
+
 // Device status word values.
 constexpr int kStatusOk = 0;
 constexpr int kStatusWaitTimeout = 1;
@@ -103,23 +123,23 @@ struct NewCounts { int32_t v[256]; };            // n_new per sequence, passed b
 struct AppendParams {
     const uint16_t *k, *v;      // fp16 [n_layers][B][Tn][Hkv][d]
     const float *Rt;            // [L][d][m]
-    unsigned char *cache;       // slab 0
+    CacheAddr ca;
     int32_t *len;               // [L][max_batch]
     int32_t *done;              // block counter of the append launch (zero between launches)
     int32_t *status;            // device status word
-    size_t slab_bytes;
+    const int32_t *seq_cap;     // [max_batch] tokens each sequence has room for: an append that would pass it is dropped
+                                // and flagged (only a replayed graph can get there: direct calls are checked on the host)
     int layer_begin, n_layers, B, Tn, Hkv, max_batch, m_words, groups;
-    int max_seq;                // capacity of a sequence: rows that would land at or beyond it are dropped and flagged
 };
 
 struct PrefillParams {          // long appends: tensor-core projection
     const uint16_t *k, *v;      // fp16 [n_layers][B][Tn][Hkv][d]
     const uint16_t *Rh;         // fp16 [L][2][m][d]: Rt^T split as fp16(Rt) + fp16(Rt - fp16(Rt))
-    unsigned char *cache;
+    CacheAddr ca;
     int32_t *len;               // [L][max_batch]
     int32_t *status;            // device status word (bounded-wait timeouts)
     int32_t *done;              // block counter (zero between launches)
-    size_t slab_bytes;
+    const int32_t *seq_cap;     // [max_batch] tokens each sequence has room for (see AppendParams)
     int layer_begin, n_layers, B, Tn, Hkv, max_batch, m_words, groups;
     int tiles_per_seq;          // 128-position tiles that can overlap the appended range of a sequence
     int tiles_per_block;        // consecutive tiles handled by one block (the projection is loaded once per block)
@@ -135,13 +155,12 @@ struct SketchParams {           // query sketch
 };
 
 struct DecodeParams {
-    const unsigned char *cache;
+    CacheAddr ca;
     const int32_t *len;         // [L][max_batch]
     const uint32_t *qwords;     // [L][max_batch][Tq][Hq][m/32]
     float *partial;             // [items][gqk][kPartStride]
     float *out;                 // fp32 [n_layers][B][Tq][Hq][d]
     int32_t *status;
-    size_t slab_bytes;
     int layer_begin, n_layers, B, Hkv, Hq, max_batch, m_words, groups;
     int splits;                 // work items per (slab, group of virtual heads): each takes an even share of the chunks
     // Several query tokens per sequence (Tq > 1): they are the sequence's last Tq cached tokens, query token i attends to

@@ -18,9 +18,10 @@ def f16_bits(t: torch.Tensor) -> np.ndarray:
     return t.detach().cpu().contiguous().view(torch.int16).numpy().view(np.uint16)
 
 
-def make_cache(w: h1b_synth.Workload, max_seq=None, Rt=None, fp16_values=False):
+def make_cache(w: h1b_synth.Workload, max_seq=None, Rt=None, fp16_values=False, page_tokens=0, n_pages=0):
     cfg = binding.make_config(w.n_layers, w.n_q_heads, w.n_kv_heads, w.head_dim, w.sketch_bits, w.group_size,
-                              max_batch=w.batch, max_seq=max_seq or w.context, fp16_values=fp16_values)
+                              max_batch=w.batch, max_seq=max_seq or w.context, fp16_values=fp16_values,
+                              page_tokens=page_tokens, n_pages=n_pages)
     if Rt is None:
         Rt = np.stack([h1b_synth.projection(h1b_synth.layer_seed(w, l, 99), w.head_dim, w.sketch_bits)
                        for l in range(w.n_layers)])
