@@ -134,6 +134,16 @@ def run_ours(args):
         w = h1b_synth.scaled(w, name=w.name + "[fp16 values]")
     if args.workload == "c5_prefill":
         return run_prefill(args, w, pdist, rank, world, local)
+    # --shard heads: the ranks split the KV heads (and their query heads) of the SAME sequences between them: every
+    # (layer, sequence, KV head) is independent, so there is still no collective on the data path; the job then
+    # produces w.batch tokens per step however many ranks there are (strong scaling)
+    shard_heads = args.shard == "heads" and world > 1
+    if shard_heads:
+        if w.n_kv_heads % world:
+            raise SystemExit("--shard heads needs the KV heads (%d) to divide by the ranks (%d)" % (w.n_kv_heads, world))
+        w = h1b_synth.scaled(w, n_q_heads=w.n_q_heads // world, n_kv_heads=w.n_kv_heads // world,
+                             name=w.name + "[1/%d of the heads per rank]" % world)
+    job_ranks = 1 if shard_heads else world           # how many ranks' tokens add up
     steps, warmup = args.steps, args.warmup
     Tq = max(1, args.query_tokens)                    # > 1: a step appends Tq tokens and attends for all of them at once
     if Tq > 1:
@@ -272,8 +282,8 @@ def run_ours(args):
     if seq_ms_total is not None:
         seq_ms_total = pdist.max_over_ranks([seq_ms_total], dev)[0]
     ms_per_step = ms_total / steps
-    value = pdist.whole_job_rate(w.batch * Tq, world, ms_per_step * 1e-3)
-    e2e_value = pdist.whole_job_rate(w.batch, world, e2e_ms_total / steps * 1e-3) if Tq == 1 else None
+    value = pdist.whole_job_rate(w.batch * Tq, job_ranks, ms_per_step * 1e-3)
+    e2e_value = pdist.whole_job_rate(w.batch, job_ranks, e2e_ms_total / steps * 1e-3) if Tq == 1 else None
 
     # roofline of the dominant kernel (split-K decode attention), per launch
     entry = binding.h1b_entry_bytes(cfg)
@@ -295,7 +305,7 @@ def run_ours(args):
                 "step_gbs": alg_bytes / (ms_per_step * 1e-3) / 1e9}
     line = {
         "metric": METRIC, "value": value, "unit": UNIT, "n_gpus": world, "steps": steps, "warmup": warmup,
-        "ms_per_step": ms_per_step, "higher_is_better": True, "scaling": "weak", "vs_baseline": None,
+        "ms_per_step": ms_per_step, "higher_is_better": True, "scaling": "strong" if shard_heads else "weak", "vs_baseline": None,
         "dtype": "f32", "data": "synthetic",
         "config": {"workload": "%s: %d layers x %d/%d heads, d=%d, m=%d, batch %d per GPU, %s; fp16 K/V ~ N(0,1)%s, one "
                                "projection per layer" % (w.name, w.n_layers, w.n_q_heads, w.n_kv_heads, w.head_dim,
@@ -312,7 +322,7 @@ def run_ours(args):
         "roofline": roofline,
     }
     if seq_ms_total is not None:                      # not the headline: the same step issued layer by layer
-        line["layer_sequential"] = {"value": pdist.whole_job_rate(w.batch, world, seq_ms_total / steps * 1e-3), "unit": UNIT,
+        line["layer_sequential"] = {"value": pdist.whole_job_rate(w.batch, job_ranks, seq_ms_total / steps * 1e-3), "unit": UNIT,
                                     "ms_per_step": seq_ms_total / steps, "launches_per_step": 3 * w.n_layers,
                                     "how": "h1b_decode_step_layers once per layer, one CUDA graph per step, replayed"}
     if rank == 0 and world == 1 and not args.no_cpu_baseline and w.name == "c2_7b_8k":
@@ -459,6 +469,9 @@ def main():
     ap.add_argument("--no-layer-sequential", action="store_true", help="skip the per-layer CUDA-graph measurement")
     ap.add_argument("--query-tokens", type=int, default=1,
                     help="> 1: each step appends this many tokens per sequence and attends for all of them (variant)")
+    ap.add_argument("--shard", default="sequences", choices=["sequences", "heads"],
+                    help="with N > 1 ranks: 'sequences' (default) = one independent sequence set per rank, weak scaling; "
+                         "'heads' = the ranks split the heads of the same sequences, strong scaling")
     ap.add_argument("--page-tokens", type=int, default=0,
                     help="> 0: a paged cache with pages of this many tokens, scattered over the pool (variant)")
     ap.add_argument("--fp16-values", action="store_true", help="keep values in fp16 (the 1-bit-keys-only ablation row)")
