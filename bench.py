@@ -477,7 +477,7 @@ def main():
     ap.add_argument("--fp16-values", action="store_true", help="keep values in fp16 (the 1-bit-keys-only ablation row)")
     ap.add_argument("--workload", default="c2_7b_8k",
                     choices=["c2_7b_8k", "c3_7b_batched", "c4_gqa_32k", "c5_prefill", "c6_60m_8k"],
-                    help="default: the configuration the metric is quoted on; the others are reported in DESIGN.md")
+                    help="default: the configuration the metric is quoted on; the others are variants and parity cases")
     args = ap.parse_args()
     if args.impl == "reference":
         run_reference(args)
