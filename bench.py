@@ -35,9 +35,9 @@ UNIT = "tokens/s"
 INV_TAU = 16.0
 # DRAM traffic of one decode_split_kernel launch (dram__bytes_read.sum + dram__bytes_write.sum) per
 # algorithmic byte, from the ncu capture summarised in profiles/decode_split_kernel_c2_7b_8k.md
-# (815.8 MB moved for 806.0 MB needed at 8199 cached tokens). Traffic grows in proportion to the cached
+# (816.5 MB moved for 806.0 MB needed at 8199 cached tokens). Traffic grows in proportion to the cached
 # tokens, so the bench scales it to the context it actually ran.
-NCU_TRAFFIC_PER_ALGORITHMIC_BYTE = 1.0122
+NCU_TRAFFIC_PER_ALGORITHMIC_BYTE = 1.0130
 
 
 def measured_peaks():
