@@ -66,7 +66,7 @@ typedef struct h1b_ctx h1b_ctx;   /* opaque, host-side */
 
 typedef struct {
     int32_t n_layers;      /* L >= 1                                                   */
-    int32_t n_q_heads;     /* Hq; Hq / Hkv must be 1, 2 or 4                           */
+    int32_t n_q_heads;     /* Hq; a multiple of Hkv, Hq / Hkv <= 16                    */
     int32_t n_kv_heads;    /* Hkv                                                      */
     int32_t head_dim;      /* d: 128, or 64 (then Hq == Hkv, even, G = 32, m <= 256)    */
     int32_t sketch_bits;   /* m: 64, 128, 256 or 512                                   */

@@ -22,6 +22,7 @@ namespace {
 constexpr long kTargetItems = 8192;   // decode work items aimed for (one warp each)
 constexpr int kMinSplitTokens = 256;
 constexpr int kMaxQueryTokens = H1B_MAX_QUERY_TOKENS;
+constexpr int kMaxGroupHeads = 16;        // query heads per KV head: the attention kernel takes them four at a time
 constexpr int kPrefillMinTokens = 64;   // appends of at least this many tokens per sequence take the tensor-core path
 
 struct Plan {
@@ -44,7 +45,7 @@ int check_config(const h1b_config *c) {
         return H1B_ERR_INVALID_ARG;
     if (c->max_batch > 256) return H1B_ERR_INVALID_ARG;
     const int gq = c->n_q_heads / c->n_kv_heads;
-    if (gq != 1 && gq != 2 && gq != 4) return H1B_ERR_UNSUPPORTED;
+    if (gq > kMaxGroupHeads) return H1B_ERR_UNSUPPORTED;
     if (c->sketch_bits != 64 && c->sketch_bits != 128 && c->sketch_bits != 256 && c->sketch_bits != 512)
         return H1B_ERR_UNSUPPORTED;
     if (c->head_dim == kHeadDim / 2) {
@@ -388,7 +389,15 @@ static int enqueue_decode(h1b_ctx *ctx, int layer_begin, int n_layers, float inv
     // (query token, query head) pairs that share a KV head, and how many of them one work item takes
     const int vheads = ctx->plan.gq * Tq, gqk = vheads >= 3 ? 4 : vheads, vgroups = (vheads + gqk - 1) / gqk;
     const size_t max_items = partial_bytes / ((size_t)gqk * kPartStride * sizeof(float));
-    const long slabs = (long)n_layers * B * ctx->cfg.n_kv_heads * vgroups;       // slabs x groups: units a split divides
+    // slabs x groups of virtual heads: the units a split divides. When the scratch cannot hold one partial for
+    // every unit of the call (many query tokens on a large batch), the layers go through it in several passes,
+    // one behind the other on the stream.
+    const long per_layer = (long)B * ctx->cfg.n_kv_heads * vgroups;
+    if ((size_t)per_layer > max_items)
+        return fail(ctx, H1B_ERR_CAPACITY, "%ld (sequence, KV head, head group) units of one layer exceed the split-K "
+                    "scratch (%zu items)", per_layer, max_items);
+    const int pass_layers = (int)std::min<size_t>((size_t)n_layers, max_items / (size_t)per_layer);
+    const long slabs = per_layer * pass_layers;
     int maxlen = 1;
     for (int l = layer_begin; l < layer_begin + n_layers; ++l)
         for (int b = 0; b < B; ++b) maxlen = std::max(maxlen, ctx->len_host[(size_t)l * ctx->cfg.max_batch + b]);
@@ -397,7 +406,7 @@ static int enqueue_decode(h1b_ctx *ctx, int layer_begin, int n_layers, float inv
     if (ctx->forced_splits <= 0 && splits > max_splits) splits = max_splits;
     if (splits < 1) splits = 1;
     if ((size_t)(slabs * splits) > max_items) {
-        if (ctx->forced_splits > 0 || (size_t)slabs > max_items)
+        if (ctx->forced_splits > 0)
             return fail(ctx, H1B_ERR_CAPACITY, "%ld splits of %ld slabs exceed the split-K scratch (%zu items)",
                         splits, slabs, max_items);
         splits = (long)(max_items / (size_t)slabs);
@@ -408,9 +417,8 @@ static int enqueue_decode(h1b_ctx *ctx, int layer_begin, int n_layers, float inv
     dp.len = at<int32_t>(ctx, ctx->plan.len);
     dp.qwords = qwords;
     dp.partial = partial;
-    dp.out = static_cast<float *>(out);
     dp.status = at<int32_t>(ctx, ctx->plan.status);
-    dp.layer_begin = layer_begin; dp.n_layers = n_layers; dp.B = B; dp.Hkv = ctx->cfg.n_kv_heads;
+    dp.B = B; dp.Hkv = ctx->cfg.n_kv_heads;
     dp.Hq = ctx->cfg.n_q_heads; dp.max_batch = ctx->cfg.max_batch; dp.m_words = ctx->plan.m_words;
     dp.groups = ctx->plan.groups;
     dp.splits = (int)splits;
@@ -419,12 +427,18 @@ static int enqueue_decode(h1b_ctx *ctx, int layer_begin, int n_layers, float inv
     dp.out_dim = ctx->ucfg.head_dim;
     dp.c2 = (float)(2.0 * (double)inv_tau * 1.4426950408889634 / (double)ctx->ucfg.sketch_bits);
     cudaEvent_t ev0 = nullptr, ev1 = nullptr;
-    if (may_profile && ctx->profiling && ctx->events_used + 2 <= ctx->events.size()) {
+    if (may_profile && pass_layers == n_layers && ctx->profiling && ctx->events_used + 2 <= ctx->events.size()) {
         ev0 = ctx->events[ctx->events_used];
         ev1 = ctx->events[ctx->events_used + 1];
         ctx->events_used += 2;
     }
-    H1B_CUDA(ctx, launch_decode(dp, st, launches, ev0, ev1));
+    const size_t layer_out = (size_t)B * Tq * ctx->cfg.n_q_heads * (size_t)ctx->ucfg.head_dim;   // floats of one layer
+    for (int done = 0; done < n_layers; done += pass_layers) {
+        dp.layer_begin = layer_begin + done;
+        dp.n_layers = std::min(pass_layers, n_layers - done);
+        dp.out = static_cast<float *>(out) + (size_t)done * layer_out;
+        H1B_CUDA(ctx, launch_decode(dp, st, launches, ev0, ev1));
+    }
     return H1B_OK;
 }
 
@@ -603,7 +617,8 @@ int h1b_decode_attention_static(h1b_ctx *ctx, int layer_begin, int n_layers, con
     const long slabs = (long)n_layers * B * ctx->cfg.n_kv_heads;
     const size_t qw_bytes = align_up((size_t)ctx->cfg.n_layers * ctx->cfg.max_batch * ctx->cfg.n_q_heads *
                                          ctx->plan.m_words * sizeof(uint32_t), 256);
-    const size_t item_bytes = (size_t)ctx->plan.gq * kPartStride * sizeof(float);
+    const int gqk = ctx->plan.gq >= 3 ? 4 : ctx->plan.gq, vgroups = (ctx->plan.gq + gqk - 1) / gqk;
+    const size_t item_bytes = (size_t)vgroups * gqk * kPartStride * sizeof(float);
     const size_t need = qw_bytes + (size_t)slabs * item_bytes;
     if (need > H1B_STATIC_SCRATCH_BYTES)
         return fail(ctx, H1B_ERR_CAPACITY,
@@ -859,7 +874,7 @@ int h1b_set_block_table(h1b_ctx *ctx, int seq, const int32_t *pages_host, int n,
 
 int h1b_set_splits(h1b_ctx *ctx, int splits) {
     if (!ctx) return H1B_ERR_NULL;
-    const size_t most = ctx->plan.partial_bytes / ((size_t)ctx->plan.gq * kPartStride * sizeof(float));
+    const size_t most = ctx->plan.partial_bytes / ((size_t)std::min(ctx->plan.gq, 4) * kPartStride * sizeof(float));
     if (splits < 0 || (size_t)splits > most)
         return fail(ctx, H1B_ERR_INVALID_ARG, "splits %d outside [0, %zu]", splits, most);
     ctx->forced_splits = splits;

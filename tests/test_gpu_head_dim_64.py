@@ -49,16 +49,28 @@ def test_fp16_values():
     out = cache.h1b_decode_attention(q.cuda(), 16.0).cpu().numpy()
     cache.h1b_poll_status()
     assert out.shape == (w.n_layers, w.batch, w.n_q_heads, 64)
+    checked = end_to_end = 0
     for l in range(w.n_layers):
         ref = oracle.layer_fp16_values(f16_bits(K[l]), f16_bits(V[l]), lens, f16_bits(q[l]), Rt[l], 16.0)
         for b in range(w.batch):
             for h in range(w.n_kv_heads):
                 n = int(lens[b])
                 assert np.array_equal(cache.h1b_export_values(l, b, h, 0, n), f16_bits(V[l, b, :n, h]))
-                words = cache.h1b_export_cache(l, b, h, 0, n)[0]
-                obits = oracle.sketch(f16_bits(K[l, b, :n, h]), Rt[l])[0]
-                if np.array_equal(binding.unpack_words(words, w.sketch_bits), obits):
+                vals = cache.h1b_export_values(l, b, h, 0, n)
+                kbits = binding.unpack_words(cache.h1b_export_cache(l, b, h, 0, n)[0], w.sketch_bits)
+                qwords, gscore = cache.h1b_debug_scores(l, b, h, q[l, b, h].contiguous().cuda(), n)
+                qbits = binding.unpack_words(qwords[None], w.sketch_bits)[0]
+                assert np.array_equal(gscore[:n], oracle.scores(qbits, kbits))
+                iso = oracle.attention_fp16_values(gscore[:n], w.sketch_bits, 16.0, vals)
+                check_output(out[l, b, h], iso, ("fp16 values, d = 64, isolated", l, b, h))
+                obits = oracle.sketch(f16_bits(K[l, b, :n, h]), Rt[l])
+                oq = oracle.sketch(f16_bits(q[l, b, h])[None], Rt[l])[0]
+                checked += 1
+                if np.array_equal(kbits, obits) and np.array_equal(qbits, oq):
                     check_output(out[l, b, h], ref[b, h], ("fp16 values, d = 64", l, b, h))
+                    end_to_end += 1
+    print("fp16 values, d = 64: units", checked, "of which end to end", end_to_end)
+    assert end_to_end > 0
     cache.close()
 
 

@@ -79,7 +79,8 @@ def _check(w, cache, Rt, K, V, q, lens, out, inv_tau, fp16_values):
 
 
 @pytest.mark.parametrize("hq, hkv, Tq", [(1, 1, 1), (1, 1, 2), (1, 1, 3), (1, 1, 4), (1, 1, 7), (2, 2, 16),
-                                         (4, 2, 3), (4, 2, 8), (4, 1, 2), (4, 1, 5), (8, 2, 16)])
+                                         (4, 2, 3), (4, 2, 8), (4, 1, 2), (4, 1, 5), (8, 2, 16),
+                                         (8, 1, 2), (7, 1, 3), (6, 2, 16), (16, 1, 16)])
 def test_head_group_shapes_and_query_counts(hq, hkv, Tq):
     w = h1b_synth.scaled(W["c1_tiny"], batch=2, n_layers=2, n_q_heads=hq, n_kv_heads=hkv)
     cache, Rt, K, V, lens = _fill(w, [333, 64])
@@ -164,4 +165,31 @@ def test_7b_shape_sampled_units():
             ref = oracle.attention(gscore[:n_i], w.sketch_bits, 16.0, codes[:n_i], scale[:n_i], zero[:n_i], w.group_size)
             check_output(out[l, b, i, g], ref, ("7B shape", l, b, g, i))
         assert np.array_equal(gscore[:n], oracle.scores(binding.unpack_words(qwords[None], w.sketch_bits)[0], kbits))
+    cache.close()
+
+
+def test_more_units_than_the_scratch_holds_run_in_layer_passes():
+    """40 layers x 4 sequences x 4 KV heads x 16 groups of four (query token, head) pairs = 10 240 units: more
+    than the split-K scratch holds at once, so the call walks the layers in passes. Bit for bit the same as the
+    same layers asked for eight at a time, and a sample of heads against the oracle."""
+    w = h1b_synth.scaled(W["c1_tiny"], n_layers=40, batch=4, n_q_heads=16, n_kv_heads=4)
+    cache, Rt, K, V, lens = _fill(w, [70, 40, 33, 16])
+    Tq = 16
+    q = _queries(w, Tq, seed=5)
+    qd = q.cuda()
+    out = cache.h1b_decode_attention_multi(qd, 16.0).cpu().numpy()
+    cache.h1b_poll_status()
+    for l0 in range(0, w.n_layers, 8):
+        part = cache.h1b_decode_attention_multi(qd[l0:l0 + 8].contiguous(), 16.0, layer_begin=l0).cpu().numpy()
+        assert np.array_equal(part, out[l0:l0 + 8]), l0
+    for (l, b, g, i, hh) in [(0, 0, 0, 0, 0), (31, 3, 3, 15, 3), (32, 0, 1, 7, 2), (39, 2, 2, 3, 1), (39, 3, 0, 0, 0)]:
+        n = int(lens[b])
+        n_i = n - Tq + i + 1
+        h = g * 4 + hh
+        words, codes, scale, zero = cache.h1b_export_cache(l, b, g, 0, n)
+        kbits = binding.unpack_words(words, w.sketch_bits)
+        qwords, gscore = cache.h1b_debug_scores(l, b, g, q[l, b, i, h].contiguous().cuda(), n)
+        assert np.array_equal(gscore[:n], oracle.scores(binding.unpack_words(qwords[None], w.sketch_bits)[0], kbits))
+        ref = oracle.attention(gscore[:n_i], w.sketch_bits, 16.0, codes[:n_i], scale[:n_i], zero[:n_i], w.group_size)
+        check_output(out[l, b, i, h], ref, ("layer passes", l, b, i, h))
     cache.close()

@@ -32,7 +32,8 @@ def test_incremental_and_ragged_appends_three_sequences():
     print("ragged", tot)
 
 
-@pytest.mark.parametrize("hq,hkv,m", [(8, 2, 256), (4, 2, 64), (2, 2, 512), (8, 2, 128), (4, 1, 64)])
+@pytest.mark.parametrize("hq,hkv,m", [(8, 2, 256), (4, 2, 64), (2, 2, 512), (8, 2, 128), (4, 1, 64),
+                                      (8, 1, 128), (3, 1, 128), (14, 2, 64), (12, 2, 256), (16, 1, 512), (5, 1, 128)])
 def test_gqa_and_sketch_widths(hq, hkv, m):
     w = small("c4_gqa_32k", n_layers=1, n_q_heads=hq, n_kv_heads=hkv, sketch_bits=m, batch=2, context=333)
     tot = full_parity(w, [333, 120])

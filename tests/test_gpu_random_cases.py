@@ -1,0 +1,40 @@
+"""GPU parity on generated cases (hypothesis, derandomised so that every run draws the same cases): head
+shapes, sketch widths, group sizes, ragged lengths, the way the rows arrive (one call, many calls, single
+tokens), forced split counts and temperatures, each checked by the full protocol (append bit for bit outside
+the decision window, isolated decode, end to end) against the fp64 oracle."""
+import numpy as np
+import pytest
+from hypothesis import HealthCheck, given, settings, strategies as st
+
+import h1b_synth
+from h1b_testlib import full_parity
+
+pytestmark = pytest.mark.gpu
+W = h1b_synth.WORKLOADS
+
+SHAPES = [(1, 1), (2, 2), (4, 4), (2, 1), (4, 1), (4, 2), (8, 2), (8, 4), (8, 1), (7, 1), (6, 2), (3, 1)]       # (query heads, kv heads)
+FORMATS = [(64, 32), (64, 128), (128, 32), (128, 128), (256, 32), (256, 128), (512, 32)]   # (sketch bits m, group size G)
+
+
+@st.composite
+def cases(draw):
+    hq, hkv = draw(st.sampled_from(SHAPES))
+    m, G = draw(st.sampled_from(FORMATS))
+    batch = draw(st.integers(1, 3))
+    lens = [draw(st.one_of(st.integers(0, 40), st.integers(0, 700))) for _ in range(batch)]
+    pieces = draw(st.lists(st.sampled_from([1, 2, 3, 15, 16, 17, 31, 32, 33, 64, 65, 100, 257]), min_size=0, max_size=6))
+    pieces.append(max(max(lens), 1))                              # whatever is left arrives in one last call
+    splits = draw(st.sampled_from([0, 0, 1, 2, 3, 5, 8, 23, 64]))
+    inv_tau = draw(st.sampled_from([1e-3, 1.0, 16.0, 50.0, 400.0]))
+    return hq, hkv, m, G, batch, lens, pieces, splits, inv_tau
+
+
+@settings(max_examples=30, deadline=None, derandomize=True, database=None,
+          suppress_health_check=list(HealthCheck))
+@given(case=cases())
+def test_generated_cases(case):
+    hq, hkv, m, G, batch, lens, pieces, splits, inv_tau = case
+    w = h1b_synth.scaled(W["c1_tiny"], batch=batch, n_layers=2, n_q_heads=hq, n_kv_heads=hkv, sketch_bits=m,
+                         group_size=G)
+    tot = full_parity(w, lens, inv_tau=inv_tau, appends=pieces, splits=splits)
+    print("generated", case, tot)
