@@ -49,6 +49,8 @@ def _load():
             lib.h1bo_half_to_double.argtypes = [ctypes.c_uint16]
             lib.h1bo_double_to_half_rne.restype = ctypes.c_uint16
             lib.h1bo_double_to_half_rne.argtypes = [ctypes.c_double]
+            lib.h1bo_rope.restype = None
+            lib.h1bo_rope.argtypes = [u16p, ctypes.c_long, ctypes.c_int, f32p, i32p, u16p]
             lib.h1bo_sketch.restype = None
             lib.h1bo_sketch.argtypes = [u16p, ctypes.c_long, ctypes.c_int, ctypes.c_int, f32p,
                                         u8p, f64p, f64p]
@@ -103,6 +105,21 @@ def half_to_double(bits: int) -> float:
 
 def double_to_half_rne(x: float) -> int:
     return int(_load().h1bo_double_to_half_rne(float(x)))
+
+
+def rope(x, table, pos):
+    """Rotary position embedding (half-split pairs) of rows ``x`` [rows, d] (fp16) at positions ``pos`` [rows] with
+    ``table`` [n_pos, d/2, 2] (fp32 cos, sin). Returns the rotated rows as fp16 bit patterns, uint16 [rows, d]."""
+    xb = _as_u16(x)
+    rows, d = xb.shape
+    table = np.ascontiguousarray(table, dtype=np.float32)
+    pos = np.ascontiguousarray(pos, dtype=np.int32)
+    assert table.ndim == 3 and table.shape[1:] == (d // 2, 2) and pos.shape == (rows,)
+    assert rows == 0 or (pos.min() >= 0 and pos.max() < table.shape[0])
+    out = np.empty((rows, d), dtype=np.uint16)
+    _load().h1bo_rope(_ptr(xb, ctypes.c_uint16), rows, d, _ptr(table, ctypes.c_float), _ptr(pos, ctypes.c_int32),
+                      _ptr(out, ctypes.c_uint16))
+    return out
 
 
 def sketch(x, Rt, want_margin: bool = False):

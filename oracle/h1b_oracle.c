@@ -31,12 +31,18 @@
  *   - Delta16 == 0 gives all-zero codes; codes are clamped to [0, 15].
  *   - alpha_t = (m - 2*Hamming)/m, no 1/sqrt(d), no unbiasing.
  *   - every cached token t in [0, len) is attended; len == 0 gives zeros.
+ *   - optional rotary position embedding of the rows that enter Eq. 2 (a
+ *     neighbour of the path, not an equation of the paper): half-split pairs,
+ *     angles from a caller's table, binary32 arithmetic in a stated order, one
+ *     rounding to binary16 (h1bo_rope).
  *
  * Pins (tests, CPU only): the +-1 inner product equals m - 2*Hamming (proof of
  * Prop. 1); bit agreement rate tracks 1 - theta/pi (Eq. 1); round trip error
  * <= Delta/2; T = 1, equal keys, tau -> infinity and tau -> 0 limits; a
  * lossless 16-level grid reduces Eq. 5 to a library softmax @ V; hand-worked
- * tiny cases; the fp16-value variant reduces to a library softmax @ V directly.
+ * tiny cases; the fp16-value variant reduces to a library softmax @ V directly;
+ * the rotation against a complex multiplication in fp64, position 0 as the
+ * identity, norm preservation and the relative-position property.
  * Parity unpinned (conventions of this build, nothing in the
  * paper fixes them): the min/max rule for Delta and zero, round-half-to-even,
  * and the value of tau.
@@ -95,6 +101,39 @@ uint16_t h1bo_double_to_half_rne(double x)
         return (uint16_t)(sign | (uint16_t)ri);
     }
     return (uint16_t)(sign | (uint16_t)((e + 15) << 10) | (uint16_t)(ri - 1024));
+}
+
+/* ------------------------------------------------------------------------ */
+/* Rotary position embedding of key or query rows before Eq. 2 (the keys a     */
+/* Llama-style model caches are the rotated ones). Not an equation of the      */
+/* paper: the rotation is the model's; the convention here is the half-split   */
+/* one (channel i pairs with channel i + d/2) with the angles handed in as a   */
+/* table, so no transcendental function is evaluated on either side.           */
+/*   x      [rows][d]        binary16 bit patterns                              */
+/*   table  [n_pos][d/2][2]  float32 (cos, sin) of position p, pair i           */
+/*   pos    [rows]           position of each row                               */
+/*   out    [rows][d]        binary16: x_i' = x_i c - x_{i+d/2} s,              */
+/*                                     x_{i+d/2}' = x_{i+d/2} c + x_i s         */
+/* The result is rounded to binary16, and that rounding is a decision every     */
+/* later step depends on, so it is taken in one stated precision: each product  */
+/* and the sum are rounded to binary32 (no fused multiply-add), then the sum    */
+/* is rounded once to binary16, to nearest even.                                */
+/* ------------------------------------------------------------------------ */
+void h1bo_rope(const uint16_t *x, long rows, int d, const float *table, const int32_t *pos, uint16_t *out)
+{
+    const int hw = d / 2;
+    for (long r = 0; r < rows; ++r) {
+        const float *t = table + (size_t)pos[r] * hw * 2;
+        for (int i = 0; i < hw; ++i) {
+            const float a = (float)h1bo_half_to_double(x[r * d + i]);          /* exact */
+            const float b = (float)h1bo_half_to_double(x[r * d + i + hw]);
+            const float c = t[2 * i], s = t[2 * i + 1];
+            volatile float ac = a * c, bs = b * s, bc = b * c, as = a * s;     /* each rounded to binary32 */
+            volatile float lo = ac - bs, hi = bc + as;
+            out[r * d + i] = h1bo_double_to_half_rne((double)lo);
+            out[r * d + i + hw] = h1bo_double_to_half_rne((double)hi);
+        }
+    }
 }
 
 /* ------------------------------------------------------------------------ */
