@@ -132,6 +132,8 @@ def run_ours(args):
                              name="%s[m=%d,G=%d]" % (w.name, args.sketch_bits or w.sketch_bits, args.group_size or w.group_size))
     if args.fp16_values:                              # Table V's "1-bit keys only" row: values stay fp16
         w = h1b_synth.scaled(w, name=w.name + "[fp16 values]")
+    if args.rope:                                     # rotary embedding fused into the append and the query sketch
+        w = h1b_synth.scaled(w, name=w.name + "[rope]")
     if args.workload == "c5_prefill":
         return run_prefill(args, w, pdist, rank, world, local)
     # --shard heads: the ranks split the KV heads (and their query heads) of the SAME sequences between them: every
@@ -156,12 +158,15 @@ def run_ours(args):
         w = h1b_synth.scaled(w, name=w.name + "[pages of %d tokens]" % page_tokens)
     cfg = binding.make_config(w.n_layers, w.n_q_heads, w.n_kv_heads, w.head_dim, w.sketch_bits, w.group_size,
                               max_batch=w.batch, max_seq=w.context - 1 + total_steps, device=local,
-                              fp16_values=args.fp16_values, page_tokens=page_tokens, n_pages=pages_per_seq * w.batch)
+                              fp16_values=args.fp16_values, page_tokens=page_tokens, n_pages=pages_per_seq * w.batch,
+                              rope=args.rope)
     # each rank is its own sequence: different seeds per rank
     wr = h1b_synth.scaled(w, index=w.index + 10 * rank)
     Rt = np.stack([h1b_synth.projection(h1b_synth.layer_seed(wr, l, 99), w.head_dim, w.sketch_bits)
                    for l in range(w.n_layers)])
     cache = binding.H1BCache(cfg, Rt=Rt)
+    if args.rope:
+        cache.h1b_set_rope_table(h1b_synth.rope_table(w.context - 1 + total_steps, w.head_dim // 2))
     if page_tokens:                                   # every sequence gets a seeded, scattered set of pool pages
         perm = np.random.default_rng(7 + rank).permutation(pages_per_seq * w.batch)
         for b in range(w.batch):
@@ -341,8 +346,11 @@ def run_prefill(args, w, pdist, rank, world, local):
     from paper_2510_05529_b200 import binding
     dev = torch.device("cuda", local)
     cfg = binding.make_config(w.n_layers, w.n_q_heads, w.n_kv_heads, w.head_dim, w.sketch_bits, w.group_size,
-                              max_batch=w.batch, max_seq=w.context, device=local, fp16_values=args.fp16_values)
+                              max_batch=w.batch, max_seq=w.context, device=local, fp16_values=args.fp16_values,
+                              rope=args.rope)
     cache = binding.H1BCache(cfg, seed=11 + rank)
+    if args.rope:
+        cache.h1b_set_rope_table(h1b_synth.rope_table(w.context, w.head_dim // 2))
     K = torch.stack([h1b_synth.kv_rows(w, l, w.context, device=str(dev))[0] for l in range(w.n_layers)])
     V = torch.stack([h1b_synth.kv_rows(w, l, w.context, device=str(dev))[1] for l in range(w.n_layers)])
     stream = torch.cuda.current_stream()
@@ -474,6 +482,8 @@ def main():
                          "'heads' = the ranks split the heads of the same sequences, strong scaling")
     ap.add_argument("--page-tokens", type=int, default=0,
                     help="> 0: a paged cache with pages of this many tokens, scattered over the pool (variant)")
+    ap.add_argument("--rope", action="store_true",
+                    help="rotate keys and queries (rotary position embedding) inside the append and the query sketch (variant)")
     ap.add_argument("--fp16-values", action="store_true", help="keep values in fp16 (the 1-bit-keys-only ablation row)")
     ap.add_argument("--workload", default="c2_7b_8k",
                     choices=["c2_7b_8k", "c3_7b_batched", "c4_gqa_32k", "c5_prefill", "c6_60m_8k"],

@@ -111,6 +111,13 @@ def queries(w: Workload, layer: int, device: str = "cpu", stream: int = 0, batch
     return normal_fp16(layer_seed(w, layer, 7001 + stream), (B, w.n_q_heads, w.head_dim), device)
 
 
+def rope_table(n_positions: int, half: int, base: float = 10000.0) -> np.ndarray:
+    """Input data for the rotary-embedding option: fp32 [n_positions, half, 2], (cos, sin) of the angle
+    position * base^(-i / half) of pair i (the usual geometric frequencies), evaluated in fp64 and rounded once."""
+    ang = np.arange(n_positions, dtype=np.float64)[:, None] * base ** (-np.arange(half, dtype=np.float64) / half)[None, :]
+    return np.stack([np.cos(ang), np.sin(ang)], axis=-1).astype(np.float32)
+
+
 def lengths(w: Workload, batch: int | None = None) -> np.ndarray:
     """Cached tokens per sequence: constant, or uniform in [context_min, context]."""
     B = w.batch if batch is None else batch

@@ -84,6 +84,20 @@ typedef struct {
  * supported value but is not used. */
 #define H1B_FLAG_FP16_VALUES 1u
 
+/* Rotary position embedding fused into the path (not a step of the paper's
+ * method: the rotation belongs to the model, and a Llama-style model caches
+ * the rotated keys; fusing it saves the model a pass over K and q). With this
+ * flag the key rows of an append are rotated at their cache positions and the
+ * query rows of a decode call at the position of their token (the sequence's
+ * last, or with Tq query tokens its last Tq) before Eq. 2; values are not
+ * touched. Pairs are (channel i, channel i + d/2) of a head:
+ *     x_i' = x_i c - x_{i+d/2} s,   x_{i+d/2}' = x_{i+d/2} c + x_i s,
+ * (c, s) = table[position][i]. Each product and the sum are rounded to fp32
+ * (no fused multiply-add) and the result once to fp16, to nearest even: the
+ * rotated row is the same fp16 bits in every kernel.
+ * h1b_set_rope_table must be called before the first append or decode. */
+#define H1B_FLAG_ROPE 2u
+
 /* Bytes of one cached token of one KV head: m/8 + d/2 + (d/G)*4 (Section IV-B
  * storage statement plus the fp16 scale and zero per group); m/8 + 2d with
  * H1B_FLAG_FP16_VALUES. 0 if invalid. */
@@ -106,6 +120,14 @@ size_t h1b_entry_bytes(const h1b_config *cfg /* HOST */);
  * H1B_ERR_INVALID_ARG on a contiguous cache, on bad page numbers, or when fewer
  * pages than the sequence's cached tokens need. */
 int h1b_set_block_table(h1b_ctx *ctx, int seq, const int32_t *pages_host, int n, void *stream);
+
+/* Rotary table (H1B_FLAG_ROPE): cos_sin_host is HOST fp32 [n_positions][d/2][2],
+ * (cos, sin) of the angle of pair i at each position, copied into the workspace
+ * (synchronous: returns when the copy is done). n_positions >= 1; positions
+ * from max_seq (rounded up to 32) on are not kept. A call that would reach a position the table does not hold
+ * fails with H1B_ERR_CAPACITY (a replayed graph: the position is clamped to the
+ * table's last). H1B_ERR_INVALID_ARG if the cache was made without the flag. */
+int h1b_set_rope_table(h1b_ctx *ctx, const float *cos_sin_host, int n_positions, void *stream);
 
 /* Bytes of device workspace the caller must provide for this configuration
  * (projection matrices, lengths, split-K scratch, staging and the packed cache

@@ -71,6 +71,7 @@ def load_library(rebuild: bool = True) -> ctypes.CDLL:
                                                   ctypes.c_int, vp]),
         "h1b_sync_lengths": (ctypes.c_int, [vp, vp]),
         "h1b_set_block_table": (ctypes.c_int, [vp, ctypes.c_int, i32p, ctypes.c_int, vp]),
+        "h1b_set_rope_table": (ctypes.c_int, [vp, vp, ctypes.c_int, vp]),
         "h1b_decode_step_host": (ctypes.c_int, [vp, vp, vp, vp, ctypes.c_float, vp, ctypes.c_int, vp]),
         "h1b_free": (ctypes.c_int, [vp]),
         "h1b_get_projection": (ctypes.c_int, [vp, ctypes.c_int, vp]),
@@ -97,13 +98,16 @@ def load_library(rebuild: bool = True) -> ctypes.CDLL:
 
 
 H1B_FLAG_FP16_VALUES = 1      # h1b_config.flags: values stay fp16 (the 1-bit-keys-only configuration)
+H1B_FLAG_ROPE = 2             # keys and queries are rotated (rotary position embedding) before they are sketched
 
 
 def make_config(n_layers, n_q_heads, n_kv_heads, head_dim=128, sketch_bits=128, group_size=32,
-                max_batch=1, max_seq=8192, device=0, fp16_values=False, page_tokens=0, n_pages=0) -> h1b_config:
+                max_batch=1, max_seq=8192, device=0, fp16_values=False, page_tokens=0, n_pages=0,
+                rope=False) -> h1b_config:
     """page_tokens > 0: a paged cache with n_pages pages of that many tokens in each layer's pool."""
+    flags = (H1B_FLAG_FP16_VALUES if fp16_values else 0) | (H1B_FLAG_ROPE if rope else 0)
     return h1b_config(n_layers, n_q_heads, n_kv_heads, head_dim, sketch_bits, group_size,
-                      max_batch, max_seq, device, H1B_FLAG_FP16_VALUES if fp16_values else 0, page_tokens, n_pages)
+                      max_batch, max_seq, device, flags, page_tokens, n_pages)
 
 
 def h1b_entry_bytes(cfg: h1b_config) -> int:
@@ -251,6 +255,13 @@ class H1BCache:
         arr = np.ascontiguousarray(pages, dtype=np.int32)
         self._check(self.lib.h1b_set_block_table(self._h, seq, arr.ctypes.data_as(ctypes.POINTER(ctypes.c_int32)),
                                                  int(arr.size), _stream_ptr(stream)))
+
+    def h1b_set_rope_table(self, cos_sin, stream=None):
+        """Rotary table: cos_sin fp32 [n_positions, d/2, 2] (numpy or CPU tensor), (cos, sin) per position and pair."""
+        arr = np.ascontiguousarray(cos_sin.numpy() if isinstance(cos_sin, torch.Tensor) else cos_sin, dtype=np.float32)
+        if arr.ndim != 3 or arr.shape[1:] != (self.cfg.head_dim // 2, 2):
+            raise ValueError("cos_sin must be [n_positions, d/2, 2]")
+        self._check(self.lib.h1b_set_rope_table(self._h, arr.ctypes.data, int(arr.shape[0]), _stream_ptr(stream)))
 
     def h1b_sync_lengths(self, stream=None):
         """After replaying a captured graph that appends: refresh the host's copy of the lengths."""

@@ -28,6 +28,7 @@ constexpr int kPrefillMinTokens = 64;   // appends of at least this many tokens 
 struct Plan {
     size_t rt, rh, len, status, qwords, partial, stage_k, stage_v, stage_q, stage_out, dbg_q, dbg_row, dbg_s, cache, total;
     size_t partial_bytes, slab_bytes;
+    size_t rope;                            // rotary table [cap_tokens][head_dim / 2][2] fp32 (H1B_FLAG_ROPE only)
     size_t table, seq_cap, layer_bytes;     // paged cache: block tables [max_batch][table_stride], capacities [max_batch]
     int table_stride, page_chunks;          // 0 when the cache is contiguous
     int cap_tokens, m_words, gq, groups;
@@ -39,7 +40,7 @@ int check_config(const h1b_config *c) {
     if (!c) return H1B_ERR_NULL;
     if (c->n_layers < 1 || c->n_q_heads < 1 || c->n_kv_heads < 1 || c->max_batch < 1 || c->max_seq < 1 ||
         c->head_dim < 1 || c->sketch_bits < 1 || c->group_size < 1 || c->device < 0 ||
-        (c->flags & ~H1B_FLAG_FP16_VALUES) != 0)
+        (c->flags & ~(H1B_FLAG_FP16_VALUES | H1B_FLAG_ROPE)) != 0)
         return H1B_ERR_INVALID_ARG;
     if (c->n_q_heads % c->n_kv_heads != 0 || c->head_dim % c->group_size != 0 || c->sketch_bits % 32 != 0)
         return H1B_ERR_INVALID_ARG;
@@ -114,6 +115,7 @@ int make_plan(const h1b_config *user, Plan *p) {
     p->dbg_s = take((size_t)p->cap_tokens * sizeof(int32_t));
     p->table = take((size_t)c->max_batch * (p->table_stride ? p->table_stride : 1) * sizeof(int32_t));
     p->seq_cap = take((size_t)c->max_batch * sizeof(int32_t));
+    p->rope = take((c->flags & H1B_FLAG_ROPE) ? (size_t)p->cap_tokens * (user->head_dim / 2) * 2 * sizeof(float) : 0);
     p->cache = take(c->page_tokens > 0 ? L * p->layer_bytes : slabs * p->slab_bytes);
     p->total = o;
     return H1B_OK;
@@ -151,6 +153,7 @@ struct h1b_ctx {
     std::vector<int32_t> len_host;     // [L][max_batch], mirror of the device lengths
     std::vector<int32_t> table_host;   // paged cache: mirror of the block tables [max_batch][table_stride], -1 = none
     std::vector<int32_t> cap_host;     // tokens each sequence has room for (max_seq, or what its pages hold)
+    int rope_positions;                // positions the rotary table holds (0: not set yet)
     int forced_splits;
     int64_t launches;
     bool profiling;
@@ -262,6 +265,7 @@ int h1b_init_projection(const h1b_config *cfg, uint64_t seed, const float *Rt_ho
     ctx->table_host.assign((size_t)cfg->max_batch * (plan.table_stride ? plan.table_stride : 1), -1);
     ctx->cap_host.assign((size_t)cfg->max_batch, plan.page_chunks ? 0 : cfg->max_seq);
     ctx->forced_splits = 0;
+    ctx->rope_positions = 0;
     ctx->launches = 0;
     ctx->profiling = false;
     ctx->events_used = 0;
@@ -328,6 +332,7 @@ int h1b_init_projection(const h1b_config *cfg, uint64_t seed, const float *Rt_ho
 // ---------------------------------------------------------------------------
 // Shared pieces of append, decode and step (static: not part of the ABI).
 // ---------------------------------------------------------------------------
+static int check_rope(h1b_ctx *ctx, int layer_begin, int n_layers, int B, const NewCounts *nn);
 static int make_new_counts(h1b_ctx *ctx, int layer_begin, int n_layers, const int32_t *n_new_host, int B, int Tn,
                            NewCounts *nn) {
     std::memset(nn, 0, sizeof *nn);
@@ -341,6 +346,28 @@ static int make_new_counts(h1b_ctx *ctx, int layer_begin, int n_layers, const in
             if ((long)ctx->len_host[(size_t)l * ctx->cfg.max_batch + b] + nn->v[b] > ctx->cap_host[b])
                 return fail(ctx, H1B_ERR_CAPACITY, "layer %d sequence %d: %d + %d tokens exceed its capacity of %d", l, b,
                             ctx->len_host[(size_t)l * ctx->cfg.max_batch + b], nn->v[b], ctx->cap_host[b]);
+    return check_rope(ctx, layer_begin, n_layers, B, nn);
+}
+
+static bool uses_rope(const h1b_ctx *ctx) { return (ctx->ucfg.flags & H1B_FLAG_ROPE) != 0; }
+static RopeRef rope_ref(h1b_ctx *ctx) {
+    RopeRef r;
+    r.table = uses_rope(ctx) ? at<float>(ctx, ctx->plan.rope) : nullptr;
+    r.half = ctx->ucfg.head_dim / 2;
+    r.n_pos = ctx->rope_positions;
+    return r;
+}
+// With rotary embedding every position that a call touches must be in the table.
+static int check_rope(h1b_ctx *ctx, int layer_begin, int n_layers, int B, const NewCounts *nn) {
+    if (!uses_rope(ctx)) return H1B_OK;
+    if (ctx->rope_positions < 1) return fail(ctx, H1B_ERR_INVALID_ARG, "H1B_FLAG_ROPE: h1b_set_rope_table has not been called");
+    for (int l = layer_begin; l < layer_begin + n_layers; ++l)
+        for (int b = 0; b < B; ++b) {
+            const int end = ctx->len_host[(size_t)l * ctx->cfg.max_batch + b] + (nn ? nn->v[b] : 0);
+            if (end > ctx->rope_positions)
+                return fail(ctx, H1B_ERR_CAPACITY, "layer %d sequence %d reaches position %d, the rotary table holds %d",
+                            l, b, end, ctx->rope_positions);
+        }
     return H1B_OK;
 }
 
@@ -358,6 +385,7 @@ static AppendParams append_params(h1b_ctx *ctx, int layer_begin, int n_layers, c
     p.layer_begin = layer_begin; p.n_layers = n_layers; p.B = B; p.Tn = Tn;
     p.Hkv = ctx->cfg.n_kv_heads; p.max_batch = ctx->cfg.max_batch; p.m_words = ctx->plan.m_words;
     p.groups = ctx->plan.groups;
+    p.rope = rope_ref(ctx);
     return p;
 }
 
@@ -371,6 +399,9 @@ static SketchParams sketch_params(h1b_ctx *ctx, int layer_begin, int n_layers, c
     sp.layer_begin = layer_begin; sp.n_layers = n_layers; sp.B = B;
     sp.Hq = ctx->paired ? ctx->cfg.n_q_heads / 2 : ctx->cfg.n_q_heads;
     sp.max_batch = ctx->cfg.max_batch; sp.m_words = ctx->plan.m_words;
+    sp.rope = rope_ref(ctx);
+    sp.len = at<int32_t>(ctx, ctx->plan.len);
+    sp.Tq = 1;
     return sp;
 }
 
@@ -449,7 +480,7 @@ static int check_decode_args(h1b_ctx *ctx, int layer_begin, int n_layers, const 
     if (!q || !out) return fail(ctx, H1B_ERR_NULL, "q or out is NULL");
     if (!(inv_tau > 0.f) || !std::isfinite(inv_tau))
         return fail(ctx, H1B_ERR_INVALID_ARG, "inv_tau must be finite and > 0");
-    return H1B_OK;
+    return check_rope(ctx, layer_begin, n_layers, B, nullptr);
 }
 
 int h1b_append_kv(h1b_ctx *ctx, int layer_begin, int n_layers, const void *k, const void *v,
@@ -470,6 +501,7 @@ int h1b_append_kv(h1b_ctx *ctx, int layer_begin, int n_layers, const void *k, co
         pp.Rh = at<uint16_t>(ctx, ctx->plan.rh);
         pp.ca = cache_addr(ctx);
         pp.seq_cap = at<int32_t>(ctx, ctx->plan.seq_cap);
+        pp.rope = rope_ref(ctx);
         pp.len = at<int32_t>(ctx, ctx->plan.len);
         pp.status = at<int32_t>(ctx, ctx->plan.status);
         pp.done = at<int32_t>(ctx, ctx->plan.status) + 4;
@@ -533,6 +565,7 @@ int h1b_decode_attention_multi(h1b_ctx *ctx, int layer_begin, int n_layers, cons
     // rows of the sketch are (sequence, query token, query head): Tq * Hq "heads" per sequence
     SketchParams sp = sketch_params(ctx, layer_begin, n_layers, q, B, at<uint32_t>(ctx, ctx->plan.qwords));
     sp.Hq = Tq * ctx->cfg.n_q_heads;
+    sp.Tq = Tq;
     NewCounts none;
     std::memset(&none, 0, sizeof none);
     H1B_CUDA(ctx, launch_prepare(nullptr, &sp, none, st, &launches));
@@ -829,6 +862,12 @@ int h1b_debug_scores(h1b_ctx *ctx, int layer, int seq, int kv_head, const void *
     sp.Rt = at<float>(ctx, ctx->plan.rt) + (size_t)layer * ctx->cfg.head_dim * ctx->cfg.sketch_bits;
     sp.qwords = at<uint32_t>(ctx, ctx->plan.dbg_q);
     sp.layer_begin = 0; sp.n_layers = 1; sp.B = 1; sp.Hq = 1; sp.max_batch = 1; sp.m_words = mw;
+    // with rotary embedding the row is turned like the query of a decode call: at the sequence's last position
+    sp.rope = rope_ref(ctx);
+    sp.len = at<int32_t>(ctx, ctx->plan.len) + (size_t)layer * ctx->cfg.max_batch + seq;
+    sp.Tq = 1;
+    if (uses_rope(ctx) && ctx->rope_positions < 1)
+        return fail(ctx, H1B_ERR_INVALID_ARG, "H1B_FLAG_ROPE: h1b_set_rope_table has not been called");
     int launches = 0;
     NewCounts none;
     std::memset(&none, 0, sizeof none);
@@ -841,6 +880,20 @@ int h1b_debug_scores(h1b_ctx *ctx, int layer, int seq, int kv_head, const void *
     if (score_host && len > 0)
         H1B_CUDA(ctx, cudaMemcpy(score_host, at<int32_t>(ctx, ctx->plan.dbg_s), (size_t)len * sizeof(int32_t),
                                  cudaMemcpyDeviceToHost));
+    return H1B_OK;
+}
+
+int h1b_set_rope_table(h1b_ctx *ctx, const float *cos_sin_host, int n_positions, void *stream) {
+    if (!ctx) return H1B_ERR_NULL;
+    if (!cos_sin_host) return fail(ctx, H1B_ERR_NULL, "cos_sin_host is NULL");
+    if (!uses_rope(ctx)) return fail(ctx, H1B_ERR_INVALID_ARG, "the cache was not made with H1B_FLAG_ROPE");
+    if (n_positions < 1) return fail(ctx, H1B_ERR_INVALID_ARG, "n_positions = %d < 1", n_positions);
+    n_positions = std::min(n_positions, ctx->plan.cap_tokens);      // positions the cache can never reach are not kept
+    cudaStream_t st = static_cast<cudaStream_t>(stream);
+    const size_t bytes = (size_t)n_positions * (ctx->ucfg.head_dim / 2) * 2 * sizeof(float);
+    H1B_CUDA(ctx, cudaMemcpyAsync(ctx->ws + ctx->plan.rope, cos_sin_host, bytes, cudaMemcpyHostToDevice, st));
+    H1B_CUDA(ctx, cudaStreamSynchronize(st));
+    ctx->rope_positions = n_positions;
     return H1B_OK;
 }
 

@@ -34,12 +34,26 @@ struct ProjSmem {
     float r[kHeadDim][32];               // Rt[:, 32*word .. 32*word+31]
     float x[kHeadDim][kProjRows + 1];    // rows, transposed
     unsigned char sig[kProjRows][4];     // sign bits, one byte per (row, warp)
+    int pos[kProjRows];                  // position of each row (rotary embedding only; set by the caller)
 };
+
+// One rotary pair: (x, y) = channels (i, i + half) of a head, (c, s) the cosine and sine of the position's angle.
+// Products and sums are rounded to fp32 one by one (no fused multiply-add) and the caller rounds once to fp16:
+// every kernel, and a CPU check that does the same, gets the same fp16 bits.
+__device__ __forceinline__ float rope_first(float x, float y, float c, float s) {
+    return __fsub_rn(__fmul_rn(x, c), __fmul_rn(y, s));
+}
+__device__ __forceinline__ float rope_second(float x, float y, float c, float s) {
+    return __fadd_rn(__fmul_rn(y, c), __fmul_rn(x, s));
+}
+__device__ __forceinline__ int rope_clamp(const RopeRef &rope, int pos) { return max(0, min(pos, rope.n_pos - 1)); }
 
 // Returns, for threads 0..31, the packed word of row `tid` of the tile (other threads: unspecified).
 // x_rows: fp16 [n_rows][128], row-contiguous; rows beyond n_rows read as zero.
+// With rope.table set, the rows are first rotated at the positions sm.pos[row] (written by the caller before the call).
 __device__ __forceinline__ uint32_t project_tile(ProjSmem &sm, const uint16_t *__restrict__ x_rows, int n_rows,
-                                                 const float *__restrict__ Rt_layer, int m, int word) {
+                                                 const float *__restrict__ Rt_layer, int m, int word,
+                                                 const RopeRef &rope) {
     const int tid = threadIdx.x, lane = tid & 31, warp = tid >> 5;
     // All global loads of the tile are issued before the first shared-memory store, so that the block pays
     // one memory round trip, not one per loop iteration.
@@ -71,6 +85,18 @@ __device__ __forceinline__ uint32_t project_tile(ProjSmem &sm, const uint16_t *_
         sm.x[2 * c2 + 1][row] = v.y;
     }
     __syncthreads();
+    if (rope.table) {                                     // block-uniform
+        const int hw = rope.half;                         // 64 or 32: a power of two
+        for (int e = tid; e < kProjRows * (kHeadDim / 2); e += kProjThreads) {
+            const int row = e & (kProjRows - 1), j = e / kProjRows;
+            const int i = j & (hw - 1), ch = (j & ~(hw - 1)) * 2 + i;           // pair (ch, ch + hw) of head j / hw
+            const float2 cs = __ldg(reinterpret_cast<const float2 *>(rope.table) + (size_t)sm.pos[row] * hw + i);
+            const float x = sm.x[ch][row], y = sm.x[ch + hw][row];
+            sm.x[ch][row] = __half2float(__float2half_rn(rope_first(x, y, cs.x, cs.y)));
+            sm.x[ch + hw][row] = __half2float(__float2half_rn(rope_second(x, y, cs.x, cs.y)));
+        }
+        __syncthreads();
+    }
     float acc[8];
 #pragma unroll
     for (int c = 0; c < 8; ++c) acc[c] = 0.f;
@@ -179,8 +205,9 @@ __global__ void __launch_bounds__(kProjThreads) prepare_kernel(AppendParams ap, 
         const int row = row0 + min((int)threadIdx.x, n_rows - 1);
         const int kvh = row % ap.Hkv, tn = (row / ap.Hkv) % ap.Tn, b = row / (ap.Hkv * ap.Tn);
         const int len0 = ap.len[layer * ap.max_batch + b];
+        if (ap.rope.table && threadIdx.x < kProjRows) sm.pos[threadIdx.x] = rope_clamp(ap.rope, len0 + tn);
         const uint32_t bits = project_tile(sm, ap.k + ((size_t)ll * k_rows + row0) * kHeadDim, n_rows,
-                                           ap.Rt + (size_t)layer * kHeadDim * m, m, word);
+                                           ap.Rt + (size_t)layer * kHeadDim * m, m, word, ap.rope);
         if ((int)threadIdx.x < n_rows) {
             if (tn < nn.v[b] && len0 + nn.v[b] <= ap.seq_cap[b]) {
                 const int t = len0 + tn;
@@ -194,8 +221,13 @@ __global__ void __launch_bounds__(kProjThreads) prepare_kernel(AppendParams ap, 
         const int layer = sp.layer_begin + ll;
         const int row0 = tile * kProjRows;
         const int n_rows = min(kProjRows, q_rows - row0);
+        if (sp.rope.table && threadIdx.x < kProjRows) {
+            const int row = row0 + min((int)threadIdx.x, n_rows - 1);
+            const int h = row % sp.Hq, b = row / sp.Hq, tq = h / (sp.Hq / sp.Tq);
+            sm.pos[threadIdx.x] = rope_clamp(sp.rope, sp.len[layer * sp.max_batch + b] + nn.v[b] - sp.Tq + tq);
+        }
         const uint32_t bits = project_tile(sm, sp.q + ((size_t)ll * q_rows + row0) * kHeadDim, n_rows,
-                                           sp.Rt + (size_t)layer * kHeadDim * m, m, word);
+                                           sp.Rt + (size_t)layer * kHeadDim * m, m, word, sp.rope);
         if ((int)threadIdx.x < n_rows) {
             const int row = row0 + threadIdx.x;
             const int h = row % sp.Hq, b = row / sp.Hq;
@@ -486,7 +518,7 @@ __global__ void __launch_bounds__(kValueWarps * 32) prefill_values_kernel(Prefil
     prefill_publish_lengths(p, nn, &is_last);
 }
 
-template <int NBC>
+template <int NBC, bool ROPE>                   // ROPE: the key tiles are rotated in shared memory before the MMAs read them
 __global__ void __launch_bounds__(kPrefillThreads, 1) prefill_kernel(PrefillParams p, NewCounts nn) {
     using SM = PrefillSmem<NBC>;
     extern __shared__ unsigned char smem_unaligned[];
@@ -500,7 +532,11 @@ __global__ void __launch_bounds__(kPrefillThreads, 1) prefill_kernel(PrefillPara
     const ChunkLayout cl = chunk_layout(p.m_words, p.groups);
     const int groups_per_slab = (p.tiles_per_seq + p.tiles_per_block - 1) / p.tiles_per_block;
     const int col_blocks = (m + NBC - 1) / NBC;
-    const long n_work = (long)p.n_layers * p.B * p.Hkv * groups_per_slab * col_blocks;
+    // ROPE: a work item is one tile of 128 positions of one (layer, sequence) across ALL its KV heads (the tiles of the
+    // item are the heads), so that the rotary table entries of those positions are fetched once, into registers,
+    // for all of them. Otherwise: a run of consecutive position tiles of one slab.
+    const long n_work = ROPE ? (long)p.n_layers * p.B * p.tiles_per_seq * col_blocks
+                             : (long)p.n_layers * p.B * p.Hkv * groups_per_slab * col_blocks;
     const uint32_t bar0 = smem_addr(&mma_bar_s[0]);
 
     // a block that starts after some other block has given up a wait does nothing (keeps a failure short)
@@ -530,18 +566,33 @@ __global__ void __launch_bounds__(kPrefillThreads, 1) prefill_kernel(PrefillPara
     int issued = 0, waited = 0;                                 // tiles (by seq) whose MMAs were issued / waited for
     for (long work = blockIdx.x; work < n_work && !skip_all; work += gridDim.x) {
         const int cbk = (int)(work % col_blocks);
-        const int tg = (int)((work / col_blocks) % groups_per_slab);
-        const long slab_local = work / ((long)col_blocks * groups_per_slab);
-        const int kvh = (int)(slab_local % p.Hkv), b = (int)((slab_local / p.Hkv) % p.B), ll = (int)(slab_local / ((long)p.Hkv * p.B));
+        int b, ll, kvh0, first_tile, n_tiles, len0, n_new;
+        if constexpr (ROPE) {
+            const int pt = (int)((work / col_blocks) % p.tiles_per_seq);
+            const long seq_local = work / ((long)col_blocks * p.tiles_per_seq);
+            b = (int)(seq_local % p.B); ll = (int)(seq_local / p.B);
+            len0 = p.len[(p.layer_begin + ll) * p.max_batch + b];
+            n_new = (len0 + nn.v[b] <= p.seq_cap[b]) ? nn.v[b] : 0;             // no room: nothing is written
+            kvh0 = 0;
+            first_tile = len0 / kPrefillTile + pt;
+            n_tiles = (first_tile * kPrefillTile < len0 + n_new) ? p.Hkv : 0;   // one tile per KV head
+        } else {
+            const int tg = (int)((work / col_blocks) % groups_per_slab);
+            const long slab_local = work / ((long)col_blocks * groups_per_slab);
+            kvh0 = (int)(slab_local % p.Hkv); b = (int)((slab_local / p.Hkv) % p.B); ll = (int)(slab_local / ((long)p.Hkv * p.B));
+            len0 = p.len[(p.layer_begin + ll) * p.max_batch + b];
+            n_new = (len0 + nn.v[b] <= p.seq_cap[b]) ? nn.v[b] : 0;             // no room: nothing is written
+            first_tile = len0 / kPrefillTile + tg * p.tiles_per_block;
+            // tiles of this work item that overlap the appended range (block-uniform)
+            n_tiles = max(0, min(p.tiles_per_block,
+                                 (len0 + n_new - first_tile * kPrefillTile + kPrefillTile - 1) / kPrefillTile));
+        }
         const int layer = p.layer_begin + ll;
         const int col0 = cbk * NBC;                             // first sketch column of this work item
-        const int len0 = p.len[layer * p.max_batch + b];
-        const int n_new = (len0 + nn.v[b] <= p.seq_cap[b]) ? nn.v[b] : 0;       // no room: nothing is written
-        const int first_tile = len0 / kPrefillTile + tg * p.tiles_per_block;
-        // tiles of this work item that overlap the appended range (block-uniform)
-        const int n_tiles = max(0, min(p.tiles_per_block,
-                                       (len0 + n_new - first_tile * kPrefillTile + kPrefillTile - 1) / kPrefillTile));
         if (n_tiles == 0) continue;
+        // tile ti of the work item: which KV head, and which position tile
+        auto tile_kvh = [&](int ti) { return ROPE ? ti : kvh0; };
+        auto tile_pos = [&](int ti) { return (ROPE ? first_tile : first_tile + ti) * kPrefillTile; };
         // ---- the two fp16 pieces of Rt[:, col0 .. col0+NBC), transposed and stacked: B[2 * NBC rows][channel].
         // (All MMAs of the previous work item have completed: its last tile was waited for.)
         if (layer != loaded_layer || col0 != loaded_col0) {
@@ -554,16 +605,62 @@ __global__ void __launch_bounds__(kPrefillThreads, 1) prefill_kernel(PrefillPara
             loaded_layer = layer;
             loaded_col0 = col0;
         }
-        const uint16_t *k_seq = p.k + (((size_t)ll * p.B + b) * p.Tn * p.Hkv + kvh) * kHeadDim + ld_c * 8;   // token 0 of this head
+        const uint16_t *k_seq0 = p.k + ((size_t)ll * p.B + b) * p.Tn * p.Hkv * kHeadDim + ld_c * 8;   // token 0, KV head 0
         // key tile ti of the work item: row r = position P0 + r; rows outside the appended range are zero
         auto load_key_tile = [&](int ti) {
-            const int tn0 = (first_tile + ti) * kPrefillTile + ld_r0 - len0;    // appended-token index of this thread's first row
+            const uint16_t *k_seq = k_seq0 + (size_t)tile_kvh(ti) * kHeadDim;
+            const int tn0 = tile_pos(ti) + ld_r0 - len0;                        // appended-token index of this thread's first row
             const uint32_t dst0 = smem_addr(As0 + ((seq + ti) % kKeyStages) * SM::kABytes) + ld_soff;
 #pragma unroll
             for (int k = 0; k < kPrefillTile / kRowsPerPass; ++k) {
                 const int tn = tn0 + k * kRowsPerPass;
                 const bool ok = tn >= 0 && tn < n_new;
                 cp_async_16(dst0 + k * (kRowsPerPass * 128), k_seq + (size_t)(ok ? tn : 0) * k_row_stride, ok ? 16u : 0u);
+            }
+        };
+        // Rotary embedding of a key tile in place, between its landing and its MMAs. A thread turns four pairs
+        // (channels 4cc .. 4cc+3 of a head's first half with the same of its second half) of rows r0 + 16 k: two 8-byte
+        // pieces per row, both copied by threads of its own half-warp, so a warp-level barrier after the copies have
+        // landed is all the ordering the reads need, and nobody else touches what it writes. The table entries of
+        // the item's 128 positions sit in registers for all the heads of the item. Rows outside the appended range
+        // are zeros and stay zeros.
+        constexpr int kRotRows = kPrefillTile / kRowsPerPass;   // 8 rows per thread
+        float2 cs[ROPE ? kRotRows : 1][ROPE ? 4 : 1];
+        int rot_lo = 0, rot_hi = 0;                             // byte offsets of the thread's two pieces of row r0
+        if constexpr (ROPE) {
+            const int hw = p.rope.half, cc = tid & 15;
+            const int ch = ((4 * cc) & ~(hw - 1)) * 2 + ((4 * cc) & (hw - 1));      // first channel of the four pairs
+            const int pair0 = (4 * cc) & (hw - 1);
+            rot_lo = kmajor_sw128_off(kPrefillTile, ld_r0, ch >> 3) + (ch & 7) * 2;
+            rot_hi = kmajor_sw128_off(kPrefillTile, ld_r0, (ch + hw) >> 3) + (ch & 7) * 2;
+#pragma unroll
+            for (int k = 0; k < kRotRows; ++k) {
+                const int pos = rope_clamp(p.rope, first_tile * kPrefillTile + ld_r0 + k * kRowsPerPass);
+                const float4 *tp = reinterpret_cast<const float4 *>(p.rope.table + ((size_t)pos * hw + pair0) * 2);
+                const float4 t0 = __ldg(tp), t1 = __ldg(tp + 1);
+                cs[k][0] = make_float2(t0.x, t0.y); cs[k][1] = make_float2(t0.z, t0.w);
+                cs[k][2] = make_float2(t1.x, t1.y); cs[k][3] = make_float2(t1.z, t1.w);
+            }
+        }
+        auto rotate_key_tile = [&](int ti) {
+            if constexpr (ROPE) {
+                unsigned char *A = As0 + ((seq + ti) % kKeyStages) * SM::kABytes;
+                __syncwarp();
+#pragma unroll
+                for (int k = 0; k < kRotRows; ++k) {
+                    uint2 *plo = reinterpret_cast<uint2 *>(A + rot_lo + k * (kRowsPerPass * 128));
+                    uint2 *phi = reinterpret_cast<uint2 *>(A + rot_hi + k * (kRowsPerPass * 128));
+                    const uint2 lo = *plo, hi = *phi;
+                    const float2 x01 = half2_bits_to_float2(lo.x), x23 = half2_bits_to_float2(lo.y);
+                    const float2 y01 = half2_bits_to_float2(hi.x), y23 = half2_bits_to_float2(hi.y);
+                    uint2 rlo, rhi;
+                    rlo.x = pack_f16x2(rope_first(x01.x, y01.x, cs[k][0].x, cs[k][0].y), rope_first(x01.y, y01.y, cs[k][1].x, cs[k][1].y));
+                    rlo.y = pack_f16x2(rope_first(x23.x, y23.x, cs[k][2].x, cs[k][2].y), rope_first(x23.y, y23.y, cs[k][3].x, cs[k][3].y));
+                    rhi.x = pack_f16x2(rope_second(x01.x, y01.x, cs[k][0].x, cs[k][0].y), rope_second(x01.y, y01.y, cs[k][1].x, cs[k][1].y));
+                    rhi.y = pack_f16x2(rope_second(x23.x, y23.x, cs[k][2].x, cs[k][2].y), rope_second(x23.y, y23.y, cs[k][3].x, cs[k][3].y));
+                    *plo = rlo;
+                    *phi = rhi;
+                }
             }
         };
         // y = K x (Rh1 + Rh2)^T for tile ti: one thread issues 2 pieces x 8 K-slices of 16 into one accumulator
@@ -592,6 +689,7 @@ __global__ void __launch_bounds__(kPrefillThreads, 1) prefill_kernel(PrefillPara
             cp_async_commit();
         }
         cp_async_wait_group<kKeyStages - 1>();
+        if constexpr (ROPE) rotate_key_tile(0);
         fence_proxy_async_smem();                               // generic-proxy writes -> visible to the tensor cores
         __syncthreads();
         issue_mma(0);
@@ -601,6 +699,7 @@ __global__ void __launch_bounds__(kPrefillThreads, 1) prefill_kernel(PrefillPara
         for (int ti = 0; ti < n_tiles; ++ti) {
             if (ti + 1 < n_tiles) {                             // start tile ti+1's MMAs behind tile ti's
                 cp_async_wait_group<kKeyStages - 2>();
+                if constexpr (ROPE) rotate_key_tile(ti + 1);
                 fence_proxy_async_smem();
                 __syncthreads();                                // also: every thread is done with the accumulator that comes next
                 if (gave_up) { stop = true; break; }
@@ -617,7 +716,7 @@ __global__ void __launch_bounds__(kPrefillThreads, 1) prefill_kernel(PrefillPara
             // ---- signs: thread = accumulator row 32*(warp%4) + lane (a warp can only read the TMEM lanes of its
             // quarter); a warp packs one key word (32 columns) per thread at a time
             if (done) {
-                const int P0 = (first_tile + ti) * kPrefillTile;
+                const int P0 = tile_pos(ti), kvh = tile_kvh(ti);
                 const int quarter = warp & 3;
                 const int pos = P0 + quarter * 32 + lane, tn = pos - len0;
                 // this warp's 32 rows are the 32 tokens of one chunk
@@ -1237,25 +1336,27 @@ cudaError_t launch_prepare(const AppendParams *ap, const SketchParams *sp, const
 }
 
 static long prefill_key_blocks(const PrefillParams &p, int nbc) {
+    const long col_blocks = (p.m_words * 32 + nbc - 1) / nbc;
+    if (p.rope.table) return (long)p.n_layers * p.B * p.tiles_per_seq * col_blocks;   // (position tile) x all KV heads
     const long groups = (p.tiles_per_seq + p.tiles_per_block - 1) / p.tiles_per_block;
-    return (long)p.n_layers * p.B * p.Hkv * groups * ((p.m_words * 32 + nbc - 1) / nbc);
+    return (long)p.n_layers * p.B * p.Hkv * groups * col_blocks;
 }
 
-template <int NBC>
+template <int NBC, bool ROPE>
 static cudaError_t launch_prefill_t(const PrefillParams &p, const NewCounts &nn, cudaStream_t st, int grid) {
     using SM = PrefillSmem<NBC>;
     static bool attr_set[64] = {};
     int dev = 0;
     cudaGetDevice(&dev);
     if (dev >= 0 && dev < 64 && !attr_set[dev]) {
-        cudaError_t e = cudaFuncSetAttribute(prefill_kernel<NBC>, cudaFuncAttributeMaxDynamicSharedMemorySize, SM::kTotal);
+        cudaError_t e = cudaFuncSetAttribute(prefill_kernel<NBC, ROPE>, cudaFuncAttributeMaxDynamicSharedMemorySize, SM::kTotal);
         if (e != cudaSuccess) return e;
         // the largest shared-memory split, not the smallest that fits this kernel: the rest is for the value kernel's blocks
-        e = cudaFuncSetAttribute(prefill_kernel<NBC>, cudaFuncAttributePreferredSharedMemoryCarveout, cudaSharedmemCarveoutMaxShared);
+        e = cudaFuncSetAttribute(prefill_kernel<NBC, ROPE>, cudaFuncAttributePreferredSharedMemoryCarveout, cudaSharedmemCarveoutMaxShared);
         if (e != cudaSuccess) return e;
         attr_set[dev] = true;
     }
-    prefill_kernel<NBC><<<(unsigned)grid, kPrefillThreads, SM::kTotal, st>>>(p, nn);
+    prefill_kernel<NBC, ROPE><<<(unsigned)grid, kPrefillThreads, SM::kTotal, st>>>(p, nn);
     return cudaGetLastError();
 }
 
@@ -1301,7 +1402,10 @@ cudaError_t launch_prefill(const PrefillParams &p_in, const NewCounts &nn, cudaS
     }
     // the key kernel first: one block of it settles on every SM (its shared memory allows no more), and the value
     // kernel's small blocks fill the registers and issue slots that are left
-    e = (nbc == 128) ? launch_prefill_t<128>(p, nn, st, (int)kblocks) : launch_prefill_t<64>(p, nn, st, (int)kblocks);
+    if (p.rope.table)
+        e = (nbc == 128) ? launch_prefill_t<128, true>(p, nn, st, (int)kblocks) : launch_prefill_t<64, true>(p, nn, st, (int)kblocks);
+    else
+        e = (nbc == 128) ? launch_prefill_t<128, false>(p, nn, st, (int)kblocks) : launch_prefill_t<64, false>(p, nn, st, (int)kblocks);
     if (e != cudaSuccess) return e;
     ++*launches;
     prefill_values_kernel<<<(unsigned)vblocks, kValueWarps * 32, 0, forked ? side : st>>>(p, nn);

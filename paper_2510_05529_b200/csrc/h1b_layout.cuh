@@ -120,6 +120,17 @@ constexpr int kStatusCapacity = 2;      // an append found a sequence full (only
 
 struct NewCounts { int32_t v[256]; };            // n_new per sequence, passed by value
 
+// Rotary position embedding of the rows that enter Eq. 2 (keys at their cache position, queries at the position of
+// the token they belong to), fused into the append and the query sketch. Half-split pairs: channel i of a head
+// turns with channel i + half by the angle whose (cos, sin) is table[position][i]. table == null: no rotation.
+// The arithmetic is fixed so that every kernel (and a CPU check) gets the same fp16 bits: each product and the
+// sum rounded to fp32, no fused multiply-add, then one rounding to fp16.
+struct RopeRef {
+    const float *table;         // fp32 [n_pos][half][2]
+    int half;                   // half the caller's head dimension (64, or 32 for 64-wide heads)
+    int n_pos;                  // positions the table holds (positions beyond are clamped: memory safety only)
+};
+
 struct AppendParams {
     const uint16_t *k, *v;      // fp16 [n_layers][B][Tn][Hkv][d]
     const float *Rt;            // [L][d][m]
@@ -130,6 +141,7 @@ struct AppendParams {
     const int32_t *seq_cap;     // [max_batch] tokens each sequence has room for: an append that would pass it is dropped
                                 // and flagged (only a replayed graph can get there: direct calls are checked on the host)
     int layer_begin, n_layers, B, Tn, Hkv, max_batch, m_words, groups;
+    RopeRef rope;
 };
 
 struct PrefillParams {          // long appends: tensor-core projection
@@ -145,6 +157,7 @@ struct PrefillParams {          // long appends: tensor-core projection
     int tiles_per_block;        // consecutive tiles handled by one block (the projection is loaded once per block)
     int total_blocks;           // blocks of the key kernel plus blocks of the value kernel: the last of them all to finish
                                 // publishes the new lengths (the two kernels may run side by side)
+    RopeRef rope;
 };
 
 struct SketchParams {           // query sketch
@@ -152,6 +165,11 @@ struct SketchParams {           // query sketch
     const float *Rt;
     uint32_t *qwords;           // [L][max_batch][Hq][m/32]
     int layer_begin, n_layers, B, Hq, max_batch, m_words;
+    // rotation of the queries: row (b, h) belongs to query token h / (Hq / Tq) of Tq, whose position is
+    // len + n_new - Tq + that index (len as the launch finds it, n_new what the same launch appends)
+    RopeRef rope;
+    const int32_t *len;         // [L][max_batch] (read only when rope.table is set)
+    int Tq;
 };
 
 struct DecodeParams {

@@ -18,14 +18,28 @@ def f16_bits(t: torch.Tensor) -> np.ndarray:
     return t.detach().cpu().contiguous().view(torch.int16).numpy().view(np.uint16)
 
 
-def make_cache(w: h1b_synth.Workload, max_seq=None, Rt=None, fp16_values=False, page_tokens=0, n_pages=0):
+def make_cache(w: h1b_synth.Workload, max_seq=None, Rt=None, fp16_values=False, page_tokens=0, n_pages=0,
+               rope_table=None):
     cfg = binding.make_config(w.n_layers, w.n_q_heads, w.n_kv_heads, w.head_dim, w.sketch_bits, w.group_size,
                               max_batch=w.batch, max_seq=max_seq or w.context, fp16_values=fp16_values,
-                              page_tokens=page_tokens, n_pages=n_pages)
+                              page_tokens=page_tokens, n_pages=n_pages, rope=rope_table is not None)
     if Rt is None:
         Rt = np.stack([h1b_synth.projection(h1b_synth.layer_seed(w, l, 99), w.head_dim, w.sketch_bits)
                        for l in range(w.n_layers)])
-    return binding.H1BCache(cfg, Rt=Rt), Rt
+    cache = binding.H1BCache(cfg, Rt=Rt)
+    if rope_table is not None:
+        cache.h1b_set_rope_table(rope_table)
+    return cache, Rt
+
+
+def rope_rows(x_bits: np.ndarray, rope_table, pos) -> np.ndarray:
+    """The oracle's rotation of fp16 rows [..., rows, d] at positions pos [rows] (or one position for all);
+    rope_table None: the rows as they are."""
+    if rope_table is None:
+        return x_bits
+    flat = x_bits.reshape(-1, x_bits.shape[-1])
+    pos = np.broadcast_to(np.asarray(pos, np.int32), (flat.shape[0],)) if np.ndim(pos) == 0 else np.asarray(pos, np.int32)
+    return oracle.rope(flat, rope_table, pos).reshape(x_bits.shape)
 
 
 def check_output(got: np.ndarray, ref: np.ndarray, what=""):
@@ -81,7 +95,7 @@ def append_parity(cache, layer, seq, kvh, K_rows, V_rows, Rt_layer, t0=0):
     return stats
 
 
-def oracle_from_export(cache, layer, seq, q_head, q_row_dev, length, inv_tau, Rt_layer):
+def oracle_from_export(cache, layer, seq, q_head, q_row_dev, length, inv_tau, Rt_layer, rope_table=None):
     """Protocol 2: the oracle's Eq. 3 + Eq. 5 on the cache the GPU wrote and on the
     GPU's own query sketch. Also checks the GPU's integer scores bit for bit."""
     c = cache.cfg
@@ -94,18 +108,21 @@ def oracle_from_export(cache, layer, seq, q_head, q_row_dev, length, inv_tau, Rt
     oscore = oracle.scores(qbits, kbits) if length > 0 else np.zeros((0,), np.int32)
     assert np.array_equal(gscore, oscore), "integer Hamming scores differ"
     # the query sketch itself: identical to the oracle's except at the sign boundary
-    oq, y, a = oracle.sketch(f16_bits(q_row_dev)[None], Rt_layer, want_margin=True)
+    # (with rotary embedding the query is turned at the sequence's last position, on both sides)
+    oq, y, a = oracle.sketch(rope_rows(f16_bits(q_row_dev)[None], rope_table, max(length - 1, 0)), Rt_layer,
+                             want_margin=True)
     d = oq[0] != qbits
     assert not (d & (np.abs(y[0]) > WINDOW * a[0])).any(), "query sketch bit differs away from the boundary"
     return oracle.attention(oscore, c.sketch_bits, inv_tau, codes, scale, zero, c.group_size), int(d.sum())
 
 
-def build_and_decode(w: h1b_synth.Workload, lens, inv_tau=16.0, appends=None, splits=0, device="cuda", max_seq=None):
+def build_and_decode(w: h1b_synth.Workload, lens, inv_tau=16.0, appends=None, splits=0, device="cuda", max_seq=None,
+                     rope_table=None):
     """Fill a cache with seeded K/V (lens[b] tokens per sequence, in `appends`
     calls), run one decode, and return everything the checks need."""
     lens = np.asarray(lens, dtype=np.int32)
     T = int(lens.max(initial=0))
-    cache, Rt = make_cache(w, max_seq=max_seq or max(T, 1))
+    cache, Rt = make_cache(w, max_seq=max_seq or max(T, 1), rope_table=rope_table)
     Ks, Vs, qs = [], [], []
     for l in range(w.n_layers):
         K, V = h1b_synth.kv_rows(w, l, max(T, 1))
@@ -135,28 +152,36 @@ def build_and_decode(w: h1b_synth.Workload, lens, inv_tau=16.0, appends=None, sp
     return dict(cache=cache, Rt=Rt, K=K, V=V, q=q, qd=qd, out=out.cpu().numpy(), lens=lens)
 
 
-def full_parity(w: h1b_synth.Workload, lens, inv_tau=16.0, appends=None, splits=0, sample=None):
+def full_parity(w: h1b_synth.Workload, lens, inv_tau=16.0, appends=None, splits=0, sample=None, rope_table=None):
     """Append parity, isolated decode parity and end-to-end parity on every (or
-    a sample of) (layer, sequence, head). Returns summary statistics."""
-    r = build_and_decode(w, lens, inv_tau, appends, splits)
+    a sample of) (layer, sequence, head). Returns summary statistics.
+    rope_table: the cache rotates keys and queries itself; the oracle is given rows rotated by its own rope()."""
+    r = build_and_decode(w, lens, inv_tau, appends, splits, rope_table=rope_table)
     cache, Rt, K, V, q, out = r["cache"], r["Rt"], r["K"], r["V"], r["q"], r["out"]
     gq = w.n_q_heads // w.n_kv_heads
     tot = {"bit_flips_in": 0, "code_flips_in": 0, "scale_flips_in": 0, "q_flips_in": 0, "max_err": 0.0, "max_err_e2e": 0.0}
     for l in range(w.n_layers):
         assert np.array_equal(cache.h1b_get_lengths(l)[:w.batch], lens)
-        ref_e2e = oracle.layer(f16_bits(K[l]), f16_bits(V[l]), lens, f16_bits(q[l]), Rt[l], inv_tau, w.group_size)
+        Kl, ql = f16_bits(K[l]), f16_bits(q[l])                       # [B, T, Hkv, d], [B, Hq, d]
+        if rope_table is not None:
+            T = Kl.shape[1]
+            Kl = np.stack([rope_rows(Kl[b].transpose(1, 0, 2), rope_table, np.tile(np.arange(T, dtype=np.int32), Kl.shape[2]))
+                           .transpose(1, 0, 2) for b in range(w.batch)])
+            ql = np.stack([rope_rows(ql[b], rope_table, max(int(lens[b]) - 1, 0)) for b in range(w.batch)])
+        ref_e2e = oracle.layer(Kl, f16_bits(V[l]), lens, ql, Rt[l], inv_tau, w.group_size)
         for b in range(w.batch):
             n = int(lens[b])
             for g in range(w.n_kv_heads):
                 if sample is not None and (l, b, g) not in sample:
                     continue
                 if n > 0:
-                    st = append_parity(cache, l, b, g, f16_bits(K[l, b, :n, g]), f16_bits(V[l, b, :n, g]), Rt[l])
+                    st = append_parity(cache, l, b, g, np.ascontiguousarray(Kl[b, :n, g]), f16_bits(V[l, b, :n, g]), Rt[l])
                     for k_ in ("bit_flips_in", "code_flips_in", "scale_flips_in"):
                         tot[k_] += st[k_]
                 for hh in range(gq):
                     h = g * gq + hh
-                    ref, qf = oracle_from_export(cache, l, b, h, r["qd"][l, b, h].contiguous(), n, inv_tau, Rt[l])
+                    ref, qf = oracle_from_export(cache, l, b, h, r["qd"][l, b, h].contiguous(), n, inv_tau, Rt[l],
+                                                 rope_table)
                     tot["q_flips_in"] += qf
                     tot["max_err"] = max(tot["max_err"], check_output(out[l, b, h], ref, ("isolated", l, b, h)))
                     if st_clean(tot):

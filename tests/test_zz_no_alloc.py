@@ -12,6 +12,8 @@ refused with a clear error instead of running past the array.
 Collected last on purpose, and written to pass both on its own in a fresh
 process and after every other test has used the library.
 """
+import gc
+
 import numpy as np
 import pytest
 import torch
@@ -32,6 +34,7 @@ def test_static_entry_matches_the_ordinary_one_twice_in_a_row():
     q2 = torch.stack([h1b_synth.queries(w, l, stream=3) for l in range(w.n_layers)]).cuda()
     ref2 = cache.h1b_decode_attention(q2, 4.0).cpu().numpy()             # second queries, another temperature
     out = torch.full(qd.shape, float("nan"), dtype=torch.float32, device="cuda")
+    gc.collect()                                                         # tensors earlier tests left in reference cycles go now, not below
     before = torch.cuda.memory_allocated()
     cache.h1b_decode_attention_static(qd, 16.0, out)                     # first call: also resolves the array
     got1 = out.cpu().numpy().copy()
