@@ -49,6 +49,13 @@ def test_entry_and_workspace_bytes(lib):
     c64 = binding.make_config(12, 8, 8, 64, 128, 32, max_batch=1, max_seq=4096)
     assert binding.h1b_entry_bytes(c64) == 56
     assert binding.h1b_cache_bytes(c64) >= 12 * 8 * 4096 * 56
+    # the rotary option adds its table: (cos, sin) fp32 per position and channel pair
+    plain = binding.h1b_cache_bytes(binding.make_config(2, 4, 4, max_seq=1024))
+    rope = binding.h1b_cache_bytes(binding.make_config(2, 4, 4, max_seq=1024, rope=True))
+    assert rope - plain == 1024 * 64 * 2 * 4
+    bad = binding.make_config(2, 4, 4, max_seq=1024)
+    bad.flags = 4                                           # an unknown flag bit
+    assert binding.h1b_cache_bytes(bad) == 0
     # capacity is rounded up to whole 32-token chunks
     a = binding.h1b_cache_bytes(binding.make_config(1, 1, 1, max_seq=33))
     b = binding.h1b_cache_bytes(binding.make_config(1, 1, 1, max_seq=64))
@@ -74,6 +81,7 @@ def test_null_context_calls_return_error_codes(lib):
     assert lib.h1b_free(None) == -2
     assert lib.h1b_poll_status(None) == -2
     assert lib.h1b_set_splits(None, 1) == -2
+    assert lib.h1b_set_rope_table(None, None, 1, None) == -2
     assert lib.h1b_launch_count(None) == 0
     # init with a NULL workspace is rejected on the host before any CUDA call
     c = binding.make_config(1, 1, 1)

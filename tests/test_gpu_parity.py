@@ -129,13 +129,14 @@ def test_scores_bit_exact_and_repeatable():
     assert np.array_equal(a["out"], out2)
 
 
-def test_host_step_equals_device_calls():
-    w = small("c2_7b_8k", n_layers=2, n_q_heads=4, n_kv_heads=4, batch=2, context=100)
+@pytest.mark.parametrize("L", [2, 1, 3])
+def test_host_step_equals_device_calls(L):
+    w = small("c2_7b_8k", n_layers=L, n_q_heads=4, n_kv_heads=4, batch=2, context=100)
     r = build_and_decode(w, [99, 50], max_seq=128)
     cache = r["cache"]
     k1, v1 = h1b_synth.kv_rows(w, 0, 1, stream=5)
-    kh = torch.stack([k1, k1 * 0.5]).contiguous().pin_memory()      # [L, B, 1, Hkv, d]
-    vh = torch.stack([v1, v1 * 2.0]).contiguous().pin_memory()
+    kh = torch.stack([k1 * 0.5 ** l for l in range(L)]).contiguous().pin_memory()      # [L, B, 1, Hkv, d]
+    vh = torch.stack([v1 * 2.0 ** l for l in range(L)]).contiguous().pin_memory()
     qh = r["q"].contiguous().pin_memory()
     outh = torch.empty(qh.shape, dtype=torch.float32).pin_memory()
     cache.h1b_decode_step_host(kh, vh, qh, 16.0, outh)
@@ -149,7 +150,7 @@ def test_host_step_equals_device_calls():
     r3 = build_and_decode(w, [99, 50], max_seq=128)
     out3 = r3["cache"].h1b_decode_step(kh.cuda(), vh.cuda(), r3["qd"], 16.0)
     assert np.array_equal(outh.numpy(), out3.cpu().numpy())
-    assert r3["cache"].h1b_get_lengths(1)[:2].tolist() == [100, 51]
+    assert r3["cache"].h1b_get_lengths(L - 1)[:2].tolist() == [100, 51]
     # ... and on a fourth one through the host entry point again, with k, v and q back to back in one pinned
     # buffer (they then travel in a single copy)
     r4 = build_and_decode(w, [99, 50], max_seq=128)
@@ -163,7 +164,7 @@ def test_host_step_equals_device_calls():
     # and against the oracle, end to end, for one sequence
     K = torch.cat([r["K"][:, :, :100], torch.zeros_like(r["K"][:, :, :1])], 2)
     V = torch.cat([r["V"][:, :, :100], torch.zeros_like(r["V"][:, :, :1])], 2)
-    for l in range(2):
+    for l in range(L):
         for b, n in enumerate((99, 50)):
             K[l, b, n] = kh[l, b, 0]
             V[l, b, n] = vh[l, b, 0]
