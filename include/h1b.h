@@ -285,6 +285,12 @@ int h1b_reset(h1b_ctx *ctx, int seq);
  * must not exceed any of their current lengths (roll back the last tokens). */
 int h1b_truncate(h1b_ctx *ctx, int seq, int new_len);
 
+/* The same, ordered on `stream` instead of waiting for the device (rejecting
+ * speculated tokens between two decode steps): the caller keeps every call that
+ * touches this cache on that one stream, or orders them with events. Both
+ * h1b_reset and h1b_truncate wait for the whole device before and after. */
+int h1b_truncate_async(h1b_ctx *ctx, int seq, int new_len, void *stream);
+
 /* Unpack cached tokens [t0, t0+n) of (layer, seq, kv_head) into a canonical
  * layout, independent of the packed device layout (all HOST, any may be NULL):
  *   words  uint32 [n][m/32]: sketch bit j is bit (j % 32) of word j / 32

@@ -78,6 +78,7 @@ def load_library(rebuild: bool = True) -> ctypes.CDLL:
         "h1b_get_lengths": (ctypes.c_int, [vp, ctypes.c_int, vp]),
         "h1b_reset": (ctypes.c_int, [vp, ctypes.c_int]),
         "h1b_truncate": (ctypes.c_int, [vp, ctypes.c_int, ctypes.c_int]),
+        "h1b_truncate_async": (ctypes.c_int, [vp, ctypes.c_int, ctypes.c_int, vp]),
         "h1b_export_cache": (ctypes.c_int, [vp, ctypes.c_int, ctypes.c_int, ctypes.c_int, ctypes.c_int,
                                             ctypes.c_int, vp, vp, vp, vp]),
         "h1b_export_values": (ctypes.c_int, [vp, ctypes.c_int, ctypes.c_int, ctypes.c_int, ctypes.c_int,
@@ -313,6 +314,10 @@ class H1BCache:
 
     def h1b_truncate(self, seq: int, new_len: int):
         self._check(self.lib.h1b_truncate(self._h, seq, new_len))
+
+    def h1b_truncate_async(self, seq: int, new_len: int, stream=None):
+        """h1b_truncate ordered on the stream, without waiting for the device."""
+        self._check(self.lib.h1b_truncate_async(self._h, seq, new_len, _stream_ptr(stream)))
 
     def h1b_export_cache(self, layer: int, seq: int, kv_head: int, t0: int, n: int):
         """-> (words uint32 [n, m/32], codes uint8 [n, d], scale uint16 [n, d/G], zero uint16 [n, d/G])."""

@@ -751,7 +751,7 @@ int h1b_get_lengths(h1b_ctx *ctx, int layer, int32_t *len_host) {
     return H1B_OK;
 }
 
-int h1b_truncate(h1b_ctx *ctx, int seq, int new_len) {
+static int truncate_impl(h1b_ctx *ctx, int seq, int new_len, bool whole_device, cudaStream_t st) {
     if (!ctx) return H1B_ERR_NULL;
     const int mb = ctx->cfg.max_batch;
     if (seq < -1 || seq >= mb) return fail(ctx, H1B_ERR_INVALID_ARG, "sequence %d out of range", seq);
@@ -761,13 +761,19 @@ int h1b_truncate(h1b_ctx *ctx, int seq, int new_len) {
             if ((seq < 0 || b == seq) && new_len > 0 && ctx->len_host[(size_t)l * mb + b] < new_len)
                 return fail(ctx, H1B_ERR_INVALID_ARG, "layer %d sequence %d holds %d < %d tokens", l, b,
                             ctx->len_host[(size_t)l * mb + b], new_len);
-    H1B_CUDA(ctx, cudaDeviceSynchronize());
-    H1B_CUDA(ctx, launch_set_len(at<int32_t>(ctx, ctx->plan.len), ctx->cfg.n_layers, mb, seq, new_len, nullptr));
-    H1B_CUDA(ctx, cudaDeviceSynchronize());
+    if (whole_device) H1B_CUDA(ctx, cudaDeviceSynchronize());
+    H1B_CUDA(ctx, launch_set_len(at<int32_t>(ctx, ctx->plan.len), ctx->cfg.n_layers, mb, seq, new_len, st));
+    if (whole_device) H1B_CUDA(ctx, cudaDeviceSynchronize());
     for (int l = 0; l < ctx->cfg.n_layers; ++l)
         for (int b = 0; b < mb; ++b)
             if (seq < 0 || b == seq) ctx->len_host[(size_t)l * mb + b] = new_len;
     return H1B_OK;
+}
+
+int h1b_truncate(h1b_ctx *ctx, int seq, int new_len) { return truncate_impl(ctx, seq, new_len, true, nullptr); }
+
+int h1b_truncate_async(h1b_ctx *ctx, int seq, int new_len, void *stream) {
+    return truncate_impl(ctx, seq, new_len, false, static_cast<cudaStream_t>(stream));
 }
 
 int h1b_reset(h1b_ctx *ctx, int seq) { return h1b_truncate(ctx, seq, 0); }

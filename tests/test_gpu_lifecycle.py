@@ -97,7 +97,7 @@ def test_speculated_tokens_verified_then_partly_rejected():
         plain.h1b_append_kv(Kd[:, :, i:i + 1].cuda(), Vd[:, :, i:i + 1].cuda())
         one = plain.h1b_decode_attention(qd[:, :, i].contiguous(), 16.0).cpu().numpy()
         np.testing.assert_allclose(verify[:, :, i], one, rtol=2e-4, atol=2e-6)
-    spec.h1b_truncate(0, 152)                             # two of the four accepted
+    spec.h1b_truncate_async(0, 152)                       # two of the four accepted: ordered on the stream, no device-wide wait
     plain.h1b_truncate(0, 152)
     qn = torch.stack([h1b_synth.queries(w, l, stream=40) for l in range(w.n_layers)]).cuda()
     a = spec.h1b_decode_step(Kn.cuda(), Vn.cuda(), qn, 16.0).cpu().numpy()
