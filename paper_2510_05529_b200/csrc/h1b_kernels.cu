@@ -519,7 +519,7 @@ __global__ void __launch_bounds__(kValueWarps * 32) prefill_values_kernel(Prefil
 }
 
 template <int NBC, bool ROPE>                   // ROPE: the key tiles are rotated in shared memory before the MMAs read them
-__global__ void __launch_bounds__(kPrefillThreads, 1) prefill_kernel(PrefillParams p, NewCounts nn) {
+__device__ __forceinline__ void prefill_body(const PrefillParams &p, const NewCounts &nn) {
     using SM = PrefillSmem<NBC>;
     extern __shared__ unsigned char smem_unaligned[];
     unsigned char *smem = smem_unaligned + ((1024u - (smem_addr(smem_unaligned) & 1023u)) & 1023u);
@@ -757,6 +757,20 @@ __global__ void __launch_bounds__(kPrefillThreads, 1) prefill_kernel(PrefillPara
     if (warp == 0 && !skip_all) { tc_fence_after_sync(); tmem_dealloc(tmem_d, 2 * NBC); }
     prefill_publish_lengths(p, nn, &is_last);
 }
+
+// The two entry points of the body above. The rotating variant keeps 64 table entries in registers; its register
+// cap is what still lets two blocks of the value kernel settle beside it on an SM.
+template <int NBC, bool ROPE> struct PrefillEntry;
+template <int NBC>
+__global__ void __launch_bounds__(kPrefillThreads, 1) prefill_kernel(PrefillParams p, NewCounts nn) {
+    prefill_body<NBC, false>(p, nn);
+}
+template <int NBC>
+__global__ void __maxnreg__(176) prefill_rope_kernel(PrefillParams p, NewCounts nn) {
+    prefill_body<NBC, true>(p, nn);
+}
+template <int NBC> struct PrefillEntry<NBC, false> { static constexpr auto fn = prefill_kernel<NBC>; };
+template <int NBC> struct PrefillEntry<NBC, true> { static constexpr auto fn = prefill_rope_kernel<NBC>; };
 
 // Rt (fp32, [L][d][m]) -> its two fp16 pieces, transposed to [L][2][m][d] (channel contiguous).
 __global__ void split_projection_kernel(const float *Rt, uint16_t *Rh, int n_layers, int m) {
@@ -1349,14 +1363,14 @@ static cudaError_t launch_prefill_t(const PrefillParams &p, const NewCounts &nn,
     int dev = 0;
     cudaGetDevice(&dev);
     if (dev >= 0 && dev < 64 && !attr_set[dev]) {
-        cudaError_t e = cudaFuncSetAttribute(prefill_kernel<NBC, ROPE>, cudaFuncAttributeMaxDynamicSharedMemorySize, SM::kTotal);
+        cudaError_t e = cudaFuncSetAttribute(PrefillEntry<NBC, ROPE>::fn, cudaFuncAttributeMaxDynamicSharedMemorySize, SM::kTotal);
         if (e != cudaSuccess) return e;
         // the largest shared-memory split, not the smallest that fits this kernel: the rest is for the value kernel's blocks
-        e = cudaFuncSetAttribute(prefill_kernel<NBC, ROPE>, cudaFuncAttributePreferredSharedMemoryCarveout, cudaSharedmemCarveoutMaxShared);
+        e = cudaFuncSetAttribute(PrefillEntry<NBC, ROPE>::fn, cudaFuncAttributePreferredSharedMemoryCarveout, cudaSharedmemCarveoutMaxShared);
         if (e != cudaSuccess) return e;
         attr_set[dev] = true;
     }
-    prefill_kernel<NBC, ROPE><<<(unsigned)grid, kPrefillThreads, SM::kTotal, st>>>(p, nn);
+    PrefillEntry<NBC, ROPE>::fn<<<(unsigned)grid, kPrefillThreads, SM::kTotal, st>>>(p, nn);
     return cudaGetLastError();
 }
 
