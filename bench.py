@@ -93,7 +93,8 @@ class ClockSampler(threading.Thread):
 
     def stop(self):
         self._stop_evt.set()
-        self.join(timeout=2)
+        if self.ident is not None:                  # started
+            self.join(timeout=2)
         med = float(np.median(self.samples)) if self.samples else None
         return {"sm_mhz": med, "sm_max_mhz": self.max_mhz, "reasons": sorted(self.reasons),
                 "samples": len(self.samples)}
@@ -356,9 +357,11 @@ def run_prefill(args, w, pdist, rank, world, local):
     stream = torch.cuda.current_stream()
     times = []
     launches0 = 0
+    sampler = ClockSampler(gpu_index())
     for i in range(args.warmup + args.steps):
         if i == args.warmup:
             launches0 = cache.h1b_launch_count()
+            sampler.start()
         cache.h1b_reset(-1)                           # synchronous, outside the timed call
         e0, e1 = torch.cuda.Event(enable_timing=True), torch.cuda.Event(enable_timing=True)
         pdist.barrier(); torch.cuda.synchronize()
@@ -368,6 +371,7 @@ def run_prefill(args, w, pdist, rank, world, local):
         torch.cuda.synchronize()
         if i >= args.warmup:
             times.append(e0.elapsed_time(e1))
+    clocks = sampler.stop()
     cache.h1b_poll_status()
     launches = cache.h1b_launch_count() - launches0
     ms = pdist.max_over_ranks([float(np.mean(times))], dev)[0]
@@ -379,7 +383,7 @@ def run_prefill(args, w, pdist, rank, world, local):
             "steps": args.steps, "warmup": args.warmup, "ms_per_step": ms, "higher_is_better": True,
             "scaling": "weak", "vs_baseline": None, "dtype": "f16 x f16 -> f32 (projection), f32 (quantiser)",
             "data": "synthetic", "config": {"workload": "%s: %s" % (w.name, w.notes), "l2": "5.1 GB per step, larger than L2"},
-            "gpu_launches": int(launches),
+            "gpu_launches": int(launches), "clocks": clocks,
             "roofline": {"bound": "hbm", "kernel": "prefill_kernel (keys, tcgen05) beside prefill_values_kernel (values), one call",
                          "achieved": alg_bytes / (ms * 1e-3) / 1e9,
                          "peak": peak, "peak_kind": peak_kind, "unit": "GB/s", "frac": alg_bytes / (ms * 1e-3) / 1e9 / peak,
