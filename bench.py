@@ -133,6 +133,8 @@ def run_ours(args):
                              name="%s[m=%d,G=%d]" % (w.name, args.sketch_bits or w.sketch_bits, args.group_size or w.group_size))
     if args.fp16_values:                              # Table V's "1-bit keys only" row: values stay fp16
         w = h1b_synth.scaled(w, name=w.name + "[fp16 values]")
+    if args.layers:                                   # fewer layers of the same shape: small enough for a profiler capture
+        w = h1b_synth.scaled(w, n_layers=args.layers, name="%s[%d layers]" % (w.name, args.layers))
     if args.rope:                                     # rotary embedding fused into the append and the query sketch
         w = h1b_synth.scaled(w, name=w.name + "[rope]")
     if args.workload == "c5_prefill":
@@ -486,6 +488,7 @@ def main():
                          "'heads' = the ranks split the heads of the same sequences, strong scaling")
     ap.add_argument("--page-tokens", type=int, default=0,
                     help="> 0: a paged cache with pages of this many tokens, scattered over the pool (variant)")
+    ap.add_argument("--layers", type=int, default=0, help="> 0: only this many layers of the workload's shape (variant)")
     ap.add_argument("--rope", action="store_true",
                     help="rotate keys and queries (rotary position embedding) inside the append and the query sketch (variant)")
     ap.add_argument("--fp16-values", action="store_true", help="keep values in fp16 (the 1-bit-keys-only ablation row)")
