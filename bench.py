@@ -448,8 +448,17 @@ def cpu_baseline(sample_layers: int = 1, steps: int = 3, warmup: int = 1, sample
         s.step()
     times = [s.step() for _ in range(max(1, steps))]
     step_s = float(np.mean(times)) * s.w.n_layers / len(s.layers)
-    return {"value": s.w.batch / step_s, "unit": UNIT, "cores": s.oracle.threads(), "kind": "oracle",
-            "sample": s.describe(len(times)), "ms_per_step": step_s * 1e3}
+    cores = s.oracle.threads()
+    out = {"value": s.w.batch / step_s, "unit": UNIT, "cores": cores, "kind": "oracle",
+           "sample": s.describe(len(times)), "ms_per_step": step_s * 1e3}
+    if cores > 1:                                       # the same sample once more on a single thread
+        s.oracle.set_threads(1)
+        try:
+            one_s = s.step() * s.w.n_layers / len(s.layers)
+        finally:
+            s.oracle.set_threads(cores)
+        out["one_thread"] = {"value": s.w.batch / one_s, "unit": UNIT, "ms_per_step": one_s * 1e3, "sample": "one timed step"}
+    return out
 
 
 def run_reference(args):

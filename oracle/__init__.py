@@ -81,6 +81,8 @@ def _load():
             lib.h1bo_entry_bytes.argtypes = [ctypes.c_int, ctypes.c_int, ctypes.c_int]
             lib.h1bo_threads.restype = ctypes.c_int
             lib.h1bo_threads.argtypes = []
+            lib.h1bo_set_threads.restype = ctypes.c_int
+            lib.h1bo_set_threads.argtypes = [ctypes.c_int]
             _lib = lib
     return _lib
 
@@ -303,3 +305,8 @@ def entry_bytes(d: int, m: int, G: int) -> int:
 
 def threads() -> int:
     return int(_load().h1bo_threads())
+
+
+def set_threads(n: int) -> int:
+    """OpenMP threads the layer drivers may use from now on; returns the previous setting."""
+    return int(_load().h1bo_set_threads(int(n)))

@@ -433,6 +433,20 @@ long h1bo_entry_bytes(int d, int m, int G)
     return (long)m / 8 + (long)d / 2 + (long)(d / G) * 4;
 }
 
+/* How many OpenMP threads the layer drivers may use from now on (n < 1: leave it). Changes no arithmetic:
+ * the units that the threads share are independent. Returns the previous setting. */
+int h1bo_set_threads(int n)
+{
+#ifdef _OPENMP
+    const int before = omp_get_max_threads();
+    if (n >= 1) omp_set_num_threads(n);
+    return before;
+#else
+    (void)n;
+    return 1;
+#endif
+}
+
 int h1bo_threads(void)
 {
 #ifdef _OPENMP
