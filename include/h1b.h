@@ -35,7 +35,7 @@
  *     All cached tokens [0, len) are attended, the one just appended included.
  *     Query head h reads KV head h / (Hq / Hkv).  An empty sequence gives zeros.
  *   - d = 64 (the paper's 60M model: 12 layers, 8 heads of 64 channels) runs
- *     through the same 128-channel kernels, two heads per cache slab; nothing
+ *     through the same 128-channel kernels, two KV heads per cache slab; nothing
  *     of that shows at this interface (shapes, exports and results are per
  *     head), except the restrictions listed at h1b_config.head_dim and that
  *     h1b_decode_attention_multi() takes one query token only.
@@ -68,7 +68,7 @@ typedef struct {
     int32_t n_layers;      /* L >= 1                                                   */
     int32_t n_q_heads;     /* Hq; a multiple of Hkv, Hq / Hkv <= 16                    */
     int32_t n_kv_heads;    /* Hkv                                                      */
-    int32_t head_dim;      /* d: 128, or 64 (then Hq == Hkv, even, G = 32, m <= 256)    */
+    int32_t head_dim;      /* d: 128, or 64 (then Hkv even, G = 32, m <= 256)           */
     int32_t sketch_bits;   /* m: 64, 128, 256 or 512                                   */
     int32_t group_size;    /* G: 32, or 128 (= d: one scale and zero per value vector)  */
     int32_t max_batch;     /* sequences the cache can hold (<= 256)                    */

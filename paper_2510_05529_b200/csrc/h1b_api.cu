@@ -50,9 +50,9 @@ int check_config(const h1b_config *c) {
     if (c->sketch_bits != 64 && c->sketch_bits != 128 && c->sketch_bits != 256 && c->sketch_bits != 512)
         return H1B_ERR_UNSUPPORTED;
     if (c->head_dim == kHeadDim / 2) {
-        // 64-wide heads travel in pairs through the 128-wide kernels: multi-head attention with an even number of
-        // heads, groups of 32 channels (or fp16 values), and both sketches of a pair within 512 bits
-        if (gq != 1 || (c->n_kv_heads & 1) || c->group_size != kGroup || c->sketch_bits > 256) return H1B_ERR_UNSUPPORTED;
+        // 64-wide heads travel in pairs through the 128-wide kernels: an even number of KV heads, groups of 32
+        // channels (or fp16 values), and both sketches of a pair within 512 bits
+        if ((c->n_kv_heads & 1) || c->group_size != kGroup || c->sketch_bits > 256) return H1B_ERR_UNSUPPORTED;
     } else if (c->head_dim != kHeadDim || (c->group_size != kGroup && c->group_size != kHeadDim)) {
         return H1B_ERR_UNSUPPORTED;
     }
@@ -418,7 +418,9 @@ static int enqueue_decode(h1b_ctx *ctx, int layer_begin, int n_layers, float inv
                           cudaStream_t st, uint32_t *qwords, float *partial, size_t partial_bytes,
                           bool may_profile, int *launches, int Tq = 1) {
     // (query token, query head) pairs that share a KV head, and how many of them one work item takes
-    const int vheads = ctx->plan.gq * Tq, gqk = vheads >= 3 ? 4 : vheads, vgroups = (vheads + gqk - 1) / gqk;
+    // (two 64-wide heads per slab: an item takes one query head of each KV head of the pair)
+    const int vheads = ctx->plan.gq * Tq, gqk = ctx->paired ? 2 : (vheads >= 3 ? 4 : vheads);
+    const int vgroups = (vheads + gqk - 1) / gqk;
     const size_t max_items = partial_bytes / ((size_t)gqk * kPartStride * sizeof(float));
     // slabs x groups of virtual heads: the units a split divides. When the scratch cannot hold one partial for
     // every unit of the call (many query tokens on a large batch), the layers go through it in several passes,

@@ -1104,8 +1104,11 @@ __global__ void __launch_bounds__(kDecodeWarps * 32, decode_min_blocks(GQ, NG)) 
         const int gq = p.Hq / p.Hkv, vheads = gq * p.Tq;
 #pragma unroll
         for (int h = 0; h < GQ; ++h) {
-            // a group's surplus slots repeat the last virtual head (their results are never read)
-            const int v = min(vg * GQ + h, vheads - 1), tq = v / gq, hq = kvh * gq + v % gq;
+            // a group's surplus slots repeat the last virtual head (their results are never read).
+            // PAIRED: the slab's query heads are [heads of its first KV head | heads of its second]; item vg takes
+            // the vg-th of each half, so that slot h reads half h of the slab
+            const int v = PAIRED ? (h * (gq >> 1) + vg) : min(vg * GQ + h, vheads - 1);
+            const int tq = PAIRED ? 0 : v / gq, hq = kvh * gq + (PAIRED ? v : v % gq);
             limit[h] = min(t_end, len - p.Tq + tq + 1);
             const uint32_t *qp = p.qwords + (((size_t)(layer * p.max_batch + b) * p.Tq + tq) * p.Hq + hq) * MWH;
 #pragma unroll
@@ -1265,7 +1268,9 @@ __global__ void __launch_bounds__(kHeadDim) combine_kernel(DecodeParams p) {
     grid_dependency_wait();                                     // the partials come from the attention kernel
     const int len = p.len[(p.layer_begin + ll) * p.max_batch + b];
     const int kvh = hq / gq;
-    const int v = tq * gq + hq % gq, vg = v / p.gqk, hh = v % p.gqk;          // virtual head, its group and slot
+    // virtual head, its group and slot (two 64-wide heads per slab: slot = which KV head of the pair, group = which of its query heads)
+    const int v = tq * gq + hq % gq;
+    const int vg = p.paired ? v % (gq >> 1) : v / p.gqk, hh = p.paired ? v / (gq >> 1) : v % p.gqk;
     const long slab_local = ((long)ll * p.B + b) * p.Hkv + kvh;
     const int n_chunks = (len + 31) >> 5, ns = p.splits;       // splits that got no chunk wrote nothing: skipped below
     const SplitShare share = split_share(n_chunks, ns);

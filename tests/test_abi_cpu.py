@@ -63,7 +63,7 @@ def test_entry_and_workspace_bytes(lib):
 
 
 @pytest.mark.parametrize("kw", [
-    dict(n_layers=0), dict(n_q_heads=3, n_kv_heads=2), dict(head_dim=32), dict(head_dim=64, n_q_heads=8, n_kv_heads=4),
+    dict(n_layers=0), dict(n_q_heads=3, n_kv_heads=2), dict(head_dim=32), dict(head_dim=64, n_q_heads=9, n_kv_heads=3),
     dict(head_dim=64, n_q_heads=3, n_kv_heads=3), dict(head_dim=64, sketch_bits=512), dict(sketch_bits=100),
     dict(sketch_bits=96), dict(group_size=64), dict(max_batch=0), dict(max_batch=257), dict(max_seq=0),
     dict(n_q_heads=17, n_kv_heads=1),

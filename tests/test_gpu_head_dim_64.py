@@ -32,6 +32,18 @@ def test_all_heads_append_and_decode(lens, appends, inv_tau, splits):
     assert tot["max_err"] < 2e-3
 
 
+@pytest.mark.parametrize("hq, hkv, fp16_like", [(8, 2, False), (16, 4, False), (6, 2, False), (14, 2, False), (32, 8, False)])
+def test_grouped_query_heads(hq, hkv, fp16_like):
+    """64-wide heads with several query heads per KV head (the small Llama-style shapes: 32/8, 14/2): the KV heads
+    still travel in pairs, and a work item takes one query head of each KV head of its pair."""
+    w = gpt2_small(n_q_heads=hq, n_kv_heads=hkv)
+    tot = full_parity(w, [333, 97], appends=[100, 40, 193], splits=0 if hq != 16 else 3)
+    print("d = 64, GQA", hq, hkv, tot)
+    tot = full_parity(gpt2_small(n_q_heads=hq, n_kv_heads=hkv, sketch_bits=256, n_layers=1), [200, 1], inv_tau=50.0,
+                      rope_table=h1b_synth.rope_table(256, 32))
+    print("d = 64, GQA, m = 256, rope", hq, hkv, tot)
+
+
 @pytest.mark.parametrize("m", [64, 256])
 def test_other_sketch_widths(m):
     tot = full_parity(gpt2_small(sketch_bits=m, n_q_heads=4, n_kv_heads=4), [200, 90])
@@ -102,7 +114,7 @@ def test_step_and_projection_round_trip_and_limits():
         cache.h1b_decode_attention_multi(torch.zeros((2, 2, 2, 4, 64), dtype=torch.float16, device="cuda"), 16.0)
     assert err.value.code == -3
     cache.close()
-    for bad in (dict(n_q_heads=8, n_kv_heads=4), dict(n_q_heads=3, n_kv_heads=3), dict(group_size=64), dict(sketch_bits=512)):
+    for bad in (dict(n_q_heads=9, n_kv_heads=3), dict(n_q_heads=3, n_kv_heads=3), dict(group_size=64), dict(sketch_bits=512)):
         cfg = binding.make_config(**{**dict(n_layers=1, n_q_heads=4, n_kv_heads=4, head_dim=64, sketch_bits=128, group_size=32),
                                      **bad})
         assert binding.h1b_cache_bytes(cfg) == 0
