@@ -37,8 +37,7 @@
  *   - d = 64 (the paper's 60M model: 12 layers, 8 heads of 64 channels) runs
  *     through the same 128-channel kernels, two KV heads per cache slab; nothing
  *     of that shows at this interface (shapes, exports and results are per
- *     head), except the restrictions listed at h1b_config.head_dim and that
- *     h1b_decode_attention_multi() takes one query token only.
+ *     head), except the restrictions listed at h1b_config.head_dim.
  *   - With H1B_FLAG_FP16_VALUES (the "1-bit keys only" row of the ablation,
  *     Table V) values are cached as the fp16 numbers they arrive as: no codes,
  *     scales or zero-points; the output is softmax(alpha/tau) * V.

@@ -555,8 +555,6 @@ int h1b_decode_attention_multi(h1b_ctx *ctx, int layer_begin, int n_layers, cons
     if (rc != H1B_OK) return rc;
     if (Tq < 1 || Tq > kMaxQueryTokens)
         return fail(ctx, H1B_ERR_INVALID_ARG, "Tq = %d outside [1, %d]", Tq, kMaxQueryTokens);
-    if (ctx->paired && Tq > 1)
-        return fail(ctx, H1B_ERR_UNSUPPORTED, "several query tokens are not built for head dimension 64");
     for (int l = layer_begin; l < layer_begin + n_layers; ++l)
         for (int b = 0; b < B; ++b)
             if (ctx->len_host[(size_t)l * ctx->cfg.max_batch + b] < Tq)
@@ -566,7 +564,7 @@ int h1b_decode_attention_multi(h1b_ctx *ctx, int layer_begin, int n_layers, cons
     int launches = 0;
     // rows of the sketch are (sequence, query token, query head): Tq * Hq "heads" per sequence
     SketchParams sp = sketch_params(ctx, layer_begin, n_layers, q, B, at<uint32_t>(ctx, ctx->plan.qwords));
-    sp.Hq = Tq * ctx->cfg.n_q_heads;
+    sp.Hq = Tq * sp.Hq;                                 // (n_q_heads, or with 64-wide heads the pairs of them)
     sp.Tq = Tq;
     NewCounts none;
     std::memset(&none, 0, sizeof none);

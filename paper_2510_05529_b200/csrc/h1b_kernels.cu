@@ -1106,9 +1106,10 @@ __global__ void __launch_bounds__(kDecodeWarps * 32, decode_min_blocks(GQ, NG)) 
         for (int h = 0; h < GQ; ++h) {
             // a group's surplus slots repeat the last virtual head (their results are never read).
             // PAIRED: the slab's query heads are [heads of its first KV head | heads of its second]; item vg takes
-            // the vg-th of each half, so that slot h reads half h of the slab
-            const int v = PAIRED ? (h * (gq >> 1) + vg) : min(vg * GQ + h, vheads - 1);
-            const int tq = PAIRED ? 0 : v / gq, hq = kvh * gq + (PAIRED ? v : v % gq);
+            // the same (query token, head in group) of each half, so that slot h reads half h of the slab
+            const int gqu = gq >> 1;                            // PAIRED: query heads per KV head
+            const int v = PAIRED ? vg : min(vg * GQ + h, vheads - 1);
+            const int tq = PAIRED ? v / gqu : v / gq, hq = kvh * gq + (PAIRED ? h * gqu + v % gqu : v % gq);
             limit[h] = min(t_end, len - p.Tq + tq + 1);
             const uint32_t *qp = p.qwords + (((size_t)(layer * p.max_batch + b) * p.Tq + tq) * p.Hq + hq) * MWH;
 #pragma unroll
@@ -1269,8 +1270,8 @@ __global__ void __launch_bounds__(kHeadDim) combine_kernel(DecodeParams p) {
     const int len = p.len[(p.layer_begin + ll) * p.max_batch + b];
     const int kvh = hq / gq;
     // virtual head, its group and slot (two 64-wide heads per slab: slot = which KV head of the pair, group = which of its query heads)
-    const int v = tq * gq + hq % gq;
-    const int vg = p.paired ? v % (gq >> 1) : v / p.gqk, hh = p.paired ? v / (gq >> 1) : v % p.gqk;
+    const int v = tq * gq + hq % gq, jj = hq % gq, gqu = gq >> 1;
+    const int vg = p.paired ? tq * gqu + jj % gqu : v / p.gqk, hh = p.paired ? jj / gqu : v % p.gqk;
     const long slab_local = ((long)ll * p.B + b) * p.Hkv + kvh;
     const int n_chunks = (len + 31) >> 5, ns = p.splits;       // splits that got no chunk wrote nothing: skipped below
     const SplitShare share = split_share(n_chunks, ns);

@@ -110,9 +110,6 @@ def test_step_and_projection_round_trip_and_limits():
             Kf[b, n] = kn[l, b, 0]; Vf[b, n] = vn[l, b, 0]
         ref = oracle.layer(f16_bits(Kf), f16_bits(Vf), lens + 1, f16_bits(qn[l]), Rt[l], 16.0, 32)
         check_output(out[l], ref, ("step, d = 64", l))
-    with pytest.raises(binding.H1BError) as err:                       # several query tokens: not built for d = 64
-        cache.h1b_decode_attention_multi(torch.zeros((2, 2, 2, 4, 64), dtype=torch.float16, device="cuda"), 16.0)
-    assert err.value.code == -3
     cache.close()
     for bad in (dict(n_q_heads=9, n_kv_heads=3), dict(n_q_heads=3, n_kv_heads=3), dict(group_size=64), dict(sketch_bits=512)):
         cfg = binding.make_config(**{**dict(n_layers=1, n_q_heads=4, n_kv_heads=4, head_dim=64, sketch_bits=128, group_size=32),

@@ -121,6 +121,21 @@ def test_other_formats(m, G, fp16_values):
     cache.close()
 
 
+@pytest.mark.parametrize("hq, hkv, Tq, m, fp16_values", [(4, 4, 3, 128, False), (8, 2, 5, 64, False), (2, 2, 16, 256, False),
+                                                         (12, 4, 2, 128, True)])
+def test_heads_of_64_channels(hq, hkv, Tq, m, fp16_values):
+    """Two KV heads per slab inside the library: an item takes the same (query token, head in group) of both."""
+    w = h1b_synth.scaled(W["c6_60m_8k"], n_layers=2, batch=2, n_q_heads=hq, n_kv_heads=hkv, sketch_bits=m, context=400)
+    cache, Rt, K, V, lens = _fill(w, [333, 70], fp16_values=fp16_values)
+    q = _queries(w, Tq, seed=11)
+    out = cache.h1b_decode_attention_multi(q.cuda(), 16.0).cpu().numpy()
+    cache.h1b_poll_status()
+    assert out.shape == (2, 2, Tq, hq, 64)
+    worst, flips = _check(w, cache, Rt, K, V, q, lens, out, 16.0, fp16_values)
+    print("multi-query, d = 64", hq, hkv, Tq, m, "max err", worst, "flips", flips)
+    cache.close()
+
+
 def test_one_query_token_is_the_decode_call_and_bad_counts_are_rejected():
     w = h1b_synth.scaled(W["c1_tiny"], batch=2, n_q_heads=4, n_kv_heads=2)
     cache, Rt, K, V, lens = _fill(w, [300, 5])
