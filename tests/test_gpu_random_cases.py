@@ -1,5 +1,5 @@
 """GPU parity on generated cases (hypothesis, derandomised so that every run draws the same cases): head
-shapes, sketch widths, group sizes, ragged lengths, the way the rows arrive (one call, many calls, single
+shapes, head dimensions, sketch widths, group sizes, rotary embedding on or off, ragged lengths, the way the rows arrive (one call, many calls, single
 tokens), forced split counts and temperatures, each checked by the full protocol (append bit for bit outside
 the decision window, isolated decode, end to end) against the fp64 oracle."""
 import numpy as np
@@ -26,15 +26,21 @@ def cases(draw):
     pieces.append(max(max(lens), 1))                              # whatever is left arrives in one last call
     splits = draw(st.sampled_from([0, 0, 1, 2, 3, 5, 8, 23, 64]))
     inv_tau = draw(st.sampled_from([1e-3, 1.0, 16.0, 50.0, 400.0]))
-    return hq, hkv, m, G, batch, lens, pieces, splits, inv_tau
+    d = draw(st.sampled_from([128, 128, 64]))
+    if d == 64:                                                   # 64-wide heads: KV heads in pairs, groups of 32, m <= 256
+        hq, hkv = draw(st.sampled_from([(2, 2), (4, 4), (8, 2), (6, 2), (16, 4)]))
+        m, G = draw(st.sampled_from([(64, 32), (128, 32), (256, 32)]))
+    rope = draw(st.booleans())
+    return hq, hkv, m, G, batch, lens, pieces, splits, inv_tau, d, rope
 
 
-@settings(max_examples=30, deadline=None, derandomize=True, database=None,
+@settings(max_examples=40, deadline=None, derandomize=True, database=None,
           suppress_health_check=list(HealthCheck))
 @given(case=cases())
 def test_generated_cases(case):
-    hq, hkv, m, G, batch, lens, pieces, splits, inv_tau = case
+    hq, hkv, m, G, batch, lens, pieces, splits, inv_tau, d, rope = case
     w = h1b_synth.scaled(W["c1_tiny"], batch=batch, n_layers=2, n_q_heads=hq, n_kv_heads=hkv, sketch_bits=m,
-                         group_size=G)
-    tot = full_parity(w, lens, inv_tau=inv_tau, appends=pieces, splits=splits)
+                         group_size=G, head_dim=d)
+    table = h1b_synth.rope_table(max(max(lens), 1), d // 2) if rope else None
+    tot = full_parity(w, lens, inv_tau=inv_tau, appends=pieces, splits=splits, rope_table=table)
     print("generated", case, tot)
