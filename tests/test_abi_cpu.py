@@ -88,3 +88,18 @@ def test_null_context_calls_return_error_codes(lib):
     h = ctypes.c_void_p()
     assert lib.h1b_init_projection(ctypes.byref(c), 0, None, None, 0, None, ctypes.byref(h)) == -2
     assert b"workspace" in lib.h1b_last_error(None)
+
+
+def test_header_is_plain_c_and_the_library_links_from_c(lib, tmp_path):
+    """include/h1b.h compiled as strict C99 by gcc, linked against the built library, run (no GPU needed)."""
+    import subprocess
+    here = os.path.dirname(os.path.abspath(__file__))
+    root = os.path.dirname(here)
+    lib_path = build.build_library()
+    libdir = os.path.dirname(lib_path)
+    exe = str(tmp_path / "abi_probe")
+    subprocess.run(["gcc", "-std=c99", "-pedantic", "-Wall", "-Wextra", "-Werror", "-I", os.path.join(root, "include"),
+                    os.path.join(here, "abi_probe.c"), "-o", exe, "-L", libdir, "-l:" + os.path.basename(lib_path),
+                    "-Wl,-rpath," + libdir], check=True)
+    out = subprocess.run([exe], check=True, capture_output=True, text=True)
+    assert out.stdout.strip() == "ok"
