@@ -130,3 +130,52 @@ def test_replay_into_a_full_cache_drops_the_rows_and_reports_it():
     assert np.array_equal(out.cpu().numpy()[0, 0], full[0, 0])
     cache.h1b_poll_status()
     cache.close()
+
+
+@pytest.mark.parametrize("fp16_values", [False, True])
+def test_a_long_append_in_a_graph_appends_at_the_current_end_every_replay(fp16_values):
+    """A chunk of 128 prompt tokens per call (the tensor-core append, whose two kernels fork onto a second stream and
+    join back) recorded once and replayed: each replay lands behind the previous one, like direct calls."""
+    w = h1b_synth.scaled(W["c1_tiny"], n_layers=2, batch=2, n_q_heads=2, n_kv_heads=2)
+    direct, Rt = make_cache(w, max_seq=600, fp16_values=fp16_values)
+    graphed, _ = make_cache(w, max_seq=600, Rt=Rt, fp16_values=fp16_values)
+    lens = np.array([50, 3], np.int32)
+    K0, V0 = _prefill(w, direct, lens)
+    _prefill(w, graphed, lens)
+    ks = torch.zeros((w.n_layers, w.batch, 128, w.n_kv_heads, w.head_dim), dtype=torch.float16, device="cuda")
+    vs = torch.zeros_like(ks)
+    chunks = []
+    graph = None
+    for s in range(3):
+        kc = torch.stack([h1b_synth.kv_rows(w, l, 128, stream=60 + s)[0] for l in range(w.n_layers)])
+        vc = torch.stack([h1b_synth.kv_rows(w, l, 128, stream=60 + s)[1] for l in range(w.n_layers)])
+        chunks.append((kc, vc))
+        direct.h1b_append_kv(kc.cuda(), vc.cuda())
+        ks.copy_(kc); vs.copy_(vc)
+        if s == 0:
+            graphed.h1b_append_kv(ks, vs)                # an ordinary call first (it also sets kernel attributes)
+            torch.cuda.synchronize()
+            graph = torch.cuda.CUDAGraph()
+            with torch.cuda.graph(graph):
+                graphed.h1b_append_kv(ks, vs)
+            # the capture itself ran nothing, but the host's copy of the lengths moved: put it back
+            graphed.h1b_sync_lengths()
+        else:
+            graph.replay()
+        torch.cuda.synchronize()
+    graphed.h1b_sync_lengths()
+    graphed.h1b_poll_status()
+    assert np.array_equal(graphed.h1b_get_lengths(1)[:2], lens + 3 * 128)
+    for l in range(w.n_layers):
+        for b in range(w.batch):
+            n = int(lens[b]) + 3 * 128
+            for g in range(w.n_kv_heads):
+                ea, eb = direct.h1b_export_cache(l, b, g, 0, n), graphed.h1b_export_cache(l, b, g, 0, n)
+                assert all(np.array_equal(x, y) for x, y in zip(ea, eb) if x is not None)
+                if fp16_values:
+                    assert np.array_equal(direct.h1b_export_values(l, b, g, 0, n), graphed.h1b_export_values(l, b, g, 0, n))
+    q = torch.stack([h1b_synth.queries(w, l) for l in range(w.n_layers)]).cuda()
+    assert np.array_equal(direct.h1b_decode_attention(q, INV_TAU).cpu().numpy(),
+                          graphed.h1b_decode_attention(q, INV_TAU).cpu().numpy())
+    direct.close()
+    graphed.close()
