@@ -376,6 +376,29 @@ def run_prefill(args, w, pdist, rank, world, local):
     clocks = sampler.stop()
     cache.h1b_poll_status()
     launches = cache.h1b_launch_count() - launches0
+    prompt_attention = None
+    if args.prompt_attention:
+        # attention for every token of the prompt over the cache just built (blocks of 16 query tokens, causal)
+        q = torch.stack([h1b_synth.normal_fp16(h1b_synth.layer_seed(w, l, 7), (w.batch, w.context, w.n_q_heads, w.head_dim),
+                                               device=str(dev)) for l in range(w.n_layers)])
+        out = torch.empty(q.shape, dtype=torch.float32, device=dev)
+        n_pa = max(1, min(args.steps, 3))
+        l0 = cache.h1b_launch_count()
+        cache.h1b_prefill_attention(q, INV_TAU, out=out)                # warm-up
+        torch.cuda.synchronize()
+        per_call = cache.h1b_launch_count() - l0
+        e0, e1 = torch.cuda.Event(enable_timing=True), torch.cuda.Event(enable_timing=True)
+        e0.record(stream)
+        for _ in range(n_pa):
+            cache.h1b_prefill_attention(q, INV_TAU, out=out)
+        e1.record(stream)
+        torch.cuda.synchronize()
+        cache.h1b_poll_status()
+        pa_ms = pdist.max_over_ranks([e0.elapsed_time(e1) / n_pa], dev)[0]
+        prompt_attention = {"value": pdist.whole_job_rate(w.batch * w.context, world, pa_ms * 1e-3), "unit": UNIT,
+                            "ms_per_call": pa_ms, "calls": n_pa, "gpu_launches_per_call": int(per_call),
+                            "how": "h1b_prefill_attention over all %d prompt tokens, %d layers at once" % (w.context, w.n_layers)}
+        del q, out
     ms = pdist.max_over_ranks([float(np.mean(times))], dev)[0]
     rows = w.n_layers * w.batch * w.context * w.n_kv_heads
     alg_bytes = rows * (2 * w.head_dim * 2 + binding.h1b_entry_bytes(cfg))       # fp16 K and V in, packed entry out
@@ -391,6 +414,8 @@ def run_prefill(args, w, pdist, rank, world, local):
                          "peak": peak, "peak_kind": peak_kind, "unit": "GB/s", "frac": alg_bytes / (ms * 1e-3) / 1e9 / peak,
                          "alg_bytes_per_launch": alg_bytes, "traffic": None,
                          "tensor_tflops": rows * w.head_dim * w.sketch_bits * 2 * 2 / (ms * 1e-3) / 1e12}}
+    if prompt_attention:
+        line["prompt_attention"] = prompt_attention
     cache.close()
     pdist.finish()
     if rank == 0:
@@ -497,6 +522,8 @@ def main():
                          "'heads' = the ranks split the heads of the same sequences, strong scaling")
     ap.add_argument("--page-tokens", type=int, default=0,
                     help="> 0: a paged cache with pages of this many tokens, scattered over the pool (variant)")
+    ap.add_argument("--prompt-attention", action="store_true",
+                    help="c5_prefill: also time attention for every prompt token over the compressed cache (variant)")
     ap.add_argument("--layers", type=int, default=0, help="> 0: only this many layers of the workload's shape (variant)")
     ap.add_argument("--rope", action="store_true",
                     help="rotate keys and queries (rotary position embedding) inside the append and the query sketch (variant)")

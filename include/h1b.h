@@ -183,6 +183,18 @@ int h1b_decode_attention(h1b_ctx *ctx, int layer_begin, int n_layers, const void
 int h1b_decode_attention_multi(h1b_ctx *ctx, int layer_begin, int n_layers, const void *q, int Tq,
                                float inv_tau, void *out, int B, void *stream);
 
+/* Attention for a whole run of Tn query tokens per sequence (a prompt, or a
+ * chunk of one): the queries are the sequences' last Tn cached tokens (append
+ * their keys and values first), query token i attends to cached tokens
+ * [0, len - Tn + i + 1). Any Tn >= 1: the call walks the run in blocks of
+ * H1B_MAX_QUERY_TOKENS query tokens, each block one pass of the same kernels
+ * over the part of the cache it may see. q: DEVICE fp16 [n_layers][B][Tn][Hq][d];
+ * out: DEVICE float32, same shape. Every sequence must hold at least Tn
+ * tokens in every layer of the call (H1B_ERR_INVALID_ARG otherwise). With the
+ * rotary option each query is rotated at the position of its token. */
+int h1b_prefill_attention(h1b_ctx *ctx, int layer_begin, int n_layers, const void *q, int Tn,
+                          float inv_tau, void *out, int B, void *stream);
+
 /* One whole decode step on device tensors, all L layers: append one new token per
  * sequence (Eq. 2, Eq. 4) and run decode attention over the grown cache (Eq. 3,
  * Eq. 5). Same result as h1b_append_kv(Tn = 1) followed by h1b_decode_attention(),

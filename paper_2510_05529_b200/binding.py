@@ -64,6 +64,8 @@ def load_library(rebuild: bool = True) -> ctypes.CDLL:
                                                 ctypes.c_int, vp]),
         "h1b_decode_attention_multi": (ctypes.c_int, [vp, ctypes.c_int, ctypes.c_int, vp, ctypes.c_int, ctypes.c_float,
                                                       vp, ctypes.c_int, vp]),
+        "h1b_prefill_attention": (ctypes.c_int, [vp, ctypes.c_int, ctypes.c_int, vp, ctypes.c_int, ctypes.c_float,
+                                                 vp, ctypes.c_int, vp]),
         "h1b_decode_attention_static": (ctypes.c_int, [vp, ctypes.c_int, ctypes.c_int, vp, ctypes.c_float, vp,
                                                        ctypes.c_int, vp]),
         "h1b_decode_step": (ctypes.c_int, [vp, vp, vp, vp, ctypes.c_float, vp, ctypes.c_int, vp]),
@@ -218,6 +220,21 @@ class H1BCache:
         op = _dev_ptr(out, torch.float32, "out")
         self._check(self.lib.h1b_decode_attention_multi(self._h, layer_begin, int(q.shape[0]), qp, int(q.shape[2]),
                                                         float(inv_tau), op, int(q.shape[1]), _stream_ptr(stream)))
+        return out
+
+    def h1b_prefill_attention(self, q: torch.Tensor, inv_tau: float, out: torch.Tensor | None = None,
+                              layer_begin: int = 0, stream=None) -> torch.Tensor:
+        """q: fp16 CUDA [n_layers, B, Tn, Hq, d], the sequences' last Tn cached tokens (any Tn) -> out fp32, same shape."""
+        qp = _dev_ptr(q, torch.float16, "q")
+        if q.dim() != 5 or q.shape[3] != self.cfg.n_q_heads or q.shape[4] != self.cfg.head_dim:
+            raise ValueError("q must be [n_layers, B, Tn, Hq, d]")
+        if out is None:
+            out = torch.empty(q.shape, dtype=torch.float32, device=q.device)
+        op = _dev_ptr(out, torch.float32, "out")
+        if out.shape != q.shape:
+            raise ValueError("out must have q's shape")
+        self._check(self.lib.h1b_prefill_attention(self._h, layer_begin, int(q.shape[0]), qp, int(q.shape[2]),
+                                                   float(inv_tau), op, int(q.shape[1]), _stream_ptr(stream)))
         return out
 
     def h1b_decode_step(self, k: torch.Tensor, v: torch.Tensor, q: torch.Tensor, inv_tau: float,

@@ -402,6 +402,8 @@ static SketchParams sketch_params(h1b_ctx *ctx, int layer_begin, int n_layers, c
     sp.rope = rope_ref(ctx);
     sp.len = at<int32_t>(ctx, ctx->plan.len);
     sp.Tq = 1;
+    sp.q_seq_rows = sp.Hq;
+    sp.q_tail = 0;
     return sp;
 }
 
@@ -416,7 +418,7 @@ static void commit_lengths(h1b_ctx *ctx, int layer_begin, int n_layers, int B, c
 // not depend on how well the host's view of the lengths matches the device's.
 static int enqueue_decode(h1b_ctx *ctx, int layer_begin, int n_layers, float inv_tau, void *out, int B,
                           cudaStream_t st, uint32_t *qwords, float *partial, size_t partial_bytes,
-                          bool may_profile, int *launches, int Tq = 1) {
+                          bool may_profile, int *launches, int Tq = 1, int q_tail = 0, int out_seq_tokens = 0) {
     // (query token, query head) pairs that share a KV head, and how many of them one work item takes
     // (two 64-wide heads per slab: an item takes one query head of each KV head of the pair)
     const int vheads = ctx->plan.gq * Tq, gqk = ctx->paired ? 2 : (vheads >= 3 ? 4 : vheads);
@@ -433,7 +435,7 @@ static int enqueue_decode(h1b_ctx *ctx, int layer_begin, int n_layers, float inv
     const long slabs = per_layer * pass_layers;
     int maxlen = 1;
     for (int l = layer_begin; l < layer_begin + n_layers; ++l)
-        for (int b = 0; b < B; ++b) maxlen = std::max(maxlen, ctx->len_host[(size_t)l * ctx->cfg.max_batch + b]);
+        for (int b = 0; b < B; ++b) maxlen = std::max(maxlen, ctx->len_host[(size_t)l * ctx->cfg.max_batch + b] - q_tail);
     long splits = ctx->forced_splits > 0 ? ctx->forced_splits : kTargetItems / slabs;
     const long max_splits = std::max(1, maxlen / kMinSplitTokens);
     if (ctx->forced_splits <= 0 && splits > max_splits) splits = max_splits;
@@ -456,6 +458,8 @@ static int enqueue_decode(h1b_ctx *ctx, int layer_begin, int n_layers, float inv
     dp.groups = ctx->plan.groups;
     dp.splits = (int)splits;
     dp.Tq = Tq; dp.gqk = gqk; dp.vgroups = vgroups;
+    dp.q_tail = q_tail;
+    dp.out_seq_rows = (out_seq_tokens > 0 ? out_seq_tokens : Tq) * ctx->cfg.n_q_heads;
     dp.paired = ctx->paired ? 1 : 0;
     dp.out_dim = ctx->ucfg.head_dim;
     dp.c2 = (float)(2.0 * (double)inv_tau * 1.4426950408889634 / (double)ctx->ucfg.sketch_bits);
@@ -465,7 +469,7 @@ static int enqueue_decode(h1b_ctx *ctx, int layer_begin, int n_layers, float inv
         ev1 = ctx->events[ctx->events_used + 1];
         ctx->events_used += 2;
     }
-    const size_t layer_out = (size_t)B * Tq * ctx->cfg.n_q_heads * (size_t)ctx->ucfg.head_dim;   // floats of one layer
+    const size_t layer_out = (size_t)B * dp.out_seq_rows * (size_t)ctx->ucfg.head_dim;           // floats of one layer
     for (int done = 0; done < n_layers; done += pass_layers) {
         dp.layer_begin = layer_begin + done;
         dp.n_layers = std::min(pass_layers, n_layers - done);
@@ -566,11 +570,47 @@ int h1b_decode_attention_multi(h1b_ctx *ctx, int layer_begin, int n_layers, cons
     SketchParams sp = sketch_params(ctx, layer_begin, n_layers, q, B, at<uint32_t>(ctx, ctx->plan.qwords));
     sp.Hq = Tq * sp.Hq;                                 // (n_q_heads, or with 64-wide heads the pairs of them)
     sp.Tq = Tq;
+    sp.q_seq_rows = sp.Hq;
     NewCounts none;
     std::memset(&none, 0, sizeof none);
     H1B_CUDA(ctx, launch_prepare(nullptr, &sp, none, st, &launches));
     rc = enqueue_decode(ctx, layer_begin, n_layers, inv_tau, out, B, st, sp.qwords, at<float>(ctx, ctx->plan.partial),
                         ctx->plan.partial_bytes, true, &launches, Tq);
+    ctx->launches += launches;
+    return rc;
+}
+
+int h1b_prefill_attention(h1b_ctx *ctx, int layer_begin, int n_layers, const void *q, int Tn, float inv_tau, void *out,
+                          int B, void *stream) {
+    int rc = check_decode_args(ctx, layer_begin, n_layers, q, inv_tau, out, B);
+    if (rc != H1B_OK) return rc;
+    if (Tn < 1) return fail(ctx, H1B_ERR_INVALID_ARG, "Tn = %d < 1", Tn);
+    for (int l = layer_begin; l < layer_begin + n_layers; ++l)
+        for (int b = 0; b < B; ++b)
+            if (ctx->len_host[(size_t)l * ctx->cfg.max_batch + b] < Tn)
+                return fail(ctx, H1B_ERR_INVALID_ARG, "layer %d sequence %d holds %d < Tn = %d tokens", l, b,
+                            ctx->len_host[(size_t)l * ctx->cfg.max_batch + b], Tn);
+    cudaStream_t st = static_cast<cudaStream_t>(stream);
+    int launches = 0;
+    NewCounts none;
+    std::memset(&none, 0, sizeof none);
+    const size_t d = ctx->ucfg.head_dim, Hq = ctx->ucfg.n_q_heads;
+    // blocks of up to kMaxQueryTokens query tokens, first to last; block j ends q_tail tokens before the sequences' ends
+    for (int t0 = 0; t0 < Tn && rc == H1B_OK; t0 += kMaxQueryTokens) {
+        const int Tq = std::min(kMaxQueryTokens, Tn - t0), q_tail = Tn - t0 - Tq;
+        SketchParams sp = sketch_params(ctx, layer_begin, n_layers,
+                                        static_cast<const uint16_t *>(q) + (size_t)t0 * Hq * d, B,
+                                        at<uint32_t>(ctx, ctx->plan.qwords));
+        const int rows_per_token = sp.Hq;               // query heads, or with 64-wide heads pairs of them
+        sp.Hq = Tq * rows_per_token;
+        sp.Tq = Tq;
+        sp.q_seq_rows = Tn * rows_per_token;
+        sp.q_tail = q_tail;
+        H1B_CUDA(ctx, launch_prepare(nullptr, &sp, none, st, &launches));
+        rc = enqueue_decode(ctx, layer_begin, n_layers, inv_tau, static_cast<float *>(out) + (size_t)t0 * Hq * d, B, st,
+                            sp.qwords, at<float>(ctx, ctx->plan.partial), ctx->plan.partial_bytes, false, &launches, Tq,
+                            q_tail, Tn);
+    }
     ctx->launches += launches;
     return rc;
 }
@@ -872,6 +912,8 @@ int h1b_debug_scores(h1b_ctx *ctx, int layer, int seq, int kv_head, const void *
     sp.rope = rope_ref(ctx);
     sp.len = at<int32_t>(ctx, ctx->plan.len) + (size_t)layer * ctx->cfg.max_batch + seq;
     sp.Tq = 1;
+    sp.q_seq_rows = 1;
+    sp.q_tail = 0;
     if (uses_rope(ctx) && ctx->rope_positions < 1)
         return fail(ctx, H1B_ERR_INVALID_ARG, "H1B_FLAG_ROPE: h1b_set_rope_table has not been called");
     int launches = 0;

@@ -51,9 +51,11 @@ __device__ __forceinline__ int rope_clamp(const RopeRef &rope, int pos) { return
 // Returns, for threads 0..31, the packed word of row `tid` of the tile (other threads: unspecified).
 // x_rows: fp16 [n_rows][128], row-contiguous; rows beyond n_rows read as zero.
 // With rope.table set, the rows are first rotated at the positions sm.pos[row] (written by the caller before the call).
+// run > 0: the tile's rows are flat rows row0 .. of a layer whose rows come in runs of `run` contiguous rows, the
+// runs `run_stride` rows apart (x_rows then points at flat row 0); run == 0: x_rows points at the tile's first row.
 __device__ __forceinline__ uint32_t project_tile(ProjSmem &sm, const uint16_t *__restrict__ x_rows, int n_rows,
                                                  const float *__restrict__ Rt_layer, int m, int word,
-                                                 const RopeRef &rope) {
+                                                 const RopeRef &rope, int row0 = 0, int run = 0, int run_stride = 0) {
     const int tid = threadIdx.x, lane = tid & 31, warp = tid >> 5;
     // All global loads of the tile are issued before the first shared-memory store, so that the block pays
     // one memory round trip, not one per loop iteration.
@@ -70,7 +72,11 @@ __device__ __forceinline__ uint32_t project_tile(ProjSmem &sm, const uint16_t *_
     for (int k = 0; k < kProjRows * (kHeadDim / 2) / kProjThreads; ++k) {
         const int e = tid + k * kProjThreads, row = e >> 6, c2 = e & 63;
         xv[k] = __float2half2_rn(0.f);
-        if (row < n_rows) xv[k] = __ldg(reinterpret_cast<const __half2 *>(x_rows + (size_t)row * kHeadDim) + c2);
+        if (row < n_rows) {
+            size_t at = (size_t)row;
+            if (run > 0) { const int flat = row0 + row; at = (size_t)(flat / run) * run_stride + flat % run; }
+            xv[k] = __ldg(reinterpret_cast<const __half2 *>(x_rows + at * kHeadDim) + c2);
+        }
     }
 #pragma unroll
     for (int k = 0; k < kHeadDim * 8 / kProjThreads; ++k) {
@@ -224,10 +230,10 @@ __global__ void __launch_bounds__(kProjThreads) prepare_kernel(AppendParams ap, 
         if (sp.rope.table && threadIdx.x < kProjRows) {
             const int row = row0 + min((int)threadIdx.x, n_rows - 1);
             const int h = row % sp.Hq, b = row / sp.Hq, tq = h / (sp.Hq / sp.Tq);
-            sm.pos[threadIdx.x] = rope_clamp(sp.rope, sp.len[layer * sp.max_batch + b] + nn.v[b] - sp.Tq + tq);
+            sm.pos[threadIdx.x] = rope_clamp(sp.rope, sp.len[layer * sp.max_batch + b] + nn.v[b] - sp.q_tail - sp.Tq + tq);
         }
-        const uint32_t bits = project_tile(sm, sp.q + ((size_t)ll * q_rows + row0) * kHeadDim, n_rows,
-                                           sp.Rt + (size_t)layer * kHeadDim * m, m, word, sp.rope);
+        const uint32_t bits = project_tile(sm, sp.q + (size_t)ll * sp.B * sp.q_seq_rows * kHeadDim, n_rows,
+                                           sp.Rt + (size_t)layer * kHeadDim * m, m, word, sp.rope, row0, sp.Hq, sp.q_seq_rows);
         if ((int)threadIdx.x < n_rows) {
             const int row = row0 + threadIdx.x;
             const int h = row % sp.Hq, b = row / sp.Hq;
@@ -1042,7 +1048,7 @@ __global__ void __launch_bounds__(kDecodeWarps * 32, decode_min_blocks(GQ, NG)) 
     const int layer = p.layer_begin + ll;
     launch_dependents();                                        // the combine grid may be scheduled behind this one
     grid_dependency_wait();                                     // lengths, query sketches and the new token come from the prepare kernel
-    const int len = p.len[layer * p.max_batch + b];
+    const int len = max(p.len[layer * p.max_batch + b] - p.q_tail, 0);
     // The sequence's chunks are dealt out evenly: split s takes chunks [s C / S, (s + 1) C / S) of the C the
     // sequence has now (whatever the host believed when it chose S), so the items of a sequence differ by one chunk at most.
     const SplitShare share = split_share((len + 31) >> 5, p.splits);
@@ -1267,7 +1273,7 @@ __global__ void __launch_bounds__(kHeadDim) combine_kernel(DecodeParams p) {
     const int b = (blockIdx.x / (p.Hq * p.Tq)) % p.B;
     const int ll = blockIdx.x / (p.Hq * p.Tq * p.B);
     grid_dependency_wait();                                     // the partials come from the attention kernel
-    const int len = p.len[(p.layer_begin + ll) * p.max_batch + b];
+    const int len = max(p.len[(p.layer_begin + ll) * p.max_batch + b] - p.q_tail, 0);
     const int kvh = hq / gq;
     // virtual head, its group and slot (two 64-wide heads per slab: slot = which KV head of the pair, group = which of its query heads)
     const int v = tq * gq + hq % gq, jj = hq % gq, gqu = gq >> 1;
@@ -1303,7 +1309,8 @@ __global__ void __launch_bounds__(kHeadDim) combine_kernel(DecodeParams p) {
     __syncthreads();
     const float n4 = (s_num[0][tid] + s_num[1][tid]) + (s_num[2][tid] + s_num[3][tid]);
     const float d4 = (s_den[0] + s_den[1]) + (s_den[2] + s_den[3]);
-    if (tid < p.out_dim) p.out[(size_t)blockIdx.x * p.out_dim + tid] = (n_chunks > 0) ? n4 / d4 : 0.f;
+    const size_t out_row = ((size_t)ll * p.B + b) * p.out_seq_rows + (size_t)tq * p.Hq + hq;
+    if (tid < p.out_dim) p.out[out_row * p.out_dim + tid] = (n_chunks > 0) ? n4 / d4 : 0.f;
 }
 
 // Test helper: score of every cached token of one slab against one sketch.

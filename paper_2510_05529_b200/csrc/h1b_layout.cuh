@@ -170,6 +170,10 @@ struct SketchParams {           // query sketch
     RopeRef rope;
     const int32_t *len;         // [L][max_batch] (read only when rope.table is set)
     int Tq;
+    // A block of query tokens out of a longer run (prompt attention): the rows of a sequence are Hq consecutive rows,
+    // sequences are q_seq_rows rows apart (== Hq: the plain contiguous layout), and q_tail cached tokens lie behind
+    // the block's last query token (their positions are counted back from there).
+    int q_seq_rows, q_tail;
 };
 
 struct DecodeParams {
@@ -185,6 +189,9 @@ struct DecodeParams {
     // tokens [0, len - Tq + i + 1). The Tq * (Hq/Hkv) (query token, query head) pairs that share a KV head are "virtual
     // heads" v = i * (Hq/Hkv) + head-in-group, handled `gqk` at a time by one work item (vgroups items per slab and split).
     int Tq, gqk, vgroups;
+    // Prompt attention: the query tokens are not the sequence's last Tq but end q_tail tokens before its end (the
+    // kernels then work on len - q_tail), and a sequence's outputs are out_seq_rows (token, head) rows apart.
+    int q_tail, out_seq_rows;
     // Head dimension 64: two heads share a 128-channel slab (head h of the pair in channels 64h.., key words [h m/32, ..)),
     // so Hkv counts pairs, Hq heads, m_words the words of both sketches, and a head's output has out_dim = 64 channels.
     int paired, out_dim;
