@@ -11,6 +11,10 @@
 //                        Hamming distances, fp16 tensor-core P.V on the integer codes
 //                        with each weight split into two fp16 parts.
 //   combine_kernel       merges the split partials (flash-decoding style).
+//   prefill_kernel /     long appends: Eq. 2 as a dense contraction on the tensor cores (tcgen05,
+//   prefill_rope_kernel  accumulators in TMEM), the second one rotating each key tile in shared
+//                        memory first (rotary position embedding);
+//   prefill_values_kernel  Eq. 4 for the same appends, side by side with the key kernel.
 #include "h1b_kernels.h"
 #include "h1b_ptx.cuh"
 
