@@ -236,8 +236,12 @@ __global__ void __launch_bounds__(kProjThreads) prepare_kernel(AppendParams ap, 
             const int h = row % sp.Hq, b = row / sp.Hq, tq = h / (sp.Hq / sp.Tq);
             sm.pos[threadIdx.x] = rope_clamp(sp.rope, sp.len[layer * sp.max_batch + b] + nn.v[b] - sp.q_tail - sp.Tq + tq);
         }
-        const uint32_t bits = project_tile(sm, sp.q + (size_t)ll * sp.B * sp.q_seq_rows * kHeadDim, n_rows,
-                                           sp.Rt + (size_t)layer * kHeadDim * m, m, word, sp.rope, row0, sp.Hq, sp.q_seq_rows);
+        // (the usual case, a sequence's rows directly behind the previous sequence's, needs no per-row address arithmetic)
+        const bool apart = sp.q_seq_rows != sp.Hq;
+        const uint16_t *q_at = apart ? sp.q + (size_t)ll * sp.B * sp.q_seq_rows * kHeadDim
+                                     : sp.q + ((size_t)ll * q_rows + row0) * kHeadDim;
+        const uint32_t bits = project_tile(sm, q_at, n_rows, sp.Rt + (size_t)layer * kHeadDim * m, m, word, sp.rope,
+                                           row0, apart ? sp.Hq : 0, sp.q_seq_rows);
         if ((int)threadIdx.x < n_rows) {
             const int row = row0 + threadIdx.x;
             const int h = row % sp.Hq, b = row / sp.Hq;
