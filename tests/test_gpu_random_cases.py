@@ -2,6 +2,8 @@
 shapes, head dimensions, sketch widths, group sizes, rotary embedding on or off, ragged lengths, the way the rows arrive (one call, many calls, single
 tokens), forced split counts and temperatures, each checked by the full protocol (append bit for bit outside
 the decision window, isolated decode, end to end) against the fp64 oracle."""
+import os
+
 import numpy as np
 import pytest
 from hypothesis import HealthCheck, given, settings, strategies as st
@@ -34,7 +36,8 @@ def cases(draw):
     return hq, hkv, m, G, batch, lens, pieces, splits, inv_tau, d, rope
 
 
-@settings(max_examples=40, deadline=None, derandomize=True, database=None,
+@settings(max_examples=int(os.environ.get("H1B_GENERATED_CASES", "40")),   # set it higher for a soak run
+          deadline=None, derandomize=True, database=None,
           suppress_health_check=list(HealthCheck))
 @given(case=cases())
 def test_generated_cases(case):
