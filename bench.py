@@ -314,7 +314,7 @@ def run_ours(args):
     line = {
         "metric": METRIC, "value": value, "unit": UNIT, "n_gpus": world, "steps": steps, "warmup": warmup,
         "ms_per_step": ms_per_step, "higher_is_better": True, "scaling": "strong" if shard_heads else "weak", "vs_baseline": None,
-        "dtype": "f32", "data": "synthetic",
+        "dtype": "u32 xor+popcount (scores), f32 (softmax), f16 x f16 -> f32 mma (P.V on 4-bit codes)", "data": "synthetic",
         "config": {"workload": "%s: %d layers x %d/%d heads, d=%d, m=%d, batch %d per GPU, %s; fp16 K/V ~ N(0,1)%s, one "
                                "projection per layer" % (w.name, w.n_layers, w.n_q_heads, w.n_kv_heads, w.head_dim,
                                                          w.sketch_bits, w.batch, w.notes,
