@@ -133,6 +133,9 @@ def run_ours(args):
                              name="%s[m=%d,G=%d]" % (w.name, args.sketch_bits or w.sketch_bits, args.group_size or w.group_size))
     if args.fp16_values:                              # Table V's "1-bit keys only" row: values stay fp16
         w = h1b_synth.scaled(w, name=w.name + "[fp16 values]")
+    if args.q_heads or args.kv_heads:                 # another head-group shape on the same workload (variant)
+        w = h1b_synth.scaled(w, n_q_heads=args.q_heads or w.n_q_heads, n_kv_heads=args.kv_heads or w.n_kv_heads,
+                             name="%s[%d/%d heads]" % (w.name, args.q_heads or w.n_q_heads, args.kv_heads or w.n_kv_heads))
     if args.layers:                                   # fewer layers of the same shape: small enough for a profiler capture
         w = h1b_synth.scaled(w, n_layers=args.layers, name="%s[%d layers]" % (w.name, args.layers))
     if args.rope:                                     # rotary embedding fused into the append and the query sketch
@@ -524,6 +527,8 @@ def main():
                     help="> 0: a paged cache with pages of this many tokens, scattered over the pool (variant)")
     ap.add_argument("--prompt-attention", action="store_true",
                     help="c5_prefill: also time attention for every prompt token over the compressed cache (variant)")
+    ap.add_argument("--q-heads", type=int, default=0, help="override the number of query heads (variant)")
+    ap.add_argument("--kv-heads", type=int, default=0, help="override the number of KV heads (variant)")
     ap.add_argument("--layers", type=int, default=0, help="> 0: only this many layers of the workload's shape (variant)")
     ap.add_argument("--rope", action="store_true",
                     help="rotate keys and queries (rotary position embedding) inside the append and the query sketch (variant)")
