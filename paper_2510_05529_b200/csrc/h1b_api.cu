@@ -421,7 +421,8 @@ static int enqueue_decode(h1b_ctx *ctx, int layer_begin, int n_layers, float inv
                           bool may_profile, int *launches, int Tq = 1, int q_tail = 0, int out_seq_tokens = 0) {
     // (query token, query head) pairs that share a KV head, and how many of them one work item takes
     // (two 64-wide heads per slab: an item takes one query head of each KV head of the pair)
-    const int vheads = ctx->plan.gq * Tq, gqk = ctx->paired ? 2 : (vheads >= 3 ? 4 : vheads);
+    // (they then come in twos or eights: one or four of them on each of the two KV heads)
+    const int vheads = ctx->plan.gq * Tq, gqk = ctx->paired ? (vheads >= 4 ? 8 : 2) : (vheads >= 3 ? 4 : vheads);
     const int vgroups = (vheads + gqk - 1) / gqk;
     const size_t max_items = partial_bytes / ((size_t)gqk * kPartStride * sizeof(float));
     // slabs x groups of virtual heads: the units a split divides. When the scratch cannot hold one partial for

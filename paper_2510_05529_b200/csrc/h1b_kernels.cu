@@ -835,7 +835,9 @@ __global__ void set_len_kernel(int32_t *len, int n_layers, int max_batch, int se
 constexpr int kDecodeWarps = H1B_DECODE_WARPS;
 constexpr int kStages = H1B_DECODE_STAGES;
 // Resident blocks per SM that the register allocation must allow: the kernel hides latency with warps.
-constexpr int decode_min_blocks(int gq, int ng) { return ng == 0 ? 3 : (gq == 1 ? 5 : (gq == 2 ? 4 : 3)); }
+constexpr int decode_min_blocks(int gq, int ng, int mw) {
+    return gq == 8 ? (mw <= 8 ? 3 : 2) : (ng == 0 ? 3 : (gq == 1 ? 5 : (gq == 2 ? 4 : 3)));
+}
 constexpr int kHamSentinel = 1 << 20;
 
 template <int MW, int GQ, int NG>                 // NG: scale/zero pairs per value vector (4 or 1); 0 = fp16 values
@@ -865,8 +867,11 @@ struct DecodeState {
 template <int MW, int GQ, int NG, bool TAIL, bool PAIRED>
 __device__ __forceinline__ void decode_chunk(DecodeState<MW, GQ, NG> &st, const unsigned char *ch, float *p_s,
                                              int lane, const int (&n_valid)[GQ], float c2) {
-    static_assert(!PAIRED || (GQ == 2 && (NG == 4 || NG == 0)), "two 64-wide heads per slab, groups of 32 or fp16 values");
-    constexpr int GQL = PAIRED ? 1 : GQ;       // heads the accumulator columns are laid out for
+    static_assert(!PAIRED || ((GQ == 2 || GQ == 8) && (NG == 4 || NG == 0)),
+                  "two 64-wide KV heads per slab (one or four heads on each), groups of 32 or fp16 values");
+    constexpr int GQH = PAIRED ? GQ / 2 : GQ;  // (virtual) heads on each KV head of the slab
+    constexpr bool P8 = PAIRED && GQ == 8;     // four heads on each half: the columns of a channel block are its own half's heads
+    constexpr int GQL = PAIRED ? (P8 ? 4 : 1) : GQ;   // heads the accumulator columns are laid out for
     constexpr int GPF = 4 / GQL;               // value groups covered by one B fragment (4 groups per vector)
     constexpr int NB = (NG == 1) ? 1 : GQL;    // B fragments per 16-token block (one scale per vector: one fragment)
     constexpr int MWH = PAIRED ? MW / 2 : MW;  // key words of one head
@@ -892,7 +897,7 @@ __device__ __forceinline__ void decode_chunk(DecodeState<MW, GQ, NG> &st, const 
     for (int h = 0; h < GQ; ++h) {
         int ham = 0;
 #pragma unroll
-        for (int w = 0; w < MWH; ++w) ham += __popc(kw[(PAIRED ? h * MWH : 0) + w] ^ st.qw[h][w]);
+        for (int w = 0; w < MWH; ++w) ham += __popc(kw[(PAIRED ? (h / GQH) * MWH : 0) + w] ^ st.qw[h][w]);
         const bool valid = !TAIL || lane < n_valid[h];
         const int cmin = __reduce_min_sync(0xffffffffu, (TAIL && !valid) ? kHamSentinel : ham);
         scl[h] = 1.f;
@@ -901,19 +906,26 @@ __device__ __forceinline__ void decode_chunk(DecodeState<MW, GQ, NG> &st, const 
             st.hmin[h] = cmin;
             st.ssum[h] *= scl[h];                           // rescale what predates this chunk
 #pragma unroll
-            for (int g = 0; g < NG; ++g) st.accz[h][g] *= scl[h];
+            for (int g = 0; g < ((P8 && NG) ? 2 : NG); ++g) st.accz[h][g] *= scl[h];
         }
         // p carries the static factor 2 of the weights (removed when the partial is written)
         float pv = ex2_approx(fmaf((float)(st.hmin[h] - ham), c2, 1.f));
         if (TAIL) pv = valid ? pv : 0.f;
         st.ssum[h] += pv;
+        // (P8: a head only ever needs the zero-point sums of the two value groups of its own half: accz[h][0..1])
 #pragma unroll
-        for (int g = 0; g < NG; ++g) st.accz[h][g] = fmaf(pv, zf[g], st.accz[h][g]);
+        for (int g = 0; g < ((P8 && NG) ? 2 : NG); ++g)
+            st.accz[h][g] = fmaf(pv, zf[(NG > 1 && P8) ? ((h / GQH) * 2 + g) : g], st.accz[h][g]);
         p_s[h * 32 + lane] = pv;
     }
     // factors by which this lane's accumulator columns 2jq, 2jq+1 shrink when a running max moved (else 1)
-    float f0, f1;
-    if (PAIRED && NG != 0) { f0 = (jq & 1) ? scl[GQ > 1 ? 1 : 0] : scl[0]; f1 = f0; }   // columns 2jq, 2jq+1: groups of head jq % 2
+    // (P8: the channel blocks of the slab's second half take the factors of heads 4..7, f0b and f1b)
+    float f0, f1, f0b = 1.f, f1b = 1.f;
+    if (P8) {
+        f0 = (jq & 1) ? scl[GQ > 2 ? 2 : 0] : scl[0]; f1 = (jq & 1) ? scl[GQ > 3 ? 3 : 0] : scl[GQ > 1 ? 1 : 0];
+        f0b = (jq & 1) ? scl[GQ > 6 ? 6 : 0] : scl[GQ > 4 ? 4 : 0]; f1b = (jq & 1) ? scl[GQ > 7 ? 7 : 0] : scl[GQ > 5 ? 5 : 0];
+    }
+    else if (PAIRED && NG != 0) { f0 = (jq & 1) ? scl[GQ > 1 ? 1 : 0] : scl[0]; f1 = f0; }   // columns 2jq, 2jq+1: groups of head jq % 2
     else if (GQ == 1) { f0 = scl[0]; f1 = scl[0]; }
     else if (GQ == 2) { f0 = scl[0]; f1 = scl[GQ > 1 ? 1 : 0]; }
     else { f0 = (jq & 1) ? scl[GQ > 2 ? 2 : 0] : scl[0]; f1 = (jq & 1) ? scl[GQ > 3 ? 3 : 0] : scl[GQ > 1 ? 1 : 0]; }
@@ -924,41 +936,47 @@ __device__ __forceinline__ void decode_chunk(DecodeState<MW, GQ, NG> &st, const 
         // they are (one 16-byte load per channel block and lane) and B = the weights p split into hi and lo parts;
         // column n = lane/4 = (part, head). Same per-chunk zero start and fold as below.
         const int part = lane >> 4, idx = (lane >> 2) & 3;
-        const int bhead = idx < GQ ? idx : 0;                   // columns of heads the group does not have: ignored
+        const int bhead = idx < (P8 ? GQH : GQ) ? idx : 0;      // columns of heads the group does not have: ignored
         const int tp = 2 * jq + 8 * part;
-        uint32_t bf[2][2];
+        constexpr int NF = P8 ? 2 : 1;                          // P8: one fragment per half of the slab (its own four heads)
+        uint32_t bf[2][NF][2];
 #pragma unroll
         for (int vb = 0; vb < 2; ++vb) {
-            const float2 pp = *reinterpret_cast<const float2 *>(p_s + bhead * 32 + vb * 16 + tp);
-            const uint32_t hi = pack_f16x2(pp.x, pp.y);
-            const float2 hf = half2_bits_to_float2(hi);
-            const uint32_t lo = pack_f16x2((pp.x - hf.x) * 2048.f, (pp.y - hf.y) * 2048.f);
-            const uint32_t got = __shfl_xor_sync(0xffffffffu, part ? hi : lo, 16);
-            bf[vb][0] = part ? got : hi;
-            bf[vb][1] = part ? lo : got;
+#pragma unroll
+            for (int f = 0; f < NF; ++f) {
+                const float2 pp = *reinterpret_cast<const float2 *>(p_s + (f * GQH + bhead) * 32 + vb * 16 + tp);
+                const uint32_t hi = pack_f16x2(pp.x, pp.y);
+                const float2 hf = half2_bits_to_float2(hi);
+                const uint32_t lo = pack_f16x2((pp.x - hf.x) * 2048.f, (pp.y - hf.y) * 2048.f);
+                const uint32_t got = __shfl_xor_sync(0xffffffffu, part ? hi : lo, 16);
+                bf[vb][f][0] = part ? got : hi;
+                bf[vb][f][1] = part ? lo : got;
+            }
         }
-        const float g0 = (jq & 1) ? (GQ > 2 ? scl[GQ > 2 ? 2 : 0] : 1.f) : scl[0];
-        const float g1 = (jq & 1) ? (GQ > 3 ? scl[GQ > 3 ? 3 : 0] : 1.f) : (GQ > 1 ? scl[GQ > 1 ? 1 : 0] : 1.f);
+        const float g0 = P8 ? f0 : ((jq & 1) ? (GQ > 2 ? scl[GQ > 2 ? 2 : 0] : 1.f) : scl[0]);
+        const float g1 = P8 ? f1 : ((jq & 1) ? (GQ > 3 ? scl[GQ > 3 ? 3 : 0] : 1.f) : (GQ > 1 ? scl[GQ > 1 ? 1 : 0] : 1.f));
 #pragma unroll
         for (int half = 0; half < 2; ++half) {
             float tmp[4][4];
+            const int f = P8 ? half : 0;
 #pragma unroll
             for (int vb = 0; vb < 2; ++vb) {
 #pragma unroll
                 for (int i = 0; i < 4; ++i) {
                     const int cb = half * 4 + i;
                     const uint4 a = *reinterpret_cast<const uint4 *>(ch + VAL + vb * kHalfBlockBytes + cb * 512 + lane * 16);
-                    if (vb == 0) mma_f16_16816_from(tmp[i], a.x, a.y, a.z, a.w, bf[vb][0], bf[vb][1], st.zero);
-                    else mma_f16_16816(tmp[i], a.x, a.y, a.z, a.w, bf[vb][0], bf[vb][1]);
+                    if (vb == 0) mma_f16_16816_from(tmp[i], a.x, a.y, a.z, a.w, bf[vb][f][0], bf[vb][f][1], st.zero);
+                    else mma_f16_16816(tmp[i], a.x, a.y, a.z, a.w, bf[vb][f][0], bf[vb][f][1]);
                 }
             }
+            const float h0 = (P8 && half) ? f0b : g0, h1 = (P8 && half) ? f1b : g1;
 #pragma unroll
             for (int i = 0; i < 4; ++i) {
                 const int cb = half * 4 + i;
-                st.acc[cb][0] = fmaf(st.acc[cb][0], g0, tmp[i][0]);
-                st.acc[cb][1] = fmaf(st.acc[cb][1], g1, tmp[i][1]);
-                st.acc[cb][2] = fmaf(st.acc[cb][2], g0, tmp[i][2]);
-                st.acc[cb][3] = fmaf(st.acc[cb][3], g1, tmp[i][3]);
+                st.acc[cb][0] = fmaf(st.acc[cb][0], h0, tmp[i][0]);
+                st.acc[cb][1] = fmaf(st.acc[cb][1], h1, tmp[i][1]);
+                st.acc[cb][2] = fmaf(st.acc[cb][2], h0, tmp[i][2]);
+                st.acc[cb][3] = fmaf(st.acc[cb][3], h1, tmp[i][3]);
             }
         }
         __syncwarp();
@@ -970,19 +988,22 @@ __device__ __forceinline__ void decode_chunk(DecodeState<MW, GQ, NG> &st, const 
     // (group in pair, head) (GQ 2) or head (GQ 4). This lane computes the weights of ONE token pair
     // (tokens 2jq, 2jq+1 if part 0, else 2jq+8, 2jq+9), both parts, and swaps one of them with lane ^ 16.
     const int part = lane >> 4, idx = (lane >> 2) & 3;
-    const int bhead = PAIRED ? (idx >> 1) : ((GQ == 1) ? 0 : (GQ == 2 ? (idx & 1) : idx));
+    const int bhead = P8 ? idx : (PAIRED ? (idx >> 1) : ((GQ == 1) ? 0 : (GQ == 2 ? (idx & 1) : idx)));
     const int bgsel = (GQL == 1) ? idx : (GQL == 2 ? (idx >> 1) : 0);
     const int tp = 2 * jq + 8 * part;                       // first token of this lane's pair within a block
     uint32_t bf[2][NB][2];
 #pragma unroll
     for (int vb = 0; vb < 2; ++vb) {
         const float2 pp = *reinterpret_cast<const float2 *>(p_s + bhead * 32 + vb * 16 + tp);
+        // P8: groups 2 and 3 (the slab's second half) take the weights of heads 4..7
+        const float2 ppb = P8 ? *reinterpret_cast<const float2 *>(p_s + (GQH + bhead) * 32 + vb * 16 + tp) : pp;
 #pragma unroll
         for (int bi = 0; bi < NB; ++bi) {
             const int g = (NG == 1) ? 0 : bi * GPF + bgsel;
             const float2 dd = half2_bits_to_float2(
                 *reinterpret_cast<const uint32_t *>(ch + SCALE + vb * (32 * NG) + g * 32 + tp * 2));
-            const float x0 = pp.x * dd.x, x1 = pp.y * dd.y;
+            const float2 pw = (P8 && bi >= 2) ? ppb : pp;
+            const float x0 = pw.x * dd.x, x1 = pw.y * dd.y;
             const uint32_t hi = pack_f16x2(x0, x1);
             const float2 hf = half2_bits_to_float2(hi);
             const uint32_t lo = pack_f16x2((x0 - hf.x) * 2048.f, (x1 - hf.y) * 2048.f);
@@ -1012,13 +1033,14 @@ __device__ __forceinline__ void decode_chunk(DecodeState<MW, GQ, NG> &st, const 
                 else mma_f16_16816(tmp[i], a[0], a[1], a[2], a[3], bf[vb][bi][0], bf[vb][bi][1]);
             }
         }
+        const float h0 = (P8 && half) ? f0b : f0, h1 = (P8 && half) ? f1b : f1;
 #pragma unroll
         for (int i = 0; i < 4; ++i) {
             const int cb = half * 4 + i;
-            st.acc[cb][0] = fmaf(st.acc[cb][0], f0, tmp[i][0]);
-            st.acc[cb][1] = fmaf(st.acc[cb][1], f1, tmp[i][1]);
-            st.acc[cb][2] = fmaf(st.acc[cb][2], f0, tmp[i][2]);
-            st.acc[cb][3] = fmaf(st.acc[cb][3], f1, tmp[i][3]);
+            st.acc[cb][0] = fmaf(st.acc[cb][0], h0, tmp[i][0]);
+            st.acc[cb][1] = fmaf(st.acc[cb][1], h1, tmp[i][1]);
+            st.acc[cb][2] = fmaf(st.acc[cb][2], h0, tmp[i][2]);
+            st.acc[cb][3] = fmaf(st.acc[cb][3], h1, tmp[i][3]);
         }
     }
     __syncwarp();
@@ -1036,7 +1058,7 @@ __device__ __forceinline__ int split_first_chunk(int s, const SplitShare &sh) { 
 __device__ __forceinline__ bool split_is_empty(int s, const SplitShare &sh) { return sh.q == 0 && s >= sh.r; }
 
 template <int MW, int GQ, int NG, bool PAIRED, bool PAGED>
-__global__ void __launch_bounds__(kDecodeWarps * 32, decode_min_blocks(GQ, NG)) decode_split_kernel(DecodeParams p) {
+__global__ void __launch_bounds__(kDecodeWarps * 32, decode_min_blocks(GQ, NG, MW)) decode_split_kernel(DecodeParams p) {
     using SM = DecodeSmem<MW, GQ, NG>;
     constexpr int MWH = PAIRED ? MW / 2 : MW;                   // key words of one head
     constexpr int CB = SM::kChunkBytes;
@@ -1120,10 +1142,12 @@ __global__ void __launch_bounds__(kDecodeWarps * 32, decode_min_blocks(GQ, NG)) 
         for (int h = 0; h < GQ; ++h) {
             // a group's surplus slots repeat the last virtual head (their results are never read).
             // PAIRED: the slab's query heads are [heads of its first KV head | heads of its second]; item vg takes
-            // the same (query token, head in group) of each half, so that slot h reads half h of the slab
+            // the same (query token, head in group) pairs of each half, GQ / 2 of them: slots 0 .. GQ/2-1 read the
+            // slab's first half, the others its second
+            constexpr int GQH = PAIRED ? GQ / 2 : GQ;           // slots on each KV head of the slab
             const int gqu = gq >> 1;                            // PAIRED: query heads per KV head
-            const int v = PAIRED ? vg : min(vg * GQ + h, vheads - 1);
-            const int tq = PAIRED ? v / gqu : v / gq, hq = kvh * gq + (PAIRED ? h * gqu + v % gqu : v % gq);
+            const int v = PAIRED ? min(vg * GQH + h % GQH, gqu * p.Tq - 1) : min(vg * GQ + h, vheads - 1);
+            const int tq = PAIRED ? v / gqu : v / gq, hq = kvh * gq + (PAIRED ? (h / GQH) * gqu + v % gqu : v % gq);
             limit[h] = min(t_end, len - p.Tq + tq + 1);
             const uint32_t *qp = p.qwords + (((size_t)(layer * p.max_batch + b) * p.Tq + tq) * p.Hq + hq) * MWH;
 #pragma unroll
@@ -1183,7 +1207,7 @@ __global__ void __launch_bounds__(kDecodeWarps * 32, decode_min_blocks(GQ, NG)) 
         for (int o = 16; o > 0; o >>= 1) {
             st.ssum[h] += __shfl_xor_sync(0xffffffffu, st.ssum[h], o);
 #pragma unroll
-            for (int g = 0; g < NG; ++g) st.accz[h][g] += __shfl_xor_sync(0xffffffffu, st.accz[h][g], o);
+            for (int g = 0; g < ((PAIRED && GQ == 8 && NG) ? 2 : NG); ++g) st.accz[h][g] += __shfl_xor_sync(0xffffffffu, st.accz[h][g], o);
         }
     }
     // Undo the scales: codes were fed as code / kCodeScaleLo (rows r) and code / kCodeScaleHi (rows r + 8), the
@@ -1207,7 +1231,11 @@ __global__ void __launch_bounds__(kDecodeWarps * 32, decode_min_blocks(GQ, NG)) 
             if (jq < 2) {
 #pragma unroll
                 for (int hh = 0; hh < 2; ++hh) {
-                    if (PAIRED) {                               // head hh owns channel blocks 4hh .. 4hh+3: its channels 0..63
+                    if (PAIRED && GQ == 8) {                    // columns = the four heads of the channel block's own half
+                        float *dst = part_out + (size_t)((cb >> 2) * 4 + 2 * jq + hh) * kPartStride;
+                        dst[(cb & 3) * 16 + r] = v[hh];
+                        dst[(cb & 3) * 16 + r + 8] = v[2 + hh];
+                    } else if (PAIRED) {                        // head hh owns channel blocks 4hh .. 4hh+3: its channels 0..63
                         if (jq == 0 && (cb >> 2) == hh) {
                             float *dst = part_out + (size_t)hh * kPartStride;
                             dst[(cb & 3) * 16 + r] = v[hh];
@@ -1218,6 +1246,18 @@ __global__ void __launch_bounds__(kDecodeWarps * 32, decode_min_blocks(GQ, NG)) 
                         dst[cb * 16 + r] = v[hh];
                         dst[cb * 16 + r + 8] = v[2 + hh];
                     }
+                }
+            }
+        } else if (PAIRED && GQ == 8) {                         // columns = the four heads of the channel block's own half
+            if (jq < 2) {
+#pragma unroll
+                for (int hh = 0; hh < 2; ++hh) {
+                    const int base = (cb >> 2) * 4;             // first slot of that half (compile-time: cb is unrolled)
+                    const float z = (jq == 0) ? st.accz[(base + hh) < GQ ? (base + hh) : 0][gz & 1]
+                                              : st.accz[(base + 2 + hh) < GQ ? (base + 2 + hh) : 0][gz & 1];
+                    float *dst = part_out + (size_t)(base + 2 * jq + hh) * kPartStride;
+                    dst[(cb & 3) * 16 + r] = v[hh] + z;
+                    dst[(cb & 3) * 16 + r + 8] = v[2 + hh] + z;
                 }
             }
         } else if (PAIRED) {                                    // group g belongs to head g / 2 = cb / 4
@@ -1284,8 +1324,9 @@ __global__ void __launch_bounds__(kHeadDim) combine_kernel(DecodeParams p) {
     const int len = max(p.len[(p.layer_begin + ll) * p.max_batch + b] - p.q_tail, 0);
     const int kvh = hq / gq;
     // virtual head, its group and slot (two 64-wide heads per slab: slot = which KV head of the pair, group = which of its query heads)
-    const int v = tq * gq + hq % gq, jj = hq % gq, gqu = gq >> 1;
-    const int vg = p.paired ? tq * gqu + jj % gqu : v / p.gqk, hh = p.paired ? jj / gqu : v % p.gqk;
+    const int v = tq * gq + hq % gq, jj = hq % gq, gqu = gq >> 1, gqh = p.gqk >> 1;
+    const int vp = tq * gqu + jj % gqu;                         // paired: (query token, head in group) on its own KV head
+    const int vg = p.paired ? vp / gqh : v / p.gqk, hh = p.paired ? (jj / gqu) * gqh + vp % gqh : v % p.gqk;
     const long slab_local = ((long)ll * p.B + b) * p.Hkv + kvh;
     const int n_chunks = (len + 31) >> 5, ns = p.splits;       // splits that got no chunk wrote nothing: skipped below
     const SplitShare share = split_share(n_chunks, ns);
@@ -1505,6 +1546,8 @@ cudaError_t launch_decode(const DecodeParams &p, cudaStream_t st, int *launches,
         if (p.paired) {                                         // two 64-wide heads per slab
             if (gq == 2 && p.groups == 4) e = launch_decode_t<MW, 2, 4, true>(p, st);
             else if (gq == 2 && p.groups == 0) e = launch_decode_t<MW, 2, 0, true>(p, st);
+            else if (gq == 8 && p.groups == 4) e = launch_decode_t<MW, 8, 4, true>(p, st);
+            else if (gq == 8 && p.groups == 0) e = launch_decode_t<MW, 8, 0, true>(p, st);
         } else if (p.groups == 4) {
             if (gq == 1) e = launch_decode_t<MW, 1, 4>(p, st);
             else if (gq == 2) e = launch_decode_t<MW, 2, 4>(p, st);

@@ -50,8 +50,9 @@ def test_other_sketch_widths(m):
     print("d = 64, m =", m, tot)
 
 
-def test_fp16_values():
-    w = gpt2_small(n_q_heads=4, n_kv_heads=4)
+@pytest.mark.parametrize("hq, hkv", [(4, 4), (8, 2), (6, 2), (20, 4)])
+def test_fp16_values(hq, hkv):
+    w = gpt2_small(n_q_heads=hq, n_kv_heads=hkv)
     lens = np.array([150, 64], np.int32)
     cache, Rt = make_cache(w, max_seq=160, fp16_values=True)
     K = torch.stack([h1b_synth.kv_rows(w, l, 150)[0] for l in range(w.n_layers)])
@@ -65,17 +66,18 @@ def test_fp16_values():
     for l in range(w.n_layers):
         ref = oracle.layer_fp16_values(f16_bits(K[l]), f16_bits(V[l]), lens, f16_bits(q[l]), Rt[l], 16.0)
         for b in range(w.batch):
-            for h in range(w.n_kv_heads):
+            for h in range(w.n_q_heads):
                 n = int(lens[b])
-                assert np.array_equal(cache.h1b_export_values(l, b, h, 0, n), f16_bits(V[l, b, :n, h]))
-                vals = cache.h1b_export_values(l, b, h, 0, n)
-                kbits = binding.unpack_words(cache.h1b_export_cache(l, b, h, 0, n)[0], w.sketch_bits)
-                qwords, gscore = cache.h1b_debug_scores(l, b, h, q[l, b, h].contiguous().cuda(), n)
+                g = h // (w.n_q_heads // w.n_kv_heads)                  # the KV head this query head reads
+                assert np.array_equal(cache.h1b_export_values(l, b, g, 0, n), f16_bits(V[l, b, :n, g]))
+                vals = cache.h1b_export_values(l, b, g, 0, n)
+                kbits = binding.unpack_words(cache.h1b_export_cache(l, b, g, 0, n)[0], w.sketch_bits)
+                qwords, gscore = cache.h1b_debug_scores(l, b, g, q[l, b, h].contiguous().cuda(), n)
                 qbits = binding.unpack_words(qwords[None], w.sketch_bits)[0]
                 assert np.array_equal(gscore[:n], oracle.scores(qbits, kbits))
                 iso = oracle.attention_fp16_values(gscore[:n], w.sketch_bits, 16.0, vals)
                 check_output(out[l, b, h], iso, ("fp16 values, d = 64, isolated", l, b, h))
-                obits = oracle.sketch(f16_bits(K[l, b, :n, h]), Rt[l])
+                obits = oracle.sketch(f16_bits(K[l, b, :n, g]), Rt[l])
                 oq = oracle.sketch(f16_bits(q[l, b, h])[None], Rt[l])[0]
                 checked += 1
                 if np.array_equal(kbits, obits) and np.array_equal(qbits, oq):
