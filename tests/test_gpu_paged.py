@@ -58,6 +58,9 @@ def _drive(cache, w, lens, appends, K, V, q, steps):
     (64, dict(n_q_heads=4, n_kv_heads=2)),
     (256, dict(n_q_heads=4, n_kv_heads=1, sketch_bits=256)),
     (128, dict(n_q_heads=4, n_kv_heads=4, head_dim=64)),  # two heads per slab
+    (64, dict(n_q_heads=16, n_kv_heads=4, head_dim=64)),  # ... with four query heads on each
+    (32, dict(n_q_heads=6, n_kv_heads=2, head_dim=64, fp16_values=True)),
+    (160, dict(n_q_heads=16, n_kv_heads=2)),             # eight query heads per KV head: two passes of four
     (96, dict(fp16_values=True)),
 ])
 def test_paged_equals_contiguous(page_tokens, kw):
