@@ -153,7 +153,9 @@ int h1b_init_projection(const h1b_config *cfg, uint64_t seed, const float *Rt_ho
  * Sequence b of the call is sequence b of the cache.  Row tn of sequence b goes
  * to position len[layer][b] + tn; afterwards len[layer][b] += n_new[b].
  * H1B_ERR_CAPACITY (nothing written) if any sequence would exceed max_seq or,
- * with a paged cache, the pages its block table holds. */
+ * with a paged cache, the pages its block table holds.
+ * Every DEVICE tensor of this interface (k, v, q, out) must start on a 16-byte
+ * boundary: H1B_ERR_INVALID_ARG otherwise, before anything is launched. */
 int h1b_append_kv(h1b_ctx *ctx, int layer_begin, int n_layers, const void *k, const void *v,
                   const int32_t *n_new_host, int B, int Tn, void *stream);
 

@@ -485,6 +485,9 @@ static int check_decode_args(h1b_ctx *ctx, int layer_begin, int n_layers, const 
     int rc = check_layers(ctx, layer_begin, n_layers, B);
     if (rc != H1B_OK) return rc;
     if (!q || !out) return fail(ctx, H1B_ERR_NULL, "q or out is NULL");
+    // the kernels read rows with 16-byte loads: a misaligned tensor would fault on the device, so it stops here
+    if ((reinterpret_cast<uintptr_t>(q) & 15u) || (reinterpret_cast<uintptr_t>(out) & 15u))
+        return fail(ctx, H1B_ERR_INVALID_ARG, "q and out must be 16-byte aligned (got %p, %p)", q, out);
     if (!(inv_tau > 0.f) || !std::isfinite(inv_tau))
         return fail(ctx, H1B_ERR_INVALID_ARG, "inv_tau must be finite and > 0");
     return check_rope(ctx, layer_begin, n_layers, B, nullptr);
@@ -495,6 +498,8 @@ int h1b_append_kv(h1b_ctx *ctx, int layer_begin, int n_layers, const void *k, co
     int rc = check_layers(ctx, layer_begin, n_layers, B);
     if (rc != H1B_OK) return rc;
     if (!k || !v) return fail(ctx, H1B_ERR_NULL, "k or v is NULL");
+    if ((reinterpret_cast<uintptr_t>(k) & 15u) || (reinterpret_cast<uintptr_t>(v) & 15u))
+        return fail(ctx, H1B_ERR_INVALID_ARG, "k and v must be 16-byte aligned (got %p, %p)", k, v);
     if (Tn < 1) return fail(ctx, H1B_ERR_INVALID_ARG, "Tn = %d < 1", Tn);
     NewCounts nn;
     rc = make_new_counts(ctx, layer_begin, n_layers, n_new_host, B, Tn, &nn);
@@ -621,6 +626,8 @@ int h1b_decode_step_layers(h1b_ctx *ctx, int layer_begin, int n_layers, const vo
     int rc = check_decode_args(ctx, layer_begin, n_layers, q, inv_tau, out, B);
     if (rc != H1B_OK) return rc;
     if (!k || !v) return fail(ctx, H1B_ERR_NULL, "k or v is NULL");
+    if ((reinterpret_cast<uintptr_t>(k) & 15u) || (reinterpret_cast<uintptr_t>(v) & 15u))
+        return fail(ctx, H1B_ERR_INVALID_ARG, "k and v must be 16-byte aligned (got %p, %p)", k, v);
     NewCounts nn;
     rc = make_new_counts(ctx, layer_begin, n_layers, nullptr, B, 1, &nn);
     if (rc != H1B_OK) return rc;

@@ -192,6 +192,17 @@ def test_error_paths_leave_the_cache_untouched():
     for bad in (0.0, -1.0, float("inf"), float("nan")):
         with pytest.raises(binding.H1BError):
             cache.h1b_decode_attention(q, bad)
+    # a tensor that does not start on a 16-byte boundary is refused on the host (the kernels use 16-byte loads)
+    flat = torch.zeros(q.numel() + 8, dtype=torch.float16, device="cuda")
+    q_odd = flat[1:1 + q.numel()].view(q.shape)
+    with pytest.raises(binding.H1BError) as e:
+        cache.h1b_decode_attention(q_odd, 1.0)
+    assert e.value.code == -1 and "aligned" in str(e.value)
+    k_flat = torch.zeros(k.numel() + 8, dtype=torch.float16, device="cuda")
+    with pytest.raises(binding.H1BError) as e:
+        cache.h1b_append_kv(k_flat[3:3 + k.numel()].view(k.shape), k, n_new=[1, 1])
+    assert e.value.code == -1 and "aligned" in str(e.value)
+    assert cache.h1b_get_lengths(0)[:2].tolist() == [30, 30]
     with pytest.raises(binding.H1BError):
         cache.h1b_export_cache(0, 0, 0, 25, 10)
     cache.h1b_truncate(1, 10)
