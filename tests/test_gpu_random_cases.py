@@ -47,3 +47,39 @@ def test_generated_cases(case):
     table = h1b_synth.rope_table(max(max(lens), 1), d // 2) if rope else None
     tot = full_parity(w, lens, inv_tau=inv_tau, appends=pieces, splits=splits, rope_table=table)
     print("generated", case, tot)
+
+
+@st.composite
+def query_run_cases(draw):
+    d = draw(st.sampled_from([128, 64]))
+    if d == 64:
+        hq, hkv = draw(st.sampled_from([(2, 2), (4, 2), (8, 2), (6, 2)]))
+        m = draw(st.sampled_from([64, 128, 256]))
+    else:
+        hq, hkv = draw(st.sampled_from([(1, 1), (2, 2), (4, 1), (3, 1), (8, 1)]))
+        m = draw(st.sampled_from([64, 128, 256, 512]))
+    batch = draw(st.integers(1, 2))
+    Tn = draw(st.one_of(st.integers(1, 16), st.integers(17, 45)))
+    lens = [draw(st.integers(Tn, Tn + 90)) for _ in range(batch)]
+    fp16_values = draw(st.booleans())
+    splits = draw(st.sampled_from([0, 0, 1, 3]))
+    return d, hq, hkv, m, batch, Tn, lens, fp16_values, splits
+
+
+@settings(max_examples=int(os.environ.get("H1B_GENERATED_CASES", "12")), deadline=None, derandomize=True, database=None,
+          suppress_health_check=list(HealthCheck))
+@given(case=query_run_cases())
+def test_generated_runs_of_query_tokens(case):
+    """h1b_prefill_attention (and through it the several-query-token kernels) on generated shapes, every
+    (query token, head) against the oracle."""
+    from test_gpu_multi_query import _check, _fill, _queries
+    d, hq, hkv, m, batch, Tn, lens, fp16_values, splits = case
+    w = h1b_synth.scaled(W["c1_tiny"], batch=batch, n_layers=1, n_q_heads=hq, n_kv_heads=hkv, sketch_bits=m, head_dim=d)
+    cache, Rt, K, V, lens = _fill(w, lens, fp16_values=fp16_values)
+    q = _queries(w, Tn, seed=1)
+    cache.h1b_set_splits(splits)
+    out = cache.h1b_prefill_attention(q.cuda(), 16.0).cpu().numpy()
+    cache.h1b_poll_status()
+    worst, flips = _check(w, cache, Rt, K, V, q, lens, out, 16.0, fp16_values)
+    print("generated run", case, "max err", worst, "flips", flips)
+    cache.close()
