@@ -22,7 +22,9 @@ def _worker(rank, world, port, out):
     ms = [10.0 + rank, 20.0 - rank]                      # rank 0: [10, 20], rank 1: [11, 19]
     mx = d.max_over_ranks(ms)
     rate = d.whole_job_rate(1.0, world, mx[0] * 1e-3)
-    out.put((rank, mx, rate))
+    # ranks that share the heads of the SAME sequences (bench.py --shard heads): the job still makes one token per step
+    rate_heads = d.whole_job_rate(1.0, 1, mx[0] * 1e-3)
+    out.put((rank, mx, rate, rate_heads))
     d.finish()
 
 
@@ -37,9 +39,10 @@ def test_two_gloo_ranks_take_the_max_and_aggregate():
     for p in procs:
         p.join(timeout=60)
         assert p.exitcode == 0
-    for rank, mx, rate in got:
+    for rank, mx, rate, rate_heads in got:
         assert mx == [11.0, 20.0]
         assert abs(rate - 2.0 / 0.011) < 1e-9           # 2 sequences' tokens over the slowest rank's time
+        assert abs(rate_heads - 1.0 / 0.011) < 1e-9     # one sequence's tokens, however many ranks split its heads
 
 
 def test_single_process_is_identity():
