@@ -193,8 +193,12 @@ __device__ __forceinline__ void store_value_row(const uint16_t *__restrict__ v_r
 //   the rest                   value rows: Eq. 4, one warp per row                    (ap.k != null)
 // When keys/values are appended, the block that finishes last adds n_new to the lengths (every block has
 // read them by then).
+// EXTRAS: the rotary option and query rows that are not contiguous from sequence to sequence (prompt attention).
+// The plain variant carries none of that code: it is the one on the latency chain of every decode step.
+template <bool EXTRAS>
 __global__ void __launch_bounds__(kProjThreads) prepare_kernel(AppendParams ap, SketchParams sp, NewCounts nn) {
     __shared__ ProjSmem sm;
+    const RopeRef no_rope = {nullptr, 0, 0};
     launch_dependents();                                        // the attention grid may be scheduled behind this one
     const bool appending = ap.k != nullptr;
     const int mw = appending ? ap.m_words : sp.m_words, m = mw * 32;
@@ -215,9 +219,9 @@ __global__ void __launch_bounds__(kProjThreads) prepare_kernel(AppendParams ap, 
         const int row = row0 + min((int)threadIdx.x, n_rows - 1);
         const int kvh = row % ap.Hkv, tn = (row / ap.Hkv) % ap.Tn, b = row / (ap.Hkv * ap.Tn);
         const int len0 = ap.len[layer * ap.max_batch + b];
-        if (ap.rope.table && threadIdx.x < kProjRows) sm.pos[threadIdx.x] = rope_clamp(ap.rope, len0 + tn);
+        if (EXTRAS && ap.rope.table && threadIdx.x < kProjRows) sm.pos[threadIdx.x] = rope_clamp(ap.rope, len0 + tn);
         const uint32_t bits = project_tile(sm, ap.k + ((size_t)ll * k_rows + row0) * kHeadDim, n_rows,
-                                           ap.Rt + (size_t)layer * kHeadDim * m, m, word, ap.rope);
+                                           ap.Rt + (size_t)layer * kHeadDim * m, m, word, EXTRAS ? ap.rope : no_rope);
         if ((int)threadIdx.x < n_rows) {
             if (tn < nn.v[b] && len0 + nn.v[b] <= ap.seq_cap[b]) {
                 const int t = len0 + tn;
@@ -231,17 +235,17 @@ __global__ void __launch_bounds__(kProjThreads) prepare_kernel(AppendParams ap, 
         const int layer = sp.layer_begin + ll;
         const int row0 = tile * kProjRows;
         const int n_rows = min(kProjRows, q_rows - row0);
-        if (sp.rope.table && threadIdx.x < kProjRows) {
+        if (EXTRAS && sp.rope.table && threadIdx.x < kProjRows) {
             const int row = row0 + min((int)threadIdx.x, n_rows - 1);
             const int h = row % sp.Hq, b = row / sp.Hq, tq = h / (sp.Hq / sp.Tq);
             sm.pos[threadIdx.x] = rope_clamp(sp.rope, sp.len[layer * sp.max_batch + b] + nn.v[b] - sp.q_tail - sp.Tq + tq);
         }
         // (the usual case, a sequence's rows directly behind the previous sequence's, needs no per-row address arithmetic)
-        const bool apart = sp.q_seq_rows != sp.Hq;
+        const bool apart = EXTRAS && sp.q_seq_rows != sp.Hq;
         const uint16_t *q_at = apart ? sp.q + (size_t)ll * sp.B * sp.q_seq_rows * kHeadDim
                                      : sp.q + ((size_t)ll * q_rows + row0) * kHeadDim;
-        const uint32_t bits = project_tile(sm, q_at, n_rows, sp.Rt + (size_t)layer * kHeadDim * m, m, word, sp.rope,
-                                           row0, apart ? sp.Hq : 0, sp.q_seq_rows);
+        const uint32_t bits = project_tile(sm, q_at, n_rows, sp.Rt + (size_t)layer * kHeadDim * m, m, word,
+                                           EXTRAS ? sp.rope : no_rope, row0, apart ? sp.Hq : 0, sp.q_seq_rows);
         if ((int)threadIdx.x < n_rows) {
             const int row = row0 + threadIdx.x;
             const int h = row % sp.Hq, b = row / sp.Hq;
@@ -1406,7 +1410,9 @@ cudaError_t launch_prepare(const AppendParams *ap, const SketchParams *sp, const
     }
     if (blocks <= 0) return cudaSuccess;
     if (blocks > 0x7fffffffL) return cudaErrorInvalidConfiguration;
-    prepare_kernel<<<(unsigned)blocks, kProjThreads, 0, st>>>(a, q, nn);
+    const bool extras = (ap && a.rope.table) || (sp && (q.rope.table || q.q_seq_rows != q.Hq));
+    if (extras) prepare_kernel<true><<<(unsigned)blocks, kProjThreads, 0, st>>>(a, q, nn);
+    else prepare_kernel<false><<<(unsigned)blocks, kProjThreads, 0, st>>>(a, q, nn);
     ++*launches;
     return cudaGetLastError();
 }
