@@ -1059,7 +1059,6 @@ __device__ __forceinline__ SplitShare split_share(int n_chunks, int n_splits) {
     return s;
 }
 __device__ __forceinline__ int split_first_chunk(int s, const SplitShare &sh) { return s * sh.q + min(s, sh.r); }
-__device__ __forceinline__ bool split_is_empty(int s, const SplitShare &sh) { return sh.q == 0 && s >= sh.r; }
 
 template <int MW, int GQ, int NG, bool PAIRED, bool PAGED>
 __global__ void __launch_bounds__(kDecodeWarps * 32, decode_min_blocks(GQ, NG, MW)) decode_split_kernel(DecodeParams p) {
@@ -1087,7 +1086,16 @@ __global__ void __launch_bounds__(kDecodeWarps * 32, decode_min_blocks(GQ, NG, M
     // sequence has now (whatever the host believed when it chose S), so the items of a sequence differ by one chunk at most.
     const SplitShare share = split_share((len + 31) >> 5, p.splits);
     const int c0 = split_first_chunk(split, share), c1 = split_first_chunk(split + 1, share);
-    if (c0 >= c1) return;                                       // empty item: the combine skips it too
+    if (c0 >= c1) {
+        // an item with no chunk says so in its partial (distance = the sentinel, weight sum 0): the combine kernel then
+        // needs neither the length nor the split arithmetic to know which partials to skip
+        if (lane < GQ) {
+            float *po = p.partial + ((size_t)item * GQ + lane) * kPartStride;
+            po[128] = (float)kHamSentinel;
+            po[129] = 0.f;
+        }
+        return;
+    }
     const int t_end = min(len, c1 * 32);
     // chunks below c_full are attended in full by every head (the earliest query token sees len - Tq + 1 tokens)
     const int c_full = min(t_end, len - p.Tq + 1) >> 5;
@@ -1325,21 +1333,34 @@ __global__ void __launch_bounds__(kHeadDim) combine_kernel(DecodeParams p) {
     const int b = (blockIdx.x / (p.Hq * p.Tq)) % p.B;
     const int ll = blockIdx.x / (p.Hq * p.Tq * p.B);
     grid_dependency_wait();                                     // the partials come from the attention kernel
-    const int len = max(p.len[(p.layer_begin + ll) * p.max_batch + b] - p.q_tail, 0);
     const int kvh = hq / gq;
     // virtual head, its group and slot (two 64-wide heads per slab: slot = which KV head of the pair, group = which of its query heads)
     const int v = tq * gq + hq % gq, jj = hq % gq, gqu = gq >> 1, gqh = p.gqk >> 1;
     const int vp = tq * gqu + jj % gqu;                         // paired: (query token, head in group) on its own KV head
     const int vg = p.paired ? vp / gqh : v / p.gqk, hh = p.paired ? (jj / gqu) * gqh + vp % gqh : v % p.gqk;
     const long slab_local = ((long)ll * p.B + b) * p.Hkv + kvh;
-    const int n_chunks = (len + 31) >> 5, ns = p.splits;       // splits that got no chunk wrote nothing: skipped below
-    const SplitShare share = split_share(n_chunks, ns);
+    const int ns = p.splits;
     const float *base = p.partial + (((size_t)slab_local * p.vgroups + vg) * p.splits * p.gqk + hh) * kPartStride;
     const size_t stride = (size_t)p.gqk * kPartStride;
-    // the smallest Hamming distance any split saw (= the largest logit)
-    float hm = 3.0e38f;
-    for (int j = tid; j < ns; j += kHeadDim)
-        if (!split_is_empty(j, share)) hm = fminf(hm, base[j * stride + 128]);
+    constexpr float kEmpty = (float)kHamSentinel;               // what a split without tokens (for this head) reports
+    // This warp's first two splits are fetched before the block agrees on the largest logit: the loads do not depend
+    // on it, so the kernel makes one trip to memory, not two.
+    const int j0 = warp, j1 = warp + 4;
+    float s0 = kEmpty, s1 = kEmpty, d0 = 0.f, d1 = 0.f;
+    float4 a0 = make_float4(0.f, 0.f, 0.f, 0.f), a1 = a0;
+    if (j0 < ns) {
+        const float *pj = base + j0 * stride;
+        s0 = pj[128]; d0 = pj[129];
+        if (lane * 4 < p.out_dim) a0 = reinterpret_cast<const float4 *>(pj)[lane];
+    }
+    if (j1 < ns) {
+        const float *pj = base + j1 * stride;
+        s1 = pj[128]; d1 = pj[129];
+        if (lane * 4 < p.out_dim) a1 = reinterpret_cast<const float4 *>(pj)[lane];
+    }
+    // the smallest Hamming distance any split saw (= the largest logit); empty splits hold the sentinel
+    float hm = fminf(s0, s1);
+    for (int j = 8 + tid; j < ns; j += kHeadDim) hm = fminf(hm, base[j * stride + 128]);
 #pragma unroll
     for (int o = 16; o > 0; o >>= 1) hm = fminf(hm, __shfl_xor_sync(0xffffffffu, hm, o));
     if (lane == 0) s_min[warp] = hm;
@@ -1347,11 +1368,23 @@ __global__ void __launch_bounds__(kHeadDim) combine_kernel(DecodeParams p) {
     hm = fminf(fminf(s_min[0], s_min[1]), fminf(s_min[2], s_min[3]));
     float4 num = make_float4(0.f, 0.f, 0.f, 0.f);
     float den = 0.f;
+    if (s0 < kEmpty) {
+        const float wgt = exp2f((hm - s0) * p.c2);
+        num.x = wgt * a0.x; num.y = wgt * a0.y; num.z = wgt * a0.z; num.w = wgt * a0.w;
+        den = wgt * d0;
+    }
+    if (s1 < kEmpty) {
+        const float wgt = exp2f((hm - s1) * p.c2);
+        num.x = fmaf(wgt, a1.x, num.x); num.y = fmaf(wgt, a1.y, num.y);
+        num.z = fmaf(wgt, a1.z, num.z); num.w = fmaf(wgt, a1.w, num.w);
+        den = fmaf(wgt, d1, den);
+    }
 #pragma unroll 4
-    for (int j = warp; j < ns; j += 4) {
-        if (split_is_empty(j, share)) continue;
+    for (int j = warp + 8; j < ns; j += 4) {
         const float *pj = base + j * stride;
-        const float wgt = exp2f((hm - pj[128]) * p.c2);
+        const float sj = pj[128];
+        if (!(sj < kEmpty)) continue;
+        const float wgt = exp2f((hm - sj) * p.c2);
         const float4 a = (lane * 4 < p.out_dim) ? reinterpret_cast<const float4 *>(pj)[lane] : make_float4(0.f, 0.f, 0.f, 0.f);
         num.x = fmaf(wgt, a.x, num.x); num.y = fmaf(wgt, a.y, num.y);
         num.z = fmaf(wgt, a.z, num.z); num.w = fmaf(wgt, a.w, num.w);
@@ -1363,7 +1396,8 @@ __global__ void __launch_bounds__(kHeadDim) combine_kernel(DecodeParams p) {
     const float n4 = (s_num[0][tid] + s_num[1][tid]) + (s_num[2][tid] + s_num[3][tid]);
     const float d4 = (s_den[0] + s_den[1]) + (s_den[2] + s_den[3]);
     const size_t out_row = ((size_t)ll * p.B + b) * p.out_seq_rows + (size_t)tq * p.Hq + hq;
-    if (tid < p.out_dim) p.out[out_row * p.out_dim + tid] = (n_chunks > 0) ? n4 / d4 : 0.f;
+    // (no split saw a token for this head: an empty sequence)
+    if (tid < p.out_dim) p.out[out_row * p.out_dim + tid] = (hm < kEmpty) ? n4 / d4 : 0.f;
 }
 
 // Test helper: score of every cached token of one slab against one sketch.
