@@ -200,7 +200,7 @@ int h1b_prefill_attention(h1b_ctx *ctx, int layer_begin, int n_layers, const voi
 /* One whole decode step on device tensors, all L layers: append one new token per
  * sequence (Eq. 2, Eq. 4) and run decode attention over the grown cache (Eq. 3,
  * Eq. 5). Same result as h1b_append_kv(Tn = 1) followed by h1b_decode_attention(),
- * in two kernel launches instead of three.
+ * in three kernel launches instead of four.
  *   k, v  DEVICE: fp16 [L][B][1][Hkv][d]      q  DEVICE: fp16 [L][B][Hq][d]
  *   out   DEVICE: float32 [L][B][Hq][d] */
 int h1b_decode_step(h1b_ctx *ctx, const void *k, const void *v, const void *q, float inv_tau,
