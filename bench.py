@@ -144,13 +144,18 @@ def run_ours(args):
         return run_prefill(args, w, pdist, rank, world, local)
     # --shard heads: the ranks split the KV heads (and their query heads) of the SAME sequences between them: every
     # (layer, sequence, KV head) is independent, so there is still no collective on the data path; the job then
-    # produces w.batch tokens per step however many ranks there are (strong scaling)
-    shard_heads = args.shard == "heads" and world > 1
-    if shard_heads:
-        if w.n_kv_heads % world:
-            raise SystemExit("--shard heads needs the KV heads (%d) to divide by the ranks (%d)" % (w.n_kv_heads, world))
-        w = h1b_synth.scaled(w, n_q_heads=w.n_q_heads // world, n_kv_heads=w.n_kv_heads // world,
+    # produces w.batch tokens per step however many ranks there are (strong scaling). Every rank draws the inputs
+    # of the whole model from the same seeds and keeps its own heads' slice.
+    shard = None
+    w_full = w
+    if args.shard == "heads" and world > 1:
+        try:
+            shard = pdist.shard_heads(w.n_q_heads, w.n_kv_heads, rank, world, w.head_dim)
+        except ValueError as e:
+            raise SystemExit("--shard heads: %s" % e)
+        w = h1b_synth.scaled(w, n_q_heads=shard.n_q, n_kv_heads=shard.n_kv,
                              name=w.name + "[1/%d of the heads per rank]" % world)
+    shard_heads = shard is not None
     job_ranks = 1 if shard_heads else world           # how many ranks' tokens add up
     steps, warmup = args.steps, args.warmup
     Tq = max(1, args.query_tokens)                    # > 1: a step appends Tq tokens and attends for all of them at once
@@ -166,8 +171,20 @@ def run_ours(args):
                               max_batch=w.batch, max_seq=w.context - 1 + total_steps, device=local,
                               fp16_values=args.fp16_values, page_tokens=page_tokens, n_pages=pages_per_seq * w.batch,
                               rope=args.rope)
-    # each rank is its own sequence: different seeds per rank
-    wr = h1b_synth.scaled(w, index=w.index + 10 * rank)
+    # replicas: each rank is its own sequence set (different seeds per rank); head shards: one model's inputs on
+    # every rank, each keeping its heads
+    wr = w_full if shard_heads else h1b_synth.scaled(w, index=w.index + 10 * rank)
+
+    def kv_rows(l, n, stream=0):
+        K, V = h1b_synth.kv_rows(wr, l, n, device=str(dev), stream=stream)
+        if shard_heads:
+            K, V = (pdist.take_heads(t, shard.kv_begin, shard.n_kv) for t in (K, V))
+        return K, V
+
+    def queries(l, stream=0):
+        q = h1b_synth.queries(wr, l, device=str(dev), stream=stream)
+        return pdist.take_heads(q, shard.q_begin, shard.n_q) if shard_heads else q
+
     Rt = np.stack([h1b_synth.projection(h1b_synth.layer_seed(wr, l, 99), w.head_dim, w.sketch_bits)
                    for l in range(w.n_layers)])
     cache = binding.H1BCache(cfg, Rt=Rt)
@@ -178,18 +195,15 @@ def run_ours(args):
         for b in range(w.batch):
             cache.h1b_set_block_table(b, perm[b * pages_per_seq:(b + 1) * pages_per_seq])
     for l in range(w.n_layers):                       # prefill, one layer at a time
-        K, V = h1b_synth.kv_rows(wr, l, w.context - 1, device=str(dev))
+        K, V = kv_rows(l, w.context - 1)
         cache.h1b_append_kv(K.unsqueeze(0), V.unsqueeze(0), layer_begin=l, n_new=lens0)
         del K, V
     torch.cuda.synchronize()
     # per-step inputs: a pool of new tokens and queries, resident in HBM
     pool = 16
-    kn = [torch.stack([h1b_synth.kv_rows(wr, l, 1, device=str(dev), stream=100 + i)[0] for l in range(w.n_layers)])
-          for i in range(pool)]
-    vn = [torch.stack([h1b_synth.kv_rows(wr, l, 1, device=str(dev), stream=100 + i)[1] for l in range(w.n_layers)])
-          for i in range(pool)]
-    qn = [torch.stack([h1b_synth.queries(wr, l, device=str(dev), stream=i) for l in range(w.n_layers)])
-          for i in range(pool)]
+    kn = [torch.stack([kv_rows(l, 1, stream=100 + i)[0] for l in range(w.n_layers)]) for i in range(pool)]
+    vn = [torch.stack([kv_rows(l, 1, stream=100 + i)[1] for l in range(w.n_layers)]) for i in range(pool)]
+    qn = [torch.stack([queries(l, stream=i) for l in range(w.n_layers)]) for i in range(pool)]
     out = torch.empty((w.n_layers, w.batch, w.n_q_heads, w.head_dim), dtype=torch.float32, device=dev)
     stream = torch.cuda.current_stream()
 
