@@ -33,10 +33,10 @@ if ROOT not in sys.path:
 METRIC = "decode-attn tokens/s (7B shape, 8k ctx): append 1 token + decode attention over 32 layers"
 UNIT = "tokens/s"
 INV_TAU = 16.0
-# DRAM traffic of one decode_split_kernel launch (dram__bytes_read.sum + dram__bytes_write.sum) per
-# algorithmic byte, from the ncu capture summarised in profiles/decode_split_kernel_c2_7b_8k.md
-# (816.5 MB moved for 806.0 MB needed at 8199 cached tokens). Traffic grows in proportion to the cached
-# tokens, so the bench scales it to the context it actually ran.
+# DRAM traffic of one decode_split_kernel launch (dram__bytes_read.sum + dram__bytes_write.sum, one ncu capture)
+# per algorithmic byte: 816.5 MB moved for 806.0 MB needed at 8199 cached tokens of the default workload. Traffic
+# grows in proportion to the cached tokens, so the bench scales it to the context it actually ran; the line says
+# where the ratio was taken (`traffic_ratio_measured_at`), so that a stale one shows.
 NCU_TRAFFIC_PER_ALGORITHMIC_BYTE = 1.0130
 
 

@@ -21,7 +21,10 @@
  *     workspace.
  *   - Asynchrony: h1b_append_kv() and h1b_decode_attention() only enqueue work
  *     on `stream` (a cudaStream_t passed as void*, NULL = the default stream).
- *     Use one stream at a time per context.
+ *     Use one stream at a time per context.  Contexts may be created and
+ *     used from several host threads (one thread at a time per context): the
+ *     per-device set-up the library keeps (kernel attributes, the address of
+ *     its built-in scratch array) is made under a lock, in h1b_init_projection().
  *   - Symbols: d = head_dim, m = sketch_bits (the paper's b), G = group_size,
  *     L = n_layers, Hq / Hkv = query / KV heads, B = sequences in the call.
  *     The projection is held as Rt[d][m] (row-major), Rt[i][j] = R[j][i] for
@@ -114,9 +117,9 @@ size_t h1b_entry_bytes(const h1b_config *cfg /* HOST */);
  * h1b_set_block_table: sequence `seq` owns pages_host[0 .. n) (HOST int32, each
  * in [0, n_pages), n * page_tokens <= max_seq rounded up to whole pages), in
  * this order. May grow or shrink a table between steps; entries that cover
- * cached tokens must keep their pages. The library does not check that two
- * sequences do not share a page. Stream-ordered like the other calls.
- * H1B_ERR_INVALID_ARG on a contiguous cache, on bad page numbers, or when fewer
+ * cached tokens must keep their pages. Stream-ordered like the other calls.
+ * H1B_ERR_INVALID_ARG on a contiguous cache, on bad page numbers, on a page
+ * that is listed twice or that another sequence's table holds, or when fewer
  * pages than the sequence's cached tokens need. */
 int h1b_set_block_table(h1b_ctx *ctx, int seq, const int32_t *pages_host, int n, void *stream);
 
@@ -180,7 +183,9 @@ int h1b_decode_attention(h1b_ctx *ctx, int layer_begin, int n_layers, const void
  *   q    DEVICE: fp16 [n_layers][B][Tq][Hq][d]      1 <= Tq <= H1B_MAX_QUERY_TOKENS
  *   out  DEVICE: float32 [n_layers][B][Tq][Hq][d]
  * H1B_ERR_INVALID_ARG if some sequence of the call holds fewer than Tq tokens.
- * Tq = 1 is h1b_decode_attention(). */
+ * Tq = 1 is h1b_decode_attention(). The split-K scratch of the workspace is
+ * sized for the largest call this allows (max_batch sequences, Tq = 16), so no
+ * valid call runs out of it. */
 #define H1B_MAX_QUERY_TOKENS 16
 int h1b_decode_attention_multi(h1b_ctx *ctx, int layer_begin, int n_layers, const void *q, int Tq,
                                float inv_tau, void *out, int B, void *stream);
@@ -216,8 +221,9 @@ int h1b_decode_step_layers(h1b_ctx *ctx, int layer_begin, int n_layers, const vo
 
 /* Stream capture. h1b_append_kv(), h1b_decode_attention(), h1b_decode_step() and
  * h1b_decode_step_layers() only enqueue kernels, so they may be recorded into a
- * CUDA graph (make one ordinary call of each kind first: the first call sets
- * kernel attributes). The kernels read the sequence lengths from device memory,
+ * CUDA graph; nothing has to be called first (every kernel attribute a context
+ * can need is set when the context is created). The kernels read the sequence
+ * lengths from device memory,
  * so every replay appends at, and attends up to, the then-current end of each
  * sequence. Frozen at capture time: the pointers, B, n_new and the number of
  * splits per sequence (which chunks a split takes is worked out on the device
@@ -249,15 +255,24 @@ int h1b_sync_lengths(h1b_ctx *ctx, void *stream);
  *
  * Same arguments, same result and same errors as h1b_decode_attention(), plus:
  *   - H1B_ERR_CAPACITY, with the needed and the available byte counts in
- *     h1b_last_error(), when even one split per sequence does not fit:
- *     n_layers * B * Hkv * (Hq/Hkv) * 528 bytes of partials plus
- *     L * max_batch * Hq * m/8 bytes of sketches must be <= 8 MiB. When more
- *     splits would fit the automatic choice, fewer are used (slower, same result
- *     up to summation order).
+ *     h1b_last_error(), when ONE layer of the call does not fit with one split
+ *     per sequence:
+ *         B * Hkv * ceil(g / k) * k * 528 bytes of partials, g = Hq / Hkv and
+ *         k = g for g <= 2, else 4 (heads go through in groups of four); with
+ *         d = 64, two KV heads share a cache slab: Hkv / 2 * ceil(2g / k) * k
+ *         with k = 2 for g = 1, else 8
+ *     plus L * max_batch * Hq * m/8 bytes of sketches (all layers and sequences
+ *     of the context, rounded up to 256) must be <= 8 MiB (8 388 608). A call
+ *     with more layers than fit at once sends them through the array in passes,
+ *     and fewer splits per sequence are used than the automatic choice when
+ *     those would not fit (slower, same result up to summation order).
  *   - the context's device must be the current device.
- *   - the first call on each device looks up the array's device address
- *     (cudaGetSymbolAddress) and keeps it; make that first call outside any
- *     stream capture.
+ *   - nothing is looked up or set up by the call itself: the array's device
+ *     address was obtained (cudaGetSymbolAddress) when the first context on
+ *     this device was created, in h1b_init_projection(), which also loaded
+ *     the kernels it launches. From its first use the call is therefore only
+ *     kernel launches; create the context outside any region in which
+ *     allocation is forbidden, and outside any stream capture.
  * All contexts and all calls in the process share the one array per device, and
  * it keeps whatever the last call left in it; nothing in it has to be
  * initialised, since a call reads only what it has written itself. Two calls
@@ -326,6 +341,33 @@ int h1b_export_values(h1b_ctx *ctx, int layer, int seq, int kv_head, int t0, int
  *   score_host   HOST, nullable: int32 [len] = m - 2 * Hamming */
 int h1b_debug_scores(h1b_ctx *ctx, int layer, int seq, int kv_head, const void *q,
                      uint32_t *qwords_host, int32_t *score_host);
+
+/* After an attention call (any of the decode / multi / prefill-attention / static
+ * entry points) has completed: what the attention kernel itself wrote for one
+ * (layer, sequence, query token, query head) of that call's LAST launch, split by
+ * split (HOST outputs, room for max_splits entries each):
+ *   n_splits_host  the number S of splits the sequence was dealt into
+ *   hmin_host[s]   the smallest Hamming distance (Eq. 3) split s saw among the
+ *                  tokens this head attends to, as a float; 1048576 if it saw none
+ *   wsum_host[s]   sum over those tokens of 2^((hmin[s] - Hamming_t) * c),
+ *                  c = 2 log2(e) / (m tau): the split's softmax denominator (Eq. 5)
+ * Split s covers chunks [s*q + min(s, r), (s+1)*q + min(s+1, r)) of the C =
+ * ceil(len / 32) chunks of 32 tokens the sequence holds, q = C / S, r = C mod S.
+ * A test compares these with a CPU statement of Eq. 3, so the scoring inside the
+ * production kernel is checked bit for bit and not only through the outputs.
+ * H1B_ERR_INVALID_ARG when the indices are not part of that launch. */
+int h1b_debug_partials(h1b_ctx *ctx, int layer, int seq, int q_token, int q_head,
+                       int32_t *n_splits_host, float *hmin_host, float *wsum_host, int max_splits);
+
+/* Failure-path probe (no counterpart in the paper). Launches one warp that waits
+ * for at most limit_ns nanoseconds (1 .. 1e9) on a barrier phase nothing will
+ * complete, with the same bounded wait the attention and long-append kernels
+ * use for their copies and tensor-core work. The wait runs out, the warp
+ * records the time-out in the device status word and the kernel returns
+ * normally: nothing traps, faults or spins on. After the stream has been
+ * synchronised h1b_poll_status() then returns H1B_ERR_TIMEOUT once and H1B_OK
+ * afterwards, and the context stays usable. Asynchronous on `stream`. */
+int h1b_debug_wait_timeout(h1b_ctx *ctx, uint64_t limit_ns, void *stream);
 
 /* Force the number of sequence splits of the decode kernel (0 = automatic).
  * H1B_ERR_INVALID_ARG if the split-K scratch cannot hold that many. */

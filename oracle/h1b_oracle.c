@@ -19,8 +19,7 @@
  * transposed, Rt[i][j] = R[j][i], row-major [d][m], so (R v)_j =
  * sum_i v_i * Rt[i][j].
  *
- * Readings of points the paper leaves open (each is also listed in the design
- * notes of the repository):
+ * Readings of points the paper leaves open:
  *   - sign(0) = +1 (bit 1).
  *   - Eq. 4's scale and zero-point come from the min and max of each group of
  *     G consecutive channels of one value vector: Delta = (max-min)/15 rounded

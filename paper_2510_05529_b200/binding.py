@@ -86,6 +86,9 @@ def load_library(rebuild: bool = True) -> ctypes.CDLL:
         "h1b_export_values": (ctypes.c_int, [vp, ctypes.c_int, ctypes.c_int, ctypes.c_int, ctypes.c_int,
                                              ctypes.c_int, vp]),
         "h1b_debug_scores": (ctypes.c_int, [vp, ctypes.c_int, ctypes.c_int, ctypes.c_int, vp, vp, vp]),
+        "h1b_debug_partials": (ctypes.c_int, [vp, ctypes.c_int, ctypes.c_int, ctypes.c_int, ctypes.c_int, i32p, vp, vp,
+                                              ctypes.c_int]),
+        "h1b_debug_wait_timeout": (ctypes.c_int, [vp, ctypes.c_uint64, vp]),
         "h1b_set_splits": (ctypes.c_int, [vp, ctypes.c_int]),
         "h1b_poll_status": (ctypes.c_int, [vp]),
         "h1b_set_profiling": (ctypes.c_int, [vp, ctypes.c_int]),
@@ -364,6 +367,19 @@ class H1BCache:
         score = np.empty((max(n_tokens, 1),), dtype=np.int32)
         self._check(self.lib.h1b_debug_scores(self._h, layer, seq, kv_head, qp, qwords.ctypes.data, score.ctypes.data))
         return qwords, score[:n_tokens]
+
+    def h1b_debug_partials(self, layer: int, seq: int, q_token: int, q_head: int, max_splits: int = 4096):
+        """After an attention call: (hmin float32 [S], wsum float32 [S]) of the last launch's splits for one head."""
+        n = ctypes.c_int32()
+        hmin = np.empty((max_splits,), dtype=np.float32)
+        wsum = np.empty((max_splits,), dtype=np.float32)
+        self._check(self.lib.h1b_debug_partials(self._h, layer, seq, q_token, q_head, ctypes.byref(n), hmin.ctypes.data,
+                                                wsum.ctypes.data, max_splits))
+        return hmin[:n.value].copy(), wsum[:n.value].copy()
+
+    def h1b_debug_wait_timeout(self, limit_ns: int, stream=None):
+        """Failure-path probe: one warp's bounded wait runs out and is recorded in the status word."""
+        self._check(self.lib.h1b_debug_wait_timeout(self._h, int(limit_ns), _stream_ptr(stream)))
 
     def h1b_set_splits(self, splits: int):
         self._check(self.lib.h1b_set_splits(self._h, splits))

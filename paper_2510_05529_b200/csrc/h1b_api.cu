@@ -6,6 +6,7 @@
 #include <cstdarg>
 #include <cstdio>
 #include <cstring>
+#include <mutex>
 #include <new>
 #include <string>
 #include <vector>
@@ -80,6 +81,16 @@ h1b_config internal_config(const h1b_config *c) {
     return ic;
 }
 
+// (query token, query head) pairs that share a KV head ("virtual heads": gq * Tq of them) go through the attention
+// kernel `gqk` at a time, one work item per group of them: vgroups items per slab and split. 128-wide heads: one, two
+// or four per item. Two 64-wide heads per slab: an item takes one or four virtual heads of EACH KV head of the pair
+// (gq counts both KV heads' query heads there), so two or eight.
+void heads_per_item(int gq, int Tq, bool paired, int *gqk, int *vgroups) {
+    const int vheads = gq * Tq;
+    *gqk = paired ? (vheads >= 4 ? 8 : 2) : (vheads >= 3 ? 4 : vheads);
+    *vgroups = (vheads + *gqk - 1) / *gqk;
+}
+
 int make_plan(const h1b_config *user, Plan *p) {
     const int rc = check_config(user);
     if (rc != H1B_OK) return rc;
@@ -95,9 +106,21 @@ int make_plan(const h1b_config *user, Plan *p) {
     p->layer_bytes = (size_t)c->n_pages * c->n_kv_heads * p->page_chunks * cl.bytes;
     const size_t L = c->n_layers, B = c->max_batch, Hq = c->n_q_heads, Hkv = c->n_kv_heads, d = c->head_dim;
     const size_t slabs = L * B * Hkv;
-    // split-K scratch: room for kTargetItems work items (or one per slab) of four (virtual) heads each
-    const size_t partial_items = slabs > (size_t)kTargetItems ? slabs : (size_t)kTargetItems;
-    p->partial_bytes = partial_items * 4 * kPartStride * sizeof(float);
+    // split-K scratch, counted in head slots (one partial of kPartStride floats each; a work item takes the slots of
+    // its heads). Room for the largest of: kTargetItems work items of four heads (the split count aimed for), one
+    // item per slab of all layers (a decode call then never needs a second pass), and ONE layer of the largest
+    // multi-query call the interface allows (H1B_MAX_QUERY_TOKENS query tokens on max_batch sequences), so that
+    // no call the header allows runs out of scratch.
+    {
+        const bool paired = is_paired(user);
+        int gqk1, vg1, gqkm, vgm;
+        heads_per_item(p->gq, 1, paired, &gqk1, &vg1);
+        heads_per_item(p->gq, kMaxQueryTokens, paired, &gqkm, &vgm);
+        size_t slots = (size_t)kTargetItems * 4;
+        slots = std::max(slots, slabs * (size_t)vg1 * gqk1);
+        slots = std::max(slots, B * Hkv * (size_t)vgm * gqkm);
+        p->partial_bytes = slots * kPartStride * sizeof(float);
+    }
     size_t o = 0;
     auto take = [&](size_t bytes) { size_t at = o; o = align_up(o + bytes, 256); return at; };
     p->rt = take(L * d * c->sketch_bits * sizeof(float));
@@ -161,6 +184,8 @@ struct h1b_ctx {
     size_t events_used;
     cudaStream_t side;                 // long appends: the value kernel runs here, beside the key kernel
     cudaEvent_t fork, join;            // ... forked from and joined back into the caller's stream
+    DecodeParams last_decode;          // the most recent attention launch (test helper: h1b_debug_partials)
+    bool have_last_decode;
     std::string err;
 };
 
@@ -230,6 +255,8 @@ int check_layers(h1b_ctx *ctx, int layer_begin, int n_layers, int B) {
 
 extern "C" {
 
+static cudaError_t resolve_static_scratch(int dev);
+
 size_t h1b_entry_bytes(const h1b_config *cfg) {
     if (check_config(cfg) != H1B_OK) return 0;
     if (cfg->flags & H1B_FLAG_FP16_VALUES) return (size_t)cfg->sketch_bits / 8 + (size_t)cfg->head_dim * 2;
@@ -270,6 +297,7 @@ int h1b_init_projection(const h1b_config *cfg, uint64_t seed, const float *Rt_ho
     ctx->profiling = false;
     ctx->events_used = 0;
     ctx->side = nullptr; ctx->fork = nullptr; ctx->join = nullptr;
+    ctx->have_last_decode = false;
     cudaStream_t st = static_cast<cudaStream_t>(stream);
     auto bail = [&](cudaError_t e, const char *what) {
         fail(nullptr, H1B_ERR_CUDA, "%s: %s", what, cudaGetErrorString(e));
@@ -315,6 +343,14 @@ int h1b_init_projection(const h1b_config *cfg, uint64_t seed, const float *Rt_ho
     if (e != cudaSuccess) return bail(e, "split_projection_kernel");
     e = cudaStreamSynchronize(st);
     if (e != cudaSuccess) return bail(e, "cudaStreamSynchronize");
+    // Set-up that would otherwise fall to the first call of some kind: the launch attributes of every kernel this
+    // cache can reach, and the device address of the built-in scratch array of h1b_decode_attention_static().
+    // Done here, no later call has anything to prepare (none needs a warm-up before a stream capture, and the
+    // array's module is loaded, its memory backed, before any region in which the caller may not allocate).
+    e = warm_kernel_attributes(plan.m_words, plan.groups, ctx->paired, plan.page_chunks > 0, (cfg->flags & H1B_FLAG_ROPE) != 0);
+    if (e != cudaSuccess) return bail(e, "kernel attributes");
+    e = resolve_static_scratch(cfg->device);
+    if (e != cudaSuccess) return bail(e, "cudaGetSymbolAddress(built-in scratch array)");
     // without these three the two long-append kernels simply run one after the other
     if (cudaStreamCreateWithFlags(&ctx->side, cudaStreamNonBlocking) != cudaSuccess ||
         cudaEventCreateWithFlags(&ctx->fork, cudaEventDisableTiming) != cudaSuccess ||
@@ -412,31 +448,35 @@ static void commit_lengths(h1b_ctx *ctx, int layer_begin, int n_layers, int B, c
         for (int b = 0; b < B; ++b) ctx->len_host[(size_t)l * ctx->cfg.max_batch + b] += nn.v[b];
 }
 
-// Enqueue the split-K attention kernel over scratch (qwords, partial). Every sequence is split so that there are
-// about kTargetItems work items, capped by what the scratch holds. The host only chooses how many splits; which
-// chunks a split takes is worked out on the device from the sequence's length at that moment, so the result does
-// not depend on how well the host's view of the lengths matches the device's.
-static int enqueue_decode(h1b_ctx *ctx, int layer_begin, int n_layers, float inv_tau, void *out, int B,
-                          cudaStream_t st, uint32_t *qwords, float *partial, size_t partial_bytes,
-                          bool may_profile, int *launches, int Tq = 1, int q_tail = 0, int out_seq_tokens = 0) {
-    // (query token, query head) pairs that share a KV head, and how many of them one work item takes
-    // (two 64-wide heads per slab: an item takes one query head of each KV head of the pair)
-    // (they then come in twos or eights: one or four of them on each of the two KV heads)
-    const int vheads = ctx->plan.gq * Tq, gqk = ctx->paired ? (vheads >= 4 ? 8 : 2) : (vheads >= 3 ? 4 : vheads);
-    const int vgroups = (vheads + gqk - 1) / gqk;
-    const size_t max_items = partial_bytes / ((size_t)gqk * kPartStride * sizeof(float));
+// How one attention call goes through the split-K scratch: decided on the host before anything is launched.
+struct DecodePlan {
+    int gqk, vgroups;       // heads per work item, items per (slab, split)
+    int pass_layers;        // layers per pass through the scratch (all of them unless the scratch is small)
+    int splits;             // work items per (slab, group of heads)
+};
+
+// Every sequence is split so that there are about kTargetItems work items, capped by what the scratch holds. The
+// host only chooses how many splits; which chunks a split takes is worked out on the device from the sequence's
+// length at that moment, so the result does not depend on how well the host's view of the lengths matches the
+// device's. `extra_tokens`: tokens the same call appends before it attends (the host's lengths do not have them yet).
+// Fails (nothing launched, nothing changed) when one layer's units do not fit the scratch.
+static int plan_decode(h1b_ctx *ctx, int layer_begin, int n_layers, int B, size_t partial_bytes, int Tq, int q_tail,
+                       int extra_tokens, DecodePlan *dpl) {
+    heads_per_item(ctx->plan.gq, Tq, ctx->paired, &dpl->gqk, &dpl->vgroups);
+    const size_t max_items = partial_bytes / ((size_t)dpl->gqk * kPartStride * sizeof(float));
     // slabs x groups of virtual heads: the units a split divides. When the scratch cannot hold one partial for
     // every unit of the call (many query tokens on a large batch), the layers go through it in several passes,
     // one behind the other on the stream.
-    const long per_layer = (long)B * ctx->cfg.n_kv_heads * vgroups;
+    const long per_layer = (long)B * ctx->cfg.n_kv_heads * dpl->vgroups;
     if ((size_t)per_layer > max_items)
         return fail(ctx, H1B_ERR_CAPACITY, "%ld (sequence, KV head, head group) units of one layer exceed the split-K "
-                    "scratch (%zu items)", per_layer, max_items);
-    const int pass_layers = (int)std::min<size_t>((size_t)n_layers, max_items / (size_t)per_layer);
-    const long slabs = per_layer * pass_layers;
+                    "scratch (%zu items of %d heads)", per_layer, max_items, dpl->gqk);
+    dpl->pass_layers = (int)std::min<size_t>((size_t)n_layers, max_items / (size_t)per_layer);
+    const long slabs = per_layer * dpl->pass_layers;
     int maxlen = 1;
     for (int l = layer_begin; l < layer_begin + n_layers; ++l)
-        for (int b = 0; b < B; ++b) maxlen = std::max(maxlen, ctx->len_host[(size_t)l * ctx->cfg.max_batch + b] - q_tail);
+        for (int b = 0; b < B; ++b)
+            maxlen = std::max(maxlen, ctx->len_host[(size_t)l * ctx->cfg.max_batch + b] + extra_tokens - q_tail);
     long splits = ctx->forced_splits > 0 ? ctx->forced_splits : kTargetItems / slabs;
     const long max_splits = std::max(1, maxlen / kMinSplitTokens);
     if (ctx->forced_splits <= 0 && splits > max_splits) splits = max_splits;
@@ -447,7 +487,14 @@ static int enqueue_decode(h1b_ctx *ctx, int layer_begin, int n_layers, float inv
                         splits, slabs, max_items);
         splits = (long)(max_items / (size_t)slabs);
     }
+    dpl->splits = (int)splits;
+    return H1B_OK;
+}
 
+// Enqueue the split-K attention kernel and the combine over scratch (qwords, partial) as planned.
+static int enqueue_decode(h1b_ctx *ctx, const DecodePlan &dpl, int layer_begin, int n_layers, float inv_tau, void *out,
+                          int B, cudaStream_t st, uint32_t *qwords, float *partial, bool may_profile, int *launches,
+                          int Tq = 1, int q_tail = 0, int out_seq_tokens = 0) {
     DecodeParams dp;
     dp.ca = cache_addr(ctx);
     dp.len = at<int32_t>(ctx, ctx->plan.len);
@@ -457,25 +504,27 @@ static int enqueue_decode(h1b_ctx *ctx, int layer_begin, int n_layers, float inv
     dp.B = B; dp.Hkv = ctx->cfg.n_kv_heads;
     dp.Hq = ctx->cfg.n_q_heads; dp.max_batch = ctx->cfg.max_batch; dp.m_words = ctx->plan.m_words;
     dp.groups = ctx->plan.groups;
-    dp.splits = (int)splits;
-    dp.Tq = Tq; dp.gqk = gqk; dp.vgroups = vgroups;
+    dp.splits = dpl.splits;
+    dp.Tq = Tq; dp.gqk = dpl.gqk; dp.vgroups = dpl.vgroups;
     dp.q_tail = q_tail;
     dp.out_seq_rows = (out_seq_tokens > 0 ? out_seq_tokens : Tq) * ctx->cfg.n_q_heads;
     dp.paired = ctx->paired ? 1 : 0;
     dp.out_dim = ctx->ucfg.head_dim;
     dp.c2 = (float)(2.0 * (double)inv_tau * 1.4426950408889634 / (double)ctx->ucfg.sketch_bits);
     cudaEvent_t ev0 = nullptr, ev1 = nullptr;
-    if (may_profile && pass_layers == n_layers && ctx->profiling && ctx->events_used + 2 <= ctx->events.size()) {
+    if (may_profile && dpl.pass_layers == n_layers && ctx->profiling && ctx->events_used + 2 <= ctx->events.size()) {
         ev0 = ctx->events[ctx->events_used];
         ev1 = ctx->events[ctx->events_used + 1];
         ctx->events_used += 2;
     }
     const size_t layer_out = (size_t)B * dp.out_seq_rows * (size_t)ctx->ucfg.head_dim;           // floats of one layer
-    for (int done = 0; done < n_layers; done += pass_layers) {
+    for (int done = 0; done < n_layers; done += dpl.pass_layers) {
         dp.layer_begin = layer_begin + done;
-        dp.n_layers = std::min(pass_layers, n_layers - done);
+        dp.n_layers = std::min(dpl.pass_layers, n_layers - done);
         dp.out = static_cast<float *>(out) + (size_t)done * layer_out;
         H1B_CUDA(ctx, launch_decode(dp, st, launches, ev0, ev1));
+        ctx->last_decode = dp;
+        ctx->have_last_decode = true;
     }
     return H1B_OK;
 }
@@ -547,14 +596,17 @@ int h1b_decode_attention(h1b_ctx *ctx, int layer_begin, int n_layers, const void
                          int B, void *stream) {
     int rc = check_decode_args(ctx, layer_begin, n_layers, q, inv_tau, out, B);
     if (rc != H1B_OK) return rc;
+    DecodePlan dpl;
+    rc = plan_decode(ctx, layer_begin, n_layers, B, ctx->plan.partial_bytes, 1, 0, 0, &dpl);
+    if (rc != H1B_OK) return rc;
     cudaStream_t st = static_cast<cudaStream_t>(stream);
     int launches = 0;
     const SketchParams sp = sketch_params(ctx, layer_begin, n_layers, q, B, at<uint32_t>(ctx, ctx->plan.qwords));
     NewCounts none;
     std::memset(&none, 0, sizeof none);
     H1B_CUDA(ctx, launch_prepare(nullptr, &sp, none, st, &launches));
-    rc = enqueue_decode(ctx, layer_begin, n_layers, inv_tau, out, B, st, sp.qwords, at<float>(ctx, ctx->plan.partial),
-                        ctx->plan.partial_bytes, true, &launches);
+    rc = enqueue_decode(ctx, dpl, layer_begin, n_layers, inv_tau, out, B, st, sp.qwords, at<float>(ctx, ctx->plan.partial),
+                        true, &launches);
     ctx->launches += launches;
     return rc;
 }
@@ -570,6 +622,9 @@ int h1b_decode_attention_multi(h1b_ctx *ctx, int layer_begin, int n_layers, cons
             if (ctx->len_host[(size_t)l * ctx->cfg.max_batch + b] < Tq)
                 return fail(ctx, H1B_ERR_INVALID_ARG, "layer %d sequence %d holds %d < Tq = %d tokens", l, b,
                             ctx->len_host[(size_t)l * ctx->cfg.max_batch + b], Tq);
+    DecodePlan dpl;
+    rc = plan_decode(ctx, layer_begin, n_layers, B, ctx->plan.partial_bytes, Tq, 0, 0, &dpl);
+    if (rc != H1B_OK) return rc;
     cudaStream_t st = static_cast<cudaStream_t>(stream);
     int launches = 0;
     // rows of the sketch are (sequence, query token, query head): Tq * Hq "heads" per sequence
@@ -580,8 +635,8 @@ int h1b_decode_attention_multi(h1b_ctx *ctx, int layer_begin, int n_layers, cons
     NewCounts none;
     std::memset(&none, 0, sizeof none);
     H1B_CUDA(ctx, launch_prepare(nullptr, &sp, none, st, &launches));
-    rc = enqueue_decode(ctx, layer_begin, n_layers, inv_tau, out, B, st, sp.qwords, at<float>(ctx, ctx->plan.partial),
-                        ctx->plan.partial_bytes, true, &launches, Tq);
+    rc = enqueue_decode(ctx, dpl, layer_begin, n_layers, inv_tau, out, B, st, sp.qwords, at<float>(ctx, ctx->plan.partial),
+                        true, &launches, Tq);
     ctx->launches += launches;
     return rc;
 }
@@ -596,6 +651,15 @@ int h1b_prefill_attention(h1b_ctx *ctx, int layer_begin, int n_layers, const voi
             if (ctx->len_host[(size_t)l * ctx->cfg.max_batch + b] < Tn)
                 return fail(ctx, H1B_ERR_INVALID_ARG, "layer %d sequence %d holds %d < Tn = %d tokens", l, b,
                             ctx->len_host[(size_t)l * ctx->cfg.max_batch + b], Tn);
+    // every block of the walk is planned before the first one is launched: a call that cannot run launches nothing
+    std::vector<DecodePlan> plans;
+    for (int t0 = 0; t0 < Tn; t0 += kMaxQueryTokens) {
+        const int Tq = std::min(kMaxQueryTokens, Tn - t0), q_tail = Tn - t0 - Tq;
+        DecodePlan dpl;
+        rc = plan_decode(ctx, layer_begin, n_layers, B, ctx->plan.partial_bytes, Tq, q_tail, 0, &dpl);
+        if (rc != H1B_OK) return rc;
+        plans.push_back(dpl);
+    }
     cudaStream_t st = static_cast<cudaStream_t>(stream);
     int launches = 0;
     NewCounts none;
@@ -604,6 +668,7 @@ int h1b_prefill_attention(h1b_ctx *ctx, int layer_begin, int n_layers, const voi
     // blocks of up to kMaxQueryTokens query tokens, first to last; block j ends q_tail tokens before the sequences' ends
     for (int t0 = 0; t0 < Tn && rc == H1B_OK; t0 += kMaxQueryTokens) {
         const int Tq = std::min(kMaxQueryTokens, Tn - t0), q_tail = Tn - t0 - Tq;
+        const DecodePlan &dpl = plans[(size_t)(t0 / kMaxQueryTokens)];
         SketchParams sp = sketch_params(ctx, layer_begin, n_layers,
                                         static_cast<const uint16_t *>(q) + (size_t)t0 * Hq * d, B,
                                         at<uint32_t>(ctx, ctx->plan.qwords));
@@ -613,9 +678,8 @@ int h1b_prefill_attention(h1b_ctx *ctx, int layer_begin, int n_layers, const voi
         sp.q_seq_rows = Tn * rows_per_token;
         sp.q_tail = q_tail;
         H1B_CUDA(ctx, launch_prepare(nullptr, &sp, none, st, &launches));
-        rc = enqueue_decode(ctx, layer_begin, n_layers, inv_tau, static_cast<float *>(out) + (size_t)t0 * Hq * d, B, st,
-                            sp.qwords, at<float>(ctx, ctx->plan.partial), ctx->plan.partial_bytes, false, &launches, Tq,
-                            q_tail, Tn);
+        rc = enqueue_decode(ctx, dpl, layer_begin, n_layers, inv_tau, static_cast<float *>(out) + (size_t)t0 * Hq * d, B, st,
+                            sp.qwords, at<float>(ctx, ctx->plan.partial), false, &launches, Tq, q_tail, Tn);
     }
     ctx->launches += launches;
     return rc;
@@ -631,14 +695,17 @@ int h1b_decode_step_layers(h1b_ctx *ctx, int layer_begin, int n_layers, const vo
     NewCounts nn;
     rc = make_new_counts(ctx, layer_begin, n_layers, nullptr, B, 1, &nn);
     if (rc != H1B_OK) return rc;
+    DecodePlan dpl;                                     // before anything is launched or the lengths move
+    rc = plan_decode(ctx, layer_begin, n_layers, B, ctx->plan.partial_bytes, 1, 0, 1, &dpl);
+    if (rc != H1B_OK) return rc;
     cudaStream_t st = static_cast<cudaStream_t>(stream);
     int launches = 0;
     const AppendParams ap = append_params(ctx, layer_begin, n_layers, k, v, B, 1);
     const SketchParams sp = sketch_params(ctx, layer_begin, n_layers, q, B, at<uint32_t>(ctx, ctx->plan.qwords));
     H1B_CUDA(ctx, launch_prepare(&ap, &sp, nn, st, &launches));
     commit_lengths(ctx, layer_begin, n_layers, B, nn);
-    rc = enqueue_decode(ctx, layer_begin, n_layers, inv_tau, out, B, st, sp.qwords, at<float>(ctx, ctx->plan.partial),
-                        ctx->plan.partial_bytes, true, &launches);
+    rc = enqueue_decode(ctx, dpl, layer_begin, n_layers, inv_tau, out, B, st, sp.qwords, at<float>(ctx, ctx->plan.partial),
+                        true, &launches);
     ctx->launches += launches;
     return rc;
 }
@@ -668,12 +735,27 @@ int h1b_sync_lengths(h1b_ctx *ctx, void *stream) {
 static __device__ __align__(256) unsigned char h1b_static_scratch[H1B_STATIC_SCRATCH_BYTES];
 
 // In host code the name above is only a stand-in for the symbol, not a device
-// address; the address each device gave the array is looked up once per device.
+// address; the address each device gave the array is looked up once per device,
+// when the first context on that device is created (h1b_init_projection, a
+// synchronous set-up call made with that device current), and kept here.
 static void *g_static_scratch_addr[64] = {};
+static std::mutex g_static_scratch_mutex;
 
 // Never launched: a device-side reference, so that the array is certain to be kept in the image.
 __global__ void h1b_static_scratch_anchor(unsigned char *dst) {
     if (dst) *dst = h1b_static_scratch[0];
+}
+
+static cudaError_t resolve_static_scratch(int dev) {
+    if (dev < 0 || dev >= 64) return cudaSuccess;       // such a device simply has no static entry point (refused there)
+    std::lock_guard<std::mutex> lock(g_static_scratch_mutex);
+    if (g_static_scratch_addr[dev]) return cudaSuccess;
+    void *p = nullptr;
+    cudaError_t e = cudaGetSymbolAddress(&p, h1b_static_scratch);
+    if (e != cudaSuccess) return e;
+    if (!p) return cudaErrorInvalidSymbol;
+    g_static_scratch_addr[dev] = p;
+    return cudaSuccess;
 }
 
 int h1b_decode_attention_static(h1b_ctx *ctx, int layer_begin, int n_layers, const void *q, float inv_tau,
@@ -686,34 +768,36 @@ int h1b_decode_attention_static(h1b_ctx *ctx, int layer_begin, int n_layers, con
     H1B_CUDA(ctx, cudaGetDevice(&cur));
     if (cur != dev)
         return fail(ctx, H1B_ERR_INVALID_ARG, "device %d must be current (current is %d)", dev, cur);
-    if (!g_static_scratch_addr[dev]) {          // first call on this device: resolve the array's address
-        void *p = nullptr;
-        H1B_CUDA(ctx, cudaGetSymbolAddress(&p, h1b_static_scratch));
-        if (!p) return fail(ctx, H1B_ERR_CUDA, "cudaGetSymbolAddress returned a null address");
-        g_static_scratch_addr[dev] = p;
+    unsigned char *scratch;
+    {
+        std::lock_guard<std::mutex> lock(g_static_scratch_mutex);
+        scratch = static_cast<unsigned char *>(g_static_scratch_addr[dev]);     // resolved when the context was made
     }
-    unsigned char *scratch = static_cast<unsigned char *>(g_static_scratch_addr[dev]);
+    if (!scratch) return fail(ctx, H1B_ERR_CUDA, "the built-in scratch array has no address on device %d", dev);
 
-    // carve: query sketches for every (layer, sequence, head) slot the kernels index, then the partials
-    const long slabs = (long)n_layers * B * ctx->cfg.n_kv_heads;
+    // carve: query sketches for every (layer, sequence, head) slot the kernels index, then the partials. What must
+    // fit is ONE layer of the call (more layers than fit go through the array in passes, fewer splits are used
+    // when the automatic choice would not fit): the same planning as the ordinary entry point, over this array.
     const size_t qw_bytes = align_up((size_t)ctx->cfg.n_layers * ctx->cfg.max_batch * ctx->cfg.n_q_heads *
                                          ctx->plan.m_words * sizeof(uint32_t), 256);
-    const int gqk = ctx->plan.gq >= 3 ? 4 : ctx->plan.gq, vgroups = (ctx->plan.gq + gqk - 1) / gqk;
-    const size_t item_bytes = (size_t)vgroups * gqk * kPartStride * sizeof(float);
-    const size_t need = qw_bytes + (size_t)slabs * item_bytes;
+    int gqk, vgroups;
+    heads_per_item(ctx->plan.gq, 1, ctx->paired, &gqk, &vgroups);
+    const size_t need = qw_bytes + (size_t)B * ctx->cfg.n_kv_heads * vgroups * gqk * kPartStride * sizeof(float);
     if (need > H1B_STATIC_SCRATCH_BYTES)
         return fail(ctx, H1B_ERR_CAPACITY,
                     "static scratch too small: this call needs at least %zu bytes, the built-in array holds %u",
                     need, (unsigned)H1B_STATIC_SCRATCH_BYTES);
-    const size_t fit_bytes = H1B_STATIC_SCRATCH_BYTES - qw_bytes;
+    DecodePlan dpl;
+    rc = plan_decode(ctx, layer_begin, n_layers, B, H1B_STATIC_SCRATCH_BYTES - qw_bytes, 1, 0, 0, &dpl);
+    if (rc != H1B_OK) return rc;
     cudaStream_t st = static_cast<cudaStream_t>(stream);
     int launches = 0;
     const SketchParams sp = sketch_params(ctx, layer_begin, n_layers, q, B, reinterpret_cast<uint32_t *>(scratch));
     NewCounts none;
     std::memset(&none, 0, sizeof none);
     H1B_CUDA(ctx, launch_prepare(nullptr, &sp, none, st, &launches));
-    rc = enqueue_decode(ctx, layer_begin, n_layers, inv_tau, out, B, st, sp.qwords,
-                        reinterpret_cast<float *>(scratch + qw_bytes), fit_bytes, false, &launches);
+    rc = enqueue_decode(ctx, dpl, layer_begin, n_layers, inv_tau, out, B, st, sp.qwords,
+                        reinterpret_cast<float *>(scratch + qw_bytes), false, &launches);
     ctx->launches += launches;
     return rc;
 }
@@ -963,6 +1047,19 @@ int h1b_set_block_table(h1b_ctx *ctx, int seq, const int32_t *pages_host, int n,
     for (int i = 0; i < n; ++i)
         if (pages_host[i] < 0 || pages_host[i] >= ctx->cfg.n_pages)
             return fail(ctx, H1B_ERR_INVALID_ARG, "page %d (entry %d) outside the pool of %d", pages_host[i], i, ctx->cfg.n_pages);
+    // no page may belong to two sequences (or twice to one): their appends would overwrite each other
+    for (int i = 0; i < n; ++i) {
+        for (int j = 0; j < i; ++j)
+            if (pages_host[j] == pages_host[i])
+                return fail(ctx, H1B_ERR_INVALID_ARG, "page %d appears twice (entries %d and %d)", pages_host[i], j, i);
+        for (int b = 0; b < ctx->cfg.max_batch; ++b) {
+            if (b == seq) continue;
+            const int32_t *other = ctx->table_host.data() + (size_t)b * ctx->plan.table_stride;
+            for (int j = 0; j < ctx->plan.table_stride; ++j)
+                if (other[j] == pages_host[i])
+                    return fail(ctx, H1B_ERR_INVALID_ARG, "page %d (entry %d) already belongs to sequence %d", pages_host[i], i, b);
+        }
+    }
     const int page_tokens = ctx->cfg.page_tokens;
     int held = 0;
     for (int l = 0; l < ctx->cfg.n_layers; ++l) held = std::max(held, ctx->len_host[(size_t)l * ctx->cfg.max_batch + seq]);
@@ -983,7 +1080,9 @@ int h1b_set_block_table(h1b_ctx *ctx, int seq, const int32_t *pages_host, int n,
 
 int h1b_set_splits(h1b_ctx *ctx, int splits) {
     if (!ctx) return H1B_ERR_NULL;
-    const size_t most = ctx->plan.partial_bytes / ((size_t)std::min(ctx->plan.gq, 4) * kPartStride * sizeof(float));
+    int gqk, vgroups;
+    heads_per_item(ctx->plan.gq, 1, ctx->paired, &gqk, &vgroups);
+    const size_t most = ctx->plan.partial_bytes / ((size_t)gqk * kPartStride * sizeof(float));
     if (splits < 0 || (size_t)splits > most)
         return fail(ctx, H1B_ERR_INVALID_ARG, "splits %d outside [0, %zu]", splits, most);
     ctx->forced_splits = splits;
@@ -999,6 +1098,45 @@ int h1b_poll_status(h1b_ctx *ctx) {
     if (s == kStatusCapacity)
         return fail(ctx, H1B_ERR_CAPACITY, "a replayed append found a sequence full: its rows were dropped");
     return fail(ctx, H1B_ERR_TIMEOUT, "a kernel gave up a bounded wait (status %d)", s);
+}
+
+int h1b_debug_wait_timeout(h1b_ctx *ctx, uint64_t limit_ns, void *stream) {
+    if (!ctx) return H1B_ERR_NULL;
+    if (limit_ns < 1 || limit_ns > 1000000000ull)
+        return fail(ctx, H1B_ERR_INVALID_ARG, "limit_ns = %llu outside [1, 1e9]", (unsigned long long)limit_ns);
+    H1B_CUDA(ctx, launch_debug_wait_timeout(at<int32_t>(ctx, ctx->plan.status), limit_ns, static_cast<cudaStream_t>(stream)));
+    ++ctx->launches;
+    return H1B_OK;
+}
+
+int h1b_debug_partials(h1b_ctx *ctx, int layer, int seq, int q_token, int q_head, int32_t *n_splits_host,
+                       float *hmin_host, float *wsum_host, int max_splits) {
+    if (!ctx) return H1B_ERR_NULL;
+    if (!n_splits_host || !hmin_host || !wsum_host) return fail(ctx, H1B_ERR_NULL, "an output pointer is NULL");
+    if (!ctx->have_last_decode) return fail(ctx, H1B_ERR_INVALID_ARG, "no attention call has been made on this context");
+    const DecodeParams &p = ctx->last_decode;
+    if (layer < p.layer_begin || layer >= p.layer_begin + p.n_layers || seq < 0 || seq >= p.B || q_token < 0 ||
+        q_token >= p.Tq || q_head < 0 || q_head >= p.Hq)
+        return fail(ctx, H1B_ERR_INVALID_ARG, "(layer %d, seq %d, query token %d, head %d) is not part of the last attention launch",
+                    layer, seq, q_token, q_head);
+    if (max_splits < p.splits) return fail(ctx, H1B_ERR_INVALID_ARG, "%d splits, room for %d", p.splits, max_splits);
+    // where the combine kernel finds this head's partials (the same arithmetic)
+    const int gq = p.Hq / p.Hkv, kvh = q_head / gq, jj = q_head % gq, gqu = gq >> 1, gqh = p.gqk >> 1;
+    const int v = q_token * gq + jj;
+    const int vp = p.paired ? q_token * gqu + jj % gqu : 0;
+    const int vg = p.paired ? vp / gqh : v / p.gqk, hh = p.paired ? (jj / gqu) * gqh + vp % gqh : v % p.gqk;
+    const long slab_local = ((long)(layer - p.layer_begin) * p.B + seq) * p.Hkv + kvh;
+    const float *base = p.partial + (((size_t)slab_local * p.vgroups + vg) * p.splits * p.gqk + hh) * kPartStride;
+    const size_t stride = (size_t)p.gqk * kPartStride;
+    H1B_CUDA(ctx, cudaDeviceSynchronize());
+    for (int s = 0; s < p.splits; ++s) {
+        float pair[2];
+        H1B_CUDA(ctx, cudaMemcpy(pair, base + (size_t)s * stride + 128, sizeof pair, cudaMemcpyDeviceToHost));
+        hmin_host[s] = pair[0];
+        wsum_host[s] = 0.5f * pair[1];                  // the kernel's weights carry a factor 2 (it cancels in the division)
+    }
+    *n_splits_host = p.splits;
+    return H1B_OK;
 }
 
 int h1b_set_profiling(h1b_ctx *ctx, int enable) {

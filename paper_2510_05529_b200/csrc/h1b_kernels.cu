@@ -15,6 +15,8 @@
 //   prefill_rope_kernel  accumulators in TMEM), the second one rotating each key tile in shared
 //                        memory first (rotary position embedding);
 //   prefill_values_kernel  Eq. 4 for the same appends, side by side with the key kernel.
+#include <mutex>
+
 #include "h1b_kernels.h"
 #include "h1b_ptx.cuh"
 
@@ -1413,9 +1415,24 @@ __global__ void debug_scores_kernel(CacheAddr ca, int layer, int b, int kvh, con
     score[t] = nw * 32 - 2 * ham;
 }
 
+// Test helper for the failure path: one warp waits, with a limit, on an mbarrier phase that nothing will ever
+// complete. The wait gives up, the warp records kStatusWaitTimeout in the status word exactly as the attention
+// and long-append kernels do when a copy or an MMA never lands, and the kernel returns normally.
+__global__ void debug_wait_timeout_kernel(int32_t *status, unsigned long long limit_ns) {
+    __shared__ __align__(8) unsigned long long bar_s;
+    const uint32_t bar = smem_addr(&bar_s);
+    if (threadIdx.x == 0) { mbar_init(bar, 1); mbar_fence_init(); }
+    __syncwarp();
+    const bool done = mbar_wait_bounded(bar, 0u, limit_ns);
+    if (!done && threadIdx.x == 0) atomicExch(status, kStatusWaitTimeout);
+}
+
 // ===========================================================================
 // Launchers
 // ===========================================================================
+// Per-device set-up that launchers do once (kernel attributes, SM counts) is guarded by this lock: two host
+// threads may make their first calls at the same time.
+static std::mutex g_setup_mutex;
 #define H1B_DISPATCH_MW(mw, ...)                                   \
     switch (mw) {                                                  \
         case 2: { constexpr int MW = 2; __VA_ARGS__; } break;      \
@@ -1459,12 +1476,14 @@ static long prefill_key_blocks(const PrefillParams &p, int nbc) {
 }
 
 template <int NBC, bool ROPE>
-static cudaError_t launch_prefill_t(const PrefillParams &p, const NewCounts &nn, cudaStream_t st, int grid) {
+static cudaError_t prefill_attributes() {
     using SM = PrefillSmem<NBC>;
     static bool attr_set[64] = {};
     int dev = 0;
     cudaGetDevice(&dev);
-    if (dev >= 0 && dev < 64 && !attr_set[dev]) {
+    if (dev < 0 || dev >= 64) return cudaErrorInvalidDevice;
+    std::lock_guard<std::mutex> lock(g_setup_mutex);
+    if (!attr_set[dev]) {
         cudaError_t e = cudaFuncSetAttribute(PrefillEntry<NBC, ROPE>::fn, cudaFuncAttributeMaxDynamicSharedMemorySize, SM::kTotal);
         if (e != cudaSuccess) return e;
         // the largest shared-memory split, not the smallest that fits this kernel: the rest is for the value kernel's blocks
@@ -1472,6 +1491,42 @@ static cudaError_t launch_prefill_t(const PrefillParams &p, const NewCounts &nn,
         if (e != cudaSuccess) return e;
         attr_set[dev] = true;
     }
+    return cudaSuccess;
+}
+static cudaError_t prefill_values_attributes() {
+    // both long-append kernels ask for the same shared-memory / L1 split, or an SM set up for one would not take the other
+    static bool attr_set[64] = {};
+    int dev = 0;
+    cudaGetDevice(&dev);
+    if (dev < 0 || dev >= 64) return cudaErrorInvalidDevice;
+    std::lock_guard<std::mutex> lock(g_setup_mutex);
+    if (!attr_set[dev]) {
+        cudaError_t e = cudaFuncSetAttribute(prefill_values_kernel, cudaFuncAttributePreferredSharedMemoryCarveout,
+                                             cudaSharedmemCarveoutMaxShared);
+        if (e != cudaSuccess) return e;
+        attr_set[dev] = true;
+    }
+    return cudaSuccess;
+}
+static cudaError_t sm_count(int *n) {
+    static int n_sm[64] = {};
+    int dev = 0;
+    cudaGetDevice(&dev);
+    if (dev < 0 || dev >= 64) return cudaErrorInvalidDevice;
+    std::lock_guard<std::mutex> lock(g_setup_mutex);
+    if (!n_sm[dev]) {
+        cudaError_t ea = cudaDeviceGetAttribute(&n_sm[dev], cudaDevAttrMultiProcessorCount, dev);
+        if (ea != cudaSuccess) return ea;
+    }
+    *n = n_sm[dev];
+    return cudaSuccess;
+}
+
+template <int NBC, bool ROPE>
+static cudaError_t launch_prefill_t(const PrefillParams &p, const NewCounts &nn, cudaStream_t st, int grid) {
+    using SM = PrefillSmem<NBC>;
+    cudaError_t e = prefill_attributes<NBC, ROPE>();
+    if (e != cudaSuccess) return e;
     PrefillEntry<NBC, ROPE>::fn<<<(unsigned)grid, kPrefillThreads, SM::kTotal, st>>>(p, nn);
     return cudaGetLastError();
 }
@@ -1487,31 +1542,15 @@ cudaError_t launch_prefill(const PrefillParams &p_in, const NewCounts &nn, cudaS
     const long vblocks = (units + kValueWarps - 1) / kValueWarps;
     // key kernel: at most one block per SM, each walking over its share of the work items, so that all of its blocks
     // are resident from the start and the value kernel's blocks can settle beside them
-    static int n_sm[64] = {};
-    int dev = 0;
-    cudaGetDevice(&dev);
-    if (dev < 0 || dev >= 64) return cudaErrorInvalidDevice;
-    if (!n_sm[dev]) {
-        cudaError_t ea = cudaDeviceGetAttribute(&n_sm[dev], cudaDevAttrMultiProcessorCount, dev);
-        if (ea != cudaSuccess) return ea;
-    }
+    int n_sm = 0;
+    cudaError_t e = sm_count(&n_sm);
+    if (e != cudaSuccess) return e;
     const long kwork = prefill_key_blocks(p, nbc);
-    const long kblocks = kwork < n_sm[dev] ? kwork : n_sm[dev];
+    const long kblocks = kwork < n_sm ? kwork : n_sm;
     if (vblocks <= 0 || kblocks <= 0 || vblocks + kblocks > 0x7fffffffL) return cudaErrorInvalidConfiguration;
     p.total_blocks = (int)(vblocks + kblocks);
     const bool forked = side && fork && join;
-    cudaError_t e;
-    {   // both kernels ask for the same shared-memory / L1 split, or an SM set up for one would not take the other
-        static bool attr_set[64] = {};
-        int dev = 0;
-        cudaGetDevice(&dev);
-        if (dev >= 0 && dev < 64 && !attr_set[dev]) {
-            e = cudaFuncSetAttribute(prefill_values_kernel, cudaFuncAttributePreferredSharedMemoryCarveout,
-                                     cudaSharedmemCarveoutMaxShared);
-            if (e != cudaSuccess) return e;
-            attr_set[dev] = true;
-        }
-    }
+    if ((e = prefill_values_attributes()) != cudaSuccess) return e;
     if (forked) {
         if ((e = cudaEventRecord(fork, st)) != cudaSuccess) return e;
         if ((e = cudaStreamWaitEvent(side, fork, 0)) != cudaSuccess) return e;
@@ -1546,17 +1585,22 @@ cudaError_t launch_set_len(int32_t *len, int n_layers, int max_batch, int seq, i
 }
 
 template <int MW, int GQ, int NG, bool PAIRED, bool PAGED>
-static cudaError_t launch_decode_tt(const DecodeParams &p, cudaStream_t st) {
+static cudaError_t launch_decode_tt(const DecodeParams &p, cudaStream_t st, bool attributes_only) {
     using SM = DecodeSmem<MW, GQ, NG>;
-    static bool attr_set[64] = {};
-    int dev = 0;
-    cudaGetDevice(&dev);
-    if (dev >= 0 && dev < 64 && !attr_set[dev]) {
-        cudaError_t e = cudaFuncSetAttribute(decode_split_kernel<MW, GQ, NG, PAIRED, PAGED>,
-                                             cudaFuncAttributeMaxDynamicSharedMemorySize, SM::kTotal);
-        if (e != cudaSuccess) return e;
-        attr_set[dev] = true;
+    {
+        static bool attr_set[64] = {};
+        int dev = 0;
+        cudaGetDevice(&dev);
+        if (dev < 0 || dev >= 64) return cudaErrorInvalidDevice;
+        std::lock_guard<std::mutex> lock(g_setup_mutex);
+        if (!attr_set[dev]) {
+            cudaError_t e = cudaFuncSetAttribute(decode_split_kernel<MW, GQ, NG, PAIRED, PAGED>,
+                                                 cudaFuncAttributeMaxDynamicSharedMemorySize, SM::kTotal);
+            if (e != cudaSuccess) return e;
+            attr_set[dev] = true;
+        }
     }
+    if (attributes_only) return cudaSuccess;
     const long items = (long)p.n_layers * p.B * p.Hkv * p.vgroups * p.splits;
     const unsigned grid = (unsigned)((items + kDecodeWarps - 1) / kDecodeWarps);
     cudaLaunchConfig_t cfg = {};
@@ -1573,35 +1617,66 @@ static cudaError_t launch_decode_tt(const DecodeParams &p, cudaStream_t st) {
 }
 
 template <int MW, int GQ, int NG, bool PAIRED = false>
-static cudaError_t launch_decode_t(const DecodeParams &p, cudaStream_t st) {
-    return p.ca.table ? launch_decode_tt<MW, GQ, NG, PAIRED, true>(p, st) : launch_decode_tt<MW, GQ, NG, PAIRED, false>(p, st);
+static cudaError_t launch_decode_t(const DecodeParams &p, cudaStream_t st, bool attributes_only) {
+    return p.ca.table ? launch_decode_tt<MW, GQ, NG, PAIRED, true>(p, st, attributes_only)
+                      : launch_decode_tt<MW, GQ, NG, PAIRED, false>(p, st, attributes_only);
+}
+
+// The attention kernel for p's shape: (key words, heads per item, scale/zero pairs, paired heads, paged cache) pick
+// the instantiation. attributes_only: set the instantiation's launch attributes on the current device and return.
+static cudaError_t dispatch_decode(const DecodeParams &p, cudaStream_t st, bool attributes_only) {
+    const int gq = p.gqk;                                       // (virtual) heads per work item
+    const bool ao = attributes_only;
+    cudaError_t e = cudaErrorInvalidValue;
+    H1B_DISPATCH_MW(p.m_words,
+        if (p.paired) {                                         // two 64-wide heads per slab
+            if (gq == 2 && p.groups == 4) e = launch_decode_t<MW, 2, 4, true>(p, st, ao);
+            else if (gq == 2 && p.groups == 0) e = launch_decode_t<MW, 2, 0, true>(p, st, ao);
+            else if (gq == 8 && p.groups == 4) e = launch_decode_t<MW, 8, 4, true>(p, st, ao);
+            else if (gq == 8 && p.groups == 0) e = launch_decode_t<MW, 8, 0, true>(p, st, ao);
+        } else if (p.groups == 4) {
+            if (gq == 1) e = launch_decode_t<MW, 1, 4>(p, st, ao);
+            else if (gq == 2) e = launch_decode_t<MW, 2, 4>(p, st, ao);
+            else if (gq == 4) e = launch_decode_t<MW, 4, 4>(p, st, ao);
+        } else if (p.groups == 1) {
+            if (gq == 1) e = launch_decode_t<MW, 1, 1>(p, st, ao);
+            else if (gq == 2) e = launch_decode_t<MW, 2, 1>(p, st, ao);
+            else if (gq == 4) e = launch_decode_t<MW, 4, 1>(p, st, ao);
+        } else if (p.groups == 0) {
+            if (gq == 1) e = launch_decode_t<MW, 1, 0>(p, st, ao);
+            else if (gq == 2) e = launch_decode_t<MW, 2, 0>(p, st, ao);
+            else if (gq == 4) e = launch_decode_t<MW, 4, 0>(p, st, ao);
+        }
+    );
+    return e;
+}
+
+// Everything the launchers would otherwise set on a kernel's first launch, for every kernel a cache of this shape
+// can reach, so that no later call (one recorded into a CUDA graph included) has anything left to set up.
+cudaError_t warm_kernel_attributes(int m_words, int groups, bool paired, bool paged, bool rope) {
+    DecodeParams p = {};
+    static const int32_t dummy_table = 0;
+    p.m_words = m_words; p.groups = groups; p.paired = paired ? 1 : 0;
+    p.ca.table = paged ? &dummy_table : nullptr;               // only its being null or not is looked at
+    const int heads_unpaired[3] = {1, 2, 4}, heads_paired[2] = {2, 8};
+    for (int i = 0; i < (paired ? 2 : 3); ++i) {
+        p.gqk = paired ? heads_paired[i] : heads_unpaired[i];
+        cudaError_t e = dispatch_decode(p, nullptr, true);
+        if (e != cudaSuccess) return e;
+    }
+    cudaError_t e;
+    if (m_words * 32 >= 128) e = rope ? prefill_attributes<128, true>() : prefill_attributes<128, false>();
+    else e = rope ? prefill_attributes<64, true>() : prefill_attributes<64, false>();
+    if (e != cudaSuccess) return e;
+    if ((e = prefill_values_attributes()) != cudaSuccess) return e;
+    int n = 0;
+    return sm_count(&n);
 }
 
 cudaError_t launch_decode(const DecodeParams &p, cudaStream_t st, int *launches, cudaEvent_t before,
                           cudaEvent_t after) {
-    const int gq = p.gqk;                                       // (virtual) heads per work item
-    cudaError_t e = cudaErrorInvalidValue;
     if (before) cudaEventRecord(before, st);
-    H1B_DISPATCH_MW(p.m_words,
-        if (p.paired) {                                         // two 64-wide heads per slab
-            if (gq == 2 && p.groups == 4) e = launch_decode_t<MW, 2, 4, true>(p, st);
-            else if (gq == 2 && p.groups == 0) e = launch_decode_t<MW, 2, 0, true>(p, st);
-            else if (gq == 8 && p.groups == 4) e = launch_decode_t<MW, 8, 4, true>(p, st);
-            else if (gq == 8 && p.groups == 0) e = launch_decode_t<MW, 8, 0, true>(p, st);
-        } else if (p.groups == 4) {
-            if (gq == 1) e = launch_decode_t<MW, 1, 4>(p, st);
-            else if (gq == 2) e = launch_decode_t<MW, 2, 4>(p, st);
-            else if (gq == 4) e = launch_decode_t<MW, 4, 4>(p, st);
-        } else if (p.groups == 1) {
-            if (gq == 1) e = launch_decode_t<MW, 1, 1>(p, st);
-            else if (gq == 2) e = launch_decode_t<MW, 2, 1>(p, st);
-            else if (gq == 4) e = launch_decode_t<MW, 4, 1>(p, st);
-        } else if (p.groups == 0) {
-            if (gq == 1) e = launch_decode_t<MW, 1, 0>(p, st);
-            else if (gq == 2) e = launch_decode_t<MW, 2, 0>(p, st);
-            else if (gq == 4) e = launch_decode_t<MW, 4, 0>(p, st);
-        }
-    );
+    cudaError_t e = dispatch_decode(p, st, false);
     if (e != cudaSuccess) return e;
     if (after) cudaEventRecord(after, st);
     ++*launches;
@@ -1619,6 +1694,11 @@ cudaError_t launch_decode(const DecodeParams &p, cudaStream_t st, int *launches,
         if (ec != cudaSuccess) return ec;
     }
     ++*launches;
+    return cudaGetLastError();
+}
+
+cudaError_t launch_debug_wait_timeout(int32_t *status, unsigned long long limit_ns, cudaStream_t st) {
+    debug_wait_timeout_kernel<<<1, 32, 0, st>>>(status, limit_ns);
     return cudaGetLastError();
 }
 

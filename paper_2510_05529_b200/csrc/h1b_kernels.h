@@ -18,6 +18,11 @@ cudaError_t launch_prefill(const PrefillParams &p, const NewCounts &nn, cudaStre
 cudaError_t launch_split_projection(const float *Rt, uint16_t *Rh, int n_layers, int m, cudaStream_t st);
 cudaError_t launch_decode(const DecodeParams &p, cudaStream_t st, int *launches, cudaEvent_t before = nullptr,
                           cudaEvent_t after = nullptr);
+// Sets, on the current device, the launch attributes of every kernel a cache of this shape can reach (thread-safe,
+// once per device and kernel): afterwards a launcher only launches.
+cudaError_t warm_kernel_attributes(int m_words, int groups, bool paired, bool paged, bool rope);
+// One warp waits for at most limit_ns on a barrier phase that never completes, then records the time-out in *status.
+cudaError_t launch_debug_wait_timeout(int32_t *status, unsigned long long limit_ns, cudaStream_t st);
 cudaError_t launch_set_len(int32_t *len, int n_layers, int max_batch, int seq, int value, cudaStream_t st);
 // Scores of key words [w0, w0 + nw) of every cached token of one slab against qwords[0 .. nw).
 cudaError_t launch_debug_scores(const CacheAddr &ca, int layer, int b, int kvh, const uint32_t *qwords, int len,

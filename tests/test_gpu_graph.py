@@ -59,7 +59,7 @@ def test_per_layer_steps_in_a_graph_replay_like_direct_calls(fp16_values):
         ref_out = direct.h1b_decode_step(kn.cuda(), vn.cuda(), qn.cuda(), INV_TAU)
         kn_s.copy_(kn); vn_s.copy_(vn); qn_s.copy_(qn)
         if s == 0:
-            per_layer_calls()                            # ordinary calls first (they also set kernel attributes)
+            per_layer_calls()                            # an ordinary step, so that direct and graphed caches stay level
             torch.cuda.synchronize()
             graph = torch.cuda.CUDAGraph()
             with torch.cuda.graph(graph):
@@ -179,3 +179,31 @@ def test_a_long_append_in_a_graph_appends_at_the_current_end_every_replay(fp16_v
                           graphed.h1b_decode_attention(q, INV_TAU).cpu().numpy())
     direct.close()
     graphed.close()
+
+
+def test_capture_as_the_very_first_call_of_a_new_context():
+    """Nothing has to be called before a capture: every kernel attribute a context can need is set when it is made.
+    The shape here (m = 512, one scale per value vector, three query heads per KV head) is used nowhere else in the
+    suite, so its kernels have never been launched in this process when they are recorded."""
+    w = h1b_synth.scaled(W["c1_tiny"], n_layers=2, batch=2, n_q_heads=3, n_kv_heads=1, sketch_bits=512, group_size=128)
+    lens = np.array([0, 0], np.int32)
+    cache, Rt = make_cache(w, max_seq=200)
+    T = 150                                              # a long append (tensor-core path) and a decode, both captured
+    K = torch.stack([h1b_synth.kv_rows(w, l, T)[0] for l in range(w.n_layers)]).cuda()
+    V = torch.stack([h1b_synth.kv_rows(w, l, T)[1] for l in range(w.n_layers)]).cuda()
+    q = torch.stack([h1b_synth.queries(w, l) for l in range(w.n_layers)]).cuda()
+    out = torch.zeros(q.shape, dtype=torch.float32, device="cuda")
+    torch.cuda.synchronize()
+    graph = torch.cuda.CUDAGraph()
+    with torch.cuda.graph(graph):
+        cache.h1b_append_kv(K, V)
+        cache.h1b_decode_attention(q, INV_TAU, out=out)
+    graph.replay()
+    torch.cuda.synchronize()
+    cache.h1b_sync_lengths()
+    cache.h1b_poll_status()
+    got = out.cpu().numpy()
+    for l in range(w.n_layers):
+        ref = oracle.layer(f16_bits(K[l]), f16_bits(V[l]), lens + T, f16_bits(q[l]), Rt[l], INV_TAU, w.group_size)
+        check_output(got[l], ref, ("captured first", l))
+    cache.close()

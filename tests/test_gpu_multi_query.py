@@ -208,3 +208,41 @@ def test_more_units_than_the_scratch_holds_run_in_layer_passes():
         ref = oracle.attention(gscore[:n_i], w.sketch_bits, 16.0, codes[:n_i], scale[:n_i], zero[:n_i], w.group_size)
         check_output(out[l, b, i, h], ref, ("layer passes", l, b, i, h))
     cache.close()
+
+
+def test_one_layer_a_large_batch_and_sixteen_query_tokens():
+    """The split-K scratch is sized for the largest multi-query call the interface allows: one layer, 128 sequences of
+    32 heads and 16 query tokens each (16384 work items of four heads) must run, and a call that cannot run must fail
+    before anything is launched or changed."""
+    w = h1b_synth.scaled(W["c1_tiny"], n_layers=1, batch=128, n_q_heads=32, n_kv_heads=32)
+    lens = np.full((128,), 40, np.int32)
+    lens[5] = 17
+    cache, Rt, K, V, lens = _fill(w, lens, max_seq=64)
+    q = _queries(w, 16)
+    out = cache.h1b_decode_attention_multi(q.cuda(), 16.0).cpu().numpy()
+    torch.cuda.synchronize()
+    cache.h1b_poll_status()
+    e2e = oracle.layer_multi(f16_bits(K[0]), f16_bits(V[0]), lens, f16_bits(q[0]), Rt[0], 16.0, w.group_size)
+    checked = 0
+    for b in (0, 5, 127):
+        words = np.stack([cache.h1b_export_cache(0, b, g, 0, int(lens[b]))[0] for g in range(w.n_kv_heads)])
+        for g in range(w.n_kv_heads):
+            kbits = binding.unpack_words(words[g], w.sketch_bits)
+            if np.array_equal(kbits, oracle.sketch(f16_bits(K[0, b, :lens[b], g]), Rt[0])):
+                check_output(out[0, b, :, g], e2e[b, :, g], ("large batch, 16 query tokens", b, g))
+                checked += 1
+    assert checked > 60
+    # a step that cannot run (forced splits beyond what the scratch holds) fails on the host before anything is
+    # launched: no kernel, no new token, lengths as they were
+    cache.h1b_set_splits(64)                             # 64 splits x 4096 slabs = 262144 work items
+    kn = torch.zeros((1, 128, 1, 32, 128), dtype=torch.float16, device="cuda")
+    qn = torch.zeros((1, 128, 32, 128), dtype=torch.float16, device="cuda")
+    n0 = cache.h1b_launch_count()
+    with pytest.raises(binding.H1BError) as err:
+        cache.h1b_decode_step(kn, kn, qn, 16.0)
+    assert err.value.code == -4 and cache.h1b_launch_count() == n0
+    assert np.array_equal(cache.h1b_get_lengths(0), lens)                # host mirror and device agree, nothing appended
+    cache.h1b_set_splits(0)
+    cache.h1b_decode_step(kn, kn, qn, 16.0)
+    assert np.array_equal(cache.h1b_get_lengths(0), lens + 1)
+    cache.close()

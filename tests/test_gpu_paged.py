@@ -137,6 +137,13 @@ def test_paged_against_the_oracle_and_table_errors():
             cache.h1b_set_block_table(0, bad)
     with pytest.raises(binding.H1BError):                # fewer pages than the cached tokens need
         cache.h1b_set_block_table(0, [5, 0])
+    for shared in ([5, 0, 2], [5, 0, 3, 4]):             # pages 2 and 4 belong to sequence 1
+        with pytest.raises(binding.H1BError) as err:
+            cache.h1b_set_block_table(0, shared)
+        assert err.value.code == -1 and "belongs to sequence 1" in str(err.value)
+    with pytest.raises(binding.H1BError):                # a page listed twice
+        cache.h1b_set_block_table(0, [5, 0, 3, 3])
+    cache.h1b_set_block_table(0, [5, 0, 3, 1])           # its own pages again plus a free one: fine
     cache.close()
     plain, _ = make_cache(w, max_seq=64)
     with pytest.raises(binding.H1BError):
