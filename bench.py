@@ -38,6 +38,8 @@ INV_TAU = 16.0
 # grows in proportion to the cached tokens, so the bench scales it to the context it actually ran; the line says
 # where the ratio was taken (`traffic_ratio_measured_at`), so that a stale one shows.
 NCU_TRAFFIC_PER_ALGORITHMIC_BYTE = 1.0130
+NCU_TRAFFIC_MEASURED_AT = {"workload": "c2_7b_8k", "tokens": 8199, "dram_bytes": 816.5e6, "algorithmic_bytes": 806.0e6,
+                           "kernel": "decode_split_kernel<4,1,4,0,0>"}
 
 
 def measured_peaks():
@@ -91,13 +93,22 @@ class ClockSampler(threading.Thread):
                 break
             time.sleep(0.002)
 
-    def stop(self):
+    def mark(self):
+        """The timed region starts here: samples taken before it (warm-up, also under load) are kept apart."""
+        self.marked_at = len(self.samples)
+
+    def stop(self, ms_per_step=None):
         self._stop_evt.set()
         if self.ident is not None:                  # started
             self.join(timeout=2)
-        med = float(np.median(self.samples)) if self.samples else None
-        return {"sm_mhz": med, "sm_max_mhz": self.max_mhz, "reasons": sorted(self.reasons),
-                "samples": len(self.samples)}
+        at = getattr(self, "marked_at", 0)
+        timed = self.samples[at:] or self.samples   # a very short timed region may have caught no sample of its own
+        med = float(np.median(timed)) if timed else None
+        out = {"sm_mhz": med, "sm_max_mhz": self.max_mhz, "reasons": sorted(self.reasons),
+               "samples": len(self.samples), "samples_in_timed_region": len(self.samples) - at}
+        if med is not None and ms_per_step is not None:
+            out["ms_per_step_x_sm_mhz"] = ms_per_step * med     # clock-normalised time: comparable from box to box
+        return out
 
 
 def gpu_index() -> int:
@@ -224,14 +235,15 @@ def run_ours(args):
         pdist.barrier()
         torch.cuda.synchronize()
 
+    sampler = ClockSampler(gpu_index())
+    sampler.start()                                   # from the warm-up on: the clocks under load, also for short runs
     for i in range(warmup):
         step(i)
     barrier()
     launches0 = cache.h1b_launch_count()
     cache.h1b_set_profiling(True)
     cache.h1b_read_profile()
-    sampler = ClockSampler(gpu_index())
-    sampler.start()
+    sampler.mark()
     ev0, ev1 = torch.cuda.Event(enable_timing=True), torch.cuda.Event(enable_timing=True)
     len_first = cache.h1b_get_lengths(0)[:w.batch].astype(np.int64) + Tq
     ctx_first = int(len_first.max())
@@ -241,8 +253,8 @@ def run_ours(args):
         step(warmup + i)
     ev1.record(stream)
     barrier()
-    clocks = sampler.stop()
     ms_total = ev0.elapsed_time(ev1)
+    clocks = sampler.stop(ms_total / steps)
     launches = cache.h1b_launch_count() - launches0
     kern_ms, kern_n = cache.h1b_read_profile()
     cache.h1b_set_profiling(False)
@@ -325,6 +337,7 @@ def run_ours(args):
                 # the capture is of the default configuration's kernel; variants have no captured traffic
                 "traffic": (NCU_TRAFFIC_PER_ALGORITHMIC_BYTE * alg_bytes) if w.name == "c2_7b_8k" else None,
                 "traffic_source": "ncu capture at 8199 tokens, scaled by algorithmic bytes" if w.name == "c2_7b_8k" else None,
+                "traffic_ratio_measured_at": NCU_TRAFFIC_MEASURED_AT if w.name == "c2_7b_8k" else None,
                 "alg_bytes_per_launch": alg_bytes,
                 "kernel_ms_avg": kern_ms_avg, "kernel_launches_timed": kern_n,
                 "step_gbs": alg_bytes / (ms_per_step * 1e-3) / 1e9}
@@ -350,8 +363,13 @@ def run_ours(args):
         line["layer_sequential"] = {"value": pdist.whole_job_rate(w.batch, job_ranks, seq_ms_total / steps * 1e-3), "unit": UNIT,
                                     "ms_per_step": seq_ms_total / steps, "launches_per_step": 3 * w.n_layers,
                                     "how": "h1b_decode_step_layers once per layer, one CUDA graph per step, replayed"}
-    if rank == 0 and world == 1 and not args.no_cpu_baseline and w.name == "c2_7b_8k":
-        line["cpu_baseline"] = cpu_baseline(sample_layers=1, steps=5, warmup=1)
+    if args.check and rank == 0:                      # after all timing: the cache just timed against the oracle
+        line["check"] = check_against_oracle(cache, w, wr, Rt, lens0, kv_rows, dev)
+    if rank == 0 and world == 1 and not args.no_cpu_baseline:
+        if w.name == "c2_7b_8k":
+            line["cpu_baseline"] = cpu_baseline(sample_layers=1, steps=5, warmup=1)
+        elif args.workload in ("c3_7b_batched", "c4_gqa_32k", "c6_60m_8k") and not (args.fp16_values or args.rope or Tq > 1):
+            line["cpu_baseline"] = cpu_baseline(steps=1, warmup=0, sample=OracleSample(1, w, sample_batch=min(w.batch, 2)))
     cache.close()
     pdist.finish()
     if rank == 0:
@@ -377,10 +395,11 @@ def run_prefill(args, w, pdist, rank, world, local):
     times = []
     launches0 = 0
     sampler = ClockSampler(gpu_index())
+    sampler.start()
     for i in range(args.warmup + args.steps):
         if i == args.warmup:
             launches0 = cache.h1b_launch_count()
-            sampler.start()
+            sampler.mark()
         cache.h1b_reset(-1)                           # synchronous, outside the timed call
         e0, e1 = torch.cuda.Event(enable_timing=True), torch.cuda.Event(enable_timing=True)
         pdist.barrier(); torch.cuda.synchronize()
@@ -431,8 +450,11 @@ def run_prefill(args, w, pdist, rank, world, local):
                          "peak": peak, "peak_kind": peak_kind, "unit": "GB/s", "frac": alg_bytes / (ms * 1e-3) / 1e9 / peak,
                          "alg_bytes_per_launch": alg_bytes, "traffic": None,
                          "tensor_tflops": rows * w.head_dim * w.sketch_bits * 2 * 2 / (ms * 1e-3) / 1e12}}
+    line["clocks"]["ms_per_step_x_sm_mhz"] = ms * clocks["sm_mhz"] if clocks.get("sm_mhz") else None
     if prompt_attention:
         line["prompt_attention"] = prompt_attention
+    if rank == 0 and world == 1 and not args.no_cpu_baseline and not (args.fp16_values or args.rope):
+        line["cpu_baseline"] = prefill_cpu_baseline(w)
     cache.close()
     pdist.finish()
     if rank == 0:
@@ -441,47 +463,57 @@ def run_prefill(args, w, pdist, rank, world, local):
 
 # --------------------------------------------------------------------------- oracle on host cores
 class OracleSample:
-    """The fp64 oracle, as it stands, on a bounded sample of the bench workload:
-    `sample_layers` of the 32 layers (all 32 heads, 8192 cached tokens each). One
-    decode step = compress the new token (Eq. 2, Eq. 4) and attend over the cached
-    history (Eq. 2 on q, Eq. 3, Eq. 5). The history is compressed once, untimed."""
+    """The fp64 oracle, as it stands, on a bounded sample of a decode workload: `sample_layers` of its layers and
+    `sample_batch` of its sequences (all heads, every cached token of those). One decode step = compress the new
+    token (Eq. 2, Eq. 4) and attend over the cached history (Eq. 2 on q, Eq. 3, Eq. 5). The history is compressed
+    once, untimed. The timed figure is scaled to the whole workload (layers and sequences are independent units)."""
 
-    def __init__(self, sample_layers: int = 1):
+    def __init__(self, sample_layers: int = 1, w=None, sample_batch: int | None = None):
         import torch
 
         import h1b_synth
         import oracle
-        self.oracle, self.w = oracle, h1b_synth.WORKLOADS["c2_7b_8k"]
+        self.oracle, self.w = oracle, (w or h1b_synth.WORKLOADS["c2_7b_8k"])
         w, T = self.w, self.w.context
+        self.sample_batch = B = min(w.batch, sample_batch or w.batch)
+        self.lens = h1b_synth.lengths(w)[:B].copy()
         self.layers = []
         for l in range(sample_layers):
             Rt = h1b_synth.projection(h1b_synth.layer_seed(w, l, 99), w.head_dim, w.sketch_bits)
-            K, V = h1b_synth.kv_rows(w, l, T)
-            q = h1b_synth.queries(w, l)
+            K, V = h1b_synth.kv_rows(w, l, T, batch=B)
+            q = h1b_synth.queries(w, l, batch=B)
             Kb = K.view(dtype=torch.int16).numpy().view(np.uint16)
             Vb = V.view(dtype=torch.int16).numpy().view(np.uint16)
             qb = q.view(dtype=torch.int16).numpy().view(np.uint16)
-            # the whole layer is compressed once; each timed step recompresses the newest token into slot T-1
-            cache = oracle.compress(Kb, Vb, Rt)
-            self.layers.append((Rt, Kb[:, T - 1:], Vb[:, T - 1:], qb, cache))
-        self.lens = np.full((w.batch,), T, dtype=np.int32)
+            # the whole layer is compressed once; each timed step recompresses every sequence's newest token
+            cache = oracle.compress(Kb, Vb, Rt, w.group_size)
+            new_k = np.stack([Kb[b, self.lens[b] - 1:self.lens[b]] for b in range(B)])
+            new_v = np.stack([Vb[b, self.lens[b] - 1:self.lens[b]] for b in range(B)])
+            self.layers.append((Rt, new_k, new_v, qb, cache))
 
     def step(self) -> float:
-        """Seconds for one decode step over the sampled layers."""
-        o, T = self.oracle, self.w.context
+        """Seconds for one decode step over the sampled layers and sequences."""
+        o, w = self.oracle, self.w
         t0 = time.perf_counter()
         for Rt, k_new, v_new, qb, cache in self.layers:
-            new = o.compress(k_new, v_new, Rt)
+            new = o.compress(k_new, v_new, Rt, w.group_size)
             for dst, src in zip(cache, new):
-                dst[:, :, T - 1:T] = src
-            o.decode_cached(cache, self.lens, qb, Rt, INV_TAU)
+                for b in range(self.sample_batch):
+                    dst[b, :, self.lens[b] - 1:self.lens[b]] = src[b]
+            o.decode_cached(cache, self.lens, qb, Rt, INV_TAU, w.group_size)
         return time.perf_counter() - t0
+
+    @property
+    def scale(self) -> float:
+        """Whole workload over the sample (independent units: layers x sequences)."""
+        return (self.w.n_layers / len(self.layers)) * (self.w.batch / self.sample_batch)
 
     def describe(self, n_timed: int):
         w = self.w
-        return ("%d of %d layers (%d heads x %d cached tokens each), mean of %d timed steps, scaled to %d layers; "
-                "history compressed once outside the timed region"
-                % (len(self.layers), w.n_layers, w.n_kv_heads, w.context, n_timed, w.n_layers))
+        return ("%s: %d of %d layers, %d of %d sequences (%d KV heads x %s cached tokens each), mean of %d timed step(s), "
+                "scaled to the whole workload (extrapolated); history compressed once outside the timed region"
+                % (w.name, len(self.layers), w.n_layers, self.sample_batch, w.batch, w.n_kv_heads,
+                   "/".join(str(int(x)) for x in self.lens), n_timed))
 
 
 def cpu_baseline(sample_layers: int = 1, steps: int = 3, warmup: int = 1, sample: OracleSample | None = None):
@@ -489,18 +521,81 @@ def cpu_baseline(sample_layers: int = 1, steps: int = 3, warmup: int = 1, sample
     for _ in range(warmup):
         s.step()
     times = [s.step() for _ in range(max(1, steps))]
-    step_s = float(np.mean(times)) * s.w.n_layers / len(s.layers)
+    step_s = float(np.mean(times)) * s.scale
     cores = s.oracle.threads()
     out = {"value": s.w.batch / step_s, "unit": UNIT, "cores": cores, "kind": "oracle",
            "sample": s.describe(len(times)), "ms_per_step": step_s * 1e3}
-    if cores > 1:                                       # the same sample once more on a single thread
+    if cores > 1 and sample is None:                    # the same sample once more on a single thread
         s.oracle.set_threads(1)
         try:
-            one_s = s.step() * s.w.n_layers / len(s.layers)
+            one_s = s.step() * s.scale
         finally:
             s.oracle.set_threads(cores)
         out["one_thread"] = {"value": s.w.batch / one_s, "unit": UNIT, "ms_per_step": one_s * 1e3, "sample": "one timed step"}
     return out
+
+
+def prefill_cpu_baseline(w, sample_tokens: int = 256):
+    """The oracle's compression (Eq. 2, Eq. 4) of `sample_tokens` prompt tokens of one layer (all KV heads), scaled to
+    the whole prompt and all layers."""
+    import torch
+
+    import h1b_synth
+    import oracle
+    Rt = h1b_synth.projection(h1b_synth.layer_seed(w, 0, 99), w.head_dim, w.sketch_bits)
+    K, V = h1b_synth.kv_rows(w, 0, sample_tokens)
+    Kb = K.view(dtype=torch.int16).numpy().view(np.uint16)
+    Vb = V.view(dtype=torch.int16).numpy().view(np.uint16)
+    oracle.compress(Kb[:, :8], Vb[:, :8], Rt, w.group_size)             # warm-up
+    t0 = time.perf_counter()
+    oracle.compress(Kb, Vb, Rt, w.group_size)
+    dt = time.perf_counter() - t0
+    step_s = dt * (w.context / sample_tokens) * w.n_layers
+    return {"value": w.batch * w.context / step_s, "unit": UNIT, "cores": oracle.threads(), "kind": "oracle",
+            "sample": "%s: %d of %d prompt tokens of 1 of %d layers (all %d KV heads), one timed pass, scaled to the whole "
+                      "prompt (extrapolated)" % (w.name, sample_tokens, w.context, w.n_layers, w.n_kv_heads),
+            "ms_per_step": step_s * 1e3}
+
+
+def check_against_oracle(cache, w, wr, Rt, lens0, kv_rows, dev, units: int = 3):
+    """Opt-in leg, after all timing: three seeded (layer, sequence, KV head) units of the cache that was just timed.
+    Their prompt part is compared with the oracle's compression of the same rows (decision flips inside the 1e-5
+    boundary windows are counted, one outside fails), and one more decode over everything they now hold is compared
+    with the oracle's Eq. 3 + Eq. 5 on the exported cache (integer scores bit for bit)."""
+    import torch
+
+    import h1b_synth
+    tests_dir = os.path.join(ROOT, "tests")
+    if tests_dir not in sys.path:
+        sys.path.insert(0, tests_dir)
+    import h1b_testlib as tl
+    rng = np.random.default_rng(20251005)
+    gq = w.n_q_heads // w.n_kv_heads
+    q = torch.stack([h1b_synth.normal_fp16(h1b_synth.layer_seed(wr, l, 31), (w.batch, w.n_q_heads, w.head_dim), str(dev))
+                     for l in range(w.n_layers)])
+    out = cache.h1b_decode_attention(q, INV_TAU).cpu().numpy()
+    cache.h1b_poll_status()
+    res = {"units": [], "flips_inside": 0, "flips_outside": 0, "max_abs": 0.0, "max_rel": 0.0}
+    for _ in range(units):
+        l, b, g = int(rng.integers(w.n_layers)), int(rng.integers(w.batch)), int(rng.integers(w.n_kv_heads))
+        n0 = int(lens0[b])
+        K, V = kv_rows(l, int(lens0.max()))
+        st = tl.append_parity(cache, l, b, g, tl.f16_bits(K[b, :n0, g]), tl.f16_bits(V[b, :n0, g]), Rt[l])   # raises on a flip outside
+        res["flips_inside"] += st["bit_flips_in"] + st["code_flips_in"] + st["scale_flips_in"]
+        n = int(cache.h1b_get_lengths(l)[b])
+        for hh in range(gq):
+            h = g * gq + hh
+            ref, qf = tl.oracle_from_export(cache, l, b, h, q[l, b, h].contiguous(), n, INV_TAU, Rt[l])
+            res["flips_inside"] += qf
+            err = np.abs(out[l, b, h].astype(np.float64) - ref)
+            big = np.abs(ref) >= 1e-3
+            res["max_abs"] = max(res["max_abs"], float(err.max()))
+            if big.any():
+                res["max_rel"] = max(res["max_rel"], float((err[big] / np.abs(ref[big])).max()))
+        res["units"].append([l, b, g])
+        del K, V
+    res["within_tolerance"] = bool(res["max_abs"] <= tl.MAX_ABS and res["max_rel"] <= tl.MAX_REL)
+    return res
 
 
 def run_reference(args):
@@ -529,6 +624,8 @@ def main():
     ap.add_argument("--warmup", type=int, default=30)
     ap.add_argument("--impl", default="ours", choices=["ours", "reference"])
     ap.add_argument("--no-cpu-baseline", action="store_true")
+    ap.add_argument("--check", action="store_true",
+                    help="after all timing: three seeded units of the timed cache against the oracle (flip counts, errors)")
     ap.add_argument("--sketch-bits", type=int, default=0, help="override m (64, 128, 256, 512)")
     ap.add_argument("--group-size", type=int, default=0, help="override G (32, or 128 = one scale per value vector)")
     ap.add_argument("--no-layer-sequential", action="store_true", help="skip the per-layer CUDA-graph measurement")

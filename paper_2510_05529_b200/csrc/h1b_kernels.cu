@@ -841,17 +841,33 @@ __global__ void set_len_kernel(int32_t *len, int n_layers, int max_batch, int se
 constexpr int kDecodeWarps = H1B_DECODE_WARPS;
 constexpr int kStages = H1B_DECODE_STAGES;
 // Resident blocks per SM that the register allocation must allow: the kernel hides latency with warps.
+#ifndef H1B_QUERY_IN_SMEM
+#define H1B_QUERY_IN_SMEM 1
+#endif
+#ifndef H1B_GQ4_BLOCKS
+#define H1B_GQ4_BLOCKS 4            // four heads per item, up to 256 sketch bits: 128 registers with the query words in shared memory
+#endif
 constexpr int decode_min_blocks(int gq, int ng, int mw) {
-    return gq == 8 ? (mw <= 8 ? 3 : 2) : (ng == 0 ? 3 : (gq == 1 ? 5 : (gq == 2 ? 4 : 3)));
+    return gq == 8 ? (mw <= 8 ? 3 : 2) : (ng == 0 ? 3 : (gq == 1 ? 5 : (gq == 2 ? 4 : (mw <= 8 ? H1B_GQ4_BLOCKS : 3))));
 }
 constexpr int kHamSentinel = 1 << 20;
+// Which variants compute the next chunk's distances inside the current chunk's tensor-core phase.
+#ifndef H1B_PIPELINE_MIN_HEADS
+#define H1B_PIPELINE_MIN_HEADS 4
+#endif
+__host__ __device__ constexpr bool decode_pipelined(int gq, int ng, bool paired) { return gq >= H1B_PIPELINE_MIN_HEADS; }
 
 template <int MW, int GQ, int NG>                 // NG: scale/zero pairs per value vector (4 or 1); 0 = fp16 values
 struct DecodeSmem {
     static constexpr int kChunkBytes = MW * 128 + (NG == 0 ? 8192 : 2048 + 128 * NG);
     // fp16-value chunks are four times larger: two in flight per warp, so that three blocks still fit an SM
     static constexpr int kNStages = (NG == 0 && kStages > 2) ? 2 : kStages;
-    static constexpr int kPerWarp = kNStages * kChunkBytes + GQ * 32 * 4 + 128;   // ring, p buffer, barriers
+    // Four or more heads per item: the query sketches (GQ * MW words, warp-uniform) stay in shared memory and are read
+    // with broadcast loads, which frees GQ * MW registers per thread: one more block of warps fits an SM.
+    static constexpr bool kQueryInSmem = H1B_QUERY_IN_SMEM && GQ == 4 && NG != 0 && MW >= 4;
+    static constexpr int kQueryBytes = kQueryInSmem ? GQ * MW * 4 : 0;
+    static constexpr int kQueryOff = kNStages * kChunkBytes + GQ * 32 * 4 + 128;
+    static constexpr int kPerWarp = kQueryOff + kQueryBytes;                      // ring, p buffer, barriers, query words
     static constexpr int kTotal = kDecodeWarps * kPerWarp;
 };
 
@@ -861,33 +877,69 @@ struct DecodeState {
     int hmin[GQ];               // running minimum Hamming distance (= running maximum logit)
     float ssum[GQ];             // per-lane partial sum of the weights
     float accz[GQ][NG ? NG : 1]; // per-lane partial sum of p * zero (unused with fp16 values)
-    uint32_t qw[GQ][MW];        // query sketches
+    static constexpr bool kQS = DecodeSmem<MW, GQ, NG>::kQueryInSmem;
+    uint32_t qw[kQS ? 1 : GQ][kQS ? 1 : MW];   // query sketches (unless they live in shared memory: qs)
+    const uint32_t *qs;         // kQS: the item's query sketches in shared memory, [GQ][MW]
     float zero[4];              // an opaque quad of zeros: C operand of each chunk's first MMA
 };
 
-// One chunk. TAIL: head h attends only to the chunk's first n_valid[h] tokens (the last chunks of a split; with
-// several query tokens, each one's causal limit).
+// One chunk is processed in three pieces, so that the kernel can run the popcounts of the NEXT chunk (the quarter-rate
+// pipe) inside the tensor-core phase of the current one (logic pipe, tensor pipe):
+//   chunk_scores   lane = token: Hamming distance to each head of the item (Eq. 3)
+//   chunk_weights  online softmax on those distances: running minimum, weights p to shared memory, sums (Eq. 5)
+//   chunk_values   the weighted sum of the chunk's values on the tensor cores (Eq. 5)
+// TAIL: head h attends only to the chunk's first n_valid[h] tokens (the last chunks of a split; with several query
+// tokens, each one's causal limit).
 // PAIRED (head dimension 64): the slab holds two heads side by side, head h in channels 64h..64h+63 and in key words
 // [h MW/2, (h+1) MW/2). GQ = 2 then counts those two heads; the accumulator columns are laid out as for one head,
 // (value group, part), and group g simply takes the weights of head g / 2.
-template <int MW, int GQ, int NG, bool TAIL, bool PAIRED>
-__device__ __forceinline__ void decode_chunk(DecodeState<MW, GQ, NG> &st, const unsigned char *ch, float *p_s,
-                                             int lane, const int (&n_valid)[GQ], float c2) {
-    static_assert(!PAIRED || ((GQ == 2 || GQ == 8) && (NG == 4 || NG == 0)),
-                  "two 64-wide KV heads per slab (one or four heads on each), groups of 32 or fp16 values");
-    constexpr int GQH = PAIRED ? GQ / 2 : GQ;  // (virtual) heads on each KV head of the slab
-    constexpr bool P8 = PAIRED && GQ == 8;     // four heads on each half: the columns of a channel block are its own half's heads
-    constexpr int GQL = PAIRED ? (P8 ? 4 : 1) : GQ;   // heads the accumulator columns are laid out for
-    constexpr int GPF = 4 / GQL;               // value groups covered by one B fragment (4 groups per vector)
-    constexpr int NB = (NG == 1) ? 1 : GQL;    // B fragments per 16-token block (one scale per vector: one fragment)
-    constexpr int MWH = PAIRED ? MW / 2 : MW;  // key words of one head
-    constexpr int VAL = MW * 128, ZERO = VAL + 2048, SCALE = ZERO + 64 * NG;
-    const int jq = lane & 3;
 
-    // ---------------- phase 1
+// Part `piece` of `pieces` of the distances of one chunk: the (head, word) pairs are dealt out over the pieces, so that
+// the caller can spread them over another phase. ham[] must start at zero; kw[] are the lane's key words.
+template <int MW, int GQ, int NG, bool PAIRED, int PIECES>
+__device__ __forceinline__ void scores_piece(const DecodeState<MW, GQ, NG> &st, const uint32_t (&kw)[MW], int (&ham)[GQ],
+                                             int piece) {
+    constexpr int GQH = PAIRED ? GQ / 2 : GQ;
+    constexpr int MWH = PAIRED ? MW / 2 : MW;
+    constexpr bool QS = DecodeState<MW, GQ, NG>::kQS;
+    // units: with the query words in shared memory one unit is (head, four words) = one broadcast 16-byte load;
+    // otherwise (head, word)
+    constexpr int UNITS = QS ? GQ * (MW / 4) : GQ * MWH;
+    constexpr int PER = (UNITS + PIECES - 1) / PIECES;
+#pragma unroll
+    for (int k = 0; k < PER; ++k) {
+        const int u = piece * PER + k;                  // compile-time once the caller's loops are unrolled
+        if (u < UNITS) {
+            if constexpr (QS) {
+                const int h = u / (MW / 4), w4 = u % (MW / 4);
+                const uint4 q4 = *reinterpret_cast<const uint4 *>(st.qs + h * MW + 4 * w4);   // every lane the same 16 bytes
+                ham[h] += __popc(kw[4 * w4] ^ q4.x) + __popc(kw[4 * w4 + 1] ^ q4.y) + __popc(kw[4 * w4 + 2] ^ q4.z) +
+                          __popc(kw[4 * w4 + 3] ^ q4.w);
+            } else {
+                const int h = u / MWH, w = u % MWH;
+                ham[h] += __popc(kw[(PAIRED ? (h / GQH) * MWH : 0) + w] ^ st.qw[h][w]);
+            }
+        }
+    }
+}
+
+template <int MW, int GQ, int NG, bool PAIRED>
+__device__ __forceinline__ void chunk_scores(const DecodeState<MW, GQ, NG> &st, const unsigned char *ch, int lane,
+                                             int (&ham)[GQ]) {
     uint32_t kw[MW];
 #pragma unroll
     for (int w = 0; w < MW; ++w) kw[w] = *reinterpret_cast<const uint32_t *>(ch + w * 128 + lane * 4);
+#pragma unroll
+    for (int h = 0; h < GQ; ++h) ham[h] = 0;
+    scores_piece<MW, GQ, NG, PAIRED, 1>(st, kw, ham, 0);
+}
+
+template <int MW, int GQ, int NG, bool TAIL, bool PAIRED>
+__device__ __forceinline__ void chunk_weights(DecodeState<MW, GQ, NG> &st, const int (&ham_in)[GQ], const unsigned char *ch,
+                                              float *p_s, int lane, const int (&n_valid)[GQ], float c2, float (&scl)[GQ]) {
+    constexpr int GQH = PAIRED ? GQ / 2 : GQ;  // (virtual) heads on each KV head of the slab
+    constexpr bool P8 = PAIRED && GQ == 8;     // four heads on each half: the columns of a channel block are its own half's heads
+    constexpr int VAL = MW * 128, ZERO = VAL + 2048;
     float zf[NG ? NG : 1];
     if (NG == 0) {
         zf[0] = 0.f;
@@ -898,12 +950,9 @@ __device__ __forceinline__ void decode_chunk(DecodeState<MW, GQ, NG> &st, const 
     } else {
         zf[0] = __half2float(*reinterpret_cast<const __half *>(ch + ZERO + lane * 2));
     }
-    float scl[GQ];
 #pragma unroll
     for (int h = 0; h < GQ; ++h) {
-        int ham = 0;
-#pragma unroll
-        for (int w = 0; w < MWH; ++w) ham += __popc(kw[(PAIRED ? (h / GQH) * MWH : 0) + w] ^ st.qw[h][w]);
+        const int ham = ham_in[h];
         const bool valid = !TAIL || lane < n_valid[h];
         const int cmin = __reduce_min_sync(0xffffffffu, (TAIL && !valid) ? kHamSentinel : ham);
         scl[h] = 1.f;
@@ -924,6 +973,32 @@ __device__ __forceinline__ void decode_chunk(DecodeState<MW, GQ, NG> &st, const 
             st.accz[h][g] = fmaf(pv, zf[(NG > 1 && P8) ? ((h / GQH) * 2 + g) : g], st.accz[h][g]);
         p_s[h * 32 + lane] = pv;
     }
+}
+
+// PIPE: the distances of the chunk at `ch_next` are computed on the way (into ham_next), a slice between the tensor-core
+// steps, so that their popcounts overlap the unpacking and the MMAs of this chunk instead of forming a phase of their own.
+template <int MW, int GQ, int NG, bool PAIRED, bool PIPE>
+__device__ __forceinline__ void chunk_values(DecodeState<MW, GQ, NG> &st, const unsigned char *ch, const float *p_s,
+                                             int lane, const float (&scl)[GQ], const unsigned char *ch_next,
+                                             int (&ham_next)[GQ]) {
+    static_assert(!PAIRED || ((GQ == 2 || GQ == 8) && (NG == 4 || NG == 0)),
+                  "two 64-wide KV heads per slab (one or four heads on each), groups of 32 or fp16 values");
+    constexpr int GQH = PAIRED ? GQ / 2 : GQ;  // (virtual) heads on each KV head of the slab
+    constexpr bool P8 = PAIRED && GQ == 8;     // four heads on each half: the columns of a channel block are its own half's heads
+    constexpr int GQL = PAIRED ? (P8 ? 4 : 1) : GQ;   // heads the accumulator columns are laid out for
+    constexpr int GPF = 4 / GQL;               // value groups covered by one B fragment (4 groups per vector)
+    constexpr int NB = (NG == 1) ? 1 : GQL;    // B fragments per 16-token block (one scale per vector: one fragment)
+    constexpr int VAL = MW * 128, ZERO = VAL + 2048, SCALE = ZERO + 64 * NG;
+    constexpr int SLOTS = 16;                  // tensor-core steps of a chunk (2 halves x 2 token blocks x 4 channel blocks)
+    const int jq = lane & 3;
+
+    uint32_t kwn[PIPE ? MW : 1];
+    if constexpr (PIPE) {
+#pragma unroll
+        for (int w = 0; w < MW; ++w) kwn[w] = *reinterpret_cast<const uint32_t *>(ch_next + w * 128 + lane * 4);
+#pragma unroll
+        for (int h = 0; h < GQ; ++h) ham_next[h] = 0;
+    }
     // factors by which this lane's accumulator columns 2jq, 2jq+1 shrink when a running max moved (else 1)
     // (P8: the channel blocks of the slab's second half take the factors of heads 4..7, f0b and f1b)
     float f0, f1, f0b = 1.f, f1b = 1.f;
@@ -935,10 +1010,9 @@ __device__ __forceinline__ void decode_chunk(DecodeState<MW, GQ, NG> &st, const 
     else if (GQ == 1) { f0 = scl[0]; f1 = scl[0]; }
     else if (GQ == 2) { f0 = scl[0]; f1 = scl[GQ > 1 ? 1 : 0]; }
     else { f0 = (jq & 1) ? scl[GQ > 2 ? 2 : 0] : scl[0]; f1 = (jq & 1) ? scl[GQ > 3 ? 3 : 0] : scl[GQ > 1 ? 1 : 0]; }
-    __syncwarp();
 
     if constexpr (NG == 0) {
-        // ---------------- phase 2, fp16 values: out^T (channels x columns) += V^T x W with A = the cached values as
+        // ---------------- fp16 values: out^T (channels x columns) += V^T x W with A = the cached values as
         // they are (one 16-byte load per channel block and lane) and B = the weights p split into hi and lo parts;
         // column n = lane/4 = (part, head). Same per-chunk zero start and fold as below.
         const int part = lane >> 4, idx = (lane >> 2) & 3;
@@ -973,6 +1047,7 @@ __device__ __forceinline__ void decode_chunk(DecodeState<MW, GQ, NG> &st, const 
                     const uint4 a = *reinterpret_cast<const uint4 *>(ch + VAL + vb * kHalfBlockBytes + cb * 512 + lane * 16);
                     if (vb == 0) mma_f16_16816_from(tmp[i], a.x, a.y, a.z, a.w, bf[vb][f][0], bf[vb][f][1], st.zero);
                     else mma_f16_16816(tmp[i], a.x, a.y, a.z, a.w, bf[vb][f][0], bf[vb][f][1]);
+                    if constexpr (PIPE) scores_piece<MW, GQ, NG, PAIRED, SLOTS>(st, kwn, ham_next, (half * 2 + vb) * 4 + i);
                 }
             }
             const float h0 = (P8 && half) ? f0b : g0, h1 = (P8 && half) ? f1b : g1;
@@ -985,11 +1060,10 @@ __device__ __forceinline__ void decode_chunk(DecodeState<MW, GQ, NG> &st, const 
                 st.acc[cb][3] = fmaf(st.acc[cb][3], h1, tmp[i][3]);
             }
         }
-        __syncwarp();
         return;
     }
 
-    // ---------------- phase 2
+    // ---------------- 4-bit values
     // Column n = lane/4 of a B fragment is (part, idx): part 0 = hi, part 1 = lo; idx = value group (GQ 1),
     // (group in pair, head) (GQ 2) or head (GQ 4). This lane computes the weights of ONE token pair
     // (tokens 2jq, 2jq+1 if part 0, else 2jq+8, 2jq+9), both parts, and swaps one of them with lane ^ 16.
@@ -1037,6 +1111,7 @@ __device__ __forceinline__ void decode_chunk(DecodeState<MW, GQ, NG> &st, const 
                 codes_to_f16x2(wv[i], a);
                 if (vb == 0) mma_f16_16816_from(tmp[i], a[0], a[1], a[2], a[3], bf[vb][bi][0], bf[vb][bi][1], st.zero);
                 else mma_f16_16816(tmp[i], a[0], a[1], a[2], a[3], bf[vb][bi][0], bf[vb][bi][1]);
+                if constexpr (PIPE) scores_piece<MW, GQ, NG, PAIRED, SLOTS>(st, kwn, ham_next, (half * 2 + vb) * 4 + i);
             }
         }
         const float h0 = (P8 && half) ? f0b : f0, h1 = (P8 && half) ? f1b : f1;
@@ -1049,7 +1124,6 @@ __device__ __forceinline__ void decode_chunk(DecodeState<MW, GQ, NG> &st, const 
             st.acc[cb][3] = fmaf(st.acc[cb][3], h1, tmp[i][3]);
         }
     }
-    __syncwarp();
 }
 
 // n_chunks chunks dealt out evenly over n_splits splits: every split gets `q`, the first `r` of them one more.
@@ -1164,9 +1238,16 @@ __global__ void __launch_bounds__(kDecodeWarps * 32, decode_min_blocks(GQ, NG, M
             const int tq = PAIRED ? v / gqu : v / gq, hq = kvh * gq + (PAIRED ? (h / GQH) * gqu + v % gqu : v % gq);
             limit[h] = min(t_end, len - p.Tq + tq + 1);
             const uint32_t *qp = p.qwords + (((size_t)(layer * p.max_batch + b) * p.Tq + tq) * p.Hq + hq) * MWH;
+            if constexpr (SM::kQueryInSmem) {
+                uint32_t *qs = reinterpret_cast<uint32_t *>(ring + SM::kQueryOff);
+                if (lane < MW) qs[h * MW + lane] = __ldg(qp + lane);
+            } else {
 #pragma unroll
-            for (int w = 0; w < MWH; ++w) st.qw[h][w] = __ldg(qp + w);
+                for (int w = 0; w < MWH; ++w) st.qw[h][w] = __ldg(qp + w);
+            }
         }
+        st.qs = reinterpret_cast<const uint32_t *>(ring + SM::kQueryOff);
+        __syncwarp();
     }
 #pragma unroll
     for (int cb = 0; cb < 8; ++cb)
@@ -1183,24 +1264,47 @@ __global__ void __launch_bounds__(kDecodeWarps * 32, decode_min_blocks(GQ, NG, M
     int stage = 0;
     uint32_t parity = 0;
     bool failed = false;
-    for (int c = c0; c < c1; ++c) {
-        if (!mbar_wait_bounded(bar0 + 8 * stage, parity, kWaitLimitNs)) { failed = true; break; }
+    // PIPE: the distances of chunk c + 1 are computed inside the tensor-core phase of chunk c. The chunk after the
+    // split's last one does not exist: its "distances" are then taken from whatever the ring's next buffer holds
+    // (shared memory of this warp, nothing is waited for) and never used.
+    constexpr bool PIPE = decode_pipelined(GQ, NG, PAIRED);
+    int ham[GQ];
+    if (PIPE) {
+        if (mbar_wait_bounded(bar0, 0u, kWaitLimitNs)) chunk_scores<MW, GQ, NG, PAIRED>(st, ring, lane, ham);
+        else failed = true;
+    }
+    for (int c = c0; c < c1 && !failed; ++c) {
+        if (!PIPE) {
+            if (!mbar_wait_bounded(bar0 + 8 * stage, parity, kWaitLimitNs)) { failed = true; break; }
+        }
         const unsigned char *ch = ring + stage * CB;
+        if (!PIPE) chunk_scores<MW, GQ, NG, PAIRED>(st, ch, lane, ham);
+        float scl[GQ];
         if (c < c_full) {
-            decode_chunk<MW, GQ, NG, false, PAIRED>(st, ch, p_s, lane, limit, p.c2);
+            chunk_weights<MW, GQ, NG, false, PAIRED>(st, ham, ch, p_s, lane, limit, p.c2, scl);
         } else {
             int n_valid[GQ];
 #pragma unroll
             for (int h = 0; h < GQ; ++h) n_valid[h] = limit[h] - c * 32;
-            decode_chunk<MW, GQ, NG, true, PAIRED>(st, ch, p_s, lane, n_valid, p.c2);
+            chunk_weights<MW, GQ, NG, true, PAIRED>(st, ham, ch, p_s, lane, n_valid, p.c2, scl);
         }
-        // every lane is done with this stage (the chunk ends with a warp barrier): refill it
+        __syncwarp();
+        int next_stage = stage + 1;
+        uint32_t next_parity = parity;
+        if (next_stage == kStages) { next_stage = 0; next_parity ^= 1; }
+        if (PIPE && c + 1 < c1) {
+            if (!mbar_wait_bounded(bar0 + 8 * next_stage, next_parity, kWaitLimitNs)) { failed = true; break; }
+        }
+        chunk_values<MW, GQ, NG, PAIRED, PIPE>(st, ch, p_s, lane, scl, ring + next_stage * CB, ham);
+        __syncwarp();
+        // every lane is done with this stage: refill it
         if (lane == 0 && requested < c1) {
             mbar_arrive_expect_tx(bar0 + 8 * stage, CB);
             bulk_copy_g2s(ring_a + stage * CB, src, CB, bar0 + 8 * stage);
             H1B_NEXT_CHUNK();
         }
-        if (++stage == kStages) { stage = 0; parity ^= 1; }
+        stage = next_stage;
+        parity = next_parity;
     }
 #undef H1B_NEXT_CHUNK
 
