@@ -63,6 +63,8 @@ extern "C" {
 #define H1B_ERR_WORKSPACE   (-5)  /* workspace too small or misaligned                 */
 #define H1B_ERR_CUDA        (-6)  /* a CUDA runtime call failed (text in last_error)   */
 #define H1B_ERR_TIMEOUT     (-7)  /* a bounded device-side wait gave up (poll_status)  */
+#define H1B_ERR_BOUNDS      (-8)  /* bounds-checked build only: a kernel's index check
+                                     failed and its access was skipped (poll_status)   */
 
 typedef struct h1b_ctx h1b_ctx;   /* opaque, host-side */
 
@@ -359,6 +361,22 @@ int h1b_debug_scores(h1b_ctx *ctx, int layer, int seq, int kv_head, const void *
 int h1b_debug_partials(h1b_ctx *ctx, int layer, int seq, int q_token, int q_head,
                        int32_t *n_splits_host, float *hmin_host, float *wsum_host, int max_splits);
 
+/* Bounds-checked build (no counterpart in the paper; a debugging aid). When the
+ * library is compiled with -DH1B_DEBUG_BOUNDS, every address a kernel derives
+ * from its parameters for global memory (cache chunks, split-K partials, query
+ * sketches) and every carve of its shared memory is range-checked before use; a
+ * failing check records its number in the device status word and the access is
+ * skipped (nothing traps or faults), and h1b_poll_status() then returns
+ * H1B_ERR_BOUNDS once. The ordinary build contains none of this.
+ *   h1b_bounds_checked       1 if this library has the checks, else 0
+ *   h1b_debug_bounds_probe   launches a kernel whose one check fails on purpose
+ *                            and verifies that its guarded store was not made;
+ *                            the next h1b_poll_status() reports H1B_ERR_BOUNDS.
+ *                            H1B_ERR_UNSUPPORTED in the ordinary build.
+ *                            Synchronises `stream`. */
+int h1b_bounds_checked(void);
+int h1b_debug_bounds_probe(h1b_ctx *ctx, void *stream);
+
 /* Failure-path probe (no counterpart in the paper). Launches one warp that waits
  * for at most limit_ns nanoseconds (1 .. 1e9) on a barrier phase nothing will
  * complete, with the same bounded wait the attention and long-append kernels
@@ -374,8 +392,9 @@ int h1b_debug_wait_timeout(h1b_ctx *ctx, uint64_t limit_ns, void *stream);
 int h1b_set_splits(h1b_ctx *ctx, int splits);
 
 /* After the stream has been synchronised: 0, H1B_ERR_TIMEOUT if a kernel gave
- * up a bounded wait since the last poll, or H1B_ERR_CAPACITY if a replayed append
- * found a sequence full (the flag is cleared). */
+ * up a bounded wait since the last poll, H1B_ERR_CAPACITY if a replayed append
+ * found a sequence full, or (bounds-checked build) H1B_ERR_BOUNDS if a kernel's
+ * index check failed (the flag is cleared). */
 int h1b_poll_status(h1b_ctx *ctx);
 
 /* Time the dominant kernel. While enabled, every h1b_decode_attention() brackets

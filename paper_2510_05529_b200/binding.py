@@ -18,7 +18,7 @@ from .build import LIB_PATH, build_library, is_stale
 H1B_OK = 0
 ERRORS = {
     -1: "H1B_ERR_INVALID_ARG", -2: "H1B_ERR_NULL", -3: "H1B_ERR_UNSUPPORTED", -4: "H1B_ERR_CAPACITY",
-    -5: "H1B_ERR_WORKSPACE", -6: "H1B_ERR_CUDA", -7: "H1B_ERR_TIMEOUT",
+    -5: "H1B_ERR_WORKSPACE", -6: "H1B_ERR_CUDA", -7: "H1B_ERR_TIMEOUT", -8: "H1B_ERR_BOUNDS",
 }
 
 
@@ -89,6 +89,8 @@ def load_library(rebuild: bool = True) -> ctypes.CDLL:
         "h1b_debug_partials": (ctypes.c_int, [vp, ctypes.c_int, ctypes.c_int, ctypes.c_int, ctypes.c_int, i32p, vp, vp,
                                               ctypes.c_int]),
         "h1b_debug_wait_timeout": (ctypes.c_int, [vp, ctypes.c_uint64, vp]),
+        "h1b_bounds_checked": (ctypes.c_int, []),
+        "h1b_debug_bounds_probe": (ctypes.c_int, [vp, vp]),
         "h1b_set_splits": (ctypes.c_int, [vp, ctypes.c_int]),
         "h1b_poll_status": (ctypes.c_int, [vp]),
         "h1b_set_profiling": (ctypes.c_int, [vp, ctypes.c_int]),
@@ -114,6 +116,11 @@ def make_config(n_layers, n_q_heads, n_kv_heads, head_dim=128, sketch_bits=128, 
     flags = (H1B_FLAG_FP16_VALUES if fp16_values else 0) | (H1B_FLAG_ROPE if rope else 0)
     return h1b_config(n_layers, n_q_heads, n_kv_heads, head_dim, sketch_bits, group_size,
                       max_batch, max_seq, device, flags, page_tokens, n_pages)
+
+
+def h1b_bounds_checked() -> bool:
+    """Whether the loaded library carries the kernels' index checks (built with H1B_DEBUG_BOUNDS=1)."""
+    return bool(load_library().h1b_bounds_checked())
 
 
 def h1b_entry_bytes(cfg: h1b_config) -> int:
@@ -376,6 +383,10 @@ class H1BCache:
         self._check(self.lib.h1b_debug_partials(self._h, layer, seq, q_token, q_head, ctypes.byref(n), hmin.ctypes.data,
                                                 wsum.ctypes.data, max_splits))
         return hmin[:n.value].copy(), wsum[:n.value].copy()
+
+    def h1b_debug_bounds_probe(self, stream=None):
+        """Bounds-checked build only: a kernel's check fails on purpose; the next h1b_poll_status() reports it."""
+        self._check(self.lib.h1b_debug_bounds_probe(self._h, _stream_ptr(stream)))
 
     def h1b_debug_wait_timeout(self, limit_ns: int, stream=None):
         """Failure-path probe: one warp's bounded wait runs out and is recorded in the status word."""

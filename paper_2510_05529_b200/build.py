@@ -7,7 +7,10 @@ import subprocess
 
 _PKG = os.path.dirname(os.path.abspath(__file__))
 _CSRC = os.path.join(_PKG, "csrc")
-LIB_PATH = os.path.join(_PKG, "libh1b.so")
+# H1B_DEBUG_BOUNDS=1 in the environment selects the bounds-checked build (the kernels' index checks compiled in): a
+# library of its own beside the ordinary one, so that both can be built ahead of time.
+DEBUG_BOUNDS = os.environ.get("H1B_DEBUG_BOUNDS", "0") not in ("", "0")
+LIB_PATH = os.path.join(_PKG, "libh1b_bounds.so" if DEBUG_BOUNDS else "libh1b.so")
 SOURCES = ["h1b_api.cu", "h1b_kernels.cu"]
 NVCC_FLAGS = ["-gencode", "arch=compute_100a,code=sm_100a", "-lineinfo", "-O3", "-std=c++17",
               "--use_fast_math=false", "-Xcompiler", "-fPIC", "-shared"]
@@ -40,7 +43,7 @@ def build_library(force: bool = False, verbose: bool = False) -> str:
     if not force and not is_stale():
         return LIB_PATH
     tmp = LIB_PATH + ".tmp.%d" % os.getpid()
-    flags = [f for f in NVCC_FLAGS if f != "--use_fast_math=false"]
+    flags = [f for f in NVCC_FLAGS if f != "--use_fast_math=false"] + (["-DH1B_DEBUG_BOUNDS"] if DEBUG_BOUNDS else [])
     cmd = [_nvcc()] + flags + (["-Xptxas", "-v"] if verbose else []) + \
           [os.path.join(_CSRC, s) for s in SOURCES] + ["-o", tmp]
     res = subprocess.run(cmd, capture_output=True, text=True)

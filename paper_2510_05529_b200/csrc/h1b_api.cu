@@ -29,6 +29,7 @@ constexpr int kPrefillMinTokens = 64;   // appends of at least this many tokens 
 struct Plan {
     size_t rt, rh, len, status, qwords, partial, stage_k, stage_v, stage_q, stage_out, dbg_q, dbg_row, dbg_s, cache, total;
     size_t partial_bytes, slab_bytes;
+    size_t qwords_words, cache_bytes;       // words of the query-sketch scratch, bytes of the cache region
     size_t rope;                            // rotary table [cap_tokens][head_dim / 2][2] fp32 (H1B_FLAG_ROPE only)
     size_t table, seq_cap, layer_bytes;     // paged cache: block tables [max_batch][table_stride], capacities [max_batch]
     int table_stride, page_chunks;          // 0 when the cache is contiguous
@@ -127,7 +128,8 @@ int make_plan(const h1b_config *user, Plan *p) {
     p->rh = take(L * 2 * d * c->sketch_bits * sizeof(uint16_t));     // fp16 pieces of Rt for the tensor-core prefill
     p->len = take(L * B * sizeof(int32_t));
     p->status = take(64);
-    p->qwords = take(L * B * Hq * kMaxQueryTokens * p->m_words * sizeof(uint32_t));
+    p->qwords_words = L * B * Hq * kMaxQueryTokens * p->m_words;
+    p->qwords = take(p->qwords_words * sizeof(uint32_t));
     p->partial = take(p->partial_bytes);
     p->stage_k = take(L * B * Hkv * d * 2);
     p->stage_v = take(L * B * Hkv * d * 2);
@@ -139,7 +141,8 @@ int make_plan(const h1b_config *user, Plan *p) {
     p->table = take((size_t)c->max_batch * (p->table_stride ? p->table_stride : 1) * sizeof(int32_t));
     p->seq_cap = take((size_t)c->max_batch * sizeof(int32_t));
     p->rope = take((c->flags & H1B_FLAG_ROPE) ? (size_t)p->cap_tokens * (user->head_dim / 2) * 2 * sizeof(float) : 0);
-    p->cache = take(c->page_tokens > 0 ? L * p->layer_bytes : slabs * p->slab_bytes);
+    p->cache_bytes = c->page_tokens > 0 ? L * p->layer_bytes : slabs * p->slab_bytes;
+    p->cache = take(p->cache_bytes);
     p->total = o;
     return H1B_OK;
 }
@@ -220,6 +223,7 @@ CacheAddr cache_addr(h1b_ctx *ctx) {
     a.layer_bytes = ctx->plan.layer_bytes;
     a.table_stride = ctx->plan.table_stride; a.page_chunks = ctx->plan.page_chunks;
     a.Hkv = ctx->cfg.n_kv_heads; a.max_batch = ctx->cfg.max_batch; a.chunk_bytes = ctx->cl.bytes;
+    a.cache_bytes = ctx->plan.cache_bytes;
     return a;
 }
 
@@ -426,8 +430,10 @@ static AppendParams append_params(h1b_ctx *ctx, int layer_begin, int n_layers, c
 }
 
 static SketchParams sketch_params(h1b_ctx *ctx, int layer_begin, int n_layers, const void *q, int B,
-                                  uint32_t *qwords) {
+                                  uint32_t *qwords, size_t qwords_words = 0 /* 0: the workspace's sketch scratch */) {
     SketchParams sp;
+    sp.qwords_words = qwords_words ? qwords_words : ctx->plan.qwords_words;
+    sp.status = at<int32_t>(ctx, ctx->plan.status);
     sp.q = static_cast<const uint16_t *>(q);
     sp.Rt = at<float>(ctx, ctx->plan.rt);
     sp.qwords = qwords;
@@ -453,6 +459,8 @@ struct DecodePlan {
     int gqk, vgroups;       // heads per work item, items per (slab, split)
     int pass_layers;        // layers per pass through the scratch (all of them unless the scratch is small)
     int splits;             // work items per (slab, group of heads)
+    size_t partial_bytes;   // what the scratch holds: partials, and words of query sketches
+    size_t qwords_words;
 };
 
 // Every sequence is split so that there are about kTargetItems work items, capped by what the scratch holds. The
@@ -463,6 +471,8 @@ struct DecodePlan {
 static int plan_decode(h1b_ctx *ctx, int layer_begin, int n_layers, int B, size_t partial_bytes, int Tq, int q_tail,
                        int extra_tokens, DecodePlan *dpl) {
     heads_per_item(ctx->plan.gq, Tq, ctx->paired, &dpl->gqk, &dpl->vgroups);
+    dpl->partial_bytes = partial_bytes;
+    dpl->qwords_words = ctx->plan.qwords_words;
     const size_t max_items = partial_bytes / ((size_t)dpl->gqk * kPartStride * sizeof(float));
     // slabs x groups of virtual heads: the units a split divides. When the scratch cannot hold one partial for
     // every unit of the call (many query tokens on a large batch), the layers go through it in several passes,
@@ -500,6 +510,8 @@ static int enqueue_decode(h1b_ctx *ctx, const DecodePlan &dpl, int layer_begin, 
     dp.len = at<int32_t>(ctx, ctx->plan.len);
     dp.qwords = qwords;
     dp.partial = partial;
+    dp.partial_floats = dpl.partial_bytes / sizeof(float);
+    dp.qwords_words = dpl.qwords_words;
     dp.status = at<int32_t>(ctx, ctx->plan.status);
     dp.B = B; dp.Hkv = ctx->cfg.n_kv_heads;
     dp.Hq = ctx->cfg.n_q_heads; dp.max_batch = ctx->cfg.max_batch; dp.m_words = ctx->plan.m_words;
@@ -790,9 +802,11 @@ int h1b_decode_attention_static(h1b_ctx *ctx, int layer_begin, int n_layers, con
     DecodePlan dpl;
     rc = plan_decode(ctx, layer_begin, n_layers, B, H1B_STATIC_SCRATCH_BYTES - qw_bytes, 1, 0, 0, &dpl);
     if (rc != H1B_OK) return rc;
+    dpl.qwords_words = qw_bytes / sizeof(uint32_t);
     cudaStream_t st = static_cast<cudaStream_t>(stream);
     int launches = 0;
-    const SketchParams sp = sketch_params(ctx, layer_begin, n_layers, q, B, reinterpret_cast<uint32_t *>(scratch));
+    const SketchParams sp = sketch_params(ctx, layer_begin, n_layers, q, B, reinterpret_cast<uint32_t *>(scratch),
+                                          qw_bytes / sizeof(uint32_t));
     NewCounts none;
     std::memset(&none, 0, sizeof none);
     H1B_CUDA(ctx, launch_prepare(nullptr, &sp, none, st, &launches));
@@ -999,6 +1013,8 @@ int h1b_debug_scores(h1b_ctx *ctx, int layer, int seq, int kv_head, const void *
     sp.q = static_cast<const uint16_t *>(q);
     sp.Rt = at<float>(ctx, ctx->plan.rt) + (size_t)layer * ctx->cfg.head_dim * ctx->cfg.sketch_bits;
     sp.qwords = at<uint32_t>(ctx, ctx->plan.dbg_q);
+    sp.qwords_words = (size_t)mw;
+    sp.status = at<int32_t>(ctx, ctx->plan.status);
     sp.layer_begin = 0; sp.n_layers = 1; sp.B = 1; sp.Hq = 1; sp.max_batch = 1; sp.m_words = mw;
     // with rotary embedding the row is turned like the query of a decode call: at the sequence's last position
     sp.rope = rope_ref(ctx);
@@ -1097,7 +1113,29 @@ int h1b_poll_status(h1b_ctx *ctx) {
     H1B_CUDA(ctx, cudaMemset(at<int32_t>(ctx, ctx->plan.status), 0, sizeof s));
     if (s == kStatusCapacity)
         return fail(ctx, H1B_ERR_CAPACITY, "a replayed append found a sequence full: its rows were dropped");
+    if (s >= kStatusBounds)
+        return fail(ctx, H1B_ERR_BOUNDS, "bounds-checked build: index check %d of a kernel failed; the access was skipped",
+                    s - kStatusBounds);
     return fail(ctx, H1B_ERR_TIMEOUT, "a kernel gave up a bounded wait (status %d)", s);
+}
+
+int h1b_bounds_checked(void) { return bounds_checked_build() ? 1 : 0; }
+
+int h1b_debug_bounds_probe(h1b_ctx *ctx, void *stream) {
+    if (!ctx) return H1B_ERR_NULL;
+    if (!bounds_checked_build())
+        return fail(ctx, H1B_ERR_UNSUPPORTED, "this library was built without the kernels' index checks (H1B_DEBUG_BOUNDS)");
+    // the word the probe would write if its check did not stop it: the debug query slot, cleared first
+    int32_t *target = at<int32_t>(ctx, ctx->plan.dbg_q);
+    cudaStream_t st = static_cast<cudaStream_t>(stream);
+    H1B_CUDA(ctx, cudaMemsetAsync(target, 0, sizeof(int32_t), st));
+    H1B_CUDA(ctx, launch_debug_bounds_probe(at<int32_t>(ctx, ctx->plan.status), target, st));
+    ++ctx->launches;
+    int32_t wrote = 0;
+    H1B_CUDA(ctx, cudaMemcpyAsync(&wrote, target, sizeof wrote, cudaMemcpyDeviceToHost, st));
+    H1B_CUDA(ctx, cudaStreamSynchronize(st));
+    if (wrote != 0) return fail(ctx, H1B_ERR_INVALID_ARG, "the guarded store of the probe was made: the checks are not in effect");
+    return H1B_OK;
 }
 
 int h1b_debug_wait_timeout(h1b_ctx *ctx, uint64_t limit_ns, void *stream) {

@@ -32,6 +32,29 @@ namespace h1b {
 // so the fp32 result is within 128 * 2^-24 of the exact projection relative to
 // the sum of absolute terms, and every launch shape gives the same bits.
 // ===========================================================================
+// Bounds-checked build (-DH1B_DEBUG_BOUNDS; compute-sanitizer's stand-in for the small test cases): every address a
+// kernel derives from its parameters for a global-memory access (cache chunks, split-K partials, query sketches) and
+// every carve of its shared memory is range-checked first. A check that fails records kStatusBounds + its number
+// in the status word (the first failure stays) and the access is NOT made: nothing traps or faults; the host reads
+// it with h1b_poll_status(). In the ordinary build the checks are the constant `true` and cost nothing.
+enum BoundsSite { kSiteKeyWord = 1, kSiteValueRow = 2, kSiteQueryStore = 3, kSitePrefillValues = 4, kSitePrefillKeys = 5,
+                  kSiteChunkCopy = 6, kSiteRing = 7, kSitePartialStore = 8, kSiteQueryLoad = 9, kSitePartialLoad = 10,
+                  kSitePrefillSmem = 11, kSiteProbe = 12 };
+#ifdef H1B_DEBUG_BOUNDS
+__device__ __forceinline__ bool bounds_ok(bool ok, int32_t *status, int site) {
+    if (!ok) atomicCAS(status, kStatusOk, kStatusBounds + site);
+    return ok;
+}
+#define H1B_IN_BOUNDS(cond, status, site) bounds_ok((cond), (status), (site))
+#else
+#define H1B_IN_BOUNDS(cond, status, site) true
+#endif
+// [ptr, ptr + bytes) lies inside the cache region
+__device__ __forceinline__ bool in_cache(const CacheAddr &ca, const void *ptr, size_t bytes) {
+    const unsigned char *q = static_cast<const unsigned char *>(ptr);
+    return q >= ca.base && q + bytes <= ca.base + ca.cache_bytes;
+}
+
 constexpr unsigned long long kWaitLimitNs = 2000000000ull;   // bounded device-side waits: 2 s, then give up
 constexpr int kProjThreads = 128;
 constexpr int kProjRows = 32;
@@ -228,7 +251,8 @@ __global__ void __launch_bounds__(kProjThreads) prepare_kernel(AppendParams ap, 
             if (tn < nn.v[b] && len0 + nn.v[b] <= ap.seq_cap[b]) {
                 const int t = len0 + tn;
                 unsigned char *chunk = chunk_ptr(ap.ca, layer, b, kvh, t >> 5);
-                *reinterpret_cast<uint32_t *>(chunk + key_word_off(word, t & 31)) = bits;
+                if (H1B_IN_BOUNDS(in_cache(ap.ca, chunk, cl.bytes), ap.status, kSiteKeyWord))
+                    *reinterpret_cast<uint32_t *>(chunk + key_word_off(word, t & 31)) = bits;
             }
         }
     } else if (blk < k_blocks + q_blocks) {
@@ -251,7 +275,8 @@ __global__ void __launch_bounds__(kProjThreads) prepare_kernel(AppendParams ap, 
         if ((int)threadIdx.x < n_rows) {
             const int row = row0 + threadIdx.x;
             const int h = row % sp.Hq, b = row / sp.Hq;
-            sp.qwords[((size_t)(layer * sp.max_batch + b) * sp.Hq + h) * mw + word] = bits;
+            const size_t at = ((size_t)(layer * sp.max_batch + b) * sp.Hq + h) * mw + word;
+            if (H1B_IN_BOUNDS(at < sp.qwords_words, sp.status, kSiteQueryStore)) sp.qwords[at] = bits;
         }
     } else {
         const long row = (long)(blk - k_blocks - q_blocks) * (kProjThreads / 32) + (threadIdx.x >> 5);
@@ -264,7 +289,8 @@ __global__ void __launch_bounds__(kProjThreads) prepare_kernel(AppendParams ap, 
             if (tn < nn.v[b] && len0 + nn.v[b] <= ap.seq_cap[b]) {
                 const int t = len0 + tn;
                 unsigned char *chunk = chunk_ptr(ap.ca, layer, b, kvh, t >> 5);
-                store_value_row(ap.v + row * kHeadDim, chunk, cl, t & 31, threadIdx.x & 31);
+                if (H1B_IN_BOUNDS(in_cache(ap.ca, chunk, cl.bytes), ap.status, kSiteValueRow))
+                    store_value_row(ap.v + row * kHeadDim, chunk, cl, t & 31, threadIdx.x & 31);
             }
         }
     }
@@ -347,6 +373,7 @@ __device__ __forceinline__ void store_value_block16(const PrefillParams &p, cons
                                                     unsigned char *vs, int lane) {
     const int tn0 = pos0 - len0;
     unsigned char *chunk = chunk_ptr(p.ca, layer, b, kvh, pos0 >> 5);
+    if (!H1B_IN_BOUNDS(in_cache(p.ca, chunk, cl.bytes), p.status, kSitePrefillValues)) return;
     const int vb = (pos0 >> 4) & 1;
     if (p.groups == 0 && tn0 >= 0 && tn0 + 16 <= n_new) {
         // fp16 values, a whole block of 16 tokens: transposed through shared memory into the A-operand
@@ -544,6 +571,7 @@ __device__ __forceinline__ void prefill_body(const PrefillParams &p, const NewCo
     extern __shared__ unsigned char smem_unaligned[];
     unsigned char *smem = smem_unaligned + ((1024u - (smem_addr(smem_unaligned) & 1023u)) & 1023u);
     unsigned char *Rs = smem, *As0 = smem + SM::kRBytes;        // key tile number t sits in buffer t % kKeyStages at As0 + that * kABytes
+    (void)H1B_IN_BOUNDS(As0 + kKeyStages * SM::kABytes <= smem_unaligned + SM::kTotal, p.status, kSitePrefillSmem);
     __shared__ uint32_t tmem_base_s;
     __shared__ __align__(8) unsigned long long mma_bar_s[2];
     __shared__ int is_last, gave_up;
@@ -755,7 +783,7 @@ __device__ __forceinline__ void prefill_body(const PrefillParams &p, const NewCo
                         for (int k = 0; k < 4; ++k)
                             part[k] = __funnelshift_l(__float_as_uint(__uint_as_float(y[8 * k + j]) + 0.f), part[k], 1);
                     const uint32_t neg = part[0] | (part[1] << 8) | (part[2] << 16) | (part[3] << 24);
-                    if (tn >= 0 && tn < n_new)
+                    if (tn >= 0 && tn < n_new && H1B_IN_BOUNDS(in_cache(p.ca, chunk, cl.bytes), p.status, kSitePrefillKeys))
                         *reinterpret_cast<uint32_t *>(chunk + lane * 4 + (col0 / 32 + w) * 128) = ~neg;
                 }
             } else if (lane == 0) {
@@ -1165,7 +1193,7 @@ __global__ void __launch_bounds__(kDecodeWarps * 32, decode_min_blocks(GQ, NG, M
     if (c0 >= c1) {
         // an item with no chunk says so in its partial (distance = the sentinel, weight sum 0): the combine kernel then
         // needs neither the length nor the split arithmetic to know which partials to skip
-        if (lane < GQ) {
+        if (lane < GQ && H1B_IN_BOUNDS(((size_t)item * GQ + GQ) * kPartStride <= p.partial_floats, p.status, kSitePartialStore)) {
             float *po = p.partial + ((size_t)item * GQ + lane) * kPartStride;
             po[128] = (float)kHamSentinel;
             po[129] = 0.f;
@@ -1180,6 +1208,7 @@ __global__ void __launch_bounds__(kDecodeWarps * 32, decode_min_blocks(GQ, NG, M
     float *p_s = reinterpret_cast<float *>(ring + kStages * CB);
     const uint32_t bar0 = smem_addr(ring + kStages * CB + GQ * 128);
     const uint32_t ring_a = smem_addr(ring);
+    (void)H1B_IN_BOUNDS((warp + 1) * SM::kPerWarp <= SM::kTotal && warp < kDecodeWarps, p.status, kSiteRing);
     if (lane == 0) {
 #pragma unroll
         for (int s = 0; s < kStages; ++s) mbar_init(bar0 + 8 * s, 1);
@@ -1213,10 +1242,13 @@ __global__ void __launch_bounds__(kDecodeWarps * 32, decode_min_blocks(GQ, NG, M
                           ? p.ca.table[(size_t)b * p.ca.table_stride + page_idx + 1] : 0;                       \
         }                                                                                                       \
     } while (0)
+    // (bounds-checked build: a source outside the cache is recorded and replaced by the cache's first chunk, so that the
+    // copy the warp waits for still happens, from memory that is the library's own)
+#define H1B_CHUNK_SOURCE() (H1B_IN_BOUNDS(in_cache(p.ca, src, CB), p.status, kSiteChunkCopy) ? src : p.ca.base)
     if (lane == 0) {
         for (int s = 0; s < kStages && requested < c1; ++s) {
             mbar_arrive_expect_tx(bar0 + 8 * s, CB);
-            bulk_copy_g2s(ring_a + s * CB, src, CB, bar0 + 8 * s);
+            bulk_copy_g2s(ring_a + s * CB, H1B_CHUNK_SOURCE(), CB, bar0 + 8 * s);
             H1B_NEXT_CHUNK();
         }
     }
@@ -1237,7 +1269,8 @@ __global__ void __launch_bounds__(kDecodeWarps * 32, decode_min_blocks(GQ, NG, M
             const int v = PAIRED ? min(vg * GQH + h % GQH, gqu * p.Tq - 1) : min(vg * GQ + h, vheads - 1);
             const int tq = PAIRED ? v / gqu : v / gq, hq = kvh * gq + (PAIRED ? (h / GQH) * gqu + v % gqu : v % gq);
             limit[h] = min(t_end, len - p.Tq + tq + 1);
-            const uint32_t *qp = p.qwords + (((size_t)(layer * p.max_batch + b) * p.Tq + tq) * p.Hq + hq) * MWH;
+            const size_t q_at = (((size_t)(layer * p.max_batch + b) * p.Tq + tq) * p.Hq + hq) * MWH;
+            const uint32_t *qp = p.qwords + (H1B_IN_BOUNDS(q_at + MWH <= p.qwords_words, p.status, kSiteQueryLoad) ? q_at : 0);
             if constexpr (SM::kQueryInSmem) {
                 uint32_t *qs = reinterpret_cast<uint32_t *>(ring + SM::kQueryOff);
                 if (lane < MW) qs[h * MW + lane] = __ldg(qp + lane);
@@ -1300,13 +1333,14 @@ __global__ void __launch_bounds__(kDecodeWarps * 32, decode_min_blocks(GQ, NG, M
         // every lane is done with this stage: refill it
         if (lane == 0 && requested < c1) {
             mbar_arrive_expect_tx(bar0 + 8 * stage, CB);
-            bulk_copy_g2s(ring_a + stage * CB, src, CB, bar0 + 8 * stage);
+            bulk_copy_g2s(ring_a + stage * CB, H1B_CHUNK_SOURCE(), CB, bar0 + 8 * stage);
             H1B_NEXT_CHUNK();
         }
         stage = next_stage;
         parity = next_parity;
     }
 #undef H1B_NEXT_CHUNK
+#undef H1B_CHUNK_SOURCE
 
     if (failed) {
         if (lane == 0) atomicExch(p.status, kStatusWaitTimeout);
@@ -1333,6 +1367,7 @@ __global__ void __launch_bounds__(kDecodeWarps * 32, decode_min_blocks(GQ, NG, M
     // the common factor 2 cancels in the final division.
     // (fp16 values: A held the values themselves, so only the low parts' 2^11 is undone and there is no zero-point term.)
     constexpr float kRowLo = NG ? kCodeScaleLo : 1.f, kRowHi = NG ? kCodeScaleHi : 1.f, kLoPart = 1.f / 2048.f;
+    if (!H1B_IN_BOUNDS(((size_t)item * GQ + GQ) * kPartStride <= p.partial_floats, p.status, kSitePartialStore)) return;
     float *part_out = p.partial + (size_t)item * GQ * kPartStride;
     const int r = lane >> 2, jq = lane & 3;
 #pragma unroll
@@ -1445,9 +1480,13 @@ __global__ void __launch_bounds__(kHeadDim) combine_kernel(DecodeParams p) {
     const int vp = tq * gqu + jj % gqu;                         // paired: (query token, head in group) on its own KV head
     const int vg = p.paired ? vp / gqh : v / p.gqk, hh = p.paired ? (jj / gqu) * gqh + vp % gqh : v % p.gqk;
     const long slab_local = ((long)ll * p.B + b) * p.Hkv + kvh;
-    const int ns = p.splits;
-    const float *base = p.partial + (((size_t)slab_local * p.vgroups + vg) * p.splits * p.gqk + hh) * kPartStride;
+    const size_t base_at = (((size_t)slab_local * p.vgroups + vg) * p.splits * p.gqk + hh) * kPartStride;
     const size_t stride = (size_t)p.gqk * kPartStride;
+    // (block-uniform: a block whose partials would lie outside the scratch reads nothing and writes zeros)
+    const bool in_scratch = H1B_IN_BOUNDS(p.splits < 1 || base_at + (size_t)(p.splits - 1) * stride + kPartStride <= p.partial_floats,
+                                          p.status, kSitePartialLoad);
+    const float *base = p.partial + (in_scratch ? base_at : 0);
+    const int ns = in_scratch ? p.splits : 0;
     constexpr float kEmpty = (float)kHamSentinel;               // what a split without tokens (for this head) reports
     // This warp's first two splits are fetched before the block agrees on the largest logit: the loads do not depend
     // on it, so the kernel makes one trip to memory, not two.
@@ -1529,6 +1568,13 @@ __global__ void debug_wait_timeout_kernel(int32_t *status, unsigned long long li
     __syncwarp();
     const bool done = mbar_wait_bounded(bar, 0u, limit_ns);
     if (!done && threadIdx.x == 0) atomicExch(status, kStatusWaitTimeout);
+}
+
+// Test helper of the bounds-checked build: one thread runs a check that must fail (index n against limit n) and
+// skips the access it guards, exactly as a real site would. In the ordinary build the check is the constant true,
+// the guarded store happens (into the word the caller handed over), and the launcher below refuses to be called.
+__global__ void debug_bounds_probe_kernel(int32_t *status, int32_t *target, int n) {
+    if (threadIdx.x == 0 && H1B_IN_BOUNDS(n < n, status, kSiteProbe)) target[0] = 1;
 }
 
 // ===========================================================================
@@ -1734,10 +1780,13 @@ static cudaError_t dispatch_decode(const DecodeParams &p, cudaStream_t st, bool 
     cudaError_t e = cudaErrorInvalidValue;
     H1B_DISPATCH_MW(p.m_words,
         if (p.paired) {                                         // two 64-wide heads per slab
-            if (gq == 2 && p.groups == 4) e = launch_decode_t<MW, 2, 4, true>(p, st, ao);
-            else if (gq == 2 && p.groups == 0) e = launch_decode_t<MW, 2, 0, true>(p, st, ao);
-            else if (gq == 8 && p.groups == 4) e = launch_decode_t<MW, 8, 4, true>(p, st, ao);
-            else if (gq == 8 && p.groups == 0) e = launch_decode_t<MW, 8, 0, true>(p, st, ao);
+            // (both heads' sketches of at least 64 bits each: four words or more; the two-word variants do not exist)
+            if constexpr (MW >= 4) {
+                if (gq == 2 && p.groups == 4) e = launch_decode_t<MW, 2, 4, true>(p, st, ao);
+                else if (gq == 2 && p.groups == 0) e = launch_decode_t<MW, 2, 0, true>(p, st, ao);
+                else if (gq == 8 && p.groups == 4) e = launch_decode_t<MW, 8, 4, true>(p, st, ao);
+                else if (gq == 8 && p.groups == 0) e = launch_decode_t<MW, 8, 0, true>(p, st, ao);
+            }
         } else if (p.groups == 4) {
             if (gq == 1) e = launch_decode_t<MW, 1, 4>(p, st, ao);
             else if (gq == 2) e = launch_decode_t<MW, 2, 4>(p, st, ao);
@@ -1798,6 +1847,19 @@ cudaError_t launch_decode(const DecodeParams &p, cudaStream_t st, int *launches,
         if (ec != cudaSuccess) return ec;
     }
     ++*launches;
+    return cudaGetLastError();
+}
+
+bool bounds_checked_build() {
+#ifdef H1B_DEBUG_BOUNDS
+    return true;
+#else
+    return false;
+#endif
+}
+
+cudaError_t launch_debug_bounds_probe(int32_t *status, int32_t *target, cudaStream_t st) {
+    debug_bounds_probe_kernel<<<1, 32, 0, st>>>(status, target, 7);
     return cudaGetLastError();
 }
 

@@ -21,6 +21,10 @@ cudaError_t launch_decode(const DecodeParams &p, cudaStream_t st, int *launches,
 // Sets, on the current device, the launch attributes of every kernel a cache of this shape can reach (thread-safe,
 // once per device and kernel): afterwards a launcher only launches.
 cudaError_t warm_kernel_attributes(int m_words, int groups, bool paired, bool paged, bool rope);
+// Whether the library was compiled with the kernels' index checks (-DH1B_DEBUG_BOUNDS), and a kernel whose one
+// check fails on purpose (records its site in *status and skips its store to *target).
+bool bounds_checked_build();
+cudaError_t launch_debug_bounds_probe(int32_t *status, int32_t *target, cudaStream_t st);
 // One warp waits for at most limit_ns on a barrier phase that never completes, then records the time-out in *status.
 cudaError_t launch_debug_wait_timeout(int32_t *status, unsigned long long limit_ns, cudaStream_t st);
 cudaError_t launch_set_len(int32_t *len, int n_layers, int max_batch, int seq, int value, cudaStream_t st);

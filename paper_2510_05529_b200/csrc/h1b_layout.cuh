@@ -102,6 +102,7 @@ struct CacheAddr {
     size_t slab_bytes;          // contiguous: bytes of one slab
     size_t layer_bytes;         // paged: bytes of one layer's pool
     int table_stride, page_chunks, Hkv, max_batch, chunk_bytes;
+    size_t cache_bytes;         // bytes of the whole cache region behind `base` (read by the bounds-checked build only)
 };
 __host__ __device__ inline size_t chunk_offset(const CacheAddr &a, const int32_t *table, int layer, int b, int kvh, int c) {
     if (!table) return ((size_t)(layer * a.max_batch + b) * a.Hkv + kvh) * a.slab_bytes + (size_t)c * a.chunk_bytes;
@@ -115,6 +116,7 @@ __device__ inline unsigned char *chunk_ptr(const CacheAddr &a, int layer, int b,
 // Device status word values.
 constexpr int kStatusOk = 0;
 constexpr int kStatusWaitTimeout = 1;
+constexpr int kStatusBounds = 16;       // bounds-checked build only: 16 + the number of the check that failed (its access was skipped)
 constexpr int kStatusCapacity = 2;      // an append found a sequence full (only reachable when a captured graph is replayed
                                         // more often than the cache has room for: direct calls are checked on the host)
 
@@ -164,6 +166,8 @@ struct SketchParams {           // query sketch
     const uint16_t *q;          // fp16 [n_layers][B][Hq][d]
     const float *Rt;
     uint32_t *qwords;           // [L][max_batch][Hq][m/32]
+    size_t qwords_words;        // words behind `qwords` (bounds-checked build)
+    int32_t *status;            // device status word
     int layer_begin, n_layers, B, Hq, max_batch, m_words;
     // rotation of the queries: row (b, h) belongs to query token h / (Hq / Tq) of Tq, whose position is
     // len + n_new - Tq + that index (len as the launch finds it, n_new what the same launch appends)
@@ -181,6 +185,8 @@ struct DecodeParams {
     const int32_t *len;         // [L][max_batch]
     const uint32_t *qwords;     // [L][max_batch][Tq][Hq][m/32]
     float *partial;             // [items][gqk][kPartStride]
+    size_t partial_floats;      // floats behind `partial`, words behind `qwords` (bounds-checked build)
+    size_t qwords_words;
     float *out;                 // fp32 [n_layers][B][Tq][Hq][d]
     int32_t *status;
     int layer_begin, n_layers, B, Hkv, Hq, max_batch, m_words, groups;
