@@ -577,7 +577,6 @@ int h1b_append_kv(h1b_ctx *ctx, int layer_begin, int n_layers, const void *k, co
         pp.rope = rope_ref(ctx);
         pp.len = at<int32_t>(ctx, ctx->plan.len);
         pp.status = at<int32_t>(ctx, ctx->plan.status);
-        pp.done = at<int32_t>(ctx, ctx->plan.status) + 4;
         pp.layer_begin = layer_begin; pp.n_layers = n_layers; pp.B = B; pp.Tn = Tn;
         pp.Hkv = ctx->cfg.n_kv_heads; pp.max_batch = ctx->cfg.max_batch; pp.m_words = ctx->plan.m_words;
         pp.groups = ctx->plan.groups;

@@ -15,7 +15,10 @@
 //   prefill_rope_kernel  accumulators in TMEM), the second one rotating each key tile in shared
 //                        memory first (rotary position embedding);
 //   prefill_values_kernel  Eq. 4 for the same appends, side by side with the key kernel.
+#include <algorithm>
 #include <mutex>
+
+#include <cuda.h>
 
 #include "h1b_kernels.h"
 #include "h1b_ptx.cuh"
@@ -461,22 +464,29 @@ __device__ __forceinline__ void store_value_block16(const PrefillParams &p, cons
             // q[i]: the bits of code + 1.5 * 2^23, i.e. the code in the low four bits and zeros up to bit 21.
             // t >= 0, and with a normal fp16 scale t / scale <= 15 / (1 - 2^-11) < 15.5: nothing to clamp. Only a
             // subnormal scale (a range below 15 * 2^-14) can overshoot.
+            // The five operations per value run two values at a time on the packed fp32 instructions of this
+            // architecture: the same IEEE operations in the same order, so the same bits.
             uint32_t q[32];
+            const float2 nmn2 = make_float2(-mn, -mn), inv2 = make_float2(inv, inv), ndelta2 = make_float2(-delta, -delta);
+            const float2 magic2 = make_float2(12582912.f, 12582912.f);
             if (delta >= 6.103515625e-05f || delta == 0.f) {
 #pragma unroll
-                for (int i = 0; i < 32; ++i) {
-                    const float t = __fsub_rn(x[i], mn);
-                    const float q0 = __fmul_rn(t, inv);
-                    const float q1 = __fmaf_rn(__fmaf_rn(-q0, delta, t), inv, q0);  // = RN(t / delta)
-                    q[i] = __float_as_uint(q1 + 12582912.f);                        // round half to even
+                for (int i = 0; i < 32; i += 2) {
+                    const float2 t = __fadd2_rn(make_float2(x[i], x[i + 1]), nmn2);                  // x - mn
+                    const float2 q0 = __fmul2_rn(t, inv2);
+                    const float2 q1 = __ffma2_rn(__ffma2_rn(q0, ndelta2, t), inv2, q0);               // = RN(t / delta)
+                    const float2 r = __fadd2_rn(q1, magic2);                                         // round half to even
+                    q[i] = __float_as_uint(r.x);
+                    q[i + 1] = __float_as_uint(r.y);
                 }
             } else {
 #pragma unroll
-                for (int i = 0; i < 32; ++i) {
-                    const float t = __fsub_rn(x[i], mn);
-                    const float q0 = __fmul_rn(t, inv);
-                    const float q1 = __fmaf_rn(__fmaf_rn(-q0, delta, t), inv, q0);
-                    q[i] = __float_as_uint(fminf(q1, 15.f) + 12582912.f);
+                for (int i = 0; i < 32; i += 2) {
+                    const float2 t = __fadd2_rn(make_float2(x[i], x[i + 1]), nmn2);
+                    const float2 q0 = __fmul2_rn(t, inv2);
+                    const float2 q1 = __ffma2_rn(__ffma2_rn(q0, ndelta2, t), inv2, q0);
+                    q[i] = __float_as_uint(fminf(q1.x, 15.f) + 12582912.f);
+                    q[i + 1] = __float_as_uint(fminf(q1.y, 15.f) + 12582912.f);
                 }
             }
             // token k = it*8 + rsub of the block; in-block byte of (channel block cb, row r): see code_byte_off
@@ -516,53 +526,41 @@ __device__ __forceinline__ void store_value_block16(const PrefillParams &p, cons
     }
 }
 
-// End of both long-append kernels: the block that finishes last of all (key and value kernel together) adds the new
-// tokens to the lengths. Every block of both kernels has read the lengths by then.
-__device__ __forceinline__ void prefill_publish_lengths(const PrefillParams &p, const NewCounts &nn, int *is_last_s) {
-    __syncthreads();
-    if (threadIdx.x == 0) {
-        __threadfence();
-        *is_last_s = (atomicAdd(p.done, 1) == p.total_blocks - 1);
-    }
-    __syncthreads();
-    if (*is_last_s) {
-        for (int i = threadIdx.x; i < p.n_layers * p.B; i += blockDim.x) {
-            int32_t *len = p.len + (p.layer_begin + i / p.B) * p.max_batch + (i % p.B);
-            const int n = nn.v[i % p.B];
-            if (*len + n <= p.seq_cap[i % p.B]) *len += n;
-            else atomicExch(p.status, kStatusCapacity);         // full: nothing of this sequence's rows was written
-        }
-        if (threadIdx.x == 0) *p.done = 0;
+// Behind both long-append kernels (stream order): the new tokens are added to the lengths. One small block.
+__global__ void prefill_publish_kernel(PrefillParams p, NewCounts nn) {
+    grid_dependency_wait();
+    for (int i = threadIdx.x; i < p.n_layers * p.B; i += blockDim.x) {
+        int32_t *len = p.len + (p.layer_begin + i / p.B) * p.max_batch + (i % p.B);
+        const int n = nn.v[i % p.B];
+        if (*len + n <= p.seq_cap[i % p.B]) *len += n;
+        else atomicExch(p.status, kStatusCapacity);             // full: nothing of this sequence's rows was written
     }
 }
 
-// Long appends, value side: one warp per block of 16 cache positions of one slab, no block-level synchronisation.
-// Units enumerate (slab, 16-position block) over the 128-aligned range that the appended tokens can touch.
+// Long appends, value side: one warp per block of 16 cache positions of one slab, no synchronisation of any kind
+// between warps (the new lengths are published by a kernel of their own behind both long-append kernels). Units
+// enumerate (slab, 16-position block) over the 128-aligned range that the appended tokens can touch.
 constexpr int kValueWarps = 4;
 __global__ void __launch_bounds__(kValueWarps * 32) prefill_values_kernel(PrefillParams p, NewCounts nn) {
     __shared__ __align__(16) unsigned char vs_all[kValueWarps][1280];
-    __shared__ int is_last;
     const int lane = threadIdx.x & 31, warp = threadIdx.x >> 5;
     const ChunkLayout cl = chunk_layout(p.m_words, p.groups);
     const int blocks_per_seq = p.tiles_per_seq * (kPrefillTile / 16);
     const long unit = (long)blockIdx.x * kValueWarps + warp;
     const long n_units = (long)p.n_layers * p.B * p.Hkv * blocks_per_seq;
-    if (unit < n_units) {
-        // KV head fastest: warps that run at the same time read the same token rows of neighbouring heads, i.e. whole
-        // contiguous [Hkv][d] rows of the input between them
-        const int kvh = (int)(unit % p.Hkv);
-        const int blk = (int)((unit / p.Hkv) % blocks_per_seq);
-        const long seq_local = unit / ((long)p.Hkv * blocks_per_seq);
-        const int b = (int)(seq_local % p.B), ll = (int)(seq_local / p.B);
-        const int layer = p.layer_begin + ll;
-        const int len0 = p.len[layer * p.max_batch + b];
-        const int n_new = (len0 + nn.v[b] <= p.seq_cap[b]) ? nn.v[b] : 0;       // no room: nothing is written
-        const int pos0 = (len0 / kPrefillTile) * kPrefillTile + blk * 16;
-        if (pos0 + 16 > len0 && pos0 < len0 + n_new) {
-            store_value_block16(p, cl, layer, ll, b, kvh, len0, n_new, pos0, vs_all[warp], lane);
-        }
-    }
-    prefill_publish_lengths(p, nn, &is_last);
+    if (unit >= n_units) return;
+    // KV head fastest: warps that run at the same time read the same token rows of neighbouring heads, i.e. whole
+    // contiguous [Hkv][d] rows of the input between them
+    const int kvh = (int)(unit % p.Hkv);
+    const int blk = (int)((unit / p.Hkv) % blocks_per_seq);
+    const long seq_local = unit / ((long)p.Hkv * blocks_per_seq);
+    const int b = (int)(seq_local % p.B), ll = (int)(seq_local / p.B);
+    const int layer = p.layer_begin + ll;
+    const int len0 = p.len[layer * p.max_batch + b];
+    const int n_new = (len0 + nn.v[b] <= p.seq_cap[b]) ? nn.v[b] : 0;           // no room: nothing is written
+    const int pos0 = (len0 / kPrefillTile) * kPrefillTile + blk * 16;
+    if (pos0 + 16 > len0 && pos0 < len0 + n_new)
+        store_value_block16(p, cl, layer, ll, b, kvh, len0, n_new, pos0, vs_all[warp], lane);
 }
 
 template <int NBC, bool ROPE>                   // ROPE: the key tiles are rotated in shared memory before the MMAs read them
@@ -574,7 +572,7 @@ __device__ __forceinline__ void prefill_body(const PrefillParams &p, const NewCo
     (void)H1B_IN_BOUNDS(As0 + kKeyStages * SM::kABytes <= smem_unaligned + SM::kTotal, p.status, kSitePrefillSmem);
     __shared__ uint32_t tmem_base_s;
     __shared__ __align__(8) unsigned long long mma_bar_s[2];
-    __shared__ int is_last, gave_up;
+    __shared__ int gave_up;
     const int tid = threadIdx.x, lane = tid & 31, warp = tid >> 5;
     const int m = p.m_words * 32;
     const ChunkLayout cl = chunk_layout(p.m_words, p.groups);
@@ -803,7 +801,6 @@ __device__ __forceinline__ void prefill_body(const PrefillParams &p, const NewCo
     tc_fence_before_sync();
     __syncthreads();
     if (warp == 0 && !skip_all) { tc_fence_after_sync(); tmem_dealloc(tmem_d, 2 * NBC); }
-    prefill_publish_lengths(p, nn, &is_last);
 }
 
 // The two entry points of the body above. The rotating variant keeps 64 table entries in registers; its register
@@ -819,6 +816,203 @@ __global__ void __maxnreg__(176) prefill_rope_kernel(PrefillParams p, NewCounts 
 }
 template <int NBC> struct PrefillEntry<NBC, false> { static constexpr auto fn = prefill_kernel<NBC>; };
 template <int NBC> struct PrefillEntry<NBC, true> { static constexpr auto fn = prefill_rope_kernel<NBC>; };
+
+// ===========================================================================
+// Long appends without rotary embedding: the same contraction with the work split by ROLE, no block-wide barrier
+// in the steady state.
+//   warp 0        producer: one elected lane requests each 128 x 128 key tile with two tiled tensor copies (TMA, one
+//                 per 64-channel half, 128-byte swizzle: the operand layout the tensor cores read), completion on the
+//                 stage's "full" barrier; the whole warp brings in the projection pieces when the layer changes
+//   warp 1        one lane issues the 16 tcgen05.mma of a tile into one of two TMEM accumulators and commits them
+//                 twice: to the stage's "empty" barrier (the producer may refill it) and to the accumulator's
+//                 "full" barrier (the epilogue may read it)
+//   warps 2..9    epilogue, two warps per TMEM lane quarter: tcgen05.ld, sign-pack, key words to the cache, then one
+//                 arrival per warp on the accumulator's "empty" barrier
+// Every role walks the same list of work items (see prefill_body) and numbers the tiles alike, so stage, accumulator
+// and barrier phase follow from the tile's number. Rows of a tile that lie outside the appended range come in as
+// whatever the tensor holds there (zeros outside it) and are never stored. Every wait is bounded; a role that gives
+// up records the time-out, and the others run into their own limits; TMEM is released by the warp that took it.
+// ===========================================================================
+constexpr int kTmaThreads = 320;
+template <int NBC>
+__global__ void __launch_bounds__(kTmaThreads, 1) prefill_tma_kernel(const __grid_constant__ CUtensorMap kmap, PrefillParams p,
+                                                                      NewCounts nn) {
+    using SM = PrefillSmem<NBC>;
+    extern __shared__ unsigned char smem_unaligned[];
+    unsigned char *smem = smem_unaligned + ((1024u - (smem_addr(smem_unaligned) & 1023u)) & 1023u);
+    unsigned char *Rs = smem, *As0 = smem + SM::kRBytes;
+    (void)H1B_IN_BOUNDS(As0 + kKeyStages * SM::kABytes <= smem_unaligned + SM::kTotal, p.status, kSitePrefillSmem);
+    __shared__ uint32_t tmem_base_s;
+    __shared__ __align__(8) unsigned long long bars[2 * kKeyStages + 5];
+    __shared__ int gave_up;
+    const int tid = threadIdx.x, lane = tid & 31, warp = tid >> 5;
+    const int m = p.m_words * 32;
+    const ChunkLayout cl = chunk_layout(p.m_words, p.groups);
+    const int col_blocks = (m + NBC - 1) / NBC;
+    // A work item is ONE tile of 128 cache positions of one (layer, sequence) across ALL its KV heads (the item's tiles
+    // are the heads): a block then reads whole contiguous [Hkv][128] token rows of the input, 128 of them in a row,
+    // whatever the other blocks are doing at that moment.
+    const long n_work = (long)p.n_layers * p.B * p.tiles_per_seq * col_blocks;
+    const uint32_t full0 = smem_addr(&bars[0]), empty0 = full0 + 8 * kKeyStages;
+    const uint32_t accf0 = empty0 + 8 * kKeyStages, acce0 = accf0 + 16, rfull = acce0 + 16;
+
+    if (tid == 0) {
+        gave_up = (*reinterpret_cast<volatile const int32_t *>(p.status) != kStatusOk);
+        for (int s = 0; s < kKeyStages; ++s) { mbar_init(full0 + 8 * s, 1); mbar_init(empty0 + 8 * s, 1); }
+        for (int a = 0; a < 2; ++a) { mbar_init(accf0 + 8 * a, 1); mbar_init(acce0 + 8 * a, 8); }
+        mbar_init(rfull, 1);
+        mbar_fence_init();
+    }
+    __syncthreads();
+    const bool skip_all = gave_up != 0;                         // a block that starts after a failure elsewhere does nothing
+    // two accumulators of 2 NBC fp32 columns: [y from the first piece | y from the second], added in the epilogue
+    if (warp == 1 && !skip_all) tmem_alloc(smem_addr(&tmem_base_s), 4 * NBC);
+    tc_fence_before_sync();
+    __syncthreads();
+    tc_fence_after_sync();
+    const uint32_t tmem_d = skip_all ? 0u : tmem_base_s;
+
+    // one work item: (slab, run of tiles, block of sketch columns), the same for every role
+    struct Item { int b, ll, layer, col0, first_tile, n_tiles, len0, n_new; };
+    auto item_of = [&](long work) {
+        Item it;
+        const int cbk = (int)(work % col_blocks);
+        const int pt = (int)((work / col_blocks) % p.tiles_per_seq);
+        const long seq_local = work / ((long)col_blocks * p.tiles_per_seq);
+        it.b = (int)(seq_local % p.B); it.ll = (int)(seq_local / p.B);
+        it.layer = p.layer_begin + it.ll;
+        it.len0 = p.len[it.layer * p.max_batch + it.b];
+        it.n_new = (it.len0 + nn.v[it.b] <= p.seq_cap[it.b]) ? nn.v[it.b] : 0;
+        it.first_tile = it.len0 / kPrefillTile + pt;
+        it.n_tiles = (it.first_tile * kPrefillTile < it.len0 + it.n_new) ? p.Hkv : 0;   // one tile per KV head
+        it.col0 = cbk * NBC;
+        return it;
+    };
+
+    int seq = 0;                                                // tiles this block has pushed through so far
+    int loaded_layer = -1, loaded_col0 = -1, r_loads = 0;
+    bool failed = false;
+    int issued = 0;                                             // (MMA lane) tiles whose MMAs were issued
+    if (!skip_all && warp == 0) {
+        // ------------------------------------------------------------------ producer
+        for (long work = blockIdx.x; work < n_work && !failed; work += gridDim.x) {
+            const Item it = item_of(work);
+            if (it.n_tiles == 0) continue;
+            if (it.layer != loaded_layer || it.col0 != loaded_col0) {
+                // the tensor cores must be done with the old pieces: the newest tile's stage has been released
+                if (seq > 0 && !mbar_wait_bounded(empty0 + 8 * ((seq - 1) % kKeyStages), (uint32_t)(((seq - 1) / kKeyStages) & 1), kWaitLimitNs)) {
+                    failed = true; break;
+                }
+                const uint16_t *src = p.Rh + ((size_t)it.layer * 2 * m + it.col0) * kHeadDim;       // [L][2][m][128]
+                for (int e = lane; e < 2 * NBC * 16; e += 32) {
+                    const int c = e & 15, n = (e >> 4) % NBC, piece = e / (16 * NBC);
+                    cp_async_16(smem_addr(Rs + kmajor_sw128_off(2 * NBC, piece * NBC + n, c)),
+                                src + ((size_t)piece * m + n) * kHeadDim + c * 8, 16);
+                }
+                cp_async_wait_all();
+                fence_proxy_async_smem();
+                __syncwarp();
+                if (lane == 0) mbar_arrive(rfull);
+                loaded_layer = it.layer; loaded_col0 = it.col0; ++r_loads;
+            }
+            if (lane == 0) {
+                for (int ti = 0; ti < it.n_tiles; ++ti) {
+                    const int sq = seq + ti, s = sq % kKeyStages;
+                    if (sq >= kKeyStages && !mbar_wait_bounded(empty0 + 8 * s, (uint32_t)((sq / kKeyStages - 1) & 1), kWaitLimitNs)) {
+                        failed = true; break;
+                    }
+                    const int zrow = (it.ll * p.B + it.b) * p.Tn + it.first_tile * kPrefillTile - it.len0;
+                    const uint32_t dst = smem_addr(As0 + s * SM::kABytes);
+                    mbar_arrive_expect_tx(full0 + 8 * s, SM::kABytes);
+                    tma_load_3d(dst, &kmap, 0, ti, zrow, full0 + 8 * s);
+                    tma_load_3d(dst + SM::kABytes / 2, &kmap, 64, ti, zrow, full0 + 8 * s);
+                }
+            }
+            failed = __any_sync(0xffffffffu, failed);
+            seq += it.n_tiles;
+        }
+    } else if (!skip_all && warp == 1) {
+        // ------------------------------------------------------------------ tensor cores: one lane issues
+        if (lane == 0) {
+            // ONE instruction per K slice covers both fp16 pieces of the projection (N = 2 NBC columns, the stacked
+            // operand): the key tile is then read from shared memory once per slice, not twice, which leaves the
+            // shared-memory bandwidth the tile copies need while the tensor cores run
+            const uint32_t idesc = umma_idesc_f16_m128(2 * NBC);
+            for (long work = blockIdx.x; work < n_work && !failed; work += gridDim.x) {
+                const Item it = item_of(work);
+                if (it.n_tiles == 0) continue;
+                if (it.layer != loaded_layer || it.col0 != loaded_col0) {
+                    if (!mbar_wait_bounded(rfull, (uint32_t)(r_loads & 1), kWaitLimitNs)) { failed = true; break; }
+                    loaded_layer = it.layer; loaded_col0 = it.col0; ++r_loads;
+                }
+                for (int ti = 0; ti < it.n_tiles; ++ti) {
+                    const int sq = seq + ti, s = sq % kKeyStages, a = sq & 1;
+                    if (!mbar_wait_bounded(full0 + 8 * s, (uint32_t)((sq / kKeyStages) & 1), kWaitLimitNs)) { failed = true; break; }
+                    if (sq >= 2 && !mbar_wait_bounded(acce0 + 8 * a, (uint32_t)((sq / 2 - 1) & 1), kWaitLimitNs)) { failed = true; break; }
+                    tc_fence_after_sync();
+                    const uint32_t a_base = smem_addr(As0 + s * SM::kABytes), r_base = smem_addr(Rs);
+                    const uint32_t acc = tmem_d + (uint32_t)(a * 2 * NBC);
+#pragma unroll
+                    for (int ks = 0; ks < kHeadDim / 16; ++ks) {
+                        const uint64_t ad = umma_desc_k_sw128(a_base + (ks >> 2) * (kPrefillTile * 128) + (ks & 3) * 32);
+                        const uint64_t bd = umma_desc_k_sw128(r_base + (ks >> 2) * (2 * NBC * 128) + (ks & 3) * 32);
+                        umma_f16(acc, ad, bd, idesc, ks ? 1u : 0u);
+                    }
+                    umma_commit(empty0 + 8 * s);
+                    umma_commit(accf0 + 8 * a);
+                    issued = sq + 1;
+                }
+                seq += it.n_tiles;
+            }
+            // after a failure: give MMAs that were issued a bounded time to finish before the TMEM goes back
+            if (failed && issued > 0)
+                (void)mbar_wait_bounded(empty0 + 8 * ((issued - 1) % kKeyStages), (uint32_t)(((issued - 1) / kKeyStages) & 1), 100000000ull);
+        }
+        __syncwarp();
+    } else if (!skip_all) {
+        // ------------------------------------------------------------------ epilogue: signs from the accumulators
+        const int quarter = warp & 3;                           // the TMEM lanes this warp may read
+        const int w_first = (warp - 2) >> 2;                    // of the quarter's two warps: even or odd key words
+        for (long work = blockIdx.x; work < n_work && !failed; work += gridDim.x) {
+            const Item it = item_of(work);
+            if (it.n_tiles == 0) continue;
+            for (int ti = 0; ti < it.n_tiles; ++ti) {
+                const int sq = seq + ti, a = sq & 1;
+                if (!mbar_wait_bounded(accf0 + 8 * a, (uint32_t)((sq / 2) & 1), kWaitLimitNs)) { failed = true; break; }
+                tc_fence_after_sync();
+                const int P0 = it.first_tile * kPrefillTile;
+                const int tn = P0 + quarter * 32 + lane - it.len0;
+                unsigned char *chunk = chunk_ptr(p.ca, it.layer, it.b, ti, (P0 >> 5) + quarter);   // this warp's 32 rows = one chunk of head ti
+#pragma unroll
+                for (int w = w_first; w < NBC / 32; w += 2) {
+                    uint32_t y[32], y2[32];
+                    tmem_ld_32cols(tmem_d + ((uint32_t)(quarter * 32) << 16) + (uint32_t)(a * 2 * NBC) + w * 32, y);
+                    tmem_ld_32cols(tmem_d + ((uint32_t)(quarter * 32) << 16) + (uint32_t)(a * 2 * NBC + NBC) + w * 32, y2);
+#pragma unroll
+                    for (int j = 0; j < 32; ++j) y[j] = __float_as_uint(__uint_as_float(y[j]) + __uint_as_float(y2[j]));
+                    // bit j = (y_j >= 0); adding +0 first turns a negative zero into a positive one (see prefill_body)
+                    uint32_t part[4] = {0u, 0u, 0u, 0u};
+#pragma unroll
+                    for (int j = 7; j >= 0; --j)
+#pragma unroll
+                        for (int k = 0; k < 4; ++k)
+                            part[k] = __funnelshift_l(__float_as_uint(__uint_as_float(y[8 * k + j]) + 0.f), part[k], 1);
+                    const uint32_t neg = part[0] | (part[1] << 8) | (part[2] << 16) | (part[3] << 24);
+                    if (tn >= 0 && tn < it.n_new && H1B_IN_BOUNDS(in_cache(p.ca, chunk, cl.bytes), p.status, kSitePrefillKeys))
+                        *reinterpret_cast<uint32_t *>(chunk + lane * 4 + (it.col0 / 32 + w) * 128) = ~neg;
+                }
+                tc_fence_before_sync();
+                __syncwarp();
+                if (lane == 0) mbar_arrive(acce0 + 8 * a);
+            }
+            seq += it.n_tiles;
+        }
+    }
+    if (failed && lane == 0) atomicExch(p.status, kStatusWaitTimeout);
+    tc_fence_before_sync();
+    __syncthreads();
+    if (warp == 1 && !skip_all) { tc_fence_after_sync(); tmem_dealloc(tmem_d, 4 * NBC); }
+}
 
 // Rt (fp32, [L][d][m]) -> its two fp16 pieces, transposed to [L][2][m][d] (channel contiguous).
 __global__ void split_projection_kernel(const float *Rt, uint16_t *Rh, int n_layers, int m) {
@@ -1672,6 +1866,66 @@ static cudaError_t sm_count(int *n) {
     return cudaSuccess;
 }
 
+// The tensor map of a call's key tensor [n_layers][B][Tn][Hkv][128] fp16 as (channel, KV head, token row): boxes of 64
+// channels x 1 head x 128 token rows, 128-byte swizzle. Made on the host for every call (the pointer is the caller's)
+// and handed to the kernel by value. The encoder is the driver's; it is looked up once.
+typedef CUresult (*EncodeTiledFn)(CUtensorMap *, CUtensorMapDataType, cuuint32_t, void *, const cuuint64_t *, const cuuint64_t *,
+                                  const cuuint32_t *, const cuuint32_t *, CUtensorMapInterleave, CUtensorMapSwizzle,
+                                  CUtensorMapL2promotion, CUtensorMapFloatOOBfill);
+static EncodeTiledFn tensor_map_encoder() {
+    static EncodeTiledFn fn = nullptr;
+    static bool looked = false;
+    std::lock_guard<std::mutex> lock(g_setup_mutex);
+    if (!looked) {
+        void *sym = nullptr;
+        cudaDriverEntryPointQueryResult q;
+        if (cudaGetDriverEntryPoint("cuTensorMapEncodeTiled", &sym, cudaEnableDefault, &q) == cudaSuccess &&
+            q == cudaDriverEntryPointSuccess)
+            fn = reinterpret_cast<EncodeTiledFn>(sym);
+        else
+            (void)cudaGetLastError();
+        looked = true;
+    }
+    return fn;
+}
+static bool key_tensor_map(const PrefillParams &p, CUtensorMap *map) {
+    const EncodeTiledFn enc = tensor_map_encoder();
+    const unsigned long long rows = (unsigned long long)p.n_layers * p.B * p.Tn;
+    if (!enc || rows >= 0x7fffff00ull) return false;            // token-row coordinates are 32-bit
+    const cuuint64_t dims[3] = {(cuuint64_t)kHeadDim, (cuuint64_t)p.Hkv, (cuuint64_t)rows};
+    const cuuint64_t strides[2] = {(cuuint64_t)kHeadDim * 2, (cuuint64_t)p.Hkv * kHeadDim * 2};     // bytes, dimensions 1 and 2
+    const cuuint32_t box[3] = {64u, 1u, (cuuint32_t)kPrefillTile}, elem[3] = {1u, 1u, 1u};
+    return enc(map, CU_TENSOR_MAP_DATA_TYPE_FLOAT16, 3, const_cast<uint16_t *>(p.k), dims, strides, box, elem,
+               CU_TENSOR_MAP_INTERLEAVE_NONE, CU_TENSOR_MAP_SWIZZLE_128B, CU_TENSOR_MAP_L2_PROMOTION_L2_256B,
+               CU_TENSOR_MAP_FLOAT_OOB_FILL_NONE) == CUDA_SUCCESS;
+}
+
+template <int NBC>
+static cudaError_t prefill_tma_attributes() {
+    using SM = PrefillSmem<NBC>;
+    static bool attr_set[64] = {};
+    int dev = 0;
+    cudaGetDevice(&dev);
+    if (dev < 0 || dev >= 64) return cudaErrorInvalidDevice;
+    std::lock_guard<std::mutex> lock(g_setup_mutex);
+    if (!attr_set[dev]) {
+        cudaError_t e = cudaFuncSetAttribute(prefill_tma_kernel<NBC>, cudaFuncAttributeMaxDynamicSharedMemorySize, SM::kTotal);
+        if (e != cudaSuccess) return e;
+        e = cudaFuncSetAttribute(prefill_tma_kernel<NBC>, cudaFuncAttributePreferredSharedMemoryCarveout, cudaSharedmemCarveoutMaxShared);
+        if (e != cudaSuccess) return e;
+        attr_set[dev] = true;
+    }
+    return cudaSuccess;
+}
+template <int NBC>
+static cudaError_t launch_prefill_tma_t(const CUtensorMap &map, const PrefillParams &p, const NewCounts &nn, cudaStream_t st, int grid) {
+    using SM = PrefillSmem<NBC>;
+    cudaError_t e = prefill_tma_attributes<NBC>();
+    if (e != cudaSuccess) return e;
+    prefill_tma_kernel<NBC><<<(unsigned)grid, kTmaThreads, SM::kTotal, st>>>(map, p, nn);
+    return cudaGetLastError();
+}
+
 template <int NBC, bool ROPE>
 static cudaError_t launch_prefill_t(const PrefillParams &p, const NewCounts &nn, cudaStream_t st, int grid) {
     using SM = PrefillSmem<NBC>;
@@ -1681,6 +1935,9 @@ static cudaError_t launch_prefill_t(const PrefillParams &p, const NewCounts &nn,
     return cudaGetLastError();
 }
 
+#ifndef H1B_PREFILL_TMA
+#define H1B_PREFILL_TMA 1
+#endif
 // The value kernel (instruction-bound) and the key kernel (latency-bound around the tensor cores) are independent
 // until the lengths are published, so they run side by side: the value kernel on `side`, forked from and joined
 // back into `st` with the two events (all three may be null: then one after the other on `st`).
@@ -1695,10 +1952,11 @@ cudaError_t launch_prefill(const PrefillParams &p_in, const NewCounts &nn, cudaS
     int n_sm = 0;
     cudaError_t e = sm_count(&n_sm);
     if (e != cudaSuccess) return e;
-    const long kwork = prefill_key_blocks(p, nbc);
+    const bool tma_path = H1B_PREFILL_TMA && !p.rope.table;
+    const long kwork = tma_path ? (long)p.n_layers * p.B * p.tiles_per_seq * ((p.m_words * 32 + nbc - 1) / nbc)
+                                : prefill_key_blocks(p, nbc);
     const long kblocks = kwork < n_sm ? kwork : n_sm;
     if (vblocks <= 0 || kblocks <= 0 || vblocks + kblocks > 0x7fffffffL) return cudaErrorInvalidConfiguration;
-    p.total_blocks = (int)(vblocks + kblocks);
     const bool forked = side && fork && join;
     if ((e = prefill_values_attributes()) != cudaSuccess) return e;
     if (forked) {
@@ -1707,8 +1965,11 @@ cudaError_t launch_prefill(const PrefillParams &p_in, const NewCounts &nn, cudaS
     }
     // the key kernel first: one block of it settles on every SM (its shared memory allows no more), and the value
     // kernel's small blocks fill the registers and issue slots that are left
+    CUtensorMap kmap;
     if (p.rope.table)
         e = (nbc == 128) ? launch_prefill_t<128, true>(p, nn, st, (int)kblocks) : launch_prefill_t<64, true>(p, nn, st, (int)kblocks);
+    else if (tma_path && key_tensor_map(p, &kmap))       // the role-split kernel fed by tiled tensor copies
+        e = (nbc == 128) ? launch_prefill_tma_t<128>(kmap, p, nn, st, (int)kblocks) : launch_prefill_tma_t<64>(kmap, p, nn, st, (int)kblocks);
     else
         e = (nbc == 128) ? launch_prefill_t<128, false>(p, nn, st, (int)kblocks) : launch_prefill_t<64, false>(p, nn, st, (int)kblocks);
     if (e != cudaSuccess) return e;
@@ -1720,6 +1981,10 @@ cudaError_t launch_prefill(const PrefillParams &p_in, const NewCounts &nn, cudaS
         if ((e = cudaEventRecord(join, side)) != cudaSuccess) return e;
         if ((e = cudaStreamWaitEvent(st, join, 0)) != cudaSuccess) return e;
     }
+    // every block of both kernels has read the old lengths by the time this runs
+    prefill_publish_kernel<<<1, 256, 0, st>>>(p, nn);
+    if ((e = cudaGetLastError()) != cudaSuccess) return e;
+    ++*launches;
     return cudaSuccess;
 }
 
@@ -1821,6 +2086,11 @@ cudaError_t warm_kernel_attributes(int m_words, int groups, bool paired, bool pa
     if (m_words * 32 >= 128) e = rope ? prefill_attributes<128, true>() : prefill_attributes<128, false>();
     else e = rope ? prefill_attributes<64, true>() : prefill_attributes<64, false>();
     if (e != cudaSuccess) return e;
+    if (!rope) {
+        e = (m_words * 32 >= 128) ? prefill_tma_attributes<128>() : prefill_tma_attributes<64>();
+        if (e != cudaSuccess) return e;
+        (void)tensor_map_encoder();
+    }
     if ((e = prefill_values_attributes()) != cudaSuccess) return e;
     int n = 0;
     return sm_count(&n);

@@ -152,13 +152,10 @@ struct PrefillParams {          // long appends: tensor-core projection
     CacheAddr ca;
     int32_t *len;               // [L][max_batch]
     int32_t *status;            // device status word (bounded-wait timeouts)
-    int32_t *done;              // block counter (zero between launches)
     const int32_t *seq_cap;     // [max_batch] tokens each sequence has room for (see AppendParams)
     int layer_begin, n_layers, B, Tn, Hkv, max_batch, m_words, groups;
     int tiles_per_seq;          // 128-position tiles that can overlap the appended range of a sequence
     int tiles_per_block;        // consecutive tiles handled by one block (the projection is loaded once per block)
-    int total_blocks;           // blocks of the key kernel plus blocks of the value kernel: the last of them all to finish
-                                // publishes the new lengths (the two kernels may run side by side)
     RopeRef rope;
 };
 

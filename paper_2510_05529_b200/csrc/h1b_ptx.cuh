@@ -63,6 +63,14 @@ __device__ __forceinline__ void bulk_copy_g2s(uint32_t dst, const void *src, uin
         ::"r"(dst), "l"(src), "r"(bytes), "r"(bar) : "memory");
 }
 
+// Tiled tensor copy (TMA) global -> this CTA's shared memory, three coordinates (x innermost; x * element size must be
+// a multiple of 16 bytes), no multicast: one destination CTA. Completion is signalled on `bar` as transferred bytes.
+__device__ __forceinline__ void tma_load_3d(uint32_t dst, const void *tensor_map, int x, int y, int z, uint32_t bar) {
+    asm volatile(
+        "cp.async.bulk.tensor.3d.shared::cluster.global.tile.mbarrier::complete_tx::bytes [%0], [%1, {%2, %3, %4}], [%5];"
+        ::"r"(dst), "l"(tensor_map), "r"(x), "r"(y), "r"(z), "r"(bar) : "memory");
+}
+
 // 16-byte async copy global -> shared; `src_bytes` = 16, or 0 to fill the 16 bytes with zeros.
 __device__ __forceinline__ void cp_async_16(uint32_t dst, const void *src, uint32_t src_bytes) {
     asm volatile("cp.async.cg.shared.global [%0], [%1], 16, %2;" ::"r"(dst), "l"(src), "r"(src_bytes) : "memory");
