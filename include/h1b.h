@@ -195,8 +195,13 @@ int h1b_decode_attention_multi(h1b_ctx *ctx, int layer_begin, int n_layers, cons
 /* Attention for a whole run of Tn query tokens per sequence (a prompt, or a
  * chunk of one): the queries are the sequences' last Tn cached tokens (append
  * their keys and values first), query token i attends to cached tokens
- * [0, len - Tn + i + 1). Any Tn >= 1: the call walks the run in blocks of
- * H1B_MAX_QUERY_TOKENS query tokens, each block one pass of the same kernels
+ * [0, len - Tn + i + 1). Any Tn >= 1. Runs of 32 tokens or more (head
+ * dimension 128, 4-bit values, m <= 256) are processed in blocks of 128 query
+ * tokens x 128 cached tokens on the tensor cores: Eq. 3 as one dense +-1
+ * contraction per block (exact integers), Eq. 5 with each tile's values
+ * dequantised once for all its queries; `out` doubles as scratch for the query
+ * sketches until its rows are written. Other runs walk in blocks of
+ * H1B_MAX_QUERY_TOKENS query tokens, each block one pass of the decode kernels
  * over the part of the cache it may see. q: DEVICE fp16 [n_layers][B][Tn][Hq][d];
  * out: DEVICE float32, same shape. Every sequence must hold at least Tn
  * tokens in every layer of the call (H1B_ERR_INVALID_ARG otherwise). With the
@@ -360,6 +365,19 @@ int h1b_debug_scores(h1b_ctx *ctx, int layer, int seq, int kv_head, const void *
  * H1B_ERR_INVALID_ARG when the indices are not part of that launch. */
 int h1b_debug_partials(h1b_ctx *ctx, int layer, int seq, int q_token, int q_head,
                        int32_t *n_splits_host, float *hmin_host, float *wsum_host, int max_splits);
+
+/* Test helpers of h1b_prefill_attention (no counterpart in the paper).
+ *   h1b_debug_prompt_scores  the NEXT h1b_prefill_attention call that takes the tile route also writes the integer
+ *                            scores m - 2 * Hamming (Eq. 3) its tensor-core contraction produced for one (layer,
+ *                            sequence, query head) to score_dev, DEVICE int32 [Tn][n_tokens] (entry [i][t] for query
+ *                            token i of the run and cached token t < n_tokens; tokens beyond the tiles that query
+ *                            block visits are not written). score_dev NULL switches it off.
+ *   h1b_debug_prompt_route   tiles = 0: h1b_prefill_attention walks every run in blocks of H1B_MAX_QUERY_TOKENS through
+ *                            the decode kernels (the route short runs take); tiles = 1 (default): runs of 32 query tokens
+ *                            or more take the 128 x 128 tile kernel where the cache format allows it (head dimension
+ *                            128, 4-bit values, m <= 256). Both routes compute the same thing. */
+int h1b_debug_prompt_scores(h1b_ctx *ctx, int layer, int seq, int q_head, int32_t *score_dev, int n_tokens);
+int h1b_debug_prompt_route(h1b_ctx *ctx, int tiles);
 
 /* Bounds-checked build (no counterpart in the paper; a debugging aid). When the
  * library is compiled with -DH1B_DEBUG_BOUNDS, every address a kernel derives

@@ -89,6 +89,8 @@ def load_library(rebuild: bool = True) -> ctypes.CDLL:
         "h1b_debug_partials": (ctypes.c_int, [vp, ctypes.c_int, ctypes.c_int, ctypes.c_int, ctypes.c_int, i32p, vp, vp,
                                               ctypes.c_int]),
         "h1b_debug_wait_timeout": (ctypes.c_int, [vp, ctypes.c_uint64, vp]),
+        "h1b_debug_prompt_scores": (ctypes.c_int, [vp, ctypes.c_int, ctypes.c_int, ctypes.c_int, vp, ctypes.c_int]),
+        "h1b_debug_prompt_route": (ctypes.c_int, [vp, ctypes.c_int]),
         "h1b_bounds_checked": (ctypes.c_int, []),
         "h1b_debug_bounds_probe": (ctypes.c_int, [vp, vp]),
         "h1b_set_splits": (ctypes.c_int, [vp, ctypes.c_int]),
@@ -383,6 +385,15 @@ class H1BCache:
         self._check(self.lib.h1b_debug_partials(self._h, layer, seq, q_token, q_head, ctypes.byref(n), hmin.ctypes.data,
                                                 wsum.ctypes.data, max_splits))
         return hmin[:n.value].copy(), wsum[:n.value].copy()
+
+    def h1b_debug_prompt_scores(self, layer: int, seq: int, q_head: int, score_dev, n_tokens: int):
+        """The next tile-route h1b_prefill_attention call exports one head's integer scores to score_dev (int32 CUDA [Tn, n_tokens])."""
+        ptr = None if score_dev is None else _dev_ptr(score_dev, torch.int32, "score_dev")
+        self._check(self.lib.h1b_debug_prompt_scores(self._h, layer, seq, q_head, ptr, n_tokens))
+
+    def h1b_debug_prompt_route(self, tiles: bool):
+        """False: prompt attention walks 16 query tokens at a time through the decode kernels, whatever the run's length."""
+        self._check(self.lib.h1b_debug_prompt_route(self._h, int(bool(tiles))))
 
     def h1b_debug_bounds_probe(self, stream=None):
         """Bounds-checked build only: a kernel's check fails on purpose; the next h1b_poll_status() reports it."""

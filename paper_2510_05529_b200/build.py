@@ -11,7 +11,7 @@ _CSRC = os.path.join(_PKG, "csrc")
 # library of its own beside the ordinary one, so that both can be built ahead of time.
 DEBUG_BOUNDS = os.environ.get("H1B_DEBUG_BOUNDS", "0") not in ("", "0")
 LIB_PATH = os.path.join(_PKG, "libh1b_bounds.so" if DEBUG_BOUNDS else "libh1b.so")
-SOURCES = ["h1b_api.cu", "h1b_kernels.cu"]
+SOURCES = ["h1b_api.cu", "h1b_kernels.cu", "h1b_prompt.cu"]
 NVCC_FLAGS = ["-gencode", "arch=compute_100a,code=sm_100a", "-lineinfo", "-O3", "-std=c++17",
               "--use_fast_math=false", "-Xcompiler", "-fPIC", "-shared"]
 

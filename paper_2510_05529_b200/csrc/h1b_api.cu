@@ -24,6 +24,7 @@ constexpr long kTargetItems = 8192;   // decode work items aimed for (one warp e
 constexpr int kMinSplitTokens = 256;
 constexpr int kMaxQueryTokens = H1B_MAX_QUERY_TOKENS;
 constexpr int kMaxGroupHeads = 16;        // query heads per KV head: the attention kernel takes them four at a time
+constexpr int kPromptMinTokens = 32;    // prompt attention: runs of at least this many query tokens take the tile kernel
 constexpr int kPrefillMinTokens = 64;   // appends of at least this many tokens per sequence take the tensor-core path
 
 struct Plan {
@@ -187,6 +188,9 @@ struct h1b_ctx {
     size_t events_used;
     cudaStream_t side;                 // long appends: the value kernel runs here, beside the key kernel
     cudaEvent_t fork, join;            // ... forked from and joined back into the caller's stream
+    bool no_prompt_tiles;              // test helper: prompt attention through the 16-token route whatever the run's length
+    int32_t *dbg_scores;               // test helper: where the next prompt-attention call exports one head's scores
+    int dbg_layer, dbg_seq, dbg_head, dbg_T;
     DecodeParams last_decode;          // the most recent attention launch (test helper: h1b_debug_partials)
     bool have_last_decode;
     std::string err;
@@ -302,6 +306,8 @@ int h1b_init_projection(const h1b_config *cfg, uint64_t seed, const float *Rt_ho
     ctx->events_used = 0;
     ctx->side = nullptr; ctx->fork = nullptr; ctx->join = nullptr;
     ctx->have_last_decode = false;
+    ctx->dbg_scores = nullptr;
+    ctx->no_prompt_tiles = false;
     cudaStream_t st = static_cast<cudaStream_t>(stream);
     auto bail = [&](cudaError_t e, const char *what) {
         fail(nullptr, H1B_ERR_CUDA, "%s: %s", what, cudaGetErrorString(e));
@@ -353,6 +359,12 @@ int h1b_init_projection(const h1b_config *cfg, uint64_t seed, const float *Rt_ho
     // array's module is loaded, its memory backed, before any region in which the caller may not allocate).
     e = warm_kernel_attributes(plan.m_words, plan.groups, ctx->paired, plan.page_chunks > 0, (cfg->flags & H1B_FLAG_ROPE) != 0);
     if (e != cudaSuccess) return bail(e, "kernel attributes");
+    if (prompt_attention_supported(plan.m_words, plan.groups, ctx->paired)) {
+        PromptParams pw = {};
+        pw.m_words = plan.m_words; pw.groups = plan.groups;
+        e = launch_prompt_attention(pw, nullptr, nullptr, true);
+        if (e != cudaSuccess) return bail(e, "kernel attributes (prompt attention)");
+    }
     e = resolve_static_scratch(cfg->device);
     if (e != cudaSuccess) return bail(e, "cudaGetSymbolAddress(built-in scratch array)");
     // without these three the two long-append kernels simply run one after the other
@@ -446,6 +458,7 @@ static SketchParams sketch_params(h1b_ctx *ctx, int layer_begin, int n_layers, c
     sp.Tq = 1;
     sp.q_seq_rows = sp.Hq;
     sp.q_tail = 0;
+    sp.qw_row_words = 0;
     return sp;
 }
 
@@ -662,6 +675,39 @@ int h1b_prefill_attention(h1b_ctx *ctx, int layer_begin, int n_layers, const voi
             if (ctx->len_host[(size_t)l * ctx->cfg.max_batch + b] < Tn)
                 return fail(ctx, H1B_ERR_INVALID_ARG, "layer %d sequence %d holds %d < Tn = %d tokens", l, b,
                             ctx->len_host[(size_t)l * ctx->cfg.max_batch + b], Tn);
+    // Runs of at least kPromptMinTokens query tokens on a cache format the tile kernel serves: scores and P.V as
+    // dense contractions over blocks of 128 queries x 128 cached tokens. The sketches of all query tokens are kept in
+    // the first words of the output rows they belong to (the kernel reads a row's words before it writes the row).
+    if (Tn >= kPromptMinTokens && !ctx->no_prompt_tiles && prompt_attention_supported(ctx->plan.m_words, ctx->plan.groups, ctx->paired) &&
+        (size_t)n_layers * B * Tn * ctx->cfg.n_q_heads < (size_t)0x7fffffff) {
+        cudaStream_t st = static_cast<cudaStream_t>(stream);
+        int launches = 0;
+        NewCounts none;
+        std::memset(&none, 0, sizeof none);
+        SketchParams sp = sketch_params(ctx, layer_begin, n_layers, q, B, static_cast<uint32_t *>(out),
+                                        (size_t)n_layers * B * Tn * ctx->cfg.n_q_heads * kHeadDim);
+        sp.Hq = Tn * sp.Hq;
+        sp.Tq = Tn;
+        sp.q_seq_rows = sp.Hq;
+        sp.qw_row_words = kHeadDim;                     // one output row (128 floats) per (token, head)
+        H1B_CUDA(ctx, launch_prepare(nullptr, &sp, none, st, &launches));
+        PromptParams pp;
+        pp.ca = cache_addr(ctx);
+        pp.len = at<int32_t>(ctx, ctx->plan.len);
+        pp.qstash = static_cast<const uint32_t *>(out);
+        pp.qstash_row_words = kHeadDim;
+        pp.out = static_cast<float *>(out);
+        pp.status = at<int32_t>(ctx, ctx->plan.status);
+        pp.layer_begin = layer_begin; pp.n_layers = n_layers; pp.B = B; pp.Hkv = ctx->cfg.n_kv_heads; pp.Hq = ctx->cfg.n_q_heads;
+        pp.max_batch = ctx->cfg.max_batch; pp.m_words = ctx->plan.m_words; pp.groups = ctx->plan.groups; pp.Tn = Tn;
+        pp.c = (float)(2.0 * (double)inv_tau * 1.4426950408889634 / (double)ctx->ucfg.sketch_bits);
+        pp.dbg_scores = ctx->dbg_scores; pp.dbg_layer = ctx->dbg_layer; pp.dbg_b = ctx->dbg_seq; pp.dbg_h = ctx->dbg_head;
+        pp.dbg_T = ctx->dbg_T;
+        ctx->dbg_scores = nullptr;                      // one call only
+        H1B_CUDA(ctx, launch_prompt_attention(pp, st, &launches));
+        ctx->launches += launches;
+        return H1B_OK;
+    }
     // every block of the walk is planned before the first one is launched: a call that cannot run launches nothing
     std::vector<DecodePlan> plans;
     for (int t0 = 0; t0 < Tn; t0 += kMaxQueryTokens) {
@@ -1021,6 +1067,7 @@ int h1b_debug_scores(h1b_ctx *ctx, int layer, int seq, int kv_head, const void *
     sp.Tq = 1;
     sp.q_seq_rows = 1;
     sp.q_tail = 0;
+    sp.qw_row_words = 0;
     if (uses_rope(ctx) && ctx->rope_positions < 1)
         return fail(ctx, H1B_ERR_INVALID_ARG, "H1B_FLAG_ROPE: h1b_set_rope_table has not been called");
     int launches = 0;
@@ -1116,6 +1163,22 @@ int h1b_poll_status(h1b_ctx *ctx) {
         return fail(ctx, H1B_ERR_BOUNDS, "bounds-checked build: index check %d of a kernel failed; the access was skipped",
                     s - kStatusBounds);
     return fail(ctx, H1B_ERR_TIMEOUT, "a kernel gave up a bounded wait (status %d)", s);
+}
+
+int h1b_debug_prompt_scores(h1b_ctx *ctx, int layer, int seq, int q_head, int32_t *score_dev, int n_tokens) {
+    if (!ctx) return H1B_ERR_NULL;
+    if (score_dev && (layer < 0 || layer >= ctx->cfg.n_layers || seq < 0 || seq >= ctx->cfg.max_batch || q_head < 0 ||
+                      q_head >= ctx->cfg.n_q_heads || n_tokens < 1))
+        return fail(ctx, H1B_ERR_INVALID_ARG, "(layer %d, seq %d, head %d, %d tokens) out of range", layer, seq, q_head, n_tokens);
+    ctx->dbg_scores = score_dev;
+    ctx->dbg_layer = layer; ctx->dbg_seq = seq; ctx->dbg_head = q_head; ctx->dbg_T = n_tokens;
+    return H1B_OK;
+}
+
+int h1b_debug_prompt_route(h1b_ctx *ctx, int tiles) {
+    if (!ctx) return H1B_ERR_NULL;
+    ctx->no_prompt_tiles = tiles == 0;
+    return H1B_OK;
 }
 
 int h1b_bounds_checked(void) { return bounds_checked_build() ? 1 : 0; }

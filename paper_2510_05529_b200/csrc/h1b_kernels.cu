@@ -278,7 +278,9 @@ __global__ void __launch_bounds__(kProjThreads) prepare_kernel(AppendParams ap, 
         if ((int)threadIdx.x < n_rows) {
             const int row = row0 + threadIdx.x;
             const int h = row % sp.Hq, b = row / sp.Hq;
-            const size_t at = ((size_t)(layer * sp.max_batch + b) * sp.Hq + h) * mw + word;
+            const size_t at = (EXTRAS && sp.qw_row_words > 0)
+                                  ? ((size_t)((layer - sp.layer_begin) * sp.B + b) * sp.Hq + h) * sp.qw_row_words + word
+                                  : ((size_t)(layer * sp.max_batch + b) * sp.Hq + h) * mw + word;
             if (H1B_IN_BOUNDS(at < sp.qwords_words, sp.status, kSiteQueryStore)) sp.qwords[at] = bits;
         }
     } else {
@@ -1805,7 +1807,7 @@ cudaError_t launch_prepare(const AppendParams *ap, const SketchParams *sp, const
     }
     if (blocks <= 0) return cudaSuccess;
     if (blocks > 0x7fffffffL) return cudaErrorInvalidConfiguration;
-    const bool extras = (ap && a.rope.table) || (sp && (q.rope.table || q.q_seq_rows != q.Hq));
+    const bool extras = (ap && a.rope.table) || (sp && (q.rope.table || q.q_seq_rows != q.Hq || q.qw_row_words > 0));
     if (extras) prepare_kernel<true><<<(unsigned)blocks, kProjThreads, 0, st>>>(a, q, nn);
     else prepare_kernel<false><<<(unsigned)blocks, kProjThreads, 0, st>>>(a, q, nn);
     ++*launches;

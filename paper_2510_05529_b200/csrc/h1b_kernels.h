@@ -27,6 +27,9 @@ bool bounds_checked_build();
 cudaError_t launch_debug_bounds_probe(int32_t *status, int32_t *target, cudaStream_t st);
 // One warp waits for at most limit_ns on a barrier phase that never completes, then records the time-out in *status.
 cudaError_t launch_debug_wait_timeout(int32_t *status, unsigned long long limit_ns, cudaStream_t st);
+// Prompt attention on the tensor cores (h1b_prompt.cu): which cache formats it serves, and its launch.
+bool prompt_attention_supported(int m_words, int groups, bool paired);
+cudaError_t launch_prompt_attention(const PromptParams &p, cudaStream_t st, int *launches, bool attributes_only = false);
 cudaError_t launch_set_len(int32_t *len, int n_layers, int max_batch, int seq, int value, cudaStream_t st);
 // Scores of key words [w0, w0 + nw) of every cached token of one slab against qwords[0 .. nw).
 cudaError_t launch_debug_scores(const CacheAddr &ca, int layer, int b, int kvh, const uint32_t *qwords, int len,

@@ -171,6 +171,10 @@ struct SketchParams {           // query sketch
     RopeRef rope;
     const int32_t *len;         // [L][max_batch] (read only when rope.table is set)
     int Tq;
+    // Where a row's words go, when not into the contiguous scratch [L][max_batch][Hq][m/32]: qw_row_words > 0 places row
+    // (layer - layer_begin, b, h) at word ((layer - layer_begin) * B + b) * Hq + h) * qw_row_words (prompt attention keeps
+    // the sketches of all its query tokens in the first words of the output rows they belong to).
+    int qw_row_words;
     // A block of query tokens out of a longer run (prompt attention): the rows of a sequence are Hq consecutive rows,
     // sequences are q_seq_rows rows apart (== Hq: the plain contiguous layout), and q_tail cached tokens lie behind
     // the block's last query token (their positions are counted back from there).
@@ -199,6 +203,21 @@ struct DecodeParams {
     // so Hkv counts pairs, Hq heads, m_words the words of both sketches, and a head's output has out_dim = 64 channels.
     int paired, out_dim;
     float c2;                   // 2 * inv_tau * log2(e) / m : log2-weight per unit of Hamming distance
+};
+
+// Attention for a run of Tn query tokens per sequence (the sequences' last Tn cached tokens), blocks of 128 queries.
+struct PromptParams {
+    CacheAddr ca;
+    const int32_t *len;         // [L][max_batch]
+    const uint32_t *qstash;     // the queries' sketch words: row ((ll * B + b) * Tn + t) * Hq + h, qstash_row_words apart
+    int qstash_row_words;
+    float *out;                 // fp32 [n_layers][B][Tn][Hq][128]
+    int32_t *status;
+    int layer_begin, n_layers, B, Hkv, Hq, max_batch, m_words, groups, Tn;
+    float c;                    // 2 * inv_tau * log2(e) / m : log2-weight per unit of Hamming distance
+    // test helper: the integer scores m - 2 Hamming of one (layer, sequence, query head), [Tn][dbg_T], null = off
+    int32_t *dbg_scores;
+    int dbg_layer, dbg_b, dbg_h, dbg_T;
 };
 
 }  // namespace h1b

@@ -100,3 +100,42 @@ def test_bad_arguments():
     with pytest.raises(binding.H1BError):
         cache.h1b_prefill_attention(_queries(w, 4).cuda(), 0.0)
     cache.close()
+
+
+@pytest.mark.parametrize("hq, hkv, m, G, lens, Tn, inv_tau", [
+    (2, 1, 128, 32, [700, 300], 300, 16.0),       # three blocks of 128 queries, up to six tiles of 128 cached tokens
+    (1, 1, 64, 32, [257, 129], 129, 50.0),        # sketches narrower than a tile row (padded with zeros)
+    (4, 2, 256, 128, [384, 200], 128, 1.0),       # two 128-byte column blocks per sketch; one scale per value vector
+    (2, 2, 128, 32, [130, 33], 33, 1e-3),         # almost uniform weights
+    (2, 2, 128, 32, [513, 512], 500, 400.0),      # peaked softmax: the running minimum moves late, accumulators are rescaled
+])
+def test_tile_route_scores_bit_for_bit_and_both_routes_agree(hq, hkv, m, G, lens, Tn, inv_tau):
+    """Runs of 32 query tokens or more go through the 128 x 128 tile kernel: its tensor-core scores (Eq. 3) are exported
+    and compared bit for bit with the oracle's, its outputs with the oracle (inside _check) and with the 16-token route."""
+    w = h1b_synth.scaled(W["c1_tiny"], batch=2, n_layers=2, n_q_heads=hq, n_kv_heads=hkv, sketch_bits=m, group_size=G)
+    cache, Rt, K, V, lens = _fill(w, lens)
+    q = _queries(w, Tn, seed=11)
+    qd = q.cuda()
+    l, b, h = 1, 0, hq - 1
+    n = int(lens[b])
+    scores = torch.full((Tn, n), -12345, dtype=torch.int32, device="cuda")
+    cache.h1b_debug_prompt_scores(l, b, h, scores, n)
+    out = cache.h1b_prefill_attention(qd, inv_tau).cpu().numpy()
+    torch.cuda.synchronize()
+    cache.h1b_poll_status()
+    got = scores.cpu().numpy()
+    g = h // (hq // hkv)
+    kbits = binding.unpack_words(cache.h1b_export_cache(l, b, g, 0, n)[0], m)
+    for i in range(Tn):
+        qwords, _ = cache.h1b_debug_scores(l, b, g, qd[l, b, i, h].contiguous(), n)
+        ref = oracle.scores(binding.unpack_words(qwords[None], m)[0], kbits)
+        lim = n - Tn + i + 1                                            # what query token i attends to
+        assert np.array_equal(got[i, :lim], ref[:lim]), ("scores of query token", i)
+    worst, flips = _check(w, cache, Rt, K, V, q, lens, out, inv_tau, False)
+    cache.h1b_debug_prompt_route(False)
+    walk = cache.h1b_prefill_attention(qd, inv_tau).cpu().numpy()
+    cache.h1b_debug_prompt_route(True)
+    cache.h1b_poll_status()
+    np.testing.assert_allclose(out, walk, rtol=2e-4, atol=5e-6)
+    print("tile route", hq, hkv, m, G, lens.tolist(), Tn, inv_tau, "max err", worst, "flips", flips)
+    cache.close()
