@@ -1,19 +1,20 @@
 // Attention for a whole run of query tokens (a prompt, or a chunk of one) over the compressed cache, on the
-// 5th-generation tensor cores (sm_100a): Eq. 3 and Eq. 5 for blocks of 128 query tokens x 128 cached tokens.
+// 5th-generation tensor cores (sm_100a): Eq. 3 and Eq. 5 for blocks of 128 query tokens x 64 cached tokens.
 //
-// One block of 128 threads per (layer, sequence, query head, block of 128 query tokens); thread r owns query row r,
-// which is also lane r of every accumulator in tensor memory (TMEM). Per tile of 128 cached tokens:
-//   1. the tile's four 32-token chunks come into shared memory with bulk copies, as the decode kernel reads them;
-//   2. scores (Eq. 3) as ONE dense +-1 contraction: the sketch bits of the 128 queries and of the 128 cached keys are
+// One block of 128 threads per (layer, sequence, query head, block of 128 query tokens), two blocks per SM; thread r
+// owns query row r, which is also lane r of every accumulator in tensor memory (TMEM). Per tile of 64 cached tokens:
+//   1. the tile's two 32-token chunks come into shared memory with bulk copies, as the decode kernel reads them;
+//   2. scores (Eq. 3) as ONE dense +-1 contraction: the sketch bits of the 128 queries and of the 64 cached keys are
 //      expanded to the 8-bit floating-point numbers +1 / -1 (e4m3), and tcgen05.mma (kind::f8f6f4, fp32 accumulate)
-//      gives S = m - 2 Hamming for the whole 128 x 128 block, exactly (sums of at most 512 terms +-1);
-//   3. online softmax on the integer distances, one query row per thread (Eq. 5): running minimum distance, weights
-//      p = 2^((hmin - Hamming) c) with the causal limit of the row, row sums; every weight is split exactly into two
-//      fp16 parts p = hi + lo 2^-11 and the 128 x 128 weight block is written to shared memory as an MMA operand;
-//   4. the tile's values are dequantised ONCE, v = code * scale + zero in fp32, split the same way into two fp16 parts,
-//      and serve all 128 queries: out += P V as three fp16 contractions (hi hi into one accumulator; hi lo and lo hi,
-//      both carrying the factor 2^11, into a second one), so that the products are exact and the sums fp32.
-// When a row's running minimum moves, its accumulator lanes are rescaled in TMEM (rare after the first tiles).
+//      gives S = m - 2 Hamming for the whole 128 x 64 block, exactly (sums of at most 256 terms +-1);
+//   3. online softmax, one query row per thread (Eq. 5): running maximum score (= minimum distance), weights
+//      p = 2^((S - Smax) c / 2) with the causal limit of the row, row sums; every weight is split into two fp16 parts
+//      p = hi + lo (to 2^-22 relative, 2^-25 of the largest weight absolute) and the 128 x 64 weight block is written
+//      to shared memory as an MMA operand;
+//   4. the tile's values are dequantised ONCE, v = code * scale + zero in fp32, split the same way into two fp16
+//      parts, and serve all 128 queries: out += P V as three fp16 contractions hi hi + hi lo + lo hi into one fp32
+//      accumulator (the products are exact).
+// When a row's running maximum moves, its accumulator lanes are rescaled in TMEM (rare after the first tiles).
 // Every wait is bounded; a block that gives up records the time-out and releases its TMEM.
 #include <mutex>
 
@@ -25,24 +26,24 @@ namespace h1b {
 namespace {
 
 constexpr int kPaThreads = 128;
-constexpr int kPaTile = 128;                       // query rows per block = cached tokens per tile
+constexpr int kPaRows = 128;                       // query rows per block
+constexpr int kPaKeys = 64;                        // cached tokens per tile (two 32-token chunks)
 constexpr unsigned long long kPaWaitNs = 2000000000ull;
-constexpr int kPaBig = 1 << 20;
 
-// Byte offset of the 16-byte piece `c16` of row `row` in a K-major operand tile of 128 rows whose rows are `row_bytes`
-// long (a multiple of 128): column blocks of 128 bytes, each [128 rows][128 B] with the 128-byte swizzle.
-__device__ __forceinline__ int pa_off(int row, int c16) {
-    return (c16 >> 3) * (kPaTile * 128) + row * 128 + (((c16 & 7) ^ (row & 7)) << 4);
+// Byte offset of the 16-byte piece `c16` of row `row` in a K-major operand tile of `rows` rows: column blocks of 128
+// bytes, each [rows][128 B] with the 128-byte swizzle.
+__device__ __forceinline__ int pa_off(int rows, int row, int c16) {
+    return (c16 >> 3) * (rows * 128) + row * 128 + (((c16 & 7) ^ (row & 7)) << 4);
 }
 
 template <int MB, int NG>          // MB: bytes of one expanded sketch row (128 for m <= 128, else 256)
 struct PaSmem {
-    static constexpr int kQ = kPaTile * MB, kK = kPaTile * MB;
-    static constexpr int kP = 2 * kPaTile * kPaTile * 2;        // weights hi | lo, [128 queries][128 tokens] fp16
-    static constexpr int kV = 2 * kPaTile * kPaTile * 2;        // values hi | lo, [128 channels][128 tokens] fp16
+    static constexpr int kQ = kPaRows * MB, kK = kPaKeys * MB;
+    static constexpr int kP1 = kPaRows * kPaKeys * 2;           // one part of the weights, [128 queries][64 tokens] fp16
+    static constexpr int kV1 = kHeadDim * kPaKeys * 2;          // one part of the values, [128 channels][64 tokens] fp16
     static constexpr int kChunkMax = (MB / 32) * 128 + 2048 + 128 * NG;
-    static constexpr int kRaw = 4 * kChunkMax;
-    static constexpr int kQOff = 0, kKOff = kQ, kPOff = kKOff + kK, kVOff = kPOff + kP, kRawOff = kVOff + kV;
+    static constexpr int kRaw = 2 * kChunkMax;
+    static constexpr int kQOff = 0, kKOff = kQ, kPOff = kKOff + kK, kVOff = kPOff + 2 * kP1, kRawOff = kVOff + 2 * kV1;
     static constexpr int kTotal = kRawOff + kRaw + 1024;        // + slack to align the operands to 1024 B
 };
 
@@ -59,10 +60,18 @@ __device__ __forceinline__ void expand_word(uint32_t w, uint4 &lo, uint4 &hi) {
     hi = make_uint4(o[4], o[5], o[6], o[7]);
 }
 
+// Two fp32 numbers -> their fp16 parts: hi = fp16(x), lo = fp16(x - hi), x = hi + lo to 2^-22 relative (2^-25 absolute)
+__device__ __forceinline__ void split2(float a, float b, uint32_t &hi, uint32_t &lo) {
+    hi = pack_f16x2(a, b);
+    const float2 hf = half2_bits_to_float2(hi);
+    lo = pack_f16x2(a - hf.x, b - hf.y);
+}
+
 }  // namespace
 
+// MASKED: some row of the block does not see the whole tile (the tiles on and near the diagonal).
 template <int MB, int NG>
-__global__ void __launch_bounds__(kPaThreads, 1) prompt_attention_kernel(PromptParams p) {
+__global__ void __launch_bounds__(kPaThreads, MB == 128 ? 2 : 1) prompt_attention_kernel(PromptParams p) {
     using SM = PaSmem<MB, NG>;
     extern __shared__ unsigned char smem_unaligned[];
     unsigned char *smem = smem_unaligned + ((1024u - (smem_addr(smem_unaligned) & 1023u)) & 1023u);
@@ -72,12 +81,12 @@ __global__ void __launch_bounds__(kPaThreads, 1) prompt_attention_kernel(PromptP
     __shared__ __align__(8) unsigned long long bars[2];         // [0] chunk copies, [1] tensor-core work
     __shared__ int gave_up;
     const int tid = threadIdx.x, lane = tid & 31, warp = tid >> 5;
-    const int mw = p.m_words, m = mw * 32;
+    const int mw = p.m_words;
     const ChunkLayout cl = chunk_layout(mw, NG);
     const int CB = cl.bytes;
 
     // ---- which block of queries
-    const int q_blocks = (p.Tn + kPaTile - 1) / kPaTile;
+    const int q_blocks = (p.Tn + kPaRows - 1) / kPaRows;
     int bid = blockIdx.x;
     const int qb = q_blocks - 1 - bid % q_blocks;               // the blocks with the longest histories first
     bid /= q_blocks;
@@ -86,11 +95,12 @@ __global__ void __launch_bounds__(kPaThreads, 1) prompt_attention_kernel(PromptP
     const int layer = p.layer_begin + ll;
     const int kvh = hq / (p.Hq / p.Hkv);
     const int len = p.len[layer * p.max_batch + b];
-    const int qi = qb * kPaTile + tid;                          // this thread's query token within the run
+    const int qi = qb * kPaRows + tid;                          // this thread's query token within the run
     const bool valid_q = qi < p.Tn;
     const int limit = valid_q ? len - p.Tn + qi + 1 : 0;        // it attends to cached tokens [0, limit)
-    const int limit_blk = len - p.Tn + min(qb * kPaTile + kPaTile - 1, p.Tn - 1) + 1;
-    const int n_tiles = limit_blk > 0 ? (limit_blk + kPaTile - 1) / kPaTile : 0;
+    const int limit_first = len - p.Tn + qb * kPaRows + 1;      // the block's first row sees this many: tiles below are unmasked
+    const int limit_blk = len - p.Tn + min(qb * kPaRows + kPaRows - 1, p.Tn - 1) + 1;
+    const int n_tiles = limit_blk > 0 ? (limit_blk + kPaKeys - 1) / kPaKeys : 0;
     const int n_chunks = (len + 31) >> 5;
 
     const uint32_t bar_copy = smem_addr(&bars[0]), bar_mma = smem_addr(&bars[1]);
@@ -105,14 +115,14 @@ __global__ void __launch_bounds__(kPaThreads, 1) prompt_attention_kernel(PromptP
     for (int e = tid; e < SM::kRaw / 16; e += kPaThreads) reinterpret_cast<uint4 *>(raw)[e] = make_uint4(0u, 0u, 0u, 0u);
     __syncthreads();
     const bool skip_all = gave_up != 0 || n_tiles == 0;         // block-uniform
-    if (warp == 0 && !skip_all) tmem_alloc(smem_addr(&tmem_base_s), 512);
+    if (warp == 0 && !skip_all) tmem_alloc(smem_addr(&tmem_base_s), 256);
     tc_fence_before_sync();
     __syncthreads();
     tc_fence_after_sync();
     if (skip_all) return;
     const uint32_t tmem = tmem_base_s;
     const uint32_t t_lane = tmem + ((uint32_t)(warp * 32) << 16);       // this warp's quarter of the TMEM lanes
-    constexpr uint32_t kColS = 0, kColO1 = 128, kColO2 = 256;
+    constexpr uint32_t kColS = 0, kColO = 128;
 
     // ---- this row's query sketch, expanded (rows past the run's end: whatever their words hold; never used)
     {
@@ -122,83 +132,95 @@ __global__ void __launch_bounds__(kPaThreads, 1) prompt_attention_kernel(PromptP
         for (int w = 0; w < MB / 32; ++w) {
             uint4 lo = make_uint4(0u, 0u, 0u, 0u), hi = lo;     // words the sketch does not have: zeros (contribute 0)
             if (w < mw) expand_word(__ldg(qw + w), lo, hi);
-            *reinterpret_cast<uint4 *>(Qs + pa_off(tid, 2 * w)) = lo;
-            *reinterpret_cast<uint4 *>(Qs + pa_off(tid, 2 * w + 1)) = hi;
+            *reinterpret_cast<uint4 *>(Qs + pa_off(kPaRows, tid, 2 * w)) = lo;
+            *reinterpret_cast<uint4 *>(Qs + pa_off(kPaRows, tid, 2 * w + 1)) = hi;
         }
     }
-    int hmin = kPaBig;
-    float lsum = 0.f;
+    // scores are handled as the floats the tensor cores deliver: S = m - 2 Hamming, so the running minimum distance is
+    // the running maximum score and p = 2^((S - Smax) c / 2)
+    const float ch2 = 0.5f * p.c;
+    float smax = -1e30f, lsum = 0.f;
     uint32_t copy_phase = 0, mma_phase = 0;
     bool failed = false;
-    const uint32_t idesc = umma_idesc_f16_m128(kPaTile);
-    const int my_cc = tid >> 5, my_tt = tid & 31;               // this thread's key of a tile: chunk and token in it
-    const int vblock = tid >> 4, vu = tid & 15;                 // value work: 16-token block of the tile, sixteenth of it
+    const uint32_t idesc_s = umma_idesc_f16_m128(kPaKeys), idesc_o = umma_idesc_f16_m128(kHeadDim);
+    // this thread's share of the tile's keys: half a key (MB / 64 words of it)
+    const int k_key = tid >> 1, k_w0 = (tid & 1) * (MB / 64);
+    // this thread's share of the tile's values: 16-token block vt, 64-channel half vh, row vr of the channel blocks,
+    // word pair vi (channel blocks 4 vh + 2 vi, + 1: one value group)
+    const int vt = tid >> 5, vh = (tid >> 4) & 1, vr = (tid >> 1) & 7, vi = tid & 1;
+    const int VAL = mw * 128, ZERO = VAL + 2048, SCALE = ZERO + 64 * NG;
+    const int vg = NG == 4 ? vh * 2 + vi : 0;                   // the value group of this thread's channels
 
     for (int j = 0; j < n_tiles; ++j) {
-        // ---- 1. the tile's chunks
+        // ---- 1. the tile's two chunks
         if (tid == 0) {
             int n_here = 0;
-            for (int cc = 0; cc < 4; ++cc) n_here += (4 * j + cc < n_chunks) ? 1 : 0;
+            for (int cc = 0; cc < 2; ++cc) n_here += (2 * j + cc < n_chunks) ? 1 : 0;
             mbar_arrive_expect_tx(bar_copy, (uint32_t)(n_here * CB));
-            for (int cc = 0; cc < 4; ++cc)
-                if (4 * j + cc < n_chunks)
-                    bulk_copy_g2s(smem_addr(raw + cc * SM::kChunkMax), chunk_ptr(p.ca, layer, b, kvh, 4 * j + cc), (uint32_t)CB, bar_copy);
+            for (int cc = 0; cc < 2; ++cc)
+                if (2 * j + cc < n_chunks)
+                    bulk_copy_g2s(smem_addr(raw + cc * SM::kChunkMax), chunk_ptr(p.ca, layer, b, kvh, 2 * j + cc), (uint32_t)CB, bar_copy);
         }
         if (!__all_sync(0xffffffffu, mbar_wait_bounded(bar_copy, copy_phase, kPaWaitNs))) { failed = true; break; }
         copy_phase ^= 1;
-        // ---- 2. this thread's key, expanded to +-1
+        // ---- 2. the keys, expanded to +-1: thread t takes half of key t / 2
         {
-            const unsigned char *ch = raw + my_cc * SM::kChunkMax;
+            const unsigned char *ch = raw + (k_key >> 5) * SM::kChunkMax;
 #pragma unroll
-            for (int w = 0; w < MB / 32; ++w) {
+            for (int ww = 0; ww < MB / 64; ++ww) {
+                const int w = k_w0 + ww;
                 uint4 lo = make_uint4(0u, 0u, 0u, 0u), hi = lo;
-                if (w < mw) expand_word(*reinterpret_cast<const uint32_t *>(ch + w * 128 + my_tt * 4), lo, hi);
-                *reinterpret_cast<uint4 *>(Ks + pa_off(tid, 2 * w)) = lo;
-                *reinterpret_cast<uint4 *>(Ks + pa_off(tid, 2 * w + 1)) = hi;
+                if (w < mw) expand_word(*reinterpret_cast<const uint32_t *>(ch + w * 128 + (k_key & 31) * 4), lo, hi);
+                *reinterpret_cast<uint4 *>(Ks + pa_off(kPaKeys, k_key, 2 * w)) = lo;
+                *reinterpret_cast<uint4 *>(Ks + pa_off(kPaKeys, k_key, 2 * w + 1)) = hi;
             }
         }
-        // ---- 3. the tile's values, dequantised once: block `vblock` of 16 tokens, code words of lanes 2 vu, 2 vu + 1
+        // ---- 3. the values, dequantised once for the 128 queries: v = code * scale + zero, split into two fp16 parts.
+        // The four lanes 4 vr .. 4 vr + 3 of a 16-token block hold, in word i, all 16 tokens of channels 16 cb + vr and
+        // 16 cb + vr + 8: a thread turns them into whole 32-byte row pieces of the operand.
         {
-            const unsigned char *ch = raw + (vblock >> 1) * SM::kChunkMax;
-            const int vb = vblock & 1;
-            const int VAL = mw * 128, ZERO = VAL + 2048, SCALE = ZERO + 64 * NG;
+            const unsigned char *ch = raw + (vt >> 1) * SM::kChunkMax;
+            const int vb = vt & 1;
+            uint2 wj[4];                                        // words 2 vi, 2 vi + 1 of the four lanes
 #pragma unroll
-            for (int hl = 0; hl < 4; ++hl) {                    // (64-channel half, lane of the pair)
-                const int half = hl >> 1, l = 2 * vu + (hl & 1), r = l >> 2, jj = l & 3;
-                const uint4 wq = *reinterpret_cast<const uint4 *>(ch + VAL + vb * 1024 + half * 512 + l * 16);
-                const uint32_t wv[4] = {wq.x, wq.y, wq.z, wq.w};
-                const int t0 = 2 * jj;                          // tokens t0, t0 + 1, t0 + 8, t0 + 9 of the block
+            for (int jj = 0; jj < 4; ++jj)
+                wj[jj] = *reinterpret_cast<const uint2 *>(ch + VAL + vb * 1024 + vh * 512 + (4 * vr + jj) * 16 + vi * 8);
+            float sc[16], zr[16];                               // scale and zero of the block's 16 tokens for this group
+            {
+                const uint4 s0 = *reinterpret_cast<const uint4 *>(ch + SCALE + vb * (32 * NG) + vg * 32);
+                const uint4 s1 = *reinterpret_cast<const uint4 *>(ch + SCALE + vb * (32 * NG) + vg * 32 + 16);
+                const uint32_t sw[8] = {s0.x, s0.y, s0.z, s0.w, s1.x, s1.y, s1.z, s1.w};
 #pragma unroll
-                for (int i = 0; i < 4; ++i) {
-                    const int cb = half * 4 + i, g = NG == 4 ? (cb >> 1) : 0;
-                    // scale and zero of the four tokens for this channel block's group
-                    const float2 d01 = half2_bits_to_float2(*reinterpret_cast<const uint32_t *>(ch + SCALE + vb * (32 * NG) + g * 32 + t0 * 2));
-                    const float2 d89 = half2_bits_to_float2(*reinterpret_cast<const uint32_t *>(ch + SCALE + vb * (32 * NG) + g * 32 + (t0 + 8) * 2));
-                    const int tk = vb * 16 + t0;                // token within the chunk
-                    const float z0 = __half2float(*reinterpret_cast<const __half *>(ch + ZERO + tk * (2 * NG) + g * 2));
-                    const float z1 = __half2float(*reinterpret_cast<const __half *>(ch + ZERO + (tk + 1) * (2 * NG) + g * 2));
-                    const float z8 = __half2float(*reinterpret_cast<const __half *>(ch + ZERO + (tk + 8) * (2 * NG) + g * 2));
-                    const float z9 = __half2float(*reinterpret_cast<const __half *>(ch + ZERO + (tk + 9) * (2 * NG) + g * 2));
-                    const uint32_t w = wv[i];
-                    // nibbles: 0 (ch r, t0)  1 (ch r+8, t0)  2 (ch r, t0+8)  3 (ch r+8, t0+8)  4..7 the same for t0+1, t0+9
-                    const float v_r_0 = fmaf((float)(w & 15u), d01.x, z0), v_r8_0 = fmaf((float)((w >> 4) & 15u), d01.x, z0);
-                    const float v_r_8 = fmaf((float)((w >> 8) & 15u), d89.x, z8), v_r8_8 = fmaf((float)((w >> 12) & 15u), d89.x, z8);
-                    const float v_r_1 = fmaf((float)((w >> 16) & 15u), d01.y, z1), v_r8_1 = fmaf((float)((w >> 20) & 15u), d01.y, z1);
-                    const float v_r_9 = fmaf((float)((w >> 24) & 15u), d89.y, z9), v_r8_9 = fmaf((float)(w >> 28), d89.y, z9);
-                    const int key0 = vblock * 16 + t0;          // key index within the tile of token t0
-                    const int ch_r = cb * 16 + r;
-                    auto put = [&](int chn, int key, float a, float bq) {
-                        const uint32_t hi = pack_f16x2(a, bq);
-                        const float2 hf = half2_bits_to_float2(hi);
-                        const uint32_t lo = pack_f16x2((a - hf.x) * 2048.f, (bq - hf.y) * 2048.f);
-                        const int off = pa_off(chn, key >> 3) + (key & 7) * 2;
-                        *reinterpret_cast<uint32_t *>(Vs + off) = hi;
-                        *reinterpret_cast<uint32_t *>(Vs + kPaTile * kPaTile * 2 + off) = lo;
-                    };
-                    put(ch_r, key0, v_r_0, v_r_1);
-                    put(ch_r, key0 + 8, v_r_8, v_r_9);
-                    put(ch_r + 8, key0, v_r8_0, v_r8_1);
-                    put(ch_r + 8, key0 + 8, v_r8_8, v_r8_9);
+                for (int k = 0; k < 8; ++k) { const float2 f = half2_bits_to_float2(sw[k]); sc[2 * k] = f.x; sc[2 * k + 1] = f.y; }
+#pragma unroll
+                for (int k = 0; k < 16; ++k)
+                    zr[k] = __half2float(*reinterpret_cast<const __half *>(ch + ZERO + (vb * 16 + k) * (2 * NG) + vg * 2));
+            }
+#pragma unroll
+            for (int ii = 0; ii < 2; ++ii) {
+                const int cb = vh * 4 + vi * 2 + ii;
+#pragma unroll
+                for (int up = 0; up < 2; ++up) {                // channel 16 cb + vr (+ 8)
+                    float v[16];
+#pragma unroll
+                    for (int jj = 0; jj < 4; ++jj) {
+                        const uint32_t w = (ii ? wj[jj].y : wj[jj].x) >> (4 * up);
+                        // nibbles 0, 2, 4, 6 of the shifted word: tokens 2jj, 2jj+8, 2jj+1, 2jj+9
+                        const int t0 = 2 * jj;
+                        v[t0] = fmaf(__int_as_float(0x4B000000 | (w & 15u)) - 8388608.f, sc[t0], zr[t0]);
+                        v[t0 + 8] = fmaf(__int_as_float(0x4B000000 | ((w >> 8) & 15u)) - 8388608.f, sc[t0 + 8], zr[t0 + 8]);
+                        v[t0 + 1] = fmaf(__int_as_float(0x4B000000 | ((w >> 16) & 15u)) - 8388608.f, sc[t0 + 1], zr[t0 + 1]);
+                        v[t0 + 9] = fmaf(__int_as_float(0x4B000000 | ((w >> 24) & 15u)) - 8388608.f, sc[t0 + 9], zr[t0 + 9]);
+                    }
+                    uint32_t hi[8], lo[8];
+#pragma unroll
+                    for (int k = 0; k < 8; ++k) split2(v[2 * k], v[2 * k + 1], hi[k], lo[k]);
+                    const int chn = cb * 16 + vr + 8 * up;
+                    const int o0 = pa_off(kHeadDim, chn, vt * 2), o1 = pa_off(kHeadDim, chn, vt * 2 + 1);
+                    *reinterpret_cast<uint4 *>(Vs + o0) = make_uint4(hi[0], hi[1], hi[2], hi[3]);
+                    *reinterpret_cast<uint4 *>(Vs + o1) = make_uint4(hi[4], hi[5], hi[6], hi[7]);
+                    *reinterpret_cast<uint4 *>(Vs + SM::kV1 + o0) = make_uint4(lo[0], lo[1], lo[2], lo[3]);
+                    *reinterpret_cast<uint4 *>(Vs + SM::kV1 + o1) = make_uint4(lo[4], lo[5], lo[6], lo[7]);
                 }
             }
         }
@@ -210,104 +232,90 @@ __global__ void __launch_bounds__(kPaThreads, 1) prompt_attention_kernel(PromptP
             tc_fence_after_sync();
 #pragma unroll
             for (int ks = 0; ks < MB / 32; ++ks) {
-                const uint64_t ad = umma_desc_k_sw128(smem_addr(Qs) + (ks >> 2) * (kPaTile * 128) + (ks & 3) * 32);
-                const uint64_t bd = umma_desc_k_sw128(smem_addr(Ks) + (ks >> 2) * (kPaTile * 128) + (ks & 3) * 32);
-                umma_f8(tmem + kColS, ad, bd, idesc, ks ? 1u : 0u);
+                const uint64_t ad = umma_desc_k_sw128(smem_addr(Qs) + (ks >> 2) * (kPaRows * 128) + (ks & 3) * 32);
+                const uint64_t bd = umma_desc_k_sw128(smem_addr(Ks) + (ks >> 2) * (kPaKeys * 128) + (ks & 3) * 32);
+                umma_f8(tmem + kColS, ad, bd, idesc_s, ks ? 1u : 0u);
             }
             umma_commit(bar_mma);
         }
         if (!__all_sync(0xffffffffu, mbar_wait_bounded(bar_mma, mma_phase, kPaWaitNs))) { failed = true; break; }
         mma_phase ^= 1;
         tc_fence_after_sync();
-        // ---- 5. online softmax on the integer distances of this row
-        const int key_base = j * kPaTile;
-        int tile_min = kPaBig;
+        // ---- 5. online softmax on this row's scores
+        const int key_base = j * kPaKeys;
+        const bool masked = key_base + kPaKeys > limit_first;   // block-uniform: some row does not see the whole tile
+        uint32_t sv[2][32];
+        tmem_ld_32cols(t_lane + kColS, sv[0]);
+        tmem_ld_32cols(t_lane + kColS + 32, sv[1]);
+        if (p.dbg_scores && layer == p.dbg_layer && b == p.dbg_b && hq == p.dbg_h && valid_q) {
 #pragma unroll
-        for (int c4 = 0; c4 < 4; ++c4) {
-            uint32_t sv[32];
-            tmem_ld_32cols(t_lane + kColS + c4 * 32, sv);
-            if (p.dbg_scores && layer == p.dbg_layer && b == p.dbg_b && hq == p.dbg_h && valid_q) {
+            for (int k = 0; k < 64; ++k)
+                if (key_base + k < p.dbg_T) p.dbg_scores[(size_t)qi * p.dbg_T + key_base + k] = (int)__uint_as_float(sv[k >> 5][k & 31]);
+        }
+        const int n_on = masked ? max(0, min(kPaKeys, limit - key_base)) : kPaKeys;     // keys of the tile this row attends to
+        float tmax = -1e30f;
 #pragma unroll
-                for (int k = 0; k < 32; ++k) {
-                    const int key = key_base + c4 * 32 + k;
-                    if (key < p.dbg_T) p.dbg_scores[(size_t)qi * p.dbg_T + key] = (int)__uint_as_float(sv[k]);
-                }
-            }
-#pragma unroll
-            for (int k = 0; k < 32; ++k) {
-                const int ham = (m - (int)__uint_as_float(sv[k])) >> 1;
-                if (key_base + c4 * 32 + k < limit) tile_min = min(tile_min, ham);
-            }
+        for (int k = 0; k < 64; ++k) {
+            const float sk = __uint_as_float(sv[k >> 5][k & 31]);
+            tmax = (!masked || k < n_on) ? fmaxf(tmax, sk) : tmax;
         }
         float factor = 1.f;
-        if (tile_min < hmin) {
-            factor = hmin == kPaBig ? 0.f : ex2_approx((float)(tile_min - hmin) * p.c);
-            hmin = tile_min;
+        if (tmax > smax) {
+            factor = ex2_approx((smax - tmax) * ch2);           // 0 the first time
+            smax = tmax;
             lsum *= factor;
         }
-        // a row whose minimum moved rescales its accumulator lanes; the loads and stores are warp-wide
+        // a row whose maximum moved rescales its accumulator lanes; the loads and stores are warp-wide
         if (j > 0 && __any_sync(0xffffffffu, factor != 1.f)) {
 #pragma unroll 1
-            for (int c = 0; c < 8; ++c) {
+            for (int c = 0; c < 4; ++c) {
                 uint32_t ov[32];
-                tmem_ld_32cols(t_lane + kColO1 + c * 32, ov);
+                tmem_ld_32cols(t_lane + kColO + c * 32, ov);
 #pragma unroll
                 for (int k = 0; k < 32; ++k) ov[k] = __float_as_uint(__uint_as_float(ov[k]) * factor);
-                tmem_st_32cols(t_lane + kColO1 + c * 32, ov);
+                tmem_st_32cols(t_lane + kColO + c * 32, ov);
             }
         }
+        {
+            const float off = -smax * ch2;
 #pragma unroll
-        for (int c4 = 0; c4 < 4; ++c4) {
-            uint32_t sv[32];
-            tmem_ld_32cols(t_lane + kColS + c4 * 32, sv);
-#pragma unroll
-            for (int k8 = 0; k8 < 4; ++k8) {
+            for (int k8 = 0; k8 < 8; ++k8) {
                 float pw[8];
 #pragma unroll
                 for (int k = 0; k < 8; ++k) {
-                    const int ham = (m - (int)__uint_as_float(sv[k8 * 8 + k])) >> 1;
-                    const bool on = key_base + c4 * 32 + k8 * 8 + k < limit;
-                    pw[k] = on ? ex2_approx((float)(hmin - ham) * p.c) : 0.f;
+                    const int kk = k8 * 8 + k;
+                    const float pv = ex2_approx(fmaf(__uint_as_float(sv[kk >> 5][kk & 31]), ch2, off));
+                    pw[k] = (!masked || kk < n_on) ? pv : 0.f;
                     lsum += pw[k];
                 }
                 uint32_t hi[4], lo[4];
 #pragma unroll
-                for (int k = 0; k < 4; ++k) {
-                    hi[k] = pack_f16x2(pw[2 * k], pw[2 * k + 1]);
-                    const float2 hf = half2_bits_to_float2(hi[k]);
-                    lo[k] = pack_f16x2((pw[2 * k] - hf.x) * 2048.f, (pw[2 * k + 1] - hf.y) * 2048.f);
-                }
-                const int off = pa_off(tid, c4 * 4 + k8);
-                *reinterpret_cast<uint4 *>(Ps + off) = make_uint4(hi[0], hi[1], hi[2], hi[3]);
-                *reinterpret_cast<uint4 *>(Ps + kPaTile * kPaTile * 2 + off) = make_uint4(lo[0], lo[1], lo[2], lo[3]);
+                for (int k = 0; k < 4; ++k) split2(pw[2 * k], pw[2 * k + 1], hi[k], lo[k]);
+                const int o = pa_off(kPaRows, tid, k8);
+                *reinterpret_cast<uint4 *>(Ps + o) = make_uint4(hi[0], hi[1], hi[2], hi[3]);
+                *reinterpret_cast<uint4 *>(Ps + SM::kP1 + o) = make_uint4(lo[0], lo[1], lo[2], lo[3]);
             }
         }
         fence_proxy_async_smem();
         tc_fence_before_sync();
         __syncthreads();
-        // ---- 6. out += P V: hi x hi into O1; hi x lo and lo x hi (both carry 2^11) into O2
+        // ---- 6. out += P V = hi hi + hi lo + lo hi (exact products, fp32 sums), one accumulator
         if (tid == 0) {
             tc_fence_after_sync();
-            const uint32_t p_hi = smem_addr(Ps), p_lo = p_hi + kPaTile * kPaTile * 2;
-            const uint32_t v_hi = smem_addr(Vs), v_lo = v_hi + kPaTile * kPaTile * 2;
+            const uint32_t p_hi = smem_addr(Ps), p_lo = p_hi + SM::kP1, v_hi = smem_addr(Vs), v_lo = v_hi + SM::kV1;
 #pragma unroll
-            for (int ks = 0; ks < kPaTile / 16; ++ks) {
-                const uint32_t ko = (ks >> 2) * (kPaTile * 128) + (ks & 3) * 32;
-                umma_f16(tmem + kColO1, umma_desc_k_sw128(p_hi + ko), umma_desc_k_sw128(v_hi + ko), idesc, (j | ks) ? 1u : 0u);
-            }
+            for (int ks = 0; ks < kPaKeys / 16; ++ks)
+                umma_f16(tmem + kColO, umma_desc_k_sw128(p_hi + ks * 32), umma_desc_k_sw128(v_hi + ks * 32), idesc_o, (j | ks) ? 1u : 0u);
 #pragma unroll
-            for (int ks = 0; ks < kPaTile / 16; ++ks) {
-                const uint32_t ko = (ks >> 2) * (kPaTile * 128) + (ks & 3) * 32;
-                umma_f16(tmem + kColO2, umma_desc_k_sw128(p_hi + ko), umma_desc_k_sw128(v_lo + ko), idesc, (j | ks) ? 1u : 0u);
-            }
+            for (int ks = 0; ks < kPaKeys / 16; ++ks)
+                umma_f16(tmem + kColO, umma_desc_k_sw128(p_hi + ks * 32), umma_desc_k_sw128(v_lo + ks * 32), idesc_o, 1u);
 #pragma unroll
-            for (int ks = 0; ks < kPaTile / 16; ++ks) {
-                const uint32_t ko = (ks >> 2) * (kPaTile * 128) + (ks & 3) * 32;
-                umma_f16(tmem + kColO2, umma_desc_k_sw128(p_lo + ko), umma_desc_k_sw128(v_hi + ko), idesc, 1u);
-            }
+            for (int ks = 0; ks < kPaKeys / 16; ++ks)
+                umma_f16(tmem + kColO, umma_desc_k_sw128(p_lo + ks * 32), umma_desc_k_sw128(v_hi + ks * 32), idesc_o, 1u);
             umma_commit(bar_mma);
         }
-        // the shared-memory operands are reused by the next tile: wait for the tensor cores here
+        // the shared-memory operands are reused by the next tile: wait for the tensor cores here (the block that
+        // shares the SM fills the gap)
         if (!__all_sync(0xffffffffu, mbar_wait_bounded(bar_mma, mma_phase, kPaWaitNs))) { failed = true; break; }
         mma_phase ^= 1;
         tc_fence_after_sync();
@@ -318,31 +326,26 @@ __global__ void __launch_bounds__(kPaThreads, 1) prompt_attention_kernel(PromptP
         // work that may still be in flight gets a bounded time before the TMEM goes back
         (void)mbar_wait_bounded(bar_mma, mma_phase, 100000000ull);
     } else {
-        // ---- the row's output: (O1 + O2 2^-11) / sum of weights. The TMEM loads are warp-wide instructions: every lane
+        // ---- the row's output: accumulator / sum of weights. The TMEM loads are warp-wide instructions: every lane
         // makes them, rows past the run's end simply do not store.
         const float inv = valid_q ? 1.f / lsum : 0.f;
         float *orow = p.out + ((((size_t)ll * p.B + b) * p.Tn + (valid_q ? qi : 0)) * p.Hq + hq) * kHeadDim;
 #pragma unroll 1
         for (int c = 0; c < 4; ++c) {
-            uint32_t o1[32], o2[32];
-            tmem_ld_32cols(t_lane + kColO1 + c * 32, o1);
-            tmem_ld_32cols(t_lane + kColO2 + c * 32, o2);
+            uint32_t o1[32];
+            tmem_ld_32cols(t_lane + kColO + c * 32, o1);
             if (valid_q) {
 #pragma unroll
-                for (int k = 0; k < 32; k += 4) {
-                    float4 v;
-                    v.x = fmaf(__uint_as_float(o2[k]), 1.f / 2048.f, __uint_as_float(o1[k])) * inv;
-                    v.y = fmaf(__uint_as_float(o2[k + 1]), 1.f / 2048.f, __uint_as_float(o1[k + 1])) * inv;
-                    v.z = fmaf(__uint_as_float(o2[k + 2]), 1.f / 2048.f, __uint_as_float(o1[k + 2])) * inv;
-                    v.w = fmaf(__uint_as_float(o2[k + 3]), 1.f / 2048.f, __uint_as_float(o1[k + 3])) * inv;
-                    *reinterpret_cast<float4 *>(orow + c * 32 + k) = v;
-                }
+                for (int k = 0; k < 32; k += 4)
+                    *reinterpret_cast<float4 *>(orow + c * 32 + k) =
+                        make_float4(__uint_as_float(o1[k]) * inv, __uint_as_float(o1[k + 1]) * inv,
+                                    __uint_as_float(o1[k + 2]) * inv, __uint_as_float(o1[k + 3]) * inv);
             }
         }
     }
     tc_fence_before_sync();
     __syncthreads();
-    if (warp == 0) { tc_fence_after_sync(); tmem_dealloc(tmem, 512); }
+    if (warp == 0) { tc_fence_after_sync(); tmem_dealloc(tmem, 256); }
 }
 
 // ---------------------------------------------------------------------------------------------------------------
@@ -363,7 +366,7 @@ static cudaError_t launch_prompt_t(const PromptParams &p, cudaStream_t st, bool 
         }
     }
     if (attributes_only) return cudaSuccess;
-    const long blocks = (long)p.n_layers * p.B * p.Hq * ((p.Tn + kPaTile - 1) / kPaTile);
+    const long blocks = (long)p.n_layers * p.B * p.Hq * ((p.Tn + kPaRows - 1) / kPaRows);
     if (blocks <= 0 || blocks > 0x7fffffffL) return cudaErrorInvalidConfiguration;
     prompt_attention_kernel<MB, NG><<<(unsigned)blocks, kPaThreads, SM::kTotal, st>>>(p);
     return cudaGetLastError();
