@@ -606,6 +606,7 @@ int h1b_append_kv(h1b_ctx *ctx, int layer_begin, int n_layers, const void *k, co
         int tpb = std::min(tiles, 32);
         while (tpb > 4 && slabs * ((tiles + tpb - 1) / tpb) < 148 * 4) tpb = (tpb + 1) / 2;
         pp.tiles_per_block = tpb;
+        pp.heads_per_item = ctx->cfg.n_kv_heads;
         H1B_CUDA(ctx, launch_prefill(pp, nn, static_cast<cudaStream_t>(stream), ctx->side, ctx->fork, ctx->join, &launches));
     } else {
         const AppendParams ap = append_params(ctx, layer_begin, n_layers, k, v, B, Tn);

@@ -854,7 +854,10 @@ __global__ void __launch_bounds__(kTmaThreads, 1) prefill_tma_kernel(const __gri
     // A work item is ONE tile of 128 cache positions of one (layer, sequence) across ALL its KV heads (the item's tiles
     // are the heads): a block then reads whole contiguous [Hkv][128] token rows of the input, 128 of them in a row,
     // whatever the other blocks are doing at that moment.
-    const long n_work = (long)p.n_layers * p.B * p.tiles_per_seq * col_blocks;
+    // (few position tiles, e.g. one layer at a time: the heads of a tile are dealt out over several items, so that
+    // every SM still has work)
+    const int head_groups = (p.Hkv + p.heads_per_item - 1) / p.heads_per_item;
+    const long n_work = (long)p.n_layers * p.B * p.tiles_per_seq * col_blocks * head_groups;
     const uint32_t full0 = smem_addr(&bars[0]), empty0 = full0 + 8 * kKeyStages;
     const uint32_t accf0 = empty0 + 8 * kKeyStages, acce0 = accf0 + 16, rfull = acce0 + 16;
 
@@ -875,9 +878,12 @@ __global__ void __launch_bounds__(kTmaThreads, 1) prefill_tma_kernel(const __gri
     const uint32_t tmem_d = skip_all ? 0u : tmem_base_s;
 
     // one work item: (slab, run of tiles, block of sketch columns), the same for every role
-    struct Item { int b, ll, layer, col0, first_tile, n_tiles, len0, n_new; };
+    struct Item { int b, ll, layer, col0, first_tile, n_tiles, len0, n_new, kvh0; };
     auto item_of = [&](long work) {
         Item it;
+        const int hgi = (int)(work % head_groups);
+        work /= head_groups;
+        it.kvh0 = hgi * p.heads_per_item;
         const int cbk = (int)(work % col_blocks);
         const int pt = (int)((work / col_blocks) % p.tiles_per_seq);
         const long seq_local = work / ((long)col_blocks * p.tiles_per_seq);
@@ -886,7 +892,7 @@ __global__ void __launch_bounds__(kTmaThreads, 1) prefill_tma_kernel(const __gri
         it.len0 = p.len[it.layer * p.max_batch + it.b];
         it.n_new = (it.len0 + nn.v[it.b] <= p.seq_cap[it.b]) ? nn.v[it.b] : 0;
         it.first_tile = it.len0 / kPrefillTile + pt;
-        it.n_tiles = (it.first_tile * kPrefillTile < it.len0 + it.n_new) ? p.Hkv : 0;   // one tile per KV head
+        it.n_tiles = (it.first_tile * kPrefillTile < it.len0 + it.n_new) ? min(p.heads_per_item, p.Hkv - it.kvh0) : 0;   // one tile per KV head
         it.col0 = cbk * NBC;
         return it;
     };
@@ -926,8 +932,8 @@ __global__ void __launch_bounds__(kTmaThreads, 1) prefill_tma_kernel(const __gri
                     const int zrow = (it.ll * p.B + it.b) * p.Tn + it.first_tile * kPrefillTile - it.len0;
                     const uint32_t dst = smem_addr(As0 + s * SM::kABytes);
                     mbar_arrive_expect_tx(full0 + 8 * s, SM::kABytes);
-                    tma_load_3d(dst, &kmap, 0, ti, zrow, full0 + 8 * s);
-                    tma_load_3d(dst + SM::kABytes / 2, &kmap, 64, ti, zrow, full0 + 8 * s);
+                    tma_load_3d(dst, &kmap, 0, it.kvh0 + ti, zrow, full0 + 8 * s);
+                    tma_load_3d(dst + SM::kABytes / 2, &kmap, 64, it.kvh0 + ti, zrow, full0 + 8 * s);
                 }
             }
             failed = __any_sync(0xffffffffu, failed);
@@ -984,7 +990,7 @@ __global__ void __launch_bounds__(kTmaThreads, 1) prefill_tma_kernel(const __gri
                 tc_fence_after_sync();
                 const int P0 = it.first_tile * kPrefillTile;
                 const int tn = P0 + quarter * 32 + lane - it.len0;
-                unsigned char *chunk = chunk_ptr(p.ca, it.layer, it.b, ti, (P0 >> 5) + quarter);   // this warp's 32 rows = one chunk of head ti
+                unsigned char *chunk = chunk_ptr(p.ca, it.layer, it.b, it.kvh0 + ti, (P0 >> 5) + quarter);   // this warp's 32 rows = one chunk of that head
 #pragma unroll
                 for (int w = w_first; w < NBC / 32; w += 2) {
                     uint32_t y[32], y2[32];
@@ -1955,8 +1961,15 @@ cudaError_t launch_prefill(const PrefillParams &p_in, const NewCounts &nn, cudaS
     cudaError_t e = sm_count(&n_sm);
     if (e != cudaSuccess) return e;
     const bool tma_path = H1B_PREFILL_TMA && !p.rope.table;
-    const long kwork = tma_path ? (long)p.n_layers * p.B * p.tiles_per_seq * ((p.m_words * 32 + nbc - 1) / nbc)
-                                : prefill_key_blocks(p, nbc);
+    long kwork = prefill_key_blocks(p, nbc);
+    if (tma_path) {
+        const long tiles = (long)p.n_layers * p.B * p.tiles_per_seq * ((p.m_words * 32 + nbc - 1) / nbc);
+        // all heads of a position tile in one item when there are tiles enough; else fewer heads per item, so that there
+        // are about two items per SM
+        p.heads_per_item = p.Hkv;
+        if (tiles < 2L * n_sm) p.heads_per_item = (int)std::max<long>(1, std::min<long>(p.Hkv, (long)p.Hkv * tiles / (2L * n_sm)));
+        kwork = tiles * ((p.Hkv + p.heads_per_item - 1) / p.heads_per_item);
+    }
     const long kblocks = kwork < n_sm ? kwork : n_sm;
     if (vblocks <= 0 || kblocks <= 0 || vblocks + kblocks > 0x7fffffffL) return cudaErrorInvalidConfiguration;
     const bool forked = side && fork && join;

@@ -156,6 +156,7 @@ struct PrefillParams {          // long appends: tensor-core projection
     int layer_begin, n_layers, B, Tn, Hkv, max_batch, m_words, groups;
     int tiles_per_seq;          // 128-position tiles that can overlap the appended range of a sequence
     int tiles_per_block;        // consecutive tiles handled by one block (the projection is loaded once per block)
+    int heads_per_item;         // role-split key kernel: KV heads of one position tile that form a work item
     RopeRef rope;
 };
 
