@@ -61,10 +61,10 @@ __device__ __forceinline__ void expand_word(uint32_t w, uint4 &lo, uint4 &hi) {
 }
 
 // Two fp32 numbers -> their fp16 parts: hi = fp16(x), lo = fp16(x - hi), x = hi + lo to 2^-22 relative (2^-25 absolute)
-__device__ __forceinline__ void split2(float a, float b, uint32_t &hi, uint32_t &lo) {
-    hi = pack_f16x2(a, b);
-    const float2 hf = half2_bits_to_float2(hi);
-    lo = pack_f16x2(a - hf.x, b - hf.y);
+__device__ __forceinline__ void split2(float2 ab, uint32_t &hi, uint32_t &lo) {
+    hi = pack_f16x2(ab.x, ab.y);
+    const float2 r = __ffma2_rn(half2_bits_to_float2(hi), make_float2(-1.f, -1.f), ab);     // ab - hi, two at a time, exact
+    lo = pack_f16x2(r.x, r.y);
 }
 
 }  // namespace
@@ -185,36 +185,36 @@ __global__ void __launch_bounds__(kPaThreads, MB == 128 ? 2 : 1) prompt_attentio
 #pragma unroll
             for (int jj = 0; jj < 4; ++jj)
                 wj[jj] = *reinterpret_cast<const uint2 *>(ch + VAL + vb * 1024 + vh * 512 + (4 * vr + jj) * 16 + vi * 8);
-            float sc[16], zr[16];                               // scale and zero of the block's 16 tokens for this group
+            float2 sc[8], zr[8];                                // scale and zero of the block's 16 tokens for this group, in pairs
             {
                 const uint4 s0 = *reinterpret_cast<const uint4 *>(ch + SCALE + vb * (32 * NG) + vg * 32);
                 const uint4 s1 = *reinterpret_cast<const uint4 *>(ch + SCALE + vb * (32 * NG) + vg * 32 + 16);
                 const uint32_t sw[8] = {s0.x, s0.y, s0.z, s0.w, s1.x, s1.y, s1.z, s1.w};
 #pragma unroll
-                for (int k = 0; k < 8; ++k) { const float2 f = half2_bits_to_float2(sw[k]); sc[2 * k] = f.x; sc[2 * k + 1] = f.y; }
-#pragma unroll
-                for (int k = 0; k < 16; ++k)
-                    zr[k] = __half2float(*reinterpret_cast<const __half *>(ch + ZERO + (vb * 16 + k) * (2 * NG) + vg * 2));
+                for (int k = 0; k < 8; ++k) {
+                    sc[k] = half2_bits_to_float2(sw[k]);
+                    zr[k].x = __half2float(*reinterpret_cast<const __half *>(ch + ZERO + (vb * 16 + 2 * k) * (2 * NG) + vg * 2));
+                    zr[k].y = __half2float(*reinterpret_cast<const __half *>(ch + ZERO + (vb * 16 + 2 * k + 1) * (2 * NG) + vg * 2));
+                }
             }
+            const float2 unbias = make_float2(-8388608.f, -8388608.f);      // (0x4B000000 | code) as a float is 2^23 + code
 #pragma unroll
             for (int ii = 0; ii < 2; ++ii) {
                 const int cb = vh * 4 + vi * 2 + ii;
 #pragma unroll
                 for (int up = 0; up < 2; ++up) {                // channel 16 cb + vr (+ 8)
-                    float v[16];
+                    uint32_t hi[8], lo[8];
 #pragma unroll
                     for (int jj = 0; jj < 4; ++jj) {
                         const uint32_t w = (ii ? wj[jj].y : wj[jj].x) >> (4 * up);
-                        // nibbles 0, 2, 4, 6 of the shifted word: tokens 2jj, 2jj+8, 2jj+1, 2jj+9
-                        const int t0 = 2 * jj;
-                        v[t0] = fmaf(__int_as_float(0x4B000000 | (w & 15u)) - 8388608.f, sc[t0], zr[t0]);
-                        v[t0 + 8] = fmaf(__int_as_float(0x4B000000 | ((w >> 8) & 15u)) - 8388608.f, sc[t0 + 8], zr[t0 + 8]);
-                        v[t0 + 1] = fmaf(__int_as_float(0x4B000000 | ((w >> 16) & 15u)) - 8388608.f, sc[t0 + 1], zr[t0 + 1]);
-                        v[t0 + 9] = fmaf(__int_as_float(0x4B000000 | ((w >> 24) & 15u)) - 8388608.f, sc[t0 + 9], zr[t0 + 9]);
+                        // nibbles 0, 4 of the shifted word: tokens 2jj, 2jj+1; nibbles 2, 6: tokens 2jj+8, 2jj+9
+                        const float2 c01 = __fadd2_rn(make_float2(__int_as_float(0x4B000000 | (w & 15u)),
+                                                                  __int_as_float(0x4B000000 | ((w >> 16) & 15u))), unbias);
+                        const float2 c89 = __fadd2_rn(make_float2(__int_as_float(0x4B000000 | ((w >> 8) & 15u)),
+                                                                  __int_as_float(0x4B000000 | ((w >> 24) & 15u))), unbias);
+                        split2(__ffma2_rn(c01, sc[jj], zr[jj]), hi[jj], lo[jj]);                 // v = code * scale + zero
+                        split2(__ffma2_rn(c89, sc[jj + 4], zr[jj + 4]), hi[jj + 4], lo[jj + 4]);
                     }
-                    uint32_t hi[8], lo[8];
-#pragma unroll
-                    for (int k = 0; k < 8; ++k) split2(v[2 * k], v[2 * k + 1], hi[k], lo[k]);
                     const int chn = cb * 16 + vr + 8 * up;
                     const int o0 = pa_off(kHeadDim, chn, vt * 2), o1 = pa_off(kHeadDim, chn, vt * 2 + 1);
                     *reinterpret_cast<uint4 *>(Vs + o0) = make_uint4(hi[0], hi[1], hi[2], hi[3]);
@@ -277,24 +277,26 @@ __global__ void __launch_bounds__(kPaThreads, MB == 128 ? 2 : 1) prompt_attentio
             }
         }
         {
-            const float off = -smax * ch2;
+            const float2 ch22 = make_float2(ch2, ch2), off2 = make_float2(-smax * ch2, -smax * ch2);
+            float2 ls2 = make_float2(0.f, 0.f);
 #pragma unroll
             for (int k8 = 0; k8 < 8; ++k8) {
-                float pw[8];
-#pragma unroll
-                for (int k = 0; k < 8; ++k) {
-                    const int kk = k8 * 8 + k;
-                    const float pv = ex2_approx(fmaf(__uint_as_float(sv[kk >> 5][kk & 31]), ch2, off));
-                    pw[k] = (!masked || kk < n_on) ? pv : 0.f;
-                    lsum += pw[k];
-                }
                 uint32_t hi[4], lo[4];
 #pragma unroll
-                for (int k = 0; k < 4; ++k) split2(pw[2 * k], pw[2 * k + 1], hi[k], lo[k]);
+                for (int k = 0; k < 4; ++k) {
+                    const int kk = k8 * 8 + 2 * k;
+                    const float2 arg = __ffma2_rn(make_float2(__uint_as_float(sv[kk >> 5][kk & 31]), __uint_as_float(sv[kk >> 5][(kk & 31) + 1])),
+                                                  ch22, off2);
+                    float2 pw = make_float2(ex2_approx(arg.x), ex2_approx(arg.y));
+                    if (masked) { pw.x = kk < n_on ? pw.x : 0.f; pw.y = kk + 1 < n_on ? pw.y : 0.f; }
+                    ls2 = __fadd2_rn(ls2, pw);
+                    split2(pw, hi[k], lo[k]);
+                }
                 const int o = pa_off(kPaRows, tid, k8);
                 *reinterpret_cast<uint4 *>(Ps + o) = make_uint4(hi[0], hi[1], hi[2], hi[3]);
                 *reinterpret_cast<uint4 *>(Ps + SM::kP1 + o) = make_uint4(lo[0], lo[1], lo[2], lo[3]);
             }
+            lsum += ls2.x + ls2.y;
         }
         fence_proxy_async_smem();
         tc_fence_before_sync();
