@@ -42,7 +42,8 @@ struct PaSmem {
     static constexpr int kP1 = kPaRows * kPaKeys * 2;           // one part of the weights, [128 queries][64 tokens] fp16
     static constexpr int kV1 = kHeadDim * kPaKeys * 2;          // one part of the values, [128 channels][64 tokens] fp16
     static constexpr int kChunkMax = (MB / 32) * 128 + 2048 + 128 * NG;
-    static constexpr int kRaw = 2 * kChunkMax;
+    static constexpr int kRaw1 = 2 * kChunkMax;                // the two chunks of one tile
+    static constexpr int kRaw = 2 * kRaw1;                      // two tiles: the next one is requested while this one is worked on
     static constexpr int kQOff = 0, kKOff = kQ, kPOff = kKOff + kK, kVOff = kPOff + 2 * kP1, kRawOff = kVOff + 2 * kV1;
     static constexpr int kTotal = kRawOff + kRaw + 1024;        // + slack to align the operands to 1024 B
 };
@@ -78,7 +79,7 @@ __global__ void __launch_bounds__(kPaThreads, MB == 128 ? 2 : 1) prompt_attentio
     unsigned char *Qs = smem + SM::kQOff, *Ks = smem + SM::kKOff, *Ps = smem + SM::kPOff, *Vs = smem + SM::kVOff;
     unsigned char *raw = smem + SM::kRawOff;
     __shared__ uint32_t tmem_base_s;
-    __shared__ __align__(8) unsigned long long bars[2];         // [0] chunk copies, [1] tensor-core work
+    __shared__ __align__(8) unsigned long long bars[3];         // [0], [1] chunk copies of even / odd tiles, [2] tensor-core work
     __shared__ int gave_up;
     const int tid = threadIdx.x, lane = tid & 31, warp = tid >> 5;
     const int mw = p.m_words;
@@ -103,10 +104,11 @@ __global__ void __launch_bounds__(kPaThreads, MB == 128 ? 2 : 1) prompt_attentio
     const int n_tiles = limit_blk > 0 ? (limit_blk + kPaKeys - 1) / kPaKeys : 0;
     const int n_chunks = (len + 31) >> 5;
 
-    const uint32_t bar_copy = smem_addr(&bars[0]), bar_mma = smem_addr(&bars[1]);
+    const uint32_t bar_copy = smem_addr(&bars[0]), bar_mma = smem_addr(&bars[2]);
     if (tid == 0) {
         gave_up = (*reinterpret_cast<volatile const int32_t *>(p.status) != kStatusOk);
         mbar_init(bar_copy, 1);
+        mbar_init(bar_copy + 8, 1);
         mbar_init(bar_mma, 1);
         mbar_fence_init();
     }
@@ -140,7 +142,7 @@ __global__ void __launch_bounds__(kPaThreads, MB == 128 ? 2 : 1) prompt_attentio
     // the running maximum score and p = 2^((S - Smax) c / 2)
     const float ch2 = 0.5f * p.c;
     float smax = -1e30f, lsum = 0.f;
-    uint32_t copy_phase = 0, mma_phase = 0;
+    uint32_t mma_phase = 0;
     bool failed = false;
     const uint32_t idesc_s = umma_idesc_f16_m128(kPaKeys), idesc_o = umma_idesc_f16_m128(kHeadDim);
     // this thread's share of the tile's keys: half a key (MB / 64 words of it)
@@ -151,21 +153,28 @@ __global__ void __launch_bounds__(kPaThreads, MB == 128 ? 2 : 1) prompt_attentio
     const int VAL = mw * 128, ZERO = VAL + 2048, SCALE = ZERO + 64 * NG;
     const int vg = NG == 4 ? vh * 2 + vi : 0;                   // the value group of this thread's channels
 
+    // tile j's chunks land in raw buffer j % 2; they are requested one tile ahead (every thread is past the buffer's
+    // previous use by then: a block-wide barrier lies between)
+    auto request_tile = [&](int j) {
+        const uint32_t bar = bar_copy + 8 * (j & 1);
+        int n_here = 0;
+        for (int cc = 0; cc < 2; ++cc) n_here += (2 * j + cc < n_chunks) ? 1 : 0;
+        mbar_arrive_expect_tx(bar, (uint32_t)(n_here * CB));
+        for (int cc = 0; cc < 2; ++cc)
+            if (2 * j + cc < n_chunks)
+                bulk_copy_g2s(smem_addr(raw + (j & 1) * SM::kRaw1 + cc * SM::kChunkMax), chunk_ptr(p.ca, layer, b, kvh, 2 * j + cc),
+                              (uint32_t)CB, bar);
+    };
+    if (tid == 0) request_tile(0);
+    bool pv_pending = false;                                    // the previous tile's P.V contractions have not been waited for yet
     for (int j = 0; j < n_tiles; ++j) {
-        // ---- 1. the tile's two chunks
-        if (tid == 0) {
-            int n_here = 0;
-            for (int cc = 0; cc < 2; ++cc) n_here += (2 * j + cc < n_chunks) ? 1 : 0;
-            mbar_arrive_expect_tx(bar_copy, (uint32_t)(n_here * CB));
-            for (int cc = 0; cc < 2; ++cc)
-                if (2 * j + cc < n_chunks)
-                    bulk_copy_g2s(smem_addr(raw + cc * SM::kChunkMax), chunk_ptr(p.ca, layer, b, kvh, 2 * j + cc), (uint32_t)CB, bar_copy);
-        }
-        if (!__all_sync(0xffffffffu, mbar_wait_bounded(bar_copy, copy_phase, kPaWaitNs))) { failed = true; break; }
-        copy_phase ^= 1;
+        // ---- 1. the tile's two chunks (requested during the previous tile); the next tile's are requested now
+        if (!__all_sync(0xffffffffu, mbar_wait_bounded(bar_copy + 8 * (j & 1), (uint32_t)((j >> 1) & 1), kPaWaitNs))) { failed = true; break; }
+        if (tid == 0 && j + 1 < n_tiles) request_tile(j + 1);
+        const unsigned char *rawj = raw + (j & 1) * SM::kRaw1;
         // ---- 2. the keys, expanded to +-1: thread t takes half of key t / 2
         {
-            const unsigned char *ch = raw + (k_key >> 5) * SM::kChunkMax;
+            const unsigned char *ch = rawj + (k_key >> 5) * SM::kChunkMax;
 #pragma unroll
             for (int ww = 0; ww < MB / 64; ++ww) {
                 const int w = k_w0 + ww;
@@ -175,11 +184,19 @@ __global__ void __launch_bounds__(kPaThreads, MB == 128 ? 2 : 1) prompt_attentio
                 *reinterpret_cast<uint4 *>(Ks + pa_off(kPaKeys, k_key, 2 * w + 1)) = hi;
             }
         }
+        // (the previous tile's P.V contractions read the value and weight operands: they must be done before those are
+        // rewritten; the key expansion above ran beside them)
+        if (pv_pending) {
+            if (!__all_sync(0xffffffffu, mbar_wait_bounded(bar_mma, mma_phase, kPaWaitNs))) { failed = true; break; }
+            mma_phase ^= 1;
+            tc_fence_after_sync();
+            pv_pending = false;
+        }
         // ---- 3. the values, dequantised once for the 128 queries: v = code * scale + zero, split into two fp16 parts.
         // The four lanes 4 vr .. 4 vr + 3 of a 16-token block hold, in word i, all 16 tokens of channels 16 cb + vr and
         // 16 cb + vr + 8: a thread turns them into whole 32-byte row pieces of the operand.
         {
-            const unsigned char *ch = raw + (vt >> 1) * SM::kChunkMax;
+            const unsigned char *ch = rawj + (vt >> 1) * SM::kChunkMax;
             const int vb = vt & 1;
             uint2 wj[4];                                        // words 2 vi, 2 vi + 1 of the four lanes
 #pragma unroll
@@ -316,9 +333,10 @@ __global__ void __launch_bounds__(kPaThreads, MB == 128 ? 2 : 1) prompt_attentio
                 umma_f16(tmem + kColO, umma_desc_k_sw128(p_lo + ks * 32), umma_desc_k_sw128(v_hi + ks * 32), idesc_o, 1u);
             umma_commit(bar_mma);
         }
-        // the shared-memory operands are reused by the next tile: wait for the tensor cores here (the block that
-        // shares the SM fills the gap)
-        if (!__all_sync(0xffffffffu, mbar_wait_bounded(bar_mma, mma_phase, kPaWaitNs))) { failed = true; break; }
+        pv_pending = true;                                      // waited for before the operands are rewritten, or after the loop
+    }
+    if (!failed && pv_pending) {
+        if (!__all_sync(0xffffffffu, mbar_wait_bounded(bar_mma, mma_phase, kPaWaitNs))) failed = true;
         mma_phase ^= 1;
         tc_fence_after_sync();
     }

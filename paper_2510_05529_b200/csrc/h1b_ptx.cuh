@@ -35,6 +35,9 @@ __device__ __forceinline__ bool mbar_try_wait(uint32_t bar, uint32_t parity) {
         : "=r"(ok) : "r"(bar), "r"(parity) : "memory");
     return ok != 0;
 }
+#ifndef H1B_WAIT_PARK_NS
+#define H1B_WAIT_PARK_NS 2000
+#endif
 __device__ __forceinline__ unsigned long long global_timer_ns() {
     unsigned long long t;
     asm volatile("mov.u64 %0, %%globaltimer;" : "=l"(t));
@@ -43,13 +46,24 @@ __device__ __forceinline__ unsigned long long global_timer_ns() {
 // Wait for a phase of an mbarrier, for at most `limit_ns`. Returns false when
 // the limit ran out (the caller records an error and leaves; nothing spins
 // forever).
+// The same probe with a suspend-time hint: the hardware may park the thread for up to about `hint_ns` while the phase is
+// incomplete, instead of returning at once, so a waiting warp does not take issue slots from the warps that work.
+__device__ __forceinline__ bool mbar_try_wait_parked(uint32_t bar, uint32_t parity, uint32_t hint_ns) {
+    uint32_t ok;
+    asm volatile(
+        "{\n\t.reg .pred p;\n\t"
+        "mbarrier.try_wait.parity.shared::cta.b64 p, [%1], %2, %3;\n\t"
+        "selp.u32 %0, 1, 0, p;\n\t}"
+        : "=r"(ok) : "r"(bar), "r"(parity), "r"(hint_ns) : "memory");
+    return ok != 0;
+}
 __device__ __forceinline__ bool mbar_wait_bounded(uint32_t bar, uint32_t parity, unsigned long long limit_ns) {
     if (mbar_try_wait(bar, parity)) return true;
     const unsigned long long t0 = global_timer_ns();
     for (;;) {
 #pragma unroll 1
-        for (int i = 0; i < 64; ++i)
-            if (mbar_try_wait(bar, parity)) return true;
+        for (int i = 0; i < 16; ++i)
+            if (mbar_try_wait_parked(bar, parity, H1B_WAIT_PARK_NS)) return true;
         if (global_timer_ns() - t0 > limit_ns) return false;
     }
 }
