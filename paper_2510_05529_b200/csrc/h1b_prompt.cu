@@ -29,6 +29,7 @@ constexpr int kPaThreads = 128;
 constexpr int kPaRows = 128;                       // query rows per block
 constexpr int kPaKeys = 64;                        // cached tokens per tile (two 32-token chunks)
 constexpr unsigned long long kPaWaitNs = 2000000000ull;
+constexpr float kPaLazy = 8.f;                     // weights stay below 2^8 (fp16 operands, fp32 sums: far from any limit)
 
 // Byte offset of the 16-byte piece `c16` of row `row` in a K-major operand tile of `rows` rows: column blocks of 128
 // bytes, each [rows][128 B] with the 128-byte swizzle.
@@ -43,8 +44,9 @@ struct PaSmem {
     static constexpr int kV1 = kHeadDim * kPaKeys * 2;          // one part of the values, [128 channels][64 tokens] fp16
     static constexpr int kChunkMax = (MB / 32) * 128 + 2048 + 128 * NG;
     static constexpr int kRaw1 = 2 * kChunkMax;                // the two chunks of one tile
-    static constexpr int kRaw = 2 * kRaw1;                      // two tiles: the next one is requested while this one is worked on
-    static constexpr int kQOff = 0, kKOff = kQ, kPOff = kKOff + kK, kVOff = kPOff + 2 * kP1, kRawOff = kVOff + 2 * kV1;
+    static constexpr int kRaw = 2 * kRaw1;                      // two tiles: tile j + 2 is requested once tile j's values are out
+    // (two key operands: the scores of tile j + 1 are contracted while the threads work on tile j)
+    static constexpr int kQOff = 0, kKOff = kQ, kPOff = kKOff + 2 * kK, kVOff = kPOff + 2 * kP1, kRawOff = kVOff + 2 * kV1;
     static constexpr int kTotal = kRawOff + kRaw + 1024;        // + slack to align the operands to 1024 B
 };
 
@@ -79,7 +81,8 @@ __global__ void __launch_bounds__(kPaThreads, MB == 128 ? 2 : 1) prompt_attentio
     unsigned char *Qs = smem + SM::kQOff, *Ks = smem + SM::kKOff, *Ps = smem + SM::kPOff, *Vs = smem + SM::kVOff;
     unsigned char *raw = smem + SM::kRawOff;
     __shared__ uint32_t tmem_base_s;
-    __shared__ __align__(8) unsigned long long bars[3];         // [0], [1] chunk copies of even / odd tiles, [2] tensor-core work
+    // [0], [1] chunk copies of tile j in [j % 2]; [2] unused; [3], [4] scores of tile j in [3 + j % 2]; [5] the P.V contractions
+    __shared__ __align__(8) unsigned long long bars[6];
     __shared__ int gave_up;
     const int tid = threadIdx.x, lane = tid & 31, warp = tid >> 5;
     const int mw = p.m_words;
@@ -104,12 +107,11 @@ __global__ void __launch_bounds__(kPaThreads, MB == 128 ? 2 : 1) prompt_attentio
     const int n_tiles = limit_blk > 0 ? (limit_blk + kPaKeys - 1) / kPaKeys : 0;
     const int n_chunks = (len + 31) >> 5;
 
-    const uint32_t bar_copy = smem_addr(&bars[0]), bar_mma = smem_addr(&bars[2]);
+    const uint32_t bar_copy = smem_addr(&bars[0]), bar_s = smem_addr(&bars[3]), bar_pv = smem_addr(&bars[5]);
     if (tid == 0) {
         gave_up = (*reinterpret_cast<volatile const int32_t *>(p.status) != kStatusOk);
-        mbar_init(bar_copy, 1);
-        mbar_init(bar_copy + 8, 1);
-        mbar_init(bar_mma, 1);
+#pragma unroll
+        for (int i = 0; i < 6; ++i) mbar_init(bar_copy + 8 * i, 1);
         mbar_fence_init();
     }
     // the raw chunk buffer starts as zeros: chunks past the sequence's end are never copied, and whatever stands in
@@ -124,7 +126,7 @@ __global__ void __launch_bounds__(kPaThreads, MB == 128 ? 2 : 1) prompt_attentio
     if (skip_all) return;
     const uint32_t tmem = tmem_base_s;
     const uint32_t t_lane = tmem + ((uint32_t)(warp * 32) << 16);       // this warp's quarter of the TMEM lanes
-    constexpr uint32_t kColS = 0, kColO = 128;
+    constexpr uint32_t kColS = 0, kColO = 128;                  // scores of tile j at columns 64 (j % 2) .., the output at 128 ..
 
     // ---- this row's query sketch, expanded (rows past the run's end: whatever their words hold; never used)
     {
@@ -142,7 +144,6 @@ __global__ void __launch_bounds__(kPaThreads, MB == 128 ? 2 : 1) prompt_attentio
     // the running maximum score and p = 2^((S - Smax) c / 2)
     const float ch2 = 0.5f * p.c;
     float smax = -1e30f, lsum = 0.f;
-    uint32_t mma_phase = 0;
     bool failed = false;
     const uint32_t idesc_s = umma_idesc_f16_m128(kPaKeys), idesc_o = umma_idesc_f16_m128(kHeadDim);
     // this thread's share of the tile's keys: half a key (MB / 64 words of it)
@@ -153,8 +154,8 @@ __global__ void __launch_bounds__(kPaThreads, MB == 128 ? 2 : 1) prompt_attentio
     const int VAL = mw * 128, ZERO = VAL + 2048, SCALE = ZERO + 64 * NG;
     const int vg = NG == 4 ? vh * 2 + vi : 0;                   // the value group of this thread's channels
 
-    // tile j's chunks land in raw buffer j % 2; they are requested one tile ahead (every thread is past the buffer's
-    // previous use by then: a block-wide barrier lies between)
+    // tile j's chunks land in raw buffer j % 2; they are requested when tile j - 2 has given up the buffer (every thread
+    // is past its use by then: a block-wide barrier lies between), more than a tile before their first use
     auto request_tile = [&](int j) {
         const uint32_t bar = bar_copy + 8 * (j & 1);
         int n_here = 0;
@@ -165,32 +166,55 @@ __global__ void __launch_bounds__(kPaThreads, MB == 128 ? 2 : 1) prompt_attentio
                 bulk_copy_g2s(smem_addr(raw + (j & 1) * SM::kRaw1 + cc * SM::kChunkMax), chunk_ptr(p.ca, layer, b, kvh, 2 * j + cc),
                               (uint32_t)CB, bar);
     };
-    if (tid == 0) request_tile(0);
-    bool pv_pending = false;                                    // the previous tile's P.V contractions have not been waited for yet
-    for (int j = 0; j < n_tiles; ++j) {
-        // ---- 1. the tile's two chunks (requested during the previous tile); the next tile's are requested now
-        if (!__all_sync(0xffffffffu, mbar_wait_bounded(bar_copy + 8 * (j & 1), (uint32_t)((j >> 1) & 1), kPaWaitNs))) { failed = true; break; }
-        if (tid == 0 && j + 1 < n_tiles) request_tile(j + 1);
-        const unsigned char *rawj = raw + (j & 1) * SM::kRaw1;
-        // ---- 2. the keys, expanded to +-1: thread t takes half of key t / 2
-        {
-            const unsigned char *ch = rawj + (k_key >> 5) * SM::kChunkMax;
+    // the keys of tile j, expanded to +-1 into key operand j % 2: thread t takes half of key t / 2
+    auto expand_keys = [&](int j) {
+        const unsigned char *ch = raw + (j & 1) * SM::kRaw1 + (k_key >> 5) * SM::kChunkMax;
+        unsigned char *Kd = Ks + (j & 1) * SM::kK;
 #pragma unroll
-            for (int ww = 0; ww < MB / 64; ++ww) {
-                const int w = k_w0 + ww;
-                uint4 lo = make_uint4(0u, 0u, 0u, 0u), hi = lo;
-                if (w < mw) expand_word(*reinterpret_cast<const uint32_t *>(ch + w * 128 + (k_key & 31) * 4), lo, hi);
-                *reinterpret_cast<uint4 *>(Ks + pa_off(kPaKeys, k_key, 2 * w)) = lo;
-                *reinterpret_cast<uint4 *>(Ks + pa_off(kPaKeys, k_key, 2 * w + 1)) = hi;
-            }
+        for (int ww = 0; ww < MB / 64; ++ww) {
+            const int w = k_w0 + ww;
+            uint4 lo = make_uint4(0u, 0u, 0u, 0u), hi = lo;
+            if (w < mw) expand_word(*reinterpret_cast<const uint32_t *>(ch + w * 128 + (k_key & 31) * 4), lo, hi);
+            *reinterpret_cast<uint4 *>(Kd + pa_off(kPaKeys, k_key, 2 * w)) = lo;
+            *reinterpret_cast<uint4 *>(Kd + pa_off(kPaKeys, k_key, 2 * w + 1)) = hi;
         }
-        // (the previous tile's P.V contractions read the value and weight operands: they must be done before those are
-        // rewritten; the key expansion above ran beside them)
-        if (pv_pending) {
-            if (!__all_sync(0xffffffffu, mbar_wait_bounded(bar_mma, mma_phase, kPaWaitNs))) { failed = true; break; }
-            mma_phase ^= 1;
+    };
+    // scores of tile j: S = Q (+-1) x K^T (+-1) into score columns j % 2 (one thread issues)
+    auto issue_scores = [&](int j) {
+        tc_fence_after_sync();
+#pragma unroll
+        for (int ks = 0; ks < MB / 32; ++ks) {
+            const uint64_t ad = umma_desc_k_sw128(smem_addr(Qs) + (ks >> 2) * (kPaRows * 128) + (ks & 3) * 32);
+            const uint64_t bd = umma_desc_k_sw128(smem_addr(Ks) + (j & 1) * SM::kK + (ks >> 2) * (kPaKeys * 128) + (ks & 3) * 32);
+            umma_f8(tmem + kColS + (j & 1) * kPaKeys, ad, bd, idesc_s, ks ? 1u : 0u);
+        }
+        umma_commit(bar_s + 8 * (j & 1));
+    };
+    // The tensor cores run one tile ahead of the threads: while the threads turn tile j's scores into weights, the scores
+    // of tile j + 1 are already being contracted, and the P.V contractions of tile j run beside the key expansion of
+    // tile j + 2.
+    if (tid == 0) {
+        request_tile(0);
+        if (n_tiles > 1) request_tile(1);
+    }
+    if (!__all_sync(0xffffffffu, mbar_wait_bounded(bar_copy, 0u, kPaWaitNs))) failed = true;
+    if (!failed) expand_keys(0);
+    fence_proxy_async_smem();
+    tc_fence_before_sync();
+    __syncthreads();
+    if (tid == 0 && !failed) issue_scores(0);
+    for (int j = 0; j < n_tiles && !failed; ++j) {
+        // ---- 1. the next tile's keys (its chunks were requested during the tile before this one)
+        if (j + 1 < n_tiles) {
+            if (!__all_sync(0xffffffffu, mbar_wait_bounded(bar_copy + 8 * ((j + 1) & 1), (uint32_t)(((j + 1) >> 1) & 1), kPaWaitNs))) { failed = true; break; }
+            expand_keys(j + 1);
+        }
+        const unsigned char *rawj = raw + (j & 1) * SM::kRaw1;
+        // ---- 2. the previous tile's P.V contractions read the value and weight operands and write the accumulator:
+        // they must be done before those are touched (the key expansion above ran beside them)
+        if (j > 0) {
+            if (!__all_sync(0xffffffffu, mbar_wait_bounded(bar_pv, (uint32_t)((j - 1) & 1), kPaWaitNs))) { failed = true; break; }
             tc_fence_after_sync();
-            pv_pending = false;
         }
         // ---- 3. the values, dequantised once for the 128 queries: v = code * scale + zero, split into two fp16 parts.
         // The four lanes 4 vr .. 4 vr + 3 of a 16-token block hold, in word i, all 16 tokens of channels 16 cb + vr and
@@ -244,40 +268,42 @@ __global__ void __launch_bounds__(kPaThreads, MB == 128 ? 2 : 1) prompt_attentio
         fence_proxy_async_smem();
         tc_fence_before_sync();
         __syncthreads();
-        // ---- 4. scores: S = Q (+-1) x K^T (+-1), one thread issues
+        // ---- 4. the next tile's scores start; this tile's chunk buffer is free for the tile after the next; this
+        // tile's scores were started one tile ago
         if (tid == 0) {
-            tc_fence_after_sync();
-#pragma unroll
-            for (int ks = 0; ks < MB / 32; ++ks) {
-                const uint64_t ad = umma_desc_k_sw128(smem_addr(Qs) + (ks >> 2) * (kPaRows * 128) + (ks & 3) * 32);
-                const uint64_t bd = umma_desc_k_sw128(smem_addr(Ks) + (ks >> 2) * (kPaKeys * 128) + (ks & 3) * 32);
-                umma_f8(tmem + kColS, ad, bd, idesc_s, ks ? 1u : 0u);
-            }
-            umma_commit(bar_mma);
+            if (j + 1 < n_tiles) issue_scores(j + 1);
+            if (j + 2 < n_tiles) request_tile(j + 2);
         }
-        if (!__all_sync(0xffffffffu, mbar_wait_bounded(bar_mma, mma_phase, kPaWaitNs))) { failed = true; break; }
-        mma_phase ^= 1;
+        if (!__all_sync(0xffffffffu, mbar_wait_bounded(bar_s + 8 * (j & 1), (uint32_t)((j >> 1) & 1), kPaWaitNs))) { failed = true; break; }
         tc_fence_after_sync();
         // ---- 5. online softmax on this row's scores
         const int key_base = j * kPaKeys;
         const bool masked = key_base + kPaKeys > limit_first;   // block-uniform: some row does not see the whole tile
         uint32_t sv[2][32];
-        tmem_ld_32cols(t_lane + kColS, sv[0]);
-        tmem_ld_32cols(t_lane + kColS + 32, sv[1]);
+        tmem_ld_32cols(t_lane + kColS + (j & 1) * kPaKeys, sv[0]);
+        tmem_ld_32cols(t_lane + kColS + (j & 1) * kPaKeys + 32, sv[1]);
         if (p.dbg_scores && layer == p.dbg_layer && b == p.dbg_b && hq == p.dbg_h && valid_q) {
 #pragma unroll
             for (int k = 0; k < 64; ++k)
                 if (key_base + k < p.dbg_T) p.dbg_scores[(size_t)qi * p.dbg_T + key_base + k] = (int)__uint_as_float(sv[k >> 5][k & 31]);
         }
         const int n_on = masked ? max(0, min(kPaKeys, limit - key_base)) : kPaKeys;     // keys of the tile this row attends to
-        float tmax = -1e30f;
+        float tmax;
+        {
+            float t4[4] = {-1e30f, -1e30f, -1e30f, -1e30f};     // four chains: the maximum does not depend on the order
 #pragma unroll
-        for (int k = 0; k < 64; ++k) {
-            const float sk = __uint_as_float(sv[k >> 5][k & 31]);
-            tmax = (!masked || k < n_on) ? fmaxf(tmax, sk) : tmax;
+            for (int k = 0; k < 64; ++k) {
+                const float sk = __uint_as_float(sv[k >> 5][k & 31]);
+                t4[k & 3] = (!masked || k < n_on) ? fmaxf(t4[k & 3], sk) : t4[k & 3];
+            }
+            tmax = fmaxf(fmaxf(t4[0], t4[1]), fmaxf(t4[2], t4[3]));
         }
+        // The reference score of a row follows its maximum lazily: weights are 2^((S - reference) c / 2), and any
+        // reference gives the same quotient out = sum(p v) / sum(p); it is moved (and the row's sums rescaled) only when
+        // a score exceeds it by so much that the weights would grow past 2^kPaLazy. After the first tile that is rare,
+        // and the pass over the accumulator in TMEM is skipped.
         float factor = 1.f;
-        if (tmax > smax) {
+        if ((tmax - smax) * ch2 > kPaLazy) {
             factor = ex2_approx((smax - tmax) * ch2);           // 0 the first time
             smax = tmax;
             lsum *= factor;
@@ -331,20 +357,18 @@ __global__ void __launch_bounds__(kPaThreads, MB == 128 ? 2 : 1) prompt_attentio
 #pragma unroll
             for (int ks = 0; ks < kPaKeys / 16; ++ks)
                 umma_f16(tmem + kColO, umma_desc_k_sw128(p_lo + ks * 32), umma_desc_k_sw128(v_hi + ks * 32), idesc_o, 1u);
-            umma_commit(bar_mma);
+            umma_commit(bar_pv);                                // waited for before the operands are rewritten, or after the loop
         }
-        pv_pending = true;                                      // waited for before the operands are rewritten, or after the loop
     }
-    if (!failed && pv_pending) {
-        if (!__all_sync(0xffffffffu, mbar_wait_bounded(bar_mma, mma_phase, kPaWaitNs))) failed = true;
-        mma_phase ^= 1;
+    if (!failed) {
+        if (!__all_sync(0xffffffffu, mbar_wait_bounded(bar_pv, (uint32_t)((n_tiles - 1) & 1), kPaWaitNs))) failed = true;
         tc_fence_after_sync();
     }
 
     if (failed) {
         if (lane == 0) atomicExch(p.status, kStatusWaitTimeout);
         // work that may still be in flight gets a bounded time before the TMEM goes back
-        (void)mbar_wait_bounded(bar_mma, mma_phase, 100000000ull);
+        (void)mbar_wait_bounded(bar_pv, (uint32_t)((n_tiles - 1) & 1), 100000000ull);
     } else {
         // ---- the row's output: accumulator / sum of weights. The TMEM loads are warp-wide instructions: every lane
         // makes them, rows past the run's end simply do not store.
