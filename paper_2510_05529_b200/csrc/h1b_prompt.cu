@@ -17,6 +17,7 @@
 // When a row's running maximum moves, its accumulator lanes are rescaled in TMEM (rare after the first tiles).
 // Every wait is bounded; a block that gives up records the time-out and releases its TMEM.
 #include <mutex>
+#include <type_traits>
 
 #include "h1b_kernels.h"
 #include "h1b_ptx.cuh"
@@ -61,6 +62,13 @@ __device__ __forceinline__ void expand_word(uint32_t w, uint4 &lo, uint4 &hi) {
     }
     lo = make_uint4(o[0], o[1], o[2], o[3]);
     hi = make_uint4(o[4], o[5], o[6], o[7]);
+}
+
+// The largest of three floats in one instruction (sm_100)
+__device__ __forceinline__ float max3(float a, float b, float c) {
+    float d;
+    asm("max.f32 %0, %1, %2, %3;" : "=f"(d) : "f"(a), "f"(b), "f"(c));
+    return d;
 }
 
 // Two fp32 numbers -> their fp16 parts: hi = fp16(x), lo = fp16(x - hi), x = hi + lo to 2^-22 relative (2^-25 absolute)
@@ -233,12 +241,12 @@ __global__ void __launch_bounds__(kPaThreads, MB == 128 ? 2 : 1) prompt_attentio
                 const uint32_t sw[8] = {s0.x, s0.y, s0.z, s0.w, s1.x, s1.y, s1.z, s1.w};
 #pragma unroll
                 for (int k = 0; k < 8; ++k) {
-                    sc[k] = half2_bits_to_float2(sw[k]);
+                    // (scales times 2^24: the codes below come as code * 2^-24; powers of two, so nothing is rounded)
+                    sc[k] = __fmul2_rn(half2_bits_to_float2(sw[k]), make_float2(16777216.f, 16777216.f));
                     zr[k].x = __half2float(*reinterpret_cast<const __half *>(ch + ZERO + (vb * 16 + 2 * k) * (2 * NG) + vg * 2));
                     zr[k].y = __half2float(*reinterpret_cast<const __half *>(ch + ZERO + (vb * 16 + 2 * k + 1) * (2 * NG) + vg * 2));
                 }
             }
-            const float2 unbias = make_float2(-8388608.f, -8388608.f);      // (0x4B000000 | code) as a float is 2^23 + code
 #pragma unroll
             for (int ii = 0; ii < 2; ++ii) {
                 const int cb = vh * 4 + vi * 2 + ii;
@@ -248,11 +256,11 @@ __global__ void __launch_bounds__(kPaThreads, MB == 128 ? 2 : 1) prompt_attentio
 #pragma unroll
                     for (int jj = 0; jj < 4; ++jj) {
                         const uint32_t w = (ii ? wj[jj].y : wj[jj].x) >> (4 * up);
-                        // nibbles 0, 4 of the shifted word: tokens 2jj, 2jj+1; nibbles 2, 6: tokens 2jj+8, 2jj+9
-                        const float2 c01 = __fadd2_rn(make_float2(__int_as_float(0x4B000000 | (w & 15u)),
-                                                                  __int_as_float(0x4B000000 | ((w >> 16) & 15u))), unbias);
-                        const float2 c89 = __fadd2_rn(make_float2(__int_as_float(0x4B000000 | ((w >> 8) & 15u)),
-                                                                  __int_as_float(0x4B000000 | ((w >> 24) & 15u))), unbias);
+                        // nibbles 0, 4 of the shifted word: tokens 2jj, 2jj+1; nibbles 2, 6: tokens 2jj+8, 2jj+9. A 4-bit
+                        // code in the low bits of a 16-bit half IS the fp16 number code * 2^-24 (a subnormal): one mask
+                        // takes two codes, and the conversion to fp32 is exact
+                        const float2 c01 = half2_bits_to_float2(w & 0x000F000Fu);
+                        const float2 c89 = half2_bits_to_float2((w >> 8) & 0x000F000Fu);
                         split2(__ffma2_rn(c01, sc[jj], zr[jj]), hi[jj], lo[jj]);                 // v = code * scale + zero
                         split2(__ffma2_rn(c89, sc[jj + 4], zr[jj + 4]), hi[jj + 4], lo[jj + 4]);
                     }
@@ -287,39 +295,46 @@ __global__ void __launch_bounds__(kPaThreads, MB == 128 ? 2 : 1) prompt_attentio
             for (int k = 0; k < 64; ++k)
                 if (key_base + k < p.dbg_T) p.dbg_scores[(size_t)qi * p.dbg_T + key_base + k] = (int)__uint_as_float(sv[k >> 5][k & 31]);
         }
-        const int n_on = masked ? max(0, min(kPaKeys, limit - key_base)) : kPaKeys;     // keys of the tile this row attends to
-        float tmax;
-        {
-            float t4[4] = {-1e30f, -1e30f, -1e30f, -1e30f};     // four chains: the maximum does not depend on the order
+        // (two copies of the code: tiles that every row sees whole, by far the most, carry no causal tests at all)
+        auto softmax_tile = [&](auto masked_c) {
+            constexpr bool MASKED = decltype(masked_c)::value;
+            const int n_on = MASKED ? max(0, min(kPaKeys, limit - key_base)) : kPaKeys;     // keys of the tile this row attends to
+            float tmax;
+            {
+                float t4[4] = {-1e30f, -1e30f, -1e30f, -1e30f};     // four chains: the maximum does not depend on the order
 #pragma unroll
-            for (int k = 0; k < 64; ++k) {
-                const float sk = __uint_as_float(sv[k >> 5][k & 31]);
-                t4[k & 3] = (!masked || k < n_on) ? fmaxf(t4[k & 3], sk) : t4[k & 3];
+                for (int k = 0; k < 64; k += 2) {
+                    const float s0 = __uint_as_float(sv[k >> 5][k & 31]), s1 = __uint_as_float(sv[k >> 5][(k & 31) + 1]);
+                    if (MASKED) {
+                        t4[(k >> 1) & 3] = k < n_on ? fmaxf(t4[(k >> 1) & 3], s0) : t4[(k >> 1) & 3];
+                        t4[(k >> 1) & 3] = k + 1 < n_on ? fmaxf(t4[(k >> 1) & 3], s1) : t4[(k >> 1) & 3];
+                    } else {
+                        t4[(k >> 1) & 3] = max3(t4[(k >> 1) & 3], s0, s1);
+                    }
+                }
+                tmax = fmaxf(fmaxf(t4[0], t4[1]), fmaxf(t4[2], t4[3]));
             }
-            tmax = fmaxf(fmaxf(t4[0], t4[1]), fmaxf(t4[2], t4[3]));
-        }
-        // The reference score of a row follows its maximum lazily: weights are 2^((S - reference) c / 2), and any
-        // reference gives the same quotient out = sum(p v) / sum(p); it is moved (and the row's sums rescaled) only when
-        // a score exceeds it by so much that the weights would grow past 2^kPaLazy. After the first tile that is rare,
-        // and the pass over the accumulator in TMEM is skipped.
-        float factor = 1.f;
-        if ((tmax - smax) * ch2 > kPaLazy) {
-            factor = ex2_approx((smax - tmax) * ch2);           // 0 the first time
-            smax = tmax;
-            lsum *= factor;
-        }
-        // a row whose maximum moved rescales its accumulator lanes; the loads and stores are warp-wide
-        if (j > 0 && __any_sync(0xffffffffu, factor != 1.f)) {
+            // The reference score of a row follows its maximum lazily: weights are 2^((S - reference) c / 2), and any
+            // reference gives the same quotient out = sum(p v) / sum(p); it is moved (and the row's sums rescaled) only
+            // when a score exceeds it by so much that the weights would grow past 2^kPaLazy. After the first tile that
+            // is rare, and the pass over the accumulator in TMEM is skipped.
+            float factor = 1.f;
+            if ((tmax - smax) * ch2 > kPaLazy) {
+                factor = ex2_approx((smax - tmax) * ch2);           // 0 the first time
+                smax = tmax;
+                lsum *= factor;
+            }
+            // a row whose maximum moved rescales its accumulator lanes; the loads and stores are warp-wide
+            if (j > 0 && __any_sync(0xffffffffu, factor != 1.f)) {
 #pragma unroll 1
-            for (int c = 0; c < 4; ++c) {
-                uint32_t ov[32];
-                tmem_ld_32cols(t_lane + kColO + c * 32, ov);
+                for (int c = 0; c < 4; ++c) {
+                    uint32_t ov[32];
+                    tmem_ld_32cols(t_lane + kColO + c * 32, ov);
 #pragma unroll
-                for (int k = 0; k < 32; ++k) ov[k] = __float_as_uint(__uint_as_float(ov[k]) * factor);
-                tmem_st_32cols(t_lane + kColO + c * 32, ov);
+                    for (int k = 0; k < 32; ++k) ov[k] = __float_as_uint(__uint_as_float(ov[k]) * factor);
+                    tmem_st_32cols(t_lane + kColO + c * 32, ov);
+                }
             }
-        }
-        {
             const float2 ch22 = make_float2(ch2, ch2), off2 = make_float2(-smax * ch2, -smax * ch2);
             float2 ls2 = make_float2(0.f, 0.f);
 #pragma unroll
@@ -331,7 +346,7 @@ __global__ void __launch_bounds__(kPaThreads, MB == 128 ? 2 : 1) prompt_attentio
                     const float2 arg = __ffma2_rn(make_float2(__uint_as_float(sv[kk >> 5][kk & 31]), __uint_as_float(sv[kk >> 5][(kk & 31) + 1])),
                                                   ch22, off2);
                     float2 pw = make_float2(ex2_approx(arg.x), ex2_approx(arg.y));
-                    if (masked) { pw.x = kk < n_on ? pw.x : 0.f; pw.y = kk + 1 < n_on ? pw.y : 0.f; }
+                    if (MASKED) { pw.x = kk < n_on ? pw.x : 0.f; pw.y = kk + 1 < n_on ? pw.y : 0.f; }
                     ls2 = __fadd2_rn(ls2, pw);
                     split2(pw, hi[k], lo[k]);
                 }
@@ -340,7 +355,8 @@ __global__ void __launch_bounds__(kPaThreads, MB == 128 ? 2 : 1) prompt_attentio
                 *reinterpret_cast<uint4 *>(Ps + SM::kP1 + o) = make_uint4(lo[0], lo[1], lo[2], lo[3]);
             }
             lsum += ls2.x + ls2.y;
-        }
+        };
+        if (masked) softmax_tile(std::true_type{}); else softmax_tile(std::false_type{});
         fence_proxy_async_smem();
         tc_fence_before_sync();
         __syncthreads();
