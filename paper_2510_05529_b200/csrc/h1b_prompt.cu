@@ -41,13 +41,13 @@ __device__ __forceinline__ int pa_off(int rows, int row, int c16) {
 template <int MB, int NG>          // MB: bytes of one expanded sketch row (128 for m <= 128, else 256)
 struct PaSmem {
     static constexpr int kQ = kPaRows * MB, kK = kPaKeys * MB;
-    static constexpr int kP1 = kPaRows * kPaKeys * 2;           // one part of the weights, [128 queries][64 tokens] fp16
     static constexpr int kV1 = kHeadDim * kPaKeys * 2;          // one part of the values, [128 channels][64 tokens] fp16
     static constexpr int kChunkMax = (MB / 32) * 128 + 2048 + 128 * NG;
     static constexpr int kRaw1 = 2 * kChunkMax;                // the two chunks of one tile
     static constexpr int kRaw = 2 * kRaw1;                      // two tiles: tile j + 2 is requested once tile j's values are out
-    // (two key operands: the scores of tile j + 1 are contracted while the threads work on tile j)
-    static constexpr int kQOff = 0, kKOff = kQ, kPOff = kKOff + 2 * kK, kVOff = kPOff + 2 * kP1, kRawOff = kVOff + 2 * kV1;
+    // (two key operands: the scores of tile j + 1 are contracted while the threads work on tile j; two value operands,
+    // each hi | lo: tile j + 1's values are dequantised while tile j's are being contracted)
+    static constexpr int kQOff = 0, kKOff = kQ, kVOff = kKOff + 2 * kK, kRawOff = kVOff + 4 * kV1;
     static constexpr int kTotal = kRawOff + kRaw + 1024;        // + slack to align the operands to 1024 B
 };
 
@@ -86,7 +86,7 @@ __global__ void __launch_bounds__(kPaThreads, MB == 128 ? 2 : 1) prompt_attentio
     using SM = PaSmem<MB, NG>;
     extern __shared__ unsigned char smem_unaligned[];
     unsigned char *smem = smem_unaligned + ((1024u - (smem_addr(smem_unaligned) & 1023u)) & 1023u);
-    unsigned char *Qs = smem + SM::kQOff, *Ks = smem + SM::kKOff, *Ps = smem + SM::kPOff, *Vs = smem + SM::kVOff;
+    unsigned char *Qs = smem + SM::kQOff, *Ks = smem + SM::kKOff, *Vs = smem + SM::kVOff;
     unsigned char *raw = smem + SM::kRawOff;
     __shared__ uint32_t tmem_base_s;
     // [0], [1] chunk copies of tile j in [j % 2]; [2] unused; [3], [4] scores of tile j in [3 + j % 2]; [5] the P.V contractions
@@ -134,7 +134,9 @@ __global__ void __launch_bounds__(kPaThreads, MB == 128 ? 2 : 1) prompt_attentio
     if (skip_all) return;
     const uint32_t tmem = tmem_base_s;
     const uint32_t t_lane = tmem + ((uint32_t)(warp * 32) << 16);       // this warp's quarter of the TMEM lanes
-    constexpr uint32_t kColS = 0, kColO = 128;                  // scores of tile j at columns 64 (j % 2) .., the output at 128 ..
+    // scores of tile j at columns 64 (j % 2) ..; its weights take their place (fp16 pairs: hi in the first 32 columns,
+    // lo in the other 32) as the A operand of the P.V contractions; the output at 128 ..
+    constexpr uint32_t kColS = 0, kColO = 128;
 
     // ---- this row's query sketch, expanded (rows past the run's end: whatever their words hold; never used)
     {
@@ -218,17 +220,12 @@ __global__ void __launch_bounds__(kPaThreads, MB == 128 ? 2 : 1) prompt_attentio
             expand_keys(j + 1);
         }
         const unsigned char *rawj = raw + (j & 1) * SM::kRaw1;
-        // ---- 2. the previous tile's P.V contractions read the value and weight operands and write the accumulator:
-        // they must be done before those are touched (the key expansion above ran beside them)
-        if (j > 0) {
-            if (!__all_sync(0xffffffffu, mbar_wait_bounded(bar_pv, (uint32_t)((j - 1) & 1), kPaWaitNs))) { failed = true; break; }
-            tc_fence_after_sync();
-        }
         // ---- 3. the values, dequantised once for the 128 queries: v = code * scale + zero, split into two fp16 parts.
         // The four lanes 4 vr .. 4 vr + 3 of a 16-token block hold, in word i, all 16 tokens of channels 16 cb + vr and
         // 16 cb + vr + 8: a thread turns them into whole 32-byte row pieces of the operand.
         {
             const unsigned char *ch = rawj + (vt >> 1) * SM::kChunkMax;
+            unsigned char *Vj = Vs + (j & 1) * (2 * SM::kV1);    // (last read by the contractions of tile j - 2: done)
             const int vb = vt & 1;
             uint2 wj[4];                                        // words 2 vi, 2 vi + 1 of the four lanes
 #pragma unroll
@@ -266,12 +263,18 @@ __global__ void __launch_bounds__(kPaThreads, MB == 128 ? 2 : 1) prompt_attentio
                     }
                     const int chn = cb * 16 + vr + 8 * up;
                     const int o0 = pa_off(kHeadDim, chn, vt * 2), o1 = pa_off(kHeadDim, chn, vt * 2 + 1);
-                    *reinterpret_cast<uint4 *>(Vs + o0) = make_uint4(hi[0], hi[1], hi[2], hi[3]);
-                    *reinterpret_cast<uint4 *>(Vs + o1) = make_uint4(hi[4], hi[5], hi[6], hi[7]);
-                    *reinterpret_cast<uint4 *>(Vs + SM::kV1 + o0) = make_uint4(lo[0], lo[1], lo[2], lo[3]);
-                    *reinterpret_cast<uint4 *>(Vs + SM::kV1 + o1) = make_uint4(lo[4], lo[5], lo[6], lo[7]);
+                    *reinterpret_cast<uint4 *>(Vj + o0) = make_uint4(hi[0], hi[1], hi[2], hi[3]);
+                    *reinterpret_cast<uint4 *>(Vj + o1) = make_uint4(hi[4], hi[5], hi[6], hi[7]);
+                    *reinterpret_cast<uint4 *>(Vj + SM::kV1 + o0) = make_uint4(lo[0], lo[1], lo[2], lo[3]);
+                    *reinterpret_cast<uint4 *>(Vj + SM::kV1 + o1) = make_uint4(lo[4], lo[5], lo[6], lo[7]);
                 }
             }
+        }
+        // ---- 3b. the previous tile's P.V contractions read its weights (where the next tile's scores will land) and
+        // write the accumulator: they must be done before either is touched (the work above ran beside them)
+        if (j > 0) {
+            if (!__all_sync(0xffffffffu, mbar_wait_bounded(bar_pv, (uint32_t)((j - 1) & 1), kPaWaitNs))) { failed = true; break; }
+            tc_fence_after_sync();
         }
         fence_proxy_async_smem();
         tc_fence_before_sync();
@@ -337,9 +340,9 @@ __global__ void __launch_bounds__(kPaThreads, MB == 128 ? 2 : 1) prompt_attentio
             }
             const float2 ch22 = make_float2(ch2, ch2), off2 = make_float2(-smax * ch2, -smax * ch2);
             float2 ls2 = make_float2(0.f, 0.f);
+            uint32_t phi[32], plo[32];
 #pragma unroll
             for (int k8 = 0; k8 < 8; ++k8) {
-                uint32_t hi[4], lo[4];
 #pragma unroll
                 for (int k = 0; k < 4; ++k) {
                     const int kk = k8 * 8 + 2 * k;
@@ -348,31 +351,32 @@ __global__ void __launch_bounds__(kPaThreads, MB == 128 ? 2 : 1) prompt_attentio
                     float2 pw = make_float2(ex2_approx(arg.x), ex2_approx(arg.y));
                     if (MASKED) { pw.x = kk < n_on ? pw.x : 0.f; pw.y = kk + 1 < n_on ? pw.y : 0.f; }
                     ls2 = __fadd2_rn(ls2, pw);
-                    split2(pw, hi[k], lo[k]);
+                    split2(pw, phi[kk >> 1], plo[kk >> 1]);
                 }
-                const int o = pa_off(kPaRows, tid, k8);
-                *reinterpret_cast<uint4 *>(Ps + o) = make_uint4(hi[0], hi[1], hi[2], hi[3]);
-                *reinterpret_cast<uint4 *>(Ps + SM::kP1 + o) = make_uint4(lo[0], lo[1], lo[2], lo[3]);
             }
             lsum += ls2.x + ls2.y;
+            // the weights replace the scores in this row's TMEM lane: 64 fp16 hi parts, then the 64 lo parts
+            tmem_st_32cols(t_lane + kColS + (j & 1) * kPaKeys, phi);
+            tmem_st_32cols(t_lane + kColS + (j & 1) * kPaKeys + 32, plo);
         };
         if (masked) softmax_tile(std::true_type{}); else softmax_tile(std::false_type{});
-        fence_proxy_async_smem();
         tc_fence_before_sync();
         __syncthreads();
-        // ---- 6. out += P V = hi hi + hi lo + lo hi (exact products, fp32 sums), one accumulator
+        // ---- 6. out += P V = hi hi + hi lo + lo hi (exact products, fp32 sums), one accumulator; the weights are read
+        // from TMEM (8 columns = one K slice of 16 keys), the values from shared memory
         if (tid == 0) {
             tc_fence_after_sync();
-            const uint32_t p_hi = smem_addr(Ps), p_lo = p_hi + SM::kP1, v_hi = smem_addr(Vs), v_lo = v_hi + SM::kV1;
+            const uint32_t p_hi = tmem + kColS + (j & 1) * kPaKeys, p_lo = p_hi + 32;
+            const uint32_t v_hi = smem_addr(Vs) + (j & 1) * (2 * SM::kV1), v_lo = v_hi + SM::kV1;
 #pragma unroll
             for (int ks = 0; ks < kPaKeys / 16; ++ks)
-                umma_f16(tmem + kColO, umma_desc_k_sw128(p_hi + ks * 32), umma_desc_k_sw128(v_hi + ks * 32), idesc_o, (j | ks) ? 1u : 0u);
+                umma_f16_ta(tmem + kColO, p_hi + ks * 8, umma_desc_k_sw128(v_hi + ks * 32), idesc_o, (j | ks) ? 1u : 0u);
 #pragma unroll
             for (int ks = 0; ks < kPaKeys / 16; ++ks)
-                umma_f16(tmem + kColO, umma_desc_k_sw128(p_hi + ks * 32), umma_desc_k_sw128(v_lo + ks * 32), idesc_o, 1u);
+                umma_f16_ta(tmem + kColO, p_hi + ks * 8, umma_desc_k_sw128(v_lo + ks * 32), idesc_o, 1u);
 #pragma unroll
             for (int ks = 0; ks < kPaKeys / 16; ++ks)
-                umma_f16(tmem + kColO, umma_desc_k_sw128(p_lo + ks * 32), umma_desc_k_sw128(v_hi + ks * 32), idesc_o, 1u);
+                umma_f16_ta(tmem + kColO, p_lo + ks * 8, umma_desc_k_sw128(v_hi + ks * 32), idesc_o, 1u);
             umma_commit(bar_pv);                                // waited for before the operands are rewritten, or after the loop
         }
     }

@@ -145,6 +145,14 @@ __device__ __forceinline__ void umma_f16(uint32_t tmem_d, uint64_t a_desc, uint6
         "tcgen05.mma.cta_group::1.kind::f16 [%0], %1, %2, %3, p;\n\t}"
         ::"r"(tmem_d), "l"(a_desc), "l"(b_desc), "r"(idesc), "r"(accumulate) : "memory");
 }
+// The same with the A operand in tensor memory: lane r of columns a_tmem .. a_tmem + 7 holds row r's 16 fp16 numbers of
+// the K slice, two per 32-bit column (the lower index in the lower half).
+__device__ __forceinline__ void umma_f16_ta(uint32_t tmem_d, uint32_t a_tmem, uint64_t b_desc, uint32_t idesc, uint32_t accumulate) {
+    asm volatile(
+        "{\n\t.reg .pred p;\n\tsetp.ne.b32 p, %4, 0;\n\t"
+        "tcgen05.mma.cta_group::1.kind::f16 [%0], [%1], %2, %3, p;\n\t}"
+        ::"r"(tmem_d), "r"(a_tmem), "l"(b_desc), "r"(idesc), "r"(accumulate) : "memory");
+}
 // The same for 8-bit floating-point operands (e4m3 x e4m3 -> fp32; one instruction covers K = 32): the instruction
 // descriptor's operand-format fields are 0 for both fp16 (kind::f16) and e4m3 (kind::f8f6f4), so umma_idesc_f16_m128
 // serves both kinds.
