@@ -26,7 +26,7 @@ namespace h1b {
 
 namespace {
 
-constexpr int kPaThreads = 128;
+constexpr int kPaThreads = 160;                     // 128 row threads (thread r owns query row r) + one warp that issues
 constexpr int kPaRows = 128;                       // query rows per block
 constexpr int kPaKeys = 64;                        // cached tokens per tile (two 32-token chunks)
 constexpr unsigned long long kPaWaitNs = 2000000000ull;
@@ -89,8 +89,9 @@ __global__ void __launch_bounds__(kPaThreads, MB == 128 ? 2 : 1) prompt_attentio
     unsigned char *Qs = smem + SM::kQOff, *Ks = smem + SM::kKOff, *Vs = smem + SM::kVOff;
     unsigned char *raw = smem + SM::kRawOff;
     __shared__ uint32_t tmem_base_s;
-    // [0], [1] chunk copies of tile j in [j % 2]; [2] unused; [3], [4] scores of tile j in [3 + j % 2]; [5] the P.V contractions
-    __shared__ __align__(8) unsigned long long bars[6];
+    // [0], [1] chunk copies of tile j in [j % 2]; [2] operands ready (keys of the next tile, values of this one);
+    // [3], [4] scores of tile j in [3 + j % 2]; [5] the P.V contractions; [6] weights ready
+    __shared__ __align__(8) unsigned long long bars[7];
     __shared__ int gave_up;
     const int tid = threadIdx.x, lane = tid & 31, warp = tid >> 5;
     const int mw = p.m_words;
@@ -115,11 +116,12 @@ __global__ void __launch_bounds__(kPaThreads, MB == 128 ? 2 : 1) prompt_attentio
     const int n_tiles = limit_blk > 0 ? (limit_blk + kPaKeys - 1) / kPaKeys : 0;
     const int n_chunks = (len + 31) >> 5;
 
-    const uint32_t bar_copy = smem_addr(&bars[0]), bar_s = smem_addr(&bars[3]), bar_pv = smem_addr(&bars[5]);
+    const uint32_t bar_copy = smem_addr(&bars[0]), bar_kv = smem_addr(&bars[2]), bar_s = smem_addr(&bars[3]);
+    const uint32_t bar_pv = smem_addr(&bars[5]), bar_p = smem_addr(&bars[6]);
     if (tid == 0) {
         gave_up = (*reinterpret_cast<volatile const int32_t *>(p.status) != kStatusOk);
 #pragma unroll
-        for (int i = 0; i < 6; ++i) mbar_init(bar_copy + 8 * i, 1);
+        for (int i = 0; i < 7; ++i) mbar_init(bar_copy + 8 * i, (i == 2 || i == 6) ? kPaRows : 1);     // every row thread arrives on [2], [6]
         mbar_fence_init();
     }
     // the raw chunk buffer starts as zeros: chunks past the sequence's end are never copied, and whatever stands in
@@ -139,7 +141,7 @@ __global__ void __launch_bounds__(kPaThreads, MB == 128 ? 2 : 1) prompt_attentio
     constexpr uint32_t kColS = 0, kColO = 128;
 
     // ---- this row's query sketch, expanded (rows past the run's end: whatever their words hold; never used)
-    {
+    if (tid < kPaRows) {
         const size_t qrow = (((size_t)ll * p.B + b) * p.Tn + (valid_q ? qi : 0)) * p.Hq + hq;
         const uint32_t *qw = p.qstash + qrow * p.qstash_row_words;
 #pragma unroll
@@ -202,17 +204,52 @@ __global__ void __launch_bounds__(kPaThreads, MB == 128 ? 2 : 1) prompt_attentio
     };
     // The tensor cores run one tile ahead of the threads: while the threads turn tile j's scores into weights, the scores
     // of tile j + 1 are already being contracted, and the P.V contractions of tile j run beside the key expansion of
-    // tile j + 2.
-    if (tid == 0) {
-        request_tile(0);
-        if (n_tiles > 1) request_tile(1);
-    }
+    // tile j + 2 and the dequantisation of tile j + 1's values. The row threads never wait for one another: they hand
+    // their operands to the issuing warp through mbarriers and wait only for tensor-core results.
+    if (warp == kPaRows / 32) {
+        // ---- the issuing warp (one lane): chunk copies, score and P.V contractions
+        if (lane == 0) {
+            request_tile(0);
+            if (n_tiles > 1) request_tile(1);
+            if (!mbar_wait_bounded(bar_kv, 0u, kPaWaitNs)) failed = true;           // the first tile's keys are expanded
+            if (!failed) issue_scores(0);
+            for (int j = 0; j < n_tiles && !failed; ++j) {
+                // tile j + 1's keys and tile j's values are in place, every row thread has seen the end of tile j - 1's
+                // P.V contractions (whose weights lie where tile j + 1's scores go) and is done with tile j's chunks
+                if (!mbar_wait_bounded(bar_kv, (uint32_t)((j + 1) & 1), kPaWaitNs)) { failed = true; break; }
+                if (j + 1 < n_tiles) issue_scores(j + 1);
+                if (j + 2 < n_tiles) request_tile(j + 2);
+                // tile j's weights are in TMEM
+                if (!mbar_wait_bounded(bar_p, (uint32_t)(j & 1), kPaWaitNs)) { failed = true; break; }
+                // out += P V = hi hi + hi lo + lo hi (exact products, fp32 sums), one accumulator; the weights are read
+                // from TMEM (8 columns = one K slice of 16 keys), the values from shared memory
+                tc_fence_after_sync();
+                const uint32_t p_hi = tmem + kColS + (j & 1) * kPaKeys, p_lo = p_hi + 32;
+                const uint32_t v_hi = smem_addr(Vs) + (j & 1) * (2 * SM::kV1), v_lo = v_hi + SM::kV1;
+#pragma unroll
+                for (int ks = 0; ks < kPaKeys / 16; ++ks)
+                    umma_f16_ta(tmem + kColO, p_hi + ks * 8, umma_desc_k_sw128(v_hi + ks * 32), idesc_o, (j | ks) ? 1u : 0u);
+#pragma unroll
+                for (int ks = 0; ks < kPaKeys / 16; ++ks)
+                    umma_f16_ta(tmem + kColO, p_hi + ks * 8, umma_desc_k_sw128(v_lo + ks * 32), idesc_o, 1u);
+#pragma unroll
+                for (int ks = 0; ks < kPaKeys / 16; ++ks)
+                    umma_f16_ta(tmem + kColO, p_lo + ks * 8, umma_desc_k_sw128(v_hi + ks * 32), idesc_o, 1u);
+                umma_commit(bar_pv);
+            }
+            if (failed) {
+                atomicExch(p.status, kStatusWaitTimeout);
+                *reinterpret_cast<volatile int *>(&gave_up) = 1;
+            }
+        }
+    } else {
+    // ---- the row threads
     if (!__all_sync(0xffffffffu, mbar_wait_bounded(bar_copy, 0u, kPaWaitNs))) failed = true;
-    if (!failed) expand_keys(0);
-    fence_proxy_async_smem();
-    tc_fence_before_sync();
-    __syncthreads();
-    if (tid == 0 && !failed) issue_scores(0);
+    if (!failed) {
+        expand_keys(0);
+        fence_proxy_async_smem();
+        mbar_arrive(bar_kv);
+    }
     for (int j = 0; j < n_tiles && !failed; ++j) {
         // ---- 1. the next tile's keys (its chunks were requested during the tile before this one)
         if (j + 1 < n_tiles) {
@@ -275,16 +312,16 @@ __global__ void __launch_bounds__(kPaThreads, MB == 128 ? 2 : 1) prompt_attentio
         if (j > 0) {
             if (!__all_sync(0xffffffffu, mbar_wait_bounded(bar_pv, (uint32_t)((j - 1) & 1), kPaWaitNs))) { failed = true; break; }
             tc_fence_after_sync();
+        } else {
+            // (the hand-over barrier must have finished its first phase, the first tile's keys, before anyone arrives
+            // on it for this tile)
+            if (!__all_sync(0xffffffffu, mbar_wait_bounded(bar_kv, 0u, kPaWaitNs))) { failed = true; break; }
         }
+        // ---- 4. hand over: the next tile's scores may start, this tile's chunk buffer may be refilled. This tile's scores
+        // were started one tile ago
         fence_proxy_async_smem();
         tc_fence_before_sync();
-        __syncthreads();
-        // ---- 4. the next tile's scores start; this tile's chunk buffer is free for the tile after the next; this
-        // tile's scores were started one tile ago
-        if (tid == 0) {
-            if (j + 1 < n_tiles) issue_scores(j + 1);
-            if (j + 2 < n_tiles) request_tile(j + 2);
-        }
+        mbar_arrive(bar_kv);
         if (!__all_sync(0xffffffffu, mbar_wait_bounded(bar_s + 8 * (j & 1), (uint32_t)((j >> 1) & 1), kPaWaitNs))) { failed = true; break; }
         tc_fence_after_sync();
         // ---- 5. online softmax on this row's scores
@@ -360,25 +397,9 @@ __global__ void __launch_bounds__(kPaThreads, MB == 128 ? 2 : 1) prompt_attentio
             tmem_st_32cols(t_lane + kColS + (j & 1) * kPaKeys + 32, plo);
         };
         if (masked) softmax_tile(std::true_type{}); else softmax_tile(std::false_type{});
+        // ---- 6. hand over the weights: the issuing warp starts out += P V
         tc_fence_before_sync();
-        __syncthreads();
-        // ---- 6. out += P V = hi hi + hi lo + lo hi (exact products, fp32 sums), one accumulator; the weights are read
-        // from TMEM (8 columns = one K slice of 16 keys), the values from shared memory
-        if (tid == 0) {
-            tc_fence_after_sync();
-            const uint32_t p_hi = tmem + kColS + (j & 1) * kPaKeys, p_lo = p_hi + 32;
-            const uint32_t v_hi = smem_addr(Vs) + (j & 1) * (2 * SM::kV1), v_lo = v_hi + SM::kV1;
-#pragma unroll
-            for (int ks = 0; ks < kPaKeys / 16; ++ks)
-                umma_f16_ta(tmem + kColO, p_hi + ks * 8, umma_desc_k_sw128(v_hi + ks * 32), idesc_o, (j | ks) ? 1u : 0u);
-#pragma unroll
-            for (int ks = 0; ks < kPaKeys / 16; ++ks)
-                umma_f16_ta(tmem + kColO, p_hi + ks * 8, umma_desc_k_sw128(v_lo + ks * 32), idesc_o, 1u);
-#pragma unroll
-            for (int ks = 0; ks < kPaKeys / 16; ++ks)
-                umma_f16_ta(tmem + kColO, p_lo + ks * 8, umma_desc_k_sw128(v_hi + ks * 32), idesc_o, 1u);
-            umma_commit(bar_pv);                                // waited for before the operands are rewritten, or after the loop
-        }
+        mbar_arrive(bar_p);
     }
     if (!failed) {
         if (!__all_sync(0xffffffffu, mbar_wait_bounded(bar_pv, (uint32_t)((n_tiles - 1) & 1), kPaWaitNs))) failed = true;
@@ -407,6 +428,7 @@ __global__ void __launch_bounds__(kPaThreads, MB == 128 ? 2 : 1) prompt_attentio
             }
         }
     }
+    }   // the row threads
     tc_fence_before_sync();
     __syncthreads();
     if (warp == 0) { tc_fence_after_sync(); tmem_dealloc(tmem, 256); }
