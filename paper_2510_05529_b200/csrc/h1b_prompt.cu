@@ -161,8 +161,9 @@ __global__ void __launch_bounds__(kPaThreads, MB == 128 ? 2 : 1) prompt_attentio
     // this thread's share of the tile's keys: half a key (MB / 64 words of it)
     const int k_key = tid >> 1, k_w0 = (tid & 1) * (MB / 64);
     // this thread's share of the tile's values: 16-token block vt, 64-channel half vh, row vr of the channel blocks,
-    // word pair vi (channel blocks 4 vh + 2 vi, + 1: one value group)
-    const int vt = tid >> 5, vh = (tid >> 4) & 1, vr = (tid >> 1) & 7, vi = tid & 1;
+    // word pair vi (channel blocks 4 vh + 2 vi, + 1: one value group). Eight consecutive threads take the eight rows vr:
+    // their 16-byte stores then fall into the eight different 16-byte columns of the swizzled operand rows.
+    const int vt = tid >> 5, vh = (tid >> 4) & 1, vi = (tid >> 3) & 1, vr = tid & 7;
     const int VAL = mw * 128, ZERO = VAL + 2048, SCALE = ZERO + 64 * NG;
     const int vg = NG == 4 ? vh * 2 + vi : 0;                   // the value group of this thread's channels
 
