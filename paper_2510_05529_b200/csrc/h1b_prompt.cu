@@ -329,8 +329,11 @@ __global__ void __launch_bounds__(kPaThreads, MB == 128 ? 2 : 1) prompt_attentio
         const int key_base = j * kPaKeys;
         const bool masked = key_base + kPaKeys > limit_first;   // block-uniform: some row does not see the whole tile
         uint32_t sv[2][32];
-        tmem_ld_32cols(t_lane + kColS + (j & 1) * kPaKeys, sv[0]);
-        tmem_ld_32cols(t_lane + kColS + (j & 1) * kPaKeys + 32, sv[1]);
+        tmem_ld_32cols_issue(t_lane + kColS + (j & 1) * kPaKeys, sv[0]);
+        tmem_ld_32cols_issue(t_lane + kColS + (j & 1) * kPaKeys + 32, sv[1]);
+        tmem_ld_wait();
+        tmem_ld_tie(sv[0]);
+        tmem_ld_tie(sv[1]);
         if (p.dbg_scores && layer == p.dbg_layer && b == p.dbg_b && hq == p.dbg_h && valid_q) {
 #pragma unroll
             for (int k = 0; k < 64; ++k)
@@ -394,8 +397,9 @@ __global__ void __launch_bounds__(kPaThreads, MB == 128 ? 2 : 1) prompt_attentio
             }
             lsum += ls2.x + ls2.y;
             // the weights replace the scores in this row's TMEM lane: 64 fp16 hi parts, then the 64 lo parts
-            tmem_st_32cols(t_lane + kColS + (j & 1) * kPaKeys, phi);
-            tmem_st_32cols(t_lane + kColS + (j & 1) * kPaKeys + 32, plo);
+            tmem_st_32cols_issue(t_lane + kColS + (j & 1) * kPaKeys, phi);
+            tmem_st_32cols_issue(t_lane + kColS + (j & 1) * kPaKeys + 32, plo);
+            tmem_st_wait();
         };
         if (masked) softmax_tile(std::true_type{}); else softmax_tile(std::false_type{});
         // ---- 6. hand over the weights: the issuing warp starts out += P V
