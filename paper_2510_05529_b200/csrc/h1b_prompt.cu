@@ -1,21 +1,24 @@
 // Attention for a whole run of query tokens (a prompt, or a chunk of one) over the compressed cache, on the
 // 5th-generation tensor cores (sm_100a): Eq. 3 and Eq. 5 for blocks of 128 query tokens x 64 cached tokens.
 //
-// One block of 128 threads per (layer, sequence, query head, block of 128 query tokens), two blocks per SM; thread r
-// owns query row r, which is also lane r of every accumulator in tensor memory (TMEM). Per tile of 64 cached tokens:
+// One block of 160 threads per (layer, sequence, query head, block of 128 query tokens), two blocks per SM: 128 row
+// threads (thread r owns query row r, which is also lane r of every accumulator in tensor memory, TMEM) and one issuing
+// warp, of which one lane requests the chunk copies and issues every contraction. The roles hand tiles to one another
+// through mbarriers; there is no block-wide barrier inside the loop. Per tile of 64 cached tokens:
 //   1. the tile's two 32-token chunks come into shared memory with bulk copies, as the decode kernel reads them;
 //   2. scores (Eq. 3) as ONE dense +-1 contraction: the sketch bits of the 128 queries and of the 64 cached keys are
 //      expanded to the 8-bit floating-point numbers +1 / -1 (e4m3), and tcgen05.mma (kind::f8f6f4, fp32 accumulate)
-//      gives S = m - 2 Hamming for the whole 128 x 64 block, exactly (sums of at most 256 terms +-1);
-//   3. online softmax, one query row per thread (Eq. 5): running maximum score (= minimum distance), weights
-//      p = 2^((S - Smax) c / 2) with the causal limit of the row, row sums; every weight is split into two fp16 parts
-//      p = hi + lo (to 2^-22 relative, 2^-25 of the largest weight absolute) and the 128 x 64 weight block is written
-//      to shared memory as an MMA operand;
+//      gives S = m - 2 Hamming for the whole 128 x 64 block, exactly (sums of at most 256 terms +-1). The scores of tile
+//      j + 1 are contracted while the row threads work on tile j (two key operands, two score accumulators);
+//   3. online softmax, one query row per thread (Eq. 5): weights p = 2^((S - reference) c / 2) with the causal limit of
+//      the row, row sums; the reference follows the row's maximum score lazily. Every weight is split into two fp16
+//      parts p = hi + lo (to 2^-22 relative, 2^-25 of the largest weight absolute); the parts are written over the
+//      row's scores in TMEM and serve from there as the A operand of the next step;
 //   4. the tile's values are dequantised ONCE, v = code * scale + zero in fp32, split the same way into two fp16
 //      parts, and serve all 128 queries: out += P V as three fp16 contractions hi hi + hi lo + lo hi into one fp32
-//      accumulator (the products are exact).
-// When a row's running maximum moves, its accumulator lanes are rescaled in TMEM (rare after the first tiles).
-// Every wait is bounded; a block that gives up records the time-out and releases its TMEM.
+//      accumulator (the products are exact). Two value operands: tile j + 1 is dequantised beside tile j's contractions.
+// When a row's reference moves, its accumulator lanes are rescaled in TMEM (rare after the first tile).
+// Every wait is bounded; a role that gives up records the time-out, and the block releases its TMEM.
 #include <mutex>
 #include <type_traits>
 
@@ -80,7 +83,6 @@ __device__ __forceinline__ void split2(float2 ab, uint32_t &hi, uint32_t &lo) {
 
 }  // namespace
 
-// MASKED: some row of the block does not see the whole tile (the tiles on and near the diagonal).
 template <int MB, int NG>
 __global__ void __launch_bounds__(kPaThreads, MB == 128 ? 2 : 1) prompt_attention_kernel(PromptParams p) {
     using SM = PaSmem<MB, NG>;
