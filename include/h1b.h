@@ -378,6 +378,14 @@ int h1b_debug_partials(h1b_ctx *ctx, int layer, int seq, int q_token, int q_head
  *                            128, 4-bit values, m <= 256). Both routes compute the same thing. */
 int h1b_debug_prompt_scores(h1b_ctx *ctx, int layer, int seq, int q_head, int32_t *score_dev, int n_tokens);
 int h1b_debug_prompt_route(h1b_ctx *ctx, int tiles);
+/*   h1b_debug_prompt_stall   the failure path of the tile kernel, exercised without harming anything: in the NEXT
+ *                            h1b_prefill_attention call that takes the tile route, the warp that requests the copies
+ *                            and issues the contractions stays idle and every wait is limited to limit_ns (1 .. 1e9).
+ *                            The row threads' first wait runs out; they record the time-out in the device status word,
+ *                            the block releases its tensor memory and the kernel returns normally. That call's output
+ *                            is undefined; h1b_poll_status() then reports H1B_ERR_TIMEOUT once, and the context keeps
+ *                            working. H1B_ERR_INVALID_ARG for a limit outside the range. */
+int h1b_debug_prompt_stall(h1b_ctx *ctx, uint64_t limit_ns);
 
 /* Bounds-checked build (no counterpart in the paper; a debugging aid). When the
  * library is compiled with -DH1B_DEBUG_BOUNDS, every address a kernel derives

@@ -91,6 +91,7 @@ def load_library(rebuild: bool = True) -> ctypes.CDLL:
         "h1b_debug_wait_timeout": (ctypes.c_int, [vp, ctypes.c_uint64, vp]),
         "h1b_debug_prompt_scores": (ctypes.c_int, [vp, ctypes.c_int, ctypes.c_int, ctypes.c_int, vp, ctypes.c_int]),
         "h1b_debug_prompt_route": (ctypes.c_int, [vp, ctypes.c_int]),
+        "h1b_debug_prompt_stall": (ctypes.c_int, [vp, ctypes.c_uint64]),
         "h1b_bounds_checked": (ctypes.c_int, []),
         "h1b_debug_bounds_probe": (ctypes.c_int, [vp, vp]),
         "h1b_set_splits": (ctypes.c_int, [vp, ctypes.c_int]),
@@ -394,6 +395,11 @@ class H1BCache:
     def h1b_debug_prompt_route(self, tiles: bool):
         """False: prompt attention walks 16 query tokens at a time through the decode kernels, whatever the run's length."""
         self._check(self.lib.h1b_debug_prompt_route(self._h, int(bool(tiles))))
+
+    def h1b_debug_prompt_stall(self, limit_ns: int):
+        """The next tile-route h1b_prefill_attention call runs with its issuing warp idle and waits limited to limit_ns:
+        its row threads time out, the next h1b_poll_status() reports it (the call's output is undefined)."""
+        self._check(self.lib.h1b_debug_prompt_stall(self._h, int(limit_ns)))
 
     def h1b_debug_bounds_probe(self, stream=None):
         """Bounds-checked build only: a kernel's check fails on purpose; the next h1b_poll_status() reports it."""

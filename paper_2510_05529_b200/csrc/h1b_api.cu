@@ -190,6 +190,7 @@ struct h1b_ctx {
     cudaEvent_t fork, join;            // ... forked from and joined back into the caller's stream
     bool no_prompt_tiles;              // test helper: prompt attention through the 16-token route whatever the run's length
     int32_t *dbg_scores;               // test helper: where the next prompt-attention call exports one head's scores
+    uint64_t dbg_prompt_stall_ns;      // test helper: the next tile-route prompt-attention call runs with its issuing warp idle
     int dbg_layer, dbg_seq, dbg_head, dbg_T;
     DecodeParams last_decode;          // the most recent attention launch (test helper: h1b_debug_partials)
     bool have_last_decode;
@@ -307,6 +308,7 @@ int h1b_init_projection(const h1b_config *cfg, uint64_t seed, const float *Rt_ho
     ctx->side = nullptr; ctx->fork = nullptr; ctx->join = nullptr;
     ctx->have_last_decode = false;
     ctx->dbg_scores = nullptr;
+    ctx->dbg_prompt_stall_ns = 0;
     ctx->no_prompt_tiles = false;
     cudaStream_t st = static_cast<cudaStream_t>(stream);
     auto bail = [&](cudaError_t e, const char *what) {
@@ -692,7 +694,7 @@ int h1b_prefill_attention(h1b_ctx *ctx, int layer_begin, int n_layers, const voi
         sp.q_seq_rows = sp.Hq;
         sp.qw_row_words = kHeadDim;                     // one output row (128 floats) per (token, head)
         H1B_CUDA(ctx, launch_prepare(nullptr, &sp, none, st, &launches));
-        PromptParams pp;
+        PromptParams pp = {};
         pp.ca = cache_addr(ctx);
         pp.len = at<int32_t>(ctx, ctx->plan.len);
         pp.qstash = static_cast<const uint32_t *>(out);
@@ -705,6 +707,9 @@ int h1b_prefill_attention(h1b_ctx *ctx, int layer_begin, int n_layers, const voi
         pp.dbg_scores = ctx->dbg_scores; pp.dbg_layer = ctx->dbg_layer; pp.dbg_b = ctx->dbg_seq; pp.dbg_h = ctx->dbg_head;
         pp.dbg_T = ctx->dbg_T;
         ctx->dbg_scores = nullptr;                      // one call only
+        pp.dbg_no_issue = ctx->dbg_prompt_stall_ns ? 1 : 0;
+        pp.wait_ns = ctx->dbg_prompt_stall_ns;
+        ctx->dbg_prompt_stall_ns = 0;
         H1B_CUDA(ctx, launch_prompt_attention(pp, st, &launches));
         ctx->launches += launches;
         return H1B_OK;
@@ -1173,6 +1178,14 @@ int h1b_debug_prompt_scores(h1b_ctx *ctx, int layer, int seq, int q_head, int32_
         return fail(ctx, H1B_ERR_INVALID_ARG, "(layer %d, seq %d, head %d, %d tokens) out of range", layer, seq, q_head, n_tokens);
     ctx->dbg_scores = score_dev;
     ctx->dbg_layer = layer; ctx->dbg_seq = seq; ctx->dbg_head = q_head; ctx->dbg_T = n_tokens;
+    return H1B_OK;
+}
+
+int h1b_debug_prompt_stall(h1b_ctx *ctx, uint64_t limit_ns) {
+    if (!ctx) return H1B_ERR_NULL;
+    if (limit_ns < 1 || limit_ns > 1000000000ull)
+        return fail(ctx, H1B_ERR_INVALID_ARG, "limit_ns = %llu outside [1, 1e9]", (unsigned long long)limit_ns);
+    ctx->dbg_prompt_stall_ns = limit_ns;
     return H1B_OK;
 }
 

@@ -837,7 +837,9 @@ template <int NBC> struct PrefillEntry<NBC, true> { static constexpr auto fn = p
 // ===========================================================================
 constexpr int kTmaThreads = 320;
 template <int NBC>
-__global__ void __launch_bounds__(kTmaThreads, 1) prefill_tma_kernel(const __grid_constant__ CUtensorMap kmap, PrefillParams p,
+// (96 registers per thread: four blocks of the value kernel then fit on the SM beside this one instead of three, which is
+// worth 3-4 % of the long append; the dozen spilled bytes cost nothing measurable)
+__global__ void __maxnreg__(96) prefill_tma_kernel(const __grid_constant__ CUtensorMap kmap, PrefillParams p,
                                                                       NewCounts nn) {
     using SM = PrefillSmem<NBC>;
     extern __shared__ unsigned char smem_unaligned[];

@@ -219,6 +219,9 @@ struct PromptParams {
     // test helper: the integer scores m - 2 Hamming of one (layer, sequence, query head), [Tn][dbg_T], null = off
     int32_t *dbg_scores;
     int dbg_layer, dbg_b, dbg_h, dbg_T;
+    // test helper of the failure path: the issuing warp stays idle and every wait is limited to wait_ns (0: the default)
+    int dbg_no_issue;
+    unsigned long long wait_ns;
 };
 
 }  // namespace h1b

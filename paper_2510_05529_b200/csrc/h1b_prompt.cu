@@ -157,6 +157,7 @@ __global__ void __launch_bounds__(kPaThreads, MB == 128 ? 2 : 1) prompt_attentio
     // scores are handled as the floats the tensor cores deliver: S = m - 2 Hamming, so the running minimum distance is
     // the running maximum score and p = 2^((S - Smax) c / 2)
     const float ch2 = 0.5f * p.c;
+    const unsigned long long wait_ns = p.wait_ns ? p.wait_ns : kPaWaitNs;
     float smax = -1e30f, lsum = 0.f;
     bool failed = false;
     const uint32_t idesc_s = umma_idesc_f16_m128(kPaKeys), idesc_o = umma_idesc_f16_m128(kHeadDim);
@@ -211,19 +212,19 @@ __global__ void __launch_bounds__(kPaThreads, MB == 128 ? 2 : 1) prompt_attentio
     // their operands to the issuing warp through mbarriers and wait only for tensor-core results.
     if (warp == kPaRows / 32) {
         // ---- the issuing warp (one lane): chunk copies, score and P.V contractions
-        if (lane == 0) {
+        if (lane == 0 && !p.dbg_no_issue) {
             request_tile(0);
             if (n_tiles > 1) request_tile(1);
-            if (!mbar_wait_bounded(bar_kv, 0u, kPaWaitNs)) failed = true;           // the first tile's keys are expanded
+            if (!mbar_wait_bounded(bar_kv, 0u, wait_ns)) failed = true;           // the first tile's keys are expanded
             if (!failed) issue_scores(0);
             for (int j = 0; j < n_tiles && !failed; ++j) {
                 // tile j + 1's keys and tile j's values are in place, every row thread has seen the end of tile j - 1's
                 // P.V contractions (whose weights lie where tile j + 1's scores go) and is done with tile j's chunks
-                if (!mbar_wait_bounded(bar_kv, (uint32_t)((j + 1) & 1), kPaWaitNs)) { failed = true; break; }
+                if (!mbar_wait_bounded(bar_kv, (uint32_t)((j + 1) & 1), wait_ns)) { failed = true; break; }
                 if (j + 1 < n_tiles) issue_scores(j + 1);
                 if (j + 2 < n_tiles) request_tile(j + 2);
                 // tile j's weights are in TMEM
-                if (!mbar_wait_bounded(bar_p, (uint32_t)(j & 1), kPaWaitNs)) { failed = true; break; }
+                if (!mbar_wait_bounded(bar_p, (uint32_t)(j & 1), wait_ns)) { failed = true; break; }
                 // out += P V = hi hi + hi lo + lo hi (exact products, fp32 sums), one accumulator; the weights are read
                 // from TMEM (8 columns = one K slice of 16 keys), the values from shared memory
                 tc_fence_after_sync();
@@ -247,7 +248,7 @@ __global__ void __launch_bounds__(kPaThreads, MB == 128 ? 2 : 1) prompt_attentio
         }
     } else {
     // ---- the row threads
-    if (!__all_sync(0xffffffffu, mbar_wait_bounded(bar_copy, 0u, kPaWaitNs))) failed = true;
+    if (!__all_sync(0xffffffffu, mbar_wait_bounded(bar_copy, 0u, wait_ns))) failed = true;
     if (!failed) {
         expand_keys(0);
         fence_proxy_async_smem();
@@ -256,7 +257,7 @@ __global__ void __launch_bounds__(kPaThreads, MB == 128 ? 2 : 1) prompt_attentio
     for (int j = 0; j < n_tiles && !failed; ++j) {
         // ---- 1. the next tile's keys (its chunks were requested during the tile before this one)
         if (j + 1 < n_tiles) {
-            if (!__all_sync(0xffffffffu, mbar_wait_bounded(bar_copy + 8 * ((j + 1) & 1), (uint32_t)(((j + 1) >> 1) & 1), kPaWaitNs))) { failed = true; break; }
+            if (!__all_sync(0xffffffffu, mbar_wait_bounded(bar_copy + 8 * ((j + 1) & 1), (uint32_t)(((j + 1) >> 1) & 1), wait_ns))) { failed = true; break; }
             expand_keys(j + 1);
         }
         const unsigned char *rawj = raw + (j & 1) * SM::kRaw1;
@@ -313,19 +314,19 @@ __global__ void __launch_bounds__(kPaThreads, MB == 128 ? 2 : 1) prompt_attentio
         // ---- 3b. the previous tile's P.V contractions read its weights (where the next tile's scores will land) and
         // write the accumulator: they must be done before either is touched (the work above ran beside them)
         if (j > 0) {
-            if (!__all_sync(0xffffffffu, mbar_wait_bounded(bar_pv, (uint32_t)((j - 1) & 1), kPaWaitNs))) { failed = true; break; }
+            if (!__all_sync(0xffffffffu, mbar_wait_bounded(bar_pv, (uint32_t)((j - 1) & 1), wait_ns))) { failed = true; break; }
             tc_fence_after_sync();
         } else {
             // (the hand-over barrier must have finished its first phase, the first tile's keys, before anyone arrives
             // on it for this tile)
-            if (!__all_sync(0xffffffffu, mbar_wait_bounded(bar_kv, 0u, kPaWaitNs))) { failed = true; break; }
+            if (!__all_sync(0xffffffffu, mbar_wait_bounded(bar_kv, 0u, wait_ns))) { failed = true; break; }
         }
         // ---- 4. hand over: the next tile's scores may start, this tile's chunk buffer may be refilled. This tile's scores
         // were started one tile ago
         fence_proxy_async_smem();
         tc_fence_before_sync();
         mbar_arrive(bar_kv);
-        if (!__all_sync(0xffffffffu, mbar_wait_bounded(bar_s + 8 * (j & 1), (uint32_t)((j >> 1) & 1), kPaWaitNs))) { failed = true; break; }
+        if (!__all_sync(0xffffffffu, mbar_wait_bounded(bar_s + 8 * (j & 1), (uint32_t)((j >> 1) & 1), wait_ns))) { failed = true; break; }
         tc_fence_after_sync();
         // ---- 5. online softmax on this row's scores
         const int key_base = j * kPaKeys;
@@ -409,14 +410,14 @@ __global__ void __launch_bounds__(kPaThreads, MB == 128 ? 2 : 1) prompt_attentio
         mbar_arrive(bar_p);
     }
     if (!failed) {
-        if (!__all_sync(0xffffffffu, mbar_wait_bounded(bar_pv, (uint32_t)((n_tiles - 1) & 1), kPaWaitNs))) failed = true;
+        if (!__all_sync(0xffffffffu, mbar_wait_bounded(bar_pv, (uint32_t)((n_tiles - 1) & 1), wait_ns))) failed = true;
         tc_fence_after_sync();
     }
 
     if (failed) {
         if (lane == 0) atomicExch(p.status, kStatusWaitTimeout);
         // work that may still be in flight gets a bounded time before the TMEM goes back
-        (void)mbar_wait_bounded(bar_pv, (uint32_t)((n_tiles - 1) & 1), 100000000ull);
+        (void)mbar_wait_bounded(bar_pv, (uint32_t)((n_tiles - 1) & 1), wait_ns < 100000000ull ? wait_ns : 100000000ull);
     } else {
         // ---- the row's output: accumulator / sum of weights. The TMEM loads are warp-wide instructions: every lane
         // makes them, rows past the run's end simply do not store.
