@@ -41,7 +41,7 @@ __device__ __forceinline__ int pa_off(int rows, int row, int c16) {
     return (c16 >> 3) * (rows * 128) + row * 128 + (((c16 & 7) ^ (row & 7)) << 4);
 }
 
-template <int MB, int NG>          // MB: bytes of one expanded sketch row (128 for m <= 128, else 256)
+template <int MB, int NG>          // MB: bytes of one expanded sketch row (128 for m <= 128, 256 for m <= 256, else 512)
 struct PaSmem {
     static constexpr int kQ = kPaRows * MB, kK = kPaKeys * MB;
     static constexpr int kV1 = kHeadDim * kPaKeys * 2;          // one part of the values, [128 channels][64 tokens] fp16
@@ -467,14 +467,19 @@ static cudaError_t launch_prompt_t(const PromptParams &p, cudaStream_t st, bool 
 }
 
 bool prompt_attention_supported(int m_words, int groups, bool paired) {
-    return !paired && (groups == 4 || groups == 1) && m_words >= 2 && m_words <= 8;
+    return !paired && (groups == 4 || groups == 1) && m_words >= 2 && m_words <= 16;
 }
 
 cudaError_t launch_prompt_attention(const PromptParams &p, cudaStream_t st, int *launches, bool attributes_only) {
     cudaError_t e = cudaErrorInvalidValue;
-    const bool wide = p.m_words > 4;
-    if (p.groups == 4) e = wide ? launch_prompt_t<256, 4>(p, st, attributes_only) : launch_prompt_t<128, 4>(p, st, attributes_only);
-    else if (p.groups == 1) e = wide ? launch_prompt_t<256, 1>(p, st, attributes_only) : launch_prompt_t<128, 1>(p, st, attributes_only);
+    // (bytes of an expanded sketch row: 128 for m <= 128, 256 for m <= 256, 512 for m <= 512)
+    const int mb = p.m_words <= 4 ? 128 : p.m_words <= 8 ? 256 : 512;
+    if (p.groups == 4)
+        e = mb == 128 ? launch_prompt_t<128, 4>(p, st, attributes_only) : mb == 256 ? launch_prompt_t<256, 4>(p, st, attributes_only)
+                                                                                     : launch_prompt_t<512, 4>(p, st, attributes_only);
+    else if (p.groups == 1)
+        e = mb == 128 ? launch_prompt_t<128, 1>(p, st, attributes_only) : mb == 256 ? launch_prompt_t<256, 1>(p, st, attributes_only)
+                                                                                     : launch_prompt_t<512, 1>(p, st, attributes_only);
     if (e == cudaSuccess && !attributes_only && launches) ++*launches;
     return e;
 }

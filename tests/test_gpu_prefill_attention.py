@@ -108,6 +108,7 @@ def test_bad_arguments():
     (4, 2, 256, 128, [384, 200], 128, 1.0),       # two 128-byte column blocks per sketch; one scale per value vector
     (2, 2, 128, 32, [130, 33], 33, 1e-3),         # almost uniform weights
     (2, 2, 128, 32, [513, 512], 500, 400.0),      # peaked softmax: the running minimum moves late, accumulators are rescaled
+    (2, 1, 512, 32, [300, 140], 140, 16.0),       # the widest sketch: four 128-byte column blocks per row
 ])
 def test_tile_route_scores_bit_for_bit_and_both_routes_agree(hq, hkv, m, G, lens, Tn, inv_tau):
     """Runs of 32 query tokens or more go through the 128 x 128 tile kernel: its tensor-core scores (Eq. 3) are exported
