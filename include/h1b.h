@@ -196,7 +196,7 @@ int h1b_decode_attention_multi(h1b_ctx *ctx, int layer_begin, int n_layers, cons
  * chunk of one): the queries are the sequences' last Tn cached tokens (append
  * their keys and values first), query token i attends to cached tokens
  * [0, len - Tn + i + 1). Any Tn >= 1. Runs of 32 tokens or more (head
- * dimension 128, 4-bit values) are processed in blocks of 128 query
+ * dimension 128) are processed in blocks of 128 query
  * tokens x 64 cached tokens on the tensor cores: Eq. 3 as one dense +-1
  * contraction per block (exact integers), Eq. 5 with each tile's values
  * dequantised once for all its queries; `out` doubles as scratch for the query
@@ -375,7 +375,7 @@ int h1b_debug_partials(h1b_ctx *ctx, int layer, int seq, int q_token, int q_head
  *   h1b_debug_prompt_route   tiles = 0: h1b_prefill_attention walks every run in blocks of H1B_MAX_QUERY_TOKENS through
  *                            the decode kernels (the route short runs take); tiles = 1 (default): runs of 32 query tokens
  *                            or more take the 128 x 64 tile kernel where the cache format allows it (head dimension
- *                            128, 4-bit values). Both routes compute the same thing. */
+ *                            128). Both routes compute the same thing. */
 int h1b_debug_prompt_scores(h1b_ctx *ctx, int layer, int seq, int q_head, int32_t *score_dev, int n_tokens);
 int h1b_debug_prompt_route(h1b_ctx *ctx, int tiles);
 /*   h1b_debug_prompt_stall   the failure path of the tile kernel, exercised without harming anything: in the NEXT

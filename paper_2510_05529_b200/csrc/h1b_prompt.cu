@@ -45,12 +45,14 @@ template <int MB, int NG>          // MB: bytes of one expanded sketch row (128 
 struct PaSmem {
     static constexpr int kQ = kPaRows * MB, kK = kPaKeys * MB;
     static constexpr int kV1 = kHeadDim * kPaKeys * 2;          // one part of the values, [128 channels][64 tokens] fp16
-    static constexpr int kChunkMax = (MB / 32) * 128 + 2048 + 128 * NG;
+    static constexpr int kVParts = NG == 0 ? 1 : 2;             // fp16 values (NG = 0) are their own, single part
+    static constexpr int kVBuf = kVParts * kV1;                 // one value operand
+    static constexpr int kChunkMax = (MB / 32) * 128 + (NG == 0 ? 2 * kHalfBlockBytes : 2 * kValBlockBytes + 128 * NG);
     static constexpr int kRaw1 = 2 * kChunkMax;                // the two chunks of one tile
     static constexpr int kRaw = 2 * kRaw1;                      // two tiles: tile j + 2 is requested once tile j's values are out
     // (two key operands: the scores of tile j + 1 are contracted while the threads work on tile j; two value operands,
     // each hi | lo: tile j + 1's values are dequantised while tile j's are being contracted)
-    static constexpr int kQOff = 0, kKOff = kQ, kVOff = kKOff + 2 * kK, kRawOff = kVOff + 4 * kV1;
+    static constexpr int kQOff = 0, kKOff = kQ, kVOff = kKOff + 2 * kK, kRawOff = kVOff + 2 * kVBuf;
     static constexpr int kTotal = kRawOff + kRaw + 1024;        // + slack to align the operands to 1024 B
 };
 
@@ -229,13 +231,15 @@ __global__ void __launch_bounds__(kPaThreads, MB == 128 ? 2 : 1) prompt_attentio
                 // from TMEM (8 columns = one K slice of 16 keys), the values from shared memory
                 tc_fence_after_sync();
                 const uint32_t p_hi = tmem + kColS + (j & 1) * kPaKeys, p_lo = p_hi + 32;
-                const uint32_t v_hi = smem_addr(Vs) + (j & 1) * (2 * SM::kV1), v_lo = v_hi + SM::kV1;
+                const uint32_t v_hi = smem_addr(Vs) + (j & 1) * SM::kVBuf, v_lo = v_hi + SM::kV1;
 #pragma unroll
                 for (int ks = 0; ks < kPaKeys / 16; ++ks)
                     umma_f16_ta(tmem + kColO, p_hi + ks * 8, umma_desc_k_sw128(v_hi + ks * 32), idesc_o, (j | ks) ? 1u : 0u);
+                if constexpr (NG != 0) {                        // (fp16 values have no lo part)
 #pragma unroll
-                for (int ks = 0; ks < kPaKeys / 16; ++ks)
-                    umma_f16_ta(tmem + kColO, p_hi + ks * 8, umma_desc_k_sw128(v_lo + ks * 32), idesc_o, 1u);
+                    for (int ks = 0; ks < kPaKeys / 16; ++ks)
+                        umma_f16_ta(tmem + kColO, p_hi + ks * 8, umma_desc_k_sw128(v_lo + ks * 32), idesc_o, 1u);
+                }
 #pragma unroll
                 for (int ks = 0; ks < kPaKeys / 16; ++ks)
                     umma_f16_ta(tmem + kColO, p_lo + ks * 8, umma_desc_k_sw128(v_hi + ks * 32), idesc_o, 1u);
@@ -264,9 +268,26 @@ __global__ void __launch_bounds__(kPaThreads, MB == 128 ? 2 : 1) prompt_attentio
         // ---- 3. the values, dequantised once for the 128 queries: v = code * scale + zero, split into two fp16 parts.
         // The four lanes 4 vr .. 4 vr + 3 of a 16-token block hold, in word i, all 16 tokens of channels 16 cb + vr and
         // 16 cb + vr + 8: a thread turns them into whole 32-byte row pieces of the operand.
-        {
+        if constexpr (NG == 0) {
+            // fp16 values ("1-bit keys only"): no arithmetic, only the way from the cache's order (lane r * 4 + jj of a
+            // 16-token block and channel block holds, in word 2 h8 + hi, tokens 2 jj + 8 h8, + 1 of channel row r + 8 hi)
+            // to K-major operand rows; a warp reads 512 contiguous bytes and writes 4-byte pieces to 32 different banks
+            unsigned char *Vj = Vs + (j & 1) * SM::kVBuf;
+#pragma unroll
+            for (int i = 0; i < 8; ++i) {
+                const int e = tid + kPaRows * i, et = e >> 8, cb = (e >> 5) & 7, ln = e & 31, r = ln >> 2, jj = ln & 3;
+                const unsigned char *ch = rawj + (et >> 1) * SM::kChunkMax;
+                const uint4 w4 = *reinterpret_cast<const uint4 *>(ch + VAL + (et & 1) * kHalfBlockBytes + cb * 512 + ln * 16);
+                const uint32_t ws[4] = {w4.x, w4.y, w4.z, w4.w};
+#pragma unroll
+                for (int h8 = 0; h8 < 2; ++h8)
+#pragma unroll
+                    for (int hi = 0; hi < 2; ++hi)
+                        *reinterpret_cast<uint32_t *>(Vj + pa_off(kHeadDim, cb * 16 + r + 8 * hi, et * 2 + h8) + jj * 4) = ws[h8 * 2 + hi];
+            }
+        } else {
             const unsigned char *ch = rawj + (vt >> 1) * SM::kChunkMax;
-            unsigned char *Vj = Vs + (j & 1) * (2 * SM::kV1);    // (last read by the contractions of tile j - 2: done)
+            unsigned char *Vj = Vs + (j & 1) * SM::kVBuf;        // (last read by the contractions of tile j - 2: done)
             const int vb = vt & 1;
             uint2 wj[4];                                        // words 2 vi, 2 vi + 1 of the four lanes
 #pragma unroll
@@ -467,7 +488,7 @@ static cudaError_t launch_prompt_t(const PromptParams &p, cudaStream_t st, bool 
 }
 
 bool prompt_attention_supported(int m_words, int groups, bool paired) {
-    return !paired && (groups == 4 || groups == 1) && m_words >= 2 && m_words <= 16;
+    return !paired && (groups == 4 || groups == 1 || groups == 0) && m_words >= 2 && m_words <= 16;
 }
 
 cudaError_t launch_prompt_attention(const PromptParams &p, cudaStream_t st, int *launches, bool attributes_only) {
@@ -480,6 +501,9 @@ cudaError_t launch_prompt_attention(const PromptParams &p, cudaStream_t st, int 
     else if (p.groups == 1)
         e = mb == 128 ? launch_prompt_t<128, 1>(p, st, attributes_only) : mb == 256 ? launch_prompt_t<256, 1>(p, st, attributes_only)
                                                                                      : launch_prompt_t<512, 1>(p, st, attributes_only);
+    else if (p.groups == 0)                                     // fp16 values
+        e = mb == 128 ? launch_prompt_t<128, 0>(p, st, attributes_only) : mb == 256 ? launch_prompt_t<256, 0>(p, st, attributes_only)
+                                                                                     : launch_prompt_t<512, 0>(p, st, attributes_only);
     if (e == cudaSuccess && !attributes_only && launches) ++*launches;
     return e;
 }

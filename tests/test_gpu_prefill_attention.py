@@ -91,6 +91,25 @@ def test_a_whole_prompt_with_rotary_embedding_end_to_end():
     cache.close()
 
 
+def test_tile_route_with_fp16_values():
+    """The "1-bit keys only" cache (values kept in fp16): the tile kernel reads the values as they are, one fp16 part, and must
+    agree with the oracle and with the 16-token route."""
+    w = h1b_synth.scaled(W["c1_tiny"], batch=2, n_layers=2, n_q_heads=4, n_kv_heads=2)
+    cache, Rt, K, V, lens = _fill(w, [300, 170], fp16_values=True)
+    q = _queries(w, 170, seed=13)
+    qd = q.cuda()
+    out = cache.h1b_prefill_attention(qd, 16.0).cpu().numpy()
+    torch.cuda.synchronize()
+    cache.h1b_poll_status()
+    _check(w, cache, Rt, K, V, q, lens, out, 16.0, True)
+    cache.h1b_debug_prompt_route(False)
+    walk = cache.h1b_prefill_attention(qd, 16.0).cpu().numpy()
+    cache.h1b_debug_prompt_route(True)
+    cache.h1b_poll_status()
+    np.testing.assert_allclose(out, walk, rtol=2e-4, atol=5e-6)
+    cache.close()
+
+
 def test_bad_arguments():
     w = h1b_synth.scaled(W["c1_tiny"], batch=2, n_layers=1, n_q_heads=2, n_kv_heads=2)
     cache, Rt, K, V, lens = _fill(w, [50, 20])
