@@ -10,6 +10,7 @@ import torch
 import h1b_synth
 import oracle
 from h1b_testlib import append_parity, check_output, f16_bits, make_cache, oracle_from_export
+from paper_2510_05529_b200 import binding
 
 pytestmark = pytest.mark.gpu
 W = h1b_synth.WORKLOADS
@@ -138,4 +139,50 @@ def test_c6_60m_shape_head_dim_64_full_size():
     cache, Rt, units, kept, q, out, lens = _run_full(w, n_samples=4)
     stats = _check_units(w, cache, Rt, units, kept, q, out, lens)
     print("c6 full size", stats)
+    cache.close()
+
+
+def test_prompt_attention_over_a_full_8k_prompt():
+    """The tile kernel at the prompt length bench.py times (8192 tokens, 32 heads; two of the 32 layers): attention for
+    every prompt token over the compressed prompt. Sampled (layer, head, query token) rows are checked one by one against
+    the oracle, which compresses the rows the token sees itself."""
+    w = h1b_synth.scaled(W["c5_prefill"], n_layers=2)
+    T = w.context
+    cache, Rt = make_cache(w, max_seq=T)
+    keep = {}
+    heads = {0: (0, 17), 1: (5, 31)}
+    for l in range(w.n_layers):
+        K, V = h1b_synth.kv_rows(w, l, T, device="cuda")
+        cache.h1b_append_kv(K.unsqueeze(0), V.unsqueeze(0), layer_begin=l)
+        for h in heads[l]:
+            keep[(l, h)] = (K[0, :, h].cpu(), V[0, :, h].cpu())
+        del K, V
+    q = torch.stack([h1b_synth.normal_fp16(h1b_synth.layer_seed(w, l, 4242), (1, T, w.n_q_heads, w.head_dim), "cuda")
+                     for l in range(w.n_layers)])
+    out = cache.h1b_prefill_attention(q, INV_TAU)
+    torch.cuda.synchronize()
+    cache.h1b_poll_status()
+    assert cache.h1b_launch_count() > 0
+    rng = np.random.default_rng(8192)
+    checked, worst = 0, 0.0
+    for (l, h), (K, V) in keep.items():
+        kbits = binding.unpack_words(cache.h1b_export_cache(l, 0, h, 0, T)[0], w.sketch_bits)
+        obits, y, a = oracle.sketch(f16_bits(K), Rt[l], want_margin=True)
+        assert not ((kbits != obits) & (np.abs(y) > 1e-5 * a)).any()
+        same = (kbits == obits).all(axis=1)                               # tokens whose key bits the oracle agrees on
+        tokens = sorted({0, 1, 63, 64, 127, 128, 4095, T - 1} | {int(t) for t in rng.integers(0, T, 6)})
+        for i in tokens:
+            if not same[:i + 1].all():
+                continue                                                 # a key bit on the sign boundary below this token
+            qi = q[l, 0, i, h].cpu()
+            _, yq, aq = oracle.sketch(f16_bits(qi)[None], Rt[l], want_margin=True)
+            if (np.abs(yq) <= 1e-5 * aq).any():
+                continue
+            n = i + 1
+            ref = oracle.layer(f16_bits(K[:n]).reshape(1, n, 1, -1), f16_bits(V[:n]).reshape(1, n, 1, -1),
+                               np.array([n], np.int32), f16_bits(qi).reshape(1, 1, -1), Rt[l], INV_TAU)[0, 0]
+            worst = max(worst, check_output(out[l, 0, i, h].cpu().numpy(), ref, ("8k prompt", l, h, i)))
+            checked += 1
+    print("prompt attention over 8192 tokens:", checked, "rows checked, max err", worst)
+    assert checked >= 20
     cache.close()
