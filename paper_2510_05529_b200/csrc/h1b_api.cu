@@ -679,7 +679,7 @@ int h1b_prefill_attention(h1b_ctx *ctx, int layer_begin, int n_layers, const voi
                 return fail(ctx, H1B_ERR_INVALID_ARG, "layer %d sequence %d holds %d < Tn = %d tokens", l, b,
                             ctx->len_host[(size_t)l * ctx->cfg.max_batch + b], Tn);
     // Runs of at least kPromptMinTokens query tokens on a cache format the tile kernel serves: scores and P.V as
-    // dense contractions over blocks of 128 queries x 128 cached tokens. The sketches of all query tokens are kept in
+    // dense contractions over blocks of 128 queries x 64 cached tokens. The sketches of all query tokens are kept in
     // the first words of the output rows they belong to (the kernel reads a row's words before it writes the row).
     if (Tn >= kPromptMinTokens && !ctx->no_prompt_tiles && prompt_attention_supported(ctx->plan.m_words, ctx->plan.groups, ctx->paired) &&
         (size_t)n_layers * B * Tn * ctx->cfg.n_q_heads < (size_t)0x7fffffff) {

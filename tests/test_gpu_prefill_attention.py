@@ -130,7 +130,7 @@ def test_bad_arguments():
     (2, 1, 512, 32, [300, 140], 140, 16.0),       # the widest sketch: four 128-byte column blocks per row
 ])
 def test_tile_route_scores_bit_for_bit_and_both_routes_agree(hq, hkv, m, G, lens, Tn, inv_tau):
-    """Runs of 32 query tokens or more go through the 128 x 128 tile kernel: its tensor-core scores (Eq. 3) are exported
+    """Runs of 32 query tokens or more go through the 128 x 64 tile kernel: its tensor-core scores (Eq. 3) are exported
     and compared bit for bit with the oracle's, its outputs with the oracle (inside _check) and with the 16-token route."""
     w = h1b_synth.scaled(W["c1_tiny"], batch=2, n_layers=2, n_q_heads=hq, n_kv_heads=hkv, sketch_bits=m, group_size=G)
     cache, Rt, K, V, lens = _fill(w, lens)
