@@ -22,6 +22,7 @@
 #include <mutex>
 #include <type_traits>
 
+#include "h1b_bounds.cuh"
 #include "h1b_kernels.h"
 #include "h1b_ptx.cuh"
 
@@ -148,10 +149,11 @@ __global__ void __launch_bounds__(kPaThreads, MB == 128 ? 2 : 1) prompt_attentio
     if (tid < kPaRows) {
         const size_t qrow = (((size_t)ll * p.B + b) * p.Tn + (valid_q ? qi : 0)) * p.Hq + hq;
         const uint32_t *qw = p.qstash + qrow * p.qstash_row_words;
+        const bool q_ok = H1B_IN_BOUNDS(ll >= 0 && qrow < (size_t)p.n_layers * p.B * p.Tn * p.Hq, p.status, kSitePromptQuery);
 #pragma unroll
         for (int w = 0; w < MB / 32; ++w) {
             uint4 lo = make_uint4(0u, 0u, 0u, 0u), hi = lo;     // words the sketch does not have: zeros (contribute 0)
-            if (w < mw) expand_word(__ldg(qw + w), lo, hi);
+            if (w < mw && q_ok) expand_word(__ldg(qw + w), lo, hi);
             *reinterpret_cast<uint4 *>(Qs + pa_off(kPaRows, tid, 2 * w)) = lo;
             *reinterpret_cast<uint4 *>(Qs + pa_off(kPaRows, tid, 2 * w + 1)) = hi;
         }
@@ -180,9 +182,13 @@ __global__ void __launch_bounds__(kPaThreads, MB == 128 ? 2 : 1) prompt_attentio
         for (int cc = 0; cc < 2; ++cc) n_here += (2 * j + cc < n_chunks) ? 1 : 0;
         mbar_arrive_expect_tx(bar, (uint32_t)(n_here * CB));
         for (int cc = 0; cc < 2; ++cc)
-            if (2 * j + cc < n_chunks)
-                bulk_copy_g2s(smem_addr(raw + (j & 1) * SM::kRaw1 + cc * SM::kChunkMax), chunk_ptr(p.ca, layer, b, kvh, 2 * j + cc),
-                              (uint32_t)CB, bar);
+            if (2 * j + cc < n_chunks) {
+                // (bounds-checked build: a source outside the cache is recorded and replaced by the cache's first chunk, so
+                // that the copy the row threads wait for still happens, from memory that is the library's own)
+                const unsigned char *src = chunk_ptr(p.ca, layer, b, kvh, 2 * j + cc);
+                if (!H1B_IN_BOUNDS(in_cache(p.ca, src, CB), p.status, kSitePromptChunk)) src = p.ca.base;
+                bulk_copy_g2s(smem_addr(raw + (j & 1) * SM::kRaw1 + cc * SM::kChunkMax), src, (uint32_t)CB, bar);
+            }
     };
     // the keys of tile j, expanded to +-1 into key operand j % 2: thread t takes half of key t / 2
     auto expand_keys = [&](int j) {
@@ -443,12 +449,14 @@ __global__ void __launch_bounds__(kPaThreads, MB == 128 ? 2 : 1) prompt_attentio
         // ---- the row's output: accumulator / sum of weights. The TMEM loads are warp-wide instructions: every lane
         // makes them, rows past the run's end simply do not store.
         const float inv = valid_q ? 1.f / lsum : 0.f;
-        float *orow = p.out + ((((size_t)ll * p.B + b) * p.Tn + (valid_q ? qi : 0)) * p.Hq + hq) * kHeadDim;
+        const size_t out_row = (((size_t)ll * p.B + b) * p.Tn + (valid_q ? qi : 0)) * p.Hq + hq;
+        const bool store = valid_q && H1B_IN_BOUNDS(ll >= 0 && out_row < (size_t)p.n_layers * p.B * p.Tn * p.Hq, p.status, kSitePromptOut);
+        float *orow = p.out + out_row * kHeadDim;
 #pragma unroll 1
         for (int c = 0; c < 4; ++c) {
             uint32_t o1[32];
             tmem_ld_32cols(t_lane + kColO + c * 32, o1);
-            if (valid_q) {
+            if (store) {
 #pragma unroll
                 for (int k = 0; k < 32; k += 4)
                     *reinterpret_cast<float4 *>(orow + c * 32 + k) =

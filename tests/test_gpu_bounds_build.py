@@ -62,6 +62,8 @@ def test_suites_pass_under_the_bounds_checked_build():
     cmd = [sys.executable, "-m", "pytest", "-x", "-q", "-m", "gpu", "-p", "no:cacheprovider",
            "tests/test_gpu_parity.py", "tests/test_gpu_paged.py", "tests/test_gpu_random_cases.py",
            "tests/test_gpu_multi_query.py", "tests/test_gpu_head_dim_64.py",
+           "tests/test_gpu_prefill_attention.py::test_tile_route_scores_bit_for_bit_and_both_routes_agree",
+           "tests/test_gpu_prefill_attention.py::test_tile_route_with_fp16_values",
            "tests/test_gpu_bounds_build.py::test_probe_under_the_bounds_checked_build"]
     res = subprocess.run(cmd, cwd=ROOT, env=env, capture_output=True, text=True, timeout=1500)
     tail = (res.stdout or "")[-3000:] + (res.stderr or "")[-1500:]
