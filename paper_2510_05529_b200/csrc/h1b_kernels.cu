@@ -976,15 +976,23 @@ __global__ void __maxnreg__(96) prefill_tma_kernel(const __grid_constant__ CUten
                     uint32_t y[32], y2[32];
                     tmem_ld_32cols(tmem_d + ((uint32_t)(quarter * 32) << 16) + (uint32_t)(a * 2 * NBC) + w * 32, y);
                     tmem_ld_32cols(tmem_d + ((uint32_t)(quarter * 32) << 16) + (uint32_t)(a * 2 * NBC + NBC) + w * 32, y2);
+                    // the two pieces' sums added, then + 0, which turns a negative zero into a positive one (see prefill_body);
+                    // both two columns at a time on the packed fp32 adder: the same IEEE additions, the same bits
 #pragma unroll
-                    for (int j = 0; j < 32; ++j) y[j] = __float_as_uint(__uint_as_float(y[j]) + __uint_as_float(y2[j]));
-                    // bit j = (y_j >= 0); adding +0 first turns a negative zero into a positive one (see prefill_body)
+                    for (int j = 0; j < 32; j += 2) {
+                        const float2 t = __fadd2_rn(__fadd2_rn(make_float2(__uint_as_float(y[j]), __uint_as_float(y[j + 1])),
+                                                                make_float2(__uint_as_float(y2[j]), __uint_as_float(y2[j + 1]))),
+                                                    make_float2(0.f, 0.f));
+                        y[j] = __float_as_uint(t.x);
+                        y[j + 1] = __float_as_uint(t.y);
+                    }
+                    // bit j = (y_j >= 0)
                     uint32_t part[4] = {0u, 0u, 0u, 0u};
 #pragma unroll
                     for (int j = 7; j >= 0; --j)
 #pragma unroll
                         for (int k = 0; k < 4; ++k)
-                            part[k] = __funnelshift_l(__float_as_uint(__uint_as_float(y[8 * k + j]) + 0.f), part[k], 1);
+                            part[k] = __funnelshift_l(y[8 * k + j], part[k], 1);
                     const uint32_t neg = part[0] | (part[1] << 8) | (part[2] << 16) | (part[3] << 24);
                     if (tn >= 0 && tn < it.n_new && H1B_IN_BOUNDS(in_cache(p.ca, chunk, cl.bytes), p.status, kSitePrefillKeys))
                         *reinterpret_cast<uint32_t *>(chunk + lane * 4 + (it.col0 / 32 + w) * 128) = ~neg;
