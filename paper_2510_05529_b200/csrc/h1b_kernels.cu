@@ -1186,9 +1186,16 @@ __device__ __forceinline__ void chunk_weights(DecodeState<MW, GQ, NG> &st, const
         if (TAIL) pv = valid ? pv : 0.f;
         st.ssum[h] += pv;
         // (P8: a head only ever needs the zero-point sums of the two value groups of its own half: accz[h][0..1])
+        if constexpr (NG == 4 && !P8) {                       // four groups: two multiply-adds on the packed fp32 instruction
+            const float2 z01 = __ffma2_rn(make_float2(pv, pv), make_float2(zf[0], zf[NG > 1 ? 1 : 0]), make_float2(st.accz[h][0], st.accz[h][NG > 1 ? 1 : 0]));
+            const float2 z23 = __ffma2_rn(make_float2(pv, pv), make_float2(zf[NG > 2 ? 2 : 0], zf[NG > 3 ? 3 : 0]),
+                                          make_float2(st.accz[h][NG > 2 ? 2 : 0], st.accz[h][NG > 3 ? 3 : 0]));
+            st.accz[h][0] = z01.x; st.accz[h][NG > 1 ? 1 : 0] = z01.y; st.accz[h][NG > 2 ? 2 : 0] = z23.x; st.accz[h][NG > 3 ? 3 : 0] = z23.y;
+        } else {
 #pragma unroll
-        for (int g = 0; g < ((P8 && NG) ? 2 : NG); ++g)
-            st.accz[h][g] = fmaf(pv, zf[(NG > 1 && P8) ? ((h / GQH) * 2 + g) : g], st.accz[h][g]);
+            for (int g = 0; g < ((P8 && NG) ? 2 : NG); ++g)
+                st.accz[h][g] = fmaf(pv, zf[(NG > 1 && P8) ? ((h / GQH) * 2 + g) : g], st.accz[h][g]);
+        }
         p_s[h * 32 + lane] = pv;
     }
 }
@@ -1244,8 +1251,8 @@ __device__ __forceinline__ void chunk_values(DecodeState<MW, GQ, NG> &st, const 
             for (int f = 0; f < NF; ++f) {
                 const float2 pp = *reinterpret_cast<const float2 *>(p_s + (f * GQH + bhead) * 32 + vb * 16 + tp);
                 const uint32_t hi = pack_f16x2(pp.x, pp.y);
-                const float2 hf = half2_bits_to_float2(hi);
-                const uint32_t lo = pack_f16x2((pp.x - hf.x) * 2048.f, (pp.y - hf.y) * 2048.f);
+                const float2 r = __fmul2_rn(__ffma2_rn(half2_bits_to_float2(hi), make_float2(-1.f, -1.f), pp), make_float2(2048.f, 2048.f));
+                const uint32_t lo = pack_f16x2(r.x, r.y);
                 const uint32_t got = __shfl_xor_sync(0xffffffffu, part ? hi : lo, 16);
                 bf[vb][f][0] = part ? got : hi;
                 bf[vb][f][1] = part ? lo : got;
@@ -1272,10 +1279,9 @@ __device__ __forceinline__ void chunk_values(DecodeState<MW, GQ, NG> &st, const 
 #pragma unroll
             for (int i = 0; i < 4; ++i) {
                 const int cb = half * 4 + i;
-                st.acc[cb][0] = fmaf(st.acc[cb][0], h0, tmp[i][0]);
-                st.acc[cb][1] = fmaf(st.acc[cb][1], h1, tmp[i][1]);
-                st.acc[cb][2] = fmaf(st.acc[cb][2], h0, tmp[i][2]);
-                st.acc[cb][3] = fmaf(st.acc[cb][3], h1, tmp[i][3]);
+                const float2 a01 = __ffma2_rn(make_float2(st.acc[cb][0], st.acc[cb][1]), make_float2(h0, h1), make_float2(tmp[i][0], tmp[i][1]));
+                const float2 a23 = __ffma2_rn(make_float2(st.acc[cb][2], st.acc[cb][3]), make_float2(h0, h1), make_float2(tmp[i][2], tmp[i][3]));
+                st.acc[cb][0] = a01.x; st.acc[cb][1] = a01.y; st.acc[cb][2] = a23.x; st.acc[cb][3] = a23.y;
             }
         }
         return;
@@ -1301,10 +1307,11 @@ __device__ __forceinline__ void chunk_values(DecodeState<MW, GQ, NG> &st, const 
             const float2 dd = half2_bits_to_float2(
                 *reinterpret_cast<const uint32_t *>(ch + SCALE + vb * (32 * NG) + g * 32 + tp * 2));
             const float2 pw = (P8 && bi >= 2) ? ppb : pp;
-            const float x0 = pw.x * dd.x, x1 = pw.y * dd.y;
-            const uint32_t hi = pack_f16x2(x0, x1);
-            const float2 hf = half2_bits_to_float2(hi);
-            const uint32_t lo = pack_f16x2((x0 - hf.x) * 2048.f, (x1 - hf.y) * 2048.f);
+            // (two tokens at a time on the packed fp32 instructions: the same IEEE operations, the same bits)
+            const float2 x = __fmul2_rn(pw, dd);
+            const uint32_t hi = pack_f16x2(x.x, x.y);
+            const float2 r = __fmul2_rn(__ffma2_rn(half2_bits_to_float2(hi), make_float2(-1.f, -1.f), x), make_float2(2048.f, 2048.f));
+            const uint32_t lo = pack_f16x2(r.x, r.y);
             const uint32_t got = __shfl_xor_sync(0xffffffffu, part ? hi : lo, 16);
             bf[vb][bi][0] = part ? got : hi;                // tokens 2jq, 2jq+1 of this lane's column
             bf[vb][bi][1] = part ? lo : got;                // tokens 2jq+8, 2jq+9
@@ -1336,10 +1343,9 @@ __device__ __forceinline__ void chunk_values(DecodeState<MW, GQ, NG> &st, const 
 #pragma unroll
         for (int i = 0; i < 4; ++i) {
             const int cb = half * 4 + i;
-            st.acc[cb][0] = fmaf(st.acc[cb][0], h0, tmp[i][0]);
-            st.acc[cb][1] = fmaf(st.acc[cb][1], h1, tmp[i][1]);
-            st.acc[cb][2] = fmaf(st.acc[cb][2], h0, tmp[i][2]);
-            st.acc[cb][3] = fmaf(st.acc[cb][3], h1, tmp[i][3]);
+            const float2 a01 = __ffma2_rn(make_float2(st.acc[cb][0], st.acc[cb][1]), make_float2(h0, h1), make_float2(tmp[i][0], tmp[i][1]));
+            const float2 a23 = __ffma2_rn(make_float2(st.acc[cb][2], st.acc[cb][3]), make_float2(h0, h1), make_float2(tmp[i][2], tmp[i][3]));
+            st.acc[cb][0] = a01.x; st.acc[cb][1] = a01.y; st.acc[cb][2] = a23.x; st.acc[cb][3] = a23.y;
         }
     }
 }
